@@ -1,0 +1,213 @@
+/*
+ * fp64 CPU oracle for non-causal linear attention with the Hedgehog feature map.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of the
+ * operator that the CUDA library is checked against.  It shares no code with
+ * the CUDA path and the product never calls it: only the tests, the smoke check
+ * and the benchmark's CPU-baseline leg may load it.
+ *
+ * What it computes, for every group g = (batch, head) independently:
+ *
+ *   Eq. 6   phi(x) = softmax(x W) (+) softmax(-x W)      W is d x d/2, (+) = concat,
+ *                                                        softmax over the d/2 features
+ *   Eq. 5   o_i = sum_j  a_ij / (sum_j a_ij) * v_j ,     a_ij = phi(q_i) . phi(k_j)   (left form)
+ *           o_i = phi(q_i) S / (phi(q_i) . z) ,          S = sum_j phi(k_j)^T v_j,
+ *                                                        z = sum_j phi(k_j)           (right form)
+ *
+ * ref_quadratic is the left form written out (the plain definition, O(n^2 d));
+ * ref_linear is the right form.  Their agreement is the identity of Eq. 5 and is
+ * one of the pins in the CPU tests.
+ *
+ * Readings taken where the paper says nothing:
+ *   - d is the per-head dimension; one W_q and one W_k per head (or one shared by
+ *     all heads when per_head == 0).
+ *   - no bias, temperature, 1/sqrt(d) scale or epsilon anywhere in the operator.
+ *   - concat order is [softmax(+u), softmax(-u)].
+ *   - each softmax subtracts its row maximum first (mathematically a no-op).
+ *   - no mask: every one of the n tokens attends to every one of the n tokens.
+ *
+ * Inputs are float (already rounded to whatever storage type the GPU receives:
+ * every bf16 value is exactly a float) and are widened to double on first use.
+ * All sums are sequential in index order, in double.
+ *
+ * Threading: OpenMP over groups (state pass) and over (group, query row) (output
+ * pass).  No reduction crosses threads, so results do not depend on thread count.
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* Eq. 6 for one row x[0..d) with W[d][m] row-major, m = d/2.  phi has d entries. */
+static void phi_row(const float *x, const float *W, int d, double *phi)
+{
+    const int m = d / 2;
+    double *u = phi + m; /* logits parked in the second half until it is overwritten */
+    for (int j = 0; j < m; ++j) {
+        double acc = 0.0;
+        for (int c = 0; c < d; ++c)
+            acc += (double)x[c] * (double)W[(size_t)c * m + j];
+        u[j] = acc;
+    }
+    double umax = u[0], umin = u[0];
+    for (int j = 1; j < m; ++j) {
+        if (u[j] > umax) umax = u[j];
+        if (u[j] < umin) umin = u[j];
+    }
+    /* softmax(+u): exp(u - max) / sum */
+    double sp = 0.0;
+    for (int j = 0; j < m; ++j) {
+        phi[j] = exp(u[j] - umax);
+        sp += phi[j];
+    }
+    for (int j = 0; j < m; ++j)
+        phi[j] /= sp;
+    /* softmax(-u): max of -u is -min(u), so exp(-u + min) / sum; overwrites u in place */
+    double sn = 0.0;
+    for (int j = 0; j < m; ++j) {
+        u[j] = exp(umin - u[j]);
+        sn += u[j];
+    }
+    for (int j = 0; j < m; ++j)
+        u[j] /= sn;
+}
+
+static const float *w_of(const float *W, int g, int H, int d, int per_head)
+{
+    return per_head ? W + (size_t)(g % H) * d * (d / 2) : W;
+}
+
+/* number of threads an OpenMP region would use here (1 without OpenMP) */
+int linattn_ref_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Eq. 6 applied to n rows: phi_out[n][d]. */
+int linattn_ref_phi(const float *x, const float *W, long n, int d, double *phi_out)
+{
+    if (d < 2 || d > 4096 || (d & 1) || n < 0) return 1;
+    for (long i = 0; i < n; ++i)
+        phi_row(x + (size_t)i * d, W, d, phi_out + (size_t)i * d);
+    return 0;
+}
+
+/*
+ * Left form of Eq. 5.
+ *   q,k,v : [G][n][d] float, G = B*H groups, group g uses head g % H
+ *   Wq,Wk : [H][d][d/2] (per_head != 0) or [d][d/2]
+ *   rows  : nrows query indices in [0,n) evaluated in every group, or NULL for all n
+ *   out   : [G][nrows or n][d] double
+ */
+int linattn_ref_quadratic(const float *q, const float *k, const float *v,
+                          const float *Wq, const float *Wk,
+                          long G, int H, long n, int d, int per_head,
+                          const long *rows, long nrows, double *out)
+{
+    if (d < 2 || d > 4096 || (d & 1) || n < 1 || G < 1 || H < 1) return 1;
+    const long nr = rows ? nrows : n;
+    int fail = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long g = 0; g < G; ++g) {
+        double *phik = (double *)malloc((size_t)n * d * sizeof(double));
+        double *a = (double *)malloc((size_t)n * sizeof(double));
+        double *phiq = (double *)malloc((size_t)d * sizeof(double));
+        if (!phik || !a || !phiq) {
+            fail = 1;
+        } else {
+            const float *kg = k + (size_t)g * n * d, *vg = v + (size_t)g * n * d;
+            const float *qg = q + (size_t)g * n * d;
+            for (long j = 0; j < n; ++j)
+                phi_row(kg + (size_t)j * d, w_of(Wk, (int)g, H, d, per_head), d, phik + (size_t)j * d);
+            for (long r = 0; r < nr; ++r) {
+                const long i = rows ? rows[r] : r;
+                double *o = out + ((size_t)g * nr + r) * d;
+                phi_row(qg + (size_t)i * d, w_of(Wq, (int)g, H, d, per_head), d, phiq);
+                double den = 0.0;
+                for (long j = 0; j < n; ++j) {
+                    double s = 0.0;
+                    for (int f = 0; f < d; ++f)
+                        s += phiq[f] * phik[(size_t)j * d + f];
+                    a[j] = s;
+                    den += s;
+                }
+                for (int c = 0; c < d; ++c) o[c] = 0.0;
+                for (long j = 0; j < n; ++j) {
+                    const double w = a[j] / den;
+                    for (int c = 0; c < d; ++c)
+                        o[c] += w * (double)vg[(size_t)j * d + c];
+                }
+            }
+        }
+        free(phik); free(a); free(phiq);
+    }
+    return fail;
+}
+
+/*
+ * Right form of Eq. 5.  Arguments as above, plus optional state outputs
+ *   S_out : [G][d][d] double, S[f][c] = sum_j phi(k_j)[f] * v_j[c]   (may be NULL)
+ *   z_out : [G][d]    double, z[f]    = sum_j phi(k_j)[f]            (may be NULL)
+ * out may be NULL when only the state is wanted.
+ */
+int linattn_ref_linear(const float *q, const float *k, const float *v,
+                       const float *Wq, const float *Wk,
+                       long G, int H, long n, int d, int per_head,
+                       const long *rows, long nrows, double *out,
+                       double *S_out, double *z_out)
+{
+    if (d < 2 || d > 4096 || (d & 1) || n < 1 || G < 1 || H < 1) return 1;
+    const long nr = rows ? nrows : n;
+    double *S_all = (double *)calloc((size_t)G * d * d, sizeof(double));
+    double *z_all = (double *)calloc((size_t)G * d, sizeof(double));
+    if (!S_all || !z_all) { free(S_all); free(z_all); return 1; }
+
+    /* state pass: S and z of every group, tokens in index order */
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long g = 0; g < G; ++g) {
+        double phik[4096]; /* d <= 4096 */
+        double *S = S_all + (size_t)g * d * d, *z = z_all + (size_t)g * d;
+        const float *kg = k + (size_t)g * n * d, *vg = v + (size_t)g * n * d;
+        for (long j = 0; j < n; ++j) {
+            phi_row(kg + (size_t)j * d, w_of(Wk, (int)g, H, d, per_head), d, phik);
+            for (int f = 0; f < d; ++f) {
+                z[f] += phik[f];
+                for (int c = 0; c < d; ++c)
+                    S[(size_t)f * d + c] += phik[f] * (double)vg[(size_t)j * d + c];
+            }
+        }
+    }
+
+    /* output pass: o_i = phi(q_i) S / (phi(q_i) . z) */
+    if (out) {
+#pragma omp parallel for collapse(2) schedule(static)
+        for (long g = 0; g < G; ++g) {
+            for (long r = 0; r < nr; ++r) {
+                double phiq[4096];
+                const long i = rows ? rows[r] : r;
+                const double *S = S_all + (size_t)g * d * d, *z = z_all + (size_t)g * d;
+                double *o = out + ((size_t)g * nr + r) * d;
+                phi_row(q + ((size_t)g * n + i) * d, w_of(Wq, (int)g, H, d, per_head), d, phiq);
+                double den = 0.0;
+                for (int f = 0; f < d; ++f)
+                    den += phiq[f] * z[f];
+                for (int c = 0; c < d; ++c) {
+                    double num = 0.0;
+                    for (int f = 0; f < d; ++f)
+                        num += phiq[f] * S[(size_t)f * d + c];
+                    o[c] = num / den;
+                }
+            }
+        }
+    }
+    if (S_out) memcpy(S_out, S_all, (size_t)G * d * d * sizeof(double));
+    if (z_out) memcpy(z_out, z_all, (size_t)G * d * sizeof(double));
+    free(S_all); free(z_all);
+    return 0;
+}

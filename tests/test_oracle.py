@@ -1,0 +1,229 @@
+"""Pins for the fp64 CPU oracle: closed forms, invariants and brute force (no GPU).
+
+Each test fixes the oracle to something other than itself, so that a dropped term,
+a wrong sign or index, or a transposed operand in it fails at least one of them.
+"""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_fractions(name):
+    out = {}
+    with open(os.path.join(GOLDEN, name)) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *vals = line.split()
+            out[key] = np.array([float(Fraction(v)) for v in vals])
+    return out
+
+
+def _rand(B, H, n, d, seed, scale=1.0, wscale=None):
+    rng = np.random.default_rng(seed)
+    q, k, v = (rng.standard_normal((B, H, n, d)).astype(np.float32) * scale for _ in range(3))
+    ws = (1.0 / (math.sqrt(d) * scale)) if wscale is None else wscale
+    Wq, Wk = (rng.standard_normal((H, d, d // 2)).astype(np.float32) * ws for _ in range(2))
+    return q, k, v, Wq.astype(np.float32), Wk.astype(np.float32)
+
+
+# ---- hand-derived worked examples (tests/golden) -------------------------------------------
+
+def test_closed_form_d4_n2():
+    """Eq. 5 + Eq. 6 against fractions derived by hand (distinct W_q / W_k, decoy coordinates)."""
+    g = _read_fractions("closed_form_d4_n2.txt")
+    ln = math.log
+    q = np.array([[ln(3), 7, 0, -2], [0, 1, ln(2), 5]], dtype=np.float32)[None, None]
+    k = np.array([[9, ln(4), -1, 0], [3, 0, 3, 0]], dtype=np.float32)[None, None]
+    v = np.array([[1, 0, -2, 4], [0, 10, 2, -4]], dtype=np.float32)[None, None]
+    Wq = np.array([[1, 0], [0, 0], [0, 1], [0, 0]], dtype=np.float32)
+    Wk = np.array([[0, 0], [1, 0], [0, 0], [0, 1]], dtype=np.float32)
+    tol = 1e-6  # ln(.) is rounded to float32 on input
+    np.testing.assert_allclose(oracle.phi(q[0, 0], Wq), np.stack([g["phi_q1"], g["phi_q2"]]), atol=tol)
+    np.testing.assert_allclose(oracle.phi(k[0, 0], Wk), np.stack([g["phi_k1"], g["phi_k2"]]), atol=tol)
+    want_o = np.stack([g["o_1"], g["o_2"]])
+    want_S = np.stack([g["S_0"], g["S_1"], g["S_2"], g["S_3"]])
+    o_lin, S, z = oracle.ref_linear(q, k, v, Wq, Wk, return_state=True)
+    np.testing.assert_allclose(o_lin[0, 0], want_o, atol=tol)
+    np.testing.assert_allclose(S[0, 0], want_S, atol=tol)
+    np.testing.assert_allclose(z[0, 0], g["z"], atol=tol)
+    np.testing.assert_allclose(oracle.ref_quadratic(q, k, v, Wq, Wk)[0, 0], want_o, atol=tol)
+    # per-head weight layout [H, d, d/2] with H = 1 gives the same
+    np.testing.assert_allclose(oracle.ref_linear(q, k, v, Wq[None], Wk[None])[0, 0], want_o, atol=tol)
+
+
+def test_closed_form_phi_d6():
+    g = _read_fractions("phi_d6.txt")
+    W = np.zeros((6, 3), dtype=np.float32)
+    W[0, 0] = 1.0
+    W[2, 2] = 0.5
+    x = np.array([[math.log(2), 5, math.log(16), 1, -3, 0]], dtype=np.float32)
+    np.testing.assert_allclose(oracle.phi(x, W)[0], g["phi"], atol=1e-6)
+
+
+# ---- Eq. 5: the two forms agree (brute force) ------------------------------------------------
+
+@pytest.mark.parametrize("B,H,n,d", [(1, 2, 1024, 64), (2, 3, 37, 8), (1, 1, 129, 128), (1, 2, 5, 2)])
+def test_linear_equals_quadratic(B, H, n, d):
+    q, k, v, Wq, Wk = _rand(B, H, n, d, seed=n + d)
+    a = oracle.ref_quadratic(q, k, v, Wq, Wk)
+    b = oracle.ref_linear(q, k, v, Wq, Wk)
+    assert np.abs(a - b).max() <= 1e-12 * max(1.0, np.abs(a).max())
+
+
+def test_rows_subset_matches_full():
+    q, k, v, Wq, Wk = _rand(1, 2, 200, 16, seed=3)
+    rows = np.array([0, 199, 57, 57, 3])
+    full = oracle.ref_linear(q, k, v, Wq, Wk)
+    np.testing.assert_array_equal(oracle.ref_linear(q, k, v, Wq, Wk, rows=rows), full[:, :, rows])
+    np.testing.assert_array_equal(oracle.ref_quadratic(q, k, v, Wq, Wk, rows=rows),
+                                  oracle.ref_quadratic(q, k, v, Wq, Wk)[:, :, rows])
+
+
+# ---- library routine with independent arithmetic --------------------------------------------
+
+def test_against_torch_sdpa_fp64():
+    """softmax(log A) is the row-normalised A, so torch's fp64 SDPA with q = 0 and additive mask
+    log A evaluates the left form of Eq. 5 through a library routine."""
+    B, H, n, d = 1, 2, 96, 16
+    q, k, v, Wq, Wk = _rand(B, H, n, d, seed=11)
+    tq, tk, tv = (torch.from_numpy(t).double() for t in (q, k, v))
+    tWq, tWk = torch.from_numpy(Wq).double(), torch.from_numpy(Wk).double()
+
+    def fmap(x, W):
+        u = torch.einsum("bhnd,hdm->bhnm", x, W)
+        return torch.cat([torch.softmax(u, -1), torch.softmax(-u, -1)], -1)
+
+    A = torch.einsum("bhif,bhjf->bhij", fmap(tq, tWq), fmap(tk, tWk))
+    want = torch.nn.functional.scaled_dot_product_attention(torch.zeros_like(tq), tk, tv, attn_mask=A.log())
+    got = oracle.ref_linear(q, k, v, Wq, Wk)
+    np.testing.assert_allclose(got, want.numpy(), rtol=0, atol=1e-12)
+
+
+# ---- closed forms and invariants ---------------------------------------------------------------
+
+def test_constant_feature_map_gives_mean_of_v():
+    """W = 0 makes phi the constant 2/d, so every output row is the mean of V."""
+    q, k, v, _, _ = _rand(2, 2, 77, 16, seed=5)
+    W0 = np.zeros((2, 16, 8), dtype=np.float32)
+    want = v.astype(np.float64).mean(axis=2, keepdims=True)
+    for fn in (oracle.ref_linear, oracle.ref_quadratic):
+        got = fn(q, k, v, W0, W0)
+        np.testing.assert_allclose(got, np.broadcast_to(want, got.shape), atol=1e-13)
+
+
+def test_d2_is_mean_of_v():
+    """d = 2: each softmax is over one feature, phi = (1, 1) whatever W is."""
+    q, k, v, Wq, Wk = _rand(1, 3, 40, 2, seed=6, wscale=3.0)
+    want = v.astype(np.float64).mean(axis=2, keepdims=True)
+    got = oracle.ref_linear(q, k, v, Wq, Wk)
+    np.testing.assert_allclose(got, np.broadcast_to(want, got.shape), atol=1e-13)
+    np.testing.assert_array_equal(oracle.phi(q[0, 0], Wq[0]), np.ones((40, 2)))
+
+
+def test_single_token_returns_v():
+    q, k, v, Wq, Wk = _rand(2, 2, 1, 32, seed=7)
+    for fn in (oracle.ref_linear, oracle.ref_quadratic):
+        np.testing.assert_allclose(fn(q, k, v, Wq, Wk), v.astype(np.float64), rtol=1e-14)
+
+
+def test_phi_structure_and_state_sums():
+    """Eq. 6: entries in (0, 1], each half sums to 1; hence sum(z) = 2 n and sum_f S[f, c] = 2 sum_j v_jc."""
+    q, k, v, Wq, Wk = _rand(1, 2, 300, 64, seed=8, wscale=0.5)
+    p = oracle.phi(k[0, 1], Wk[1])
+    assert (p > 0).all() and (p <= 1).all()
+    np.testing.assert_allclose(p[:, :32].sum(-1), 1.0, rtol=1e-14)
+    np.testing.assert_allclose(p[:, 32:].sum(-1), 1.0, rtol=1e-14)
+    # the second half is the first half's map applied to the negated input
+    np.testing.assert_allclose(p[:, 32:], oracle.phi(-k[0, 1], Wk[1])[:, :32], rtol=1e-14)
+    _, S, z = oracle.ref_linear(q, k, v, Wq, Wk, return_state=True)
+    np.testing.assert_allclose(z.sum(-1), 2.0 * 300, rtol=1e-13)
+    np.testing.assert_allclose(S.sum(-2), 2.0 * v.astype(np.float64).sum(2), atol=1e-11)
+    # z and S restated from phi with numpy
+    np.testing.assert_allclose(z[0, 1], p.sum(0), rtol=1e-13)
+    np.testing.assert_allclose(S[0, 1], p.T @ v[0, 1].astype(np.float64), atol=1e-11)
+
+
+def test_phi_is_shift_stable():
+    """Large logits must not overflow: softmax is invariant to adding a constant to all logits."""
+    W = np.zeros((4, 2), dtype=np.float32)
+    W[0, 0] = 1.0
+    W[1, 1] = 1.0
+    x = np.array([[1000.0, 999.0, 0, 0], [-1000.0, -1001.0, 0, 0]], dtype=np.float32)
+    e = math.e
+    want = np.array([e / (1 + e), 1 / (1 + e), 1 / (1 + e), e / (1 + e)])
+    got = oracle.phi(x, W)
+    np.testing.assert_allclose(got[0], want, rtol=1e-14)
+    np.testing.assert_allclose(got[1], want, rtol=1e-14)
+
+
+def test_key_value_permutation_invariance_and_query_equivariance():
+    q, k, v, Wq, Wk = _rand(1, 2, 150, 16, seed=9)
+    base = oracle.ref_linear(q, k, v, Wq, Wk)
+    perm = np.random.default_rng(1).permutation(150)
+    np.testing.assert_allclose(oracle.ref_linear(q, k[:, :, perm], v[:, :, perm], Wq, Wk), base, atol=1e-13)
+    np.testing.assert_allclose(oracle.ref_linear(q[:, :, perm], k, v, Wq, Wk), base[:, :, perm], atol=1e-15)
+    # permuting only the keys (not the values) must change the result: k_j and v_j are paired
+    assert np.abs(oracle.ref_linear(q, k[:, :, perm], v, Wq, Wk) - base).max() > 1e-3
+
+
+def test_convex_combination_shift_and_linearity_in_v():
+    q, k, v, Wq, Wk = _rand(1, 2, 120, 16, seed=10)
+    o = oracle.ref_linear(q, k, v, Wq, Wk)
+    v64 = v.astype(np.float64)
+    assert (o <= v64.max(axis=2, keepdims=True) + 1e-12).all()
+    assert (o >= v64.min(axis=2, keepdims=True) - 1e-12).all()
+    shift = np.float32(2.0)  # exact in float32 for these magnitudes? compare against the shifted floats
+    v2 = (v + shift).astype(np.float32)
+    np.testing.assert_allclose(oracle.ref_linear(q, k, v2, Wq, Wk) - o,
+                               (v2.astype(np.float64) - v64).mean() * np.ones_like(o), atol=1e-6)
+    np.testing.assert_allclose(oracle.ref_linear(q, k, (2 * v).astype(np.float32), Wq, Wk), 2 * o, rtol=1e-14)
+
+
+def test_duplicating_every_key_value_pair_changes_nothing():
+    q, k, v, Wq, Wk = _rand(1, 2, 60, 16, seed=12)
+    base = oracle.ref_linear(q, k, v, Wq, Wk)
+    k2, v2 = np.repeat(k, 2, axis=2), np.repeat(v, 2, axis=2)
+    q2 = np.concatenate([q, q], axis=2)
+    o2, S2, z2 = oracle.ref_linear(q2, k2, v2, Wq, Wk, return_state=True)
+    _, S, z = oracle.ref_linear(q, k, v, Wq, Wk, return_state=True)
+    np.testing.assert_allclose(o2[:, :, :60], base, atol=1e-13)
+    np.testing.assert_allclose(S2, 2 * S, atol=1e-12)
+    np.testing.assert_allclose(z2, 2 * z, atol=1e-12)
+
+
+def test_heads_and_batches_are_independent_and_use_their_own_weights():
+    q, k, v, Wq, Wk = _rand(2, 3, 50, 8, seed=13)
+    full = oracle.ref_linear(q, k, v, Wq, Wk)
+    for b in range(2):
+        for h in range(3):
+            one = oracle.ref_linear(q[b:b + 1, h:h + 1], k[b:b + 1, h:h + 1], v[b:b + 1, h:h + 1], Wq[h], Wk[h])
+            np.testing.assert_array_equal(one[0, 0], full[b, h])
+    # shared-weights mode equals per-head mode with the same matrix repeated
+    shared = oracle.ref_linear(q, k, v, Wq[1], Wk[2])
+    rep = oracle.ref_linear(q, k, v, np.repeat(Wq[1:2], 3, 0), np.repeat(Wk[2:3], 3, 0))
+    np.testing.assert_array_equal(shared, rep)
+
+
+def test_query_and_key_weights_are_not_interchangeable():
+    q, k, v, Wq, Wk = _rand(1, 1, 64, 16, seed=14, wscale=1.0)
+    a = oracle.ref_linear(q, k, v, Wq, Wk)
+    b = oracle.ref_linear(q, k, v, Wk, Wq)
+    assert np.abs(a - b).max() > 1e-3
+
+
+def test_bad_arguments_are_rejected():
+    q, k, v, Wq, Wk = _rand(1, 1, 4, 4, seed=15)
+    with pytest.raises(AssertionError):
+        oracle.ref_linear(q, k, v[:, :, :3], Wq, Wk)
+    with pytest.raises(AssertionError):
+        oracle.ref_linear(q, k, v, Wq, Wk, rows=np.array([4]))
