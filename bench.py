@@ -1,0 +1,291 @@
+#!/usr/bin/env python
+"""Benchmark of the linear-attention forward (Eq. 5 with the feature map of Eq. 6) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C]
+
+One step = one `linattn_forward` over one batch of synthetic Wan-shaped input (default: the
+Wan-1.3B 480p layer, B=1, H=12, n=32760, d=128, bf16).  Prints ONE JSON line on rank 0.
+With N > 1 (under torchrun) every rank runs an independent replica on its own inputs: the
+operator has no cross-GPU exchange, so there is no data-path collective (weak scaling).
+`--impl reference` times the fp64 CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_08318_b200 import dist as ladist  # noqa: E402
+from paper_2510_08318_b200 import synth  # noqa: E402
+
+METRIC = "linear-attention fwd tokens/s"
+UNIT = "tokens/s"
+ROTATE = 3  # input sets cycled through, so that a step's inputs were last touched > 2 x L2 ago
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [nm for i, nm in enumerate(names) if any(len(r) >= 6 and r[2 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def time_oracle(x, budget_s: float):
+    """Oracle (right-hand form of Eq. 5, fp64, as it stands) on a bounded sample: the first n_s tokens of
+    every head.  Its cost is linear in tokens, so tokens/s on the sample stands for the workload."""
+    import oracle
+    B, H, n, d = x["q"].shape
+    probe = min(n, 2048)
+
+    def run(ns):
+        sl = {k_: (x[k_][:, :, :ns].contiguous() if k_ in ("q", "k", "v") else x[k_]) for k_ in x}
+        t0 = time.perf_counter()
+        oracle.ref_linear(sl["q"], sl["k"], sl["v"], sl["Wq"], sl["Wk"])
+        return time.perf_counter() - t0
+
+    run(min(n, 256))  # builds / loads the oracle, warms the thread pool
+    rate = probe / run(probe)
+    ns = int(max(probe, min(n, rate * budget_s)))
+    secs = run(ns)
+    return {"tokens": B * ns, "seconds": secs, "value": B * ns / secs, "cores": oracle.threads(),
+            "sample": f"first {ns} of n={n} tokens of all {B}x{H} heads, 1 run, {secs:.2f} s"}
+
+
+def reference_arm(args, wl):
+    """--impl reference: the CPU oracle, timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    x = synth.make_inputs(args.config)
+    total = args.steps + args.warmup
+    budget = max(0.2, min(10.0, 150.0 / max(1, total)))
+    import oracle
+    B, H, n, d = x["q"].shape
+    probe = min(n, 1024)
+    sl = lambda ns: [x[k_][:, :, :ns].contiguous() for k_ in ("q", "k", "v")] + [x["Wq"], x["Wk"]]
+    t0 = time.perf_counter(); oracle.ref_linear(*sl(probe)); rate = probe / (time.perf_counter() - t0)
+    ns = int(max(probe, min(n, rate * budget)))
+    a = sl(ns)
+    for _ in range(args.warmup):
+        oracle.ref_linear(*a)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.ref_linear(*a)
+    secs = time.perf_counter() - t0
+    value = B * ns * args.steps / secs
+    sample = f"first {ns} of n={n} tokens of all {B}x{H} heads per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl_name(args.config, wl), "B": B, "H": H, "n": n, "d": d, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def wl_name(config, wl):
+    return f"config {config}: {wl.name} B={wl.B} H={wl.H} n={wl.n} d={wl.d} {wl.dtype}"
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--no-baselines", action="store_true", help="skip the oracle and SDPA context baselines")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    wl = synth.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        reference_arm(args, wl)
+        return
+
+    from paper_2510_08318_b200 import linattn
+
+    rank, world, local = ladist.init_from_env("nccl")
+    assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torchrun --nproc-per-node {args.gpus}"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    # inputs: ROTATE independent sets per rank (different layers' seeds), resident in HBM
+    B, H, n, d = wl.B, wl.H, wl.n, wl.d
+    sets = []
+    host0 = None
+    for r in range(ROTATE):
+        x = synth.make_inputs(args.config, layer=(rank * ROTATE + r) % max(wl.layers, 30))
+        if r == 0:
+            host0 = x
+        sets.append({k_: t.to(dev) for k_, t in x.items()})
+    outs = [torch.empty_like(s["q"]) for s in sets]
+    ctxs = []
+    for s in sets:  # one context per input set: its own feature map, as one layer would have
+        c = linattn.LinAttn(H, d, max_B=B, max_n=n, device=local)
+        c.set_option(linattn.OPT_PATH, args.path)
+        c.set_option(linattn.OPT_SPLITS, args.splits)
+        c.set_feature_map(s["Wq"], s["Wk"])
+        ctxs.append(c)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        j = i % ROTATE
+        ctxs[j].forward(sets[j]["q"], sets[j]["k"], sets[j]["v"], out=outs[j], stream=stream)
+
+    for i in range(args.warmup):
+        step(i)
+    ctxs[0].check()
+    launches_per_step = ctxs[0].last_launch_count()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ladist.barrier()
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ladist.barrier()
+    ms_total = ladist.max_over_ranks(ev0.elapsed_time(ev1))
+    clocks = sampler.stop() if rank == 0 else None
+    for c in ctxs:
+        c.check()
+    ms_step = ms_total / args.steps
+    tokens_per_step = ladist.sum_over_ranks(float(B * n))
+    value = tokens_per_step / (ms_step * 1e-3)
+
+    # per-kernel durations: a second pass of the same steps with events around every launch
+    e = 2 if wl.dtype == "bf16" else 4
+    alg_total = 4.0 * B * H * n * d * e
+    for c in ctxs:
+        c.set_option(linattn.OPT_PROFILE, 1)
+    for i in range(args.steps):
+        step(i)
+    torch.cuda.synchronize()
+    kernels = ctxs[0].kernel_times()  # [(name, mean ms, launches, algorithmic bytes per launch)]
+    for c in ctxs:
+        c.set_option(linattn.OPT_PROFILE, 0)
+    peaks = load_peaks()
+    dom = max(kernels, key=lambda kt: kt["ms"])
+    achieved = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom["name"], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                "kernel_ms": dom["ms"], "algorithmic_bytes_per_launch": dom["bytes"],
+                "timing": "mean over a second pass of the timed steps with CUDA events around each launch",
+                "kernels": kernels,
+                "whole_step": {"achieved": alg_total / (ms_step * 1e-3) / 1e9,
+                               "frac": alg_total / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                               "frac_of_nominal_8TBs": alg_total / (ms_step * 1e-3) / 1e9 / 8000.0,
+                               "algorithmic_bytes": alg_total}}
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        roofline["traffic"] = json.load(open(traffic_file)).get(dom["name"])
+
+    # end to end through the host-buffer entry point: pinned host tensors in, pinned host tensor out
+    pin = {k_: host0[k_].pin_memory() for k_ in ("q", "k", "v")}
+    hout = torch.empty_like(host0["q"]).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    ctxs[0].forward_host(pin["q"], pin["k"], pin["v"], hout, stream=stream)  # allocates the staging buffers
+    ladist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        ctxs[0].forward_host(pin["q"], pin["k"], pin["v"], hout, stream=stream)
+    torch.cuda.synchronize()
+    e2e_s = ladist.max_over_ranks(time.perf_counter() - t0) / e2e_steps
+    nbytes = B * H * n * d * e
+    e2e = {"value": tokens_per_step / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
+           "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "entry_point": "linattn_forward_host (pinned host buffers)"}
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": wl_name(args.config, wl), "B": B, "H": H, "n": n, "d": d, "path": args.path,
+                   "l2": f"inputs larger than L2 and {ROTATE} input sets rotated (no set is re-read within {ROTATE - 1} steps)",
+                   "multi_gpu": "replicas only: independent inputs per rank, no collective on the data path"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1 and not args.no_baselines:
+        cb = time_oracle(host0, budget_s=12.0)
+        result["cpu_baseline"] = {"value": cb["value"], "unit": UNIT, "cores": cb["cores"], "kind": "oracle", "sample": cb["sample"]}
+        # context only: softmax attention of the same shape through torch SDPA
+        try:
+            s = sets[0]
+            for _ in range(2):
+                torch.nn.functional.scaled_dot_product_attention(s["q"], s["k"], s["v"])
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            for _ in range(5):
+                torch.nn.functional.scaled_dot_product_attention(s["q"], s["k"], s["v"])
+            a1.record()
+            torch.cuda.synchronize()
+            sd = a0.elapsed_time(a1) / 5
+            result["sdpa_baseline"] = {"ms_per_step": sd, "value": B * n / (sd * 1e-3), "unit": UNIT,
+                                       "kind": "torch scaled_dot_product_attention, same [B,H,n,d] bf16, non-causal"}
+        except Exception as exc:  # context number only
+            result["sdpa_baseline"] = {"error": str(exc)[:200]}
+
+    for c in ctxs:
+        c.destroy()
+    if rank == 0:
+        print(json.dumps(result))
+    ladist.shutdown()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,134 @@
+/*
+ * linattn — non-causal O(n) linear attention with the Hedgehog feature map, for NVIDIA B200 (sm_100a).
+ *
+ * The operator (per batch b and head h, all n tokens attend to all n tokens):
+ *
+ *   phi(x) = softmax(x W) (+) softmax(-x W)            Eq. 6; W is d x d/2, (+) is concatenation,
+ *                                                      both softmaxes run over the d/2 features
+ *   S = sum_j phi(k_j)^T v_j   (d x d)                 Eq. 5, numerator bracket of the right-hand form
+ *   z = sum_j phi(k_j)         (d)                     Eq. 5, denominator bracket
+ *   o_i = phi(q_i) S / (phi(q_i) . z)                  Eq. 5, right-hand form
+ *
+ * with W = W_q for queries and W = W_k for keys.  There is no bias, no temperature, no
+ * 1/sqrt(d) factor, no epsilon and no mask inside the operator.
+ *
+ * Every entry point returns a status and never throws, aborts or prints.  Nothing here falls
+ * back to the CPU: an unsupported request is an error.  Unless an entry point says otherwise its
+ * pointers are DEVICE pointers on the context's device, work is enqueued on the caller's stream
+ * and the call returns without synchronising.
+ */
+#ifndef LINATTN_H
+#define LINATTN_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct linattn_ctx linattn_ctx; /* opaque: feature-map weights + workspace of one attention layer */
+
+typedef enum {
+    LINATTN_OK = 0,
+    LINATTN_ERR_INVALID_ARG = 1,    /* null pointer, size out of range, shape differs from create, misaligned pointer */
+    LINATTN_ERR_UNSUPPORTED = 2,    /* d not in {64, 128}, unknown dtype, device is not sm_100 */
+    LINATTN_ERR_NO_FEATURE_MAP = 3, /* forward before set_feature_map */
+    LINATTN_ERR_WORKSPACE = 4,      /* request exceeds what create reserved */
+    LINATTN_ERR_CUDA = 5,           /* a CUDA call failed; text via linattn_last_error */
+    LINATTN_ERR_TIMEOUT = 6         /* a bounded device-side wait gave up (reported by linattn_check) */
+} linattn_status;
+
+typedef enum { LINATTN_F32 = 0, LINATTN_BF16 = 1 } linattn_dtype;
+
+/* Options for linattn_set_option. */
+typedef enum {
+    LINATTN_OPT_SPLITS = 0, /* number of key-side partial reductions per (b,h); 0 = automatic (default) */
+    LINATTN_OPT_PATH = 1,   /* 0 = automatic (default), 1 = CUDA-core kernels, 2 = tensor-core (tcgen05 + TMA) kernels */
+    LINATTN_OPT_PROFILE = 2 /* 1 = record CUDA events around every kernel of each forward (see linattn_profile_get);
+                               switching it on clears the accumulated figures; 0 = off (default) */
+} linattn_option;
+
+/*
+ * Create a context for one attention layer with H heads of dimension d (Eq. 5-6 are per head;
+ * the paper writes a single head).  Allocates, on `device`, room for the feature-map weights and
+ * the workspace that holds the partial and final S and z (Eq. 5) for up to max_B * H (b,h) pairs.
+ * max_n bounds the sequence length later calls may use.  *ctx is written only on success.
+ * Errors: INVALID_ARG (null ctx, H/max_B/max_n < 1), UNSUPPORTED (d not 64 or 128, device not
+ * compute capability 10.x), CUDA (allocation failed).
+ */
+linattn_status linattn_create(linattn_ctx** ctx, int device, int H, int d, long long max_B, long long max_n);
+
+/*
+ * Set W_q and W_k of Eq. 6.  Wq, Wk: device pointers, row-major [H][d][d/2] when per_head != 0, or
+ * [d][d/2] shared by all heads when per_head == 0, of type wdtype.  The values are COPIED (and
+ * converted) into the context on `stream`; the caller may free its buffers once that stream has
+ * passed this point.  Errors: INVALID_ARG, UNSUPPORTED (wdtype), CUDA.
+ */
+linattn_status linattn_set_feature_map(linattn_ctx* ctx, const void* Wq, const void* Wk, int per_head,
+                                       linattn_dtype wdtype, void* stream);
+
+/*
+ * Eq. 5 (right-hand form) with the feature map of Eq. 6, for all B*H (b,h) pairs.
+ *   q, k, v : device, contiguous row-major [B][H][n][d] of `dtype`, 16-byte aligned, read-only
+ *   out     : device, same shape and type, written in full; must not overlap q, k or v
+ *   H, d    : must equal the values given to create;  1 <= B <= max_B;  1 <= n <= max_n
+ *   dtype   : LINATTN_BF16 (bf16 in, bf16 out, round-to-nearest-even) or LINATTN_F32
+ *   stream  : a cudaStream_t of the context's device (NULL = default stream)
+ * All accumulation (S, z, numerator, denominator) is fp32.  The call allocates nothing, does not
+ * synchronise, and is deterministic: the same inputs give bit-identical outputs.  Calls on one
+ * context must be stream-ordered (they share the context's workspace).
+ * Errors: INVALID_ARG, UNSUPPORTED, NO_FEATURE_MAP, WORKSPACE, CUDA (launch failure).
+ */
+linattn_status linattn_forward(linattn_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                               int B, int H, int n, int d, linattn_dtype dtype, void* stream);
+
+/*
+ * The same operation on HOST buffers (pageable or pinned): copies q, k, v to device staging
+ * buffers owned by the context, runs linattn_forward, copies the result into `out`, and waits
+ * for `stream` before returning.  The staging buffers are allocated (or grown) on the first call
+ * that needs them and released by destroy.  Same argument rules and errors as linattn_forward,
+ * except that the pointers are host pointers with no alignment requirement.
+ */
+linattn_status linattn_forward_host(linattn_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                                    int B, int H, int n, int d, linattn_dtype dtype, void* stream);
+
+/*
+ * Copy the S and z (Eq. 5) left in the workspace by the most recent forward to HOST memory:
+ * S_host [B][H][d][d] floats with S[f][c] = sum_j phi(k_j)[f] v_j[c], z_host [B][H][d] floats.
+ * Waits for `stream`.  Either pointer may be NULL.  For tests and debugging.
+ */
+linattn_status linattn_read_state(linattn_ctx* ctx, float* S_host, float* z_host, int B, void* stream);
+
+/* Tuning and test knobs; see linattn_option.  Errors: INVALID_ARG (unknown option or value). */
+linattn_status linattn_set_option(linattn_ctx* ctx, linattn_option opt, long long value);
+
+/*
+ * Wait for `stream` and report whether any kernel of this context gave up a bounded wait
+ * (TIMEOUT) or the stream hit a CUDA error (CUDA); clears the device-side error word.
+ */
+linattn_status linattn_check(linattn_ctx* ctx, void* stream);
+
+/*
+ * Per-kernel timing gathered while LINATTN_OPT_PROFILE is on.  index = position of the kernel in the
+ * forward's launch order.  Returns 1 and fills the outputs (any may be NULL) if that kernel has been
+ * timed at least once, else 0: *name (static string), *mean_ms (mean duration between the CUDA events
+ * around its launches), *launches, *algorithmic_bytes (bytes of q/k/v/out one launch must move:
+ * K+V for the key side, Q+O for the query side).  Waits for the last profiled forward to finish.
+ */
+int linattn_profile_get(linattn_ctx* ctx, int index, const char** name, double* mean_ms, long long* launches,
+                        double* algorithmic_bytes);
+
+/* Number of kernels the most recent linattn_forward on this context launched (0 before any). */
+int linattn_last_launch_count(const linattn_ctx* ctx);
+
+/* Text of the last CUDA error seen by this context ("" if none).  Valid until the next call on ctx. */
+const char* linattn_last_error(const linattn_ctx* ctx);
+
+/* Release everything the context owns.  Waits for the device.  NULL is accepted. */
+linattn_status linattn_destroy(linattn_ctx* ctx);
+
+/* Static text for a status code. */
+const char* linattn_status_string(linattn_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LINATTN_H */

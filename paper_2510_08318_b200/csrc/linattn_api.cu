@@ -1,0 +1,438 @@
+// C-ABI boundary of the linear-attention library: context, argument checks, kernel dispatch.
+// The entry points and their contracts are declared in include/linattn.h.
+#include "linattn.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "simt_kernels.cuh"
+
+using namespace linattn;
+
+namespace {
+
+constexpr int kTargetCtas = 296;  // key-side CTAs aimed for: two waves of the 148 SMs
+constexpr int kMaxSplits = 512;
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct linattn_ctx {
+    int device = 0;
+    int H = 0, d = 0;
+    long long max_B = 0, max_n = 0;
+    bool have_map = false;
+    // weights, fp32 [H][d][d/2]
+    float* Wq = nullptr;
+    float* Wk = nullptr;
+    // workspace
+    float* partial = nullptr;   // [partial_slots][d*d + d]
+    long long partial_slots = 0;
+    float* state = nullptr;     // [max_B*H][d*d + d]
+    unsigned int* err_word = nullptr;
+    // host-call staging
+    void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
+    size_t stage_bytes = 0;
+    // options
+    int opt_splits = 0;
+    int opt_path = 0;
+    // per-kernel timing (LINATTN_OPT_PROFILE)
+    static constexpr int kMaxKernels = 4;
+    bool profile = false;
+    bool prof_pending = false;
+    int prof_n = 0;                       // kernels in the forward being timed
+    cudaEvent_t prof_ev[kMaxKernels + 1] = {};
+    const char* prof_name[kMaxKernels] = {};
+    double prof_bytes[kMaxKernels] = {};
+    double prof_ms[kMaxKernels] = {};
+    long long prof_cnt[kMaxKernels] = {};
+    // bookkeeping
+    int last_launches = 0;
+    int last_B = 0;
+    char err_text[256] = {0};
+};
+
+namespace {
+
+linattn_status cuda_fail(linattn_ctx* c, cudaError_t e, const char* what)
+{
+    if (c) snprintf(c->err_text, sizeof(c->err_text), "%s: %s", what, cudaGetErrorString(e));
+    return LINATTN_ERR_CUDA;
+}
+
+#define LA_CUDA(ctx, call)                                         \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call); \
+    } while (0)
+
+size_t elem_size(linattn_dtype t) { return t == LINATTN_BF16 ? 2 : 4; }
+
+// Per-kernel timing: events are recorded around every launch of a forward and read back (after a
+// wait on the last one) at the start of the next profiled forward or when the figures are queried.
+void prof_flush(linattn_ctx* c)
+{
+    if (!c->prof_pending) return;
+    c->prof_pending = false;
+    if (cudaEventSynchronize(c->prof_ev[c->prof_n]) != cudaSuccess) {
+        cudaGetLastError();
+        return;
+    }
+    for (int i = 0; i < c->prof_n; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]) == cudaSuccess) {
+            c->prof_ms[i] += ms;
+            c->prof_cnt[i] += 1;
+        }
+    }
+}
+
+void prof_begin(linattn_ctx* c, cudaStream_t st)
+{
+    if (!c->profile) return;
+    prof_flush(c);
+    c->prof_n = 0;
+    cudaEventRecord(c->prof_ev[0], st);
+}
+
+void prof_mark(linattn_ctx* c, cudaStream_t st, const char* name, double alg_bytes)
+{
+    if (!c->profile || c->prof_n >= linattn_ctx::kMaxKernels) return;
+    const int i = c->prof_n++;
+    c->prof_name[i] = name;
+    c->prof_bytes[i] = alg_bytes;
+    cudaEventRecord(c->prof_ev[i + 1], st);
+    c->prof_pending = true;
+}
+
+// Splits of the token range per (b,h) for the key-side reduction: enough CTAs to fill the GPU,
+// never shorter than 256 tokens each; a function of (G, n) only, so results are reproducible.
+int choose_splits(long long G, int n, int forced)
+{
+    long long s = forced > 0 ? forced : (kTargetCtas + G - 1) / G;
+    const long long by_len = (n + 255) / 256;
+    if (forced <= 0 && s > by_len) s = by_len;
+    if (s > n) s = n;
+    if (s > kMaxSplits) s = kMaxSplits;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+template <typename T, int D>
+linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int n,
+                           cudaStream_t st)
+{
+    const long long G = (long long)B * c->H;
+    int splits = choose_splits(G, n, c->opt_splits);
+    // token chunk per split, rounded up to the kernel's 32-token step; drop splits left empty
+    int chunk = (n + splits - 1) / splits;
+    chunk = (chunk + kSimtTokens - 1) / kSimtTokens * kSimtTokens;
+    splits = (n + chunk - 1) / chunk;
+    if (G * splits > c->partial_slots) return LINATTN_ERR_WORKSPACE;
+    constexpr int E = D * D + D;
+
+    static bool attr_done = false;  // per process and template instance; setting it twice is harmless
+    if (!attr_done) {
+        LA_CUDA(c, cudaFuncSetAttribute(kside_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kside_simt_smem<D>()));
+        LA_CUDA(c, cudaFuncSetAttribute(qside_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)qside_simt_smem<D>()));
+        attr_done = true;
+    }
+    const double side_bytes = 2.0 * (double)G * n * D * sizeof(T);  // K+V read, or Q read + O written
+    prof_begin(c, st);
+    kside_simt<T, D><<<dim3(splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
+        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "kside_simt", side_bytes);
+    combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, c->state, splits, E);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "combine_state", 0.0);
+    const int nchunks = (n + kSimtTokens - 1) / kSimtTokens;
+    long long per_group = (2LL * 148 + G - 1) / G;
+    if (per_group > nchunks) per_group = nchunks;
+    if (per_group < 1) per_group = 1;
+    qside_simt<T, D><<<dim3((unsigned)per_group, (unsigned)G), kSimtThreads, qside_simt_smem<D>(), st>>>(
+        (const T*)q, c->Wq, c->state, (T*)out, c->H, n);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "qside_simt", side_bytes);
+    c->last_launches = 3;
+    return LINATTN_OK;
+}
+
+bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+bool overlaps(const void* a, const void* b, size_t bytes)
+{
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + bytes && y < x + bytes;
+}
+
+linattn_status check_forward_args(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B,
+                                  int H, int n, int d, linattn_dtype dtype)
+{
+    if (!c || !q || !k || !v || !out) return LINATTN_ERR_INVALID_ARG;
+    if (dtype != LINATTN_F32 && dtype != LINATTN_BF16) return LINATTN_ERR_UNSUPPORTED;
+    if (d != 64 && d != 128) return LINATTN_ERR_UNSUPPORTED;
+    if (H != c->H || d != c->d) return LINATTN_ERR_INVALID_ARG;
+    if (B < 1 || n < 1) return LINATTN_ERR_INVALID_ARG;
+    if (B > c->max_B || n > c->max_n) return LINATTN_ERR_WORKSPACE;
+    if (!c->have_map) return LINATTN_ERR_NO_FEATURE_MAP;
+    return LINATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* linattn_status_string(linattn_status s)
+{
+    switch (s) {
+        case LINATTN_OK: return "ok";
+        case LINATTN_ERR_INVALID_ARG: return "invalid argument";
+        case LINATTN_ERR_UNSUPPORTED: return "unsupported head dimension, dtype or device";
+        case LINATTN_ERR_NO_FEATURE_MAP: return "feature map not set";
+        case LINATTN_ERR_WORKSPACE: return "request exceeds the workspace reserved at create";
+        case LINATTN_ERR_CUDA: return "CUDA error";
+        case LINATTN_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, long long max_B, long long max_n)
+{
+    if (!out_ctx || H < 1 || max_B < 1 || max_n < 1 || device < 0) return LINATTN_ERR_INVALID_ARG;
+    if (max_n > 0x7fffffffLL || max_B * H > 65535) return LINATTN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return LINATTN_ERR_UNSUPPORTED;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device >= ndev) {
+        cudaGetLastError();
+        return LINATTN_ERR_CUDA;
+    }
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess)
+        return LINATTN_ERR_CUDA;
+    if (major != 10) return LINATTN_ERR_UNSUPPORTED;
+
+    linattn_ctx* c = new (std::nothrow) linattn_ctx();
+    if (!c) return LINATTN_ERR_INVALID_ARG;
+    c->device = device;
+    c->H = H;
+    c->d = d;
+    c->max_B = max_B;
+    c->max_n = max_n;
+    DeviceGuard guard(device);
+    const size_t E = (size_t)d * d + d;
+    const size_t wbytes = sizeof(float) * (size_t)H * d * (d / 2);
+    const long long G = max_B * H;
+    c->partial_slots = kTargetCtas + G;
+    cudaError_t e = cudaSuccess;
+    if (e == cudaSuccess) e = cudaMalloc(&c->Wq, wbytes);
+    if (e == cudaSuccess) e = cudaMalloc(&c->Wk, wbytes);
+    if (e == cudaSuccess) e = cudaMalloc(&c->partial, sizeof(float) * E * (size_t)c->partial_slots);
+    if (e == cudaSuccess) e = cudaMalloc(&c->state, sizeof(float) * E * (size_t)G);
+    if (e == cudaSuccess) e = cudaMalloc(&c->err_word, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(c->err_word, 0, sizeof(unsigned int));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        linattn_destroy(c);
+        return LINATTN_ERR_CUDA;
+    }
+    *out_ctx = c;
+    return LINATTN_OK;
+}
+
+linattn_status linattn_destroy(linattn_ctx* c)
+{
+    if (!c) return LINATTN_OK;
+    DeviceGuard guard(c->device);
+    cudaDeviceSynchronize();
+    cudaFree(c->Wq);
+    cudaFree(c->Wk);
+    cudaFree(c->partial);
+    cudaFree(c->state);
+    cudaFree(c->err_word);
+    for (void* p : c->stage) cudaFree(p);
+    for (cudaEvent_t ev : c->prof_ev)
+        if (ev) cudaEventDestroy(ev);
+    cudaGetLastError();
+    delete c;
+    return LINATTN_OK;
+}
+
+linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const void* Wk, int per_head,
+                                       linattn_dtype wdtype, void* stream)
+{
+    if (!c || !Wq || !Wk) return LINATTN_ERR_INVALID_ARG;
+    if (wdtype != LINATTN_F32 && wdtype != LINATTN_BF16) return LINATTN_ERR_UNSUPPORTED;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const int DM = c->d * (c->d / 2);
+    const size_t total = (size_t)c->H * DM;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    if (wdtype == LINATTN_F32) {
+        convert_weights<float><<<blocks, 256, 0, st>>>((const float*)Wq, c->Wq, c->H, DM, per_head ? 1 : 0);
+        convert_weights<float><<<blocks, 256, 0, st>>>((const float*)Wk, c->Wk, c->H, DM, per_head ? 1 : 0);
+    } else {
+        convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wq, c->H, DM, per_head ? 1 : 0);
+        convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wk, c->H, DM, per_head ? 1 : 0);
+    }
+    LA_CUDA(c, cudaGetLastError());
+    c->have_map = true;
+    return LINATTN_OK;
+}
+
+linattn_status linattn_forward(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int H,
+                               int n, int d, linattn_dtype dtype, void* stream)
+{
+    linattn_status s = check_forward_args(c, q, k, v, out, B, H, n, d, dtype);
+    if (s != LINATTN_OK) return s;
+    if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(out)) return LINATTN_ERR_INVALID_ARG;
+    const size_t bytes = (size_t)B * H * n * d * elem_size(dtype);
+    if (overlaps(out, q, bytes) || overlaps(out, k, bytes) || overlaps(out, v, bytes)) return LINATTN_ERR_INVALID_ARG;
+    if (c->opt_path == 2) return LINATTN_ERR_UNSUPPORTED;  // tensor-core path not built into this library
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    c->last_B = B;
+    if (dtype == LINATTN_BF16) {
+        return d == 128 ? launch_simt<__nv_bfloat16, 128>(c, q, k, v, out, B, n, st)
+                        : launch_simt<__nv_bfloat16, 64>(c, q, k, v, out, B, n, st);
+    }
+    return d == 128 ? launch_simt<float, 128>(c, q, k, v, out, B, n, st)
+                    : launch_simt<float, 64>(c, q, k, v, out, B, n, st);
+}
+
+linattn_status linattn_forward_host(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B,
+                                    int H, int n, int d, linattn_dtype dtype, void* stream)
+{
+    linattn_status s = check_forward_args(c, q, k, v, out, B, H, n, d, dtype);
+    if (s != LINATTN_OK) return s;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = (size_t)B * H * n * d * elem_size(dtype);
+    if (bytes > c->stage_bytes) {
+        LA_CUDA(c, cudaStreamSynchronize(st));
+        for (void*& p : c->stage) {
+            cudaFree(p);
+            p = nullptr;
+        }
+        c->stage_bytes = 0;
+        for (void*& p : c->stage) LA_CUDA(c, cudaMalloc(&p, bytes));
+        c->stage_bytes = bytes;
+    }
+    LA_CUDA(c, cudaMemcpyAsync(c->stage[0], q, bytes, cudaMemcpyHostToDevice, st));
+    LA_CUDA(c, cudaMemcpyAsync(c->stage[1], k, bytes, cudaMemcpyHostToDevice, st));
+    LA_CUDA(c, cudaMemcpyAsync(c->stage[2], v, bytes, cudaMemcpyHostToDevice, st));
+    s = linattn_forward(c, c->stage[0], c->stage[1], c->stage[2], c->stage[3], B, H, n, d, dtype, stream);
+    if (s != LINATTN_OK) return s;
+    LA_CUDA(c, cudaMemcpyAsync(out, c->stage[3], bytes, cudaMemcpyDeviceToHost, st));
+    LA_CUDA(c, cudaStreamSynchronize(st));
+    return LINATTN_OK;
+}
+
+linattn_status linattn_read_state(linattn_ctx* c, float* S_host, float* z_host, int B, void* stream)
+{
+    if (!c || B < 1 || B > c->max_B) return LINATTN_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t dd = (size_t)c->d * c->d, E = dd + c->d;
+    const size_t G = (size_t)B * c->H;
+    if (S_host)
+        LA_CUDA(c, cudaMemcpy2DAsync(S_host, dd * sizeof(float), c->state, E * sizeof(float), dd * sizeof(float), G,
+                                     cudaMemcpyDeviceToHost, st));
+    if (z_host)
+        LA_CUDA(c, cudaMemcpy2DAsync(z_host, c->d * sizeof(float), c->state + dd, E * sizeof(float),
+                                     c->d * sizeof(float), G, cudaMemcpyDeviceToHost, st));
+    LA_CUDA(c, cudaStreamSynchronize(st));
+    return LINATTN_OK;
+}
+
+linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long value)
+{
+    if (!c) return LINATTN_ERR_INVALID_ARG;
+    switch (opt) {
+        case LINATTN_OPT_SPLITS:
+            if (value < 0 || value > kMaxSplits) return LINATTN_ERR_INVALID_ARG;
+            c->opt_splits = (int)value;
+            return LINATTN_OK;
+        case LINATTN_OPT_PATH:
+            if (value < 0 || value > 2) return LINATTN_ERR_INVALID_ARG;
+            c->opt_path = (int)value;
+            return LINATTN_OK;
+        case LINATTN_OPT_PROFILE: {
+            if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
+            DeviceGuard guard(c->device);
+            if (value == 1) {
+                for (cudaEvent_t& ev : c->prof_ev)
+                    if (!ev) LA_CUDA(c, cudaEventCreate(&ev));
+                if (!c->profile) {  // a fresh measurement
+                    for (int i = 0; i < linattn_ctx::kMaxKernels; ++i) {
+                        c->prof_ms[i] = 0.0;
+                        c->prof_cnt[i] = 0;
+                    }
+                }
+            } else {
+                prof_flush(c);
+            }
+            c->profile = (value == 1);
+            return LINATTN_OK;
+        }
+    }
+    return LINATTN_ERR_INVALID_ARG;
+}
+
+linattn_status linattn_check(linattn_ctx* c, void* stream)
+{
+    if (!c) return LINATTN_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    LA_CUDA(c, cudaStreamSynchronize(st));
+    unsigned int w = 0;
+    LA_CUDA(c, cudaMemcpyAsync(&w, c->err_word, sizeof(w), cudaMemcpyDeviceToHost, st));
+    LA_CUDA(c, cudaStreamSynchronize(st));
+    if (w != 0) {
+        LA_CUDA(c, cudaMemsetAsync(c->err_word, 0, sizeof(w), st));
+        snprintf(c->err_text, sizeof(c->err_text), "device-side wait gave up (code 0x%x)", w);
+        return LINATTN_ERR_TIMEOUT;
+    }
+    return LINATTN_OK;
+}
+
+int linattn_profile_get(linattn_ctx* c, int index, const char** name, double* mean_ms, long long* launches,
+                        double* algorithmic_bytes)
+{
+    if (!c || index < 0) return 0;
+    {
+        DeviceGuard guard(c->device);
+        prof_flush(c);
+    }
+    if (index >= c->prof_n || c->prof_cnt[index] == 0) return 0;
+    if (name) *name = c->prof_name[index];
+    if (mean_ms) *mean_ms = c->prof_ms[index] / (double)c->prof_cnt[index];
+    if (launches) *launches = c->prof_cnt[index];
+    if (algorithmic_bytes) *algorithmic_bytes = c->prof_bytes[index];
+    return 1;
+}
+
+int linattn_last_launch_count(const linattn_ctx* c) { return c ? c->last_launches : 0; }
+
+const char* linattn_last_error(const linattn_ctx* c) { return c ? c->err_text : ""; }
+
+}  // extern "C"

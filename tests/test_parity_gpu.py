@@ -1,0 +1,206 @@
+"""GPU parity: the CUDA library, called through its C-ABI, against the fp64 CPU oracle.
+
+Tolerances (on the whole output tensor, outputs widened to fp64):
+    relative L2 <= 5e-3 and max-abs <= 2e-2.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_08318_b200 import linattn, synth
+from util import assert_parity, errors, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [linattn.PATH_AUTO, linattn.PATH_SIMT]
+
+
+def small_inputs(B, H, n, d, dtype, seed, wmode="random"):
+    """Inputs with the value distributions of the bf16 workloads (N(0,1)/sqrt(d), unit-variance logits)."""
+    g = torch.Generator().manual_seed(seed)
+    sx = 1.0 / math.sqrt(d)
+    q, k, v = (torch.randn(B, H, n, d, generator=g) * sx for _ in range(3))
+    if wmode == "random":
+        Wq, Wk = (torch.randn(H, d, d // 2, generator=g) / (math.sqrt(d) * sx) for _ in range(2))
+    elif wmode == "zero":
+        Wq = Wk = torch.zeros(H, d, d // 2)
+    elif wmode == "identity":  # truncated identity [I ; 0], near-identity initialisation of the feature map
+        Wq = Wk = torch.eye(d)[:, : d // 2].expand(H, d, d // 2).contiguous() * 8.0
+    elif wmode == "shared":
+        Wq, Wk = (torch.randn(d, d // 2, generator=g) / (math.sqrt(d) * sx) for _ in range(2))
+    return {"q": q.to(dtype), "k": k.to(dtype), "v": v.to(dtype), "Wq": Wq.to(dtype), "Wk": Wk.to(dtype)}
+
+
+def oracle_out(x, rows=None):
+    return oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], rows=rows)
+
+
+# ---- config 1: the tiny fp32 case against the O(n^2) brute-force form --------------------------
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config1_tiny_against_quadratic_form(path):
+    x = synth.make_inputs(1)
+    got, S, z = run_gpu(x, path=path, return_state=True)
+    want = oracle.ref_quadratic(x["q"], x["k"], x["v"], x["Wq"], x["Wk"])
+    assert_parity(got, want, "config 1 vs quadratic form")
+    _, S_ref, z_ref = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], return_state=True)
+    assert errors(S, S_ref)[0] <= 5e-3 and errors(z, z_ref)[0] <= 5e-3
+
+
+# ---- ragged sizes: several tiles plus a tail, the degenerate n = 1, 2 -----------------------------
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n", [1, 2, 127, 129, 1000, 4097])
+def test_ragged_lengths(n, d, dtype, path):
+    x = small_inputs(2, 3, n, d, dtype, seed=1000 + n + d)
+    got, S, z = run_gpu(x, path=path, return_state=True)
+    assert_parity(got, oracle_out(x), f"n={n} d={d} {dtype}")
+    _, S_ref, z_ref = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], return_state=True)
+    assert errors(z, z_ref)[0] <= 5e-3, "z"
+    assert abs(z.sum(-1) - 2.0 * n).max() <= 2e-3 * 2.0 * n, "sum(z) must be 2n: padded rows leaked into z"
+    if n == 1:
+        assert_parity(got, x["v"].double().numpy(), "n=1 returns v")
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("splits", [1, 2, 3, 7, 33])
+def test_split_count_does_not_change_the_answer(splits, path):
+    x = small_inputs(1, 2, 2500, 128, torch.bfloat16, seed=77)
+    got = run_gpu(x, path=path, splits=splits)
+    assert_parity(got, oracle_out(x), f"splits={splits}")
+
+
+# ---- special feature maps ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_zero_weights_give_the_mean_of_v(dtype, path):
+    x = small_inputs(1, 2, 777, 128, dtype, seed=5, wmode="zero")
+    got = run_gpu(x, path=path)
+    mean_v = x["v"].double().numpy().mean(axis=2, keepdims=True)
+    assert_parity(got, np.broadcast_to(mean_v, got.shape), "W=0 -> mean of V")
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("wmode", ["identity", "shared"])
+def test_identity_and_shared_weights(wmode, path):
+    x = small_inputs(2, 2, 900, 128, torch.bfloat16, seed=6, wmode=wmode)
+    assert_parity(run_gpu(x, path=path), oracle_out(x), wmode)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_large_logits_do_not_overflow(path):
+    """Logits of magnitude ~50: exp without max subtraction would overflow fp32 sums / underflow to 0/0."""
+    x = small_inputs(1, 2, 600, 128, torch.bfloat16, seed=8)
+    x["Wq"] = (x["Wq"].float() * 40).to(torch.bfloat16)
+    x["Wk"] = (x["Wk"].float() * 40).to(torch.bfloat16)
+    assert_parity(run_gpu(x, path=path), oracle_out(x), "large logits")
+
+
+# ---- reduced-size versions of the bf16 workloads (same distributions, fewer heads / tokens) ----------
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("config,H,n", [(2, 3, 4216), (3, 4, 4216), (4, 2, 9300), (5, 3, 4216)])
+def test_reduced_workloads(config, H, n, path):
+    x = synth.make_inputs(config, H=H, n=n)
+    assert_parity(run_gpu(x, path=path), oracle_out(x), f"config {config} reduced")
+
+
+# ---- determinism and context reuse --------------------------------------------------------------------
+
+@pytest.mark.parametrize("path", PATHS)
+def test_bit_identical_across_runs_and_context_reuse(path):
+    x = small_inputs(2, 4, 3000, 128, torch.bfloat16, seed=9)
+    ctx = linattn.LinAttn(4, 128, max_B=2, max_n=4000)
+    try:
+        ctx.set_option(linattn.OPT_PATH, path)
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        q, k, v = x["q"].cuda(), x["k"].cuda(), x["v"].cuda()
+        first = ctx.forward(q, k, v).clone()
+        for _ in range(20):
+            again = ctx.forward(q, k, v)
+            assert torch.equal(first, again)
+        # a different, shorter problem on the same context, then the first one again
+        y = small_inputs(1, 4, 333, 128, torch.bfloat16, seed=10)
+        ctx.set_feature_map(y["Wq"].cuda(), y["Wk"].cuda())
+        got = ctx.forward(y["q"].cuda(), y["k"].cuda(), y["v"].cuda()).cpu().double().numpy()
+        assert_parity(got, oracle_out(y), "second problem on the same context")
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        assert torch.equal(first, ctx.forward(q, k, v))
+        ctx.check()
+    finally:
+        ctx.destroy()
+
+
+def test_output_guard_bands_are_untouched():
+    """The kernels must write exactly B*H*n*d elements: canaries on both sides of `out` survive."""
+    x = small_inputs(1, 2, 1000, 128, torch.bfloat16, seed=11)
+    B, H, n, d = x["q"].shape
+    pad = 4096
+    buf = torch.full((pad + B * H * n * d + pad,), 7.0, dtype=torch.bfloat16, device="cuda")
+    out = buf[pad:pad + B * H * n * d].view(B, H, n, d)
+    ctx = linattn.LinAttn(H, d, max_B=B, max_n=n)
+    try:
+        for path in PATHS:
+            ctx.set_option(linattn.OPT_PATH, path)
+            ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+            ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda(), out=out)
+            ctx.check()
+            assert (buf[:pad] == 7.0).all() and (buf[-pad:] == 7.0).all()
+            assert_parity(out.cpu().double().numpy(), oracle_out(x), "guarded output")
+    finally:
+        ctx.destroy()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    x = small_inputs(1, 2, 1500, 128, torch.bfloat16, seed=12)
+    ctx = linattn.LinAttn(2, 128, max_B=1, max_n=1500)
+    try:
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        dev = ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda()).cpu()
+        host_out = torch.empty_like(x["q"])
+        ctx.forward_host(x["q"], x["k"], x["v"], host_out)
+        assert torch.equal(dev, host_out)
+        pin = {k_: x[k_].pin_memory() for k_ in ("q", "k", "v")}
+        host_out2 = torch.empty_like(x["q"]).pin_memory()
+        ctx.forward_host(pin["q"], pin["k"], pin["v"], host_out2)
+        assert torch.equal(dev, host_out2)
+    finally:
+        ctx.destroy()
+
+
+# ---- argument checking on a live context (host-side; nothing invalid reaches a kernel) ------------------
+
+def test_forward_argument_errors():
+    lib = linattn.load_library()
+    x = small_inputs(1, 2, 256, 128, torch.bfloat16, seed=13)
+    q, k, v = x["q"].cuda(), x["k"].cuda(), x["v"].cuda()
+    out = torch.empty_like(q)
+    ctx = linattn.LinAttn(2, 128, max_B=1, max_n=256)
+    try:
+        def fwd(qp, kp, vp, op, B=1, H=2, n=256, d=128, dt=linattn.BF16):
+            return lib.linattn_forward(ctx._h, qp, kp, vp, op, B, H, n, d, dt, None)
+        P = (q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr())
+        assert fwd(*P) == linattn.ERR_NO_FEATURE_MAP
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        assert fwd(*P) == linattn.OK
+        assert fwd(None, P[1], P[2], P[3]) == linattn.ERR_INVALID_ARG
+        assert fwd(P[0] + 2, P[1], P[2], P[3]) == linattn.ERR_INVALID_ARG       # misaligned
+        assert fwd(P[0], P[1], P[2], P[0]) == linattn.ERR_INVALID_ARG           # out aliases q
+        assert fwd(*P, H=3) == linattn.ERR_INVALID_ARG
+        assert fwd(*P, d=64) == linattn.ERR_INVALID_ARG
+        assert fwd(*P, d=96) == linattn.ERR_UNSUPPORTED
+        assert fwd(*P, dt=7) == linattn.ERR_UNSUPPORTED
+        assert fwd(*P, n=0) == linattn.ERR_INVALID_ARG
+        assert fwd(*P, n=257) == linattn.ERR_WORKSPACE
+        assert fwd(*P, B=2) == linattn.ERR_WORKSPACE
+        assert lib.linattn_set_option(ctx._h, 99, 0) == linattn.ERR_INVALID_ARG
+        assert lib.linattn_set_option(ctx._h, linattn.OPT_SPLITS, -1) == linattn.ERR_INVALID_ARG
+        ctx.check()
+    finally:
+        ctx.destroy()
