@@ -97,6 +97,32 @@ linattn_status linattn_forward_host(linattn_ctx* ctx, const void* q, const void*
  */
 linattn_status linattn_read_state(linattn_ctx* ctx, float* S_host, float* z_host, int B, void* stream);
 
+/*
+ * The forward for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a property of the library, not of the method.)  Typical cases: a plug-in that is handed
+ * pointers and a stream by a framework whose memory pool it may not touch; a latency-critical
+ * serving thread, where cudaMalloc / cudaFree would synchronise the whole device; code that must
+ * not fail for lack of memory at call time.  It needs no context: the feature-map weights are
+ * passed in, and the scratch for the partial and combined S, z of Eq. 5 is a fixed array inside
+ * the library's device image (about 5.3 MB, held by every GPU that loads the library until the
+ * process exits).  It calls no allocator of any kind and computes the same operation as
+ * linattn_forward with the CUDA-core kernels.
+ *   q, k, v, out : as for linattn_forward (device, [B][H][n][d] of `dtype`, 16-byte aligned)
+ *   Wq, Wk       : device, fp32, 16-byte aligned, [H][d][d/2] (per_head != 0) or [d][d/2]; read, not copied
+ *   limits       : B * H <= 16 and d in {64, 128}; any n >= 1.  A larger B * H returns
+ *                  LINATTN_ERR_WORKSPACE ("request exceeds the workspace ...") and launches nothing.
+ * Runs on the CURRENT device.  The first call on each device looks up the device address of the
+ * scratch array and raises the kernels' shared-memory limit; make that first call before any
+ * stream capture begins.  All calls on a device share the one scratch array: it keeps the previous
+ * call's contents, every element a call reads is first written by that same call (nothing needs
+ * clearing), and two calls whose kernels overlap on the GPU (different streams, no ordering) race
+ * on it and give wrong results -- keep calls on one device stream-ordered.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ */
+linattn_status linattn_forward_noalloc(const void* q, const void* k, const void* v, void* out,
+                                       const float* Wq, const float* Wk, int per_head,
+                                       int B, int H, int n, int d, linattn_dtype dtype, void* stream);
+
 /* Tuning and test knobs; see linattn_option.  Errors: INVALID_ARG (unknown option or value). */
 linattn_status linattn_set_option(linattn_ctx* ctx, linattn_option opt, long long value);
 

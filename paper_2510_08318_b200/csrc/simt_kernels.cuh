@@ -168,7 +168,7 @@ kside_simt(const T* __restrict__ k, const T* __restrict__ v, const float* __rest
 }
 
 // state[g][e] = sum_{s=0..splits-1} partial[g][s][e], s ascending.  grid = (ceil(E/256), G), E = D*D + D.
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 combine_state(const float* __restrict__ partial, float* __restrict__ state, int splits, int E)
 {
     const int e = blockIdx.x * 256 + threadIdx.x;

@@ -28,6 +28,7 @@ SIGNATURES = {
     "linattn_set_feature_map": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "linattn_forward": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_host": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "linattn_forward_noalloc": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "linattn_read_state": (_i, [_vp, _vp, _vp, _i, _vp]),
     "linattn_set_option": (_i, [_vp, _i, _ll]),
     "linattn_check": (_i, [_vp, _vp]),
@@ -72,6 +73,28 @@ def _stream_ptr(stream) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
     return stream.cuda_stream
+
+
+def forward_noalloc(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, Wq: torch.Tensor, Wk: torch.Tensor,
+                    out: torch.Tensor, stream=None) -> torch.Tensor:
+    """``linattn_forward_noalloc``: the forward for callers that may not allocate device memory.
+
+    No context and no allocation inside the library: q, k, v, out are contiguous CUDA tensors
+    [B, H, n, d] (the caller provides ``out``), Wq and Wk are fp32 CUDA tensors [H, d, d/2] or
+    [d, d/2], and the scratch lives in a fixed device array of the library (B * H <= 16).
+    Runs on the current device; calls on one device must be stream-ordered."""
+    lib = load_library()
+    for t in (q, k, v, out, Wq, Wk):
+        assert t.is_cuda and t.is_contiguous()
+    assert q.shape == k.shape == v.shape == out.shape and q.dtype == k.dtype == v.dtype == out.dtype
+    assert Wq.dtype == torch.float32 and Wk.dtype == torch.float32 and Wq.shape == Wk.shape
+    B, H, n, d = q.shape
+    st = lib.linattn_forward_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), Wq.data_ptr(),
+                                     Wk.data_ptr(), 1 if Wq.dim() == 3 else 0, B, H, n, d, _DTYPES[q.dtype],
+                                     _stream_ptr(stream))
+    if st != OK:
+        raise LinAttnError(st, status_string(st))
+    return out
 
 
 class LinAttn:
