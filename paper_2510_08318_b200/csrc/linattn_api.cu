@@ -11,6 +11,8 @@
 #include <new>
 
 #include "simt_kernels.cuh"
+#include "sm100_kernels.cuh"
+#include "tensor_map.hpp"
 
 using namespace linattn;
 
@@ -42,6 +44,13 @@ struct linattn_ctx {
     // weights, fp32 [H][d][d/2]
     float* Wq = nullptr;
     float* Wk = nullptr;
+    // weights for the tensor-core path: bf16 W^T [H][d/2][d] (d = 128 only)
+    __nv_bfloat16* Wqt = nullptr;
+    __nv_bfloat16* Wkt = nullptr;
+    bool map_is_bf16 = false;   // the caller supplied bf16 weights (the tensor-core path uses them unrounded)
+    __nv_bfloat16* s_img = nullptr;  // [max_B*H][128*128] bf16 image of S for the query-side TMA
+    __nv_bfloat16* z_img = nullptr;  // [max_B*H][2048] bf16 operand image of z (hi, lo)
+    int num_sms = 0;
     // workspace
     float* partial = nullptr;   // [partial_slots][d*d + d]
     long long partial_slots = 0;
@@ -177,6 +186,58 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     return LINATTN_OK;
 }
 
+// Tensor-core path: bf16, d = 128.
+linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int n,
+                         cudaStream_t st)
+{
+    using namespace linattn::tc;
+    const long long G = (long long)B * c->H;
+    const long long Tn = ((long long)n + kTile - 1) / kTile;
+    const long long T = G * Tn;
+    long long Pq = c->num_sms < T ? c->num_sms : T;
+    long long Pk = Pq;
+    if (c->opt_splits > 0) {
+        Pk = G * c->opt_splits;
+        if (Pk > T) Pk = T;
+    }
+    if (Pk + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
+
+    CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmS;
+    const bool ok = make_tmap_bf16_3d(&tmK, k, kD, (uint64_t)n, (uint64_t)G, kTile) &&
+                    make_tmap_bf16_3d(&tmV, v, kD, (uint64_t)n, (uint64_t)G, kTile) &&
+                    make_tmap_bf16_3d(&tmQ, q, kD, (uint64_t)n, (uint64_t)G, kTile) &&
+                    make_tmap_bf16_3d(&tmO, out, kD, (uint64_t)n, (uint64_t)G, kTile) &&
+                    make_tmap_bf16_3d(&tmWk, c->Wkt, kD, kM, (uint64_t)c->H, kM) &&
+                    make_tmap_bf16_3d(&tmWq, c->Wqt, kD, kM, (uint64_t)c->H, kM) &&
+                    make_tmap_bf16_3d(&tmS, c->s_img, kD, kD, (uint64_t)G, kTile);
+    if (!ok) {
+        snprintf(c->err_text, sizeof(c->err_text), "cuTensorMapEncodeTiled failed");
+        return LINATTN_ERR_CUDA;
+    }
+    static bool attr_done = false;
+    if (!attr_done) {
+        LA_CUDA(c, cudaFuncSetAttribute(kside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KSideSmem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(qside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QSideSmem::kTotal));
+        attr_done = true;
+    }
+    const double side_bytes = 2.0 * (double)G * n * kD * 2;
+    prof_begin(c, st);
+    KSideArgs ka{c->partial, c->err_word, n, c->H, Tn, T};
+    kside_tc<<<(unsigned)Pk, kThreads, KSideSmem::kTotal, st>>>(tmK, tmV, tmWk, ka);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "kside_tc", side_bytes);
+    CombineArgs ca{c->partial, c->state, c->s_img, c->z_img, Tn, T, Pk};
+    combine_tc<<<dim3((kE + 255) / 256, (unsigned)G), 256, 0, st>>>(ca);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "combine_tc", 0.0);
+    QSideArgs qa{c->z_img, c->err_word, n, c->H, Tn, T};
+    qside_tc<<<(unsigned)Pq, kQThreads, QSideSmem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, qa);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "qside_tc", side_bytes);
+    c->last_launches = 3;
+    return LINATTN_OK;
+}
+
 bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
 bool overlaps(const void* a, const void* b, size_t bytes)
@@ -248,6 +309,15 @@ linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, l
     if (e == cudaSuccess) e = cudaMalloc(&c->Wk, wbytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->partial, sizeof(float) * E * (size_t)c->partial_slots);
     if (e == cudaSuccess) e = cudaMalloc(&c->state, sizeof(float) * E * (size_t)G);
+    if (e == cudaSuccess && d == 128) {
+        const size_t wt = sizeof(__nv_bfloat16) * (size_t)H * d * (d / 2);
+        e = cudaMalloc(&c->Wqt, wt);
+        if (e == cudaSuccess) e = cudaMalloc(&c->Wkt, wt);
+        if (e == cudaSuccess) e = cudaMalloc(&c->s_img, sizeof(__nv_bfloat16) * (size_t)G * d * d);
+        if (e == cudaSuccess) e = cudaMalloc(&c->z_img, (size_t)G * linattn::tc::kZBlkBytes);
+        if (e == cudaSuccess) e = cudaMemset(c->z_img, 0, (size_t)G * linattn::tc::kZBlkBytes);
+    }
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaMalloc(&c->err_word, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->err_word, 0, sizeof(unsigned int));
     if (e != cudaSuccess) {
@@ -269,6 +339,10 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->partial);
     cudaFree(c->state);
     cudaFree(c->err_word);
+    cudaFree(c->Wqt);
+    cudaFree(c->Wkt);
+    cudaFree(c->s_img);
+    cudaFree(c->z_img);
     for (void* p : c->stage) cudaFree(p);
     for (cudaEvent_t ev : c->prof_ev)
         if (ev) cudaEventDestroy(ev);
@@ -294,7 +368,18 @@ linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const voi
         convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wq, c->H, DM, per_head ? 1 : 0);
         convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wk, c->H, DM, per_head ? 1 : 0);
     }
+    if (c->d == 128) {
+        const unsigned tb = (unsigned)(((size_t)c->H * DM + 255) / 256);
+        if (wdtype == LINATTN_F32) {
+            tc::transpose_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
+            tc::transpose_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
+        } else {
+            tc::transpose_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
+            tc::transpose_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
+        }
+    }
     LA_CUDA(c, cudaGetLastError());
+    c->map_is_bf16 = (wdtype == LINATTN_BF16);
     c->have_map = true;
     return LINATTN_OK;
 }
@@ -307,10 +392,14 @@ linattn_status linattn_forward(linattn_ctx* c, const void* q, const void* k, con
     if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(out)) return LINATTN_ERR_INVALID_ARG;
     const size_t bytes = (size_t)B * H * n * d * elem_size(dtype);
     if (overlaps(out, q, bytes) || overlaps(out, k, bytes) || overlaps(out, v, bytes)) return LINATTN_ERR_INVALID_ARG;
-    if (c->opt_path == 2) return LINATTN_ERR_UNSUPPORTED;  // tensor-core path not built into this library
+    // The tensor-core kernels cover bf16 activations with head dimension 128 and bf16 feature-map weights;
+    // everything else runs on the CUDA-core kernels.
+    const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && c->map_is_bf16);
+    if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     c->last_B = B;
+    if (tc_ok && c->opt_path != 1) return launch_tc(c, q, k, v, out, B, n, st);
     if (dtype == LINATTN_BF16) {
         return d == 128 ? launch_simt<__nv_bfloat16, 128>(c, q, k, v, out, B, n, st)
                         : launch_simt<__nv_bfloat16, 64>(c, q, k, v, out, B, n, st);
