@@ -222,15 +222,15 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     }
     const double side_bytes = 2.0 * (double)G * n * kD * 2;
     prof_begin(c, st);
-    KSideArgs ka{c->partial, c->err_word, n, c->H, Tn, T};
-    kside_tc<<<(unsigned)Pk, kThreads, KSideSmem::kTotal, st>>>(tmK, tmV, tmWk, ka);
+    KSideArgs ka{c->partial, c->err_word, n, c->H, (int)Tn, T};
+    kside_tc<<<(unsigned)Pk, kKThreads, KSideSmem::kTotal, st>>>(tmK, tmV, tmWk, ka);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_tc", side_bytes);
     CombineArgs ca{c->partial, c->state, c->s_img, c->z_img, Tn, T, Pk};
     combine_tc<<<dim3((kE + 255) / 256, (unsigned)G), 256, 0, st>>>(ca);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_tc", 0.0);
-    QSideArgs qa{c->z_img, c->err_word, n, c->H, Tn, T};
+    QSideArgs qa{c->z_img, c->err_word, n, c->H, (int)Tn, T};
     qside_tc<<<(unsigned)Pq, kQThreads, QSideSmem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, qa);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);

@@ -16,9 +16,10 @@
 //
 // Work split: the G * ceil(n/128) tiles form one sequence (head-major); CTA c of P owns the contiguous
 // run [c*T/P, (c+1)*T/P).  A run may cross head boundaries; each (CTA, head) piece is a "segment".
-// Warp roles in both streaming kernels: warps 0-3 feature map of softmax(+U) / output columns 0-63,
-// warps 4-7 softmax(-U) / columns 64-127, warp 8 TMA producer, warp 9 MMA issuer, and (query side only)
-// warp 10 issues the TMA stores.
+// Warp roles: warps 0-3 feature map of softmax(+U) / output columns 0-63, warps 4-7 softmax(-U) / columns
+// 64-127, warp 8 TMA producer, warp 9 issues the logits MMAs, warp 10 issues the accumulation MMAs, and
+// (query side only) warp 11 issues the TMA stores.  Role loops are warp-uniform; single-thread work
+// (TMA and MMA issue) is predicated inside them.
 // Every wait is bounded: on time-out the kernel records a code in *err and unwinds.
 #pragma once
 #include <cuda.h>
@@ -36,8 +37,8 @@ using namespace ptx;
 constexpr int kD = 128;             // head dimension
 constexpr int kM = 64;              // features per softmax half
 constexpr int kTile = 128;          // tokens per tile
-constexpr int kThreads = 320;        // key side
-constexpr int kQThreads = 352;       // query side: one more warp for the stores
+constexpr int kKThreads = 352;      // key side: 11 warps
+constexpr int kQThreads = 384;      // query side: 12 warps
 constexpr int kE = kD * kD + kD;    // floats per (S, z) record
 constexpr uint32_t kTileBytes = kTile * kD * 2;       // 32 KB: one [128 x 128] bf16 tile
 constexpr uint32_t kHalfTileBytes = kTileBytes / 2;   // one 64-column block of a tile
@@ -52,19 +53,61 @@ enum : uint32_t {
     kErrSoftmaxU = 32u, kErrDrain = 64u, kErrEpilogue = 128u, kErrSeg = 256u, kErrStore = 512u
 };
 
-struct Run {
-    long long first, count;  // this CTA's tiles in the global tile sequence
-};
-__device__ __forceinline__ Run cta_run(long long total_tiles)
-{
-    const long long P = gridDim.x, c = blockIdx.x;
-    const long long a = c * total_tiles / P, b = (c + 1) * total_tiles / P;
-    return Run{a, b - a};
-}
-// CTA that owns tile t when T tiles are split over P CTAs as above.
+// CTA that owns tile t when T tiles are split over P CTAs (CTA c owns [c*T/P, (c+1)*T/P)).
 __host__ __device__ __forceinline__ long long tile_owner(long long t, long long T, long long P)
 {
     return ((t + 1) * P - 1) / T;
+}
+
+// Walks this CTA's run of tiles.  g = (batch, head) index, lt = tile within the head, seg = number of
+// head boundaries crossed so far; first / last mark the ends of a segment.
+struct TileWalk {
+    int count, i, g, lt, seg, tiles_per_head;
+    __device__ __forceinline__ void init(long long total_tiles, int tph)
+    {
+        const long long P = gridDim.x, c = blockIdx.x;
+        const long long a = c * total_tiles / P, b = (c + 1) * total_tiles / P;
+        count = (int)(b - a);
+        tiles_per_head = tph;
+        g = (int)(a / tph);
+        lt = (int)(a % tph);
+        i = 0;
+        seg = 0;
+    }
+    __device__ __forceinline__ bool done() const { return i >= count; }
+    __device__ __forceinline__ bool first() const { return i == 0 || lt == 0; }
+    __device__ __forceinline__ bool last() const { return i == count - 1 || lt == tiles_per_head - 1; }
+    __device__ __forceinline__ void next()
+    {
+        ++i;
+        if (++lt == tiles_per_head) {
+            lt = 0;
+            ++g;
+            ++seg;
+        }
+    }
+};
+
+// Ring position: slot index and the parity of the phase a consumer waits for on its n-th visit.
+template <int N> struct Ring {
+    int s = 0;
+    uint32_t ph = 0;
+    __device__ __forceinline__ void next()
+    {
+        if (++s == N) {
+            s = 0;
+            ph ^= 1u;
+        }
+    }
+};
+
+// All lanes wait (bounded); the verdict is made warp-uniform so that role loops never diverge.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, uint32_t* err, uint32_t code)
+{
+    const bool ok = mbar_wait(bar, parity, kWaitLimitNs);
+    const bool all = __all_sync(0xffffffffu, ok);
+    if (!all && (threadIdx.x & 31) == 0) atomicOr(err, code);
+    return all;
 }
 
 __device__ __forceinline__ float ex2_approx(float x)
@@ -122,20 +165,35 @@ __device__ __forceinline__ void load_logits(uint32_t taddr, float (&u)[kM])
     for (int j = 0; j < kM; ++j) u[j] = __uint_as_float(r[j]);
 }
 
-#define LA_WAIT(bar, parity, code)                         \
-    if (!mbar_wait((bar), (parity), kWaitLimitNs)) {       \
-        atomicOr(err, (uint32_t)(code));                   \
-        break;                                             \
-    }
+// Optional per-tile timestamps for tuning (compiled out unless LINATTN_TRACE is defined):
+// trace[((cta * 4 + role) * kTraceTiles + tile) * 4 + event] = clock64.
+#ifdef LINATTN_TRACE
+constexpr int kTraceTiles = 64;
+#define LA_TRACE(role, tile, ev)                                                                         \
+    do {                                                                                                 \
+        if (a.trace && (tile) < kTraceTiles && (threadIdx.x & 31) == 0)                                  \
+            a.trace[(((size_t)blockIdx.x * 4 + (role)) * kTraceTiles + (tile)) * 4 + (ev)] = clock64(); \
+    } while (0)
+#else
+#define LA_TRACE(role, tile, ev) do { } while (0)
+#endif
+
+// Shared-memory descriptor with the address field replaced: descriptors of one operand family differ
+// only in their start address, so the constant part is built once.
+__device__ __forceinline__ uint64_t desc_at(uint64_t base_desc, uint32_t smem_addr)
+{
+    return base_desc | (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+}
 
 // U = X W (Eq. 6 logits) for one tile: A = X tile (K-major), B = W^T (K-major), D = 128 x 64 fp32.
 __device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_smem, uint32_t w_smem)
 {
     constexpr uint32_t idesc = make_idesc_bf16(kTile, kM, 0, 0);
+    const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
 #pragma unroll
     for (int k = 0; k < kD / 16; ++k) {
-        const uint64_t da = make_desc_sw128(x_smem + (k >> 2) * kHalfTileBytes + (k & 3) * 32, 16, 1024);
-        const uint64_t db = make_desc_sw128(w_smem + (k >> 2) * (kWBytes / 2) + (k & 3) * 32, 16, 1024);
+        const uint64_t da = desc_at(kmajor, x_smem + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
+        const uint64_t db = desc_at(kmajor, w_smem + (k >> 2) * (kWBytes / 2) + (k & 3) * 32);
         mma_bf16_ss(d_tmem, da, db, idesc, k > 0);
     }
 }
@@ -157,10 +215,14 @@ struct KSideArgs {
     float* partial;   // [slots][kE]
     uint32_t* err;
     int n, H;
-    long long tiles_per_head, total_tiles;
+    int tiles_per_head;
+    long long total_tiles;
+#ifdef LINATTN_TRACE
+    long long* trace;
+#endif
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kKThreads, 1)
 kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
          const __grid_constant__ CUtensorMap tmW, const KSideArgs a)
 {
@@ -168,14 +230,13 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + KSideSmem::kBars);
-    // barrier indices
     enum { FULL = 0, EMPTY = 3, UFULL = 6, UEMPTY = 8, PHIFULL = 10, WFULL = 13, WFREE = 15, ACCFULL = 17, ACCFREE = 18, NBARS = 19 };
-    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+    const uint32_t bar0 = smem_u32(bars);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[NBARS]);
     uint32_t* err = a.err;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const Run run = cta_run(a.total_tiles);
 
     if (tid == 0) {
         for (int i = 0; i < kKStages; ++i) { mbar_init(bar(FULL + i), 1); mbar_init(bar(EMPTY + i), 1); mbar_init(bar(PHIFULL + i), 8); }
@@ -193,7 +254,7 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
         tma_prefetch_desc(&tmV);
         tma_prefetch_desc(&tmW);
     }
-    for (int i = tid; i < 512; i += kThreads) reinterpret_cast<__nv_bfloat16*>(smem + KSideSmem::kOnes)[i] = __float2bfloat16(1.0f);
+    for (int i = tid; i < 512; i += kKThreads) reinterpret_cast<__nv_bfloat16*>(smem + KSideSmem::kOnes)[i] = __float2bfloat16(1.0f);
     fence_proxy_async_smem();
     tcgen05_fence_before();
     __syncthreads();
@@ -203,149 +264,138 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
     const uint32_t tmem_s = tmem + 128;      // 128 columns: S[f][c], lane = f
     const uint32_t tmem_z = tmem + 256;      // 16 columns: z[f] (all 16 equal)
 
-    if (run.count > 0) {
-        if (warp == 8) {
-            // ---------------- TMA producer ----------------
-            if (lane == 0) {
-                int seg = -1;
-                long long issued = 0;
-                for (long long i = 0; i < run.count; ++i) {
-                    const long long t = run.first + i;
-                    const int g = (int)(t / a.tiles_per_head);
-                    const int lt = (int)(t % a.tiles_per_head);
-                    if (i == 0 || lt == 0) {
-                        ++seg;
-                        const int wb = seg & 1;
-                        if (seg >= 2) LA_WAIT(bar(WFREE + wb), ((seg >> 1) - 1) & 1, kErrProducer);
-                        mbar_arrive_expect_tx(bar(WFULL + wb), kWBytes);
-                        const uint32_t wdst = sbase + KSideSmem::kW + wb * kWBytes;
-                        tma_load_3d(wdst, &tmW, bar(WFULL + wb), 0, 0, g % a.H);
-                        tma_load_3d(wdst + kWBytes / 2, &tmW, bar(WFULL + wb), 64, 0, g % a.H);
-                    }
-                    const int s = (int)(i % kKStages);
-                    if (i >= kKStages) LA_WAIT(bar(EMPTY + s), ((i / kKStages) - 1) & 1, kErrProducer);
-                    mbar_arrive_expect_tx(bar(FULL + s), 2 * kTileBytes);
-                    const uint32_t kdst = sbase + s * KSideSmem::kStage, vdst = kdst + kTileBytes;
-                    tma_load_3d(kdst, &tmK, bar(FULL + s), 0, lt * kTile, g);
-                    tma_load_3d(kdst + kHalfTileBytes, &tmK, bar(FULL + s), 64, lt * kTile, g);
-                    tma_load_3d(vdst, &tmV, bar(FULL + s), 0, lt * kTile, g);
-                    tma_load_3d(vdst + kHalfTileBytes, &tmV, bar(FULL + s), 64, lt * kTile, g);
-                    issued = i + 1;
-                }
-                if (issued < run.count) {
-                    // unwinding after a time-out: let the copies already in flight land before the CTA exits
-                    for (long long i = (issued > kKStages ? issued - kKStages : 0); i < issued; ++i)
-                        mbar_wait(bar(FULL + (int)(i % kKStages)), (i / kKStages) & 1, kWaitLimitNs);
+    TileWalk w;
+    w.init(a.total_tiles, a.tiles_per_head);
+
+    if (warp == 8) {
+        // ---------------- TMA producer ----------------
+        Ring<kKStages> r;
+        int issued = 0;
+        for (; !w.done(); w.next(), r.next()) {
+            if (w.first()) {
+                const int wb = w.seg & 1;
+                if (w.seg >= 2 && !warp_wait(bar(WFREE + wb), ((w.seg >> 1) - 1) & 1, err, kErrProducer)) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar(WFULL + wb), kWBytes);
+                    const uint32_t wdst = sbase + KSideSmem::kW + wb * kWBytes;
+                    tma_load_3d(wdst, &tmW, bar(WFULL + wb), 0, 0, w.g % a.H);
+                    tma_load_3d(wdst + kWBytes / 2, &tmW, bar(WFULL + wb), 64, 0, w.g % a.H);
                 }
             }
-        } else if (warp == 9) {
-            // ---------------- MMA issuer ----------------
+            if (w.i >= kKStages && !warp_wait(bar(EMPTY + r.s), r.ph ^ 1u, err, kErrProducer)) break;
+            LA_TRACE(0, w.i, 0);
             if (lane == 0) {
-                constexpr uint32_t idesc_s = make_idesc_bf16(kD, kD, 1, 1);   // A = phi^T (MN-major), B = V (MN-major)
-                constexpr uint32_t idesc_z = make_idesc_bf16(kD, 16, 1, 0);   // B = ones (K-major, no swizzle)
-                const uint64_t ones_desc = make_desc_noswizzle(sbase + KSideSmem::kOnes, 128, 256);
-                int seg1 = -1;  // segment counter of the logits stream
-                int seg2 = -1;  // segment counter of the accumulation stream
-                bool ok = true;
-                auto do_mma1 = [&](long long i) {
-                    const long long t = run.first + i;
-                    const int lt = (int)(t % a.tiles_per_head);
-                    const bool first = (i == 0 || lt == 0);
-                    const bool last = (i == run.count - 1 || lt == a.tiles_per_head - 1);
-                    if (first) {
-                        ++seg1;
-                        if (!mbar_wait(bar(WFULL + (seg1 & 1)), (seg1 >> 1) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaLoad); ok = false; return; }
-                    }
-                    const int s = (int)(i % kKStages), ub = (int)(i & 1);
-                    if (!mbar_wait(bar(FULL + s), (i / kKStages) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaLoad); ok = false; return; }
-                    if (i >= 2 && !mbar_wait(bar(UEMPTY + ub), ((i >> 1) - 1) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaU); ok = false; return; }
-                    tcgen05_fence_after();
-                    issue_logits_mma(tmem_u + ub * kM, sbase + s * KSideSmem::kStage, sbase + KSideSmem::kW + (seg1 & 1) * kWBytes);
-                    mma_commit(bar(UFULL + ub));
-                    if (last) mma_commit(bar(WFREE + (seg1 & 1)));
-                };
-                auto do_mma2 = [&](long long j) {
-                    const long long t = run.first + j;
-                    const int lt = (int)(t % a.tiles_per_head);
-                    const bool first = (j == 0 || lt == 0);
-                    const bool last = (j == run.count - 1 || lt == a.tiles_per_head - 1);
-                    const int s = (int)(j % kKStages);
-                    if (!mbar_wait(bar(PHIFULL + s), (j / kKStages) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaPhi); ok = false; return; }
-                    if (first) {
-                        ++seg2;
-                        if (seg2 >= 1 && !mbar_wait(bar(ACCFREE), (seg2 - 1) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaAcc); ok = false; return; }
-                    }
-                    tcgen05_fence_after();
-                    const uint32_t phi = sbase + s * KSideSmem::kStage, vt = phi + kTileBytes;
+                mbar_arrive_expect_tx(bar(FULL + r.s), 2 * kTileBytes);
+                const uint32_t kdst = sbase + r.s * KSideSmem::kStage, vdst = kdst + kTileBytes;
+                tma_load_3d(kdst, &tmK, bar(FULL + r.s), 0, w.lt * kTile, w.g);
+                tma_load_3d(kdst + kHalfTileBytes, &tmK, bar(FULL + r.s), 64, w.lt * kTile, w.g);
+                tma_load_3d(vdst, &tmV, bar(FULL + r.s), 0, w.lt * kTile, w.g);
+                tma_load_3d(vdst + kHalfTileBytes, &tmV, bar(FULL + r.s), 64, w.lt * kTile, w.g);
+            }
+            issued = w.i + 1;
+        }
+        if (issued < w.count) {
+            // unwinding after a time-out: let the copies already in flight land before the CTA exits
+            for (int i = (issued > kKStages ? issued - kKStages : 0); i < issued; ++i)
+                mbar_wait(bar(FULL + i % kKStages), (uint32_t)(i / kKStages) & 1u, kWaitLimitNs);
+        }
+    } else if (warp == 9) {
+        // ---------------- logits MMA issuer: U = K W_k ----------------
+        Ring<kKStages> r;
+        Ring<2> ur;
+        for (; !w.done(); w.next(), r.next(), ur.next()) {
+            const int wb = w.seg & 1;
+            if (w.first() && !warp_wait(bar(WFULL + wb), (uint32_t)(w.seg >> 1) & 1u, err, kErrMmaLoad)) break;
+            if (!warp_wait(bar(FULL + r.s), r.ph, err, kErrMmaLoad)) break;
+            LA_TRACE(1, w.i, 0);
+            if (w.i >= 2 && !warp_wait(bar(UEMPTY + ur.s), ur.ph ^ 1u, err, kErrMmaU)) break;
+            tcgen05_fence_after();
+            if (elect_one()) {
+                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * KSideSmem::kStage, sbase + KSideSmem::kW + wb * kWBytes);
+                mma_commit(bar(UFULL + ur.s));
+                if (w.last()) mma_commit(bar(WFREE + wb));
+            }
+            __syncwarp();
+            LA_TRACE(1, w.i, 1);
+        }
+    } else if (warp == 10) {
+        // ---------------- accumulation MMA issuer: S += phi^T V, z += phi^T 1 ----------------
+        constexpr uint32_t idesc_s = make_idesc_bf16(kD, kD, 1, 1);   // A = phi^T (MN-major), B = V (MN-major)
+        constexpr uint32_t idesc_z = make_idesc_bf16(kD, 16, 1, 0);   // B = ones (K-major, no swizzle)
+        const uint64_t ones_desc = make_desc_noswizzle(sbase + KSideSmem::kOnes, 128, 256);
+        const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
+        Ring<kKStages> r;
+        for (; !w.done(); w.next(), r.next()) {
+            if (!warp_wait(bar(PHIFULL + r.s), r.ph, err, kErrMmaPhi)) break;
+            LA_TRACE(1, w.i, 2);
+            const bool first = w.first();
+            if (first && w.seg >= 1 && !warp_wait(bar(ACCFREE), (uint32_t)(w.seg - 1) & 1u, err, kErrMmaAcc)) break;
+            tcgen05_fence_after();
+            if (elect_one()) {
+                const uint32_t phi = sbase + r.s * KSideSmem::kStage, vt = phi + kTileBytes;
 #pragma unroll
-                    for (int k = 0; k < kTile / 16; ++k) {
-                        const uint64_t da = make_desc_sw128(phi + k * 2048, kHalfTileBytes, 1024);
-                        const uint64_t db = make_desc_sw128(vt + k * 2048, kHalfTileBytes, 1024);
-                        const uint32_t acc = (first && k == 0) ? 0u : 1u;
-                        mma_bf16_ss(tmem_s, da, db, idesc_s, acc);
-                        mma_bf16_ss(tmem_z, da, ones_desc, idesc_z, acc);
-                    }
-                    mma_commit(bar(EMPTY + s));
-                    if (last) mma_commit(bar(ACCFULL));
-                };
-                for (long long i = 0; i < run.count && ok; ++i) {
-                    do_mma1(i);
-                    if (ok && i >= 1) do_mma2(i - 1);
+                for (int k = 0; k < kTile / 16; ++k) {
+                    const uint64_t da = desc_at(mnmajor, phi + k * 2048);
+                    const uint64_t db = desc_at(mnmajor, vt + k * 2048);
+                    const uint32_t acc = (first && k == 0) ? 0u : 1u;
+                    mma_bf16_ss(tmem_s, da, db, idesc_s, acc);
+                    mma_bf16_ss(tmem_z, da, ones_desc, idesc_z, acc);
                 }
-                if (ok) do_mma2(run.count - 1);
+                mma_commit(bar(EMPTY + r.s));
+                if (w.last()) mma_commit(bar(ACCFULL));
             }
-        } else {
-            // ---------------- feature map + drain (warps 0-7) ----------------
-            const int half = warp >> 2;                       // 0: softmax(+U), 1: softmax(-U)
-            const int row = (warp & 3) * 32 + lane;           // token within the tile == TMEM lane
-            const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-            int seg = -1;
-            for (long long i = 0; i < run.count; ++i) {
-                const long long t = run.first + i;
-                const int g = (int)(t / a.tiles_per_head);
-                const int lt = (int)(t % a.tiles_per_head);
-                if (i == 0 || lt == 0) ++seg;
-                const bool last = (i == run.count - 1 || lt == a.tiles_per_head - 1);
-                const int s = (int)(i % kKStages), ub = (int)(i & 1);
-                LA_WAIT(bar(UFULL + ub), (i >> 1) & 1, kErrSoftmaxU);
+            __syncwarp();
+            LA_TRACE(1, w.i, 3);
+        }
+    } else {
+        // ---------------- feature map + drain (warps 0-7) ----------------
+        const int half = warp >> 2;                       // 0: softmax(+U), 1: softmax(-U)
+        const int row = (warp & 3) * 32 + lane;           // token within the tile == TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        Ring<kKStages> r;
+        Ring<2> ur;
+        for (; !w.done(); w.next(), r.next(), ur.next()) {
+            if (!warp_wait(bar(UFULL + ur.s), ur.ph, err, kErrSoftmaxU)) break;
+            if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 0);
+            tcgen05_fence_after();
+            float u[kM];
+            load_logits(tmem_u + lane_base + ur.s * kM, u);
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(UEMPTY + ur.s));
+            if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 1);
+            const float keep = (w.lt * kTile + row < a.n) ? 1.f : 0.f;
+            uint8_t* dst = smem + r.s * KSideSmem::kStage + half * kHalfTileBytes + row * 128;
+            if (half == 0) softmax_half_to_smem<false>(u, keep, dst, row);
+            else softmax_half_to_smem<true>(u, keep, dst, row);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(PHIFULL + r.s));
+            if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 2);
+            if (w.last()) {
+                // drain the accumulators of this segment: thread = feature f, this half's 64 columns of S
+                if (!warp_wait(bar(ACCFULL), (uint32_t)w.seg & 1u, err, kErrDrain)) break;
                 tcgen05_fence_after();
-                float u[kM];
-                load_logits(tmem_u + lane_base + ub * kM, u);
+                float* rec = a.partial + (size_t)(blockIdx.x + w.g) * kE;
+                float* srow = rec + (size_t)row * kD + half * 64;
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld_x32(tmem_s + lane_base + half * 64 + c0, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int q4 = 0; q4 < 8; ++q4)
+                        *reinterpret_cast<uint4*>(srow + c0 + 4 * q4) = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+                }
+                if (half == 0) {
+                    uint32_t zr[2];
+                    tmem_ld_x2(tmem_z + lane_base, zr);
+                    tmem_wait_ld();
+                    rec[kD * kD + row] = __uint_as_float(zr[0]);
+                }
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(UEMPTY + ub));
-                const float keep = (lt * kTile + row < a.n) ? 1.f : 0.f;
-                uint8_t* dst = smem + s * KSideSmem::kStage + half * kHalfTileBytes + row * 128;
-                if (half == 0) softmax_half_to_smem<false>(u, keep, dst, row);
-                else softmax_half_to_smem<true>(u, keep, dst, row);
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(PHIFULL + s));
-                if (last) {
-                    // drain the accumulators of this segment: thread = feature f, this half's 64 columns of S
-                    LA_WAIT(bar(ACCFULL), seg & 1, kErrDrain);
-                    tcgen05_fence_after();
-                    float* rec = a.partial + (size_t)(blockIdx.x + g) * kE;
-                    float* srow = rec + (size_t)row * kD + half * 64;
-#pragma unroll
-                    for (int c0 = 0; c0 < 64; c0 += 32) {
-                        uint32_t r[32];
-                        tmem_ld_x32(tmem_s + lane_base + half * 64 + c0, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4)
-                            *reinterpret_cast<uint4*>(srow + c0 + 4 * q4) = make_uint4(r[4 * q4], r[4 * q4 + 1], r[4 * q4 + 2], r[4 * q4 + 3]);
-                    }
-                    if (half == 0) {
-                        uint32_t zr[2];
-                        tmem_ld_x2(tmem_z + lane_base, zr);
-                        tmem_wait_ld();
-                        rec[kD * kD + row] = __uint_as_float(zr[0]);
-                    }
-                    tcgen05_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(ACCFREE));
-                }
+                if (lane == 0) mbar_arrive(bar(ACCFREE));
             }
         }
     }
@@ -374,8 +424,18 @@ static __global__ void __launch_bounds__(256) combine_tc(const CombineArgs a)
     const long long g = blockIdx.y;
     const long long c0 = tile_owner(g * a.tiles_per_head, a.total_tiles, a.P);
     const long long c1 = tile_owner((g + 1) * a.tiles_per_head - 1, a.total_tiles, a.P);
+    const float* p = a.partial + (size_t)(c0 + g) * kE + e;
+    const int cnt = (int)(c1 - c0) + 1;
     float acc = 0.f;
-    for (long long c = c0; c <= c1; ++c) acc += a.partial[(size_t)(c + g) * kE + e];
+    int c = 0;
+    for (; c + 8 <= cnt; c += 8) {  // loads first (independent), then the adds in CTA order
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = p[(size_t)(c + u) * kE];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc += v[u];
+    }
+    for (; c < cnt; ++c) acc += p[(size_t)c * kE];
     a.state[(size_t)g * kE + e] = acc;
     if (e < kD * kD) {
         a.s_img[(size_t)g * kD * kD + e] = __float2bfloat16_rn(acc);
@@ -408,7 +468,11 @@ struct QSideArgs {
     const __nv_bfloat16* z_img;  // [G][kZBlkBytes / 2]
     uint32_t* err;
     int n, H;
-    long long tiles_per_head, total_tiles;
+    int tiles_per_head;
+    long long total_tiles;
+#ifdef LINATTN_TRACE
+    long long* trace;
+#endif
 };
 
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar)
@@ -427,12 +491,12 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
     const uint32_t sbase = smem_u32(smem);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + QSideSmem::kBars);
     enum { QFULL = 0, QEMPTY = 5, PHIFULL = 10, OFULL = 15, UFULL = 20, UEMPTY = 22, DFULL = 24, DEMPTY = 26, SEGFULL = 28, SEGFREE = 29, NBARS = 30 };
-    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+    const uint32_t bar0 = smem_u32(bars);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[NBARS]);
     uint32_t* err = a.err;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const Run run = cta_run(a.total_tiles);
 
     if (tid == 0) {
         for (int i = 0; i < kQStages; ++i) { mbar_init(bar(QFULL + i), 1); mbar_init(bar(QEMPTY + i), 1); mbar_init(bar(PHIFULL + i), 8); mbar_init(bar(OFULL + i), 8); }
@@ -459,156 +523,148 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
     auto tmem_num = [&](int db) { return tmem + 128 + db * 160; };   // 128 columns: num[token][c]
     auto tmem_den = [&](int db) { return tmem + 256 + db * 160; };   // 16 columns: [hi(z) part, lo(z) part, ...]
 
-    if (run.count > 0) {
-        if (warp == 8) {
-            // ---------------- TMA producer ----------------
-            if (lane == 0) {
-                int seg = -1;
-                long long issued = 0;
-                for (long long i = 0; i < run.count; ++i) {
-                    const long long t = run.first + i;
-                    const int g = (int)(t / a.tiles_per_head);
-                    const int lt = (int)(t % a.tiles_per_head);
-                    if (i == 0 || lt == 0) {
-                        ++seg;
-                        if (seg >= 1) LA_WAIT(bar(SEGFREE), (seg - 1) & 1, kErrSeg);
-                        mbar_arrive_expect_tx(bar(SEGFULL), kWBytes + kTileBytes + kZBlkBytes);
-                        tma_load_3d(sbase + QSideSmem::kW, &tmW, bar(SEGFULL), 0, 0, g % a.H);
-                        tma_load_3d(sbase + QSideSmem::kW + kWBytes / 2, &tmW, bar(SEGFULL), 64, 0, g % a.H);
-                        tma_load_3d(sbase + QSideSmem::kS, &tmS, bar(SEGFULL), 0, 0, g);
-                        tma_load_3d(sbase + QSideSmem::kS + kHalfTileBytes, &tmS, bar(SEGFULL), 64, 0, g);
-                        bulk_load_1d(sbase + QSideSmem::kZ, a.z_img + (size_t)g * (kZBlkBytes / 2), kZBlkBytes, bar(SEGFULL));
-                    }
-                    const int s = (int)(i % kQStages);
-                    if (i >= kQStages) LA_WAIT(bar(QEMPTY + s), ((i / kQStages) - 1) & 1, kErrProducer);
-                    mbar_arrive_expect_tx(bar(QFULL + s), kTileBytes);
-                    tma_load_3d(sbase + s * kTileBytes, &tmQ, bar(QFULL + s), 0, lt * kTile, g);
-                    tma_load_3d(sbase + s * kTileBytes + kHalfTileBytes, &tmQ, bar(QFULL + s), 64, lt * kTile, g);
-                    issued = i + 1;
-                }
-                if (issued < run.count) {
-                    for (long long i = (issued > kQStages ? issued - kQStages : 0); i < issued; ++i)
-                        mbar_wait(bar(QFULL + (int)(i % kQStages)), (i / kQStages) & 1, kWaitLimitNs);
+    TileWalk w;
+    w.init(a.total_tiles, a.tiles_per_head);
+
+    if (warp == 8) {
+        // ---------------- TMA producer ----------------
+        Ring<kQStages> r;
+        int issued = 0;
+        for (; !w.done(); w.next(), r.next()) {
+            if (w.first()) {
+                if (w.seg >= 1 && !warp_wait(bar(SEGFREE), (uint32_t)(w.seg - 1) & 1u, err, kErrSeg)) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar(SEGFULL), kWBytes + kTileBytes + kZBlkBytes);
+                    tma_load_3d(sbase + QSideSmem::kW, &tmW, bar(SEGFULL), 0, 0, w.g % a.H);
+                    tma_load_3d(sbase + QSideSmem::kW + kWBytes / 2, &tmW, bar(SEGFULL), 64, 0, w.g % a.H);
+                    tma_load_3d(sbase + QSideSmem::kS, &tmS, bar(SEGFULL), 0, 0, w.g);
+                    tma_load_3d(sbase + QSideSmem::kS + kHalfTileBytes, &tmS, bar(SEGFULL), 64, 0, w.g);
+                    bulk_load_1d(sbase + QSideSmem::kZ, a.z_img + (size_t)w.g * (kZBlkBytes / 2), kZBlkBytes, bar(SEGFULL));
                 }
             }
-        } else if (warp == 9) {
-            // ---------------- MMA issuer ----------------
+            if (w.i >= kQStages && !warp_wait(bar(QEMPTY + r.s), r.ph ^ 1u, err, kErrProducer)) break;
             if (lane == 0) {
-                constexpr uint32_t idesc_n = make_idesc_bf16(kTile, kD, 0, 1);   // A = phi(q) (K-major), B = S (MN-major)
-                constexpr uint32_t idesc_d = make_idesc_bf16(kTile, 16, 0, 0);   // B = z operand (K-major)
-                int seg = -1;
-                bool ok = true;
-                auto do_mma1 = [&](long long i) {
-                    const long long t = run.first + i;
-                    const int lt = (int)(t % a.tiles_per_head);
-                    if (i == 0 || lt == 0) {
-                        ++seg;
-                        if (!mbar_wait(bar(SEGFULL), seg & 1, kWaitLimitNs)) { atomicOr(err, kErrSeg); ok = false; return; }
-                    }
-                    const int s = (int)(i % kQStages), ub = (int)(i & 1);
-                    if (!mbar_wait(bar(QFULL + s), (i / kQStages) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaLoad); ok = false; return; }
-                    if (i >= 2 && !mbar_wait(bar(UEMPTY + ub), ((i >> 1) - 1) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaU); ok = false; return; }
-                    tcgen05_fence_after();
-                    issue_logits_mma(tmem_u + ub * kM, sbase + s * kTileBytes, sbase + QSideSmem::kW);
-                    mma_commit(bar(UFULL + ub));
-                };
-                auto do_mma2 = [&](long long j) {
-                    const long long t = run.first + j;
-                    const int lt = (int)(t % a.tiles_per_head);
-                    const bool last = (j == run.count - 1 || lt == a.tiles_per_head - 1);
-                    const int s = (int)(j % kQStages), db = (int)(j & 1);
-                    if (!mbar_wait(bar(PHIFULL + s), (j / kQStages) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaPhi); ok = false; return; }
-                    if (j >= 2 && !mbar_wait(bar(DEMPTY + db), ((j >> 1) - 1) & 1, kWaitLimitNs)) { atomicOr(err, kErrMmaAcc); ok = false; return; }
-                    tcgen05_fence_after();
-                    const uint32_t phi = sbase + s * kTileBytes;
+                mbar_arrive_expect_tx(bar(QFULL + r.s), kTileBytes);
+                tma_load_3d(sbase + r.s * kTileBytes, &tmQ, bar(QFULL + r.s), 0, w.lt * kTile, w.g);
+                tma_load_3d(sbase + r.s * kTileBytes + kHalfTileBytes, &tmQ, bar(QFULL + r.s), 64, w.lt * kTile, w.g);
+            }
+            issued = w.i + 1;
+        }
+        if (issued < w.count) {
+            for (int i = (issued > kQStages ? issued - kQStages : 0); i < issued; ++i)
+                mbar_wait(bar(QFULL + i % kQStages), (uint32_t)(i / kQStages) & 1u, kWaitLimitNs);
+        }
+    } else if (warp == 9) {
+        // ---------------- logits MMA issuer: U = Q W_q ----------------
+        Ring<kQStages> r;
+        Ring<2> ur;
+        for (; !w.done(); w.next(), r.next(), ur.next()) {
+            if (w.first() && !warp_wait(bar(SEGFULL), (uint32_t)w.seg & 1u, err, kErrSeg)) break;
+            if (!warp_wait(bar(QFULL + r.s), r.ph, err, kErrMmaLoad)) break;
+            if (w.i >= 2 && !warp_wait(bar(UEMPTY + ur.s), ur.ph ^ 1u, err, kErrMmaU)) break;
+            tcgen05_fence_after();
+            if (elect_one()) {
+                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + QSideSmem::kW);
+                mma_commit(bar(UFULL + ur.s));
+            }
+            __syncwarp();
+        }
+    } else if (warp == 10) {
+        // ---------------- numerator / denominator MMA issuer: num = phi(q) S, den = phi(q) . z ----------------
+        constexpr uint32_t idesc_n = make_idesc_bf16(kTile, kD, 0, 1);   // A = phi(q) (K-major), B = S (MN-major)
+        constexpr uint32_t idesc_d = make_idesc_bf16(kTile, 16, 0, 0);   // B = z operand (K-major)
+        const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
+        const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
+        Ring<kQStages> r;
+        Ring<2> dr;
+        for (; !w.done(); w.next(), r.next(), dr.next()) {
+            if (w.first() && !warp_wait(bar(SEGFULL), (uint32_t)w.seg & 1u, err, kErrSeg)) break;
+            if (!warp_wait(bar(PHIFULL + r.s), r.ph, err, kErrMmaPhi)) break;
+            if (w.i >= 2 && !warp_wait(bar(DEMPTY + dr.s), dr.ph ^ 1u, err, kErrMmaAcc)) break;
+            tcgen05_fence_after();
+            if (elect_one()) {
+                const uint32_t phi = sbase + r.s * kTileBytes;
 #pragma unroll
-                    for (int k = 0; k < kD / 16; ++k) {
-                        const uint64_t da = make_desc_sw128(phi + (k >> 2) * kHalfTileBytes + (k & 3) * 32, 16, 1024);
-                        const uint64_t db_s = make_desc_sw128(sbase + QSideSmem::kS + k * 2048, kHalfTileBytes, 1024);
-                        const uint64_t db_z = make_desc_sw128(sbase + QSideSmem::kZ + (k >> 2) * 2048 + (k & 3) * 32, 16, 1024);
-                        mma_bf16_ss(tmem_num(db), da, db_s, idesc_n, k > 0);
-                        mma_bf16_ss(tmem_den(db), da, db_z, idesc_d, k > 0);
-                    }
-                    mma_commit(bar(DFULL + db));
-                    if (last) mma_commit(bar(SEGFREE));
-                };
-                for (long long i = 0; i < run.count && ok; ++i) {
-                    const int lt = (int)((run.first + i) % a.tiles_per_head);
-                    const bool boundary = (i >= 1 && lt == 0);
-                    if (boundary) do_mma2(i - 1);      // finish the previous head before its S, z, W are replaced
-                    if (ok) do_mma1(i);
-                    if (ok && i >= 1 && !boundary) do_mma2(i - 1);
+                for (int k = 0; k < kD / 16; ++k) {
+                    const uint64_t da = desc_at(kmajor, phi + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
+                    const uint64_t db_s = desc_at(mnmajor, sbase + QSideSmem::kS + k * 2048);
+                    const uint64_t db_z = desc_at(kmajor, sbase + QSideSmem::kZ + (k >> 2) * 2048 + (k & 3) * 32);
+                    mma_bf16_ss(tmem_num(dr.s), da, db_s, idesc_n, k > 0);
+                    mma_bf16_ss(tmem_den(dr.s), da, db_z, idesc_d, k > 0);
                 }
-                if (ok) do_mma2(run.count - 1);
+                mma_commit(bar(DFULL + dr.s));
+                if (w.last()) mma_commit(bar(SEGFREE));   // this head's S, z and W may now be replaced
             }
-        } else if (warp == 10) {
-            // ---------------- TMA stores of finished output tiles ----------------
+            __syncwarp();
+        }
+    } else if (warp == 11) {
+        // ---------------- TMA stores of finished output tiles ----------------
+        Ring<kQStages> r;
+        for (; !w.done(); w.next(), r.next()) {
+            if (!warp_wait(bar(OFULL + r.s), r.ph, err, kErrStore)) break;
             if (lane == 0) {
-                for (long long j = 0; j < run.count; ++j) {
-                    const long long t = run.first + j;
-                    const int g = (int)(t / a.tiles_per_head);
-                    const int lt = (int)(t % a.tiles_per_head);
-                    const int s = (int)(j % kQStages);
-                    LA_WAIT(bar(OFULL + s), (j / kQStages) & 1, kErrStore);
-                    tma_store_3d(&tmO, sbase + s * kTileBytes, 0, lt * kTile, g);
-                    tma_store_3d(&tmO, sbase + s * kTileBytes + kHalfTileBytes, 64, lt * kTile, g);
-                    bulk_commit_group();
-                    bulk_wait_group_read<0>();   // the slot has been read out: hand it back to the producer
-                    mbar_arrive(bar(QEMPTY + s));
-                }
-                bulk_wait_group<0>();
+                tma_store_3d(&tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g);
+                tma_store_3d(&tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g);
+                bulk_commit_group();
+                bulk_wait_group_read<0>();   // the slot has been read out: hand it back to the producer
+                mbar_arrive(bar(QEMPTY + r.s));
             }
-        } else {
-            // ---------------- feature map + epilogue (warps 0-7) ----------------
-            const int half = warp >> 2;
-            const int row = (warp & 3) * 32 + lane;
-            const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-            for (long long i = 0; i <= run.count; ++i) {
-                if (i < run.count) {
-                    const int s = (int)(i % kQStages), ub = (int)(i & 1);
-                    LA_WAIT(bar(UFULL + ub), (i >> 1) & 1, kErrSoftmaxU);
-                    tcgen05_fence_after();
-                    float u[kM];
-                    load_logits(tmem_u + lane_base + ub * kM, u);
-                    tcgen05_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(UEMPTY + ub));
-                    uint8_t* dst = smem + s * kTileBytes + half * kHalfTileBytes + row * 128;
-                    if (half == 0) softmax_half_to_smem<false>(u, 1.f, dst, row);
-                    else softmax_half_to_smem<true>(u, 1.f, dst, row);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(PHIFULL + s));
-                }
-                if (i >= 1) {
-                    const long long j = i - 1;
-                    const int s = (int)(j % kQStages), db = (int)(j & 1);
-                    LA_WAIT(bar(DFULL + db), (j >> 1) & 1, kErrEpilogue);
-                    tcgen05_fence_after();
-                    uint32_t r[64], dr[2];
-                    tmem_ld_x32(tmem_num(db) + lane_base + half * 64, r);
-                    tmem_ld_x32(tmem_num(db) + lane_base + half * 64 + 32, r + 32);
-                    tmem_ld_x2(tmem_den(db) + lane_base, dr);
-                    tmem_wait_ld();
-                    tcgen05_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(DEMPTY + db));
-                    const float inv = __fdividef(1.f, __uint_as_float(dr[0]) + __uint_as_float(dr[1]));
-                    uint8_t* dst = smem + s * kTileBytes + half * kHalfTileBytes + row * 128;
-                    const int sw = row & 7;
+            __syncwarp();
+        }
+        if (lane == 0) bulk_wait_group<0>();
+    } else {
+        // ---------------- feature map + epilogue (warps 0-7) ----------------
+        const int half = warp >> 2;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        Ring<kQStages> r, er;   // feature-map ring position, epilogue ring position (one tile behind)
+        Ring<2> ur, dr;
+        for (int i = 0; i <= w.count; ++i) {
+            if (i < w.count) {
+                if (!warp_wait(bar(UFULL + ur.s), ur.ph, err, kErrSoftmaxU)) break;
+                tcgen05_fence_after();
+                float u[kM];
+                load_logits(tmem_u + lane_base + ur.s * kM, u);
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(UEMPTY + ur.s));
+                uint8_t* dst = smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                if (half == 0) softmax_half_to_smem<false>(u, 1.f, dst, row);
+                else softmax_half_to_smem<true>(u, 1.f, dst, row);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(PHIFULL + r.s));
+                r.next();
+                ur.next();
+            }
+            if (i >= 1) {
+                if (!warp_wait(bar(DFULL + dr.s), dr.ph, err, kErrEpilogue)) break;
+                tcgen05_fence_after();
+                uint32_t v[64], dv[2];
+                tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64, v);
+                tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64 + 32, v + 32);
+                tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
+                tmem_wait_ld();
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(DEMPTY + dr.s));
+                const float inv = __fdividef(1.f, __uint_as_float(dv[0]) + __uint_as_float(dv[1]));
+                uint8_t* dst = smem + er.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                const int sw = row & 7;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        uint4 v;
-                        v.x = pack_bf16(__uint_as_float(r[8 * c + 0]) * inv, __uint_as_float(r[8 * c + 1]) * inv);
-                        v.y = pack_bf16(__uint_as_float(r[8 * c + 2]) * inv, __uint_as_float(r[8 * c + 3]) * inv);
-                        v.z = pack_bf16(__uint_as_float(r[8 * c + 4]) * inv, __uint_as_float(r[8 * c + 5]) * inv);
-                        v.w = pack_bf16(__uint_as_float(r[8 * c + 6]) * inv, __uint_as_float(r[8 * c + 7]) * inv);
-                        *reinterpret_cast<uint4*>(dst + ((c ^ sw) << 4)) = v;
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(OFULL + s));
+                for (int c = 0; c < 8; ++c) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(v[8 * c + 0]) * inv, __uint_as_float(v[8 * c + 1]) * inv);
+                    o.y = pack_bf16(__uint_as_float(v[8 * c + 2]) * inv, __uint_as_float(v[8 * c + 3]) * inv);
+                    o.z = pack_bf16(__uint_as_float(v[8 * c + 4]) * inv, __uint_as_float(v[8 * c + 5]) * inv);
+                    o.w = pack_bf16(__uint_as_float(v[8 * c + 6]) * inv, __uint_as_float(v[8 * c + 7]) * inv);
+                    *reinterpret_cast<uint4*>(dst + ((c ^ sw) << 4)) = o;
                 }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(OFULL + er.s));
+                er.next();
+                dr.next();
             }
         }
     }
@@ -616,8 +672,6 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
     __syncthreads();
     if (warp == 9) tmem_dealloc(tmem, 512);
 }
-
-#undef LA_WAIT
 
 // W [H][128 d][64 j] (any supported type) -> W^T bf16 [H][64 j][128 d]; per_head == 0 replicates one matrix.
 template <typename T>
