@@ -51,6 +51,8 @@ struct linattn_ctx {
     __nv_bfloat16* s_img = nullptr;  // [max_B*H][128*128] bf16 image of S for the query-side TMA
     __nv_bfloat16* z_img = nullptr;  // [max_B*H][2048] bf16 operand image of z (hi, lo)
     int num_sms = 0;
+    bool coop_ok = false;            // device supports cooperative launches
+    uint32_t* sync_words = nullptr;  // grid-barrier counter and generation of the fused kernel
     // workspace
     float* partial = nullptr;   // [partial_slots][d*d + d]
     long long partial_slots = 0;
@@ -62,6 +64,7 @@ struct linattn_ctx {
     // options
     int opt_splits = 0;
     int opt_path = 0;
+    int opt_fuse = 1;
     // per-kernel timing (LINATTN_OPT_PROFILE)
     static constexpr int kMaxKernels = 4;
     bool profile = false;
@@ -216,22 +219,41 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     }
     static bool attr_done = false;
     if (!attr_done) {
-        LA_CUDA(c, cudaFuncSetAttribute(kside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KSideSmem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(qside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QSideSmem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(kside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(qside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(linattn_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
         attr_done = true;
     }
     const double side_bytes = 2.0 * (double)G * n * kD * 2;
+    Args a{};
+    a.partial = c->partial;
+    a.state = c->state;
+    a.s_img = c->s_img;
+    a.z_img = c->z_img;
+    a.err = c->err_word;
+    a.sync = c->sync_words;
+    a.n = n;
+    a.H = c->H;
+    a.G = (int)G;
+    a.tiles_per_head = (int)Tn;
+    a.total_tiles = T;
     prof_begin(c, st);
-    KSideArgs ka{c->partial, c->err_word, n, c->H, (int)Tn, T};
-    kside_tc<<<(unsigned)Pk, kKThreads, KSideSmem::kTotal, st>>>(tmK, tmV, tmWk, ka);
+    if (c->opt_fuse && c->coop_ok && Pk == Pq) {
+        // one cooperative launch: key side, grid barrier, combine, grid barrier, query side
+        void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &a};
+        LA_CUDA(c, cudaLaunchCooperativeKernel((const void*)linattn_fused_tc, dim3((unsigned)Pq), dim3(kThreads), params,
+                                               Smem::kTotal, st));
+        prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
+        c->last_launches = 1;
+        return LINATTN_OK;
+    }
+    kside_tc<<<(unsigned)Pk, kThreads, Smem::kTotal, st>>>(tmK, tmV, tmWk, a);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_tc", side_bytes);
-    CombineArgs ca{c->partial, c->state, c->s_img, c->z_img, Tn, T, Pk};
-    combine_tc<<<dim3((kE + 255) / 256, (unsigned)G), 256, 0, st>>>(ca);
+    combine_tc<<<dim3((kE / 4 + 255) / 256, (unsigned)G), 256, 0, st>>>(a, Pk);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_tc", 0.0);
-    QSideArgs qa{c->z_img, c->err_word, n, c->H, (int)Tn, T};
-    qside_tc<<<(unsigned)Pq, kQThreads, QSideSmem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, qa);
+    qside_tc<<<(unsigned)Pq, kThreads, Smem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, a);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);
     c->last_launches = 3;
@@ -318,6 +340,13 @@ linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, l
         if (e == cudaSuccess) e = cudaMemset(c->z_img, 0, (size_t)G * linattn::tc::kZBlkBytes);
     }
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) {
+        int coop = 0;
+        e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device);
+        c->coop_ok = (coop != 0);
+    }
+    if (e == cudaSuccess) e = cudaMalloc(&c->sync_words, 2 * sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->sync_words, 0, 2 * sizeof(uint32_t));
     if (e == cudaSuccess) e = cudaMalloc(&c->err_word, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->err_word, 0, sizeof(unsigned int));
     if (e != cudaSuccess) {
@@ -339,6 +368,7 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->partial);
     cudaFree(c->state);
     cudaFree(c->err_word);
+    cudaFree(c->sync_words);
     cudaFree(c->Wqt);
     cudaFree(c->Wkt);
     cudaFree(c->s_img);
@@ -465,6 +495,10 @@ linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long 
             if (value < 0 || value > 2) return LINATTN_ERR_INVALID_ARG;
             c->opt_path = (int)value;
             return LINATTN_OK;
+        case LINATTN_OPT_FUSE:
+            if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
+            c->opt_fuse = (int)value;
+            return LINATTN_OK;
         case LINATTN_OPT_PROFILE: {
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
             DeviceGuard guard(c->device);
@@ -498,6 +532,7 @@ linattn_status linattn_check(linattn_ctx* c, void* stream)
     LA_CUDA(c, cudaStreamSynchronize(st));
     if (w != 0) {
         LA_CUDA(c, cudaMemsetAsync(c->err_word, 0, sizeof(w), st));
+        LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, 2 * sizeof(uint32_t), st));  // an aborted grid barrier leaves them inconsistent
         snprintf(c->err_text, sizeof(c->err_text), "device-side wait gave up (code 0x%x)", w);
         return LINATTN_ERR_TIMEOUT;
     }

@@ -1,5 +1,7 @@
 // Tensor-core kernels (tcgen05 + TMEM + TMA) for linear attention with the Hedgehog feature map,
-// bf16 storage, head dimension 128.  Three launches per forward:
+// bf16 storage, head dimension 128.  The forward has three steps, run either as ONE persistent
+// cooperative kernel (linattn_fused_tc: key side, grid barrier, combine, grid barrier, query side) or as
+// three launches:
 //
 //   kside_tc   : persistent CTAs stream 128-token tiles of K and V.  Per tile
 //                  U = K W_k          (tcgen05.mma, 128x64x128, fp32 in TMEM)                 Eq. 6
@@ -20,7 +22,8 @@
 // 64-127, warp 8 TMA producer, warp 9 issues the logits MMAs, warp 10 issues the accumulation MMAs, and
 // (query side only) warp 11 issues the TMA stores.  Role loops are warp-uniform; single-thread work
 // (TMA and MMA issue) is predicated inside them.
-// Every wait is bounded: on time-out the kernel records a code in *err and unwinds.
+// Every wait is bounded: on time-out the kernel records a code in *err, raises the CTA's abort word so
+// that the other roles stop waiting too, and unwinds.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -37,8 +40,6 @@ using namespace ptx;
 constexpr int kD = 128;             // head dimension
 constexpr int kM = 64;              // features per softmax half
 constexpr int kTile = 128;          // tokens per tile
-constexpr int kKThreads = 352;      // key side: 11 warps
-constexpr int kQThreads = 384;      // query side: 12 warps
 constexpr int kE = kD * kD + kD;    // floats per (S, z) record
 constexpr uint32_t kTileBytes = kTile * kD * 2;       // 32 KB: one [128 x 128] bf16 tile
 constexpr uint32_t kHalfTileBytes = kTileBytes / 2;   // one 64-column block of a tile
@@ -50,7 +51,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 // error codes OR-ed into *err (which wait gave up)
 enum : uint32_t {
     kErrProducer = 1u, kErrMmaLoad = 2u, kErrMmaU = 4u, kErrMmaPhi = 8u, kErrMmaAcc = 16u,
-    kErrSoftmaxU = 32u, kErrDrain = 64u, kErrEpilogue = 128u, kErrSeg = 256u, kErrStore = 512u
+    kErrSoftmaxU = 32u, kErrDrain = 64u, kErrEpilogue = 128u, kErrSeg = 256u, kErrStore = 512u, kErrGrid = 1024u
 };
 
 // CTA that owns tile t when T tiles are split over P CTAs (CTA c owns [c*T/P, (c+1)*T/P)).
@@ -101,12 +102,21 @@ template <int N> struct Ring {
     }
 };
 
+// What every role needs to wait on a barrier and to report a failed wait.
+struct WaitCtx {
+    uint32_t* err;        // global error word
+    uint32_t abort_smem;  // shared-memory address of the CTA's abort word
+};
+
 // All lanes wait (bounded); the verdict is made warp-uniform so that role loops never diverge.
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, uint32_t* err, uint32_t code)
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc, uint32_t code)
 {
-    const bool ok = mbar_wait(bar, parity, kWaitLimitNs);
+    const bool ok = mbar_wait_abortable(bar, parity, kWaitLimitNs, wc.abort_smem);
     const bool all = __all_sync(0xffffffffu, ok);
-    if (!all && (threadIdx.x & 31) == 0) atomicOr(err, code);
+    if (!all && (threadIdx.x & 31) == 0) {
+        atomicOr(wc.err, code);
+        asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(wc.abort_smem), "r"(1u) : "memory");
+    }
     return all;
 }
 
@@ -174,8 +184,14 @@ constexpr int kTraceTiles = 64;
         if (a.trace && (tile) < kTraceTiles && (threadIdx.x & 31) == 0)                                  \
             a.trace[(((size_t)blockIdx.x * 4 + (role)) * kTraceTiles + (tile)) * 4 + (ev)] = clock64(); \
     } while (0)
+#define LA_TRACE_NS(role, tile, ev)                                                                             \
+    do {                                                                                                        \
+        if (a.trace && threadIdx.x == 0)                                                                        \
+            a.trace[(((size_t)blockIdx.x * 4 + (role)) * kTraceTiles + (tile)) * 4 + (ev)] = (long long)globaltimer_ns(); \
+    } while (0)
 #else
 #define LA_TRACE(role, tile, ev) do { } while (0)
+#define LA_TRACE_NS(role, tile, ev) do { } while (0)
 #endif
 
 // Shared-memory descriptor with the address field replaced: descriptors of one operand family differ
@@ -199,22 +215,54 @@ __device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_sme
 }
 
 // ======================================================================================================
-// Key side
+// Shared-memory layout, barriers and per-CTA state common to all three kernels
 // ======================================================================================================
 
-constexpr int kKStages = 3;
-struct KSideSmem {
-    static constexpr uint32_t kStage = 2 * kTileBytes;                    // K (later phi) + V
-    static constexpr uint32_t kW = kKStages * kStage;                     // 2 x W^T
-    static constexpr uint32_t kOnes = kW + 2 * kWBytes;                   // 1 KB of bf16 ones
-    static constexpr uint32_t kBars = kOnes + 1024;
-    static constexpr uint32_t kTotal = kBars + 256 + 1024;                // + barriers + alignment slack
+constexpr int kKStages = 3;   // key side: stages of (K tile, V tile)
+constexpr int kQStages = 5;   // query side: stages of one Q tile (reused for phi(q) and then the output tile)
+constexpr int kThreads = 384; // 12 warps
+
+struct Smem {
+    // key side
+    static constexpr uint32_t kKStage = 2 * kTileBytes;                   // K (later phi) + V
+    static constexpr uint32_t kKW = kKStages * kKStage;                   // 2 x W_k^T
+    static constexpr uint32_t kOnes = kKW + 2 * kWBytes;                  // 1 KB of bf16 ones
+    static constexpr uint32_t kKEnd = kOnes + 1024;
+    // query side (overlays the key-side region)
+    static constexpr uint32_t kQS = kQStages * kTileBytes;                // S image (32 KB)
+    static constexpr uint32_t kQW = kQS + kTileBytes;                     // W_q^T (16 KB)
+    static constexpr uint32_t kQZ = kQW + kWBytes;                        // z operand (4 KB)
+    static constexpr uint32_t kQEnd = kQZ + kZBlkBytes;
+    static constexpr uint32_t kBars = kKEnd > kQEnd ? kKEnd : kQEnd;      // mbarriers, TMEM slot, abort word
+    static constexpr uint32_t kTotal = kBars + 512 + 1024;                // + alignment slack
 };
 
-struct KSideArgs {
-    float* partial;   // [slots][kE]
-    uint32_t* err;
-    int n, H;
+// mbarrier indices
+enum : int {
+    // key side
+    K_FULL = 0, K_EMPTY = 3, K_UFULL = 6, K_UEMPTY = 8, K_PHIFULL = 10, K_WFULL = 13, K_WFREE = 15, K_ACCFULL = 17, K_ACCFREE = 18,
+    // query side
+    Q_FULL = 19, Q_EMPTY = 24, Q_PHIFULL = 29, Q_OFULL = 34, Q_UFULL = 39, Q_UEMPTY = 41, Q_DFULL = 43, Q_DEMPTY = 45,
+    Q_SEGFULL = 47, Q_SEGFREE = 48, Q_SREADY = 49, Q_WFULL = 50,
+    NBARS = 51
+};
+
+struct Cta {
+    uint8_t* smem;
+    uint32_t sbase, bar0, tmem;
+    int warp, lane;
+    WaitCtx wc;
+    __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * (uint32_t)i; }
+};
+
+struct Args {
+    float* partial;              // [slots][kE] partial (S, z) records, slot = cta + g
+    float* state;                // [G][kE] combined S, z (fp32)
+    __nv_bfloat16* s_img;        // [G][128][128] bf16 image of S
+    __nv_bfloat16* z_img;        // [G][kZBlkBytes / 2] bf16 operand image of z (hi, lo)
+    uint32_t* err;               // error word
+    uint32_t* sync;              // [0] grid-barrier arrival counter, [1] generation (fused kernel only)
+    int n, H, G;
     int tiles_per_head;
     long long total_tiles;
 #ifdef LINATTN_TRACE
@@ -222,82 +270,110 @@ struct KSideArgs {
 #endif
 };
 
-__global__ void __launch_bounds__(kKThreads, 1)
-kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-         const __grid_constant__ CUtensorMap tmW, const KSideArgs a)
+// Common prologue: barrier init, TMEM allocation (512 columns, warp 9), abort word.
+__device__ __forceinline__ Cta cta_setup(uint8_t* smem_raw, const Args& a, bool init_k, bool init_q)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const uint32_t sbase = smem_u32(smem);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + KSideSmem::kBars);
-    enum { FULL = 0, EMPTY = 3, UFULL = 6, UEMPTY = 8, PHIFULL = 10, WFULL = 13, WFREE = 15, ACCFULL = 17, ACCFREE = 18, NBARS = 19 };
-    const uint32_t bar0 = smem_u32(bars);
-    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    Cta c;
+    c.smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    c.sbase = smem_u32(c.smem);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(c.smem + Smem::kBars);
+    c.bar0 = smem_u32(bars);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[NBARS]);
-    uint32_t* err = a.err;
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    if (tid == 0) {
-        for (int i = 0; i < kKStages; ++i) { mbar_init(bar(FULL + i), 1); mbar_init(bar(EMPTY + i), 1); mbar_init(bar(PHIFULL + i), 8); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(UFULL + i), 1); mbar_init(bar(UEMPTY + i), 8); mbar_init(bar(WFULL + i), 1); mbar_init(bar(WFREE + i), 1); }
-        mbar_init(bar(ACCFULL), 1);
-        mbar_init(bar(ACCFREE), 8);
+    uint32_t* abort_word = tmem_slot + 1;
+    c.warp = threadIdx.x >> 5;
+    c.lane = threadIdx.x & 31;
+    c.wc.err = a.err;
+    c.wc.abort_smem = smem_u32(abort_word);
+    if (threadIdx.x == 0) {
+        *abort_word = 0u;
+        if (init_k) {
+            for (int i = 0; i < kKStages; ++i) { mbar_init(c.bar(K_FULL + i), 1); mbar_init(c.bar(K_EMPTY + i), 1); mbar_init(c.bar(K_PHIFULL + i), 8); }
+            for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_UFULL + i), 1); mbar_init(c.bar(K_UEMPTY + i), 8); mbar_init(c.bar(K_WFULL + i), 1); mbar_init(c.bar(K_WFREE + i), 1); }
+            mbar_init(c.bar(K_ACCFULL), 1);
+            mbar_init(c.bar(K_ACCFREE), 8);
+        }
+        if (init_q) {
+            for (int i = 0; i < kQStages; ++i) { mbar_init(c.bar(Q_FULL + i), 1); mbar_init(c.bar(Q_EMPTY + i), 1); mbar_init(c.bar(Q_PHIFULL + i), 8); mbar_init(c.bar(Q_OFULL + i), 8); }
+            for (int i = 0; i < 2; ++i) { mbar_init(c.bar(Q_UFULL + i), 1); mbar_init(c.bar(Q_UEMPTY + i), 8); mbar_init(c.bar(Q_DFULL + i), 1); mbar_init(c.bar(Q_DEMPTY + i), 8); }
+            mbar_init(c.bar(Q_SEGFULL), 1);
+            mbar_init(c.bar(Q_SEGFREE), 1);
+            mbar_init(c.bar(Q_SREADY), 8);
+            mbar_init(c.bar(Q_WFULL), 1);
+        }
         fence_mbar_init();
     }
-    if (warp == 9) {
+    if (c.warp == 9) {
         tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
     }
-    if (warp == 8 && lane == 0) {
-        tma_prefetch_desc(&tmK);
-        tma_prefetch_desc(&tmV);
-        tma_prefetch_desc(&tmW);
-    }
-    for (int i = tid; i < 512; i += kKThreads) reinterpret_cast<__nv_bfloat16*>(smem + KSideSmem::kOnes)[i] = __float2bfloat16(1.0f);
+    if (init_k)
+        for (int i = threadIdx.x; i < 512; i += blockDim.x) reinterpret_cast<__nv_bfloat16*>(c.smem + Smem::kOnes)[i] = __float2bfloat16(1.0f);
     fence_proxy_async_smem();
     tcgen05_fence_before();
     __syncthreads();
     tcgen05_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    const uint32_t tmem_u = tmem;            // 2 x 64 columns of logits
-    const uint32_t tmem_s = tmem + 128;      // 128 columns: S[f][c], lane = f
-    const uint32_t tmem_z = tmem + 256;      // 16 columns: z[f] (all 16 equal)
+    c.tmem = *tmem_slot;
+    return c;
+}
 
+__device__ __forceinline__ void cta_teardown(const Cta& c)
+{
+    tcgen05_fence_before();
+    __syncthreads();
+    if (c.warp == 9) tmem_dealloc(c.tmem, 512);
+}
+
+// ======================================================================================================
+// Key side: partial S = sum phi(k)^T v and z = sum phi(k) over this CTA's tiles (Eq. 5 brackets, Eq. 6)
+// ======================================================================================================
+
+__device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const CUtensorMap* tmK, const CUtensorMap* tmV,
+                                            const CUtensorMap* tmW)
+{
+    const uint32_t tmem_u = c.tmem;            // 2 x 64 columns of logits
+    const uint32_t tmem_s = c.tmem + 128;      // 128 columns: S[f][c], lane = f
+    const uint32_t tmem_z = c.tmem + 256;      // 16 columns: z[f] (all 16 equal)
+    const int warp = c.warp, lane = c.lane;
+    const uint32_t sbase = c.sbase;
     TileWalk w;
     w.init(a.total_tiles, a.tiles_per_head);
 
     if (warp == 8) {
         // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            tma_prefetch_desc(tmK);
+            tma_prefetch_desc(tmV);
+            tma_prefetch_desc(tmW);
+        }
         Ring<kKStages> r;
         int issued = 0;
         for (; !w.done(); w.next(), r.next()) {
             if (w.first()) {
                 const int wb = w.seg & 1;
-                if (w.seg >= 2 && !warp_wait(bar(WFREE + wb), ((w.seg >> 1) - 1) & 1, err, kErrProducer)) break;
+                if (w.seg >= 2 && !warp_wait(c.bar(K_WFREE + wb), ((w.seg >> 1) - 1) & 1, c.wc, kErrProducer)) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(bar(WFULL + wb), kWBytes);
-                    const uint32_t wdst = sbase + KSideSmem::kW + wb * kWBytes;
-                    tma_load_3d(wdst, &tmW, bar(WFULL + wb), 0, 0, w.g % a.H);
-                    tma_load_3d(wdst + kWBytes / 2, &tmW, bar(WFULL + wb), 64, 0, w.g % a.H);
+                    mbar_arrive_expect_tx(c.bar(K_WFULL + wb), kWBytes);
+                    const uint32_t wdst = sbase + Smem::kKW + wb * kWBytes;
+                    tma_load_3d(wdst, tmW, c.bar(K_WFULL + wb), 0, 0, w.g % a.H);
+                    tma_load_3d(wdst + kWBytes / 2, tmW, c.bar(K_WFULL + wb), 64, 0, w.g % a.H);
                 }
             }
-            if (w.i >= kKStages && !warp_wait(bar(EMPTY + r.s), r.ph ^ 1u, err, kErrProducer)) break;
+            if (w.i >= kKStages && !warp_wait(c.bar(K_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) break;
             LA_TRACE(0, w.i, 0);
             if (lane == 0) {
-                mbar_arrive_expect_tx(bar(FULL + r.s), 2 * kTileBytes);
-                const uint32_t kdst = sbase + r.s * KSideSmem::kStage, vdst = kdst + kTileBytes;
-                tma_load_3d(kdst, &tmK, bar(FULL + r.s), 0, w.lt * kTile, w.g);
-                tma_load_3d(kdst + kHalfTileBytes, &tmK, bar(FULL + r.s), 64, w.lt * kTile, w.g);
-                tma_load_3d(vdst, &tmV, bar(FULL + r.s), 0, w.lt * kTile, w.g);
-                tma_load_3d(vdst + kHalfTileBytes, &tmV, bar(FULL + r.s), 64, w.lt * kTile, w.g);
+                mbar_arrive_expect_tx(c.bar(K_FULL + r.s), 2 * kTileBytes);
+                const uint32_t kdst = sbase + r.s * Smem::kKStage, vdst = kdst + kTileBytes;
+                tma_load_3d(kdst, tmK, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g);
+                tma_load_3d(kdst + kHalfTileBytes, tmK, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g);
+                tma_load_3d(vdst, tmV, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g);
+                tma_load_3d(vdst + kHalfTileBytes, tmV, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g);
             }
             issued = w.i + 1;
         }
         if (issued < w.count) {
-            // unwinding after a time-out: let the copies already in flight land before the CTA exits
+            // unwinding after a time-out: let the copies already in flight land before the CTA moves on
             for (int i = (issued > kKStages ? issued - kKStages : 0); i < issued; ++i)
-                mbar_wait(bar(FULL + i % kKStages), (uint32_t)(i / kKStages) & 1u, kWaitLimitNs);
+                mbar_wait(c.bar(K_FULL + i % kKStages), (uint32_t)(i / kKStages) & 1u, kWaitLimitNs);
         }
     } else if (warp == 9) {
         // ---------------- logits MMA issuer: U = K W_k ----------------
@@ -305,15 +381,15 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
         Ring<2> ur;
         for (; !w.done(); w.next(), r.next(), ur.next()) {
             const int wb = w.seg & 1;
-            if (w.first() && !warp_wait(bar(WFULL + wb), (uint32_t)(w.seg >> 1) & 1u, err, kErrMmaLoad)) break;
-            if (!warp_wait(bar(FULL + r.s), r.ph, err, kErrMmaLoad)) break;
+            if (w.first() && !warp_wait(c.bar(K_WFULL + wb), (uint32_t)(w.seg >> 1) & 1u, c.wc, kErrMmaLoad)) break;
+            if (!warp_wait(c.bar(K_FULL + r.s), r.ph, c.wc, kErrMmaLoad)) break;
             LA_TRACE(1, w.i, 0);
-            if (w.i >= 2 && !warp_wait(bar(UEMPTY + ur.s), ur.ph ^ 1u, err, kErrMmaU)) break;
+            if (w.i >= 2 && !warp_wait(c.bar(K_UEMPTY + ur.s), ur.ph ^ 1u, c.wc, kErrMmaU)) break;
             tcgen05_fence_after();
             if (elect_one()) {
-                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * KSideSmem::kStage, sbase + KSideSmem::kW + wb * kWBytes);
-                mma_commit(bar(UFULL + ur.s));
-                if (w.last()) mma_commit(bar(WFREE + wb));
+                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * Smem::kKStage, sbase + Smem::kKW + wb * kWBytes);
+                mma_commit(c.bar(K_UFULL + ur.s));
+                if (w.last()) mma_commit(c.bar(K_WFREE + wb));
             }
             __syncwarp();
             LA_TRACE(1, w.i, 1);
@@ -322,17 +398,17 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
         // ---------------- accumulation MMA issuer: S += phi^T V, z += phi^T 1 ----------------
         constexpr uint32_t idesc_s = make_idesc_bf16(kD, kD, 1, 1);   // A = phi^T (MN-major), B = V (MN-major)
         constexpr uint32_t idesc_z = make_idesc_bf16(kD, 16, 1, 0);   // B = ones (K-major, no swizzle)
-        const uint64_t ones_desc = make_desc_noswizzle(sbase + KSideSmem::kOnes, 128, 256);
+        const uint64_t ones_desc = make_desc_noswizzle(sbase + Smem::kOnes, 128, 256);
         const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
         Ring<kKStages> r;
         for (; !w.done(); w.next(), r.next()) {
-            if (!warp_wait(bar(PHIFULL + r.s), r.ph, err, kErrMmaPhi)) break;
+            if (!warp_wait(c.bar(K_PHIFULL + r.s), r.ph, c.wc, kErrMmaPhi)) break;
             LA_TRACE(1, w.i, 2);
             const bool first = w.first();
-            if (first && w.seg >= 1 && !warp_wait(bar(ACCFREE), (uint32_t)(w.seg - 1) & 1u, err, kErrMmaAcc)) break;
+            if (first && w.seg >= 1 && !warp_wait(c.bar(K_ACCFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrMmaAcc)) break;
             tcgen05_fence_after();
             if (elect_one()) {
-                const uint32_t phi = sbase + r.s * KSideSmem::kStage, vt = phi + kTileBytes;
+                const uint32_t phi = sbase + r.s * Smem::kKStage, vt = phi + kTileBytes;
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k) {
                     const uint64_t da = desc_at(mnmajor, phi + k * 2048);
@@ -341,13 +417,13 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
                     mma_bf16_ss(tmem_s, da, db, idesc_s, acc);
                     mma_bf16_ss(tmem_z, da, ones_desc, idesc_z, acc);
                 }
-                mma_commit(bar(EMPTY + r.s));
-                if (w.last()) mma_commit(bar(ACCFULL));
+                mma_commit(c.bar(K_EMPTY + r.s));
+                if (w.last()) mma_commit(c.bar(K_ACCFULL));
             }
             __syncwarp();
             LA_TRACE(1, w.i, 3);
         }
-    } else {
+    } else if (warp < 8) {
         // ---------------- feature map + drain (warps 0-7) ----------------
         const int half = warp >> 2;                       // 0: softmax(+U), 1: softmax(-U)
         const int row = (warp & 3) * 32 + lane;           // token within the tile == TMEM lane
@@ -355,26 +431,26 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
         Ring<kKStages> r;
         Ring<2> ur;
         for (; !w.done(); w.next(), r.next(), ur.next()) {
-            if (!warp_wait(bar(UFULL + ur.s), ur.ph, err, kErrSoftmaxU)) break;
+            if (!warp_wait(c.bar(K_UFULL + ur.s), ur.ph, c.wc, kErrSoftmaxU)) break;
             if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 0);
             tcgen05_fence_after();
             float u[kM];
             load_logits(tmem_u + lane_base + ur.s * kM, u);
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(UEMPTY + ur.s));
+            if (lane == 0) mbar_arrive(c.bar(K_UEMPTY + ur.s));
             if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 1);
             const float keep = (w.lt * kTile + row < a.n) ? 1.f : 0.f;
-            uint8_t* dst = smem + r.s * KSideSmem::kStage + half * kHalfTileBytes + row * 128;
+            uint8_t* dst = c.smem + r.s * Smem::kKStage + half * kHalfTileBytes + row * 128;
             if (half == 0) softmax_half_to_smem<false>(u, keep, dst, row);
             else softmax_half_to_smem<true>(u, keep, dst, row);
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(PHIFULL + r.s));
+            if (lane == 0) mbar_arrive(c.bar(K_PHIFULL + r.s));
             if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 2);
             if (w.last()) {
                 // drain the accumulators of this segment: thread = feature f, this half's 64 columns of S
-                if (!warp_wait(bar(ACCFULL), (uint32_t)w.seg & 1u, err, kErrDrain)) break;
+                if (!warp_wait(c.bar(K_ACCFULL), (uint32_t)w.seg & 1u, c.wc, kErrDrain)) break;
                 tcgen05_fence_after();
                 float* rec = a.partial + (size_t)(blockIdx.x + w.g) * kE;
                 float* srow = rec + (size_t)row * kD + half * 64;
@@ -395,85 +471,67 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
                 }
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(ACCFREE));
+                if (lane == 0) mbar_arrive(c.bar(K_ACCFREE));
             }
         }
     }
-    tcgen05_fence_before();
-    __syncthreads();
-    if (warp == 9) tmem_dealloc(tmem, 512);
 }
 
 // ======================================================================================================
-// Combine
+// Combine: S = sum of partials, z likewise, in CTA order; bf16 images for the query side
 // ======================================================================================================
 
-struct CombineArgs {
-    const float* partial;       // [slots][kE]
-    float* state;               // [G][kE] fp32 (S row-major [f][c], then z)
-    __nv_bfloat16* s_img;       // [G][128][128] bf16, S[f][c] row-major
-    __nv_bfloat16* z_img;       // [G][2][16][64] bf16 operand image: row 0 = hi(z), row 1 = lo(z), swizzled
-    long long tiles_per_head, total_tiles, P;
-};
-
-// grid = (ceil(kE / 256), G).  Sums the partials of head g over the CTAs that touched it, in CTA order.
-static __global__ void __launch_bounds__(256) combine_tc(const CombineArgs a)
+// Four consecutive elements (e4 .. e4+3, e4 a multiple of 4) of head g's record: sum the partials of the
+// CTAs that touched the head in ascending CTA index (so the result does not depend on timing), store the
+// fp32 state and the bf16 operand images.  All loads of a batch are issued before the first add.
+__device__ __forceinline__ void combine_quad(const Args& a, long long P, int g, int e4)
 {
-    const int e = blockIdx.x * 256 + threadIdx.x;
-    if (e >= kE) return;
-    const long long g = blockIdx.y;
-    const long long c0 = tile_owner(g * a.tiles_per_head, a.total_tiles, a.P);
-    const long long c1 = tile_owner((g + 1) * a.tiles_per_head - 1, a.total_tiles, a.P);
-    const float* p = a.partial + (size_t)(c0 + g) * kE + e;
+    const long long c0 = tile_owner((long long)g * a.tiles_per_head, a.total_tiles, P);
+    const long long c1 = tile_owner((long long)(g + 1) * a.tiles_per_head - 1, a.total_tiles, P);
+    const float4* p = reinterpret_cast<const float4*>(a.partial + (size_t)(c0 + g) * kE + e4);
     const int cnt = (int)(c1 - c0) + 1;
-    float acc = 0.f;
-    int c = 0;
-    for (; c + 8 <= cnt; c += 8) {  // loads first (independent), then the adds in CTA order
-        float v[8];
+    constexpr int kBatch = 16;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = 0; base < cnt; base += kBatch) {
+        float4 v[kBatch];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = p[(size_t)(c + u) * kE];
+        for (int u = 0; u < kBatch; ++u)
+            v[u] = (base + u < cnt) ? __ldcg(p + (size_t)(base + u) * (kE / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) acc += v[u];
+        for (int u = 0; u < kBatch; ++u) {
+            if (base + u < cnt) {
+                acc.x += v[u].x;
+                acc.y += v[u].y;
+                acc.z += v[u].z;
+                acc.w += v[u].w;
+            }
+        }
     }
-    for (; c < cnt; ++c) acc += p[(size_t)c * kE];
-    a.state[(size_t)g * kE + e] = acc;
-    if (e < kD * kD) {
-        a.s_img[(size_t)g * kD * kD + e] = __float2bfloat16_rn(acc);
+    *reinterpret_cast<float4*>(a.state + (size_t)g * kE + e4) = acc;
+    const float r[4] = {acc.x, acc.y, acc.z, acc.w};
+    if (e4 < kD * kD) {
+        uint2 packed;
+        packed.x = pack_bf16(r[0], r[1]);
+        packed.y = pack_bf16(r[2], r[3]);
+        *reinterpret_cast<uint2*>(a.s_img + (size_t)g * kD * kD + e4) = packed;
     } else {
         // z[f]: hi and lo bf16 parts into rows 0 and 1 of the K-major operand block of feature block f / 64
-        const int f = e - kD * kD;
-        const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(acc - __bfloat162float(hi));
-        __nv_bfloat16* blk = a.z_img + (size_t)g * (kZBlkBytes / 2) + (f >> 6) * (16 * 64);
-        const int fi = f & 63, chunk = fi >> 3, within = fi & 7;
-        blk[0 * 64 + ((chunk ^ 0) << 3) + within] = hi;  // row 0: swizzle term (row & 7) = 0
-        blk[1 * 64 + ((chunk ^ 1) << 3) + within] = lo;  // row 1: swizzle term 1
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int f = e4 - kD * kD + t;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(r[t]);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(r[t] - __bfloat162float(hi));
+            __nv_bfloat16* blk = a.z_img + (size_t)g * (kZBlkBytes / 2) + (f >> 6) * (16 * 64);
+            const int fi = f & 63, chunk = fi >> 3, within = fi & 7;
+            blk[0 * 64 + ((chunk ^ 0) << 3) + within] = hi;  // row 0: swizzle term (row & 7) = 0
+            blk[1 * 64 + ((chunk ^ 1) << 3) + within] = lo;  // row 1: swizzle term 1
+        }
     }
 }
 
 // ======================================================================================================
-// Query side
+// Query side: o = phi(q) S / (phi(q) . z)  (Eq. 5, Eq. 6)
 // ======================================================================================================
-
-constexpr int kQStages = 5;
-struct QSideSmem {
-    static constexpr uint32_t kS = kQStages * kTileBytes;   // S image (32 KB)
-    static constexpr uint32_t kW = kS + kTileBytes;         // W^T (16 KB)
-    static constexpr uint32_t kZ = kW + kWBytes;            // z operand (4 KB)
-    static constexpr uint32_t kBars = kZ + kZBlkBytes;
-    static constexpr uint32_t kTotal = kBars + 512 + 1024;
-};
-
-struct QSideArgs {
-    const __nv_bfloat16* z_img;  // [G][kZBlkBytes / 2]
-    uint32_t* err;
-    int n, H;
-    int tiles_per_head;
-    long long total_tiles;
-#ifdef LINATTN_TRACE
-    long long* trace;
-#endif
-};
 
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar)
 {
@@ -482,90 +540,82 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
                  : "memory");
 }
 
-__global__ void __launch_bounds__(kQThreads, 1)
-qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
-         const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS, const QSideArgs a)
+// wait_state: the S and z images are produced earlier in the same kernel (fused path); loads of them
+// must wait for the Q_SREADY barrier.  Otherwise they were written by a previous launch.
+__device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
+                                            const CUtensorMap* tmW, const CUtensorMap* tmS, bool wait_state)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const uint32_t sbase = smem_u32(smem);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + QSideSmem::kBars);
-    enum { QFULL = 0, QEMPTY = 5, PHIFULL = 10, OFULL = 15, UFULL = 20, UEMPTY = 22, DFULL = 24, DEMPTY = 26, SEGFULL = 28, SEGFREE = 29, NBARS = 30 };
-    const uint32_t bar0 = smem_u32(bars);
-    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[NBARS]);
-    uint32_t* err = a.err;
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    if (tid == 0) {
-        for (int i = 0; i < kQStages; ++i) { mbar_init(bar(QFULL + i), 1); mbar_init(bar(QEMPTY + i), 1); mbar_init(bar(PHIFULL + i), 8); mbar_init(bar(OFULL + i), 8); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(UFULL + i), 1); mbar_init(bar(UEMPTY + i), 8); mbar_init(bar(DFULL + i), 1); mbar_init(bar(DEMPTY + i), 8); }
-        mbar_init(bar(SEGFULL), 1);
-        mbar_init(bar(SEGFREE), 1);
-        fence_mbar_init();
-    }
-    if (warp == 9) {
-        tmem_alloc(smem_u32(tmem_slot), 512);
-        tmem_relinquish();
-    }
-    if (warp == 8 && lane == 0) {
-        tma_prefetch_desc(&tmQ);
-        tma_prefetch_desc(&tmO);
-        tma_prefetch_desc(&tmW);
-        tma_prefetch_desc(&tmS);
-    }
-    tcgen05_fence_before();
-    __syncthreads();
-    tcgen05_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    const uint32_t tmem_u = tmem;  // 2 x 64 columns of logits
-    auto tmem_num = [&](int db) { return tmem + 128 + db * 160; };   // 128 columns: num[token][c]
-    auto tmem_den = [&](int db) { return tmem + 256 + db * 160; };   // 16 columns: [hi(z) part, lo(z) part, ...]
-
+    const uint32_t tmem_u = c.tmem;  // 2 x 64 columns of logits
+    auto tmem_num = [&](int db) { return c.tmem + 128 + db * 160; };   // 128 columns: num[token][c]
+    auto tmem_den = [&](int db) { return c.tmem + 256 + db * 160; };   // 16 columns: [hi(z) part, lo(z) part, ...]
+    const int warp = c.warp, lane = c.lane;
+    const uint32_t sbase = c.sbase;
     TileWalk w;
     w.init(a.total_tiles, a.tiles_per_head);
 
     if (warp == 8) {
         // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            tma_prefetch_desc(tmQ);
+            tma_prefetch_desc(tmW);
+            tma_prefetch_desc(tmS);
+        }
         Ring<kQStages> r;
         int issued = 0;
-        for (; !w.done(); w.next(), r.next()) {
-            if (w.first()) {
-                if (w.seg >= 1 && !warp_wait(bar(SEGFREE), (uint32_t)(w.seg - 1) & 1u, err, kErrSeg)) break;
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(bar(SEGFULL), kWBytes + kTileBytes + kZBlkBytes);
-                    tma_load_3d(sbase + QSideSmem::kW, &tmW, bar(SEGFULL), 0, 0, w.g % a.H);
-                    tma_load_3d(sbase + QSideSmem::kW + kWBytes / 2, &tmW, bar(SEGFULL), 64, 0, w.g % a.H);
-                    tma_load_3d(sbase + QSideSmem::kS, &tmS, bar(SEGFULL), 0, 0, w.g);
-                    tma_load_3d(sbase + QSideSmem::kS + kHalfTileBytes, &tmS, bar(SEGFULL), 64, 0, w.g);
-                    bulk_load_1d(sbase + QSideSmem::kZ, a.z_img + (size_t)w.g * (kZBlkBytes / 2), kZBlkBytes, bar(SEGFULL));
-                }
-            }
-            if (w.i >= kQStages && !warp_wait(bar(QEMPTY + r.s), r.ph ^ 1u, err, kErrProducer)) break;
+        int state_g = -1;   // head whose S, z still have to be loaded (W already on its way)
+        bool ok = true;
+        auto load_state = [&]() {
+            // S and z of head state_g; in the fused kernel they were written by other CTAs with ordinary
+            // stores and become readable once the grid barrier behind Q_SREADY has been passed
+            if (wait_state && !warp_wait(c.bar(Q_SREADY), 0u, c.wc, kErrSeg)) { ok = false; return; }
             if (lane == 0) {
-                mbar_arrive_expect_tx(bar(QFULL + r.s), kTileBytes);
-                tma_load_3d(sbase + r.s * kTileBytes, &tmQ, bar(QFULL + r.s), 0, w.lt * kTile, w.g);
-                tma_load_3d(sbase + r.s * kTileBytes + kHalfTileBytes, &tmQ, bar(QFULL + r.s), 64, w.lt * kTile, w.g);
+                if (wait_state) fence_proxy_async_all();
+                mbar_arrive_expect_tx(c.bar(Q_SEGFULL), kTileBytes + kZBlkBytes);
+                tma_load_3d(sbase + Smem::kQS, tmS, c.bar(Q_SEGFULL), 0, 0, state_g);
+                tma_load_3d(sbase + Smem::kQS + kHalfTileBytes, tmS, c.bar(Q_SEGFULL), 64, 0, state_g);
+                bulk_load_1d(sbase + Smem::kQZ, a.z_img + (size_t)state_g * (kZBlkBytes / 2), kZBlkBytes, c.bar(Q_SEGFULL));
+            }
+            state_g = -1;
+        };
+        for (; !w.done() && ok; w.next(), r.next()) {
+            if (w.first()) {
+                if (w.seg >= 1 && !warp_wait(c.bar(Q_SEGFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrSeg)) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(c.bar(Q_WFULL), kWBytes);
+                    tma_load_3d(sbase + Smem::kQW, tmW, c.bar(Q_WFULL), 0, 0, w.g % a.H);
+                    tma_load_3d(sbase + Smem::kQW + kWBytes / 2, tmW, c.bar(Q_WFULL), 64, 0, w.g % a.H);
+                }
+                state_g = w.g;
+                // the first head's state may not exist yet: get the first Q tiles moving before waiting for it
+                if (!(wait_state && w.seg == 0)) load_state();
+            }
+            if (state_g >= 0 && w.i >= kQStages) load_state();
+            if (!ok) break;
+            if (w.i >= kQStages && !warp_wait(c.bar(Q_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) break;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(c.bar(Q_FULL + r.s), kTileBytes);
+                tma_load_3d(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g);
+                tma_load_3d(sbase + r.s * kTileBytes + kHalfTileBytes, tmQ, c.bar(Q_FULL + r.s), 64, w.lt * kTile, w.g);
             }
             issued = w.i + 1;
         }
+        if (ok && state_g >= 0) load_state();
         if (issued < w.count) {
             for (int i = (issued > kQStages ? issued - kQStages : 0); i < issued; ++i)
-                mbar_wait(bar(QFULL + i % kQStages), (uint32_t)(i / kQStages) & 1u, kWaitLimitNs);
+                mbar_wait(c.bar(Q_FULL + i % kQStages), (uint32_t)(i / kQStages) & 1u, kWaitLimitNs);
         }
     } else if (warp == 9) {
         // ---------------- logits MMA issuer: U = Q W_q ----------------
         Ring<kQStages> r;
         Ring<2> ur;
         for (; !w.done(); w.next(), r.next(), ur.next()) {
-            if (w.first() && !warp_wait(bar(SEGFULL), (uint32_t)w.seg & 1u, err, kErrSeg)) break;
-            if (!warp_wait(bar(QFULL + r.s), r.ph, err, kErrMmaLoad)) break;
-            if (w.i >= 2 && !warp_wait(bar(UEMPTY + ur.s), ur.ph ^ 1u, err, kErrMmaU)) break;
+            if (w.first() && !warp_wait(c.bar(Q_WFULL), (uint32_t)w.seg & 1u, c.wc, kErrSeg)) break;
+            if (!warp_wait(c.bar(Q_FULL + r.s), r.ph, c.wc, kErrMmaLoad)) break;
+            if (w.i >= 2 && !warp_wait(c.bar(Q_UEMPTY + ur.s), ur.ph ^ 1u, c.wc, kErrMmaU)) break;
             tcgen05_fence_after();
             if (elect_one()) {
-                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + QSideSmem::kW);
-                mma_commit(bar(UFULL + ur.s));
+                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + Smem::kQW);
+                mma_commit(c.bar(Q_UFULL + ur.s));
             }
             __syncwarp();
         }
@@ -578,41 +628,42 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
         Ring<kQStages> r;
         Ring<2> dr;
         for (; !w.done(); w.next(), r.next(), dr.next()) {
-            if (w.first() && !warp_wait(bar(SEGFULL), (uint32_t)w.seg & 1u, err, kErrSeg)) break;
-            if (!warp_wait(bar(PHIFULL + r.s), r.ph, err, kErrMmaPhi)) break;
-            if (w.i >= 2 && !warp_wait(bar(DEMPTY + dr.s), dr.ph ^ 1u, err, kErrMmaAcc)) break;
+            if (w.first() && !warp_wait(c.bar(Q_SEGFULL), (uint32_t)w.seg & 1u, c.wc, kErrSeg)) break;
+            if (!warp_wait(c.bar(Q_PHIFULL + r.s), r.ph, c.wc, kErrMmaPhi)) break;
+            if (w.i >= 2 && !warp_wait(c.bar(Q_DEMPTY + dr.s), dr.ph ^ 1u, c.wc, kErrMmaAcc)) break;
             tcgen05_fence_after();
             if (elect_one()) {
                 const uint32_t phi = sbase + r.s * kTileBytes;
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) {
                     const uint64_t da = desc_at(kmajor, phi + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
-                    const uint64_t db_s = desc_at(mnmajor, sbase + QSideSmem::kS + k * 2048);
-                    const uint64_t db_z = desc_at(kmajor, sbase + QSideSmem::kZ + (k >> 2) * 2048 + (k & 3) * 32);
+                    const uint64_t db_s = desc_at(mnmajor, sbase + Smem::kQS + k * 2048);
+                    const uint64_t db_z = desc_at(kmajor, sbase + Smem::kQZ + (k >> 2) * 2048 + (k & 3) * 32);
                     mma_bf16_ss(tmem_num(dr.s), da, db_s, idesc_n, k > 0);
                     mma_bf16_ss(tmem_den(dr.s), da, db_z, idesc_d, k > 0);
                 }
-                mma_commit(bar(DFULL + dr.s));
-                if (w.last()) mma_commit(bar(SEGFREE));   // this head's S, z and W may now be replaced
+                mma_commit(c.bar(Q_DFULL + dr.s));
+                if (w.last()) mma_commit(c.bar(Q_SEGFREE));   // this head's S, z and W may now be replaced
             }
             __syncwarp();
         }
     } else if (warp == 11) {
         // ---------------- TMA stores of finished output tiles ----------------
+        if (lane == 0) tma_prefetch_desc(tmO);
         Ring<kQStages> r;
         for (; !w.done(); w.next(), r.next()) {
-            if (!warp_wait(bar(OFULL + r.s), r.ph, err, kErrStore)) break;
+            if (!warp_wait(c.bar(Q_OFULL + r.s), r.ph, c.wc, kErrStore)) break;
             if (lane == 0) {
-                tma_store_3d(&tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g);
-                tma_store_3d(&tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g);
+                tma_store_3d(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g);
+                tma_store_3d(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g);
                 bulk_commit_group();
                 bulk_wait_group_read<0>();   // the slot has been read out: hand it back to the producer
-                mbar_arrive(bar(QEMPTY + r.s));
+                mbar_arrive(c.bar(Q_EMPTY + r.s));
             }
             __syncwarp();
         }
         if (lane == 0) bulk_wait_group<0>();
-    } else {
+    } else if (warp < 8) {
         // ---------------- feature map + epilogue (warps 0-7) ----------------
         const int half = warp >> 2;
         const int row = (warp & 3) * 32 + lane;
@@ -621,24 +672,24 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
         Ring<2> ur, dr;
         for (int i = 0; i <= w.count; ++i) {
             if (i < w.count) {
-                if (!warp_wait(bar(UFULL + ur.s), ur.ph, err, kErrSoftmaxU)) break;
+                if (!warp_wait(c.bar(Q_UFULL + ur.s), ur.ph, c.wc, kErrSoftmaxU)) break;
                 tcgen05_fence_after();
                 float u[kM];
                 load_logits(tmem_u + lane_base + ur.s * kM, u);
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(UEMPTY + ur.s));
-                uint8_t* dst = smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                if (lane == 0) mbar_arrive(c.bar(Q_UEMPTY + ur.s));
+                uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
                 if (half == 0) softmax_half_to_smem<false>(u, 1.f, dst, row);
                 else softmax_half_to_smem<true>(u, 1.f, dst, row);
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(PHIFULL + r.s));
+                if (lane == 0) mbar_arrive(c.bar(Q_PHIFULL + r.s));
                 r.next();
                 ur.next();
             }
             if (i >= 1) {
-                if (!warp_wait(bar(DFULL + dr.s), dr.ph, err, kErrEpilogue)) break;
+                if (!warp_wait(c.bar(Q_DFULL + dr.s), dr.ph, c.wc, kErrEpilogue)) break;
                 tcgen05_fence_after();
                 uint32_t v[64], dv[2];
                 tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64, v);
@@ -647,30 +698,135 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
                 tmem_wait_ld();
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(DEMPTY + dr.s));
+                if (lane == 0) mbar_arrive(c.bar(Q_DEMPTY + dr.s));
                 const float inv = __fdividef(1.f, __uint_as_float(dv[0]) + __uint_as_float(dv[1]));
-                uint8_t* dst = smem + er.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                uint8_t* dst = c.smem + er.s * kTileBytes + half * kHalfTileBytes + row * 128;
                 const int sw = row & 7;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
+                for (int cc = 0; cc < 8; ++cc) {
                     uint4 o;
-                    o.x = pack_bf16(__uint_as_float(v[8 * c + 0]) * inv, __uint_as_float(v[8 * c + 1]) * inv);
-                    o.y = pack_bf16(__uint_as_float(v[8 * c + 2]) * inv, __uint_as_float(v[8 * c + 3]) * inv);
-                    o.z = pack_bf16(__uint_as_float(v[8 * c + 4]) * inv, __uint_as_float(v[8 * c + 5]) * inv);
-                    o.w = pack_bf16(__uint_as_float(v[8 * c + 6]) * inv, __uint_as_float(v[8 * c + 7]) * inv);
-                    *reinterpret_cast<uint4*>(dst + ((c ^ sw) << 4)) = o;
+                    o.x = pack_bf16(__uint_as_float(v[8 * cc + 0]) * inv, __uint_as_float(v[8 * cc + 1]) * inv);
+                    o.y = pack_bf16(__uint_as_float(v[8 * cc + 2]) * inv, __uint_as_float(v[8 * cc + 3]) * inv);
+                    o.z = pack_bf16(__uint_as_float(v[8 * cc + 4]) * inv, __uint_as_float(v[8 * cc + 5]) * inv);
+                    o.w = pack_bf16(__uint_as_float(v[8 * cc + 6]) * inv, __uint_as_float(v[8 * cc + 7]) * inv);
+                    *reinterpret_cast<uint4*>(dst + ((cc ^ sw) << 4)) = o;
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(OFULL + er.s));
+                if (lane == 0) mbar_arrive(c.bar(Q_OFULL + er.s));
                 er.next();
                 dr.next();
             }
         }
     }
+}
+
+// ======================================================================================================
+// Kernels
+// ======================================================================================================
+
+__global__ void __launch_bounds__(kThreads, 1)
+kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+         const __grid_constant__ CUtensorMap tmW, const Args a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const Cta c = cta_setup(smem_raw, a, true, false);
+    kside_phase(c, a, &tmK, &tmV, &tmW);
+    cta_teardown(c);
+}
+
+// grid = (ceil(kE / 4 / 256), G)
+static __global__ void __launch_bounds__(256) combine_tc(const Args a, long long P)
+{
+    const int q4 = blockIdx.x * 256 + threadIdx.x;
+    if (q4 < kE / 4) combine_quad(a, P, blockIdx.y, q4 * 4);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
+         const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS, const Args a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const Cta c = cta_setup(smem_raw, a, false, true);
+    qside_phase(c, a, &tmQ, &tmO, &tmW, &tmS, false);
+    cta_teardown(c);
+}
+
+// Grid-wide barrier for a cooperative launch (all CTAs resident).  Called by ONE thread per CTA after a
+// CTA-level barrier.  sync[0] counts arrivals and wraps to 0 by itself; sync[1] is the generation that the
+// last arriver advances.  The wait is bounded: returns false on time-out.
+__device__ __forceinline__ bool grid_barrier(uint32_t* sync, uint32_t P)
+{
+    const uint32_t gen0 = ld_acquire_gpu(sync + 1);
+    __threadfence();
+    const uint32_t old = atomicInc(sync, P - 1);
+    if (old == P - 1) {
+        __threadfence();
+        atomicAdd(sync + 1, 1u);
+    } else {
+        const uint64_t t0 = globaltimer_ns();
+        uint32_t spins = 0;
+        while (ld_acquire_gpu(sync + 1) == gen0) {
+            if ((++spins & 63u) == 0u && globaltimer_ns() - t0 > kWaitLimitNs) return false;
+        }
+    }
+    __threadfence();
+    return true;
+}
+
+// The whole forward in one cooperative launch of P <= #SMs persistent CTAs.
+__global__ void __launch_bounds__(kThreads, 1)
+linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                 const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmQ,
+                 const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmWq,
+                 const __grid_constant__ CUtensorMap tmS, const Args a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    LA_TRACE_NS(0, 60, 0);
+    const Cta c = cta_setup(smem_raw, a, true, true);
+    LA_TRACE_NS(0, 60, 1);
+    kside_phase(c, a, &tmK, &tmV, &tmWk);
+    // every role is done with the key-side buffers; the partials of this CTA are written
     tcgen05_fence_before();
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tmem, 512);
+    tcgen05_fence_after();
+    LA_TRACE_NS(0, 60, 2);
+    if (c.warp < 8) {
+        // warps 0-7: grid barrier, combine (spread over all CTAs), grid barrier, then release the query side.
+        // The other warps go straight on: Q tiles, W_q and the first logits do not depend on S.
+        __shared__ uint32_t gb_ok;
+        const uint32_t P = gridDim.x;
+        if (threadIdx.x == 0) {
+            gb_ok = grid_barrier(a.sync, P) ? 1u : 0u;
+            if (!gb_ok) {
+                atomicOr(a.err, (uint32_t)kErrGrid);
+                asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
+            }
+        }
+        named_barrier_sync(1, 256);
+        LA_TRACE_NS(0, 60, 3);
+        if (gb_ok) {
+            const int total = a.G * (kE / 4);   // float4 groups over all heads
+            for (int x = blockIdx.x * 256 + threadIdx.x; x < total; x += (int)P * 256)
+                combine_quad(a, P, x / (kE / 4), (x % (kE / 4)) * 4);
+        }
+        named_barrier_sync(1, 256);
+        LA_TRACE_NS(0, 61, 0);
+        if (threadIdx.x == 0 && gb_ok) {
+            if (!grid_barrier(a.sync, P)) {
+                gb_ok = 0u;
+                atomicOr(a.err, (uint32_t)kErrGrid);
+                asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
+            }
+        }
+        named_barrier_sync(1, 256);
+        if (c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
+        LA_TRACE_NS(0, 61, 1);
+    }
+    qside_phase(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
+    LA_TRACE_NS(0, 61, 2);
+    cta_teardown(c);
+    LA_TRACE_NS(0, 61, 3);
 }
 
 // W [H][128 d][64 j] (any supported type) -> W^T bf16 [H][64 j][128 d]; per_head == 0 replicates one matrix.

@@ -68,6 +68,33 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_
     }
     return true;
 }
+// The same, but also gives up as soon as the CTA's abort word (shared memory) is non-zero, so that
+// after one wait has timed out the other roles unwind at once instead of each running out its own limit.
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, uint64_t limit_ns, uint32_t abort_smem)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0u) {
+            uint32_t ab;
+            asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(ab) : "r"(abort_smem) : "memory");
+            if (ab != 0u || globaltimer_ns() - t0 > limit_ns) return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Orders earlier generic-proxy accesses (after an acquire) before later async-proxy (TMA) accesses.
+__device__ __forceinline__ void fence_proxy_async_all()
+{
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
 
 // ---- proxies and fences --------------------------------------------------------------------------
 

@@ -15,7 +15,18 @@ from util import assert_parity, errors, run_gpu
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [linattn.PATH_AUTO, linattn.PATH_SIMT]
+# (path option, fuse option): automatic choice (one fused tensor-core kernel where it applies), the
+# tensor-core kernels as three launches, and the CUDA-core kernels
+MODES = [(linattn.PATH_AUTO, 1), (linattn.PATH_AUTO, 0), (linattn.PATH_SIMT, 0)]
+MODE_IDS = ["auto", "unfused", "simt"]
+
+
+def mode_param():
+    return pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+
+
+def run_mode(x, mode, **kw):
+    return run_gpu(x, path=mode[0], fuse=mode[1], **kw)
 
 
 def small_inputs(B, H, n, d, dtype, seed, wmode="random"):
@@ -40,10 +51,10 @@ def oracle_out(x, rows=None):
 
 # ---- config 1: the tiny fp32 case against the O(n^2) brute-force form --------------------------
 
-@pytest.mark.parametrize("path", PATHS)
-def test_config1_tiny_against_quadratic_form(path):
+@mode_param()
+def test_config1_tiny_against_quadratic_form(mode):
     x = synth.make_inputs(1)
-    got, S, z = run_gpu(x, path=path, return_state=True)
+    got, S, z = run_mode(x, mode, return_state=True)
     want = oracle.ref_quadratic(x["q"], x["k"], x["v"], x["Wq"], x["Wk"])
     assert_parity(got, want, "config 1 vs quadratic form")
     _, S_ref, z_ref = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], return_state=True)
@@ -52,13 +63,13 @@ def test_config1_tiny_against_quadratic_form(path):
 
 # ---- ragged sizes: several tiles plus a tail, the degenerate n = 1, 2 -----------------------------
 
-@pytest.mark.parametrize("path", PATHS)
+@mode_param()
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("d", [64, 128])
 @pytest.mark.parametrize("n", [1, 2, 127, 129, 1000, 4097])
-def test_ragged_lengths(n, d, dtype, path):
+def test_ragged_lengths(n, d, dtype, mode):
     x = small_inputs(2, 3, n, d, dtype, seed=1000 + n + d)
-    got, S, z = run_gpu(x, path=path, return_state=True)
+    got, S, z = run_mode(x, mode, return_state=True)
     assert_parity(got, oracle_out(x), f"n={n} d={d} {dtype}")
     _, S_ref, z_ref = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], return_state=True)
     assert errors(z, z_ref)[0] <= 5e-3, "z"
@@ -67,58 +78,59 @@ def test_ragged_lengths(n, d, dtype, path):
         assert_parity(got, x["v"].double().numpy(), "n=1 returns v")
 
 
-@pytest.mark.parametrize("path", PATHS)
+@mode_param()
 @pytest.mark.parametrize("splits", [1, 2, 3, 7, 33])
-def test_split_count_does_not_change_the_answer(splits, path):
+def test_split_count_does_not_change_the_answer(splits, mode):
     x = small_inputs(1, 2, 2500, 128, torch.bfloat16, seed=77)
-    got = run_gpu(x, path=path, splits=splits)
+    got = run_mode(x, mode, splits=splits)
     assert_parity(got, oracle_out(x), f"splits={splits}")
 
 
 # ---- special feature maps ---------------------------------------------------------------------------
 
-@pytest.mark.parametrize("path", PATHS)
+@mode_param()
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_zero_weights_give_the_mean_of_v(dtype, path):
+def test_zero_weights_give_the_mean_of_v(dtype, mode):
     x = small_inputs(1, 2, 777, 128, dtype, seed=5, wmode="zero")
-    got = run_gpu(x, path=path)
+    got = run_mode(x, mode)
     mean_v = x["v"].double().numpy().mean(axis=2, keepdims=True)
     assert_parity(got, np.broadcast_to(mean_v, got.shape), "W=0 -> mean of V")
 
 
-@pytest.mark.parametrize("path", PATHS)
+@mode_param()
 @pytest.mark.parametrize("wmode", ["identity", "shared"])
-def test_identity_and_shared_weights(wmode, path):
+def test_identity_and_shared_weights(wmode, mode):
     x = small_inputs(2, 2, 900, 128, torch.bfloat16, seed=6, wmode=wmode)
-    assert_parity(run_gpu(x, path=path), oracle_out(x), wmode)
+    assert_parity(run_mode(x, mode), oracle_out(x), wmode)
 
 
-@pytest.mark.parametrize("path", PATHS)
-def test_large_logits_do_not_overflow(path):
+@mode_param()
+def test_large_logits_do_not_overflow(mode):
     """Logits of magnitude ~50: exp without max subtraction would overflow fp32 sums / underflow to 0/0."""
     x = small_inputs(1, 2, 600, 128, torch.bfloat16, seed=8)
     x["Wq"] = (x["Wq"].float() * 40).to(torch.bfloat16)
     x["Wk"] = (x["Wk"].float() * 40).to(torch.bfloat16)
-    assert_parity(run_gpu(x, path=path), oracle_out(x), "large logits")
+    assert_parity(run_mode(x, mode), oracle_out(x), "large logits")
 
 
 # ---- reduced-size versions of the bf16 workloads (same distributions, fewer heads / tokens) ----------
 
-@pytest.mark.parametrize("path", PATHS)
+@mode_param()
 @pytest.mark.parametrize("config,H,n", [(2, 3, 4216), (3, 4, 4216), (4, 2, 9300), (5, 3, 4216)])
-def test_reduced_workloads(config, H, n, path):
+def test_reduced_workloads(config, H, n, mode):
     x = synth.make_inputs(config, H=H, n=n)
-    assert_parity(run_gpu(x, path=path), oracle_out(x), f"config {config} reduced")
+    assert_parity(run_mode(x, mode), oracle_out(x), f"config {config} reduced")
 
 
 # ---- determinism and context reuse --------------------------------------------------------------------
 
-@pytest.mark.parametrize("path", PATHS)
-def test_bit_identical_across_runs_and_context_reuse(path):
+@mode_param()
+def test_bit_identical_across_runs_and_context_reuse(mode):
     x = small_inputs(2, 4, 3000, 128, torch.bfloat16, seed=9)
     ctx = linattn.LinAttn(4, 128, max_B=2, max_n=4000)
     try:
-        ctx.set_option(linattn.OPT_PATH, path)
+        ctx.set_option(linattn.OPT_PATH, mode[0])
+        ctx.set_option(linattn.OPT_FUSE, mode[1])
         ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
         q, k, v = x["q"].cuda(), x["k"].cuda(), x["v"].cuda()
         first = ctx.forward(q, k, v).clone()
@@ -146,8 +158,9 @@ def test_output_guard_bands_are_untouched():
     out = buf[pad:pad + B * H * n * d].view(B, H, n, d)
     ctx = linattn.LinAttn(H, d, max_B=B, max_n=n)
     try:
-        for path in PATHS:
-            ctx.set_option(linattn.OPT_PATH, path)
+        for mode in MODES:
+            ctx.set_option(linattn.OPT_PATH, mode[0])
+            ctx.set_option(linattn.OPT_FUSE, mode[1])
             ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
             ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda(), out=out)
             ctx.check()
@@ -170,6 +183,38 @@ def test_host_buffer_entry_point_matches_device_entry_point():
         host_out2 = torch.empty_like(x["q"]).pin_memory()
         ctx.forward_host(pin["q"], pin["k"], pin["v"], host_out2)
         assert torch.equal(dev, host_out2)
+    finally:
+        ctx.destroy()
+
+
+def test_which_kernels_run():
+    """bf16, d = 128, bf16 weights -> the tensor-core kernels (one fused launch by default); fp32 -> CUDA cores."""
+    x = small_inputs(1, 2, 700, 128, torch.bfloat16, seed=14)
+    ctx = linattn.LinAttn(2, 128, max_B=1, max_n=700)
+    try:
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        q, k, v = x["q"].cuda(), x["k"].cuda(), x["v"].cuda()
+
+        def names(path, fuse):
+            ctx.set_option(linattn.OPT_PATH, path)
+            ctx.set_option(linattn.OPT_FUSE, fuse)
+            ctx.set_option(linattn.OPT_PROFILE, 1)
+            ctx.forward(q, k, v)
+            got = [kt["name"] for kt in ctx.kernel_times()]
+            ctx.set_option(linattn.OPT_PROFILE, 0)
+            return got, ctx.last_launch_count()
+
+        assert names(linattn.PATH_AUTO, 1) == (["linattn_fused_tc"], 1)
+        assert names(linattn.PATH_TENSOR, 0) == (["kside_tc", "combine_tc", "qside_tc"], 3)
+        assert names(linattn.PATH_SIMT, 1) == (["kside_simt", "combine_state", "qside_simt"], 3)
+        ctx.check()
+        # fp32 weights with bf16 activations: the tensor-core path would have to round them, so it is not taken
+        ctx.set_feature_map(x["Wq"].float().cuda(), x["Wk"].float().cuda())
+        assert names(linattn.PATH_AUTO, 1)[0][0] == "kside_simt"
+        lib = linattn.load_library()
+        ctx.set_option(linattn.OPT_PATH, linattn.PATH_TENSOR)
+        assert lib.linattn_forward(ctx._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), torch.empty_like(q).data_ptr(),
+                                   1, 2, 700, 128, linattn.BF16, None) == linattn.ERR_UNSUPPORTED
     finally:
         ctx.destroy()
 
