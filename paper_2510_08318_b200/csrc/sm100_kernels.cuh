@@ -18,10 +18,11 @@
 //
 // Work split: the G * ceil(n/128) tiles form one sequence (head-major); CTA c of P owns the contiguous
 // run [c*T/P, (c+1)*T/P).  A run may cross head boundaries; each (CTA, head) piece is a "segment".
-// Warp roles: warps 0-3 feature map of softmax(+U) / output columns 0-63, warps 4-7 softmax(-U) / columns
-// 64-127, warp 8 TMA producer, warp 9 issues the logits MMAs, warp 10 issues the accumulation MMAs, and
-// (query side only) warp 11 issues the TMA stores.  Role loops are warp-uniform; single-thread work
-// (TMA and MMA issue) is predicated inside them.
+// Warp roles (16 warps): warps 0-3 feature map softmax(+U), warps 4-7 softmax(-U) (one token per thread),
+// warp 8 TMA producer, warp 9 issues the logits MMAs, warp 10 issues the accumulation MMAs, warp 11 issues
+// the TMA stores (query side), warps 12-15 query-side epilogue (num / den -> bf16 output tile) and, in the
+// fused kernel, the grid barriers and the combine step between the two sides.  Role loops are
+// warp-uniform; single-thread work (TMA and MMA issue) is predicated inside them.
 // Every wait is bounded: on time-out the kernel records a code in *err, raises the CTA's abort word so
 // that the other roles stop waiting too, and unwinds.
 #pragma once
@@ -132,35 +133,118 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// ---- packed fp32 pairs (one instruction for two lanes of arithmetic) ----------------------------------
+using f32x2 = uint64_t;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+__device__ __forceinline__ float min3(float a, float b, float c)
+{
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// 2^x for a pair of x <= 0 on the FMA pipe (no special-function unit): x = i + f with i = round(x),
+// f in [-1/2, 1/2]; 2^f by a cubic (relative error < 7.5e-5, far below the bf16 rounding applied to the
+// result), then i is added into the exponent field.  x is clamped at -126 (result ~1e-38).
+__device__ __forceinline__ f32x2 exp2_poly2(f32x2 x)
+{
+    float x0, x1;
+    unpack2(x, x0, x1);
+    x = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const float magic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    const f32x2 t = add2(x, pack2(magic, magic));
+    const f32x2 fi = add2(t, pack2(-magic, -magic));
+    const f32x2 f = fma2(fi, pack2(-1.f, -1.f), x);
+    f32x2 p = fma2(f, pack2(0.055171459913253784f, 0.055171459913253784f), pack2(0.2426108568906784f, 0.2426108568906784f));
+    p = fma2(p, f, pack2(0.6932609677314758f, 0.6932609677314758f));
+    p = fma2(p, f, pack2(0.9999281167984009f, 0.9999281167984009f));
+    float p0, p1, t0, t1;
+    unpack2(p, p0, p1);
+    unpack2(t, t0, t1);
+    const float r0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+    const float r1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+    return pack2(r0, r1);
+}
+
 // One softmax half of Eq. 6 for one token.  u[64] holds the logits of this thread's token on entry.
 // kNeg = false: softmax(+u); kNeg = true: softmax(-u).  The 64 results, scaled by `keep` (0 for rows
 // past the end of the sequence), are written as bf16 to `row_base` = start of this token's 128-byte row
 // in the 64-feature block, 16-byte chunk c stored at chunk c ^ (row & 7) (the 128-byte swizzle).
+// Arithmetic is fp32, two lanes per instruction; one pair in four takes its exponentials on the FMA
+// pipe (exp2_poly2) so that the special-function unit and the FMA pipe finish together.
 template <bool kNeg>
 __device__ __forceinline__ void softmax_half_to_smem(float (&u)[kM], float keep, uint8_t* row_base, int row)
 {
-    float m = u[0];
+    float m = kNeg ? min3(u[0], u[1], u[2]) : max3(u[0], u[1], u[2]);
 #pragma unroll
-    for (int j = 1; j < kM; ++j) m = kNeg ? fminf(m, u[j]) : fmaxf(m, u[j]);
+    for (int j = 3; j < kM - 1; j += 2) m = kNeg ? min3(m, u[j], u[j + 1]) : max3(m, u[j], u[j + 1]);
+    m = kNeg ? fminf(m, u[kM - 1]) : fmaxf(m, u[kM - 1]);
     // exp(u - max) = 2^(u*log2e - max*log2e);   exp(-u - max(-u)) = 2^(min*log2e - u*log2e)
-    const float mL = m * kLog2e;
-    float sum = 0.f;
+    const float sL = kNeg ? -kLog2e : kLog2e;
+    const float off = kNeg ? m * kLog2e : -m * kLog2e;
+    const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
+    f32x2 e[kM / 2];
+    f32x2 sum2 = pack2(0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < kM; ++j) {
-        const float e = kNeg ? ex2_approx(fmaf(-u[j], kLog2e, mL)) : ex2_approx(fmaf(u[j], kLog2e, -mL));
-        u[j] = e;
-        sum += e;
+    for (int p = 0; p < kM / 2; ++p) {
+        const f32x2 x = fma2(pack2(u[2 * p], u[2 * p + 1]), scale, offset);
+        if ((p & 3) == 3) {
+            e[p] = exp2_poly2(x);
+        } else {
+            float x0, x1;
+            unpack2(x, x0, x1);
+            e[p] = pack2(ex2_approx(x0), ex2_approx(x1));
+        }
+        sum2 = add2(sum2, e[p]);
     }
-    const float inv = __fdividef(keep, sum);
+    float s0, s1;
+    unpack2(sum2, s0, s1);
+    const float inv = __fdividef(keep, s0 + s1);
+    const f32x2 inv2 = pack2(inv, inv);
     const int sw = row & 7;
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-        uint4 v;
-        v.x = pack_bf16(u[8 * c + 0] * inv, u[8 * c + 1] * inv);
-        v.y = pack_bf16(u[8 * c + 2] * inv, u[8 * c + 3] * inv);
-        v.z = pack_bf16(u[8 * c + 4] * inv, u[8 * c + 5] * inv);
-        v.w = pack_bf16(u[8 * c + 6] * inv, u[8 * c + 7] * inv);
-        *reinterpret_cast<uint4*>(row_base + ((c ^ sw) << 4)) = v;
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float a, b;
+            unpack2(mul2(e[4 * c + q], inv2), a, b);
+            w[q] = pack_bf16(a, b);
+        }
+        *reinterpret_cast<uint4*>(row_base + ((c ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -189,9 +273,15 @@ constexpr int kTraceTiles = 64;
         if (a.trace && threadIdx.x == 0)                                                                        \
             a.trace[(((size_t)blockIdx.x * 4 + (role)) * kTraceTiles + (tile)) * 4 + (ev)] = (long long)globaltimer_ns(); \
     } while (0)
+#define LA_TRACE_NS1(role, tile, ev)                                                                            \
+    do {                                                                                                        \
+        if (a.trace)                                                                                            \
+            a.trace[(((size_t)blockIdx.x * 4 + (role)) * kTraceTiles + (tile)) * 4 + (ev)] = (long long)globaltimer_ns(); \
+    } while (0)
 #else
 #define LA_TRACE(role, tile, ev) do { } while (0)
 #define LA_TRACE_NS(role, tile, ev) do { } while (0)
+#define LA_TRACE_NS1(role, tile, ev) do { } while (0)
 #endif
 
 // Shared-memory descriptor with the address field replaced: descriptors of one operand family differ
@@ -220,7 +310,7 @@ __device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_sme
 
 constexpr int kKStages = 3;   // key side: stages of (K tile, V tile)
 constexpr int kQStages = 5;   // query side: stages of one Q tile (reused for phi(q) and then the output tile)
-constexpr int kThreads = 384; // 12 warps
+constexpr int kThreads = 512; // 16 warps
 
 struct Smem {
     // key side
@@ -293,11 +383,11 @@ __device__ __forceinline__ Cta cta_setup(uint8_t* smem_raw, const Args& a, bool 
             mbar_init(c.bar(K_ACCFREE), 8);
         }
         if (init_q) {
-            for (int i = 0; i < kQStages; ++i) { mbar_init(c.bar(Q_FULL + i), 1); mbar_init(c.bar(Q_EMPTY + i), 1); mbar_init(c.bar(Q_PHIFULL + i), 8); mbar_init(c.bar(Q_OFULL + i), 8); }
-            for (int i = 0; i < 2; ++i) { mbar_init(c.bar(Q_UFULL + i), 1); mbar_init(c.bar(Q_UEMPTY + i), 8); mbar_init(c.bar(Q_DFULL + i), 1); mbar_init(c.bar(Q_DEMPTY + i), 8); }
+            for (int i = 0; i < kQStages; ++i) { mbar_init(c.bar(Q_FULL + i), 1); mbar_init(c.bar(Q_EMPTY + i), 1); mbar_init(c.bar(Q_PHIFULL + i), 8); mbar_init(c.bar(Q_OFULL + i), 4); }
+            for (int i = 0; i < 2; ++i) { mbar_init(c.bar(Q_UFULL + i), 1); mbar_init(c.bar(Q_UEMPTY + i), 8); mbar_init(c.bar(Q_DFULL + i), 1); mbar_init(c.bar(Q_DEMPTY + i), 4); }
             mbar_init(c.bar(Q_SEGFULL), 1);
             mbar_init(c.bar(Q_SEGFREE), 1);
-            mbar_init(c.bar(Q_SREADY), 8);
+            mbar_init(c.bar(Q_SREADY), 4);
             mbar_init(c.bar(Q_WFULL), 1);
         }
         fence_mbar_init();
@@ -592,6 +682,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             if (state_g >= 0 && w.i >= kQStages) load_state();
             if (!ok) break;
             if (w.i >= kQStages && !warp_wait(c.bar(Q_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) break;
+            LA_TRACE(0, 24 + w.i, 0);
             if (lane == 0) {
                 mbar_arrive_expect_tx(c.bar(Q_FULL + r.s), kTileBytes);
                 tma_load_3d(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g);
@@ -611,6 +702,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         for (; !w.done(); w.next(), r.next(), ur.next()) {
             if (w.first() && !warp_wait(c.bar(Q_WFULL), (uint32_t)w.seg & 1u, c.wc, kErrSeg)) break;
             if (!warp_wait(c.bar(Q_FULL + r.s), r.ph, c.wc, kErrMmaLoad)) break;
+            LA_TRACE(1, 24 + w.i, 0);
             if (w.i >= 2 && !warp_wait(c.bar(Q_UEMPTY + ur.s), ur.ph ^ 1u, c.wc, kErrMmaU)) break;
             tcgen05_fence_after();
             if (elect_one()) {
@@ -618,6 +710,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 mma_commit(c.bar(Q_UFULL + ur.s));
             }
             __syncwarp();
+            LA_TRACE(1, 24 + w.i, 1);
         }
     } else if (warp == 10) {
         // ---------------- numerator / denominator MMA issuer: num = phi(q) S, den = phi(q) . z ----------------
@@ -631,6 +724,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             if (w.first() && !warp_wait(c.bar(Q_SEGFULL), (uint32_t)w.seg & 1u, c.wc, kErrSeg)) break;
             if (!warp_wait(c.bar(Q_PHIFULL + r.s), r.ph, c.wc, kErrMmaPhi)) break;
             if (w.i >= 2 && !warp_wait(c.bar(Q_DEMPTY + dr.s), dr.ph ^ 1u, c.wc, kErrMmaAcc)) break;
+            LA_TRACE(1, 24 + w.i, 2);
             tcgen05_fence_after();
             if (elect_one()) {
                 const uint32_t phi = sbase + r.s * kTileBytes;
@@ -646,77 +740,101 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 if (w.last()) mma_commit(c.bar(Q_SEGFREE));   // this head's S, z and W may now be replaced
             }
             __syncwarp();
+            LA_TRACE(1, 24 + w.i, 3);
         }
     } else if (warp == 11) {
         // ---------------- TMA stores of finished output tiles ----------------
+        // Two stores may be in flight: after issuing tile j's store the warp waits only until tile j-1's
+        // store has read its slot, then hands that slot back to the producer.
         if (lane == 0) tma_prefetch_desc(tmO);
         Ring<kQStages> r;
+        int prev_slot = -1;
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(Q_OFULL + r.s), r.ph, c.wc, kErrStore)) break;
             if (lane == 0) {
                 tma_store_3d(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g);
                 tma_store_3d(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g);
                 bulk_commit_group();
-                bulk_wait_group_read<0>();   // the slot has been read out: hand it back to the producer
-                mbar_arrive(c.bar(Q_EMPTY + r.s));
+                bulk_wait_group_read<1>();
+                if (prev_slot >= 0) mbar_arrive(c.bar(Q_EMPTY + prev_slot));
             }
+            prev_slot = r.s;
             __syncwarp();
+            LA_TRACE(0, 24 + w.i, 1);
         }
-        if (lane == 0) bulk_wait_group<0>();
+        if (lane == 0) {
+            bulk_wait_group_read<0>();
+            if (prev_slot >= 0) mbar_arrive(c.bar(Q_EMPTY + prev_slot));
+            bulk_wait_group<0>();
+        }
     } else if (warp < 8) {
-        // ---------------- feature map + epilogue (warps 0-7) ----------------
+        // ---------------- feature map (warps 0-7) ----------------
         const int half = warp >> 2;
         const int row = (warp & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        Ring<kQStages> r, er;   // feature-map ring position, epilogue ring position (one tile behind)
-        Ring<2> ur, dr;
-        for (int i = 0; i <= w.count; ++i) {
-            if (i < w.count) {
-                if (!warp_wait(c.bar(Q_UFULL + ur.s), ur.ph, c.wc, kErrSoftmaxU)) break;
-                tcgen05_fence_after();
-                float u[kM];
-                load_logits(tmem_u + lane_base + ur.s * kM, u);
-                tcgen05_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(c.bar(Q_UEMPTY + ur.s));
-                uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
-                if (half == 0) softmax_half_to_smem<false>(u, 1.f, dst, row);
-                else softmax_half_to_smem<true>(u, 1.f, dst, row);
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(c.bar(Q_PHIFULL + r.s));
-                r.next();
-                ur.next();
-            }
-            if (i >= 1) {
-                if (!warp_wait(c.bar(Q_DFULL + dr.s), dr.ph, c.wc, kErrEpilogue)) break;
-                tcgen05_fence_after();
-                uint32_t v[64], dv[2];
+        Ring<kQStages> r;
+        Ring<2> ur;
+        for (; !w.done(); w.next(), r.next(), ur.next()) {
+            if (!warp_wait(c.bar(Q_UFULL + ur.s), ur.ph, c.wc, kErrSoftmaxU)) break;
+            if (warp == 0) LA_TRACE(2, 24 + w.i, 0);
+            tcgen05_fence_after();
+            float u[kM];
+            load_logits(tmem_u + lane_base + ur.s * kM, u);
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c.bar(Q_UEMPTY + ur.s));
+            uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
+            if (half == 0) softmax_half_to_smem<false>(u, 1.f, dst, row);
+            else softmax_half_to_smem<true>(u, 1.f, dst, row);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c.bar(Q_PHIFULL + r.s));
+            if (warp == 0) LA_TRACE(2, 24 + w.i, 1);
+        }
+    } else if (warp >= 12) {
+        // ---------------- epilogue (warps 12-15): o = num / den, bf16, into the tile's slot ----------------
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const int sw = row & 7;
+        Ring<kQStages> r;
+        Ring<2> dr;
+        for (; !w.done(); w.next(), r.next(), dr.next()) {
+            if (!warp_wait(c.bar(Q_DFULL + dr.s), dr.ph, c.wc, kErrEpilogue)) break;
+            if (warp == 12) LA_TRACE(3, 24 + w.i, 0);
+            tcgen05_fence_after();
+            uint32_t dv[2];
+            tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t v[64];
                 tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64, v);
                 tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64 + 32, v + 32);
-                tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
                 tmem_wait_ld();
-                tcgen05_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(c.bar(Q_DEMPTY + dr.s));
+                if (half == 1) {
+                    // everything this tile needs from TMEM is in registers: release the accumulator
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(c.bar(Q_DEMPTY + dr.s));
+                }
                 const float inv = __fdividef(1.f, __uint_as_float(dv[0]) + __uint_as_float(dv[1]));
-                uint8_t* dst = c.smem + er.s * kTileBytes + half * kHalfTileBytes + row * 128;
-                const int sw = row & 7;
+                const f32x2 inv2 = pack2(inv, inv);
+                uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
 #pragma unroll
                 for (int cc = 0; cc < 8; ++cc) {
-                    uint4 o;
-                    o.x = pack_bf16(__uint_as_float(v[8 * cc + 0]) * inv, __uint_as_float(v[8 * cc + 1]) * inv);
-                    o.y = pack_bf16(__uint_as_float(v[8 * cc + 2]) * inv, __uint_as_float(v[8 * cc + 3]) * inv);
-                    o.z = pack_bf16(__uint_as_float(v[8 * cc + 4]) * inv, __uint_as_float(v[8 * cc + 5]) * inv);
-                    o.w = pack_bf16(__uint_as_float(v[8 * cc + 6]) * inv, __uint_as_float(v[8 * cc + 7]) * inv);
-                    *reinterpret_cast<uint4*>(dst + ((cc ^ sw) << 4)) = o;
+                    uint32_t o[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float x, y;
+                        unpack2(mul2(pack2(__uint_as_float(v[8 * cc + 2 * q]), __uint_as_float(v[8 * cc + 2 * q + 1])), inv2), x, y);
+                        o[q] = pack_bf16(x, y);
+                    }
+                    *reinterpret_cast<uint4*>(dst + ((cc ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(c.bar(Q_OFULL + er.s));
-                er.next();
-                dr.next();
             }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c.bar(Q_OFULL + r.s));
+            if (warp == 12) LA_TRACE(3, 24 + w.i, 1);
         }
     }
 }
@@ -791,37 +909,38 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __syncthreads();
     tcgen05_fence_after();
     LA_TRACE_NS(0, 60, 2);
-    if (c.warp < 8) {
-        // warps 0-7: grid barrier, combine (spread over all CTAs), grid barrier, then release the query side.
-        // The other warps go straight on: Q tiles, W_q and the first logits do not depend on S.
+    if (c.warp >= 12) {
+        // warps 12-15: grid barrier, combine (spread over all CTAs), grid barrier, then release the query side.
+        // The other warps go straight on: Q tiles, W_q, the first logits and feature maps do not depend on S.
         __shared__ uint32_t gb_ok;
         const uint32_t P = gridDim.x;
-        if (threadIdx.x == 0) {
+        const int it = threadIdx.x - 12 * 32;   // 0..127
+        if (it == 0) {
             gb_ok = grid_barrier(a.sync, P) ? 1u : 0u;
             if (!gb_ok) {
                 atomicOr(a.err, (uint32_t)kErrGrid);
                 asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
             }
         }
-        named_barrier_sync(1, 256);
-        LA_TRACE_NS(0, 60, 3);
+        named_barrier_sync(1, 128);
+        if (it == 0) LA_TRACE_NS1(0, 60, 3);
         if (gb_ok) {
             const int total = a.G * (kE / 4);   // float4 groups over all heads
-            for (int x = blockIdx.x * 256 + threadIdx.x; x < total; x += (int)P * 256)
+            for (int x = blockIdx.x * 128 + it; x < total; x += (int)P * 128)
                 combine_quad(a, P, x / (kE / 4), (x % (kE / 4)) * 4);
         }
-        named_barrier_sync(1, 256);
-        LA_TRACE_NS(0, 61, 0);
-        if (threadIdx.x == 0 && gb_ok) {
+        named_barrier_sync(1, 128);
+        if (it == 0) LA_TRACE_NS1(0, 61, 0);
+        if (it == 0 && gb_ok) {
             if (!grid_barrier(a.sync, P)) {
                 gb_ok = 0u;
                 atomicOr(a.err, (uint32_t)kErrGrid);
                 asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
             }
         }
-        named_barrier_sync(1, 256);
+        named_barrier_sync(1, 128);
         if (c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
-        LA_TRACE_NS(0, 61, 1);
+        if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
     qside_phase(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
     LA_TRACE_NS(0, 61, 2);
