@@ -44,8 +44,6 @@ typedef enum {
     LINATTN_OPT_PATH = 1,   /* 0 = automatic (default), 1 = CUDA-core kernels, 2 = tensor-core (tcgen05 + TMA) kernels */
     LINATTN_OPT_FUSE = 3,   /* tensor-core path: 1 = one cooperative kernel for the whole forward (default, used when the
                                device allows it), 0 = three launches (key side, combine, query side) */
-    LINATTN_OPT_WAVES = 4,  /* fused kernel: 0 = automatic (default), 1 = all heads in one wave, 2 = two waves of heads
-                               (the query side of the first wave streams while the second wave is being combined) */
     LINATTN_OPT_PROFILE = 2 /* 1 = record CUDA events around every kernel of each forward (see linattn_profile_get);
                                switching it on clears the accumulated figures; 0 = off (default) */
 } linattn_option;

@@ -12,7 +12,6 @@
 
 #include "simt_kernels.cuh"
 #include "sm100_kernels.cuh"
-#include "sm100_stream.cuh"
 #include "tensor_map.hpp"
 
 using namespace linattn;
@@ -53,9 +52,7 @@ struct linattn_ctx {
     __nv_bfloat16* z_img = nullptr;  // [max_B*H][2048] bf16 operand image of z (hi, lo)
     int num_sms = 0;
     bool coop_ok = false;            // device supports cooperative launches
-    uint32_t* sync_words = nullptr;  // [0..1] unused, [2..5] wave counters of the fused kernel (monotonic)
-    uint32_t kdone_total[2] = {0, 0};  // values the wave counters have after the launches enqueued so far
-    uint32_t cdone_total[2] = {0, 0};
+    uint32_t* sync_words = nullptr;  // grid-barrier counter and generation of the fused kernel
     // workspace
     float* partial = nullptr;   // [partial_slots][d*d + d]
     long long partial_slots = 0;
@@ -68,7 +65,6 @@ struct linattn_ctx {
     int opt_splits = 0;
     int opt_path = 0;
     int opt_fuse = 1;
-    int opt_waves = 0;
     // per-kernel timing (LINATTN_OPT_PROFILE)
     static constexpr int kMaxKernels = 4;
     bool profile = false;
@@ -82,7 +78,6 @@ struct linattn_ctx {
     // bookkeeping
     int last_launches = 0;
     int last_B = 0;
-    bool state_transposed = false;  // the last forward left S in the workspace as [c][f] (fused kernel) rather than [f][c]
     char err_text[256] = {0};
 #ifdef LINATTN_TRACE
     long long* trace = nullptr;  // tuning builds only: device buffer for per-tile timestamps
@@ -229,7 +224,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     if (!attr_done) {
         LA_CUDA(c, cudaFuncSetAttribute(kside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
         LA_CUDA(c, cudaFuncSetAttribute(qside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(linattn_stream_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmemStream::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(linattn_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
         attr_done = true;
     }
     const double side_bytes = 2.0 * (double)G * n * kD * 2;
@@ -250,41 +245,12 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
 #endif
     prof_begin(c, st);
     if (c->opt_fuse && c->coop_ok && Pk == Pq) {
-        // one cooperative launch for the whole forward; heads go in two waves when there is enough work per CTA
-        int waves = c->opt_waves;
-        if (waves == 0) waves = (G >= 2 && T >= 16 * Pq) ? 2 : 1;
-        if (waves == 2 && G < 2) waves = 1;
-        const long long gsplit = waves == 2 ? G / 2 : G;
-        // every CTA gets at least one tile of every wave (the combine step relies on it)
-        const long long Pf = Pq < gsplit * Tn ? Pq : gsplit * Tn;
-        if (2 * Pf + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
-        StreamArgs sa{};
-        sa.partial = c->partial;
-        sa.state = c->state;
-        sa.s_img = c->s_img;
-        sa.err = c->err_word;
-        sa.cnt = c->sync_words + 2;
-        sa.n = n;
-        sa.H = c->H;
-        sa.G = (int)G;
-        sa.tph = (int)Tn;
-        sa.waves = waves;
-        sa.gsplit = (int)gsplit;
-        for (int wv = 0; wv < waves; ++wv) {
-            c->kdone_total[wv] += 4u * (uint32_t)Pf;
-            c->cdone_total[wv] += 4u * (uint32_t)Pf;
-            sa.kdone_target[wv] = c->kdone_total[wv];
-            sa.cdone_target[wv] = c->cdone_total[wv];
-        }
-#ifdef LINATTN_TRACE
-        sa.trace = c->trace;
-#endif
-        void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &sa};
-        LA_CUDA(c, cudaLaunchCooperativeKernel((const void*)linattn_stream_tc, dim3((unsigned)Pf), dim3(kThreads), params,
-                                               SmemStream::kTotal, st));
-        prof_mark(c, st, "linattn_stream_tc", 2.0 * side_bytes);
+        // one cooperative launch: key side, grid barrier, combine, grid barrier, query side
+        void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &a};
+        LA_CUDA(c, cudaLaunchCooperativeKernel((const void*)linattn_fused_tc, dim3((unsigned)Pq), dim3(kThreads), params,
+                                               Smem::kTotal, st));
+        prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
         c->last_launches = 1;
-        c->state_transposed = true;
         return LINATTN_OK;
     }
     kside_tc<<<(unsigned)Pk, kThreads, Smem::kTotal, st>>>(tmK, tmV, tmWk, a);
@@ -365,14 +331,11 @@ linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, l
     const size_t E = (size_t)d * d + d;
     const size_t wbytes = sizeof(float) * (size_t)H * d * (d / 2);
     const long long G = max_B * H;
-    cudaError_t e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
-    // partial records: the CUDA-core path uses up to kTargetCtas + G of E floats, the fused tensor-core kernel
-    // up to 2 * #SMs + G of tc::kRec floats (two waves of heads)
-    c->partial_slots = (kTargetCtas > 2 * c->num_sms ? kTargetCtas : 2 * c->num_sms) + G;
-    const size_t rec_floats = d == 128 ? (size_t)linattn::tc::kRec : E;
+    c->partial_slots = kTargetCtas + G;
+    cudaError_t e = cudaSuccess;
     if (e == cudaSuccess) e = cudaMalloc(&c->Wq, wbytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->Wk, wbytes);
-    if (e == cudaSuccess) e = cudaMalloc(&c->partial, sizeof(float) * rec_floats * (size_t)c->partial_slots);
+    if (e == cudaSuccess) e = cudaMalloc(&c->partial, sizeof(float) * E * (size_t)c->partial_slots);
     if (e == cudaSuccess) e = cudaMalloc(&c->state, sizeof(float) * E * (size_t)G);
     if (e == cudaSuccess && d == 128) {
         const size_t wt = sizeof(__nv_bfloat16) * (size_t)H * d * (d / 2);
@@ -382,13 +345,14 @@ linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, l
         if (e == cudaSuccess) e = cudaMalloc(&c->z_img, (size_t)G * linattn::tc::kZBlkBytes);
         if (e == cudaSuccess) e = cudaMemset(c->z_img, 0, (size_t)G * linattn::tc::kZBlkBytes);
     }
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) {
         int coop = 0;
         e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device);
         c->coop_ok = (coop != 0);
     }
-    if (e == cudaSuccess) e = cudaMalloc(&c->sync_words, 8 * sizeof(uint32_t));
-    if (e == cudaSuccess) e = cudaMemset(c->sync_words, 0, 8 * sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&c->sync_words, 2 * sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMemset(c->sync_words, 0, 2 * sizeof(uint32_t));
     if (e == cudaSuccess) e = cudaMalloc(&c->err_word, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->err_word, 0, sizeof(unsigned int));
     if (e != cudaSuccess) {
@@ -471,7 +435,6 @@ linattn_status linattn_forward(linattn_ctx* c, const void* q, const void* k, con
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     c->last_B = B;
-    c->state_transposed = false;
     if (tc_ok && c->opt_path != 1) return launch_tc(c, q, k, v, out, B, n, st);
     if (dtype == LINATTN_BF16) {
         return d == 128 ? launch_simt<__nv_bfloat16, 128>(c, q, k, v, out, B, n, st)
@@ -523,19 +486,6 @@ linattn_status linattn_read_state(linattn_ctx* c, float* S_host, float* z_host, 
         LA_CUDA(c, cudaMemcpy2DAsync(z_host, c->d * sizeof(float), c->state + dd, E * sizeof(float),
                                      c->d * sizeof(float), G, cudaMemcpyDeviceToHost, st));
     LA_CUDA(c, cudaStreamSynchronize(st));
-    if (S_host && c->state_transposed) {
-        // the fused kernel keeps S as [c][f]; the documented layout is [f][c]
-        const int d = c->d;
-        for (size_t g = 0; g < G; ++g) {
-            float* m = S_host + g * dd;
-            for (int i = 0; i < d; ++i)
-                for (int j = i + 1; j < d; ++j) {
-                    const float t = m[(size_t)i * d + j];
-                    m[(size_t)i * d + j] = m[(size_t)j * d + i];
-                    m[(size_t)j * d + i] = t;
-                }
-        }
-    }
     return LINATTN_OK;
 }
 
@@ -554,10 +504,6 @@ linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long 
         case LINATTN_OPT_FUSE:
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
             c->opt_fuse = (int)value;
-            return LINATTN_OK;
-        case LINATTN_OPT_WAVES:
-            if (value < 0 || value > 2) return LINATTN_ERR_INVALID_ARG;
-            c->opt_waves = (int)value;
             return LINATTN_OK;
         case LINATTN_OPT_PROFILE: {
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
@@ -592,8 +538,7 @@ linattn_status linattn_check(linattn_ctx* c, void* stream)
     LA_CUDA(c, cudaStreamSynchronize(st));
     if (w != 0) {
         LA_CUDA(c, cudaMemsetAsync(c->err_word, 0, sizeof(w), st));
-        LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, 8 * sizeof(uint32_t), st));  // an aborted launch leaves the wave counters short
-        c->kdone_total[0] = c->kdone_total[1] = c->cdone_total[0] = c->cdone_total[1] = 0;
+        LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, 2 * sizeof(uint32_t), st));  // an aborted grid barrier leaves them inconsistent
         snprintf(c->err_text, sizeof(c->err_text), "device-side wait gave up (code 0x%x)", w);
         return LINATTN_ERR_TIMEOUT;
     }

@@ -110,8 +110,7 @@ struct WaitCtx {
 };
 
 // All lanes wait (bounded); the verdict is made warp-uniform so that role loops never diverge.
-// Out of line: the kernels wait in dozens of places and their code has to stay within the instruction cache.
-__device__ __noinline__ bool warp_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc, uint32_t code)
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc, uint32_t code)
 {
     const bool ok = mbar_wait_abortable(bar, parity, kWaitLimitNs, wc.abort_smem);
     const bool all = __all_sync(0xffffffffu, ok);

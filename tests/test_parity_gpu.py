@@ -15,11 +15,10 @@ from util import assert_parity, errors, run_gpu
 
 pytestmark = pytest.mark.gpu
 
-# (path option, fuse option, waves option): automatic choice (one fused tensor-core kernel where it applies,
-# heads in one wave at these sizes), the fused kernel forced to two waves of heads, the tensor-core kernels as
-# three launches, and the CUDA-core kernels
-MODES = [(linattn.PATH_AUTO, 1, 0), (linattn.PATH_AUTO, 1, 2), (linattn.PATH_AUTO, 0, 0), (linattn.PATH_SIMT, 0, 0)]
-MODE_IDS = ["auto", "twowaves", "unfused", "simt"]
+# (path option, fuse option): automatic choice (one fused tensor-core kernel where it applies), the
+# tensor-core kernels as three launches, and the CUDA-core kernels
+MODES = [(linattn.PATH_AUTO, 1), (linattn.PATH_AUTO, 0), (linattn.PATH_SIMT, 0)]
+MODE_IDS = ["auto", "unfused", "simt"]
 
 
 def mode_param():
@@ -27,7 +26,7 @@ def mode_param():
 
 
 def run_mode(x, mode, **kw):
-    return run_gpu(x, path=mode[0], fuse=mode[1], waves=mode[2], **kw)
+    return run_gpu(x, path=mode[0], fuse=mode[1], **kw)
 
 
 def small_inputs(B, H, n, d, dtype, seed, wmode="random"):
@@ -132,7 +131,6 @@ def test_bit_identical_across_runs_and_context_reuse(mode):
     try:
         ctx.set_option(linattn.OPT_PATH, mode[0])
         ctx.set_option(linattn.OPT_FUSE, mode[1])
-        ctx.set_option(linattn.OPT_WAVES, mode[2])
         ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
         q, k, v = x["q"].cuda(), x["k"].cuda(), x["v"].cuda()
         first = ctx.forward(q, k, v).clone()
@@ -163,7 +161,6 @@ def test_output_guard_bands_are_untouched():
         for mode in MODES:
             ctx.set_option(linattn.OPT_PATH, mode[0])
             ctx.set_option(linattn.OPT_FUSE, mode[1])
-            ctx.set_option(linattn.OPT_WAVES, mode[2])
             ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
             ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda(), out=out)
             ctx.check()
@@ -207,7 +204,7 @@ def test_which_kernels_run():
             ctx.set_option(linattn.OPT_PROFILE, 0)
             return got, ctx.last_launch_count()
 
-        assert names(linattn.PATH_AUTO, 1) == (["linattn_stream_tc"], 1)
+        assert names(linattn.PATH_AUTO, 1) == (["linattn_fused_tc"], 1)
         assert names(linattn.PATH_TENSOR, 0) == (["kside_tc", "combine_tc", "qside_tc"], 3)
         assert names(linattn.PATH_SIMT, 1) == (["kside_simt", "combine_state", "qside_simt"], 3)
         ctx.check()

@@ -22,7 +22,7 @@ def assert_parity(got, want, what=""):
     return rel, mx
 
 
-def run_gpu(x, path=0, splits=0, ctx=None, return_state=False, fuse=1, waves=0):
+def run_gpu(x, path=0, splits=0, ctx=None, return_state=False, fuse=1):
     """Run the CUDA library on the CPU tensors of `x` (q, k, v, Wq, Wk); returns a CPU float64 array."""
     from paper_2510_08318_b200 import linattn
     q = x["q"]
@@ -34,7 +34,6 @@ def run_gpu(x, path=0, splits=0, ctx=None, return_state=False, fuse=1, waves=0):
         ctx.set_option(linattn.OPT_PATH, path)
         ctx.set_option(linattn.OPT_SPLITS, splits)
         ctx.set_option(linattn.OPT_FUSE, fuse)
-        ctx.set_option(linattn.OPT_WAVES, waves)
         ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
         out = ctx.forward(q.cuda(), x["k"].cuda(), x["v"].cuda())
         ctx.check()
