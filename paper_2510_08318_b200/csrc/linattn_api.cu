@@ -78,6 +78,7 @@ struct linattn_ctx {
     // bookkeeping
     int last_launches = 0;
     int last_B = 0;
+    bool state_transposed = false;  // the last forward left S in the workspace as [c][f] (tensor-core kernels) rather than [f][c]
     char err_text[256] = {0};
 #ifdef LINATTN_TRACE
     long long* trace = nullptr;  // tuning builds only: device buffer for per-tile timestamps
@@ -435,7 +436,8 @@ linattn_status linattn_forward(linattn_ctx* c, const void* q, const void* k, con
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     c->last_B = B;
-    if (tc_ok && c->opt_path != 1) return launch_tc(c, q, k, v, out, B, n, st);
+    c->state_transposed = tc_ok && c->opt_path != 1;
+    if (c->state_transposed) return launch_tc(c, q, k, v, out, B, n, st);
     if (dtype == LINATTN_BF16) {
         return d == 128 ? launch_simt<__nv_bfloat16, 128>(c, q, k, v, out, B, n, st)
                         : launch_simt<__nv_bfloat16, 64>(c, q, k, v, out, B, n, st);
@@ -486,6 +488,19 @@ linattn_status linattn_read_state(linattn_ctx* c, float* S_host, float* z_host, 
         LA_CUDA(c, cudaMemcpy2DAsync(z_host, c->d * sizeof(float), c->state + dd, E * sizeof(float),
                                      c->d * sizeof(float), G, cudaMemcpyDeviceToHost, st));
     LA_CUDA(c, cudaStreamSynchronize(st));
+    if (S_host && c->state_transposed) {
+        // the tensor-core kernels keep S as [c][f]; the documented layout is [f][c]
+        const int d = c->d;
+        for (size_t g = 0; g < G; ++g) {
+            float* m = S_host + g * dd;
+            for (int i = 0; i < d; ++i)
+                for (int j = i + 1; j < d; ++j) {
+                    const float t = m[(size_t)i * d + j];
+                    m[(size_t)i * d + j] = m[(size_t)j * d + i];
+                    m[(size_t)j * d + i] = t;
+                }
+        }
+    }
     return LINATTN_OK;
 }
 

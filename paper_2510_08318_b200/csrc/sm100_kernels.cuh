@@ -330,11 +330,11 @@ struct Smem {
 // mbarrier indices
 enum : int {
     // key side
-    K_FULL = 0, K_EMPTY = 3, K_UFULL = 6, K_UEMPTY = 8, K_PHIFULL = 10, K_WFULL = 13, K_WFREE = 15, K_ACCFULL = 17, K_ACCFREE = 18,
+    K_FULL = 0, K_EMPTY = 3, K_UFULL = 6, K_UEMPTY = 8, K_PHIFULL = 10, K_WFULL = 13, K_WFREE = 15, K_ACCFULL = 17, K_ACCFREE = 19,
     // query side
-    Q_FULL = 19, Q_EMPTY = 24, Q_PHIFULL = 29, Q_OFULL = 34, Q_UFULL = 39, Q_UEMPTY = 41, Q_DFULL = 43, Q_DEMPTY = 45,
-    Q_SEGFULL = 47, Q_SEGFREE = 48, Q_SREADY = 49, Q_WFULL = 50,
-    NBARS = 51
+    Q_FULL = 21, Q_EMPTY = 26, Q_PHIFULL = 31, Q_OFULL = 36, Q_UFULL = 41, Q_UEMPTY = 43, Q_DFULL = 45, Q_DEMPTY = 47,
+    Q_SEGFULL = 49, Q_SEGFREE = 50, Q_SREADY = 51, Q_WFULL = 52,
+    NBARS = 53
 };
 
 struct Cta {
@@ -346,9 +346,9 @@ struct Cta {
 };
 
 struct Args {
-    float* partial;              // [slots][kE] partial (S, z) records, slot = cta + g
-    float* state;                // [G][kE] combined S, z (fp32)
-    __nv_bfloat16* s_img;        // [G][128][128] bf16 image of S
+    float* partial;              // [slots][kE] partial (S, z) records, slot = cta + g; S as [c][f] (c = column of V, f = feature)
+    float* state;                // [G][kE] combined S, z (fp32), same layout
+    __nv_bfloat16* s_img;        // [G][128][128] bf16 image of S, [c][f]
     __nv_bfloat16* z_img;        // [G][kZBlkBytes / 2] bf16 operand image of z (hi, lo)
     uint32_t* err;               // error word
     uint32_t* sync;              // [0] grid-barrier arrival counter, [1] generation (fused kernel only)
@@ -379,8 +379,7 @@ __device__ __forceinline__ Cta cta_setup(uint8_t* smem_raw, const Args& a, bool 
         if (init_k) {
             for (int i = 0; i < kKStages; ++i) { mbar_init(c.bar(K_FULL + i), 1); mbar_init(c.bar(K_EMPTY + i), 1); mbar_init(c.bar(K_PHIFULL + i), 8); }
             for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_UFULL + i), 1); mbar_init(c.bar(K_UEMPTY + i), 8); mbar_init(c.bar(K_WFULL + i), 1); mbar_init(c.bar(K_WFREE + i), 1); }
-            mbar_init(c.bar(K_ACCFULL), 1);
-            mbar_init(c.bar(K_ACCFREE), 8);
+            for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_ACCFULL + i), 1); mbar_init(c.bar(K_ACCFREE + i), 4); }
         }
         if (init_q) {
             for (int i = 0; i < kQStages; ++i) { mbar_init(c.bar(Q_FULL + i), 1); mbar_init(c.bar(Q_EMPTY + i), 1); mbar_init(c.bar(Q_PHIFULL + i), 8); mbar_init(c.bar(Q_OFULL + i), 4); }
@@ -421,8 +420,9 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
                                             const CUtensorMap* tmW)
 {
     const uint32_t tmem_u = c.tmem;            // 2 x 64 columns of logits
-    const uint32_t tmem_s = c.tmem + 128;      // 128 columns: S[f][c], lane = f
-    const uint32_t tmem_z = c.tmem + 256;      // 16 columns: z[f] (all 16 equal)
+    // two accumulator sets, alternating by segment, so that one drains while the next accumulates
+    auto tmem_s = [&](int b) { return c.tmem + 128 + b * 144; };   // 128 columns: S[f][c], lane = f
+    auto tmem_z = [&](int b) { return c.tmem + 256 + b * 144; };   // 16 columns: z[f] (all 16 equal)
     const int warp = c.warp, lane = c.lane;
     const uint32_t sbase = c.sbase;
     TileWalk w;
@@ -495,7 +495,8 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             if (!warp_wait(c.bar(K_PHIFULL + r.s), r.ph, c.wc, kErrMmaPhi)) break;
             LA_TRACE(1, w.i, 2);
             const bool first = w.first();
-            if (first && w.seg >= 1 && !warp_wait(c.bar(K_ACCFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrMmaAcc)) break;
+            const int b = w.seg & 1;
+            if (first && w.seg >= 2 && !warp_wait(c.bar(K_ACCFREE + b), (uint32_t)((w.seg >> 1) - 1) & 1u, c.wc, kErrMmaAcc)) break;
             tcgen05_fence_after();
             if (elect_one()) {
                 const uint32_t phi = sbase + r.s * Smem::kKStage, vt = phi + kTileBytes;
@@ -504,11 +505,11 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
                     const uint64_t da = desc_at(mnmajor, phi + k * 2048);
                     const uint64_t db = desc_at(mnmajor, vt + k * 2048);
                     const uint32_t acc = (first && k == 0) ? 0u : 1u;
-                    mma_bf16_ss(tmem_s, da, db, idesc_s, acc);
-                    mma_bf16_ss(tmem_z, da, ones_desc, idesc_z, acc);
+                    mma_bf16_ss(tmem_s(b), da, db, idesc_s, acc);
+                    mma_bf16_ss(tmem_z(b), da, ones_desc, idesc_z, acc);
                 }
                 mma_commit(c.bar(K_EMPTY + r.s));
-                if (w.last()) mma_commit(c.bar(K_ACCFULL));
+                if (w.last()) mma_commit(c.bar(K_ACCFULL + b));
             }
             __syncwarp();
             LA_TRACE(1, w.i, 3);
@@ -538,31 +539,35 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             __syncwarp();
             if (lane == 0) mbar_arrive(c.bar(K_PHIFULL + r.s));
             if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 2);
-            if (w.last()) {
-                // drain the accumulators of this segment: thread = feature f, this half's 64 columns of S
-                if (!warp_wait(c.bar(K_ACCFULL), (uint32_t)w.seg & 1u, c.wc, kErrDrain)) break;
-                tcgen05_fence_after();
-                float* rec = a.partial + (size_t)(blockIdx.x + w.g) * kE;
-                float* srow = rec + (size_t)row * kD + half * 64;
+        }
+    } else if (warp >= 12) {
+        // ---------------- drain (warps 12-15): at the end of a segment the accumulators go to the partial record ---
+        // thread = feature f = TMEM lane.  The record holds S as [c][f] (c = column of V), so that the 32 lanes
+        // of a warp write 128 contiguous bytes per column; z follows.
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        for (; !w.done(); w.next()) {
+            if (!w.last()) continue;
+            const int b = w.seg & 1;
+            if (!warp_wait(c.bar(K_ACCFULL + b), (uint32_t)(w.seg >> 1) & 1u, c.wc, kErrDrain)) break;
+            tcgen05_fence_after();
+            float* rec = a.partial + (size_t)(blockIdx.x + w.g) * kE;
+            float* scol = rec + row;
 #pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld_x32(tmem_s + lane_base + half * 64 + c0, v);
-                    tmem_wait_ld();
+            for (int c0 = 0; c0 < kD; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_x32(tmem_s(b) + lane_base + c0, v);
+                tmem_wait_ld();
 #pragma unroll
-                    for (int q4 = 0; q4 < 8; ++q4)
-                        *reinterpret_cast<uint4*>(srow + c0 + 4 * q4) = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
-                }
-                if (half == 0) {
-                    uint32_t zr[2];
-                    tmem_ld_x2(tmem_z + lane_base, zr);
-                    tmem_wait_ld();
-                    rec[kD * kD + row] = __uint_as_float(zr[0]);
-                }
-                tcgen05_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(c.bar(K_ACCFREE));
+                for (int j = 0; j < 32; ++j) scol[(size_t)(c0 + j) * kD] = __uint_as_float(v[j]);
             }
+            uint32_t zr[2];
+            tmem_ld_x2(tmem_z(b) + lane_base, zr);
+            tmem_wait_ld();
+            rec[kD * kD + row] = __uint_as_float(zr[0]);
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c.bar(K_ACCFREE + b));
         }
     }
 }
@@ -714,7 +719,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         }
     } else if (warp == 10) {
         // ---------------- numerator / denominator MMA issuer: num = phi(q) S, den = phi(q) . z ----------------
-        constexpr uint32_t idesc_n = make_idesc_bf16(kTile, kD, 0, 1);   // A = phi(q) (K-major), B = S (MN-major)
+        constexpr uint32_t idesc_n = make_idesc_bf16(kTile, kD, 0, 0);   // A = phi(q) (K-major), B = S image [c][f] (K-major)
         constexpr uint32_t idesc_d = make_idesc_bf16(kTile, 16, 0, 0);   // B = z operand (K-major)
         const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
         const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
@@ -731,7 +736,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) {
                     const uint64_t da = desc_at(kmajor, phi + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
-                    const uint64_t db_s = desc_at(mnmajor, sbase + Smem::kQS + k * 2048);
+                    const uint64_t db_s = desc_at(kmajor, sbase + Smem::kQS + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
                     const uint64_t db_z = desc_at(kmajor, sbase + Smem::kQZ + (k >> 2) * 2048 + (k & 3) * 32);
                     mma_bf16_ss(tmem_num(dr.s), da, db_s, idesc_n, k > 0);
                     mma_bf16_ss(tmem_den(dr.s), da, db_z, idesc_d, k > 0);
