@@ -52,7 +52,8 @@ struct linattn_ctx {
     __nv_bfloat16* z_img = nullptr;  // [max_B*H][2048] bf16 operand image of z (hi, lo)
     int num_sms = 0;
     bool coop_ok = false;            // device supports cooperative launches
-    uint32_t* sync_words = nullptr;  // grid-barrier counter and generation of the fused kernel
+    uint32_t* sync_words = nullptr;  // grid-barrier arrival counter of the fused kernel (only ever grows)
+    uint32_t bar_total = 0;          // its value after the launches enqueued so far
     // workspace
     float* partial = nullptr;   // [partial_slots][d*d + d]
     long long partial_slots = 0;
@@ -247,6 +248,9 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     prof_begin(c, st);
     if (c->opt_fuse && c->coop_ok && Pk == Pq) {
         // one cooperative launch: key side, grid barrier, combine, grid barrier, query side
+        a.bar_target[0] = c->bar_total + (uint32_t)Pq;
+        a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
+        c->bar_total += 2u * (uint32_t)Pq;
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &a};
         LA_CUDA(c, cudaLaunchCooperativeKernel((const void*)linattn_fused_tc, dim3((unsigned)Pq), dim3(kThreads), params,
                                                Smem::kTotal, st));
@@ -553,7 +557,8 @@ linattn_status linattn_check(linattn_ctx* c, void* stream)
     LA_CUDA(c, cudaStreamSynchronize(st));
     if (w != 0) {
         LA_CUDA(c, cudaMemsetAsync(c->err_word, 0, sizeof(w), st));
-        LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, 2 * sizeof(uint32_t), st));  // an aborted grid barrier leaves them inconsistent
+        LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, 2 * sizeof(uint32_t), st));  // an aborted launch leaves the counter short
+        c->bar_total = 0;
         snprintf(c->err_text, sizeof(c->err_text), "device-side wait gave up (code 0x%x)", w);
         return LINATTN_ERR_TIMEOUT;
     }

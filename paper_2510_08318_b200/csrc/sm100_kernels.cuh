@@ -351,7 +351,8 @@ struct Args {
     __nv_bfloat16* s_img;        // [G][128][128] bf16 image of S, [c][f]
     __nv_bfloat16* z_img;        // [G][kZBlkBytes / 2] bf16 operand image of z (hi, lo)
     uint32_t* err;               // error word
-    uint32_t* sync;              // [0] grid-barrier arrival counter, [1] generation (fused kernel only)
+    uint32_t* sync;              // grid-barrier arrival counter of the fused kernel (monotonic over launches)
+    uint32_t bar_target[2];      // its value once every CTA has arrived at the first / second barrier of this launch
     int n, H, G;
     int tiles_per_head;
     long long total_tiles;
@@ -876,22 +877,17 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
 }
 
 // Grid-wide barrier for a cooperative launch (all CTAs resident).  Called by ONE thread per CTA after a
-// CTA-level barrier.  sync[0] counts arrivals and wraps to 0 by itself; sync[1] is the generation that the
-// last arriver advances.  The wait is bounded: returns false on time-out.
-__device__ __forceinline__ bool grid_barrier(uint32_t* sync, uint32_t P)
+// CTA-level barrier.  *counter only ever grows (over launches too); `target` is the value it has once all P
+// CTAs have arrived at this barrier, which the host knows when it enqueues the launch.  One fire-and-forget
+// add and a poll: no value has to come back before the wait can start.  Bounded: returns false on time-out.
+__device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target)
 {
-    const uint32_t gen0 = ld_acquire_gpu(sync + 1);
     __threadfence();
-    const uint32_t old = atomicInc(sync, P - 1);
-    if (old == P - 1) {
-        __threadfence();
-        atomicAdd(sync + 1, 1u);
-    } else {
-        const uint64_t t0 = globaltimer_ns();
-        uint32_t spins = 0;
-        while (ld_acquire_gpu(sync + 1) == gen0) {
-            if ((++spins & 63u) == 0u && globaltimer_ns() - t0 > kWaitLimitNs) return false;
-        }
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while ((int32_t)(ld_acquire_gpu(counter) - target) < 0) {
+        if ((++spins & 63u) == 0u && globaltimer_ns() - t0 > kWaitLimitNs) return false;
     }
     __threadfence();
     return true;
@@ -914,37 +910,39 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __syncthreads();
     tcgen05_fence_after();
     LA_TRACE_NS(0, 60, 2);
-    if (c.warp >= 12) {
-        // warps 12-15: grid barrier, combine (spread over all CTAs), grid barrier, then release the query side.
-        // The other warps go straight on: Q tiles, W_q, the first logits and feature maps do not depend on S.
+    constexpr int kHoleWarp0 = 10, kHoleThreads = (16 - kHoleWarp0) * 32;
+    if (c.warp >= kHoleWarp0) {
+        // warps 10-15 (idle until S exists): grid barrier, combine (spread over all CTAs), grid barrier, then
+        // release the query side.  The other warps go straight on: Q tiles, W_q, the first logits and feature
+        // maps do not depend on S.
         __shared__ uint32_t gb_ok;
         const uint32_t P = gridDim.x;
-        const int it = threadIdx.x - 12 * 32;   // 0..127
+        const int it = threadIdx.x - kHoleWarp0 * 32;
         if (it == 0) {
-            gb_ok = grid_barrier(a.sync, P) ? 1u : 0u;
+            gb_ok = grid_barrier(a.sync, a.bar_target[0]) ? 1u : 0u;
             if (!gb_ok) {
                 atomicOr(a.err, (uint32_t)kErrGrid);
                 asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
             }
         }
-        named_barrier_sync(1, 128);
+        named_barrier_sync(1, kHoleThreads);
         if (it == 0) LA_TRACE_NS1(0, 60, 3);
         if (gb_ok) {
             const int total = a.G * (kE / 4);   // float4 groups over all heads
-            for (int x = blockIdx.x * 128 + it; x < total; x += (int)P * 128)
+            for (int x = blockIdx.x * kHoleThreads + it; x < total; x += (int)P * kHoleThreads)
                 combine_quad(a, P, x / (kE / 4), (x % (kE / 4)) * 4);
         }
-        named_barrier_sync(1, 128);
+        named_barrier_sync(1, kHoleThreads);
         if (it == 0) LA_TRACE_NS1(0, 61, 0);
         if (it == 0 && gb_ok) {
-            if (!grid_barrier(a.sync, P)) {
+            if (!grid_barrier(a.sync, a.bar_target[1])) {
                 gb_ok = 0u;
                 atomicOr(a.err, (uint32_t)kErrGrid);
                 asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
             }
         }
-        named_barrier_sync(1, 128);
-        if (c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
+        named_barrier_sync(1, kHoleThreads);
+        if (c.warp >= 12 && c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
     qside_phase(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
