@@ -311,6 +311,7 @@ __device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_sme
 constexpr int kKStages = 3;   // key side: stages of (K tile, V tile)
 constexpr int kQStages = 5;   // query side: stages of one Q tile (reused for phi(q) and then the output tile)
 constexpr int kThreads = 512; // 16 warps
+constexpr int kQPrefetchL2 = 3;   // fused kernel: Q tiles pulled into L2 while the CTA waits for S (measured: 2-3 best, 6+ slows the combine)
 
 struct Smem {
     // key side
@@ -685,7 +686,32 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 // the first head's state may not exist yet: get the first Q tiles moving before waiting for it
                 if (!(wait_state && w.seg == 0)) load_state();
             }
-            if (state_g >= 0 && w.i >= kQStages) load_state();
+            if (state_g >= 0 && w.i >= kQStages) {
+                if (wait_state && w.seg == 0) {
+                    // The ring is full and S does not exist yet.  Once every CTA has drained its accumulators
+                    // (first grid barrier) HBM has nothing to do until the query side starts: use the time to pull
+                    // the next Q tiles of this run into L2.
+                    bool passed = false;
+                    if (lane == 0) {
+                        const uint64_t t0 = globaltimer_ns();
+                        while (!(passed = (int32_t)(ld_acquire_gpu(a.sync) - a.bar_target[0]) >= 0)) {
+                            __nanosleep(200);
+                            uint32_t ab;
+                            asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(ab) : "r"(c.wc.abort_smem) : "memory");
+                            if (ab != 0u || globaltimer_ns() - t0 > kWaitLimitNs) break;
+                        }
+                        if (passed) {
+                            TileWalk pw = w;
+                            for (int j = 0; j < kQPrefetchL2 && !pw.done(); ++j, pw.next()) {
+                                tma_prefetch_l2_3d(tmQ, 0, pw.lt * kTile, pw.g);
+                                tma_prefetch_l2_3d(tmQ, 64, pw.lt * kTile, pw.g);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                }
+                load_state();
+            }
             if (!ok) break;
             if (w.i >= kQStages && !warp_wait(c.bar(Q_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) break;
             LA_TRACE(0, 24 + w.i, 0);
