@@ -18,6 +18,11 @@
  * ref_linear is the right form.  Their agreement is the identity of Eq. 5 and is
  * one of the pins in the CPU tests.
  *
+ *   Eq. 8   o_i = r^ * softmax-attention_i + (1 - r^) * linear-attention_i,  r^ = clip(r, 0, 1)
+ *
+ * ref_softmax is the first term (Eq. 4 with sim = exp) and ref_mix the blend; both at the
+ * end of the file.
+ *
  * Readings taken where the paper says nothing:
  *   - d is the per-head dimension; one W_q and one W_k per head (or one shared by
  *     all heads when per_head == 0).
@@ -209,5 +214,68 @@ int linattn_ref_linear(const float *q, const float *k, const float *v,
     if (S_out) memcpy(S_out, S_all, (size_t)G * d * d * sizeof(double));
     if (z_out) memcpy(z_out, z_all, (size_t)G * d * sizeof(double));
     free(S_all); free(z_all);
+    return 0;
+}
+
+/*
+ * First term of Eq. 8 (Eq. 4 with sim = exp): softmax attention,
+ *   o_i = sum_j exp(scale * q_i . k_j) v_j / sum_j exp(scale * q_i . k_j),
+ * all n tokens attending to all n tokens.  The paper prints the scale as 1/sqrt(d) in the text
+ * under Eq. 4 and as 1/d inside Eq. 8; it is an argument here.  The row maximum is subtracted
+ * before exponentiating (mathematically a no-op).
+ *   q,k,v : [G][n][d] float;  rows : nrows query indices, or NULL for all n
+ *   out   : [G][nrows or n][d] double
+ */
+int linattn_ref_softmax(const float *q, const float *k, const float *v,
+                        long G, long n, int d, double scale,
+                        const long *rows, long nrows, double *out)
+{
+    if (d < 1 || n < 1 || G < 1) return 1;
+    const long nr = rows ? nrows : n;
+    int fail = 0;
+#pragma omp parallel for schedule(dynamic, 8) collapse(2)
+    for (long g = 0; g < G; ++g) {
+        for (long r = 0; r < nr; ++r) {
+            double *s = (double *)malloc((size_t)n * sizeof(double));
+            if (!s) {
+                fail = 1;
+                continue;
+            }
+            const long i = rows ? rows[r] : r;
+            const float *qi = q + ((size_t)g * n + i) * d;
+            const float *kg = k + (size_t)g * n * d, *vg = v + (size_t)g * n * d;
+            double smax = 0.0;
+            for (long j = 0; j < n; ++j) {
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c) acc += (double)qi[c] * (double)kg[(size_t)j * d + c];
+                s[j] = scale * acc;
+                if (j == 0 || s[j] > smax) smax = s[j];
+            }
+            double den = 0.0;
+            for (long j = 0; j < n; ++j) {
+                s[j] = exp(s[j] - smax);
+                den += s[j];
+            }
+            double *o = out + ((size_t)g * nr + r) * d;
+            for (int c = 0; c < d; ++c) o[c] = 0.0;
+            for (long j = 0; j < n; ++j) {
+                const double w = s[j] / den;
+                for (int c = 0; c < d; ++c) o[c] += w * (double)vg[(size_t)j * d + c];
+            }
+            free(s);
+        }
+    }
+    return fail;
+}
+
+/*
+ * Eq. 8: out = r^ * o_softmax + (1 - r^) * o_linear, element by element, with the learnable
+ * score r clipped into [0, 1] first (footnote to Eq. 8): r^ = min(max(r, 0), 1).
+ */
+int linattn_ref_mix(const double *o_softmax, const double *o_linear, long count, double r, double *out)
+{
+    if (count < 0) return 1;
+    const double rc = r < 0.0 ? 0.0 : (r > 1.0 ? 1.0 : r);
+    for (long e = 0; e < count; ++e) out[e] = rc * o_softmax[e] + (1.0 - rc) * o_linear[e];
     return 0;
 }

@@ -47,6 +47,9 @@ def _load():
         lib.linattn_ref_linear.argtypes = [fp, fp, fp, fp, fp, ctypes.c_long, ctypes.c_int,
                                            ctypes.c_long, ctypes.c_int, ctypes.c_int,
                                            lp, ctypes.c_long, dp, dp, dp]
+        lib.linattn_ref_softmax.argtypes = [fp, fp, fp, ctypes.c_long, ctypes.c_long, ctypes.c_int, ctypes.c_double,
+                                            lp, ctypes.c_long, dp]
+        lib.linattn_ref_mix.argtypes = [dp, dp, ctypes.c_long, ctypes.c_double, dp]
         _lib = lib
     return _lib
 
@@ -134,3 +137,30 @@ def ref_linear(q, k, v, Wq, Wk, rows=None, return_state: bool = False):
     if rc:
         raise ValueError("oracle rejected the arguments or ran out of memory")
     return (out, S, z) if return_state else out
+
+
+def ref_softmax(q, k, v, scale: float, rows=None) -> np.ndarray:
+    """Softmax attention, the first term of Eq. 8, with an explicit scale on q.k. float64 [B, H, len(rows) or n, d]."""
+    q, k, v = (_f32(t) for t in (q, k, v))
+    assert q.ndim == 4 and q.shape == k.shape == v.shape
+    B, H, n, d = q.shape
+    r, nr = _rows(rows, n)
+    out = np.empty((B, H, nr, d), dtype=np.float64)
+    F = ctypes.c_float
+    rc = _load().linattn_ref_softmax(_ptr(q, F), _ptr(k, F), _ptr(v, F), B * H, n, d, float(scale),
+                                     _ptr(r, ctypes.c_long), nr, _ptr(out, ctypes.c_double))
+    if rc:
+        raise ValueError("oracle rejected the arguments or ran out of memory")
+    return out
+
+
+def ref_mix(o_softmax, o_linear, r: float) -> np.ndarray:
+    """Eq. 8: clip(r, 0, 1) * o_softmax + (1 - clip(r, 0, 1)) * o_linear, in float64."""
+    a = np.ascontiguousarray(o_softmax, dtype=np.float64)
+    b = np.ascontiguousarray(o_linear, dtype=np.float64)
+    assert a.shape == b.shape
+    out = np.empty_like(a)
+    D = ctypes.c_double
+    if _load().linattn_ref_mix(_ptr(a, D), _ptr(b, D), a.size, float(r), _ptr(out, D)):
+        raise ValueError("oracle rejected the arguments")
+    return out

@@ -227,3 +227,64 @@ def test_bad_arguments_are_rejected():
         oracle.ref_linear(q, k, v[:, :, :3], Wq, Wk)
     with pytest.raises(AssertionError):
         oracle.ref_linear(q, k, v, Wq, Wk, rows=np.array([4]))
+
+
+# ---- Eq. 8: softmax-attention term and the blend ---------------------------------------------------
+
+def test_mixed_attention_hand_example():
+    gold = _read_fractions("mixed_n2_d2.txt")
+    q = np.array([[[[1.0, 0.0], [0.0, 1.0]]]], dtype=np.float32)
+    k = np.array([[[[math.log(3.0), math.log(4.0)], [0.0, 0.0]]]], dtype=np.float32)
+    v = np.array([[[[4.0, 8.0], [0.0, -4.0]]]], dtype=np.float32)
+    o = oracle.ref_softmax(q, k, v, scale=1.0)
+    np.testing.assert_allclose(o[0, 0, 0], gold["softmax_o1"], rtol=0, atol=1e-6)
+    np.testing.assert_allclose(o[0, 0, 1], gold["softmax_o2"], rtol=0, atol=1e-6)
+    lin = np.ones_like(o)
+    want = np.stack([gold["mix_o1"], gold["mix_o2"]])[None, None]
+    np.testing.assert_allclose(oracle.ref_mix(o, lin, 0.25), want, rtol=0, atol=1e-6)
+    np.testing.assert_array_equal(oracle.ref_mix(o, lin, 1.75), o)      # clipped to 1: the softmax term alone
+    np.testing.assert_array_equal(oracle.ref_mix(o, lin, -0.5), lin)    # clipped to 0: the linear term alone
+
+
+@pytest.mark.parametrize("scale", [1.0, 0.25, 1.0 / 8.0])
+def test_softmax_term_matches_library_attention(scale):
+    """torch's fp64 scaled_dot_product_attention is an independent implementation of the same definition."""
+    rng = np.random.default_rng(5)
+    q, k, v = (rng.standard_normal((2, 3, 37, 16)).astype(np.float32) for _ in range(3))
+    got = oracle.ref_softmax(q, k, v, scale=scale)
+    want = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q).double(), torch.from_numpy(k).double(), torch.from_numpy(v).double(), scale=scale).numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-10, atol=1e-12)
+    rows = np.array([0, 5, 36])
+    np.testing.assert_allclose(oracle.ref_softmax(q, k, v, scale=scale, rows=rows), want[:, :, rows], rtol=1e-10, atol=1e-12)
+
+
+def test_softmax_term_special_cases():
+    rng = np.random.default_rng(6)
+    q, k, v = (rng.standard_normal((1, 2, 50, 8)).astype(np.float32) for _ in range(3))
+    # all keys equal -> uniform weights -> the mean of V, for every query
+    kc = np.broadcast_to(k[:, :, :1], k.shape).copy()
+    mean_v = v.astype(np.float64).mean(axis=2, keepdims=True)
+    np.testing.assert_allclose(oracle.ref_softmax(q, kc, v, scale=0.7), np.broadcast_to(mean_v, v.shape), rtol=1e-12, atol=1e-12)
+    # a very sharp softmax picks the value of the best-matching key
+    o = oracle.ref_softmax(q, k, v, scale=1e4)
+    best = np.einsum("bhid,bhjd->bhij", q.astype(np.float64), k.astype(np.float64)).argmax(-1)
+    np.testing.assert_allclose(o, np.take_along_axis(v.astype(np.float64), best[..., None], axis=2), rtol=0, atol=1e-9)
+    # logits of +-1e4 must not overflow
+    assert np.isfinite(o).all()
+    # joint permutation of (k, v) changes nothing
+    perm = rng.permutation(50)
+    np.testing.assert_allclose(oracle.ref_softmax(q, k[:, :, perm], v[:, :, perm], scale=0.3),
+                               oracle.ref_softmax(q, k, v, scale=0.3), rtol=1e-12, atol=1e-13)
+
+
+def test_mix_is_affine_in_the_clipped_score():
+    rng = np.random.default_rng(7)
+    a, b = rng.standard_normal((2, 3, 4, 5)), rng.standard_normal((2, 3, 4, 5))
+    m0, m1 = oracle.ref_mix(a, b, 0.0), oracle.ref_mix(a, b, 1.0)
+    np.testing.assert_array_equal(m0, b)
+    np.testing.assert_array_equal(m1, a)
+    for r in (0.1, 0.5, 0.9):
+        np.testing.assert_allclose(oracle.ref_mix(a, b, r), m0 + r * (m1 - m0), rtol=1e-13, atol=1e-14)
+    np.testing.assert_array_equal(oracle.ref_mix(a, b, 3.0), m1)
+    np.testing.assert_array_equal(oracle.ref_mix(a, b, -3.0), m0)
