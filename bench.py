@@ -169,6 +169,9 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-baselines", action="store_true", help="skip the oracle and SDPA context baselines")
+    ap.add_argument("--mixed", type=float, default=None, metavar="R",
+                    help="time mixed attention (Eq. 8) with score R instead: linattn_forward_mixed on a resident "
+                         "softmax-branch output (5 tensors of traffic instead of 4)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     wl = synth.CONFIGS[args.config]
@@ -194,6 +197,7 @@ def main():
             host0 = x
         sets.append({k_: t.to(dev) for k_, t in x.items()})
     outs = [torch.empty_like(s["q"]) for s in sets]
+    softs = [torch.randn_like(s["q"]) for s in sets] if args.mixed is not None else None
     ctxs = []
     for s in sets:  # one context per input set: its own feature map, as one layer would have
         c = linattn.LinAttn(H, d, max_B=B, max_n=n, device=local)
@@ -205,7 +209,10 @@ def main():
 
     def step(i):
         j = i % ROTATE
-        ctxs[j].forward(sets[j]["q"], sets[j]["k"], sets[j]["v"], out=outs[j], stream=stream)
+        if softs is None:
+            ctxs[j].forward(sets[j]["q"], sets[j]["k"], sets[j]["v"], out=outs[j], stream=stream)
+        else:
+            ctxs[j].forward_mixed(sets[j]["q"], sets[j]["k"], sets[j]["v"], softs[j], args.mixed, out=outs[j], stream=stream)
 
     for i in range(args.warmup):
         step(i)
@@ -234,7 +241,7 @@ def main():
 
     # per-kernel durations: a second pass of the same steps with events around every launch
     e = 2 if wl.dtype == "bf16" else 4
-    alg_total = 4.0 * B * H * n * d * e
+    alg_total = (4.0 if softs is None else 5.0) * B * H * n * d * e
     for c in ctxs:
         c.set_option(linattn.OPT_PROFILE, 1)
     for i in range(args.steps):
@@ -245,6 +252,8 @@ def main():
         c.set_option(linattn.OPT_PROFILE, 0)
     peaks = load_peaks()
     dom = max(kernels, key=lambda kt: kt["ms"])
+    if softs is not None:
+        dom["bytes"] += 1.0 * B * H * n * d * e   # the softmax branch's output is read once more
     achieved = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom["name"], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
@@ -255,7 +264,7 @@ def main():
                                "frac": alg_total / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                "frac_of_nominal_8TBs": alg_total / (ms_step * 1e-3) / 1e9 / 8000.0,
                                "algorithmic_bytes": alg_total}}
-    roofline["traffic"] = recorded_traffic(dom["name"])
+    roofline["traffic"] = recorded_traffic(dom["name"]) if softs is None else None
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host tensor out
     pin = {k_: host0[k_].pin_memory() for k_ in ("q", "k", "v")}
@@ -274,7 +283,8 @@ def main():
            "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "entry_point": "linattn_forward_host (pinned host buffers)"}
 
     result = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC if softs is None else "mixed-attention (Eq. 8) fwd tokens/s", "value": value, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": wl_name(args.config, wl), "B": B, "H": H, "n": n, "d": d, "path": args.path,

@@ -83,6 +83,23 @@ linattn_status linattn_forward(linattn_ctx* ctx, const void* q, const void* k, c
                                int B, int H, int n, int d, linattn_dtype dtype, void* stream);
 
 /*
+ * Mixed attention, Eq. 8: the layer's output while softmax attention is being transferred to linear attention,
+ *   out = r^ * o_softmax + (1 - r^) * [Eq. 5 applied to q, k, v],    r^ = min(max(r, 0), 1)
+ * (the footnote to Eq. 8 clips the learnable score r into [0, 1] before use).  o_softmax is the output of the
+ * softmax-attention branch of the same layer, computed by the caller with whatever attention kernel and
+ * scale it uses (the paper prints 1/sqrt(d) under Eq. 4 and 1/d inside Eq. 8); the blend is fused into the
+ * query side's epilogue: fp32, rounded once to the output type.  r^ = 0 gives linattn_forward's result bit
+ * for bit, r^ = 1 returns o_softmax.
+ *   o_softmax : device, [B][H][n][d] of `dtype`, 16-byte aligned, read-only; it may be the SAME buffer as `out`
+ *               (in place); any other overlap with `out` is an error
+ *   r         : the layer's score (host value); NaN is an error
+ * Everything else as for linattn_forward.  Errors: as linattn_forward, plus INVALID_ARG for the above.
+ */
+linattn_status linattn_forward_mixed(linattn_ctx* ctx, const void* q, const void* k, const void* v,
+                                     const void* o_softmax, float r, void* out, int B, int H, int n, int d,
+                                     linattn_dtype dtype, void* stream);
+
+/*
  * The same operation on HOST buffers (pageable or pinned): copies q, k, v to device staging
  * buffers owned by the context, runs linattn_forward, copies the result into `out`, and waits
  * for `stream` before returning.  The staging buffers are allocated (or grown) on the first call

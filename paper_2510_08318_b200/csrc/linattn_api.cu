@@ -154,7 +154,7 @@ int choose_splits(long long G, int n, int forced)
 
 template <typename T, int D>
 linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int n,
-                           cudaStream_t st)
+                           cudaStream_t st, const void* mix, float mix_r)
 {
     const long long G = (long long)B * c->H;
     int splits = choose_splits(G, n, c->opt_splits);
@@ -187,7 +187,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     if (per_group > nchunks) per_group = nchunks;
     if (per_group < 1) per_group = 1;
     qside_simt<T, D><<<dim3((unsigned)per_group, (unsigned)G), kSimtThreads, qside_simt_smem<D>(), st>>>(
-        (const T*)q, c->Wq, c->state, (T*)out, c->H, n);
+        (const T*)q, c->Wq, c->state, (T*)out, c->H, n, (const T*)mix, mix_r);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_simt", side_bytes);
     c->last_launches = 3;
@@ -196,7 +196,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
 
 // Tensor-core path: bf16, d = 128.
 linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int n,
-                         cudaStream_t st)
+                         cudaStream_t st, const void* mix, float mix_r)
 {
     using namespace linattn::tc;
     const long long G = (long long)B * c->H;
@@ -237,6 +237,8 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.z_img = c->z_img;
     a.err = c->err_word;
     a.sync = c->sync_words;
+    a.mix_src = (const __nv_bfloat16*)mix;
+    a.mix_r = mix_r;
     a.n = n;
     a.H = c->H;
     a.G = (int)G;
@@ -425,14 +427,22 @@ linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const voi
     return LINATTN_OK;
 }
 
-linattn_status linattn_forward(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int H,
-                               int n, int d, linattn_dtype dtype, void* stream)
+// Shared by linattn_forward (mix == NULL) and linattn_forward_mixed.
+static linattn_status forward_impl(linattn_ctx* c, const void* q, const void* k, const void* v, void* out,
+                                   const void* mix, float mix_r, int B, int H, int n, int d, linattn_dtype dtype,
+                                   void* stream)
 {
     linattn_status s = check_forward_args(c, q, k, v, out, B, H, n, d, dtype);
     if (s != LINATTN_OK) return s;
     if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(out)) return LINATTN_ERR_INVALID_ARG;
     const size_t bytes = (size_t)B * H * n * d * elem_size(dtype);
     if (overlaps(out, q, bytes) || overlaps(out, k, bytes) || overlaps(out, v, bytes)) return LINATTN_ERR_INVALID_ARG;
+    if (mix) {
+        if (misaligned16(mix)) return LINATTN_ERR_INVALID_ARG;
+        if (mix != out && overlaps(out, mix, bytes)) return LINATTN_ERR_INVALID_ARG;  // in place is fine, a partial overlap is not
+        if (!(mix_r == mix_r)) return LINATTN_ERR_INVALID_ARG;                         // NaN
+        mix_r = mix_r < 0.f ? 0.f : (mix_r > 1.f ? 1.f : mix_r);                       // footnote to Eq. 8: r is clipped into [0, 1]
+    }
     // The tensor-core kernels cover bf16 activations with head dimension 128 and bf16 feature-map weights;
     // everything else runs on the CUDA-core kernels.
     const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && c->map_is_bf16);
@@ -441,13 +451,27 @@ linattn_status linattn_forward(linattn_ctx* c, const void* q, const void* k, con
     cudaStream_t st = (cudaStream_t)stream;
     c->last_B = B;
     c->state_transposed = tc_ok && c->opt_path != 1;
-    if (c->state_transposed) return launch_tc(c, q, k, v, out, B, n, st);
+    if (c->state_transposed) return launch_tc(c, q, k, v, out, B, n, st, mix, mix_r);
     if (dtype == LINATTN_BF16) {
-        return d == 128 ? launch_simt<__nv_bfloat16, 128>(c, q, k, v, out, B, n, st)
-                        : launch_simt<__nv_bfloat16, 64>(c, q, k, v, out, B, n, st);
+        return d == 128 ? launch_simt<__nv_bfloat16, 128>(c, q, k, v, out, B, n, st, mix, mix_r)
+                        : launch_simt<__nv_bfloat16, 64>(c, q, k, v, out, B, n, st, mix, mix_r);
     }
-    return d == 128 ? launch_simt<float, 128>(c, q, k, v, out, B, n, st)
-                    : launch_simt<float, 64>(c, q, k, v, out, B, n, st);
+    return d == 128 ? launch_simt<float, 128>(c, q, k, v, out, B, n, st, mix, mix_r)
+                    : launch_simt<float, 64>(c, q, k, v, out, B, n, st, mix, mix_r);
+}
+
+linattn_status linattn_forward(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int H,
+                               int n, int d, linattn_dtype dtype, void* stream)
+{
+    return forward_impl(c, q, k, v, out, nullptr, 0.f, B, H, n, d, dtype, stream);
+}
+
+linattn_status linattn_forward_mixed(linattn_ctx* c, const void* q, const void* k, const void* v,
+                                     const void* o_softmax, float r, void* out, int B, int H, int n, int d,
+                                     linattn_dtype dtype, void* stream)
+{
+    if (!o_softmax) return LINATTN_ERR_INVALID_ARG;
+    return forward_impl(c, q, k, v, out, o_softmax, r, B, H, n, d, dtype, stream);
 }
 
 linattn_status linattn_forward_host(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B,

@@ -81,7 +81,7 @@ linattn_status run(int dev, int slot, float* scratch, const T* q, const T* k, co
     long long per_group = (2LL * 148 + G - 1) / G;
     if (per_group > nchunks) per_group = nchunks;
     qside_simt<T, D><<<dim3((unsigned)per_group, (unsigned)G), kSimtThreads, qside_simt_smem<D>(), st>>>(
-        q, Wq, state, out, Hw, n);
+        q, Wq, state, out, Hw, n, (const T*)nullptr, 0.f);
     if (cudaGetLastError() != cudaSuccess) return LINATTN_ERR_CUDA;
     return LINATTN_OK;
 }

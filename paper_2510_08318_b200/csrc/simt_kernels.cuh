@@ -187,10 +187,12 @@ template <int D> constexpr size_t qside_simt_smem()
 
 // grid = (blocks_per_group, G).  Block x handles chunks x, x + gridDim.x, ... of kSimtTokens tokens.
 // state: [G][D*D + D] floats (S then z).
+// mix != nullptr: Eq. 8, out = mix_r * mix + (1 - mix_r) * (Eq. 5), mix = output of the softmax-attention branch
+// ([G][n][D], may be the same buffer as out), mix_r already clipped into [0, 1].
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* __restrict__ state,
-           T* __restrict__ out, int H, int n)
+           T* out, int H, int n, const T* mix, float mix_r)
 {
     constexpr int M = SimtShape<D>::M, P = SimtShape<D>::PITCH;
     constexpr int CG = D / 32;  // float4 column groups per thread (4 or 2)
@@ -242,11 +244,15 @@ qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* _
         }
         if (tt < valid) {
             const float inv = 1.f / den;
+            const T* mg = mix ? mix + (size_t)g * n * D : nullptr;
 #pragma unroll
             for (int r = 0; r < CG; ++r)
 #pragma unroll
-                for (int b = 0; b < 4; ++b)
-                    store_out(&og[(size_t)(t + tt) * D + r * 32 + cg * 4 + b], num[r][b] * inv);
+                for (int b = 0; b < 4; ++b) {
+                    const size_t e = (size_t)(t + tt) * D + r * 32 + cg * 4 + b;
+                    const float lin = num[r][b] * inv;
+                    store_out(&og[e], mg ? fmaf(lin, 1.f - mix_r, mix_r * to_f32(mg[e])) : lin);
+                }
         }
     }
 }

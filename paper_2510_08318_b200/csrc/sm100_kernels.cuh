@@ -354,6 +354,8 @@ struct Args {
     uint32_t* err;               // error word
     uint32_t* sync;              // grid-barrier arrival counter of the fused kernel (monotonic over launches)
     uint32_t bar_target[2];      // its value once every CTA has arrived at the first / second barrier of this launch
+    const __nv_bfloat16* mix_src;  // Eq. 8: output of the softmax-attention branch [G][n][128], or nullptr (plain Eq. 5)
+    float mix_r;                 // Eq. 8: the score r, already clipped into [0, 1]
     int n, H, G;
     int tiles_per_head;
     long long total_tiles;
@@ -720,6 +722,15 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 tma_load_3d(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g);
                 tma_load_3d(sbase + r.s * kTileBytes + kHalfTileBytes, tmQ, c.bar(Q_FULL + r.s), 64, w.lt * kTile, w.g);
             }
+            if (a.mix_src != nullptr) {
+                // Eq. 8: the epilogue will read this tile's rows of the softmax branch's output straight from
+                // global memory a few microseconds from now; start them on their way into L2 (the rows of a tile
+                // are contiguous: 256 lines of 128 bytes, fewer in the ragged tail tile)
+                const int rows = min(kTile, a.n - w.lt * kTile);
+                const char* base = reinterpret_cast<const char*>(a.mix_src + ((size_t)w.g * a.n + (size_t)w.lt * kTile) * kD);
+                for (int line = lane; line < rows * 2; line += 32)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (size_t)line * 128));
+            }
             issued = w.i + 1;
         }
         if (ok && state_g >= 0) load_state();
@@ -836,8 +847,19 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             tcgen05_fence_after();
             uint32_t dv[2];
             tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
+            // Eq. 8 (mixed attention): this token's row of the softmax branch's output, read straight from global
+            // memory (the row is 256 contiguous bytes; rows past the end of the sequence are not touched)
+            const bool mix = a.mix_src != nullptr;
+            const bool in_range = w.lt * kTile + row < a.n;
+            const uint4* mrow = reinterpret_cast<const uint4*>(
+                a.mix_src + ((size_t)w.g * a.n + (size_t)(w.lt * kTile + (in_range ? row : 0))) * kD);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
+                uint4 av[8];
+                if (mix) {
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc) av[cc] = in_range ? __ldg(mrow + half * 8 + cc) : make_uint4(0u, 0u, 0u, 0u);
+                }
                 uint32_t v[64];
                 tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64, v);
                 tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64 + 32, v + 32);
@@ -849,18 +871,38 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                     if (lane == 0) mbar_arrive(c.bar(Q_DEMPTY + dr.s));
                 }
                 const float inv = __fdividef(1.f, __uint_as_float(dv[0]) + __uint_as_float(dv[1]));
-                const f32x2 inv2 = pack2(inv, inv);
                 uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                if (!mix) {
+                    const f32x2 inv2 = pack2(inv, inv);
 #pragma unroll
-                for (int cc = 0; cc < 8; ++cc) {
-                    uint32_t o[4];
+                    for (int cc = 0; cc < 8; ++cc) {
+                        uint32_t o[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float x, y;
-                        unpack2(mul2(pack2(__uint_as_float(v[8 * cc + 2 * q]), __uint_as_float(v[8 * cc + 2 * q + 1])), inv2), x, y);
-                        o[q] = pack_bf16(x, y);
+                        for (int q = 0; q < 4; ++q) {
+                            float x, y;
+                            unpack2(mul2(pack2(__uint_as_float(v[8 * cc + 2 * q]), __uint_as_float(v[8 * cc + 2 * q + 1])), inv2), x, y);
+                            o[q] = pack_bf16(x, y);
+                        }
+                        *reinterpret_cast<uint4*>(dst + ((cc ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
-                    *reinterpret_cast<uint4*>(dst + ((cc ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                } else {
+                    // o = r * softmax branch + (1 - r) * num / den, in fp32, rounded once
+                    const float lin = (1.f - a.mix_r) * inv;
+                    const f32x2 lin2 = pack2(lin, lin), r2 = pack2(a.mix_r, a.mix_r);
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc) {
+                        const uint32_t aw4[4] = {av[cc].x, av[cc].y, av[cc].z, av[cc].w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const f32x2 soft = pack2(__uint_as_float(aw4[q] << 16), __uint_as_float(aw4[q] & 0xffff0000u));
+                            float x, y;
+                            unpack2(fma2(pack2(__uint_as_float(v[8 * cc + 2 * q]), __uint_as_float(v[8 * cc + 2 * q + 1])), lin2,
+                                         mul2(soft, r2)), x, y);
+                            o[q] = pack_bf16(x, y);
+                        }
+                        *reinterpret_cast<uint4*>(dst + ((cc ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
                 }
             }
             fence_proxy_async_smem();

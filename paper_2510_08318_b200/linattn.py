@@ -27,6 +27,7 @@ SIGNATURES = {
     "linattn_create": (_i, [ctypes.POINTER(_vp), _i, _i, _i, _ll, _ll]),
     "linattn_set_feature_map": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "linattn_forward": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "linattn_forward_mixed": (_i, [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_host": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_noalloc": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "linattn_read_state": (_i, [_vp, _vp, _vp, _i, _vp]),
@@ -140,6 +141,20 @@ class LinAttn:
         B, H, n, d = q.shape
         self._call(self._lib.linattn_forward, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                    B, H, n, d, _DTYPES[q.dtype], _stream_ptr(stream))
+        return out
+
+    def forward_mixed(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, o_softmax: torch.Tensor, r: float,
+                      out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+        """Eq. 8: clip(r, 0, 1) * o_softmax + (1 - clip(r, 0, 1)) * linear attention.  ``o_softmax`` is the output of
+        the layer's softmax-attention branch, [B, H, n, d]; ``out`` may be ``o_softmax`` itself (in place)."""
+        assert q.is_cuda and q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and o_softmax.is_contiguous()
+        assert q.shape == k.shape == v.shape == o_softmax.shape and q.dtype == k.dtype == v.dtype == o_softmax.dtype
+        if out is None:
+            out = torch.empty_like(q)
+        assert out.is_contiguous() and out.shape == q.shape and out.dtype == q.dtype
+        B, H, n, d = q.shape
+        self._call(self._lib.linattn_forward_mixed, q.data_ptr(), k.data_ptr(), v.data_ptr(), o_softmax.data_ptr(),
+                   float(r), out.data_ptr(), B, H, n, d, _DTYPES[q.dtype], _stream_ptr(stream))
         return out
 
     def forward_host(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
