@@ -16,7 +16,9 @@ mx = dist.max_over_ranks(10.0 + rank)          # slowest rank's time
 sm = dist.sum_over_ranks(100.0 * (rank + 1))   # units processed by all ranks
 lo, hi = dist.shard_range(25, rank, world)
 n_units = dist.sum_over_ranks(float(hi - lo))
-print(f"RESULT {rank} {mx} {sm} {lo} {hi} {n_units}")
+# one file per rank: two processes printing to one pipe can interleave their lines
+with open(os.path.join(os.environ["LA_OUT"], f"rank{rank}.txt"), "w") as fh:
+    fh.write(f"{rank} {mx} {sm} {lo} {hi} {n_units}\n")
 dist.shutdown()
 """
 
@@ -24,12 +26,12 @@ dist.shutdown()
 def test_two_gloo_ranks_reduce_and_shard(tmp_path):
     script = tmp_path / "worker.py"
     script.write_text(WORKER)
-    env = dict(os.environ, LA_ROOT=ROOT)
+    env = dict(os.environ, LA_ROOT=ROOT, LA_OUT=str(tmp_path))
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
            "--master-addr", "127.0.0.1", "--master-port", "29617", str(script)]
     res = subprocess.run(cmd, capture_output=True, text=True, env=env, timeout=240)
     assert res.returncode == 0, res.stderr[-2000:]
-    rows = sorted(line.split()[1:] for line in res.stdout.splitlines() if line.startswith("RESULT"))
+    rows = sorted((tmp_path / f"rank{r}.txt").read_text().split() for r in range(2))
     assert len(rows) == 2
     for rank, row in enumerate(rows):
         assert int(row[0]) == rank
