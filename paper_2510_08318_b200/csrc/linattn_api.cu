@@ -225,8 +225,10 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     static bool attr_done = false;
     if (!attr_done) {
         LA_CUDA(c, cudaFuncSetAttribute(kside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(qside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(linattn_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(qside_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(qside_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(linattn_fused_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        LA_CUDA(c, cudaFuncSetAttribute(linattn_fused_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
         attr_done = true;
     }
     const double side_bytes = 2.0 * (double)G * n * kD * 2;
@@ -254,7 +256,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
         c->bar_total += 2u * (uint32_t)Pq;
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &a};
-        LA_CUDA(c, cudaLaunchCooperativeKernel((const void*)linattn_fused_tc, dim3((unsigned)Pq), dim3(kThreads), params,
+        LA_CUDA(c, cudaLaunchCooperativeKernel(mix ? (const void*)linattn_fused_tc<true> : (const void*)linattn_fused_tc<false>, dim3((unsigned)Pq), dim3(kThreads), params,
                                                Smem::kTotal, st));
         prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
         c->last_launches = 1;
@@ -266,7 +268,8 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     combine_tc<<<dim3((kE / 4 + 255) / 256, (unsigned)G), 256, 0, st>>>(a, Pk);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_tc", 0.0);
-    qside_tc<<<(unsigned)Pq, kThreads, Smem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, a);
+    if (mix) qside_tc<true><<<(unsigned)Pq, kThreads, Smem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, a);
+    else qside_tc<false><<<(unsigned)Pq, kThreads, Smem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, a);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);
     c->last_launches = 3;

@@ -641,6 +641,7 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
 
 // wait_state: the S and z images are produced earlier in the same kernel (fused path); loads of them
 // must wait for the Q_SREADY barrier.  Otherwise they were written by a previous launch.
+template <bool kMix>
 __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
                                             const CUtensorMap* tmW, const CUtensorMap* tmS, bool wait_state)
 {
@@ -722,7 +723,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 tma_load_3d(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g);
                 tma_load_3d(sbase + r.s * kTileBytes + kHalfTileBytes, tmQ, c.bar(Q_FULL + r.s), 64, w.lt * kTile, w.g);
             }
-            if (a.mix_src != nullptr) {
+            if (kMix) {
                 // Eq. 8: the epilogue will read this tile's rows of the softmax branch's output straight from
                 // global memory a few microseconds from now; start them on their way into L2 (the rows of a tile
                 // are contiguous: 256 lines of 128 bytes, fewer in the ragged tail tile)
@@ -849,7 +850,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
             // Eq. 8 (mixed attention): this token's row of the softmax branch's output, read straight from global
             // memory (the row is 256 contiguous bytes; rows past the end of the sequence are not touched)
-            const bool mix = a.mix_src != nullptr;
+            constexpr bool mix = kMix;   // compile-time: the plain forward carries none of the blend's registers
             const bool in_range = w.lt * kTile + row < a.n;
             const uint4* mrow = reinterpret_cast<const uint4*>(
                 a.mix_src + ((size_t)w.g * a.n + (size_t)(w.lt * kTile + (in_range ? row : 0))) * kD);
@@ -934,13 +935,14 @@ static __global__ void __launch_bounds__(256) combine_tc(const Args a, long long
     if (q4 < kE / 4) combine_quad(a, P, blockIdx.y, q4 * 4);
 }
 
+template <bool kMix>
 __global__ void __launch_bounds__(kThreads, 1)
 qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
          const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, false, true);
-    qside_phase(c, a, &tmQ, &tmO, &tmW, &tmS, false);
+    qside_phase<kMix>(c, a, &tmQ, &tmO, &tmW, &tmS, false);
     cta_teardown(c);
 }
 
@@ -962,6 +964,7 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target)
 }
 
 // The whole forward in one cooperative launch of P <= #SMs persistent CTAs.
+template <bool kMix>
 __global__ void __launch_bounds__(kThreads, 1)
 linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmQ,
@@ -1013,7 +1016,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (c.warp >= 12 && c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
-    qside_phase(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
+    qside_phase<kMix>(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
     LA_TRACE_NS(0, 61, 2);
     cta_teardown(c);
     LA_TRACE_NS(0, 61, 3);
