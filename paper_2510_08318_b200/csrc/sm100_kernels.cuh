@@ -788,29 +788,24 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         }
     } else if (warp == 11) {
         // ---------------- TMA stores of finished output tiles ----------------
-        // Two stores may be in flight: after issuing tile j's store the warp waits only until tile j-1's
-        // store has read its slot, then hands that slot back to the producer.
+        // The slot goes back to the producer as soon as the store has READ it (the write to global memory goes on
+        // by itself): the query side runs at the rate at which slots come back, so every microsecond a slot is
+        // held longer than needed costs throughput.
         if (lane == 0) tma_prefetch_desc(tmO);
         Ring<kQStages> r;
-        int prev_slot = -1;
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(Q_OFULL + r.s), r.ph, c.wc, kErrStore)) break;
             if (lane == 0) {
                 tma_store_3d(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g);
                 tma_store_3d(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g);
                 bulk_commit_group();
-                bulk_wait_group_read<1>();
-                if (prev_slot >= 0) mbar_arrive(c.bar(Q_EMPTY + prev_slot));
+                bulk_wait_group_read<0>();
+                mbar_arrive(c.bar(Q_EMPTY + r.s));
             }
-            prev_slot = r.s;
             __syncwarp();
             LA_TRACE(0, 24 + w.i, 1);
         }
-        if (lane == 0) {
-            bulk_wait_group_read<0>();
-            if (prev_slot >= 0) mbar_arrive(c.bar(Q_EMPTY + prev_slot));
-            bulk_wait_group<0>();
-        }
+        if (lane == 0) bulk_wait_group<0>();
     } else if (warp < 8) {
         // ---------------- feature map (warps 0-7) ----------------
         const int half = warp >> 2;
