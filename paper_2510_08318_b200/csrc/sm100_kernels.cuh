@@ -320,10 +320,12 @@ struct Smem {
     static constexpr uint32_t kOnes = kKW + 2 * kWBytes;                  // 1 KB of bf16 ones
     static constexpr uint32_t kKEnd = kOnes + 1024;
     // query side (overlays the key-side region)
-    static constexpr uint32_t kQS = kQStages * kTileBytes;                // S image (32 KB)
-    static constexpr uint32_t kQW = kQS + kTileBytes;                     // W_q^T (16 KB)
-    static constexpr uint32_t kQZ = kQW + kWBytes;                        // z operand (4 KB)
-    static constexpr uint32_t kQEnd = kQZ + kZBlkBytes;
+    // [S | z] operand of the query side: per 64-feature block 144 rows of 128 bytes, rows 0-127 = S image [c][f],
+    // rows 128-143 = z operand (hi, lo, zeros): ONE MMA of N = 144 per K step gives numerator and denominator
+    static constexpr uint32_t kSZBlock = kHalfTileBytes + kZBlkBytes / 2; // 18 KB
+    static constexpr uint32_t kQS = kQStages * kTileBytes;                // 2 blocks (36 KB)
+    static constexpr uint32_t kQW = kQS + 2 * kSZBlock;                   // W_q^T (16 KB)
+    static constexpr uint32_t kQEnd = kQW + kWBytes;
     static constexpr uint32_t kBars = kKEnd > kQEnd ? kKEnd : kQEnd;      // mbarriers, TMEM slot, abort word
     static constexpr uint32_t kTotal = kBars + 512 + 1024;                // + alignment slack
 };
@@ -646,8 +648,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                                             const CUtensorMap* tmW, const CUtensorMap* tmS, bool wait_state)
 {
     const uint32_t tmem_u = c.tmem;  // 2 x 64 columns of logits
-    auto tmem_num = [&](int db) { return c.tmem + 128 + db * 160; };   // 128 columns: num[token][c]
-    auto tmem_den = [&](int db) { return c.tmem + 256 + db * 160; };   // 16 columns: [hi(z) part, lo(z) part, ...]
+    auto tmem_num = [&](int db) { return c.tmem + 128 + db * 160; };   // 144 columns: num[token][c], c = 0..127, then
+    auto tmem_den = [&](int db) { return c.tmem + 256 + db * 160; };   // 16 columns: [phi(q).z_hi, phi(q).z_lo, 0...]
     const int warp = c.warp, lane = c.lane;
     const uint32_t sbase = c.sbase;
     TileWalk w;
@@ -671,9 +673,12 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             if (lane == 0) {
                 if (wait_state) fence_proxy_async_all();
                 mbar_arrive_expect_tx(c.bar(Q_SEGFULL), kTileBytes + kZBlkBytes);
-                tma_load_3d(sbase + Smem::kQS, tmS, c.bar(Q_SEGFULL), 0, 0, state_g);
-                tma_load_3d(sbase + Smem::kQS + kHalfTileBytes, tmS, c.bar(Q_SEGFULL), 64, 0, state_g);
-                bulk_load_1d(sbase + Smem::kQZ, a.z_img + (size_t)state_g * (kZBlkBytes / 2), kZBlkBytes, c.bar(Q_SEGFULL));
+                const __nv_bfloat16* zsrc = a.z_img + (size_t)state_g * (kZBlkBytes / 2);
+                for (int blk = 0; blk < 2; ++blk) {
+                    const uint32_t dst = sbase + Smem::kQS + blk * Smem::kSZBlock;
+                    tma_load_3d(dst, tmS, c.bar(Q_SEGFULL), 64 * blk, 0, state_g);
+                    bulk_load_1d(dst + kHalfTileBytes, zsrc + blk * (kZBlkBytes / 4), kZBlkBytes / 2, c.bar(Q_SEGFULL));
+                }
             }
             state_g = -1;
         };
@@ -758,8 +763,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         }
     } else if (warp == 10) {
         // ---------------- numerator / denominator MMA issuer: num = phi(q) S, den = phi(q) . z ----------------
-        constexpr uint32_t idesc_n = make_idesc_bf16(kTile, kD, 0, 0);   // A = phi(q) (K-major), B = S image [c][f] (K-major)
-        constexpr uint32_t idesc_d = make_idesc_bf16(kTile, 16, 0, 0);   // B = z operand (K-major)
+        constexpr uint32_t idesc_n = make_idesc_bf16(kTile, kD + 16, 0, 0);   // A = phi(q) (K-major), B = [S image [c][f]; z operand] (K-major)
         const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
         const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
         Ring<kQStages> r;
@@ -775,10 +779,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) {
                     const uint64_t da = desc_at(kmajor, phi + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
-                    const uint64_t db_s = desc_at(kmajor, sbase + Smem::kQS + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
-                    const uint64_t db_z = desc_at(kmajor, sbase + Smem::kQZ + (k >> 2) * 2048 + (k & 3) * 32);
-                    mma_bf16_ss(tmem_num(dr.s), da, db_s, idesc_n, k > 0);
-                    mma_bf16_ss(tmem_den(dr.s), da, db_z, idesc_d, k > 0);
+                    const uint64_t db = desc_at(kmajor, sbase + Smem::kQS + (k >> 2) * Smem::kSZBlock + (k & 3) * 32);
+                    mma_bf16_ss(tmem_num(dr.s), da, db, idesc_n, k > 0);
                 }
                 mma_commit(c.bar(Q_DFULL + dr.s));
                 if (w.last()) mma_commit(c.bar(Q_SEGFREE));   // this head's S, z and W may now be replaced
