@@ -44,6 +44,9 @@ typedef enum {
     LINATTN_OPT_PATH = 1,   /* 0 = automatic (default), 1 = CUDA-core kernels, 2 = tensor-core (tcgen05 + TMA) kernels */
     LINATTN_OPT_FUSE = 3,   /* tensor-core path: 1 = one cooperative kernel for the whole forward (default, used when the
                                device allows it), 0 = three launches (key side, combine, query side) */
+    LINATTN_OPT_LAYOUT = 4, /* memory order of q, k, v, out (and o_softmax): 0 = [B][H][n][d] (default), 1 = [B][n][H][d],
+                               the order in which a DiT's projection layers leave them (no transposes around the call);
+                               d is contiguous in both */
     LINATTN_OPT_PROFILE = 2 /* 1 = record CUDA events around every kernel of each forward (see linattn_profile_get);
                                switching it on clears the accumulated figures; 0 = off (default) */
 } linattn_option;
@@ -69,7 +72,8 @@ linattn_status linattn_set_feature_map(linattn_ctx* ctx, const void* Wq, const v
 
 /*
  * Eq. 5 (right-hand form) with the feature map of Eq. 6, for all B*H (b,h) pairs.
- *   q, k, v : device, contiguous row-major [B][H][n][d] of `dtype`, 16-byte aligned, read-only
+ *   q, k, v : device, contiguous [B][H][n][d] (or [B][n][H][d], see LINATTN_OPT_LAYOUT) of `dtype`, 16-byte aligned,
+ *             read-only
  *   out     : device, same shape and type, written in full; must not overlap q, k or v
  *   H, d    : must equal the values given to create;  1 <= B <= max_B;  1 <= n <= max_n
  *   dtype   : LINATTN_BF16 (bf16 in, bf16 out, round-to-nearest-even) or LINATTN_F32

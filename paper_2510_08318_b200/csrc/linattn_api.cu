@@ -66,6 +66,7 @@ struct linattn_ctx {
     int opt_splits = 0;
     int opt_path = 0;
     int opt_fuse = 1;
+    int opt_layout = 0;   // 0: [B][H][n][d], 1: [B][n][H][d]
     // per-kernel timing (LINATTN_OPT_PROFILE)
     static constexpr int kMaxKernels = 4;
     bool profile = false;
@@ -101,6 +102,14 @@ linattn_status cuda_fail(linattn_ctx* c, cudaError_t e, const char* what)
     } while (0)
 
 size_t elem_size(linattn_dtype t) { return t == LINATTN_BF16 ? 2 : 4; }
+
+// Element strides of q, k, v, out for the context's layout option.
+ActStrides act_strides(const linattn_ctx* c, int n)
+{
+    const long long d = c->d, H = c->H;
+    if (c->opt_layout == 1) return ActStrides{H * d, d, (long long)n * H * d};   // [B][n][H][d]
+    return ActStrides{d, (long long)n * d, H * (long long)n * d};                 // [B][H][n][d]
+}
 
 // Per-kernel timing: events are recorded around every launch of a forward and read back (after a
 // wait on the last one) at the start of the next profiled forward or when the figures are queried.
@@ -176,7 +185,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     const double side_bytes = 2.0 * (double)G * n * D * sizeof(T);  // K+V read, or Q read + O written
     prof_begin(c, st);
     kside_simt<T, D><<<dim3(splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
-        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk);
+        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, act_strides(c, n));
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_simt", side_bytes);
     combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, c->state, splits, E);
@@ -187,7 +196,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     if (per_group > nchunks) per_group = nchunks;
     if (per_group < 1) per_group = 1;
     qside_simt<T, D><<<dim3((unsigned)per_group, (unsigned)G), kSimtThreads, qside_simt_smem<D>(), st>>>(
-        (const T*)q, c->Wq, c->state, (T*)out, c->H, n, (const T*)mix, mix_r);
+        (const T*)q, c->Wq, c->state, (T*)out, c->H, n, (const T*)mix, mix_r, act_strides(c, n));
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_simt", side_bytes);
     c->last_launches = 3;
@@ -211,10 +220,14 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     if (Pk + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
 
     CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmS;
-    const bool ok = make_tmap_bf16_3d(&tmK, k, kD, (uint64_t)n, (uint64_t)G, kTile) &&
-                    make_tmap_bf16_3d(&tmV, v, kD, (uint64_t)n, (uint64_t)G, kTile) &&
-                    make_tmap_bf16_3d(&tmQ, q, kD, (uint64_t)n, (uint64_t)G, kTile) &&
-                    make_tmap_bf16_3d(&tmO, out, kD, (uint64_t)n, (uint64_t)G, kTile) &&
+    const ActStrides as = act_strides(c, n);
+    const int layout = c->opt_layout;
+    auto act_map = [&](CUtensorMap* m, const void* base) {
+        if (layout == 0) return make_tmap_bf16_3d(m, base, kD, (uint64_t)n, (uint64_t)G, kTile);
+        return make_tmap_bf16_act(m, base, kD, (uint64_t)n, (uint64_t)c->H, (uint64_t)B, (uint64_t)as.token * 2,
+                                  (uint64_t)as.head * 2, (uint64_t)as.batch * 2, kTile);
+    };
+    const bool ok = act_map(&tmK, k) && act_map(&tmV, v) && act_map(&tmQ, q) && act_map(&tmO, out) &&
                     make_tmap_bf16_3d(&tmWk, c->Wkt, kD, kM, (uint64_t)c->H, kM) &&
                     make_tmap_bf16_3d(&tmWq, c->Wqt, kD, kM, (uint64_t)c->H, kM) &&
                     make_tmap_bf16_3d(&tmS, c->s_img, kD, kD, (uint64_t)G, kTile);
@@ -222,13 +235,21 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         snprintf(c->err_text, sizeof(c->err_text), "cuTensorMapEncodeTiled failed");
         return LINATTN_ERR_CUDA;
     }
+    // one instantiation per (mixed attention or not, memory layout)
+    const void* k_fused[2][2] = {{(const void*)linattn_fused_tc<false, 0>, (const void*)linattn_fused_tc<false, 1>},
+                                 {(const void*)linattn_fused_tc<true, 0>, (const void*)linattn_fused_tc<true, 1>}};
+    const void* k_qside[2][2] = {{(const void*)qside_tc<false, 0>, (const void*)qside_tc<false, 1>},
+                                 {(const void*)qside_tc<true, 0>, (const void*)qside_tc<true, 1>}};
+    const void* k_kside[2] = {(const void*)kside_tc<0>, (const void*)kside_tc<1>};
     static bool attr_done = false;
     if (!attr_done) {
-        LA_CUDA(c, cudaFuncSetAttribute(kside_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(qside_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(qside_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(linattn_fused_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-        LA_CUDA(c, cudaFuncSetAttribute(linattn_fused_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        for (int i = 0; i < 2; ++i) {
+            LA_CUDA(c, cudaFuncSetAttribute(k_kside[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+            for (int j = 0; j < 2; ++j) {
+                LA_CUDA(c, cudaFuncSetAttribute(k_fused[i][j], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                LA_CUDA(c, cudaFuncSetAttribute(k_qside[i][j], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+            }
+        }
         attr_done = true;
     }
     const double side_bytes = 2.0 * (double)G * n * kD * 2;
@@ -241,6 +262,9 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.sync = c->sync_words;
     a.mix_src = (const __nv_bfloat16*)mix;
     a.mix_r = mix_r;
+    a.str_token = as.token;
+    a.str_head = as.head;
+    a.str_batch = as.batch;
     a.n = n;
     a.H = c->H;
     a.G = (int)G;
@@ -256,20 +280,25 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
         c->bar_total += 2u * (uint32_t)Pq;
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &a};
-        LA_CUDA(c, cudaLaunchCooperativeKernel(mix ? (const void*)linattn_fused_tc<true> : (const void*)linattn_fused_tc<false>, dim3((unsigned)Pq), dim3(kThreads), params,
+        LA_CUDA(c, cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads), params,
                                                Smem::kTotal, st));
         prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
         c->last_launches = 1;
         return LINATTN_OK;
     }
-    kside_tc<<<(unsigned)Pk, kThreads, Smem::kTotal, st>>>(tmK, tmV, tmWk, a);
+    {
+        void* kp[] = {&tmK, &tmV, &tmWk, &a};
+        LA_CUDA(c, cudaLaunchKernel(k_kside[layout], dim3((unsigned)Pk), dim3(kThreads), kp, Smem::kTotal, st));
+    }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_tc", side_bytes);
     combine_tc<<<dim3((kE / 4 + 255) / 256, (unsigned)G), 256, 0, st>>>(a, Pk);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_tc", 0.0);
-    if (mix) qside_tc<true><<<(unsigned)Pq, kThreads, Smem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, a);
-    else qside_tc<false><<<(unsigned)Pq, kThreads, Smem::kTotal, st>>>(tmQ, tmO, tmWq, tmS, a);
+    {
+        void* qp[] = {&tmQ, &tmO, &tmWq, &tmS, &a};
+        LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
+    }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);
     c->last_launches = 3;
@@ -546,6 +575,10 @@ linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long 
         case LINATTN_OPT_PATH:
             if (value < 0 || value > 2) return LINATTN_ERR_INVALID_ARG;
             c->opt_path = (int)value;
+            return LINATTN_OK;
+        case LINATTN_OPT_LAYOUT:
+            if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
+            c->opt_layout = (int)value;
             return LINATTN_OK;
         case LINATTN_OPT_FUSE:
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;

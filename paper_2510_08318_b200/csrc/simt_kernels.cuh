@@ -81,14 +81,20 @@ __device__ __forceinline__ void feature_map_chunk(const float* __restrict__ x_s,
 // Load `rows` x D elements starting at src (row-major, contiguous) into dst (fp32, pitch PITCH);
 // rows in [valid, kSimtTokens) are zero-filled.
 template <typename T, int D>
-__device__ __forceinline__ void load_chunk(const T* __restrict__ src, float* __restrict__ dst, int valid)
+__device__ __forceinline__ void load_chunk(const T* __restrict__ src, long long row_stride, float* __restrict__ dst, int valid)
 {
     constexpr int P = SimtShape<D>::PITCH;
     for (int e = threadIdx.x; e < kSimtTokens * D; e += kSimtThreads) {
         const int r = e / D, c = e % D;
-        dst[r * P + c] = (r < valid) ? to_f32(src[(size_t)r * D + c]) : 0.f;
+        dst[r * P + c] = (r < valid) ? to_f32(src[(size_t)r * row_stride + c]) : 0.f;
     }
 }
+
+// Element strides of the activations [batch][head][token][feature] (feature contiguous) in memory.
+struct ActStrides {
+    long long token, head, batch;
+    __device__ __forceinline__ size_t base(int g, int H) const { return (size_t)(g / H) * batch + (size_t)(g % H) * head; }
+};
 
 template <int D> constexpr size_t kside_simt_smem()
 {
@@ -100,7 +106,7 @@ template <int D> constexpr size_t kside_simt_smem()
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 kside_simt(const T* __restrict__ k, const T* __restrict__ v, const float* __restrict__ Wk /*[H][D][M]*/,
-           float* __restrict__ partial, int H, int n, int chunk)
+           float* __restrict__ partial, int H, int n, int chunk, ActStrides st)
 {
     constexpr int M = SimtShape<D>::M, P = SimtShape<D>::PITCH;
     constexpr int FB = D / 16;           // f rows per thread (8 or 4)
@@ -126,14 +132,14 @@ kside_simt(const T* __restrict__ k, const T* __restrict__ v, const float* __rest
 #pragma unroll
         for (int b = 0; b < CB; ++b) acc[a][b] = 0.f;
     }
-    const T* kg = k + (size_t)g * n * D;
-    const T* vg = v + (size_t)g * n * D;
+    const T* kg = k + st.base(g, H);
+    const T* vg = v + st.base(g, H);
 
     for (int t = t0; t < t1; t += kSimtTokens) {
         const int valid = min(kSimtTokens, t1 - t);
         __syncthreads();  // previous chunk fully consumed (and W_s visible on the first pass)
-        load_chunk<T, D>(kg + (size_t)t * D, k_s, valid);
-        load_chunk<T, D>(vg + (size_t)t * D, v_s, valid);
+        load_chunk<T, D>(kg + (size_t)t * st.token, st.token, k_s, valid);
+        load_chunk<T, D>(vg + (size_t)t * st.token, st.token, v_s, valid);
         __syncthreads();
         feature_map_chunk<D>(k_s, W_s, phi_s, valid);
         __syncthreads();
@@ -192,7 +198,7 @@ template <int D> constexpr size_t qside_simt_smem()
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* __restrict__ state,
-           T* out, int H, int n, const T* mix, float mix_r)
+           T* out, int H, int n, const T* mix, float mix_r, ActStrides st)
 {
     constexpr int M = SimtShape<D>::M, P = SimtShape<D>::PITCH;
     constexpr int CG = D / 32;  // float4 column groups per thread (4 or 2)
@@ -209,8 +215,8 @@ qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* _
     for (int e = tid; e < D * M; e += kSimtThreads) W_s[e] = Wg[e];
     for (int e = tid; e < D * D + D; e += kSimtThreads) S_s[e] = Sg[e];  // z_s follows S_s
 
-    const T* qg = q + (size_t)g * n * D;
-    T* og = out + (size_t)g * n * D;
+    const T* qg = q + st.base(g, H);
+    T* og = out + st.base(g, H);
     const int tt = tid >> 3, cg = tid & 7;
     const int nchunks = (n + kSimtTokens - 1) / kSimtTokens;
 
@@ -218,7 +224,7 @@ qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* _
         const int t = ch * kSimtTokens;
         const int valid = min(kSimtTokens, n - t);
         __syncthreads();
-        load_chunk<T, D>(qg + (size_t)t * D, q_s, valid);
+        load_chunk<T, D>(qg + (size_t)t * st.token, st.token, q_s, valid);
         __syncthreads();
         feature_map_chunk<D>(q_s, W_s, phi_s, kSimtTokens);  // tail rows see zero-filled q: finite phi, never stored
         __syncthreads();
@@ -244,12 +250,12 @@ qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* _
         }
         if (tt < valid) {
             const float inv = 1.f / den;
-            const T* mg = mix ? mix + (size_t)g * n * D : nullptr;
+            const T* mg = mix ? mix + st.base(g, H) : nullptr;
 #pragma unroll
             for (int r = 0; r < CG; ++r)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {
-                    const size_t e = (size_t)(t + tt) * D + r * 32 + cg * 4 + b;
+                    const size_t e = (size_t)(t + tt) * st.token + r * 32 + cg * 4 + b;
                     const float lin = num[r][b] * inv;
                     store_out(&og[e], mg ? fmaf(lin, 1.f - mix_r, mix_r * to_f32(mg[e])) : lin);
                 }

@@ -358,6 +358,7 @@ struct Args {
     uint32_t bar_target[2];      // its value once every CTA has arrived at the first / second barrier of this launch
     const __nv_bfloat16* mix_src;  // Eq. 8: output of the softmax-attention branch [G][n][128], or nullptr (plain Eq. 5)
     float mix_r;                 // Eq. 8: the score r, already clipped into [0, 1]
+    long long str_token, str_head, str_batch;  // element strides of q, k, v, out (and mix_src) between tokens, heads, batches
     int n, H, G;
     int tiles_per_head;
     long long total_tiles;
@@ -418,10 +419,33 @@ __device__ __forceinline__ void cta_teardown(const Cta& c)
     if (c.warp == 9) tmem_dealloc(c.tmem, 512);
 }
 
+// Activations q, k, v, out as TMA sees them.  kLayout 0: [B][H][n][d], a rank-3 map (feature, token, b*H + h);
+// kLayout 1: [B][n][H][d], a rank-4 map (feature, token, head, batch).  The rank-3 form is measurably faster
+// (1.5 us per forward at B=1, H=12, n=32760), so the default layout keeps it.
+template <int kLayout>
+__device__ __forceinline__ void act_load(uint32_t dst, const void* tm, uint32_t bar, int x, int t, int g, int H)
+{
+    if (kLayout == 0) tma_load_3d(dst, tm, bar, x, t, g);
+    else tma_load_4d(dst, tm, bar, x, t, g % H, g / H);
+}
+template <int kLayout>
+__device__ __forceinline__ void act_store(const void* tm, uint32_t src, int x, int t, int g, int H)
+{
+    if (kLayout == 0) tma_store_3d(tm, src, x, t, g);
+    else tma_store_4d(tm, src, x, t, g % H, g / H);
+}
+template <int kLayout>
+__device__ __forceinline__ void act_prefetch_l2(const void* tm, int x, int t, int g, int H)
+{
+    if (kLayout == 0) tma_prefetch_l2_3d(tm, x, t, g);
+    else tma_prefetch_l2_4d(tm, x, t, g % H, g / H);
+}
+
 // ======================================================================================================
 // Key side: partial S = sum phi(k)^T v and z = sum phi(k) over this CTA's tiles (Eq. 5 brackets, Eq. 6)
 // ======================================================================================================
 
+template <int kLayout>
 __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const CUtensorMap* tmK, const CUtensorMap* tmV,
                                             const CUtensorMap* tmW)
 {
@@ -459,10 +483,10 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             if (lane == 0) {
                 mbar_arrive_expect_tx(c.bar(K_FULL + r.s), 2 * kTileBytes);
                 const uint32_t kdst = sbase + r.s * Smem::kKStage, vdst = kdst + kTileBytes;
-                tma_load_3d(kdst, tmK, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g);
-                tma_load_3d(kdst + kHalfTileBytes, tmK, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g);
-                tma_load_3d(vdst, tmV, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g);
-                tma_load_3d(vdst + kHalfTileBytes, tmV, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g);
+                act_load<kLayout>(kdst, tmK, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                act_load<kLayout>(kdst + kHalfTileBytes, tmK, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
+                act_load<kLayout>(vdst, tmV, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                act_load<kLayout>(vdst + kHalfTileBytes, tmV, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
             }
             issued = w.i + 1;
         }
@@ -643,7 +667,7 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
 
 // wait_state: the S and z images are produced earlier in the same kernel (fused path); loads of them
 // must wait for the Q_SREADY barrier.  Otherwise they were written by a previous launch.
-template <bool kMix>
+template <bool kMix, int kLayout>
 __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
                                             const CUtensorMap* tmW, const CUtensorMap* tmS, bool wait_state)
 {
@@ -711,8 +735,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                         if (passed) {
                             TileWalk pw = w;
                             for (int j = 0; j < kQPrefetchL2 && !pw.done(); ++j, pw.next()) {
-                                tma_prefetch_l2_3d(tmQ, 0, pw.lt * kTile, pw.g);
-                                tma_prefetch_l2_3d(tmQ, 64, pw.lt * kTile, pw.g);
+                                act_prefetch_l2<kLayout>(tmQ, 0, pw.lt * kTile, pw.g, a.H);
+                                act_prefetch_l2<kLayout>(tmQ, 64, pw.lt * kTile, pw.g, a.H);
                             }
                         }
                     }
@@ -725,17 +749,18 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             LA_TRACE(0, 24 + w.i, 0);
             if (lane == 0) {
                 mbar_arrive_expect_tx(c.bar(Q_FULL + r.s), kTileBytes);
-                tma_load_3d(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g);
-                tma_load_3d(sbase + r.s * kTileBytes + kHalfTileBytes, tmQ, c.bar(Q_FULL + r.s), 64, w.lt * kTile, w.g);
+                act_load<kLayout>(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                act_load<kLayout>(sbase + r.s * kTileBytes + kHalfTileBytes, tmQ, c.bar(Q_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
             }
             if (kMix) {
                 // Eq. 8: the epilogue will read this tile's rows of the softmax branch's output straight from
                 // global memory a few microseconds from now; start them on their way into L2 (the rows of a tile
                 // are contiguous: 256 lines of 128 bytes, fewer in the ragged tail tile)
                 const int rows = min(kTile, a.n - w.lt * kTile);
-                const char* base = reinterpret_cast<const char*>(a.mix_src + ((size_t)w.g * a.n + (size_t)w.lt * kTile) * kD);
-                for (int line = lane; line < rows * 2; line += 32)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (size_t)line * 128));
+                const __nv_bfloat16* base = a.mix_src + (size_t)(w.g / a.H) * a.str_batch + (size_t)(w.g % a.H) * a.str_head +
+                                            (size_t)w.lt * kTile * a.str_token;
+                for (int line = lane; line < rows * 2; line += 32)   // two 128-byte lines per row of 128 bf16
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (size_t)(line >> 1) * a.str_token + (line & 1) * 64));
             }
             issued = w.i + 1;
         }
@@ -798,8 +823,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(Q_OFULL + r.s), r.ph, c.wc, kErrStore)) break;
             if (lane == 0) {
-                tma_store_3d(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g);
-                tma_store_3d(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g);
+                act_store<kLayout>(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g, a.H);
+                act_store<kLayout>(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g, a.H);
                 bulk_commit_group();
                 bulk_wait_group_read<0>();
                 mbar_arrive(c.bar(Q_EMPTY + r.s));
@@ -850,7 +875,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             constexpr bool mix = kMix;   // compile-time: the plain forward carries none of the blend's registers
             const bool in_range = w.lt * kTile + row < a.n;
             const uint4* mrow = reinterpret_cast<const uint4*>(
-                a.mix_src + ((size_t)w.g * a.n + (size_t)(w.lt * kTile + (in_range ? row : 0))) * kD);
+                a.mix_src + (size_t)(w.g / a.H) * a.str_batch + (size_t)(w.g % a.H) * a.str_head +
+                (size_t)(w.lt * kTile + (in_range ? row : 0)) * a.str_token);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint4 av[8];
@@ -915,13 +941,14 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
 // Kernels
 // ======================================================================================================
 
+template <int kLayout>
 __global__ void __launch_bounds__(kThreads, 1)
 kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
          const __grid_constant__ CUtensorMap tmW, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, true, false);
-    kside_phase(c, a, &tmK, &tmV, &tmW);
+    kside_phase<kLayout>(c, a, &tmK, &tmV, &tmW);
     cta_teardown(c);
 }
 
@@ -932,14 +959,14 @@ static __global__ void __launch_bounds__(256) combine_tc(const Args a, long long
     if (q4 < kE / 4) combine_quad(a, P, blockIdx.y, q4 * 4);
 }
 
-template <bool kMix>
+template <bool kMix, int kLayout>
 __global__ void __launch_bounds__(kThreads, 1)
 qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
          const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, false, true);
-    qside_phase<kMix>(c, a, &tmQ, &tmO, &tmW, &tmS, false);
+    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmW, &tmS, false);
     cta_teardown(c);
 }
 
@@ -961,7 +988,7 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target)
 }
 
 // The whole forward in one cooperative launch of P <= #SMs persistent CTAs.
-template <bool kMix>
+template <bool kMix, int kLayout>
 __global__ void __launch_bounds__(kThreads, 1)
 linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmQ,
@@ -972,7 +999,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     LA_TRACE_NS(0, 60, 0);
     const Cta c = cta_setup(smem_raw, a, true, true);
     LA_TRACE_NS(0, 60, 1);
-    kside_phase(c, a, &tmK, &tmV, &tmWk);
+    kside_phase<kLayout>(c, a, &tmK, &tmV, &tmWk);
     // every role is done with the key-side buffers; the partials of this CTA are written
     tcgen05_fence_before();
     __syncthreads();
@@ -1013,7 +1040,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (c.warp >= 12 && c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
-    qside_phase<kMix>(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
+    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
     LA_TRACE_NS(0, 61, 2);
     cta_teardown(c);
     LA_TRACE_NS(0, 61, 3);

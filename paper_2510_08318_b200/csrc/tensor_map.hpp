@@ -43,4 +43,22 @@ inline bool make_tmap_bf16_3d(CUtensorMap* map, const void* base, uint64_t cols,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 activations [batch][head][token][feature] in any memory order with the feature dimension contiguous:
+// a rank-4 map (feature, token, head, batch) with the byte strides of token, head and batch; tiles of box_rows
+// tokens x 64 features of one (batch, head), 128-byte swizzle; tokens past n read as zero and are not written.
+// `base` must be 16-byte aligned and every stride a multiple of 16 bytes.  Returns false on failure.
+inline bool make_tmap_bf16_act(CUtensorMap* map, const void* base, uint64_t d, uint64_t n, uint64_t H, uint64_t B,
+                               uint64_t stride_token, uint64_t stride_head, uint64_t stride_batch, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {d, n, H, B};
+    const cuuint64_t strides[3] = {stride_token, stride_head, stride_batch};
+    const cuuint32_t box[4] = {64, box_rows, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace linattn
