@@ -219,7 +219,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     }
     if (Pk + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
 
-    CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmS;
+    CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmS, tmA;   // tmA: the softmax branch's output (mixed attention), else a copy of tmQ
     const ActStrides as = act_strides(c, n);
     const int layout = c->opt_layout;
     auto act_map = [&](CUtensorMap* m, const void* base) {
@@ -227,7 +227,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         return make_tmap_bf16_act(m, base, kD, (uint64_t)n, (uint64_t)c->H, (uint64_t)B, (uint64_t)as.token * 2,
                                   (uint64_t)as.head * 2, (uint64_t)as.batch * 2, kTile);
     };
-    const bool ok = act_map(&tmK, k) && act_map(&tmV, v) && act_map(&tmQ, q) && act_map(&tmO, out) &&
+    const bool ok = act_map(&tmK, k) && act_map(&tmV, v) && act_map(&tmQ, q) && act_map(&tmO, out) && act_map(&tmA, mix ? mix : q) &&
                     make_tmap_bf16_3d(&tmWk, c->Wkt, kD, kM, (uint64_t)c->H, kM) &&
                     make_tmap_bf16_3d(&tmWq, c->Wqt, kD, kM, (uint64_t)c->H, kM) &&
                     make_tmap_bf16_3d(&tmS, c->s_img, kD, kD, (uint64_t)G, kTile);
@@ -279,7 +279,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         a.bar_target[0] = c->bar_total + (uint32_t)Pq;
         a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
         c->bar_total += 2u * (uint32_t)Pq;
-        void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &a};
+        void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
         LA_CUDA(c, cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads), params,
                                                Smem::kTotal, st));
         prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
@@ -296,7 +296,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_tc", 0.0);
     {
-        void* qp[] = {&tmQ, &tmO, &tmWq, &tmS, &a};
+        void* qp[] = {&tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
         LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
     }
     LA_CUDA(c, cudaGetLastError());

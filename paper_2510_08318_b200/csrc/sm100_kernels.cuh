@@ -336,8 +336,8 @@ enum : int {
     K_FULL = 0, K_EMPTY = 3, K_UFULL = 6, K_UEMPTY = 8, K_PHIFULL = 10, K_WFULL = 13, K_WFREE = 15, K_ACCFULL = 17, K_ACCFREE = 19,
     // query side
     Q_FULL = 21, Q_EMPTY = 26, Q_PHIFULL = 31, Q_OFULL = 36, Q_UFULL = 41, Q_UEMPTY = 43, Q_DFULL = 45, Q_DEMPTY = 47,
-    Q_SEGFULL = 49, Q_SEGFREE = 50, Q_SREADY = 51, Q_WFULL = 52,
-    NBARS = 53
+    Q_SEGFULL = 49, Q_SEGFREE = 50, Q_SREADY = 51, Q_WFULL = 52, Q_AFULL = 53,
+    NBARS = 58
 };
 
 struct Cta {
@@ -389,7 +389,7 @@ __device__ __forceinline__ Cta cta_setup(uint8_t* smem_raw, const Args& a, bool 
             for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_ACCFULL + i), 1); mbar_init(c.bar(K_ACCFREE + i), 4); }
         }
         if (init_q) {
-            for (int i = 0; i < kQStages; ++i) { mbar_init(c.bar(Q_FULL + i), 1); mbar_init(c.bar(Q_EMPTY + i), 1); mbar_init(c.bar(Q_PHIFULL + i), 8); mbar_init(c.bar(Q_OFULL + i), 4); }
+            for (int i = 0; i < kQStages; ++i) { mbar_init(c.bar(Q_FULL + i), 1); mbar_init(c.bar(Q_EMPTY + i), 1); mbar_init(c.bar(Q_PHIFULL + i), 8); mbar_init(c.bar(Q_OFULL + i), 4); mbar_init(c.bar(Q_AFULL + i), 1); }
             for (int i = 0; i < 2; ++i) { mbar_init(c.bar(Q_UFULL + i), 1); mbar_init(c.bar(Q_UEMPTY + i), 8); mbar_init(c.bar(Q_DFULL + i), 1); mbar_init(c.bar(Q_DEMPTY + i), 4); }
             mbar_init(c.bar(Q_SEGFULL), 1);
             mbar_init(c.bar(Q_SEGFREE), 1);
@@ -669,7 +669,7 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
 // must wait for the Q_SREADY barrier.  Otherwise they were written by a previous launch.
 template <bool kMix, int kLayout>
 __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
-                                            const CUtensorMap* tmW, const CUtensorMap* tmS, bool wait_state)
+                                            const CUtensorMap* tmW, const CUtensorMap* tmS, const CUtensorMap* tmA, bool wait_state)
 {
     const uint32_t tmem_u = c.tmem;  // 2 x 64 columns of logits
     auto tmem_num = [&](int db) { return c.tmem + 128 + db * 160; };   // 144 columns: num[token][c], c = 0..127, then
@@ -870,20 +870,20 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             tcgen05_fence_after();
             uint32_t dv[2];
             tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
-            // Eq. 8 (mixed attention): this token's row of the softmax branch's output, read straight from global
-            // memory (the row is 256 contiguous bytes; rows past the end of the sequence are not touched)
-            constexpr bool mix = kMix;   // compile-time: the plain forward carries none of the blend's registers
-            const bool in_range = w.lt * kTile + row < a.n;
-            const uint4* mrow = reinterpret_cast<const uint4*>(
-                a.mix_src + (size_t)(w.g / a.H) * a.str_batch + (size_t)(w.g % a.H) * a.str_head +
-                (size_t)(w.lt * kTile + (in_range ? row : 0)) * a.str_token);
+            constexpr bool mix = kMix;   // compile-time: the plain forward carries none of the blend's code
+            if (mix) {
+                // Eq. 8 (mixed attention): the tensor core is done with phi(q) in this slot (that is what the barrier
+                // above says), so the tile of the softmax branch's output is brought into the very same slot by TMA
+                // (its lines are already on their way into L2), blended in place and stored from there.
+                if (warp == 12 && lane == 0) {
+                    mbar_arrive_expect_tx(c.bar(Q_AFULL + r.s), kTileBytes);
+                    act_load<kLayout>(sbase + r.s * kTileBytes, tmA, c.bar(Q_AFULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                    act_load<kLayout>(sbase + r.s * kTileBytes + kHalfTileBytes, tmA, c.bar(Q_AFULL + r.s), 64, w.lt * kTile, w.g, a.H);
+                }
+                if (!warp_wait(c.bar(Q_AFULL + r.s), r.ph, c.wc, kErrEpilogue)) break;
+            }
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                uint4 av[8];
-                if (mix) {
-#pragma unroll
-                    for (int cc = 0; cc < 8; ++cc) av[cc] = in_range ? __ldg(mrow + half * 8 + cc) : make_uint4(0u, 0u, 0u, 0u);
-                }
                 uint32_t v[64];
                 tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64, v);
                 tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64 + 32, v + 32);
@@ -915,7 +915,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                     const f32x2 lin2 = pack2(lin, lin), r2 = pack2(a.mix_r, a.mix_r);
 #pragma unroll
                     for (int cc = 0; cc < 8; ++cc) {
-                        const uint32_t aw4[4] = {av[cc].x, av[cc].y, av[cc].z, av[cc].w};
+                        const uint4 av = *reinterpret_cast<const uint4*>(dst + ((cc ^ sw) << 4));
+                        const uint32_t aw4[4] = {av.x, av.y, av.z, av.w};
                         uint32_t o[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
@@ -962,11 +963,12 @@ static __global__ void __launch_bounds__(256) combine_tc(const Args a, long long
 template <bool kMix, int kLayout>
 __global__ void __launch_bounds__(kThreads, 1)
 qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
-         const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS, const Args a)
+         const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS,
+         const __grid_constant__ CUtensorMap tmA, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, false, true);
-    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmW, &tmS, false);
+    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmW, &tmS, &tmA, false);
     cta_teardown(c);
 }
 
@@ -993,7 +995,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmWq,
-                 const __grid_constant__ CUtensorMap tmS, const Args a)
+                 const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmA, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     LA_TRACE_NS(0, 60, 0);
@@ -1040,7 +1042,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (c.warp >= 12 && c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
-    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmWq, &tmS, true);
+    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmWq, &tmS, &tmA, true);
     LA_TRACE_NS(0, 61, 2);
     cta_teardown(c);
     LA_TRACE_NS(0, 61, 3);
