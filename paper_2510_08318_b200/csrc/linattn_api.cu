@@ -280,11 +280,19 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
         c->bar_total += 2u * (uint32_t)Pq;
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
-        LA_CUDA(c, cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads), params,
-                                               Smem::kTotal, st));
-        prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
-        c->last_launches = 1;
-        return LINATTN_OK;
+        const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads),
+                                                           params, Smem::kTotal, st);
+        if (le == cudaSuccess) {
+            prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
+            c->last_launches = 1;
+            return LINATTN_OK;
+        }
+        if (le != cudaErrorCooperativeLaunchTooLarge) return cuda_fail(c, le, "cudaLaunchCooperativeKernel");
+        // Not all CTAs can be resident at once (part of the GPU is taken, e.g. MIG or MPS limits): nothing was
+        // launched; use the three-launch form from now on, which needs no co-residency.
+        cudaGetLastError();
+        c->bar_total -= 2u * (uint32_t)Pq;
+        c->coop_ok = false;
     }
     {
         void* kp[] = {&tmK, &tmV, &tmWk, &a};
