@@ -1,2 +1,2 @@
 """fp64 CPU oracle (test infrastructure; the product never imports this package)."""
-from .ref import build, phi, ref_linear, ref_mix, ref_quadratic, ref_softmax, threads  # noqa: F401
+from .ref import build, phi, ref_backward, ref_linear, ref_mix, ref_quadratic, ref_softmax, threads  # noqa: F401

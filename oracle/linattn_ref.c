@@ -279,3 +279,114 @@ int linattn_ref_mix(const double *o_softmax, const double *o_linear, long count,
     for (long e = 0; e < count; ++e) out[e] = rc * o_softmax[e] + (1.0 - rc) * o_linear[e];
     return 0;
 }
+
+/*
+ * Gradients of the operator (what the post-training objective of Eq. 14 back-propagates through every
+ * linear-attention layer): for L = sum_{i,c} dO[i][c] * o_i[c] with o from the right form of Eq. 5 and
+ * phi from Eq. 6, the derivatives of L with respect to q, k, v, W_q and W_k, by the chain rule written out:
+ *
+ *   dnum_i = dO_i / den_i                      dden_i = -(dO_i . o_i) / den_i
+ *   dphi(q_i) = S dnum_i + dden_i z            dS = sum_i phi(q_i)^T dnum_i        dz = sum_i dden_i phi(q_i)
+ *   dphi(k_j) = dS v_j + dz                    dv_j = dS^T phi(k_j)
+ *   through phi (two softmaxes p+ = softmax(u), p- = softmax(-u), u = x W):
+ *       du = p+ (.) (dphi+ - p+ . dphi+)  -  p- (.) (dphi- - p- . dphi-)
+ *       dx = du W^T                            dW += x^T du
+ *
+ * dW_q, dW_k are summed over the batch (groups g with the same head g % H) and, when per_head == 0, over the
+ * heads as well.  All arrays [G][n][d] except dWq, dWk: [H][d][d/2] (per_head) or [d][d/2].  Outputs in double.
+ */
+static void phi_backward_row(const float *x, const float *W, int d, const double *phi, const double *dphi,
+                             double *dx, double *dW)
+{
+    const int m = d / 2;
+    double dotp = 0.0, dotn = 0.0;
+    for (int j = 0; j < m; ++j) {
+        dotp += phi[j] * dphi[j];
+        dotn += phi[m + j] * dphi[m + j];
+    }
+    for (int c = 0; c < d; ++c) dx[c] = 0.0;
+    for (int j = 0; j < m; ++j) {
+        const double du = phi[j] * (dphi[j] - dotp) - phi[m + j] * (dphi[m + j] - dotn);
+        for (int c = 0; c < d; ++c) {
+            dx[c] += du * (double)W[(size_t)c * m + j];
+            dW[(size_t)c * m + j] += (double)x[c] * du;
+        }
+    }
+}
+
+int linattn_ref_backward(const float *q, const float *k, const float *v, const float *Wq, const float *Wk,
+                         const float *dout, long G, int H, long n, int d, int per_head,
+                         double *dq, double *dk, double *dv, double *dWq, double *dWk)
+{
+    if (d < 2 || d > 4096 || (d & 1) || n < 1 || G < 1 || H < 1) return 1;
+    const int m = d / 2;
+    const size_t wsz = (size_t)d * m;
+    const long nW = per_head ? H : 1;
+    for (size_t e = 0; e < (size_t)nW * wsz; ++e) dWq[e] = dWk[e] = 0.0;
+    int fail = 0;
+    /* one group at a time (the weight gradients are shared between groups, so no threading across groups) */
+    for (long g = 0; g < G && !fail; ++g) {
+        const float *qg = q + (size_t)g * n * d, *kg = k + (size_t)g * n * d, *vg = v + (size_t)g * n * d;
+        const float *gg = dout + (size_t)g * n * d;
+        const float *wq = w_of(Wq, (int)g, H, d, per_head), *wk = w_of(Wk, (int)g, H, d, per_head);
+        double *dwq = dWq + (per_head ? (size_t)(g % H) * wsz : 0), *dwk = dWk + (per_head ? (size_t)(g % H) * wsz : 0);
+        double *S = (double *)calloc((size_t)d * d, sizeof(double)), *z = (double *)calloc(d, sizeof(double));
+        double *dS = (double *)calloc((size_t)d * d, sizeof(double)), *dz = (double *)calloc(d, sizeof(double));
+        double *phi = (double *)malloc((size_t)d * sizeof(double)), *dphi = (double *)malloc((size_t)d * sizeof(double));
+        double *o = (double *)malloc((size_t)d * sizeof(double)), *dnum = (double *)malloc((size_t)d * sizeof(double));
+        if (!S || !z || !dS || !dz || !phi || !dphi || !o || !dnum) {
+            fail = 1;
+        } else {
+            /* forward state */
+            for (long j = 0; j < n; ++j) {
+                phi_row(kg + (size_t)j * d, wk, d, phi);
+                for (int f = 0; f < d; ++f) {
+                    z[f] += phi[f];
+                    for (int c = 0; c < d; ++c) S[(size_t)f * d + c] += phi[f] * (double)vg[(size_t)j * d + c];
+                }
+            }
+            /* query side: dq, dWq, and the gradients of the state */
+            for (long i = 0; i < n; ++i) {
+                phi_row(qg + (size_t)i * d, wq, d, phi);
+                double den = 0.0;
+                for (int f = 0; f < d; ++f) den += phi[f] * z[f];
+                double go = 0.0;
+                for (int c = 0; c < d; ++c) {
+                    double num = 0.0;
+                    for (int f = 0; f < d; ++f) num += phi[f] * S[(size_t)f * d + c];
+                    o[c] = num / den;
+                    go += (double)gg[(size_t)i * d + c] * o[c];
+                    dnum[c] = (double)gg[(size_t)i * d + c] / den;
+                }
+                const double dden = -go / den;
+                for (int f = 0; f < d; ++f) {
+                    double acc = dden * z[f];
+                    for (int c = 0; c < d; ++c) {
+                        acc += S[(size_t)f * d + c] * dnum[c];
+                        dS[(size_t)f * d + c] += phi[f] * dnum[c];
+                    }
+                    dphi[f] = acc;
+                    dz[f] += dden * phi[f];
+                }
+                phi_backward_row(qg + (size_t)i * d, wq, d, phi, dphi, dq + ((size_t)g * n + i) * d, dwq);
+            }
+            /* key side: dk, dv, dWk */
+            for (long j = 0; j < n; ++j) {
+                phi_row(kg + (size_t)j * d, wk, d, phi);
+                double *dvj = dv + ((size_t)g * n + j) * d;
+                for (int c = 0; c < d; ++c) dvj[c] = 0.0;
+                for (int f = 0; f < d; ++f) {
+                    double acc = dz[f];
+                    for (int c = 0; c < d; ++c) {
+                        acc += dS[(size_t)f * d + c] * (double)vg[(size_t)j * d + c];
+                        dvj[c] += phi[f] * dS[(size_t)f * d + c];
+                    }
+                    dphi[f] = acc;
+                }
+                phi_backward_row(kg + (size_t)j * d, wk, d, phi, dphi, dk + ((size_t)g * n + j) * d, dwk);
+            }
+        }
+        free(S); free(z); free(dS); free(dz); free(phi); free(dphi); free(o); free(dnum);
+    }
+    return fail;
+}

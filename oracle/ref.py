@@ -50,6 +50,8 @@ def _load():
         lib.linattn_ref_softmax.argtypes = [fp, fp, fp, ctypes.c_long, ctypes.c_long, ctypes.c_int, ctypes.c_double,
                                             lp, ctypes.c_long, dp]
         lib.linattn_ref_mix.argtypes = [dp, dp, ctypes.c_long, ctypes.c_double, dp]
+        lib.linattn_ref_backward.argtypes = [fp, fp, fp, fp, fp, fp, ctypes.c_long, ctypes.c_int, ctypes.c_long,
+                                             ctypes.c_int, ctypes.c_int, dp, dp, dp, dp, dp]
         _lib = lib
     return _lib
 
@@ -164,3 +166,20 @@ def ref_mix(o_softmax, o_linear, r: float) -> np.ndarray:
     if _load().linattn_ref_mix(_ptr(a, D), _ptr(b, D), a.size, float(r), _ptr(out, D)):
         raise ValueError("oracle rejected the arguments")
     return out
+
+
+def ref_backward(q, k, v, Wq, Wk, dout):
+    """Gradients of sum(dout * o) with respect to q, k, v, Wq, Wk (o = right form of Eq. 5 with the phi of Eq. 6).
+    Returns float64 (dq, dk, dv, dWq, dWk); the weight gradients have the shape of the weights."""
+    q, k, v, Wq, Wk, B, H, n, d, per_head = _prep(q, k, v, Wq, Wk)
+    g = _f32(dout)
+    assert g.shape == q.shape
+    dq, dk, dv = (np.empty(q.shape, dtype=np.float64) for _ in range(3))
+    dWq, dWk = (np.empty(Wq.shape, dtype=np.float64) for _ in range(2))
+    F, D = ctypes.c_float, ctypes.c_double
+    rc = _load().linattn_ref_backward(_ptr(q, F), _ptr(k, F), _ptr(v, F), _ptr(Wq, F), _ptr(Wk, F), _ptr(g, F),
+                                      B * H, H, n, d, per_head, _ptr(dq, D), _ptr(dk, D), _ptr(dv, D),
+                                      _ptr(dWq, D), _ptr(dWk, D))
+    if rc:
+        raise ValueError("oracle rejected the arguments or ran out of memory")
+    return dq, dk, dv, dWq, dWk

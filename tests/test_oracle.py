@@ -288,3 +288,69 @@ def test_mix_is_affine_in_the_clipped_score():
         np.testing.assert_allclose(oracle.ref_mix(a, b, r), m0 + r * (m1 - m0), rtol=1e-13, atol=1e-14)
     np.testing.assert_array_equal(oracle.ref_mix(a, b, 3.0), m1)
     np.testing.assert_array_equal(oracle.ref_mix(a, b, -3.0), m0)
+
+
+# ---- gradients (what Eq. 14 back-propagates through the operator) ----------------------------------------
+
+def _torch_forward(q, k, v, Wq, Wk):
+    """The operator in plain torch fp64 (Eq. 5 left form, Eq. 6), written independently of the C oracle so that
+    autograd gives a second opinion on its hand-derived chain rule."""
+    def phi(x, W):
+        u = torch.einsum("bhnd,hdm->bhnm", x, W)
+        return torch.cat([torch.softmax(u, -1), torch.softmax(-u, -1)], -1)
+    a = torch.einsum("bhif,bhjf->bhij", phi(q, Wq), phi(k, Wk))
+    return torch.einsum("bhij,bhjd->bhid", a / a.sum(-1, keepdim=True), v)
+
+
+@pytest.mark.parametrize("B,H,n,d", [(1, 1, 5, 4), (2, 2, 9, 8), (1, 3, 17, 16)])
+def test_backward_matches_autograd_of_an_independent_forward(B, H, n, d):
+    q, k, v, Wq, Wk = _rand(B, H, n, d, seed=50 + n)
+    g = np.random.default_rng(51).standard_normal((B, H, n, d)).astype(np.float32)
+    t = [torch.from_numpy(x).double().requires_grad_(True) for x in (q, k, v, Wq, Wk)]
+    (_torch_forward(*t) * torch.from_numpy(g).double()).sum().backward()
+    got = oracle.ref_backward(q, k, v, Wq, Wk, g)
+    for name, a, b in zip(("dq", "dk", "dv", "dWq", "dWk"), got, t):
+        np.testing.assert_allclose(a, b.grad.numpy(), rtol=1e-9, atol=1e-12, err_msg=name)
+
+
+def test_backward_matches_central_differences_of_the_forward_oracle():
+    """The forward oracle is pinned above; its central differences pin every gradient of the backward oracle."""
+    B, H, n, d = 1, 2, 6, 4
+    q, k, v, Wq, Wk = _rand(B, H, n, d, seed=60)
+    g = np.random.default_rng(61).standard_normal((B, H, n, d))
+    # inputs must be exactly representable in float32 after +-h: use a power of two
+    h = 2.0 ** -10
+    grads = oracle.ref_backward(q, k, v, Wq, Wk, g.astype(np.float32))
+    g32 = g.astype(np.float32).astype(np.float64)
+    args = [q, k, v, Wq, Wk]
+    rng = np.random.default_rng(62)
+    for a_i, (arr, grad) in enumerate(zip(args, grads)):
+        for _ in range(6):
+            idx = tuple(rng.integers(0, s) for s in arr.shape)
+            plus, minus = [x.copy() for x in args], [x.copy() for x in args]
+            plus[a_i][idx] += h
+            minus[a_i][idx] -= h
+            fd = ((oracle.ref_linear(*plus) - oracle.ref_linear(*minus)) * g32).sum() / (2 * h)
+            assert abs(fd - grad[idx]) <= 1e-5 * max(1.0, abs(grad[idx])), (a_i, idx, fd, grad[idx])
+
+
+def test_backward_shared_weights_sum_over_heads_and_invariances():
+    B, H, n, d = 2, 3, 7, 8
+    q, k, v, Wq, Wk = _rand(B, H, n, d, seed=70)
+    g = np.random.default_rng(71).standard_normal((B, H, n, d)).astype(np.float32)
+    shared_q, shared_k = Wq[0].copy(), Wk[0].copy()
+    rep = lambda W: np.broadcast_to(W, (H,) + W.shape).copy()
+    per = oracle.ref_backward(q, k, v, rep(shared_q), rep(shared_k), g)
+    sh = oracle.ref_backward(q, k, v, shared_q, shared_k, g)
+    for a, b in zip(per[:3], sh[:3]):
+        np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(per[3].sum(0), sh[3], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(per[4].sum(0), sh[4], rtol=1e-11, atol=1e-13)
+    # dO = 0 gives all-zero gradients
+    zero = oracle.ref_backward(q, k, v, Wq, Wk, np.zeros_like(g))
+    assert all(np.all(x == 0.0) for x in zero)
+    # and the gradients are linear in dO
+    two = oracle.ref_backward(q, k, v, Wq, Wk, 2.0 * g)
+    one = oracle.ref_backward(q, k, v, Wq, Wk, g)
+    for a, b in zip(two, one):
+        np.testing.assert_allclose(a, 2.0 * b, rtol=1e-12, atol=1e-14)
