@@ -104,6 +104,25 @@ linattn_status linattn_forward_mixed(linattn_ctx* ctx, const void* q, const void
                                      linattn_dtype dtype, void* stream);
 
 /*
+ * Gradients of linattn_forward: what the training objective (Eq. 14) back-propagates through a layer that uses
+ * Eq. 5 with the feature map of Eq. 6.  Given dout = dL/d(out), writes dL/dq, dL/dk, dL/dv and the gradients of
+ * the two feature-map weight matrices.  S and z are recomputed from k, v (no forward needs to precede the call).
+ *   q, k, v, dout : device, as q, k, v of linattn_forward (same layout option), read-only
+ *   dq, dk, dv    : device, same shape, type and layout; written in full; must not overlap any input or each other
+ *   dWq, dWk      : device, fp32, 16-byte aligned, written in full: [H][d][d/2] when per_head != 0 (each head's
+ *                   gradient summed over the batch), [d][d/2] when per_head == 0 (one shared matrix: summed over
+ *                   batch and heads).  The weights differentiated are the ones given to set_feature_map.
+ * Arithmetic is fp32 on the CUDA cores (the stored q, k, v, dout are the only rounded quantities); dq, dk, dv are
+ * rounded once to `dtype`.  All sums have a fixed order: the same inputs give bit-identical gradients.  The first
+ * call allocates the backward workspace (it synchronises the device once); later calls allocate nothing.  After
+ * the call the context holds the S, z of these k, v (linattn_read_state returns them).
+ * Errors: INVALID_ARG, UNSUPPORTED, NO_FEATURE_MAP, WORKSPACE, CUDA.
+ */
+linattn_status linattn_backward(linattn_ctx* ctx, const void* q, const void* k, const void* v, const void* dout,
+                                void* dq, void* dk, void* dv, float* dWq, float* dWk, int per_head,
+                                int B, int H, int n, int d, linattn_dtype dtype, void* stream);
+
+/*
  * The same operation on HOST buffers (pageable or pinned): copies q, k, v to device staging
  * buffers owned by the context, runs linattn_forward, copies the result into `out`, and waits
  * for `stream` before returning.  The staging buffers are allocated (or grown) on the first call
@@ -165,7 +184,7 @@ linattn_status linattn_check(linattn_ctx* ctx, void* stream);
 int linattn_profile_get(linattn_ctx* ctx, int index, const char** name, double* mean_ms, long long* launches,
                         double* algorithmic_bytes);
 
-/* Number of kernels the most recent linattn_forward on this context launched (0 before any). */
+/* Number of kernels the most recent linattn_forward or linattn_backward on this context launched (0 before any). */
 int linattn_last_launch_count(const linattn_ctx* ctx);
 
 /* Text of the last CUDA error seen by this context ("" if none).  Valid until the next call on ctx. */

@@ -11,6 +11,7 @@
 #include <new>
 
 #include "simt_kernels.cuh"
+#include "simt_backward.cuh"
 #include "sm100_kernels.cuh"
 #include "tensor_map.hpp"
 
@@ -59,6 +60,10 @@ struct linattn_ctx {
     long long partial_slots = 0;
     float* state = nullptr;     // [max_B*H][d*d + d]
     unsigned int* err_word = nullptr;
+    // workspace of the backward pass, allocated by the first linattn_backward
+    float* bwd_part_state = nullptr;  // [partial_slots][d*d + d]  per-block sums of dS, dz
+    float* bwd_part_w = nullptr;      // [partial_slots][d*d/2]    per-block sums of dW
+    float* bwd_dstate = nullptr;      // [max_B*H][d*d + d]        dS, dz
     // host-call staging
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     size_t stage_bytes = 0;
@@ -68,7 +73,7 @@ struct linattn_ctx {
     int opt_fuse = 1;
     int opt_layout = 0;   // 0: [B][H][n][d], 1: [B][n][H][d]
     // per-kernel timing (LINATTN_OPT_PROFILE)
-    static constexpr int kMaxKernels = 4;
+    static constexpr int kMaxKernels = 8;
     bool profile = false;
     bool prof_pending = false;
     int prof_n = 0;                       // kernels in the forward being timed
@@ -200,6 +205,62 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_simt", side_bytes);
     c->last_launches = 3;
+    return LINATTN_OK;
+}
+
+// Gradients on the CUDA-core kernels: S, z as in the forward, then the query side (dq, dS, dz, dW_q), then the key
+// side (dk, dv, dW_k).
+template <typename T, int D>
+linattn_status launch_backward_simt(linattn_ctx* c, const void* q, const void* k, const void* v, const void* dout, void* dq,
+                                    void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int n, cudaStream_t st)
+{
+    const long long G = (long long)B * c->H;
+    int splits = choose_splits(G, n, c->opt_splits);
+    int chunk = (n + splits - 1) / splits;
+    chunk = (chunk + kSimtTokens - 1) / kSimtTokens * kSimtTokens;
+    splits = (n + chunk - 1) / chunk;
+    const int nchunks = (n + kSimtTokens - 1) / kSimtTokens;
+    long long blocks = (kTargetCtas + G - 1) / G;   // blocks per (b,h) of the two gradient kernels
+    if (blocks > nchunks) blocks = nchunks;
+    if (G * splits > c->partial_slots || G * blocks > c->partial_slots) return LINATTN_ERR_WORKSPACE;
+    constexpr int E = D * D + D, DM = D * (D / 2);
+
+    static bool attr_done = false;
+    if (!attr_done) {
+        LA_CUDA(c, cudaFuncSetAttribute(kside_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kside_simt_smem<D>()));
+        LA_CUDA(c, cudaFuncSetAttribute(qside_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bwd_smem<D>()));
+        LA_CUDA(c, cudaFuncSetAttribute(kside_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bwd_smem<D>()));
+        attr_done = true;
+    }
+    const ActStrides as = act_strides(c, n);
+    const double tensor_bytes = (double)G * n * D * sizeof(T);
+    const dim3 grid((unsigned)blocks, (unsigned)G);
+    prof_begin(c, st);
+    kside_simt<T, D><<<dim3(splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
+        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, as);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "kside_simt", 2.0 * tensor_bytes);
+    combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, c->state, splits, E);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "combine_state", 0.0);
+    qside_bwd<T, D><<<grid, kSimtThreads, bwd_smem<D>(), st>>>((const T*)q, (const T*)dout, c->Wq, c->state, (T*)dq,
+                                                              c->bwd_part_state, c->bwd_part_w, c->H, n, as);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "qside_bwd", 3.0 * tensor_bytes);
+    combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->bwd_part_state, c->bwd_dstate, (int)blocks, E);
+    LA_CUDA(c, cudaGetLastError());
+    const dim3 wgrid((DM + 255) / 256, per_head ? (unsigned)c->H : 1u);
+    combine_wgrad<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWq, (int)blocks, (int)G, c->H, DM, per_head);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "combine_dstate_dWq", 0.0);
+    kside_bwd<T, D><<<grid, kSimtThreads, bwd_smem<D>(), st>>>((const T*)k, (const T*)v, c->Wk, c->bwd_dstate, (T*)dk, (T*)dv,
+                                                              c->bwd_part_w, c->H, n, as);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "kside_bwd", 4.0 * tensor_bytes);
+    combine_wgrad<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWk, (int)blocks, (int)G, c->H, DM, per_head);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "combine_dWk", 0.0);
+    c->last_launches = 7;
     return LINATTN_OK;
 }
 
@@ -426,6 +487,9 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->Wkt);
     cudaFree(c->s_img);
     cudaFree(c->z_img);
+    cudaFree(c->bwd_part_state);
+    cudaFree(c->bwd_part_w);
+    cudaFree(c->bwd_dstate);
     for (void* p : c->stage) cudaFree(p);
     for (cudaEvent_t ev : c->prof_ev)
         if (ev) cudaEventDestroy(ev);
@@ -512,6 +576,45 @@ linattn_status linattn_forward_mixed(linattn_ctx* c, const void* q, const void* 
 {
     if (!o_softmax) return LINATTN_ERR_INVALID_ARG;
     return forward_impl(c, q, k, v, out, o_softmax, r, B, H, n, d, dtype, stream);
+}
+
+linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, const void* v, const void* dout, void* dq,
+                                void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int H, int n, int d,
+                                linattn_dtype dtype, void* stream)
+{
+    if (!dout || !dk || !dv || !dWq || !dWk) return LINATTN_ERR_INVALID_ARG;
+    linattn_status s = check_forward_args(c, q, k, v, dq, B, H, n, d, dtype);
+    if (s != LINATTN_OK) return s;
+    const void* ins[4] = {q, k, v, dout};
+    void* outs[3] = {dq, dk, dv};
+    const size_t bytes = (size_t)B * H * n * d * elem_size(dtype);
+    for (const void* p : ins)
+        if (misaligned16(p)) return LINATTN_ERR_INVALID_ARG;
+    for (int i = 0; i < 3; ++i) {
+        if (misaligned16(outs[i])) return LINATTN_ERR_INVALID_ARG;
+        for (const void* p : ins)
+            if (overlaps(outs[i], p, bytes)) return LINATTN_ERR_INVALID_ARG;
+        for (int j = 0; j < i; ++j)
+            if (overlaps(outs[i], outs[j], bytes)) return LINATTN_ERR_INVALID_ARG;
+    }
+    if (misaligned16(dWq) || misaligned16(dWk) || dWq == dWk) return LINATTN_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!c->bwd_dstate) {
+        const size_t E = (size_t)d * d + d;
+        LA_CUDA(c, cudaMalloc(&c->bwd_part_state, sizeof(float) * E * (size_t)c->partial_slots));
+        LA_CUDA(c, cudaMalloc(&c->bwd_part_w, sizeof(float) * (size_t)d * (d / 2) * (size_t)c->partial_slots));
+        LA_CUDA(c, cudaMalloc(&c->bwd_dstate, sizeof(float) * E * (size_t)(c->max_B * c->H)));
+    }
+    c->last_B = B;
+    c->state_transposed = false;
+    const int ph = per_head ? 1 : 0;
+    if (dtype == LINATTN_BF16) {
+        return d == 128 ? launch_backward_simt<__nv_bfloat16, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st)
+                        : launch_backward_simt<__nv_bfloat16, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
+    }
+    return d == 128 ? launch_backward_simt<float, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st)
+                    : launch_backward_simt<float, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
 }
 
 linattn_status linattn_forward_host(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B,

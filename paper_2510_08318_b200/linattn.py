@@ -29,6 +29,7 @@ SIGNATURES = {
     "linattn_set_feature_map": (_i, [_vp, _vp, _vp, _i, _i, _vp]),
     "linattn_forward": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_mixed": (_i, [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i, _i, _i, _i, _i, _vp]),
+    "linattn_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_host": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_noalloc": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "linattn_read_state": (_i, [_vp, _vp, _vp, _i, _vp]),
@@ -157,6 +158,23 @@ class LinAttn:
         self._call(self._lib.linattn_forward_mixed, q.data_ptr(), k.data_ptr(), v.data_ptr(), o_softmax.data_ptr(),
                    float(r), out.data_ptr(), B, H, n, d, _DTYPES[q.dtype], _stream_ptr(stream))
         return out
+
+    def backward(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, dout: torch.Tensor, per_head: bool = True,
+                 stream=None):
+        """Gradients of ``forward``: returns (dq, dk, dv, dWq, dWk); dq, dk, dv like q, the weight gradients fp32
+        [H, d, d/2] (``per_head``) or [d, d/2] (one shared matrix)."""
+        for t in (q, k, v, dout):
+            assert t.is_cuda and t.is_contiguous()
+        assert q.shape == k.shape == v.shape == dout.shape and q.dtype == k.dtype == v.dtype == dout.dtype
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+        wshape = (self.H, self.d, self.d // 2) if per_head else (self.d, self.d // 2)
+        dWq = torch.empty(wshape, dtype=torch.float32, device=q.device)
+        dWk = torch.empty(wshape, dtype=torch.float32, device=q.device)
+        B, H, n, d = q.shape
+        self._call(self._lib.linattn_backward, q.data_ptr(), k.data_ptr(), v.data_ptr(), dout.data_ptr(), dq.data_ptr(),
+                   dk.data_ptr(), dv.data_ptr(), dWq.data_ptr(), dWk.data_ptr(), 1 if per_head else 0, B, H, n, d,
+                   _DTYPES[q.dtype], _stream_ptr(stream))
+        return dq, dk, dv, dWq, dWk
 
     def forward_host(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
                      stream=None) -> torch.Tensor:

@@ -1,0 +1,146 @@
+"""GPU parity of linattn_backward against the oracle's gradients (the chain rule through Eq. 5 and Eq. 6, which
+is what the objective of Eq. 14 back-propagates through a linear-attention layer).
+
+Both sides get the same stored (rounded) q, k, v, dO and weights.  Gradients have no natural scale (dv is of
+order |dO| / n), so the absolute bound is taken relative to the largest reference entry: relative L2 <= 5e-3
+over each gradient tensor and max-abs <= 2e-2 * max|reference|.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_08318_b200 import linattn
+from util import errors
+
+pytestmark = pytest.mark.gpu
+
+NAMES = ("dq", "dk", "dv", "dWq", "dWk")
+
+
+def _inputs(B, H, n, d, dtype, seed, shared=False):
+    g = torch.Generator().manual_seed(seed)
+    sx = 1.0 / math.sqrt(d)
+    q, k, v = (torch.randn(B, H, n, d, generator=g) * sx for _ in range(3))
+    wshape = (d, d // 2) if shared else (H, d, d // 2)
+    Wq, Wk = (torch.randn(*wshape, generator=g) / (math.sqrt(d) * sx) for _ in range(2))
+    dout = torch.randn(B, H, n, d, generator=g)
+    return {"q": q.to(dtype), "k": k.to(dtype), "v": v.to(dtype), "Wq": Wq.to(dtype), "Wk": Wk.to(dtype),
+            "dout": dout.to(dtype)}
+
+
+def _assert_grads(got, want, what):
+    for name, a, b in zip(NAMES, got, want):
+        a = a.detach().cpu().double().numpy()
+        assert np.isfinite(a).all(), f"{what}: {name} has non-finite entries"
+        rel, mx = errors(a, b)
+        scale = float(np.abs(b).max())
+        assert rel <= 5e-3 and mx <= 2e-2 * scale, f"{what}: {name} rel-L2 {rel:.3e}, max-abs {mx:.3e} (largest reference entry {scale:.3e})"
+
+
+def _run(x, per_head=True, layout=linattn.LAYOUT_BHND):
+    B, H, n, d = x["q"].shape
+    ctx = linattn.LinAttn(H, d, max_B=B, max_n=n)
+    try:
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        ctx.set_option(linattn.OPT_LAYOUT, layout)
+        args = [x[s].cuda() for s in ("q", "k", "v", "dout")]
+        if layout == linattn.LAYOUT_BNHD:
+            args = [t.permute(0, 2, 1, 3).contiguous().view(B, H, n, d) for t in args]
+        got = ctx.backward(*args, per_head=per_head)
+        again = ctx.backward(*args, per_head=per_head)
+        ctx.check()
+        assert ctx.last_launch_count() == 7
+        for a, b in zip(got, again):
+            assert torch.equal(a, b), "the gradients are not bit-reproducible"
+        if layout == linattn.LAYOUT_BNHD:
+            got = tuple(t.view(B, n, H, d).permute(0, 2, 1, 3) for t in got[:3]) + tuple(got[3:])
+        return got, ctx.read_state(B)
+    finally:
+        ctx.destroy()
+
+
+@pytest.mark.parametrize("B,H,n,d,dtype", [
+    (2, 2, 300, 64, torch.float32),      # several chunks and a ragged tail
+    (1, 3, 257, 128, torch.float32),
+    (2, 2, 1000, 128, torch.bfloat16),
+    (1, 2, 129, 64, torch.bfloat16),
+    (1, 1, 1, 128, torch.float32),       # one token: o = v, so dq = dk = 0 and dv = dO
+    (3, 1, 31, 64, torch.float32),       # less than one chunk
+    (1, 12, 2048, 128, torch.bfloat16),  # the small workload's shape
+])
+def test_gradients_match_the_oracle(B, H, n, d, dtype):
+    x = _inputs(B, H, n, d, dtype, seed=200 + n)
+    want = oracle.ref_backward(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], x["dout"])
+    got, (S, z) = _run(x)
+    if n == 1:
+        # o = v whatever q and k are: every gradient but dv vanishes, so only absolute checks make sense
+        for name, t in zip(NAMES, got):
+            if name != "dv":
+                assert float(t.abs().max()) <= 1e-5, f"{name} must vanish for a single token"
+        assert torch.allclose(got[2].cpu().float(), x["dout"].float(), rtol=1e-6, atol=0)
+        assert np.abs(want[2] - x["dout"].double().numpy()).max() <= 1e-12
+        return
+    _assert_grads(got, want, f"B={B} H={H} n={n} d={d} {dtype}")
+    # the call leaves the forward state of these k, v in the context
+    _, S_ref, z_ref = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], rows=np.array([0]), return_state=True)
+    assert errors(S.double().numpy(), S_ref)[0] <= 5e-3 and errors(z.double().numpy(), z_ref)[0] <= 5e-3
+
+
+def test_shared_feature_map_sums_the_weight_gradients_over_heads():
+    x = _inputs(2, 3, 200, 64, torch.float32, seed=31, shared=True)
+    want = oracle.ref_backward(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], x["dout"])
+    got, _ = _run(x, per_head=False)
+    assert tuple(got[3].shape) == (64, 32)
+    _assert_grads(got, want, "shared map")
+
+
+def test_token_major_layout():
+    x = _inputs(2, 3, 333, 128, torch.bfloat16, seed=32)
+    ref, _ = _run(x)
+    got, _ = _run(x, layout=linattn.LAYOUT_BNHD)
+    for name, a, b in zip(NAMES, got, ref):
+        assert torch.equal(a, b), f"{name}: the [B][n][H][d] layout must give the same bits"
+
+
+def test_heavy_tailed_keys():
+    """Keys with a few large entries (the recipe of the heavy-tailed workload) make phi(k) nearly one-hot."""
+    x = _inputs(1, 2, 600, 128, torch.bfloat16, seed=33)
+    g = torch.Generator().manual_seed(34)
+    k = x["k"].float()
+    mask = torch.rand(k.shape, generator=g) < 0.01
+    x["k"] = torch.where(mask, k * 12.0, k).to(torch.bfloat16)
+    want = oracle.ref_backward(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], x["dout"])
+    got, _ = _run(x)
+    _assert_grads(got, want, "heavy-tailed keys")
+
+
+def test_argument_errors():
+    lib = linattn.load_library()
+    x = _inputs(1, 2, 128, 64, torch.float32, seed=35)
+    ctx = linattn.LinAttn(2, 64, max_B=1, max_n=128)
+    try:
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        q, k, v, g = (x[s].cuda() for s in ("q", "k", "v", "dout"))
+        dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+        dWq, dWk = (torch.empty(2, 64, 32, device="cuda") for _ in range(2))
+
+        def call(**kw):
+            a = dict(q=q.data_ptr(), k=k.data_ptr(), v=v.data_ptr(), g=g.data_ptr(), dq=dq.data_ptr(), dk=dk.data_ptr(),
+                     dv=dv.data_ptr(), dWq=dWq.data_ptr(), dWk=dWk.data_ptr(), n=128)
+            a.update(kw)
+            return lib.linattn_backward(ctx._h, a["q"], a["k"], a["v"], a["g"], a["dq"], a["dk"], a["dv"], a["dWq"],
+                                        a["dWk"], 1, 1, 2, a["n"], 64, linattn.F32, None)
+        assert call() == linattn.OK
+        assert call(g=None) == linattn.ERR_INVALID_ARG
+        assert call(dWk=None) == linattn.ERR_INVALID_ARG
+        assert call(dk=dq.data_ptr()) == linattn.ERR_INVALID_ARG          # two outputs in one buffer
+        assert call(dv=g.data_ptr()) == linattn.ERR_INVALID_ARG           # an output over an input
+        assert call(dq=dq.data_ptr() + 4) == linattn.ERR_INVALID_ARG      # misaligned
+        assert call(dWk=dWq.data_ptr()) == linattn.ERR_INVALID_ARG
+        assert call(n=129) == linattn.ERR_WORKSPACE
+        ctx.check()
+    finally:
+        ctx.destroy()
