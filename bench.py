@@ -172,6 +172,8 @@ def main():
     ap.add_argument("--mixed", type=float, default=None, metavar="R",
                     help="time mixed attention (Eq. 8) with score R instead: linattn_forward_mixed on a resident "
                          "softmax-branch output (5 tensors of traffic instead of 4)")
+    ap.add_argument("--backward", action="store_true",
+                    help="time linattn_backward (gradients of the operator, CUDA-core kernels) instead of the forward")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     wl = synth.CONFIGS[args.config]
@@ -200,6 +202,7 @@ def main():
         sets.append({k_: t.to(dev) for k_, t in x.items()})
     outs = [torch.empty_like(s["q"]) for s in sets]
     softs = [torch.randn_like(s["q"]) for s in sets] if args.mixed is not None else None
+    douts = [torch.randn_like(s["q"]) for s in sets] if args.backward else None
     ctxs = []
     for s in sets:  # one context per input set: its own feature map, as one layer would have
         c = linattn.LinAttn(H, d, max_B=B, max_n=n, device=local)
@@ -211,7 +214,9 @@ def main():
 
     def step(i):
         j = i % rotate
-        if softs is None:
+        if douts is not None:
+            ctxs[j].backward(sets[j]["q"], sets[j]["k"], sets[j]["v"], douts[j], stream=stream)
+        elif softs is None:
             ctxs[j].forward(sets[j]["q"], sets[j]["k"], sets[j]["v"], out=outs[j], stream=stream)
         else:
             ctxs[j].forward_mixed(sets[j]["q"], sets[j]["k"], sets[j]["v"], softs[j], args.mixed, out=outs[j], stream=stream)
@@ -243,7 +248,9 @@ def main():
 
     # per-kernel durations: a second pass of the same steps with events around every launch
     e = 2 if wl.dtype == "bf16" else 4
-    alg_total = (4.0 if softs is None else 5.0) * B * H * n * d * e
+    # tensors of [B,H,n,d] one step must move: q, k, v in and o out; + the softmax branch for Eq. 8; for the
+    # gradients q, k, v, dO in and dq, dk, dv out
+    alg_total = (7.0 if douts is not None else 4.0 if softs is None else 5.0) * B * H * n * d * e
     for c in ctxs:
         c.set_option(linattn.OPT_PROFILE, 1)
     for i in range(args.steps):
@@ -266,7 +273,7 @@ def main():
                                "frac": alg_total / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                "frac_of_nominal_8TBs": alg_total / (ms_step * 1e-3) / 1e9 / 8000.0,
                                "algorithmic_bytes": alg_total}}
-    roofline["traffic"] = recorded_traffic(dom["name"]) if softs is None else None
+    roofline["traffic"] = recorded_traffic(dom["name"]) if softs is None and douts is None else None
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host tensor out
     pin = {k_: host0[k_].pin_memory() for k_ in ("q", "k", "v")}
@@ -284,8 +291,11 @@ def main():
     e2e = {"value": tokens_per_step / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
            "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "entry_point": "linattn_forward_host (pinned host buffers)"}
 
+    if douts is not None:
+        e2e["note"] = "this is the forward's host-buffer entry point; the backward has no host-buffer form"
     result = {
-        "metric": METRIC if softs is None else "mixed-attention (Eq. 8) fwd tokens/s", "value": value, "unit": UNIT,
+        "metric": ("linear-attention bwd tokens/s" if douts is not None else METRIC if softs is None
+                   else "mixed-attention (Eq. 8) fwd tokens/s"), "value": value, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",

@@ -117,6 +117,21 @@ def test_heavy_tailed_keys():
     _assert_grads(got, want, "heavy-tailed keys")
 
 
+def test_config2_full_size_two_heads_against_the_oracle():
+    """Full size of the headline workload.  The heads are independent, so the oracle's gradients for two of the
+    twelve heads (computed on those heads alone) pin the corresponding slices of the full-size result."""
+    from paper_2510_08318_b200 import synth
+    x = synth.make_inputs(2)
+    B, H, n, d = x["q"].shape
+    x["dout"] = torch.randn(B, H, n, d, generator=torch.Generator().manual_seed(36)).to(x["q"].dtype)
+    got, _ = _run(x)
+    for h in (0, 7):
+        sl = {s: x[s][:, h:h + 1].contiguous() for s in ("q", "k", "v", "dout")}
+        want = oracle.ref_backward(sl["q"], sl["k"], sl["v"], x["Wq"][h:h + 1].contiguous(), x["Wk"][h:h + 1].contiguous(), sl["dout"])
+        mine = tuple(t[:, h:h + 1] for t in got[:3]) + tuple(t[h:h + 1] for t in got[3:])
+        _assert_grads(mine, want, f"config 2, head {h}")
+
+
 def test_argument_errors():
     lib = linattn.load_library()
     x = _inputs(1, 2, 128, 64, torch.float32, seed=35)
