@@ -390,3 +390,88 @@ int linattn_ref_backward(const float *q, const float *k, const float *v, const f
     }
     return fail;
 }
+
+/*
+ * The ReLU kernel function of the paper's ablation over kernel functions (the table "Comparison across kernel
+ * functions"; the paper names the kernel and prints no formula).  Reading taken: the standard ReLU feature map of
+ * the linear-attention literature the ablation follows, phi(x) = max(x, 0) element by element on the d features of
+ * the head, no learnable matrix; Eq. 5 is otherwise unchanged (no epsilon: a query whose phi is orthogonal to z
+ * divides by zero and gives a non-finite row, on both sides).  Left and right forms as for the Hedgehog map.
+ *   q,k,v : [G][n][d] float;  rows : nrows query indices, or NULL for all n;  out : [G][nrows or n][d] double
+ */
+static double relu(float x) { return x > 0.0f ? (double)x : 0.0; }
+
+int linattn_ref_relu_quadratic(const float *q, const float *k, const float *v, long G, long n, int d,
+                               const long *rows, long nrows, double *out)
+{
+    if (d < 1 || n < 1 || G < 1) return 1;
+    const long nr = rows ? nrows : n;
+    int fail = 0;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long g = 0; g < G; ++g) {
+        for (long r = 0; r < nr; ++r) {
+            const long i = rows ? rows[r] : r;
+            const float *qi = q + ((size_t)g * n + i) * d;
+            const float *kg = k + (size_t)g * n * d, *vg = v + (size_t)g * n * d;
+            double *o = out + ((size_t)g * nr + r) * d;
+            double *a = (double *)malloc((size_t)n * sizeof(double));
+            if (!a) { fail = 1; continue; }
+            double den = 0.0;
+            for (long j = 0; j < n; ++j) {
+                double s = 0.0;
+                for (int f = 0; f < d; ++f) s += relu(qi[f]) * relu(kg[(size_t)j * d + f]);
+                a[j] = s;
+                den += s;
+            }
+            for (int c = 0; c < d; ++c) o[c] = 0.0;
+            for (long j = 0; j < n; ++j)
+                for (int c = 0; c < d; ++c) o[c] += a[j] / den * (double)vg[(size_t)j * d + c];
+            free(a);
+        }
+    }
+    return fail;
+}
+
+int linattn_ref_relu_linear(const float *q, const float *k, const float *v, long G, long n, int d,
+                            const long *rows, long nrows, double *out, double *S_out, double *z_out)
+{
+    if (d < 1 || n < 1 || G < 1) return 1;
+    const long nr = rows ? nrows : n;
+    double *S_all = (double *)calloc((size_t)G * d * d, sizeof(double));
+    double *z_all = (double *)calloc((size_t)G * d, sizeof(double));
+    if (!S_all || !z_all) { free(S_all); free(z_all); return 1; }
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long g = 0; g < G; ++g) {
+        double *S = S_all + (size_t)g * d * d, *z = z_all + (size_t)g * d;
+        for (long j = 0; j < n; ++j) {
+            const float *kj = k + ((size_t)g * n + j) * d, *vj = v + ((size_t)g * n + j) * d;
+            for (int f = 0; f < d; ++f) {
+                const double p = relu(kj[f]);
+                z[f] += p;
+                for (int c = 0; c < d; ++c) S[(size_t)f * d + c] += p * (double)vj[c];
+            }
+        }
+    }
+    if (out) {
+#pragma omp parallel for collapse(2) schedule(static)
+        for (long g = 0; g < G; ++g) {
+            for (long r = 0; r < nr; ++r) {
+                const long i = rows ? rows[r] : r;
+                const float *qi = q + ((size_t)g * n + i) * d;
+                const double *S = S_all + (size_t)g * d * d, *z = z_all + (size_t)g * d;
+                double *o = out + ((size_t)g * nr + r) * d;
+                double den = 0.0;
+                for (int f = 0; f < d; ++f) den += relu(qi[f]) * z[f];
+                for (int c = 0; c < d; ++c) {
+                    double num = 0.0;
+                    for (int f = 0; f < d; ++f) num += relu(qi[f]) * S[(size_t)f * d + c];
+                    o[c] = num / den;
+                }
+            }
+        }
+    }
+    if (S_out) memcpy(S_out, S_all, (size_t)G * d * d * sizeof(double));
+    if (z_out) memcpy(z_out, z_all, (size_t)G * d * sizeof(double));
+    free(S_all); free(z_all);
+    return 0;
+}

@@ -52,6 +52,9 @@ def _load():
         lib.linattn_ref_mix.argtypes = [dp, dp, ctypes.c_long, ctypes.c_double, dp]
         lib.linattn_ref_backward.argtypes = [fp, fp, fp, fp, fp, fp, ctypes.c_long, ctypes.c_int, ctypes.c_long,
                                              ctypes.c_int, ctypes.c_int, dp, dp, dp, dp, dp]
+        lib.linattn_ref_relu_quadratic.argtypes = [fp, fp, fp, ctypes.c_long, ctypes.c_long, ctypes.c_int, lp, ctypes.c_long, dp]
+        lib.linattn_ref_relu_linear.argtypes = [fp, fp, fp, ctypes.c_long, ctypes.c_long, ctypes.c_int, lp, ctypes.c_long,
+                                                dp, dp, dp]
         _lib = lib
     return _lib
 
@@ -183,3 +186,35 @@ def ref_backward(q, k, v, Wq, Wk, dout):
     if rc:
         raise ValueError("oracle rejected the arguments or ran out of memory")
     return dq, dk, dv, dWq, dWk
+
+
+def ref_relu_quadratic(q, k, v, rows=None) -> np.ndarray:
+    """Left form of Eq. 5 with the ReLU kernel function phi(x) = max(x, 0). float64 [B, H, len(rows) or n, d]."""
+    q, k, v = (_f32(t) for t in (q, k, v))
+    assert q.ndim == 4 and q.shape == k.shape == v.shape
+    B, H, n, d = q.shape
+    r, nr = _rows(rows, n)
+    out = np.empty((B, H, nr, d), dtype=np.float64)
+    F = ctypes.c_float
+    rc = _load().linattn_ref_relu_quadratic(_ptr(q, F), _ptr(k, F), _ptr(v, F), B * H, n, d, _ptr(r, ctypes.c_long), nr,
+                                            _ptr(out, ctypes.c_double))
+    if rc:
+        raise ValueError("oracle rejected the arguments or ran out of memory")
+    return out
+
+
+def ref_relu_linear(q, k, v, rows=None, return_state: bool = False):
+    """Right form of Eq. 5 with the ReLU kernel function; as ``ref_linear``."""
+    q, k, v = (_f32(t) for t in (q, k, v))
+    assert q.ndim == 4 and q.shape == k.shape == v.shape
+    B, H, n, d = q.shape
+    r, nr = _rows(rows, n)
+    out = np.empty((B, H, nr, d), dtype=np.float64)
+    S = np.empty((B, H, d, d), dtype=np.float64) if return_state else None
+    z = np.empty((B, H, d), dtype=np.float64) if return_state else None
+    F, D = ctypes.c_float, ctypes.c_double
+    rc = _load().linattn_ref_relu_linear(_ptr(q, F), _ptr(k, F), _ptr(v, F), B * H, n, d, _ptr(r, ctypes.c_long), nr,
+                                         _ptr(out, D), _ptr(S, D), _ptr(z, D))
+    if rc:
+        raise ValueError("oracle rejected the arguments or ran out of memory")
+    return (out, S, z) if return_state else out

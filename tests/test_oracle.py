@@ -354,3 +354,52 @@ def test_backward_shared_weights_sum_over_heads_and_invariances():
     one = oracle.ref_backward(q, k, v, Wq, Wk, g)
     for a, b in zip(two, one):
         np.testing.assert_allclose(a, 2.0 * b, rtol=1e-12, atol=1e-14)
+
+
+# ---- the ReLU kernel function of the paper's kernel-function ablation ---------------------------------------
+
+def _qkv(B, H, n, d, seed):
+    rng = np.random.default_rng(seed)
+    return tuple(rng.standard_normal((B, H, n, d)).astype(np.float32) for _ in range(3))
+
+
+@pytest.mark.parametrize("B,H,n,d", [(1, 1, 7, 4), (2, 2, 33, 8), (1, 2, 300, 64)])
+def test_relu_linear_form_equals_quadratic_form_and_a_library_computation(B, H, n, d):
+    q, k, v = _qkv(B, H, n, d, seed=80 + n)
+    lin, S, z = oracle.ref_relu_linear(q, k, v, return_state=True)
+    quad = oracle.ref_relu_quadratic(q, k, v)
+    np.testing.assert_allclose(lin, quad, rtol=1e-10, atol=1e-12)
+    # the same through torch's matmuls in fp64: A = relu(Q) relu(K)^T, O = (A / rowsum) V
+    tq, tk, tv = (torch.from_numpy(x).double() for x in (q, k, v))
+    A = torch.relu(tq) @ torch.relu(tk).transpose(-1, -2)
+    want = (A / A.sum(-1, keepdim=True)) @ tv
+    np.testing.assert_allclose(quad, want.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(S, (torch.relu(tk).transpose(-1, -2) @ tv).numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(z, torch.relu(tk).sum(-2).numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_relu_closed_forms():
+    B, H, n, d = 1, 2, 40, 8
+    q, k, v = _qkv(B, H, n, d, seed=90)
+    base = oracle.ref_relu_linear(q, k, v)
+    # positively homogeneous: scaling q or k by a positive (power-of-two) factor leaves o unchanged
+    np.testing.assert_allclose(oracle.ref_relu_linear(4.0 * q, 0.25 * k, v), base, rtol=1e-12, atol=1e-14)
+    # negative entries are ignored: replacing them by other negative values changes nothing
+    q2 = np.where(q < 0, 3.0 * q, q).astype(np.float32)
+    k2 = np.where(k < 0, -1.0, k).astype(np.float32)
+    np.testing.assert_array_equal(oracle.ref_relu_linear(q2, k2, v), base)
+    # keys that are all equal and positive: every weight is equal, o = mean of V
+    kc = np.ones_like(k)
+    np.testing.assert_allclose(oracle.ref_relu_linear(np.abs(q), kc, v), np.broadcast_to(v.astype(np.float64).mean(2, keepdims=True), v.shape),
+                               rtol=1e-12, atol=1e-13)
+    # one-hot queries and keys pick out the average of the values whose key shares the query's feature
+    e = np.zeros((1, 1, 4, 4), dtype=np.float32)
+    e[0, 0, np.arange(4), [0, 1, 0, 1]] = 1.0
+    vv = np.arange(16, dtype=np.float32).reshape(1, 1, 4, 4)
+    o = oracle.ref_relu_linear(e, e, vv)
+    np.testing.assert_allclose(o[0, 0, 0], (vv[0, 0, 0] + vv[0, 0, 2]) / 2)
+    np.testing.assert_allclose(o[0, 0, 1], (vv[0, 0, 1] + vv[0, 0, 3]) / 2)
+    # rows subset
+    rows = np.array([3, 17, 39])
+    np.testing.assert_array_equal(oracle.ref_relu_linear(q, k, v, rows=rows), base[:, :, rows])
+    np.testing.assert_allclose(oracle.ref_relu_quadratic(q, k, v, rows=rows), base[:, :, rows], rtol=1e-10, atol=1e-12)
