@@ -172,6 +172,8 @@ def main():
     ap.add_argument("--mixed", type=float, default=None, metavar="R",
                     help="time mixed attention (Eq. 8) with score R instead: linattn_forward_mixed on a resident "
                          "softmax-branch output (5 tensors of traffic instead of 4)")
+    ap.add_argument("--phi", default="hedgehog", choices=["hedgehog", "relu"],
+                    help="kernel function: the Hedgehog feature map of Eq. 6 (the metric's) or the ReLU of the paper's ablation")
     ap.add_argument("--backward", action="store_true",
                     help="time linattn_backward (gradients of the operator, CUDA-core kernels) instead of the forward")
     args = ap.parse_args()
@@ -208,6 +210,7 @@ def main():
         c = linattn.LinAttn(H, d, max_B=B, max_n=n, device=local)
         c.set_option(linattn.OPT_PATH, args.path)
         c.set_option(linattn.OPT_SPLITS, args.splits)
+        c.set_option(linattn.OPT_KERNEL_FUNCTION, linattn.PHI_RELU if args.phi == "relu" else linattn.PHI_HEDGEHOG)
         c.set_feature_map(s["Wq"], s["Wk"])
         ctxs.append(c)
     stream = torch.cuda.current_stream()
@@ -273,7 +276,7 @@ def main():
                                "frac": alg_total / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                "frac_of_nominal_8TBs": alg_total / (ms_step * 1e-3) / 1e9 / 8000.0,
                                "algorithmic_bytes": alg_total}}
-    roofline["traffic"] = recorded_traffic(dom["name"]) if softs is None and douts is None else None
+    roofline["traffic"] = recorded_traffic(dom["name"]) if softs is None and douts is None and args.phi == "hedgehog" else None
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host tensor out
     pin = {k_: host0[k_].pin_memory() for k_ in ("q", "k", "v")}
@@ -294,8 +297,8 @@ def main():
     if douts is not None:
         e2e["note"] = "this is the forward's host-buffer entry point; the backward has no host-buffer form"
     result = {
-        "metric": ("linear-attention bwd tokens/s" if douts is not None else METRIC if softs is None
-                   else "mixed-attention (Eq. 8) fwd tokens/s"), "value": value, "unit": UNIT,
+        "metric": ("linear-attention bwd tokens/s" if douts is not None else "mixed-attention (Eq. 8) fwd tokens/s" if softs is not None
+                   else "linear-attention (ReLU kernel function) fwd tokens/s" if args.phi == "relu" else METRIC), "value": value, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",

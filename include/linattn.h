@@ -47,6 +47,12 @@ typedef enum {
     LINATTN_OPT_LAYOUT = 4, /* memory order of q, k, v, out (and o_softmax): 0 = [B][H][n][d] (default), 1 = [B][n][H][d],
                                the order in which a DiT's projection layers leave them (no transposes around the call);
                                d is contiguous in both */
+    LINATTN_OPT_KERNEL_FUNCTION = 5, /* the map phi of Eq. 5: 0 = the Hedgehog feature map of Eq. 6 (default); 1 = the ReLU
+                               kernel function of the paper's comparison across kernel functions, phi(x) = max(x, 0)
+                               element by element on the d features of the head: no weights (set_feature_map is not
+                               needed), no epsilon (a query whose phi is orthogonal to every key's gives a non-finite
+                               row).  Applies to linattn_forward, _mixed and _host; linattn_backward then returns
+                               UNSUPPORTED */
     LINATTN_OPT_PROFILE = 2 /* 1 = record CUDA events around every kernel of each forward (see linattn_profile_get);
                                switching it on clears the accumulated figures; 0 = off (default) */
 } linattn_option;

@@ -72,6 +72,7 @@ struct linattn_ctx {
     int opt_path = 0;
     int opt_fuse = 1;
     int opt_layout = 0;   // 0: [B][H][n][d], 1: [B][n][H][d]
+    int opt_phi = 0;      // 0: Hedgehog feature map (Eq. 6), 1: ReLU kernel function
     // per-kernel timing (LINATTN_OPT_PROFILE)
     static constexpr int kMaxKernels = 8;
     bool profile = false;
@@ -190,7 +191,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     const double side_bytes = 2.0 * (double)G * n * D * sizeof(T);  // K+V read, or Q read + O written
     prof_begin(c, st);
     kside_simt<T, D><<<dim3(splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
-        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, act_strides(c, n));
+        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, act_strides(c, n), c->opt_phi);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_simt", side_bytes);
     combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, c->state, splits, E);
@@ -201,7 +202,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     if (per_group > nchunks) per_group = nchunks;
     if (per_group < 1) per_group = 1;
     qside_simt<T, D><<<dim3((unsigned)per_group, (unsigned)G), kSimtThreads, qside_simt_smem<D>(), st>>>(
-        (const T*)q, c->Wq, c->state, (T*)out, c->H, n, (const T*)mix, mix_r, act_strides(c, n));
+        (const T*)q, c->Wq, c->state, (T*)out, c->H, n, (const T*)mix, mix_r, act_strides(c, n), c->opt_phi);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_simt", side_bytes);
     c->last_launches = 3;
@@ -237,7 +238,7 @@ linattn_status launch_backward_simt(linattn_ctx* c, const void* q, const void* k
     const dim3 grid((unsigned)blocks, (unsigned)G);
     prof_begin(c, st);
     kside_simt<T, D><<<dim3(splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
-        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, as);
+        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, as, 0);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_simt", 2.0 * tensor_bytes);
     combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, c->state, splits, E);
@@ -297,20 +298,24 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         return LINATTN_ERR_CUDA;
     }
     // one instantiation per (mixed attention or not, memory layout)
-    const void* k_fused[2][2] = {{(const void*)linattn_fused_tc<false, 0>, (const void*)linattn_fused_tc<false, 1>},
-                                 {(const void*)linattn_fused_tc<true, 0>, (const void*)linattn_fused_tc<true, 1>}};
-    const void* k_qside[2][2] = {{(const void*)qside_tc<false, 0>, (const void*)qside_tc<false, 1>},
-                                 {(const void*)qside_tc<true, 0>, (const void*)qside_tc<true, 1>}};
-    const void* k_kside[2] = {(const void*)kside_tc<0>, (const void*)kside_tc<1>};
+#define LA_BY_PHI(K, ...) {(const void*)K<__VA_ARGS__, 0>, (const void*)K<__VA_ARGS__, 1>}
+    const void* k_fused[2][2][2] = {{LA_BY_PHI(linattn_fused_tc, false, 0), LA_BY_PHI(linattn_fused_tc, false, 1)},
+                                    {LA_BY_PHI(linattn_fused_tc, true, 0), LA_BY_PHI(linattn_fused_tc, true, 1)}};
+    const void* k_qside[2][2][2] = {{LA_BY_PHI(qside_tc, false, 0), LA_BY_PHI(qside_tc, false, 1)},
+                                    {LA_BY_PHI(qside_tc, true, 0), LA_BY_PHI(qside_tc, true, 1)}};
+    const void* k_kside[2][2] = {LA_BY_PHI(kside_tc, 0), LA_BY_PHI(kside_tc, 1)};
+#undef LA_BY_PHI
+    const int phi = c->opt_phi;
     static bool attr_done = false;
     if (!attr_done) {
-        for (int i = 0; i < 2; ++i) {
-            LA_CUDA(c, cudaFuncSetAttribute(k_kside[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-            for (int j = 0; j < 2; ++j) {
-                LA_CUDA(c, cudaFuncSetAttribute(k_fused[i][j], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-                LA_CUDA(c, cudaFuncSetAttribute(k_qside[i][j], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+        for (int i = 0; i < 2; ++i)
+            for (int p = 0; p < 2; ++p) {
+                LA_CUDA(c, cudaFuncSetAttribute(k_kside[i][p], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                for (int j = 0; j < 2; ++j) {
+                    LA_CUDA(c, cudaFuncSetAttribute(k_fused[i][j][p], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                    LA_CUDA(c, cudaFuncSetAttribute(k_qside[i][j][p], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                }
             }
-        }
         attr_done = true;
     }
     const double side_bytes = 2.0 * (double)G * n * kD * 2;
@@ -341,7 +346,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
         c->bar_total += 2u * (uint32_t)Pq;
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
-        const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads),
+        const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout][phi], dim3((unsigned)Pq), dim3(kThreads),
                                                            params, Smem::kTotal, st);
         if (le == cudaSuccess) {
             prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
@@ -357,7 +362,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     }
     {
         void* kp[] = {&tmK, &tmV, &tmWk, &a};
-        LA_CUDA(c, cudaLaunchKernel(k_kside[layout], dim3((unsigned)Pk), dim3(kThreads), kp, Smem::kTotal, st));
+        LA_CUDA(c, cudaLaunchKernel(k_kside[layout][phi], dim3((unsigned)Pk), dim3(kThreads), kp, Smem::kTotal, st));
     }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_tc", side_bytes);
@@ -366,7 +371,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     prof_mark(c, st, "combine_tc", 0.0);
     {
         void* qp[] = {&tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
-        LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
+        LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout][phi], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
     }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);
@@ -391,7 +396,7 @@ linattn_status check_forward_args(linattn_ctx* c, const void* q, const void* k, 
     if (H != c->H || d != c->d) return LINATTN_ERR_INVALID_ARG;
     if (B < 1 || n < 1) return LINATTN_ERR_INVALID_ARG;
     if (B > c->max_B || n > c->max_n) return LINATTN_ERR_WORKSPACE;
-    if (!c->have_map) return LINATTN_ERR_NO_FEATURE_MAP;
+    if (!c->have_map && c->opt_phi == 0) return LINATTN_ERR_NO_FEATURE_MAP;   // the ReLU kernel function has no weights
     return LINATTN_OK;
 }
 
@@ -549,7 +554,7 @@ static linattn_status forward_impl(linattn_ctx* c, const void* q, const void* k,
     }
     // The tensor-core kernels cover bf16 activations with head dimension 128 and bf16 feature-map weights;
     // everything else runs on the CUDA-core kernels.
-    const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && c->map_is_bf16);
+    const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && (c->map_is_bf16 || c->opt_phi == 1));
     if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
@@ -583,6 +588,7 @@ linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, co
                                 linattn_dtype dtype, void* stream)
 {
     if (!dout || !dk || !dv || !dWq || !dWk) return LINATTN_ERR_INVALID_ARG;
+    if (c && c->opt_phi != 0) return LINATTN_ERR_UNSUPPORTED;   // gradients exist for the feature map of Eq. 6 only
     linattn_status s = check_forward_args(c, q, k, v, dq, B, H, n, d, dtype);
     if (s != LINATTN_OK) return s;
     const void* ins[4] = {q, k, v, dout};
@@ -690,6 +696,10 @@ linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long 
         case LINATTN_OPT_LAYOUT:
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
             c->opt_layout = (int)value;
+            return LINATTN_OK;
+        case LINATTN_OPT_KERNEL_FUNCTION:
+            if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
+            c->opt_phi = (int)value;
             return LINATTN_OK;
         case LINATTN_OPT_FUSE:
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;

@@ -75,13 +75,13 @@ linattn_status run(int dev, int slot, float* scratch, const T* q, const T* k, co
     float* partial = scratch;                                              // [G*splits][E], fully overwritten
     float* state = scratch + (size_t)kNoAllocPartialSlots * kNoAllocMaxE;  // [G][E], fully overwritten
     kside_simt<T, D><<<dim3((unsigned)splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
-        k, v, Wk, partial, Hw, n, chunk, ActStrides{D, (long long)n * D, (long long)Hw * n * D});
+        k, v, Wk, partial, Hw, n, chunk, ActStrides{D, (long long)n * D, (long long)Hw * n * D}, 0);
     combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(partial, state, (int)splits, E);
     const int nchunks = (n + kSimtTokens - 1) / kSimtTokens;
     long long per_group = (2LL * 148 + G - 1) / G;
     if (per_group > nchunks) per_group = nchunks;
     qside_simt<T, D><<<dim3((unsigned)per_group, (unsigned)G), kSimtThreads, qside_simt_smem<D>(), st>>>(
-        q, Wq, state, out, Hw, n, (const T*)nullptr, 0.f, ActStrides{D, (long long)n * D, (long long)Hw * n * D});
+        q, Wq, state, out, Hw, n, (const T*)nullptr, 0.f, ActStrides{D, (long long)n * D, (long long)Hw * n * D}, 0);
     if (cudaGetLastError() != cudaSuccess) return LINATTN_ERR_CUDA;
     return LINATTN_OK;
 }

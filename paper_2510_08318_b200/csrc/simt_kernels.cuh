@@ -78,6 +78,17 @@ __device__ __forceinline__ void feature_map_chunk(const float* __restrict__ x_s,
     }
 }
 
+// The ReLU kernel function, phi(x) = max(x, 0) element by element, for the chunk; rows >= valid get phi = 0.
+template <int D>
+__device__ __forceinline__ void relu_chunk(const float* __restrict__ x_s, float* __restrict__ phi_s, int valid)
+{
+    constexpr int P = SimtShape<D>::PITCH;
+    for (int e = threadIdx.x; e < kSimtTokens * D; e += kSimtThreads) {
+        const int r = e / D, c = e % D;
+        phi_s[r * P + c] = (r < valid) ? fmaxf(x_s[r * P + c], 0.f) : 0.f;
+    }
+}
+
 // Load `rows` x D elements starting at src (row-major, contiguous) into dst (fp32, pitch PITCH);
 // rows in [valid, kSimtTokens) are zero-filled.
 template <typename T, int D>
@@ -106,7 +117,7 @@ template <int D> constexpr size_t kside_simt_smem()
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 kside_simt(const T* __restrict__ k, const T* __restrict__ v, const float* __restrict__ Wk /*[H][D][M]*/,
-           float* __restrict__ partial, int H, int n, int chunk, ActStrides st)
+           float* __restrict__ partial, int H, int n, int chunk, ActStrides st, int relu)
 {
     constexpr int M = SimtShape<D>::M, P = SimtShape<D>::PITCH;
     constexpr int FB = D / 16;           // f rows per thread (8 or 4)
@@ -141,7 +152,8 @@ kside_simt(const T* __restrict__ k, const T* __restrict__ v, const float* __rest
         load_chunk<T, D>(kg + (size_t)t * st.token, st.token, k_s, valid);
         load_chunk<T, D>(vg + (size_t)t * st.token, st.token, v_s, valid);
         __syncthreads();
-        feature_map_chunk<D>(k_s, W_s, phi_s, valid);
+        if (relu) relu_chunk<D>(k_s, phi_s, valid);
+        else feature_map_chunk<D>(k_s, W_s, phi_s, valid);
         __syncthreads();
 #pragma unroll 2
         for (int r = 0; r < kSimtTokens; ++r) {
@@ -193,12 +205,13 @@ template <int D> constexpr size_t qside_simt_smem()
 
 // grid = (blocks_per_group, G).  Block x handles chunks x, x + gridDim.x, ... of kSimtTokens tokens.
 // state: [G][D*D + D] floats (S then z).
+// relu != 0: the ReLU kernel function instead of Eq. 6 (Wq / Wk are then loaded but not used).
 // mix != nullptr: Eq. 8, out = mix_r * mix + (1 - mix_r) * (Eq. 5), mix = output of the softmax-attention branch
 // ([G][n][D], may be the same buffer as out), mix_r already clipped into [0, 1].
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* __restrict__ state,
-           T* out, int H, int n, const T* mix, float mix_r, ActStrides st)
+           T* out, int H, int n, const T* mix, float mix_r, ActStrides st, int relu)
 {
     constexpr int M = SimtShape<D>::M, P = SimtShape<D>::PITCH;
     constexpr int CG = D / 32;  // float4 column groups per thread (4 or 2)
@@ -226,7 +239,9 @@ qside_simt(const T* __restrict__ q, const float* __restrict__ Wq, const float* _
         __syncthreads();
         load_chunk<T, D>(qg + (size_t)t * st.token, st.token, q_s, valid);
         __syncthreads();
-        feature_map_chunk<D>(q_s, W_s, phi_s, kSimtTokens);  // tail rows see zero-filled q: finite phi, never stored
+        // tail rows see zero-filled q: their phi is finite (Eq. 6) or zero (ReLU); their outputs are never stored
+        if (relu) relu_chunk<D>(q_s, phi_s, kSimtTokens);
+        else feature_map_chunk<D>(q_s, W_s, phi_s, kSimtTokens);
         __syncthreads();
         float num[CG][4];
 #pragma unroll

@@ -441,11 +441,30 @@ __device__ __forceinline__ void act_prefetch_l2(const void* tm, int x, int t, in
     else tma_prefetch_l2_4d(tm, x, t, g % H, g / H);
 }
 
+// ReLU kernel function, phi(x) = max(x, 0) element by element: applied in place to a 128 x 128 bf16 tile exactly as
+// TMA left it in shared memory (element-wise, so the swizzled operand layout is kept); 256 threads, 128 bytes each.
+// Rows past the end of the sequence were zero-filled by TMA and stay zero.
+__device__ __forceinline__ void relu_tile_in_place(uint8_t* tile, int t)
+{
+#pragma unroll
+    for (int j = 0; j < kTileBytes / (256 * 16); ++j) {
+        uint4* p = reinterpret_cast<uint4*>(tile) + j * 256 + t;
+        uint4 v = *p;
+        asm("max.bf16x2 %0, %0, %1;" : "+r"(v.x) : "r"(0u));
+        asm("max.bf16x2 %0, %0, %1;" : "+r"(v.y) : "r"(0u));
+        asm("max.bf16x2 %0, %0, %1;" : "+r"(v.z) : "r"(0u));
+        asm("max.bf16x2 %0, %0, %1;" : "+r"(v.w) : "r"(0u));
+        *p = v;
+    }
+}
+
 // ======================================================================================================
 // Key side: partial S = sum phi(k)^T v and z = sum phi(k) over this CTA's tiles (Eq. 5 brackets, Eq. 6)
 // ======================================================================================================
 
-template <int kLayout>
+// kPhi: 0 = the Hedgehog feature map of Eq. 6; 1 = the ReLU kernel function (no projection, no softmax: the logits
+// warp idles and warps 0-7 rectify the K tile in place).
+template <int kLayout, int kPhi>
 __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const CUtensorMap* tmK, const CUtensorMap* tmV,
                                             const CUtensorMap* tmW)
 {
@@ -468,7 +487,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
         Ring<kKStages> r;
         int issued = 0;
         for (; !w.done(); w.next(), r.next()) {
-            if (w.first()) {
+            if (kPhi == 0 && w.first()) {
                 const int wb = w.seg & 1;
                 if (w.seg >= 2 && !warp_wait(c.bar(K_WFREE + wb), ((w.seg >> 1) - 1) & 1, c.wc, kErrProducer)) break;
                 if (lane == 0) {
@@ -499,7 +518,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
         // ---------------- logits MMA issuer: U = K W_k ----------------
         Ring<kKStages> r;
         Ring<2> ur;
-        for (; !w.done(); w.next(), r.next(), ur.next()) {
+        for (; kPhi == 0 && !w.done(); w.next(), r.next(), ur.next()) {
             const int wb = w.seg & 1;
             if (w.first() && !warp_wait(c.bar(K_WFULL + wb), (uint32_t)(w.seg >> 1) & 1u, c.wc, kErrMmaLoad)) break;
             if (!warp_wait(c.bar(K_FULL + r.s), r.ph, c.wc, kErrMmaLoad)) break;
@@ -543,6 +562,16 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             }
             __syncwarp();
             LA_TRACE(1, w.i, 3);
+        }
+    } else if (warp < 8 && kPhi == 1) {
+        // ---------------- ReLU kernel function (warps 0-7) ----------------
+        Ring<kKStages> r;
+        for (; !w.done(); w.next(), r.next()) {
+            if (!warp_wait(c.bar(K_FULL + r.s), r.ph, c.wc, kErrSoftmaxU)) break;
+            relu_tile_in_place(c.smem + r.s * Smem::kKStage, threadIdx.x);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c.bar(K_PHIFULL + r.s));
         }
     } else if (warp < 8) {
         // ---------------- feature map + drain (warps 0-7) ----------------
@@ -667,7 +696,7 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
 
 // wait_state: the S and z images are produced earlier in the same kernel (fused path); loads of them
 // must wait for the Q_SREADY barrier.  Otherwise they were written by a previous launch.
-template <bool kMix, int kLayout>
+template <bool kMix, int kLayout, int kPhi>
 __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
                                             const CUtensorMap* tmW, const CUtensorMap* tmS, const CUtensorMap* tmA, bool wait_state)
 {
@@ -709,7 +738,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         for (; !w.done() && ok; w.next(), r.next()) {
             if (w.first()) {
                 if (w.seg >= 1 && !warp_wait(c.bar(Q_SEGFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrSeg)) break;
-                if (lane == 0) {
+                if (kPhi == 0 && lane == 0) {
                     mbar_arrive_expect_tx(c.bar(Q_WFULL), kWBytes);
                     tma_load_3d(sbase + Smem::kQW, tmW, c.bar(Q_WFULL), 0, 0, w.g % a.H);
                     tma_load_3d(sbase + Smem::kQW + kWBytes / 2, tmW, c.bar(Q_WFULL), 64, 0, w.g % a.H);
@@ -773,7 +802,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         // ---------------- logits MMA issuer: U = Q W_q ----------------
         Ring<kQStages> r;
         Ring<2> ur;
-        for (; !w.done(); w.next(), r.next(), ur.next()) {
+        for (; kPhi == 0 && !w.done(); w.next(), r.next(), ur.next()) {
             if (w.first() && !warp_wait(c.bar(Q_WFULL), (uint32_t)w.seg & 1u, c.wc, kErrSeg)) break;
             if (!warp_wait(c.bar(Q_FULL + r.s), r.ph, c.wc, kErrMmaLoad)) break;
             LA_TRACE(1, 24 + w.i, 0);
@@ -833,6 +862,16 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             LA_TRACE(0, 24 + w.i, 1);
         }
         if (lane == 0) bulk_wait_group<0>();
+    } else if (warp < 8 && kPhi == 1) {
+        // ---------------- ReLU kernel function (warps 0-7): phi(q) in place in the tile's slot ----------------
+        Ring<kQStages> r;
+        for (; !w.done(); w.next(), r.next()) {
+            if (!warp_wait(c.bar(Q_FULL + r.s), r.ph, c.wc, kErrSoftmaxU)) break;
+            relu_tile_in_place(c.smem + r.s * kTileBytes, threadIdx.x);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c.bar(Q_PHIFULL + r.s));
+        }
     } else if (warp < 8) {
         // ---------------- feature map (warps 0-7) ----------------
         const int half = warp >> 2;
@@ -942,14 +981,14 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
 // Kernels
 // ======================================================================================================
 
-template <int kLayout>
+template <int kLayout, int kPhi>
 __global__ void __launch_bounds__(kThreads, 1)
 kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
          const __grid_constant__ CUtensorMap tmW, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, true, false);
-    kside_phase<kLayout>(c, a, &tmK, &tmV, &tmW);
+    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmW);
     cta_teardown(c);
 }
 
@@ -960,7 +999,7 @@ static __global__ void __launch_bounds__(256) combine_tc(const Args a, long long
     if (q4 < kE / 4) combine_quad(a, P, blockIdx.y, q4 * 4);
 }
 
-template <bool kMix, int kLayout>
+template <bool kMix, int kLayout, int kPhi>
 __global__ void __launch_bounds__(kThreads, 1)
 qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
          const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS,
@@ -968,7 +1007,7 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, false, true);
-    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmW, &tmS, &tmA, false);
+    qside_phase<kMix, kLayout, kPhi>(c, a, &tmQ, &tmO, &tmW, &tmS, &tmA, false);
     cta_teardown(c);
 }
 
@@ -990,7 +1029,7 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target)
 }
 
 // The whole forward in one cooperative launch of P <= #SMs persistent CTAs.
-template <bool kMix, int kLayout>
+template <bool kMix, int kLayout, int kPhi>
 __global__ void __launch_bounds__(kThreads, 1)
 linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmQ,
@@ -1001,7 +1040,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     LA_TRACE_NS(0, 60, 0);
     const Cta c = cta_setup(smem_raw, a, true, true);
     LA_TRACE_NS(0, 60, 1);
-    kside_phase<kLayout>(c, a, &tmK, &tmV, &tmWk);
+    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmWk);
     // every role is done with the key-side buffers; the partials of this CTA are written
     tcgen05_fence_before();
     __syncthreads();
@@ -1042,7 +1081,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (c.warp >= 12 && c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
-    qside_phase<kMix, kLayout>(c, a, &tmQ, &tmO, &tmWq, &tmS, &tmA, true);
+    qside_phase<kMix, kLayout, kPhi>(c, a, &tmQ, &tmO, &tmWq, &tmS, &tmA, true);
     LA_TRACE_NS(0, 61, 2);
     cta_teardown(c);
     LA_TRACE_NS(0, 61, 3);
