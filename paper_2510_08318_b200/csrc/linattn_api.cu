@@ -84,6 +84,7 @@ struct linattn_ctx {
     double prof_ms[kMaxKernels] = {};
     long long prof_cnt[kMaxKernels] = {};
     // bookkeeping
+    bool attr_done[9] = {};   // shared-memory limit raised on this context's device, per kernel family (function attributes are per device)
     int last_launches = 0;
     int last_B = 0;
     bool state_transposed = false;  // the last forward left S in the workspace as [c][f] (tensor-core kernels) rather than [f][c]
@@ -180,7 +181,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     if (G * splits > c->partial_slots) return LINATTN_ERR_WORKSPACE;
     constexpr int E = D * D + D;
 
-    static bool attr_done = false;  // per process and template instance; setting it twice is harmless
+    bool& attr_done = c->attr_done[(sizeof(T) == 2 ? 2 : 0) + (D == 128 ? 1 : 0)];
     if (!attr_done) {
         LA_CUDA(c, cudaFuncSetAttribute(kside_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kside_simt_smem<D>()));
@@ -226,7 +227,7 @@ linattn_status launch_backward_simt(linattn_ctx* c, const void* q, const void* k
     if (G * splits > c->partial_slots || G * blocks > c->partial_slots) return LINATTN_ERR_WORKSPACE;
     constexpr int E = D * D + D, DM = D * (D / 2);
 
-    static bool attr_done = false;
+    bool& attr_done = c->attr_done[4 + (sizeof(T) == 2 ? 2 : 0) + (D == 128 ? 1 : 0)];
     if (!attr_done) {
         LA_CUDA(c, cudaFuncSetAttribute(kside_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kside_simt_smem<D>()));
         LA_CUDA(c, cudaFuncSetAttribute(qside_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bwd_smem<D>()));
@@ -306,7 +307,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     const void* k_kside[2][2] = {LA_BY_PHI(kside_tc, 0), LA_BY_PHI(kside_tc, 1)};
 #undef LA_BY_PHI
     const int phi = c->opt_phi;
-    static bool attr_done = false;
+    bool& attr_done = c->attr_done[8];
     if (!attr_done) {
         for (int i = 0; i < 2; ++i)
             for (int p = 0; p < 2; ++p) {
