@@ -129,11 +129,16 @@ linattn_status linattn_backward(linattn_ctx* ctx, const void* q, const void* k, 
                                 int B, int H, int n, int d, linattn_dtype dtype, void* stream);
 
 /*
- * The same operation on HOST buffers (pageable or pinned): copies q, k, v to device staging
- * buffers owned by the context, runs linattn_forward, copies the result into `out`, and waits
- * for `stream` before returning.  The staging buffers are allocated (or grown) on the first call
- * that needs them and released by destroy.  Same argument rules and errors as linattn_forward,
- * except that the pointers are host pointers with no alignment requirement.
+ * The same operation on HOST buffers (pageable or pinned; pinned buffers let the copies overlap).  For the
+ * default [B][H][n][d] layout the (b,h) pairs, which are independent and contiguous, go through a three-stage
+ * pipeline inside the call: copies to the device on one internal stream, the forward of one pair on `stream`,
+ * copies of finished pairs back on a second internal stream, so that both copy directions and the compute
+ * overlap; the call returns when `out` is complete.  For the token-major layout the problem goes in one piece.
+ * The staging buffers (four of the problem's size) are allocated, or grown, on the first call that needs them
+ * and released by destroy.  Same argument rules and errors as linattn_forward, except that the pointers are
+ * host pointers with no alignment requirement.  Each pair is reduced with the split of a one-pair problem, so
+ * the result agrees with linattn_forward's to rounding (not bit for bit); it is deterministic like every entry
+ * point.  linattn_read_state afterwards returns the S, z of all pairs as usual.
  */
 linattn_status linattn_forward_host(linattn_ctx* ctx, const void* q, const void* k, const void* v, void* out,
                                     int B, int H, int n, int d, linattn_dtype dtype, void* stream);

@@ -64,9 +64,15 @@ struct linattn_ctx {
     float* bwd_part_state = nullptr;  // [partial_slots][d*d + d]  per-block sums of dS, dz
     float* bwd_part_w = nullptr;      // [partial_slots][d*d/2]    per-block sums of dW
     float* bwd_dstate = nullptr;      // [max_B*H][d*d + d]        dS, dz
-    // host-call staging
+    // host-call staging and its pipeline: copies in, compute and copies out run on three streams, one (b,h) at a time
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     size_t stage_bytes = 0;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_in = nullptr, ev_done = nullptr, ev_start = nullptr;
+    // while linattn_forward_host walks over the (b,h) pairs, the launchers see ONE group: head view_head0's weights,
+    // the state slots of group view_g0 (view_H == 0: the whole problem, the normal case)
+    int view_H = 0, view_head0 = 0;
+    long long view_g0 = 0;
     // options
     int opt_splits = 0;
     int opt_path = 0;
@@ -117,6 +123,8 @@ ActStrides act_strides(const linattn_ctx* c, int n)
     if (c->opt_layout == 1) return ActStrides{H * d, d, (long long)n * H * d};   // [B][n][H][d]
     return ActStrides{d, (long long)n * d, H * (long long)n * d};                 // [B][H][n][d]
 }
+
+int view_heads(const linattn_ctx* c) { return c->view_H ? c->view_H : c->H; }
 
 // Per-kernel timing: events are recorded around every launch of a forward and read back (after a
 // wait on the last one) at the start of the next profiled forward or when the figures are queried.
@@ -172,7 +180,11 @@ template <typename T, int D>
 linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int n,
                            cudaStream_t st, const void* mix, float mix_r)
 {
-    const long long G = (long long)B * c->H;
+    const int Hv = view_heads(c);
+    const long long G = (long long)B * Hv;
+    const float* Wq = c->Wq + (size_t)c->view_head0 * D * (D / 2);
+    const float* Wk = c->Wk + (size_t)c->view_head0 * D * (D / 2);
+    float* state = c->state + (size_t)c->view_g0 * (D * D + D);
     int splits = choose_splits(G, n, c->opt_splits);
     // token chunk per split, rounded up to the kernel's 32-token step; drop splits left empty
     int chunk = (n + splits - 1) / splits;
@@ -192,10 +204,10 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     const double side_bytes = 2.0 * (double)G * n * D * sizeof(T);  // K+V read, or Q read + O written
     prof_begin(c, st);
     kside_simt<T, D><<<dim3(splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
-        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, act_strides(c, n), c->opt_phi);
+        (const T*)k, (const T*)v, Wk, c->partial, Hv, n, chunk, act_strides(c, n), c->opt_phi);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_simt", side_bytes);
-    combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, c->state, splits, E);
+    combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, state, splits, E);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_state", 0.0);
     const int nchunks = (n + kSimtTokens - 1) / kSimtTokens;
@@ -203,7 +215,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     if (per_group > nchunks) per_group = nchunks;
     if (per_group < 1) per_group = 1;
     qside_simt<T, D><<<dim3((unsigned)per_group, (unsigned)G), kSimtThreads, qside_simt_smem<D>(), st>>>(
-        (const T*)q, c->Wq, c->state, (T*)out, c->H, n, (const T*)mix, mix_r, act_strides(c, n), c->opt_phi);
+        (const T*)q, Wq, state, (T*)out, Hv, n, (const T*)mix, mix_r, act_strides(c, n), c->opt_phi);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_simt", side_bytes);
     c->last_launches = 3;
@@ -271,7 +283,8 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
                          cudaStream_t st, const void* mix, float mix_r)
 {
     using namespace linattn::tc;
-    const long long G = (long long)B * c->H;
+    const int Hv = view_heads(c);
+    const long long G = (long long)B * Hv;
     const long long Tn = ((long long)n + kTile - 1) / kTile;
     const long long T = G * Tn;
     long long Pq = c->num_sms < T ? c->num_sms : T;
@@ -287,13 +300,13 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     const int layout = c->opt_layout;
     auto act_map = [&](CUtensorMap* m, const void* base) {
         if (layout == 0) return make_tmap_bf16_3d(m, base, kD, (uint64_t)n, (uint64_t)G, kTile);
-        return make_tmap_bf16_act(m, base, kD, (uint64_t)n, (uint64_t)c->H, (uint64_t)B, (uint64_t)as.token * 2,
+        return make_tmap_bf16_act(m, base, kD, (uint64_t)n, (uint64_t)Hv, (uint64_t)B, (uint64_t)as.token * 2,
                                   (uint64_t)as.head * 2, (uint64_t)as.batch * 2, kTile);
     };
     const bool ok = act_map(&tmK, k) && act_map(&tmV, v) && act_map(&tmQ, q) && act_map(&tmO, out) && act_map(&tmA, mix ? mix : q) &&
-                    make_tmap_bf16_3d(&tmWk, c->Wkt, kD, kM, (uint64_t)c->H, kM) &&
-                    make_tmap_bf16_3d(&tmWq, c->Wqt, kD, kM, (uint64_t)c->H, kM) &&
-                    make_tmap_bf16_3d(&tmS, c->s_img, kD, kD, (uint64_t)G, kTile);
+                    make_tmap_bf16_3d(&tmWk, c->Wkt + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
+                    make_tmap_bf16_3d(&tmWq, c->Wqt + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
+                    make_tmap_bf16_3d(&tmS, c->s_img + (size_t)c->view_g0 * kD * kD, kD, kD, (uint64_t)G, kTile);
     if (!ok) {
         snprintf(c->err_text, sizeof(c->err_text), "cuTensorMapEncodeTiled failed");
         return LINATTN_ERR_CUDA;
@@ -322,9 +335,9 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     const double side_bytes = 2.0 * (double)G * n * kD * 2;
     Args a{};
     a.partial = c->partial;
-    a.state = c->state;
-    a.s_img = c->s_img;
-    a.z_img = c->z_img;
+    a.state = c->state + (size_t)c->view_g0 * kE;
+    a.s_img = c->s_img + (size_t)c->view_g0 * kD * kD;
+    a.z_img = c->z_img + (size_t)c->view_g0 * (kZBlkBytes / 2);
     a.err = c->err_word;
     a.sync = c->sync_words;
     a.mix_src = (const __nv_bfloat16*)mix;
@@ -333,7 +346,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.str_head = as.head;
     a.str_batch = as.batch;
     a.n = n;
-    a.H = c->H;
+    a.H = Hv;
     a.G = (int)G;
     a.tiles_per_head = (int)Tn;
     a.total_tiles = T;
@@ -497,6 +510,11 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->bwd_part_w);
     cudaFree(c->bwd_dstate);
     for (void* p : c->stage) cudaFree(p);
+    if (c->copy_in) cudaStreamDestroy(c->copy_in);
+    if (c->copy_out) cudaStreamDestroy(c->copy_out);
+    if (c->ev_in) cudaEventDestroy(c->ev_in);
+    if (c->ev_done) cudaEventDestroy(c->ev_done);
+    if (c->ev_start) cudaEventDestroy(c->ev_start);
     for (cudaEvent_t ev : c->prof_ev)
         if (ev) cudaEventDestroy(ev);
     cudaGetLastError();
@@ -537,6 +555,9 @@ linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const voi
     return LINATTN_OK;
 }
 
+static linattn_status dispatch_forward(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, const void* mix,
+                                       float mix_r, int B, int n, int d, linattn_dtype dtype, cudaStream_t st);
+
 // Shared by linattn_forward (mix == NULL) and linattn_forward_mixed.
 static linattn_status forward_impl(linattn_ctx* c, const void* q, const void* k, const void* v, void* out,
                                    const void* mix, float mix_r, int B, int H, int n, int d, linattn_dtype dtype,
@@ -553,12 +574,17 @@ static linattn_status forward_impl(linattn_ctx* c, const void* q, const void* k,
         if (!(mix_r == mix_r)) return LINATTN_ERR_INVALID_ARG;                         // NaN
         mix_r = mix_r < 0.f ? 0.f : (mix_r > 1.f ? 1.f : mix_r);                       // footnote to Eq. 8: r is clipped into [0, 1]
     }
-    // The tensor-core kernels cover bf16 activations with head dimension 128 and bf16 feature-map weights;
-    // everything else runs on the CUDA-core kernels.
+    DeviceGuard guard(c->device);
+    return dispatch_forward(c, q, k, v, out, mix, mix_r, B, n, d, dtype, (cudaStream_t)stream);
+}
+
+// Choice of kernels for checked arguments.  The tensor-core kernels cover bf16 activations with head dimension 128
+// and bf16 feature-map weights; everything else runs on the CUDA-core kernels.
+static linattn_status dispatch_forward(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, const void* mix,
+                                       float mix_r, int B, int n, int d, linattn_dtype dtype, cudaStream_t st)
+{
     const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && (c->map_is_bf16 || c->opt_phi == 1));
     if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
-    DeviceGuard guard(c->device);
-    cudaStream_t st = (cudaStream_t)stream;
     c->last_B = B;
     c->state_transposed = tc_ok && c->opt_path != 1;
     if (c->state_transposed) return launch_tc(c, q, k, v, out, B, n, st, mix, mix_r);
@@ -642,13 +668,69 @@ linattn_status linattn_forward_host(linattn_ctx* c, const void* q, const void* k
         for (void*& p : c->stage) LA_CUDA(c, cudaMalloc(&p, bytes));
         c->stage_bytes = bytes;
     }
-    LA_CUDA(c, cudaMemcpyAsync(c->stage[0], q, bytes, cudaMemcpyHostToDevice, st));
-    LA_CUDA(c, cudaMemcpyAsync(c->stage[1], k, bytes, cudaMemcpyHostToDevice, st));
-    LA_CUDA(c, cudaMemcpyAsync(c->stage[2], v, bytes, cudaMemcpyHostToDevice, st));
-    s = linattn_forward(c, c->stage[0], c->stage[1], c->stage[2], c->stage[3], B, H, n, d, dtype, stream);
-    if (s != LINATTN_OK) return s;
-    LA_CUDA(c, cudaMemcpyAsync(out, c->stage[3], bytes, cudaMemcpyDeviceToHost, st));
-    LA_CUDA(c, cudaStreamSynchronize(st));
+    if (!c->copy_in) {
+        LA_CUDA(c, cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking));
+        LA_CUDA(c, cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking));
+        LA_CUDA(c, cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming));
+        LA_CUDA(c, cudaEventCreateWithFlags(&c->ev_done, cudaEventDisableTiming));
+        LA_CUDA(c, cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming));
+    }
+    char* sq = (char*)c->stage[0];
+    char* sk = (char*)c->stage[1];
+    char* sv = (char*)c->stage[2];
+    char* so = (char*)c->stage[3];
+    if (c->opt_layout != 0) {
+        // token-major layout: the heads are interleaved in memory, so the whole problem goes in one piece
+        LA_CUDA(c, cudaMemcpyAsync(sq, q, bytes, cudaMemcpyHostToDevice, st));
+        LA_CUDA(c, cudaMemcpyAsync(sk, k, bytes, cudaMemcpyHostToDevice, st));
+        LA_CUDA(c, cudaMemcpyAsync(sv, v, bytes, cudaMemcpyHostToDevice, st));
+        s = dispatch_forward(c, sq, sk, sv, so, nullptr, 0.f, B, n, d, dtype, st);
+        if (s != LINATTN_OK) return s;
+        LA_CUDA(c, cudaMemcpyAsync(out, so, bytes, cudaMemcpyDeviceToHost, st));
+        LA_CUDA(c, cudaStreamSynchronize(st));
+        return LINATTN_OK;
+    }
+    // [B][H][n][d]: the (b,h) pairs are independent and each is contiguous, so they go through a three-stage pipeline:
+    // copies in on one stream, the forward of one pair on the caller's stream, copies out on a third.  The two copy
+    // directions overlap, and the first pair is being computed while the rest is still arriving.
+    const size_t gbytes = (size_t)n * d * elem_size(dtype);
+    const long long G = (long long)B * H;
+    LA_CUDA(c, cudaEventRecord(c->ev_start, st));          // work queued on the caller's stream may still use the staging buffers
+    LA_CUDA(c, cudaStreamWaitEvent(c->copy_in, c->ev_start, 0));
+    LA_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->ev_start, 0));
+    linattn_status res = LINATTN_OK;
+    cudaError_t ce = cudaSuccess;
+    int launches = 0;
+    for (long long g = 0; g < G && res == LINATTN_OK && ce == cudaSuccess; ++g) {
+        const size_t off = (size_t)g * gbytes;
+        ce = cudaMemcpyAsync(sk + off, (const char*)k + off, gbytes, cudaMemcpyHostToDevice, c->copy_in);
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync(sv + off, (const char*)v + off, gbytes, cudaMemcpyHostToDevice, c->copy_in);
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync(sq + off, (const char*)q + off, gbytes, cudaMemcpyHostToDevice, c->copy_in);
+        if (ce == cudaSuccess) ce = cudaEventRecord(c->ev_in, c->copy_in);
+        if (ce == cudaSuccess) ce = cudaStreamWaitEvent(st, c->ev_in, 0);
+        if (ce != cudaSuccess) break;
+        c->view_H = 1;
+        c->view_head0 = (int)(g % H);
+        c->view_g0 = g;
+        res = dispatch_forward(c, sq + off, sk + off, sv + off, so + off, nullptr, 0.f, 1, n, d, dtype, st);
+        launches += c->last_launches;
+        c->view_H = 0;
+        c->view_head0 = 0;
+        c->view_g0 = 0;
+        if (res != LINATTN_OK) break;
+        ce = cudaEventRecord(c->ev_done, st);
+        if (ce == cudaSuccess) ce = cudaStreamWaitEvent(c->copy_out, c->ev_done, 0);
+        if (ce == cudaSuccess) ce = cudaMemcpyAsync((char*)out + off, so + off, gbytes, cudaMemcpyDeviceToHost, c->copy_out);
+    }
+    // drain all three streams whatever happened, so that no copy is left in flight on buffers the caller owns
+    const cudaError_t e1 = cudaStreamSynchronize(c->copy_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(c->copy_out);
+    c->last_B = B;
+    c->last_launches = launches;
+    if (res != LINATTN_OK) return res;
+    if (ce != cudaSuccess) return cuda_fail(c, ce, "pipelined host copy");
+    if (e1 != cudaSuccess) return cuda_fail(c, e1, "cudaStreamSynchronize(copy_in)");
+    if (e2 != cudaSuccess) return cuda_fail(c, e2, "cudaStreamSynchronize(stream)");
+    if (e3 != cudaSuccess) return cuda_fail(c, e3, "cudaStreamSynchronize(copy_out)");
     return LINATTN_OK;
 }
 

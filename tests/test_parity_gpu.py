@@ -170,19 +170,39 @@ def test_output_guard_bands_are_untouched():
         ctx.destroy()
 
 
-def test_host_buffer_entry_point_matches_device_entry_point():
-    x = small_inputs(1, 2, 1500, 128, torch.bfloat16, seed=12)
-    ctx = linattn.LinAttn(2, 128, max_B=1, max_n=1500)
+@pytest.mark.parametrize("B,H,n,d,dtype", [(1, 2, 1500, 128, torch.bfloat16), (2, 3, 700, 128, torch.bfloat16),
+                                           (2, 2, 300, 64, torch.float32)])
+def test_host_buffer_entry_point(B, H, n, d, dtype):
+    """Host buffers in, host buffer out; inside, the (b,h) pairs are pipelined one by one over three streams."""
+    x = small_inputs(B, H, n, d, dtype, seed=12 + B)
+    ctx = linattn.LinAttn(H, d, max_B=B, max_n=n)
     try:
         ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
-        dev = ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda()).cpu()
+        want, S_ref, z_ref = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], return_state=True)
         host_out = torch.empty_like(x["q"])
-        ctx.forward_host(x["q"], x["k"], x["v"], host_out)
-        assert torch.equal(dev, host_out)
+        ctx.forward_host(x["q"], x["k"], x["v"], host_out)          # pageable memory
+        ctx.check()
+        assert_parity(host_out.double().numpy(), want, "host entry point")
+        S, z = ctx.read_state(B)
+        assert errors(S.double().numpy(), S_ref)[0] <= 5e-3 and errors(z.double().numpy(), z_ref)[0] <= 5e-3
         pin = {k_: x[k_].pin_memory() for k_ in ("q", "k", "v")}
         host_out2 = torch.empty_like(x["q"]).pin_memory()
-        ctx.forward_host(pin["q"], pin["k"], pin["v"], host_out2)
-        assert torch.equal(dev, host_out2)
+        for _ in range(3):                                              # pinned memory: the copies overlap
+            host_out2.zero_()
+            ctx.forward_host(pin["q"], pin["k"], pin["v"], host_out2)
+            assert torch.equal(host_out, host_out2)
+        # the device entry point on the same context afterwards is undisturbed
+        dev = ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda()).cpu()
+        ctx.check()
+        assert_parity(dev.double().numpy(), want, "device entry point after the host one")
+        rel, _ = errors(host_out.double().numpy(), dev.double().numpy())
+        assert rel <= 5e-3
+        # token-major layout: one piece
+        ctx.set_option(linattn.OPT_LAYOUT, linattn.LAYOUT_BNHD)
+        tm = lambda t: t.permute(0, 2, 1, 3).contiguous().view(B, H, n, d)
+        host_out3 = torch.empty_like(x["q"])
+        ctx.forward_host(tm(x["q"]), tm(x["k"]), tm(x["v"]), host_out3)
+        assert torch.equal(host_out3.view(B, n, H, d).permute(0, 2, 1, 3), dev)
     finally:
         ctx.destroy()
 
