@@ -13,6 +13,7 @@
 #include "simt_kernels.cuh"
 #include "simt_backward.cuh"
 #include "sm100_kernels.cuh"
+#include "sm100_backward.cuh"
 #include "tensor_map.hpp"
 
 using namespace linattn;
@@ -64,6 +65,7 @@ struct linattn_ctx {
     float* bwd_part_state = nullptr;  // [partial_slots][d*d + d]  per-block sums of dS, dz
     float* bwd_part_w = nullptr;      // [partial_slots][d*d/2]    per-block sums of dW
     float* bwd_dstate = nullptr;      // [max_B*H][d*d + d]        dS, dz
+    __nv_bfloat16* bwd_img[3] = {nullptr, nullptr, nullptr};   // tensor-core backward: lo image of S, hi and lo images of dS
     // host-call staging and its pipeline: copies in, compute and copies out run on three streams, one (b,h) at a time
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     size_t stage_bytes = 0;
@@ -280,7 +282,7 @@ linattn_status launch_backward_simt(linattn_ctx* c, const void* q, const void* k
 
 // Tensor-core path: bf16, d = 128.
 linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int n,
-                         cudaStream_t st, const void* mix, float mix_r)
+                         cudaStream_t st, const void* mix, float mix_r, bool state_only = false)
 {
     using namespace linattn::tc;
     const int Hv = view_heads(c);
@@ -354,7 +356,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.trace = c->trace;
 #endif
     prof_begin(c, st);
-    if (c->opt_fuse && c->coop_ok && Pk == Pq) {
+    if (c->opt_fuse && c->coop_ok && Pk == Pq && !state_only) {
         // one cooperative launch: key side, grid barrier, combine, grid barrier, query side
         a.bar_target[0] = c->bar_total + (uint32_t)Pq;
         a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
@@ -383,6 +385,10 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     combine_tc<<<dim3((kE / 4 + 255) / 256, (unsigned)G), 256, 0, st>>>(a, Pk);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_tc", 0.0);
+    if (state_only) {   // the backward pass wants S and z only
+        c->last_launches = 2;
+        return LINATTN_OK;
+    }
     {
         void* qp[] = {&tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
         LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout][phi], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
@@ -390,6 +396,88 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);
     c->last_launches = 3;
+    return LINATTN_OK;
+}
+
+// Gradients on the tensor-core kernels (bf16, d = 128, bf16 feature-map weights): S, z by the forward's key-side
+// kernels, then the query side (dq; dS, dz, dW_q records), the combines, and the key side (dk, dv; dW_k records).
+linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, const void* v, const void* dout, void* dq,
+                                  void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int n, cudaStream_t st)
+{
+    using namespace linattn::tc;
+    const long long G = (long long)B * c->H;
+    const long long Tn = ((long long)n + kTile - 1) / kTile;
+    const long long T = G * Tn;
+    const long long P = c->num_sms < T ? c->num_sms : T;
+    if (P + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
+    // forward state (S as [c][f], z) and the hi image of S; q and out are not touched by the first two kernels
+    linattn_status s = launch_tc(c, k, k, v, dk, B, n, st, nullptr, 0.f, true);
+    if (s != LINATTN_OK) return s;
+
+    const ActStrides as = act_strides(c, n);
+    const int layout = c->opt_layout;
+    auto act_map = [&](CUtensorMap* m, const void* base) {
+        if (layout == 0) return make_tmap_bf16_3d(m, base, kD, (uint64_t)n, (uint64_t)G, kTile);
+        return make_tmap_bf16_act(m, base, kD, (uint64_t)n, (uint64_t)c->H, (uint64_t)B, (uint64_t)as.token * 2,
+                                  (uint64_t)as.head * 2, (uint64_t)as.batch * 2, kTile);
+    };
+    auto img_map = [&](CUtensorMap* m, const void* base) { return make_tmap_bf16_3d(m, base, kD, kD, (uint64_t)G, kTile); };
+    CUtensorMap tmQ, tmG, tmDQ, tmK, tmV, tmDK, tmDV, tmWq, tmWk, tmShi, tmSlo, tmDShi, tmDSlo;
+    const bool ok = act_map(&tmQ, q) && act_map(&tmG, dout) && act_map(&tmDQ, dq) && act_map(&tmK, k) && act_map(&tmV, v) &&
+                    act_map(&tmDK, dk) && act_map(&tmDV, dv) &&
+                    make_tmap_bf16_3d(&tmWq, c->Wqt, kD, kM, (uint64_t)c->H, kM) &&
+                    make_tmap_bf16_3d(&tmWk, c->Wkt, kD, kM, (uint64_t)c->H, kM) && img_map(&tmShi, c->s_img) &&
+                    img_map(&tmSlo, c->bwd_img[0]) && img_map(&tmDShi, c->bwd_img[1]) && img_map(&tmDSlo, c->bwd_img[2]);
+    if (!ok) {
+        snprintf(c->err_text, sizeof(c->err_text), "cuTensorMapEncodeTiled failed");
+        return LINATTN_ERR_CUDA;
+    }
+    const void* k_q[2] = {(const void*)qside_bwd_tc<0>, (const void*)qside_bwd_tc<1>};
+    const void* k_k[2] = {(const void*)kside_bwd_tc<0>, (const void*)kside_bwd_tc<1>};
+    bool& attr_done = c->attr_done[9];
+    if (!attr_done) {
+        for (int i = 0; i < 2; ++i) {
+            LA_CUDA(c, cudaFuncSetAttribute(k_q[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemQ));
+            LA_CUDA(c, cudaFuncSetAttribute(k_k[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemK));
+        }
+        attr_done = true;
+    }
+    const double tensor_bytes = (double)G * n * kD * 2;
+    BwdArgs a{};
+    a.part_state = c->bwd_part_state;
+    a.part_w = c->bwd_part_w;
+    a.state = c->state;
+    a.err = c->err_word;
+    a.n = n;
+    a.H = c->H;
+    a.G = (int)G;
+    a.tiles_per_head = (int)Tn;
+    a.total_tiles = T;
+    const dim3 wgrid(kWRec / 256, per_head ? (unsigned)c->H : 1u);
+    hilo_images<<<dim3(kD * kD / 256, (unsigned)G), 256, 0, st>>>(c->state, nullptr, c->bwd_img[0]);
+    LA_CUDA(c, cudaGetLastError());
+    {
+        void* p[] = {&tmQ, &tmG, &tmDQ, &tmWq, &tmShi, &tmSlo, &a};
+        LA_CUDA(c, cudaLaunchKernel(k_q[layout], dim3((unsigned)P), dim3(kBwdThreads), p, kBwdSmemQ, st));
+    }
+    prof_mark(c, st, "qside_bwd_tc", 3.0 * tensor_bytes);
+    combine_slots<<<dim3((kE + 255) / 256, (unsigned)G), 256, 0, st>>>(c->bwd_part_state, c->bwd_dstate, kE, (int)Tn, T, P);
+    LA_CUDA(c, cudaGetLastError());
+    hilo_images<<<dim3(kD * kD / 256, (unsigned)G), 256, 0, st>>>(c->bwd_dstate, c->bwd_img[1], c->bwd_img[2]);
+    LA_CUDA(c, cudaGetLastError());
+    combine_wgrad_slots<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWq, (int)G, c->H, per_head, (int)Tn, T, P);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "combine_dstate_dWq", 0.0);
+    a.state = c->bwd_dstate;
+    {
+        void* p[] = {&tmK, &tmV, &tmDK, &tmDV, &tmWk, &tmDShi, &tmDSlo, &a};
+        LA_CUDA(c, cudaLaunchKernel(k_k[layout], dim3((unsigned)P), dim3(kBwdThreads), p, kBwdSmemK, st));
+    }
+    prof_mark(c, st, "kside_bwd_tc", 4.0 * tensor_bytes);
+    combine_wgrad_slots<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWk, (int)G, c->H, per_head, (int)Tn, T, P);
+    LA_CUDA(c, cudaGetLastError());
+    prof_mark(c, st, "combine_dWk", 0.0);
+    c->last_launches = 9;
     return LINATTN_OK;
 }
 
@@ -509,6 +597,7 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->bwd_part_state);
     cudaFree(c->bwd_part_w);
     cudaFree(c->bwd_dstate);
+    for (void* p : c->bwd_img) cudaFree(p);
     for (void* p : c->stage) cudaFree(p);
     if (c->copy_in) cudaStreamDestroy(c->copy_in);
     if (c->copy_out) cudaStreamDestroy(c->copy_out);
@@ -638,10 +727,19 @@ linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, co
         LA_CUDA(c, cudaMalloc(&c->bwd_part_state, sizeof(float) * E * (size_t)c->partial_slots));
         LA_CUDA(c, cudaMalloc(&c->bwd_part_w, sizeof(float) * (size_t)d * (d / 2) * (size_t)c->partial_slots));
         LA_CUDA(c, cudaMalloc(&c->bwd_dstate, sizeof(float) * E * (size_t)(c->max_B * c->H)));
+        if (d == 128)
+            for (__nv_bfloat16*& p : c->bwd_img) LA_CUDA(c, cudaMalloc(&p, sizeof(__nv_bfloat16) * (size_t)d * d * (size_t)(c->max_B * c->H)));
     }
     c->last_B = B;
-    c->state_transposed = false;
     const int ph = per_head ? 1 : 0;
+    const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && c->map_is_bf16);
+    if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
+    if (tc_ok && c->opt_path != 1) {
+        c->state_transposed = true;
+        prof_begin(c, st);
+        return launch_backward_tc(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
+    }
+    c->state_transposed = false;
     if (dtype == LINATTN_BF16) {
         return d == 128 ? launch_backward_simt<__nv_bfloat16, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st)
                         : launch_backward_simt<__nv_bfloat16, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);

@@ -1,0 +1,652 @@
+// Tensor-core kernels (tcgen05 + TMEM + TMA) for the gradients of linear attention with the Hedgehog feature map
+// (what Eq. 14 back-propagates through Eq. 5 and Eq. 6), bf16 storage, head dimension 128.
+//
+// With dO the incoming gradient, den_i = phi(q_i).z, o_i = phi(q_i) S / den_i:
+//     dnum_i = dO_i / den_i                  dden_i = -(dO_i . o_i) / den_i
+//     dphi(q_i) = S dnum_i + dden_i z        dS = sum_i phi(q_i)^T dnum_i       dz = sum_i dden_i phi(q_i)
+//     dphi(k_j) = dS v_j + dz                dv_j = dS^T phi(k_j)
+//     du = p+ (.) (dphi+ - p+ . dphi+) - p- (.) (dphi- - p- . dphi-)       dx = du W^T       dW += x^T du
+//
+// Two kernels of persistent CTAs, each walking its contiguous run of 128-token tiles one tile at a time; the
+// stages of a tile run one after the other (no software pipeline: the first aim here is a correct tensor-core
+// path; every matrix product is a tcgen05.mma with fp32 accumulators in TMEM, every element-wise step runs on all
+// 256 threads, thread = (token, half of the features)):
+//
+//   qside_bwd_tc : U = Q W_q -> phi(q) -> num = phi S, den -> dnum, dden -> dphi = dnum S^T (+ dden z),
+//                  dS += phi^T dnum, dz += phi^T dden -> du -> dq = du W_q^T (TMA store), dW_q += Q^T du
+//   kside_bwd_tc : U = K W_k -> phi(k) -> dphi = V dS^T (+ dz), dv = phi dS (TMA store) -> du ->
+//                  dk = du W_k^T (TMA store), dW_k += K^T du
+//
+// Operands that carry a difference of nearly equal terms downstream are split into bf16 hi + lo parts and
+// multiplied in two or three passes: S and dS (images written by the combine kernels) and dnum.  phi and du are
+// single bf16 operands, as phi is in the forward.
+// Accumulators that live across tiles (dS, dW) are written as one record per (CTA, head) and summed in CTA
+// order by the combine kernels, so the gradients are bit-reproducible.  Every wait is bounded.
+#pragma once
+#include "sm100_kernels.cuh"
+
+namespace linattn {
+namespace tc {
+
+constexpr int kBwdThreads = 256;
+constexpr int kWRec = kM * kD;   // floats per weight-gradient record, stored [j][c]
+
+struct BwdArgs {
+    float* part_state;     // [slots][kE]: per (CTA, head) sums of dS as [c][f], then dz   (query side writes)
+    float* part_w;         // [slots][kWRec]: per (CTA, head) sums of dW as [j][c]
+    const float* state;    // [G][kE]: query side: S as [c][f], then z; key side: dS as [c][f], then dz
+    uint32_t* err;
+    int n, H, G, tiles_per_head;
+    long long total_tiles;
+};
+
+struct BwdSmemQ {   // query side
+    static constexpr uint32_t kX = 0;                        // Q tile
+    static constexpr uint32_t kG = kX + kTileBytes;          // dO tile -> dnum (hi) -> du (first 16 KB)
+    static constexpr uint32_t kL = kG + kTileBytes;          // dnum (lo) -> fp32 scratch for du
+    static constexpr uint32_t kP = kL + kTileBytes;          // phi(q) -> dq staging
+    static constexpr uint32_t kShi = kP + kTileBytes;        // S image [c][f], hi part
+    static constexpr uint32_t kSlo = kShi + kTileBytes;      // lo part
+    static constexpr uint32_t kW = kSlo + kTileBytes;        // W_q^T [64][128]
+    static constexpr uint32_t kMisc = kW + kWBytes;
+};
+struct BwdSmemK {   // key side
+    static constexpr uint32_t kX = 0;                        // K tile
+    static constexpr uint32_t kV = kX + kTileBytes;          // V tile -> fp32 scratch for du -> dk staging
+    static constexpr uint32_t kP = kV + kTileBytes;          // phi(k) -> dv staging
+    static constexpr uint32_t kShi = kP + kTileBytes;        // dS image [c][f], hi part
+    static constexpr uint32_t kSlo = kShi + kTileBytes;
+    static constexpr uint32_t kW = kSlo + kTileBytes;        // W_k^T [64][128]
+    static constexpr uint32_t kDu = kW + kWBytes;            // du tile [128][64] bf16
+    static constexpr uint32_t kMisc = kDu + kWBytes;
+};
+// misc block: z / dz vector, per-token scalars, barriers, TMEM slot, abort word
+struct BwdMisc {
+    static constexpr uint32_t kVec = 0;           // 128 floats: z (query side) or dz (key side)
+    static constexpr uint32_t kA = 512;           // 2 x 128 floats: den halves, later dz halves
+    static constexpr uint32_t kB = 1536;          // 2 x 128 floats: (dO . o) halves
+    static constexpr uint32_t kDd = 2560;         // 128 floats: dden
+    static constexpr uint32_t kBars = 3072;       // 3 mbarriers, TMEM slot, abort word
+    static constexpr uint32_t kBytes = 3072 + 64;
+};
+constexpr uint32_t kBwdSmemQ = BwdSmemQ::kMisc + BwdMisc::kBytes + 1024;
+constexpr uint32_t kBwdSmemK = BwdSmemK::kMisc + BwdMisc::kBytes + 1024;
+
+enum : int { BW_LOAD = 0, BW_SEG = 1, BW_MMA = 2 };
+
+struct BwdCta {
+    uint8_t* smem;
+    uint32_t sbase, bar0, tmem;
+    float* misc;
+    WaitCtx wc;
+    __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * (uint32_t)i; }
+};
+
+__device__ __forceinline__ BwdCta bwd_setup(uint8_t* smem_raw, uint32_t misc_off, uint32_t* err)
+{
+    BwdCta c;
+    c.smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    c.sbase = smem_u32(c.smem);
+    c.misc = reinterpret_cast<float*>(c.smem + misc_off);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(c.smem + misc_off + BwdMisc::kBars);
+    c.bar0 = smem_u32(bars);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[3]);
+    uint32_t* abort_word = tmem_slot + 1;
+    c.wc.err = err;
+    c.wc.abort_smem = smem_u32(abort_word);
+    if (threadIdx.x == 0) {
+        *abort_word = 0u;
+        for (int i = 0; i < 3; ++i) mbar_init(c.bar(i), 1);
+        fence_mbar_init();
+    }
+    if ((threadIdx.x >> 5) == 1) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    fence_proxy_async_smem();
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    c.tmem = *tmem_slot;
+    return c;
+}
+
+__device__ __forceinline__ void bwd_teardown(const BwdCta& c)
+{
+    if (threadIdx.x == 0) bulk_wait_group<0>();
+    tcgen05_fence_before();
+    __syncthreads();
+    if ((threadIdx.x >> 5) == 1) tmem_dealloc(c.tmem, 512);
+}
+
+// All threads of the CTA wait (bounded) for the barrier's phase; the verdict is the same for every thread, so the
+// stage loop never leaves some threads behind at a CTA barrier.
+__device__ __forceinline__ bool cta_wait(const BwdCta& c, int b, uint32_t& phase, uint32_t code)
+{
+    const bool ok = warp_wait(c.bar(b), phase, c.wc, code);
+    phase ^= 1u;
+    const bool all = __syncthreads_and(ok ? 1 : 0) != 0;
+    tcgen05_fence_after();
+    return all;
+}
+
+// Byte offset of 16-byte chunk `ch` (8 bf16) of row `row` inside a 64-column block of a TMA tile (128-byte swizzle).
+__device__ __forceinline__ uint32_t sw_chunk(int row, int ch) { return (uint32_t)row * 128u + (uint32_t)((ch ^ (row & 7)) << 4); }
+
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+// One softmax half of Eq. 6 for one token: u[64] logits in, p[64] (fp32) out in place; the bf16 values go to the
+// token's 128-byte row of the half's 64-feature block (operand layout).  Returns sum_j bf16(p_j) * vec[j].
+template <bool kNeg>
+__device__ __forceinline__ float softmax_half_keep(float (&u)[kM], uint8_t* blk, int row, const float* vec)
+{
+    float m = u[0];
+#pragma unroll
+    for (int j = 1; j < kM; ++j) m = kNeg ? fminf(m, u[j]) : fmaxf(m, u[j]);
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < kM; ++j) {
+        u[j] = ex2_approx((kNeg ? m - u[j] : u[j] - m) * kLog2e);
+        sum += u[j];
+    }
+    const float inv = 1.f / sum;
+    float dot = 0.f;
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int j = 8 * ch + 2 * q;
+            u[j] *= inv;
+            u[j + 1] *= inv;
+            w[q] = pack_bf16(u[j], u[j + 1]);
+            dot = fmaf(bf16_round(u[j]), vec[j], dot);
+            dot = fmaf(bf16_round(u[j + 1]), vec[j + 1], dot);
+        }
+        *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    return dot;
+}
+
+__device__ __forceinline__ void load64(uint32_t taddr, float (&x)[kM])
+{
+    uint32_t r[kM];
+    tmem_ld_x32(taddr, r);
+    tmem_ld_x32(taddr + 32, r + 32);
+    tmem_wait_ld();
+#pragma unroll
+    for (int j = 0; j < kM; ++j) x[j] = __uint_as_float(r[j]);
+}
+
+// 64 floats of one token -> bf16 row of a 64-column block (operand / TMA-store layout).
+__device__ __forceinline__ void store_row_bf16(uint8_t* blk, int row, const float (&x)[kM])
+{
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) w[q] = pack_bf16(x[8 * ch + 2 * q], x[8 * ch + 2 * q + 1]);
+        *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+// fp32 scratch tile [128 tokens][64]: 16-byte chunk ch of row r sits at chunk ch ^ (r & 15) (no bank conflicts
+// when the threads of a warp, one row each, touch the same logical chunk).
+__device__ __forceinline__ float4* scratch_chunk(uint8_t* scratch, int row, int ch)
+{
+    return reinterpret_cast<float4*>(scratch + (size_t)row * 256 + ((ch ^ (row & 15)) << 4));
+}
+
+// Softmax backward of Eq. 6 for one token, split between the two threads of the token (half 0: softmax(+u),
+// half 1: softmax(-u)): each forms p (.) (dphi - p . dphi) for its half; half 1 parks its values in the scratch
+// tile, and after a CTA barrier half 0 subtracts them and writes du (bf16) to its row of the du tile.
+__device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint8_t* scratch,
+                                            uint8_t* du_tile)
+{
+    float dot = 0.f;
+#pragma unroll
+    for (int j = 0; j < kM; ++j) dot = fmaf(p[j], dphi[j], dot);
+#pragma unroll
+    for (int j = 0; j < kM; ++j) dphi[j] = p[j] * (dphi[j] - dot);
+    if (half == 1) {
+#pragma unroll
+        for (int ch = 0; ch < 16; ++ch)
+            *scratch_chunk(scratch, row, ch) = make_float4(dphi[4 * ch], dphi[4 * ch + 1], dphi[4 * ch + 2], dphi[4 * ch + 3]);
+    }
+    __syncthreads();
+    if (half == 0) {
+#pragma unroll
+        for (int ch = 0; ch < 16; ++ch) {
+            const float4 o = *scratch_chunk(scratch, row, ch);
+            dphi[4 * ch] -= o.x;
+            dphi[4 * ch + 1] -= o.y;
+            dphi[4 * ch + 2] -= o.z;
+            dphi[4 * ch + 3] -= o.w;
+        }
+        store_row_bf16(du_tile, row, dphi);
+    }
+}
+
+// K-major operand (rows x K, K contiguous in 64-element blocks `blk_bytes` apart): address of K step k (16 elements).
+__device__ __forceinline__ uint32_t kstep_kmajor(uint32_t base, int k, uint32_t blk_bytes) { return base + (uint32_t)(k >> 2) * blk_bytes + (uint32_t)(k & 3) * 32u; }
+
+// dx = du W^T and dW += x^T du for one tile (issued by one thread): A of the first product is the du tile (K-major,
+// K = 64), B the W^T image [j][c] read MN-major; the second product reads the x tile MN-major (x^T) and du MN-major.
+__device__ __forceinline__ void issue_dx_dw(uint32_t t_dx, uint32_t t_dw, uint32_t du, uint32_t x, uint32_t w, bool first_of_segment)
+{
+    constexpr uint32_t idesc_dx = make_idesc_bf16(kTile, kD, 0, 1);
+    constexpr uint32_t idesc_dw = make_idesc_bf16(kD, kM, 1, 1);
+    const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
+    const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
+    const uint64_t mn_w = make_desc_sw128(0, kWBytes / 2, 1024);
+#pragma unroll
+    for (int k = 0; k < kM / 16; ++k)
+        mma_bf16_ss(t_dx, desc_at(kmajor, du + k * 32), desc_at(mn_w, w + k * 2048), idesc_dx, k > 0);
+#pragma unroll
+    for (int k = 0; k < kTile / 16; ++k)
+        mma_bf16_ss(t_dw, desc_at(mn_tile, x + k * 2048), desc_at(mn_tile, du + k * 2048), idesc_dw, (first_of_segment && k == 0) ? 0u : 1u);
+}
+
+// Write the weight-gradient accumulator (TMEM: lane = input feature c, 64 columns = logits j) as a [j][c] record.
+__device__ __forceinline__ void drain_dw(uint32_t t_dw, uint32_t lane_base, int half, int row, float* rec)
+{
+    uint32_t v[32];
+    tmem_ld_x32(t_dw + lane_base + half * 32, v);
+    tmem_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) rec[(size_t)(half * 32 + j) * kD + row] = __uint_as_float(v[j]);
+}
+
+template <int kLayout>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
+             const __grid_constant__ CUtensorMap tmDQ, const __grid_constant__ CUtensorMap tmW,
+             const __grid_constant__ CUtensorMap tmShi, const __grid_constant__ CUtensorMap tmSlo, const BwdArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    using L = BwdSmemQ;
+    const BwdCta c = bwd_setup(smem_raw, L::kMisc, a.err);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int half = warp >> 2, row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t t_u = c.tmem, t_work = c.tmem + 64, t_ds = c.tmem + 208, t_dw = c.tmem + 336;
+    float* vec = c.misc + BwdMisc::kVec / 4;
+    float* sa = c.misc + BwdMisc::kA / 4;
+    float* sb = c.misc + BwdMisc::kB / 4;
+    float* sdd = c.misc + BwdMisc::kDd / 4;
+    const uint32_t sb0 = c.sbase;
+    const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
+    const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
+    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0;
+    float dz_acc = 0.f;   // thread (f = tid & 127, token half = tid >> 7)
+    TileWalk w;
+    w.init(a.total_tiles, a.tiles_per_head);
+    if (tid == 0) {
+        tma_prefetch_desc(&tmQ);
+        tma_prefetch_desc(&tmG);
+        tma_prefetch_desc(&tmDQ);
+    }
+
+    for (; !w.done(); w.next()) {
+        const bool first = w.first(), last = w.last();
+        // ---- loads: per head S (hi, lo), W_q^T, z; per tile Q and dO ----
+        if (tid == 0) {
+            if (first) {
+                mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, w.g);
+                    tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, w.g);
+                    tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, w.g % a.H);
+                }
+            }
+            mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
+            for (int b = 0; b < 2; ++b) {
+                act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmQ, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
+                act_load<kLayout>(sb0 + L::kG + b * kHalfTileBytes, &tmG, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
+            }
+            TileWalk nx = w;   // the next tile's rows start on their way into L2 while this one is worked on
+            nx.next();
+            if (!nx.done())
+                for (int b = 0; b < 2; ++b) {
+                    act_prefetch_l2<kLayout>(&tmQ, 64 * b, nx.lt * kTile, nx.g, a.H);
+                    act_prefetch_l2<kLayout>(&tmG, 64 * b, nx.lt * kTile, nx.g, a.H);
+                }
+        }
+        if (first) {
+            if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];
+            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) break;
+        }
+        if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) break;
+        // ---- U = Q W_q ----
+        if (tid == 0) {
+            issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
+            mma_commit(c.bar(BW_MMA));
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
+        // ---- phi(q): bf16 operand tile; p stays in registers; den = phi . z from the rounded values ----
+        float p[kM];
+        load64(t_u + lane_base, p);
+        {
+            uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
+            sa[half * kTile + row] = half == 0 ? softmax_half_keep<false>(p, blk, row, vec) : softmax_half_keep<true>(p, blk, row, vec + kM);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        // ---- num = phi (S_hi + S_lo) ----
+        if (tid == 0) {
+            tcgen05_fence_after();
+            constexpr uint32_t idesc = make_idesc_bf16(kTile, kD, 0, 0);
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass)
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k)
+                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)),
+                                desc_at(kmajor, kstep_kmajor(sb0 + (pass == 0 ? L::kShi : L::kSlo), k, kHalfTileBytes)), idesc,
+                                (pass | k) != 0);
+            mma_commit(c.bar(BW_MMA));
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrEpilogue)) break;
+        // ---- dnum = dO / den (hi over dO in place, lo beside it), (dO . o) per half ----
+        float inv;
+        {
+            float x[kM];
+            load64(t_work + lane_base + half * kM, x);
+            inv = 1.f / (sa[row] + sa[kTile + row]);
+            uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
+            uint8_t* lblk = c.smem + L::kL + half * kHalfTileBytes;
+            float go = 0.f;
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+                const uint32_t off = sw_chunk(row, ch);
+                const uint4 gv = *reinterpret_cast<const uint4*>(gblk + off);
+                const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float g0 = __uint_as_float(gw[q] << 16), g1 = __uint_as_float(gw[q] & 0xffff0000u);
+                    go = fmaf(g0, x[8 * ch + 2 * q] * inv, go);
+                    go = fmaf(g1, x[8 * ch + 2 * q + 1] * inv, go);
+                    const float d0 = g0 * inv, d1 = g1 * inv;
+                    const float h0 = bf16_round(d0), h1 = bf16_round(d1);
+                    hi[q] = pack_bf16(h0, h1);
+                    lo[q] = pack_bf16(d0 - h0, d1 - h1);
+                }
+                *reinterpret_cast<uint4*>(gblk + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(lblk + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+            sb[half * kTile + row] = go;
+        }
+        tcgen05_fence_before();
+        __syncthreads();
+        const float dden = -(sb[row] + sb[kTile + row]) * inv;
+        if (half == 0) sdd[row] = dden;
+        fence_proxy_async_smem();
+        __syncthreads();
+        // ---- dphi = dnum S^T (three hi/lo passes), dS += phi^T dnum (two passes) ----
+        if (tid == 0) {
+            tcgen05_fence_after();
+            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = dnum (K-major over c), B = S image [c][f] (rows = K)
+            constexpr uint32_t idesc_ds = make_idesc_bf16(kD, kD, 1, 1);        // A = phi^T, B = dnum, both read MN-major
+#pragma unroll
+            for (int pass = 0; pass < 3; ++pass) {
+                const uint32_t at = sb0 + (pass == 1 ? L::kL : L::kG), st = sb0 + (pass == 2 ? L::kSlo : L::kShi);
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k)
+                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(at, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
+                                (pass | k) != 0);
+            }
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass)
+#pragma unroll
+                for (int k = 0; k < kTile / 16; ++k)
+                    mma_bf16_ss(t_ds, desc_at(mn_tile, sb0 + L::kP + k * 2048), desc_at(mn_tile, sb0 + (pass == 0 ? L::kG : L::kL) + k * 2048),
+                                idesc_ds, (first && pass == 0 && k == 0) ? 0u : 1u);
+            mma_commit(c.bar(BW_MMA));
+        }
+        {
+            // dz += phi^T dden on the CUDA cores while the tensor core works: thread = (feature f, half of the tokens)
+            const int f = tid & (kD - 1), t0 = (tid >> 7) * (kTile / 2);
+            const uint8_t* blk = c.smem + L::kP + (f >> 6) * kHalfTileBytes;
+            const int ch = (f & 63) >> 3, e = (f & 7) * 2;
+#pragma unroll 8
+            for (int t = t0; t < t0 + kTile / 2; ++t) {
+                const __nv_bfloat16 pv = *reinterpret_cast<const __nv_bfloat16*>(blk + sw_chunk(t, ch) + e);
+                dz_acc = fmaf(sdd[t], __bfloat162float(pv), dz_acc);
+            }
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrMmaAcc)) break;
+        // ---- du (through the softmax of Eq. 6) ----
+        {
+            float x[kM];
+            load64(t_work + lane_base + half * kM, x);
+#pragma unroll
+            for (int j = 0; j < kM; ++j) x[j] = fmaf(dden, vec[half * kM + j], x[j]);
+            du_exchange(half, row, p, x, c.smem + L::kL, c.smem + L::kG);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        // ---- dq = du W_q^T, dW_q += Q^T du ----
+        if (tid == 0) {
+            tcgen05_fence_after();
+            issue_dx_dw(t_work, t_dw, sb0 + L::kG, sb0 + L::kX, sb0 + L::kW, first);
+            mma_commit(c.bar(BW_MMA));
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
+        {
+            float x[kM];
+            load64(t_work + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+            bulk_commit_group();
+        }
+        // ---- end of this CTA's part of the head: the accumulators go to the (CTA, head) records ----
+        if (last) {
+            tcgen05_fence_after();
+            float* rec = a.part_state + (size_t)(blockIdx.x + w.g) * kE;
+            {
+                float x[kM];
+                load64(t_ds + lane_base + half * kM, x);   // lane = feature f, columns = c
+#pragma unroll
+                for (int j = 0; j < kM; ++j) rec[(size_t)(half * kM + j) * kD + row] = x[j];
+            }
+            drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
+            sa[tid] = dz_acc;
+            dz_acc = 0.f;
+            __syncthreads();
+            if (tid < kD) rec[kD * kD + tid] = sa[tid] + sa[kD + tid];
+        }
+        if (tid == 0) bulk_wait_group_read<0>();   // the staging tile is phi's home again at the next tile
+        tcgen05_fence_before();
+        __syncthreads();
+    }
+    bwd_teardown(c);
+}
+
+template <int kLayout>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+             const __grid_constant__ CUtensorMap tmDK, const __grid_constant__ CUtensorMap tmDV,
+             const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmShi,
+             const __grid_constant__ CUtensorMap tmSlo, const BwdArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    using L = BwdSmemK;
+    const BwdCta c = bwd_setup(smem_raw, L::kMisc, a.err);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int half = warp >> 2, row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t t_u = c.tmem, t_w1 = c.tmem + 64, t_w2 = c.tmem + 192, t_dw = c.tmem + 320;
+    float* vec = c.misc + BwdMisc::kVec / 4;
+    const uint32_t sb0 = c.sbase;
+    const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
+    const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
+    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0;
+    TileWalk w;
+    w.init(a.total_tiles, a.tiles_per_head);
+    if (tid == 0) {
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+        tma_prefetch_desc(&tmDK);
+        tma_prefetch_desc(&tmDV);
+    }
+
+    for (; !w.done(); w.next()) {
+        const bool first = w.first(), last = w.last();
+        if (tid == 0) {
+            if (first) {
+                mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, w.g);
+                    tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, w.g);
+                    tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, w.g % a.H);
+                }
+            }
+            mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
+            for (int b = 0; b < 2; ++b) {
+                act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmK, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
+                act_load<kLayout>(sb0 + L::kV + b * kHalfTileBytes, &tmV, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
+            }
+            TileWalk nx = w;
+            nx.next();
+            if (!nx.done())
+                for (int b = 0; b < 2; ++b) {
+                    act_prefetch_l2<kLayout>(&tmK, 64 * b, nx.lt * kTile, nx.g, a.H);
+                    act_prefetch_l2<kLayout>(&tmV, 64 * b, nx.lt * kTile, nx.g, a.H);
+                }
+        }
+        if (first) {
+            if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // dz
+            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) break;
+        }
+        if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) break;
+        // ---- U = K W_k ----
+        if (tid == 0) {
+            issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
+            mma_commit(c.bar(BW_MMA));
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
+        float p[kM];
+        load64(t_u + lane_base, p);
+        {
+            uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
+            if (half == 0) softmax_half_keep<false>(p, blk, row, vec);
+            else softmax_half_keep<true>(p, blk, row, vec + kM);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        // ---- dphi = V dS^T, dv = phi dS (hi and lo parts of dS) ----
+        if (tid == 0) {
+            tcgen05_fence_after();
+            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = V (K-major over c), B = dS image [c][f] (rows = K)
+            constexpr uint32_t idesc_dv = make_idesc_bf16(kTile, kD, 0, 0);     // A = phi (K-major over f), B = dS image [c][f] (rows = N)
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass) {
+                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k) {
+                    mma_bf16_ss(t_w1, desc_at(kmajor, kstep_kmajor(sb0 + L::kV, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
+                                (pass | k) != 0);
+                    mma_bf16_ss(t_w2, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)), desc_at(kmajor, kstep_kmajor(st, k, kHalfTileBytes)),
+                                idesc_dv, (pass | k) != 0);
+                }
+            }
+            mma_commit(c.bar(BW_MMA));
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrMmaAcc)) break;
+        // ---- du; dv leaves through phi's tile ----
+        {
+            float x[kM];
+            load64(t_w1 + lane_base + half * kM, x);
+#pragma unroll
+            for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
+            du_exchange(half, row, p, x, c.smem + L::kV, c.smem + L::kDu);
+            load64(t_w2 + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        // ---- dk = du W_k^T, dW_k += K^T du ----
+        if (tid == 0) {
+            tcgen05_fence_after();
+            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+            bulk_commit_group();
+            issue_dx_dw(t_w1, t_dw, sb0 + L::kDu, sb0 + L::kX, sb0 + L::kW, first);
+            mma_commit(c.bar(BW_MMA));
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
+        {
+            float x[kM];
+            load64(t_w1 + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kV + half * kHalfTileBytes, row, x);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, sb0 + L::kV + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+            bulk_commit_group();
+        }
+        if (last) {
+            tcgen05_fence_after();
+            drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
+        }
+        if (tid == 0) bulk_wait_group_read<0>();
+        tcgen05_fence_before();
+        __syncthreads();
+    }
+    bwd_teardown(c);
+}
+
+// out[g][e] = sum over the CTAs that own tiles of head g, ascending, of part[(cta + g)][e].  grid = (ceil(E/256), G).
+static __global__ void __launch_bounds__(256)
+combine_slots(const float* __restrict__ part, float* __restrict__ out, int E, int tiles_per_head, long long total_tiles, long long P)
+{
+    const int e = blockIdx.x * 256 + threadIdx.x;
+    if (e >= E) return;
+    const int g = blockIdx.y;
+    const long long c0 = tile_owner((long long)g * tiles_per_head, total_tiles, P);
+    const long long c1 = tile_owner((long long)(g + 1) * tiles_per_head - 1, total_tiles, P);
+    float acc = 0.f;
+    for (long long cta = c0; cta <= c1; ++cta) acc += part[(size_t)(cta + g) * E + e];
+    out[(size_t)g * E + e] = acc;
+}
+
+// Matrix part of a state record ([c][f] fp32) -> bf16 hi and lo images (either may be NULL).  grid = (64, G).
+static __global__ void __launch_bounds__(256)
+hilo_images(const float* __restrict__ state, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo)
+{
+    const int e = blockIdx.x * 256 + threadIdx.x, g = blockIdx.y;
+    const float x = state[(size_t)g * kE + e];
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    if (hi) hi[(size_t)g * kD * kD + e] = h;
+    if (lo) lo[(size_t)g * kD * kD + e] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+// dW[w][c][j] = sum over the heads g that use weight matrix w (per_head: g % H == w; shared: all), ascending, and
+// over the CTAs of each, ascending, of part_w[(cta + g)][j][c].  grid = (kWRec / 256, per_head ? H : 1).
+static __global__ void __launch_bounds__(256)
+combine_wgrad_slots(const float* __restrict__ part_w, float* __restrict__ dW, int G, int H, int per_head, int tiles_per_head,
+                    long long total_tiles, long long P)
+{
+    const int o = blockIdx.x * 256 + threadIdx.x;   // output index c * 64 + j
+    const int cc = o / kM, j = o % kM, wsel = blockIdx.y;
+    float acc = 0.f;
+    for (int g = per_head ? wsel : 0; g < G; g += per_head ? H : 1) {
+        const long long c0 = tile_owner((long long)g * tiles_per_head, total_tiles, P);
+        const long long c1 = tile_owner((long long)(g + 1) * tiles_per_head - 1, total_tiles, P);
+        for (long long cta = c0; cta <= c1; ++cta) acc += part_w[(size_t)(cta + g) * kWRec + (size_t)j * kD + cc];
+    }
+    dW[(size_t)wsel * kWRec + o] = acc;
+}
+
+}  // namespace tc
+}  // namespace linattn
