@@ -53,6 +53,11 @@ typedef enum {
                                needed), no epsilon (a query whose phi is orthogonal to every key's gives a non-finite
                                row).  Applies to linattn_forward, _mixed and _host; linattn_backward then returns
                                UNSUPPORTED */
+    LINATTN_OPT_REUSE_STATE = 6, /* 1 = linattn_backward (tensor-core path) takes S and z from the workspace instead of
+                               recomputing them when the most recent state-producing call on this context was a forward
+                               (or backward) on the same k and v POINTERS, B, n and layout, with the same feature map.
+                               The caller promises that the contents of k and v have not changed in between (the
+                               forward -> backward order of a training step).  0 = always recompute (default) */
     LINATTN_OPT_PROFILE = 2 /* 1 = record CUDA events around every kernel of each forward (see linattn_profile_get);
                                switching it on clears the accumulated figures; 0 = off (default) */
 } linattn_option;

@@ -81,6 +81,14 @@ struct linattn_ctx {
     int opt_fuse = 1;
     int opt_layout = 0;   // 0: [B][H][n][d], 1: [B][n][H][d]
     int opt_phi = 0;      // 0: Hedgehog feature map (Eq. 6), 1: ReLU kernel function
+    int opt_reuse = 0;    // 1: linattn_backward may take S, z from the forward that just ran on the same k, v
+    // which problem the S, z (tensor-core layout, with the bf16 image of S) in the workspace belong to
+    struct StateKey {
+        const void* k = nullptr;
+        const void* v = nullptr;
+        int B = 0, n = 0, layout = 0;
+        bool valid = false;
+    } state_key;
     // per-kernel timing (LINATTN_OPT_PROFILE)
     static constexpr int kMaxKernels = 8;
     bool profile = false;
@@ -410,9 +418,20 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     const long long T = G * Tn;
     const long long P = c->num_sms < T ? c->num_sms : T;
     if (P + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
-    // forward state (S as [c][f], z) and the hi image of S; q and out are not touched by the first two kernels
-    linattn_status s = launch_tc(c, k, k, v, dk, B, n, st, nullptr, 0.f, true);
-    if (s != LINATTN_OK) return s;
+    // forward state (S as [c][f], z) and the hi image of S: left by the forward that just ran on these k, v (if the
+    // caller allows it), else recomputed; q and out are not touched by the first two kernels of the forward
+    const linattn_ctx::StateKey& sk = c->state_key;
+    const bool reuse = c->opt_reuse && sk.valid && sk.k == k && sk.v == v && sk.B == B && sk.n == n && sk.layout == c->opt_layout;
+    int launches = 7;
+    if (reuse) {
+        prof_begin(c, st);
+    } else {
+        c->state_key.valid = false;
+        const linattn_status s = launch_tc(c, k, k, v, dk, B, n, st, nullptr, 0.f, true);
+        if (s != LINATTN_OK) return s;
+        c->state_key = {k, v, B, n, c->opt_layout, true};
+        launches = 9;
+    }
 
     const ActStrides as = act_strides(c, n);
     const int layout = c->opt_layout;
@@ -477,7 +496,7 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     combine_wgrad_slots<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWk, (int)G, c->H, per_head, (int)Tn, T, P);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_dWk", 0.0);
-    c->last_launches = 9;
+    c->last_launches = launches;
     return LINATTN_OK;
 }
 
@@ -641,6 +660,7 @@ linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const voi
     LA_CUDA(c, cudaGetLastError());
     c->map_is_bf16 = (wdtype == LINATTN_BF16);
     c->have_map = true;
+    c->state_key.valid = false;
     return LINATTN_OK;
 }
 
@@ -676,7 +696,12 @@ static linattn_status dispatch_forward(linattn_ctx* c, const void* q, const void
     if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
     c->last_B = B;
     c->state_transposed = tc_ok && c->opt_path != 1;
-    if (c->state_transposed) return launch_tc(c, q, k, v, out, B, n, st, mix, mix_r);
+    c->state_key.valid = false;
+    if (c->state_transposed) {
+        const linattn_status s = launch_tc(c, q, k, v, out, B, n, st, mix, mix_r);
+        if (s == LINATTN_OK && c->opt_phi == 0 && c->view_H == 0) c->state_key = {k, v, B, n, c->opt_layout, true};
+        return s;
+    }
     if (dtype == LINATTN_BF16) {
         return d == 128 ? launch_simt<__nv_bfloat16, 128>(c, q, k, v, out, B, n, st, mix, mix_r)
                         : launch_simt<__nv_bfloat16, 64>(c, q, k, v, out, B, n, st, mix, mix_r);
@@ -736,10 +761,10 @@ linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, co
     if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
     if (tc_ok && c->opt_path != 1) {
         c->state_transposed = true;
-        prof_begin(c, st);
         return launch_backward_tc(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
     }
     c->state_transposed = false;
+    c->state_key.valid = false;
     if (dtype == LINATTN_BF16) {
         return d == 128 ? launch_backward_simt<__nv_bfloat16, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st)
                         : launch_backward_simt<__nv_bfloat16, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
@@ -824,6 +849,7 @@ linattn_status linattn_forward_host(linattn_ctx* c, const void* q, const void* k
     const cudaError_t e1 = cudaStreamSynchronize(c->copy_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(c->copy_out);
     c->last_B = B;
     c->last_launches = launches;
+    c->state_key.valid = false;
     if (res != LINATTN_OK) return res;
     if (ce != cudaSuccess) return cuda_fail(c, ce, "pipelined host copy");
     if (e1 != cudaSuccess) return cuda_fail(c, e1, "cudaStreamSynchronize(copy_in)");
@@ -881,6 +907,10 @@ linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long 
         case LINATTN_OPT_KERNEL_FUNCTION:
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
             c->opt_phi = (int)value;
+            return LINATTN_OK;
+        case LINATTN_OPT_REUSE_STATE:
+            if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
+            c->opt_reuse = (int)value;
             return LINATTN_OK;
         case LINATTN_OPT_FUSE:
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;

@@ -159,6 +159,43 @@ def test_config2_full_size_two_heads_against_the_oracle():
         _assert_grads(mine, want, f"config 2, head {h}")
 
 
+def test_state_left_by_the_forward_is_reused_only_when_it_belongs_to_the_same_problem():
+    x = _inputs(1, 3, 900, 128, torch.bfloat16, seed=38)
+    y = _inputs(1, 3, 900, 128, torch.bfloat16, seed=39)
+    ctx = linattn.LinAttn(3, 128, max_B=1, max_n=900)
+    try:
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        dx = [x[s].cuda() for s in ("q", "k", "v", "dout")]
+        dy = [y[s].cuda() for s in ("q", "k", "v", "dout")]
+        ref_x = ctx.backward(*dx)
+        ref_y = ctx.backward(*dy)
+        assert ctx.last_launch_count() == 9
+        ctx.set_option(linattn.OPT_REUSE_STATE, 1)
+        ctx.forward(dx[0], dx[1], dx[2])
+        got = ctx.backward(*dx)                       # same k, v as the forward: S, z are taken over
+        assert ctx.last_launch_count() == 7
+        for a, b in zip(got, ref_x):
+            assert torch.equal(a, b)
+        got = ctx.backward(*dy)                       # other k, v: recomputed
+        assert ctx.last_launch_count() == 9
+        for a, b in zip(got, ref_y):
+            assert torch.equal(a, b)
+        got = ctx.backward(*dy)                       # the backward's own state counts too
+        assert ctx.last_launch_count() == 7
+        for a, b in zip(got, ref_y):
+            assert torch.equal(a, b)
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())   # new weights: nothing is taken over
+        ctx.backward(*dy)
+        assert ctx.last_launch_count() == 9
+        ctx.forward(dx[0], dx[1], dx[2])
+        ctx.set_option(linattn.OPT_REUSE_STATE, 0)
+        ctx.backward(*dx)
+        assert ctx.last_launch_count() == 9
+        ctx.check()
+    finally:
+        ctx.destroy()
+
+
 def test_argument_errors():
     lib = linattn.load_library()
     x = _inputs(1, 2, 128, 64, torch.float32, seed=35)
