@@ -472,6 +472,9 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     a.G = (int)G;
     a.tiles_per_head = (int)Tn;
     a.total_tiles = T;
+#ifdef LINATTN_TRACE
+    a.trace = c->trace;
+#endif
     const dim3 wgrid(kWRec / 256, per_head ? (unsigned)c->H : 1u);
     hilo_images<<<dim3(kD * kD / 256, (unsigned)G), 256, 0, st>>>(c->state, nullptr, c->bwd_img[0]);
     LA_CUDA(c, cudaGetLastError());

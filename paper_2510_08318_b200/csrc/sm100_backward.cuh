@@ -38,7 +38,19 @@ struct BwdArgs {
     uint32_t* err;
     int n, H, G, tiles_per_head;
     long long total_tiles;
+#ifdef LINATTN_TRACE
+    long long* trace;      // tuning builds: [CTA][tile < 8][16] clock64 stamps of the stages of a tile
+#endif
 };
+
+#ifdef LINATTN_TRACE
+#define LB_TRACE(ev)                                                                                                  \
+    do {                                                                                                              \
+        if (a.trace && threadIdx.x == 0 && w.i < 8) a.trace[((size_t)blockIdx.x * 8 + w.i) * 16 + (ev)] = clock64(); \
+    } while (0)
+#else
+#define LB_TRACE(ev) do { } while (0)
+#endif
 
 struct BwdSmemQ {   // query side
     static constexpr uint32_t kX = 0;                        // Q tile
@@ -52,8 +64,8 @@ struct BwdSmemQ {   // query side
 };
 struct BwdSmemK {   // key side
     static constexpr uint32_t kX = 0;                        // K tile
-    static constexpr uint32_t kV = kX + kTileBytes;          // V tile -> fp32 scratch for du -> dk staging
-    static constexpr uint32_t kP = kV + kTileBytes;          // phi(k) -> dv staging
+    static constexpr uint32_t kV = kX + kTileBytes;          // V tile -> fp32 scratch for du
+    static constexpr uint32_t kP = kV + kTileBytes;          // phi(k) -> dv staging -> dk staging
     static constexpr uint32_t kShi = kP + kTileBytes;        // dS image [c][f], hi part
     static constexpr uint32_t kSlo = kShi + kTileBytes;
     static constexpr uint32_t kW = kSlo + kTileBytes;        // W_k^T [64][128]
@@ -133,24 +145,27 @@ __device__ __forceinline__ bool cta_wait(const BwdCta& c, int b, uint32_t& phase
 // Byte offset of 16-byte chunk `ch` (8 bf16) of row `row` inside a 64-column block of a TMA tile (128-byte swizzle).
 __device__ __forceinline__ uint32_t sw_chunk(int row, int ch) { return (uint32_t)row * 128u + (uint32_t)((ch ^ (row & 7)) << 4); }
 
-__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
-
 // One softmax half of Eq. 6 for one token: u[64] logits in, p[64] (fp32) out in place; the bf16 values go to the
 // token's 128-byte row of the half's 64-feature block (operand layout).  Returns sum_j bf16(p_j) * vec[j].
 template <bool kNeg>
 __device__ __forceinline__ float softmax_half_keep(float (&u)[kM], uint8_t* blk, int row, const float* vec)
 {
-    float m = u[0];
+    float m = kNeg ? min3(u[0], u[1], u[2]) : max3(u[0], u[1], u[2]);
 #pragma unroll
-    for (int j = 1; j < kM; ++j) m = kNeg ? fminf(m, u[j]) : fmaxf(m, u[j]);
-    float sum = 0.f;
+    for (int j = 3; j < kM - 1; j += 2) m = kNeg ? min3(m, u[j], u[j + 1]) : max3(m, u[j], u[j + 1]);
+    m = kNeg ? fminf(m, u[kM - 1]) : fmaxf(m, u[kM - 1]);
+    // exp(u - max) = 2^(u*log2e - max*log2e);   exp(-u - max(-u)) = 2^(min*log2e - u*log2e)
+    const float sL = kNeg ? -kLog2e : kLog2e, off = kNeg ? m * kLog2e : -m * kLog2e;
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int j = 0; j < kM; ++j) {
-        u[j] = ex2_approx((kNeg ? m - u[j] : u[j] - m) * kLog2e);
-        sum += u[j];
+    for (int j = 0; j < kM; j += 2) {
+        u[j] = ex2_approx(fmaf(u[j], sL, off));
+        u[j + 1] = ex2_approx(fmaf(u[j + 1], sL, off));
+        s0 += u[j];
+        s1 += u[j + 1];
     }
-    const float inv = 1.f / sum;
-    float dot = 0.f;
+    const float inv = __fdividef(1.f, s0 + s1);
+    float d0 = 0.f, d1 = 0.f;
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch) {
         uint32_t w[4];
@@ -160,12 +175,12 @@ __device__ __forceinline__ float softmax_half_keep(float (&u)[kM], uint8_t* blk,
             u[j] *= inv;
             u[j + 1] *= inv;
             w[q] = pack_bf16(u[j], u[j + 1]);
-            dot = fmaf(bf16_round(u[j]), vec[j], dot);
-            dot = fmaf(bf16_round(u[j + 1]), vec[j + 1], dot);
+            d0 = fmaf(__uint_as_float(w[q] << 16), vec[j], d0);            // the rounded values, as the tensor core sees them
+            d1 = fmaf(__uint_as_float(w[q] & 0xffff0000u), vec[j + 1], d1);
         }
         *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    return dot;
+    return d0 + d1;
 }
 
 __device__ __forceinline__ void load64(uint32_t taddr, float (&x)[kM])
@@ -278,7 +293,9 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
     const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
     uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0;
-    float dz_acc = 0.f;   // thread (f = tid & 127, token half = tid >> 7)
+    float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dz_acc[e] = 0.f;
     TileWalk w;
     w.init(a.total_tiles, a.tiles_per_head);
     if (tid == 0) {
@@ -287,42 +304,50 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         tma_prefetch_desc(&tmDQ);
     }
 
+    // Loads of one tile (issued by one thread): Q and dO, at the start of a head also S (hi, lo) and W_q^T; the tile
+    // after it starts on its way into L2.
+    auto issue_loads = [&](const TileWalk& t) {
+        if (t.first()) {
+            mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
+            for (int b = 0; b < 2; ++b) {
+                tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
+                tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
+                tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
+            }
+        }
+        mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
+        for (int b = 0; b < 2; ++b) {
+            act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmQ, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+            act_load<kLayout>(sb0 + L::kG + b * kHalfTileBytes, &tmG, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+        }
+        TileWalk nx = t;
+        nx.next();
+        if (!nx.done())
+            for (int b = 0; b < 2; ++b) {
+                act_prefetch_l2<kLayout>(&tmQ, 64 * b, nx.lt * kTile, nx.g, a.H);
+                act_prefetch_l2<kLayout>(&tmG, 64 * b, nx.lt * kTile, nx.g, a.H);
+            }
+    };
+    if (tid == 0 && !w.done()) issue_loads(w);
+
     for (; !w.done(); w.next()) {
         const bool first = w.first(), last = w.last();
-        // ---- loads: per head S (hi, lo), W_q^T, z; per tile Q and dO ----
-        if (tid == 0) {
-            if (first) {
-                mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
-                for (int b = 0; b < 2; ++b) {
-                    tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, w.g);
-                    tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, w.g);
-                    tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, w.g % a.H);
-                }
-            }
-            mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
-            for (int b = 0; b < 2; ++b) {
-                act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmQ, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
-                act_load<kLayout>(sb0 + L::kG + b * kHalfTileBytes, &tmG, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
-            }
-            TileWalk nx = w;   // the next tile's rows start on their way into L2 while this one is worked on
-            nx.next();
-            if (!nx.done())
-                for (int b = 0; b < 2; ++b) {
-                    act_prefetch_l2<kLayout>(&tmQ, 64 * b, nx.lt * kTile, nx.g, a.H);
-                    act_prefetch_l2<kLayout>(&tmG, 64 * b, nx.lt * kTile, nx.g, a.H);
-                }
-        }
+        LB_TRACE(0);
+        // ---- this tile's Q and dO (and, at the start of a head, S hi/lo, W_q^T) were requested one tile ago ----
         if (first) {
             if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];
             if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) break;
         }
         if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) break;
+        LB_TRACE(1);
         // ---- U = Q W_q ----
         if (tid == 0) {
             issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
             mma_commit(c.bar(BW_MMA));
+            bulk_wait_group_read<0>();   // the previous tile's dq has left the staging tile, which is phi's home again
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
+        LB_TRACE(2);
         // ---- phi(q): bf16 operand tile; p stays in registers; den = phi . z from the rounded values ----
         float p[kM];
         load64(t_u + lane_base, p);
@@ -333,6 +358,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
+        LB_TRACE(3);
         // ---- num = phi (S_hi + S_lo) ----
         if (tid == 0) {
             tcgen05_fence_after();
@@ -347,6 +373,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             mma_commit(c.bar(BW_MMA));
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrEpilogue)) break;
+        LB_TRACE(4);
         // ---- dnum = dO / den (hi over dO in place, lo beside it), (dO . o) per half ----
         float inv;
         {
@@ -368,9 +395,8 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     go = fmaf(g0, x[8 * ch + 2 * q] * inv, go);
                     go = fmaf(g1, x[8 * ch + 2 * q + 1] * inv, go);
                     const float d0 = g0 * inv, d1 = g1 * inv;
-                    const float h0 = bf16_round(d0), h1 = bf16_round(d1);
-                    hi[q] = pack_bf16(h0, h1);
-                    lo[q] = pack_bf16(d0 - h0, d1 - h1);
+                    hi[q] = pack_bf16(d0, d1);
+                    lo[q] = pack_bf16(d0 - __uint_as_float(hi[q] << 16), d1 - __uint_as_float(hi[q] & 0xffff0000u));
                 }
                 *reinterpret_cast<uint4*>(gblk + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<uint4*>(lblk + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
@@ -383,6 +409,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (half == 0) sdd[row] = dden;
         fence_proxy_async_smem();
         __syncthreads();
+        LB_TRACE(5);
         // ---- dphi = dnum S^T (three hi/lo passes), dS += phi^T dnum (two passes) ----
         if (tid == 0) {
             tcgen05_fence_after();
@@ -405,17 +432,25 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             mma_commit(c.bar(BW_MMA));
         }
         {
-            // dz += phi^T dden on the CUDA cores while the tensor core works: thread = (feature f, half of the tokens)
-            const int f = tid & (kD - 1), t0 = (tid >> 7) * (kTile / 2);
-            const uint8_t* blk = c.smem + L::kP + (f >> 6) * kHalfTileBytes;
-            const int ch = (f & 63) >> 3, e = (f & 7) * 2;
-#pragma unroll 8
-            for (int t = t0; t < t0 + kTile / 2; ++t) {
-                const __nv_bfloat16 pv = *reinterpret_cast<const __nv_bfloat16*>(blk + sw_chunk(t, ch) + e);
-                dz_acc = fmaf(sdd[t], __bfloat162float(pv), dz_acc);
+            // dz += phi^T dden on the CUDA cores while the tensor core works: thread = (16-byte chunk of 8 features,
+            // group of 8 tokens)
+            const int fc = tid & 15, t0 = (tid >> 4) * 8;
+            const uint8_t* blk = c.smem + L::kP + (fc >> 3) * kHalfTileBytes;
+#pragma unroll
+            for (int t = t0; t < t0 + 8; ++t) {
+                const uint4 pv = *reinterpret_cast<const uint4*>(blk + sw_chunk(t, fc & 7));
+                const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
+                const float dd = sdd[t];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    dz_acc[2 * q] = fmaf(dd, __uint_as_float(pw[q] << 16), dz_acc[2 * q]);
+                    dz_acc[2 * q + 1] = fmaf(dd, __uint_as_float(pw[q] & 0xffff0000u), dz_acc[2 * q + 1]);
+                }
             }
         }
+        LB_TRACE(6);
         if (!cta_wait(c, BW_MMA, ph_mma, kErrMmaAcc)) break;
+        LB_TRACE(7);
         // ---- du (through the softmax of Eq. 6) ----
         {
             float x[kM];
@@ -427,6 +462,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
+        LB_TRACE(8);
         // ---- dq = du W_q^T, dW_q += Q^T du ----
         if (tid == 0) {
             tcgen05_fence_after();
@@ -434,6 +470,13 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             mma_commit(c.bar(BW_MMA));
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
+        LB_TRACE(9);
+        if (tid == 0) {
+            // every operand tile of this tile has been consumed: the next tile's loads overlap the store of this one
+            TileWalk nx = w;
+            nx.next();
+            if (!nx.done()) issue_loads(nx);
+        }
         {
             float x[kM];
             load64(t_work + lane_base + half * kM, x);
@@ -442,6 +485,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
+        LB_TRACE(10);
         if (tid == 0) {
             for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
             bulk_commit_group();
@@ -457,14 +501,24 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 for (int j = 0; j < kM; ++j) rec[(size_t)(half * kM + j) * kD + row] = x[j];
             }
             drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
-            sa[tid] = dz_acc;
-            dz_acc = 0.f;
+            // dz: the 16 token groups' sums, in group order (the scratch tile is free at this point)
+            float* red = reinterpret_cast<float*>(c.smem + L::kL);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                red[(tid >> 4) * kD + (tid & 15) * 8 + e] = dz_acc[e];
+                dz_acc[e] = 0.f;
+            }
             __syncthreads();
-            if (tid < kD) rec[kD * kD + tid] = sa[tid] + sa[kD + tid];
+            if (tid < kD) {
+                float acc = 0.f;
+#pragma unroll
+                for (int gidx = 0; gidx < 16; ++gidx) acc += red[gidx * kD + tid];
+                rec[kD * kD + tid] = acc;
+            }
         }
-        if (tid == 0) bulk_wait_group_read<0>();   // the staging tile is phi's home again at the next tile
         tcgen05_fence_before();
         __syncthreads();
+        LB_TRACE(11);
     }
     bwd_teardown(c);
 }
@@ -497,30 +551,33 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tma_prefetch_desc(&tmDV);
     }
 
+    // Loads of one tile (issued by one thread): K and V, at the start of a head also dS (hi, lo) and W_k^T.
+    auto issue_loads = [&](const TileWalk& t) {
+        if (t.first()) {
+            mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
+            for (int b = 0; b < 2; ++b) {
+                tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
+                tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
+                tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
+            }
+        }
+        mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
+        for (int b = 0; b < 2; ++b) {
+            act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmK, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+            act_load<kLayout>(sb0 + L::kV + b * kHalfTileBytes, &tmV, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+        }
+        TileWalk nx = t;
+        nx.next();
+        if (!nx.done())
+            for (int b = 0; b < 2; ++b) {
+                act_prefetch_l2<kLayout>(&tmK, 64 * b, nx.lt * kTile, nx.g, a.H);
+                act_prefetch_l2<kLayout>(&tmV, 64 * b, nx.lt * kTile, nx.g, a.H);
+            }
+    };
+    if (tid == 0 && !w.done()) issue_loads(w);
+
     for (; !w.done(); w.next()) {
         const bool first = w.first(), last = w.last();
-        if (tid == 0) {
-            if (first) {
-                mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
-                for (int b = 0; b < 2; ++b) {
-                    tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, w.g);
-                    tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, w.g);
-                    tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, w.g % a.H);
-                }
-            }
-            mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
-            for (int b = 0; b < 2; ++b) {
-                act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmK, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
-                act_load<kLayout>(sb0 + L::kV + b * kHalfTileBytes, &tmV, c.bar(BW_LOAD), 64 * b, w.lt * kTile, w.g, a.H);
-            }
-            TileWalk nx = w;
-            nx.next();
-            if (!nx.done())
-                for (int b = 0; b < 2; ++b) {
-                    act_prefetch_l2<kLayout>(&tmK, 64 * b, nx.lt * kTile, nx.g, a.H);
-                    act_prefetch_l2<kLayout>(&tmV, 64 * b, nx.lt * kTile, nx.g, a.H);
-                }
-        }
         if (first) {
             if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // dz
             if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) break;
@@ -530,6 +587,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         if (tid == 0) {
             issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
             mma_commit(c.bar(BW_MMA));
+            bulk_wait_group_read<0>();   // the previous tile's dk has left phi's tile
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
         float p[kM];
@@ -583,23 +641,31 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             mma_commit(c.bar(BW_MMA));
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
+        if (tid == 0) {
+            // K, V (its tile served as scratch) and the du tile have been consumed: the next tile's loads start now and
+            // overlap this tile's stores; dk is staged in phi's tile once dv has left it
+            TileWalk nx = w;
+            nx.next();
+            if (!nx.done()) issue_loads(nx);
+            bulk_wait_group_read<0>();
+        }
+        __syncthreads();
         {
             float x[kM];
             load64(t_w1 + lane_base + half * kM, x);
-            store_row_bf16(c.smem + L::kV + half * kHalfTileBytes, row, x);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
         }
         fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
         if (tid == 0) {
-            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, sb0 + L::kV + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
             bulk_commit_group();
         }
         if (last) {
             tcgen05_fence_after();
             drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
         }
-        if (tid == 0) bulk_wait_group_read<0>();
         tcgen05_fence_before();
         __syncthreads();
     }
@@ -637,15 +703,15 @@ static __global__ void __launch_bounds__(256)
 combine_wgrad_slots(const float* __restrict__ part_w, float* __restrict__ dW, int G, int H, int per_head, int tiles_per_head,
                     long long total_tiles, long long P)
 {
-    const int o = blockIdx.x * 256 + threadIdx.x;   // output index c * 64 + j
-    const int cc = o / kM, j = o % kM, wsel = blockIdx.y;
+    const int r = blockIdx.x * 256 + threadIdx.x;   // index in a record, j * 128 + c: neighbouring threads read neighbouring words
+    const int j = r / kD, cc = r % kD, wsel = blockIdx.y;
     float acc = 0.f;
     for (int g = per_head ? wsel : 0; g < G; g += per_head ? H : 1) {
         const long long c0 = tile_owner((long long)g * tiles_per_head, total_tiles, P);
         const long long c1 = tile_owner((long long)(g + 1) * tiles_per_head - 1, total_tiles, P);
-        for (long long cta = c0; cta <= c1; ++cta) acc += part_w[(size_t)(cta + g) * kWRec + (size_t)j * kD + cc];
+        for (long long cta = c0; cta <= c1; ++cta) acc += part_w[(size_t)(cta + g) * kWRec + r];
     }
-    dW[(size_t)wsel * kWRec + o] = acc;
+    dW[(size_t)wsel * kWRec + (size_t)cc * kM + j] = acc;
 }
 
 }  // namespace tc
