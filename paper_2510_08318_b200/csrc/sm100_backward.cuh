@@ -12,14 +12,16 @@
 // path; every matrix product is a tcgen05.mma with fp32 accumulators in TMEM, every element-wise step runs on all
 // 256 threads, thread = (token, half of the features)):
 //
-//   qside_bwd_tc : U = Q W_q -> phi(q) -> num = phi S, den -> dnum, dden -> dphi = dnum S^T (+ dden z),
-//                  dS += phi^T dnum, dz += phi^T dden -> du -> dq = du W_q^T (TMA store), dW_q += Q^T du
+//   qside_bwd_tc : U = Q W_q -> phi(q) -> num = phi S, den, dO . o -> dphi = (dO S^T - (dO . o) z) / den,
+//                  dS += (phi / den)^T dO, dz += (phi / den)^T (dden den) -> du -> dq = du W_q^T (TMA store),
+//                  dW_q += Q^T du
 //   kside_bwd_tc : U = K W_k -> phi(k) -> dphi = V dS^T (+ dz), dv = phi dS (TMA store) -> du ->
 //                  dk = du W_k^T (TMA store), dW_k += K^T du
 //
-// Operands that carry a difference of nearly equal terms downstream are split into bf16 hi + lo parts and
-// multiplied in two or three passes: S and dS (images written by the combine kernels) and dnum.  phi and du are
-// single bf16 operands, as phi is in the forward.
+// Operands that carry a difference of nearly equal terms downstream are kept exact or split into bf16 hi + lo
+// parts: S and dS are hi + lo images written by the combine kernels (two passes each); dnum = dO / den is never
+// formed: its per-token factor 1 / den is applied to the accumulator (dphi) or folded into phi (dS), so that the
+// dO tile, exact in bf16, is the operand.  phi, phi / den and du are single bf16 operands, as phi is in the forward.
 // Accumulators that live across tiles (dS, dW) are written as one record per (CTA, head) and summed in CTA
 // order by the combine kernels, so the gradients are bit-reproducible.  Every wait is bounded.
 #pragma once
@@ -54,9 +56,9 @@ struct BwdArgs {
 
 struct BwdSmemQ {   // query side
     static constexpr uint32_t kX = 0;                        // Q tile
-    static constexpr uint32_t kG = kX + kTileBytes;          // dO tile -> dnum (hi) -> du (first 16 KB)
-    static constexpr uint32_t kL = kG + kTileBytes;          // dnum (lo) -> fp32 scratch for du
-    static constexpr uint32_t kP = kL + kTileBytes;          // phi(q) -> dq staging
+    static constexpr uint32_t kG = kX + kTileBytes;          // dO tile -> du (first 16 KB)
+    static constexpr uint32_t kL = kG + kTileBytes;          // fp32 scratch for du, and for the dz sums at the end of a head
+    static constexpr uint32_t kP = kL + kTileBytes;          // phi(q) -> phi(q) / den -> dq staging
     static constexpr uint32_t kShi = kP + kTileBytes;        // S image [c][f], hi part
     static constexpr uint32_t kSlo = kShi + kTileBytes;      // lo part
     static constexpr uint32_t kW = kSlo + kTileBytes;        // W_q^T [64][128]
@@ -374,66 +376,62 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrEpilogue)) break;
         LB_TRACE(4);
-        // ---- dnum = dO / den (hi over dO in place, lo beside it), (dO . o) per half ----
+        // ---- den, dO . o.  The per-token factor 1 / den of dnum = dO / den is kept OUT of the tensor-core operands: dphi
+        // = (dO S^T) / den is scaled in the accumulator's epilogue, and dS = (phi / den)^T dO takes it into phi, so
+        // the dO tile itself, exact in bf16, is the operand of both products ----
         float inv;
         {
             float x[kM];
             load64(t_work + lane_base + half * kM, x);
             inv = 1.f / (sa[row] + sa[kTile + row]);
-            uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
-            uint8_t* lblk = c.smem + L::kL + half * kHalfTileBytes;
-            float go = 0.f;
+            const uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
+            float g0s = 0.f, g1s = 0.f;
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
-                const uint32_t off = sw_chunk(row, ch);
-                const uint4 gv = *reinterpret_cast<const uint4*>(gblk + off);
+                const uint4 gv = *reinterpret_cast<const uint4*>(gblk + sw_chunk(row, ch));
                 const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
-                uint32_t hi[4], lo[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const float g0 = __uint_as_float(gw[q] << 16), g1 = __uint_as_float(gw[q] & 0xffff0000u);
-                    go = fmaf(g0, x[8 * ch + 2 * q] * inv, go);
-                    go = fmaf(g1, x[8 * ch + 2 * q + 1] * inv, go);
-                    const float d0 = g0 * inv, d1 = g1 * inv;
-                    hi[q] = pack_bf16(d0, d1);
-                    lo[q] = pack_bf16(d0 - __uint_as_float(hi[q] << 16), d1 - __uint_as_float(hi[q] & 0xffff0000u));
+                    g0s = fmaf(__uint_as_float(gw[q] << 16), x[8 * ch + 2 * q], g0s);
+                    g1s = fmaf(__uint_as_float(gw[q] & 0xffff0000u), x[8 * ch + 2 * q + 1], g1s);
                 }
-                *reinterpret_cast<uint4*>(gblk + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4*>(lblk + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
-            sb[half * kTile + row] = go;
+            sb[half * kTile + row] = (g0s + g1s) * inv;   // this half's part of dO . o
+            // phi / den over phi (the numerator MMA is done with it); p itself stays in registers for the softmax Jacobian
+            float ps[kM];
+#pragma unroll
+            for (int j = 0; j < kM; ++j) ps[j] = p[j] * inv;
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, ps);
         }
+        fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
-        const float dden = -(sb[row] + sb[kTile + row]) * inv;
-        if (half == 0) sdd[row] = dden;
-        fence_proxy_async_smem();
+        const float ngo = -(sb[row] + sb[kTile + row]);   // -(dO . o) = dden * den
+        if (half == 0) sdd[row] = ngo;
         __syncthreads();
         LB_TRACE(5);
-        // ---- dphi = dnum S^T (three hi/lo passes), dS += phi^T dnum (two passes) ----
+        // ---- dphi * den = dO S^T (S_hi, S_lo), dS += (phi / den)^T dO ----
         if (tid == 0) {
             tcgen05_fence_after();
-            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = dnum (K-major over c), B = S image [c][f] (rows = K)
-            constexpr uint32_t idesc_ds = make_idesc_bf16(kD, kD, 1, 1);        // A = phi^T, B = dnum, both read MN-major
+            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = dO (K-major over c), B = S image [c][f] (rows = K)
+            constexpr uint32_t idesc_ds = make_idesc_bf16(kD, kD, 1, 1);        // A = (phi / den)^T, B = dO, both read MN-major
 #pragma unroll
-            for (int pass = 0; pass < 3; ++pass) {
-                const uint32_t at = sb0 + (pass == 1 ? L::kL : L::kG), st = sb0 + (pass == 2 ? L::kSlo : L::kShi);
+            for (int pass = 0; pass < 2; ++pass) {
+                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k)
-                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(at, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
+                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kG, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
                                 (pass | k) != 0);
             }
 #pragma unroll
-            for (int pass = 0; pass < 2; ++pass)
-#pragma unroll
-                for (int k = 0; k < kTile / 16; ++k)
-                    mma_bf16_ss(t_ds, desc_at(mn_tile, sb0 + L::kP + k * 2048), desc_at(mn_tile, sb0 + (pass == 0 ? L::kG : L::kL) + k * 2048),
-                                idesc_ds, (first && pass == 0 && k == 0) ? 0u : 1u);
+            for (int k = 0; k < kTile / 16; ++k)
+                mma_bf16_ss(t_ds, desc_at(mn_tile, sb0 + L::kP + k * 2048), desc_at(mn_tile, sb0 + L::kG + k * 2048), idesc_ds,
+                            (first && k == 0) ? 0u : 1u);
             mma_commit(c.bar(BW_MMA));
         }
         {
-            // dz += phi^T dden on the CUDA cores while the tensor core works: thread = (16-byte chunk of 8 features,
-            // group of 8 tokens)
+            // dz += phi^T dden = (phi / den)^T (dden den) on the CUDA cores while the tensor core works: thread =
+            // (16-byte chunk of 8 features, group of 8 tokens)
             const int fc = tid & 15, t0 = (tid >> 4) * 8;
             const uint8_t* blk = c.smem + L::kP + (fc >> 3) * kHalfTileBytes;
 #pragma unroll
@@ -456,7 +454,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             float x[kM];
             load64(t_work + lane_base + half * kM, x);
 #pragma unroll
-            for (int j = 0; j < kM; ++j) x[j] = fmaf(dden, vec[half * kM + j], x[j]);
+            for (int j = 0; j < kM; ++j) x[j] = inv * fmaf(ngo, vec[half * kM + j], x[j]);   // dphi = (dO S^T - (dO . o) z) / den
             du_exchange(half, row, p, x, c.smem + L::kL, c.smem + L::kG);
         }
         fence_proxy_async_smem();
