@@ -266,11 +266,20 @@ def main():
     dom = max(kernels, key=lambda kt: kt["ms"])
     if softs is not None:
         dom["bytes"] += 1.0 * B * H * n * d * e   # the softmax branch's output is read once more
-    achieved = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9
+    # Average launch duration of the dominant kernel.  When a step is ONE launch, that is the timed region itself (CUDA
+    # events around it) divided by its launches: no event sits between launches and the clocks are those of the timed
+    # region.  With several kernels per step it comes from the second pass, which has events around every launch.
+    if launches_per_step == 1:
+        kernel_ms = ms_step
+        timing = "timed region (CUDA events around it) / launches in it; the step is this one kernel"
+    else:
+        kernel_ms = dom["ms"]
+        timing = "mean over a second pass of the timed steps with CUDA events around each launch"
+    achieved = dom["bytes"] / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom["name"], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
-                "kernel_ms": dom["ms"], "algorithmic_bytes_per_launch": dom["bytes"],
-                "timing": "mean over a second pass of the timed steps with CUDA events around each launch",
+                "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": dom["bytes"],
+                "timing": timing,
                 "kernels": kernels,
                 "whole_step": {"achieved": alg_total / (ms_step * 1e-3) / 1e9,
                                "frac": alg_total / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
