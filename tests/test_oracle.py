@@ -403,3 +403,26 @@ def test_relu_closed_forms():
     rows = np.array([3, 17, 39])
     np.testing.assert_array_equal(oracle.ref_relu_linear(q, k, v, rows=rows), base[:, :, rows])
     np.testing.assert_allclose(oracle.ref_relu_quadratic(q, k, v, rows=rows), base[:, :, rows], rtol=1e-10, atol=1e-12)
+
+
+def test_backward_closed_forms():
+    """Cases where the gradients are known without any computation.
+    d = 2: one logit per half, so phi = [1, 1] whatever q, k, W are: o_i is the mean of V, dq = dk = dW = 0 and every
+    dv_j is the mean of dO over the queries.  n = 1: o_1 = v_1, so dv = dO and the rest vanishes."""
+    rng = np.random.default_rng(95)
+    B, H, n, d = 2, 2, 6, 2
+    q, k, v = (rng.standard_normal((B, H, n, d)).astype(np.float32) for _ in range(3))
+    Wq, Wk = (rng.standard_normal((H, d, 1)).astype(np.float32) for _ in range(2))
+    g = rng.standard_normal((B, H, n, d)).astype(np.float32)
+    dq, dk, dv, dWq, dWk = oracle.ref_backward(q, k, v, Wq, Wk, g)
+    for z in (dq, dk, dWq, dWk):
+        assert np.abs(z).max() <= 1e-15
+    np.testing.assert_allclose(dv, np.broadcast_to(g.astype(np.float64).mean(2, keepdims=True), g.shape), rtol=1e-13, atol=1e-15)
+    B, H, n, d = 1, 3, 1, 8
+    q, k, v = (rng.standard_normal((B, H, n, d)).astype(np.float32) for _ in range(3))
+    Wq, Wk = (rng.standard_normal((H, d, d // 2)).astype(np.float32) for _ in range(2))
+    g = rng.standard_normal((B, H, n, d)).astype(np.float32)
+    dq, dk, dv, dWq, dWk = oracle.ref_backward(q, k, v, Wq, Wk, g)
+    for z in (dq, dk, dWq, dWk):
+        assert np.abs(z).max() <= 1e-12
+    np.testing.assert_allclose(dv, g.astype(np.float64), rtol=1e-13, atol=1e-15)
