@@ -117,13 +117,18 @@ linattn_status linattn_forward_mixed(linattn_ctx* ctx, const void* q, const void
 /*
  * Gradients of linattn_forward: what the training objective (Eq. 14) back-propagates through a layer that uses
  * Eq. 5 with the feature map of Eq. 6.  Given dout = dL/d(out), writes dL/dq, dL/dk, dL/dv and the gradients of
- * the two feature-map weight matrices.  S and z are recomputed from k, v (no forward needs to precede the call).
+ * the two feature-map weight matrices.  S and z are recomputed from k, v (no forward needs to precede the call;
+ * see LINATTN_OPT_REUSE_STATE for taking them over from the forward).
  *   q, k, v, dout : device, as q, k, v of linattn_forward (same layout option), read-only
  *   dq, dk, dv    : device, same shape, type and layout; written in full; must not overlap any input or each other
  *   dWq, dWk      : device, fp32, 16-byte aligned, written in full: [H][d][d/2] when per_head != 0 (each head's
  *                   gradient summed over the batch), [d][d/2] when per_head == 0 (one shared matrix: summed over
  *                   batch and heads).  The weights differentiated are the ones given to set_feature_map.
- * Arithmetic is fp32 on the CUDA cores (the stored q, k, v, dout are the only rounded quantities); dq, dk, dv are
+ * Two sets of kernels, chosen like the forward's (LINATTN_OPT_PATH): for bf16 activations with d = 128 and bf16
+ * feature-map weights the products run on the tensor cores (bf16 operands, fp32 accumulation; S and dS enter as
+ * bf16 hi + lo pairs and dO itself, exact in bf16, is the operand where dO / den is needed, so that gradients stay
+ * accurate when V has a large mean; relative L2 error about 3e-3 per gradient); everything else, or path 1, runs in
+ * fp32 on the CUDA cores (the stored q, k, v, dout are then the only rounded quantities).  dq, dk, dv are
  * rounded once to `dtype`.  All sums have a fixed order: the same inputs give bit-identical gradients.  The first
  * call allocates the backward workspace (it synchronises the device once); later calls allocate nothing.  After
  * the call the context holds the S, z of these k, v (linattn_read_state returns them).
