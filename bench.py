@@ -224,7 +224,8 @@ def main():
         else:
             ctxs[j].forward_mixed(sets[j]["q"], sets[j]["k"], sets[j]["v"], softs[j], args.mixed, out=outs[j], stream=stream)
 
-    for i in range(args.warmup):
+    # the backward allocates its workspace on a context's first call: every context gets one call before the warm-up
+    for i in range(max(args.warmup, rotate if douts is not None else 0)):
         step(i)
     ctxs[0].check()
     launches_per_step = ctxs[0].last_launch_count()
