@@ -158,31 +158,39 @@ __device__ __forceinline__ float softmax_half_keep(float (&u)[kM], uint8_t* blk,
     m = kNeg ? fminf(m, u[kM - 1]) : fmaxf(m, u[kM - 1]);
     // exp(u - max) = 2^(u*log2e - max*log2e);   exp(-u - max(-u)) = 2^(min*log2e - u*log2e)
     const float sL = kNeg ? -kLog2e : kLog2e, off = kNeg ? m * kLog2e : -m * kLog2e;
-    float s0 = 0.f, s1 = 0.f;
+    // two lanes of arithmetic per instruction (packed fp32 pairs), as in the forward
+    const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
+    f32x2 sum2 = pack2(0.f, 0.f);
 #pragma unroll
     for (int j = 0; j < kM; j += 2) {
-        u[j] = ex2_approx(fmaf(u[j], sL, off));
-        u[j + 1] = ex2_approx(fmaf(u[j + 1], sL, off));
-        s0 += u[j];
-        s1 += u[j + 1];
+        float x0, x1;
+        unpack2(fma2(pack2(u[j], u[j + 1]), scale, offset), x0, x1);
+        u[j] = ex2_approx(x0);
+        u[j + 1] = ex2_approx(x1);
+        sum2 = add2(sum2, pack2(u[j], u[j + 1]));
     }
+    float s0, s1;
+    unpack2(sum2, s0, s1);
     const float inv = __fdividef(1.f, s0 + s1);
-    float d0 = 0.f, d1 = 0.f;
+    const f32x2 inv2 = pack2(inv, inv);
+    f32x2 dot2 = pack2(0.f, 0.f);
+    const float2* vec2 = reinterpret_cast<const float2*>(vec);
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch) {
         uint32_t w[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const int j = 8 * ch + 2 * q;
-            u[j] *= inv;
-            u[j + 1] *= inv;
+            unpack2(mul2(pack2(u[j], u[j + 1]), inv2), u[j], u[j + 1]);
             w[q] = pack_bf16(u[j], u[j + 1]);
-            d0 = fmaf(__uint_as_float(w[q] << 16), vec[j], d0);            // the rounded values, as the tensor core sees them
-            d1 = fmaf(__uint_as_float(w[q] & 0xffff0000u), vec[j + 1], d1);
+            const float2 zv = vec2[j >> 1];
+            // the rounded values, as the tensor core sees them
+            dot2 = fma2(pack2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xffff0000u)), pack2(zv.x, zv.y), dot2);
         }
         *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    return d0 + d1;
+    unpack2(dot2, s0, s1);
+    return s0 + s1;
 }
 
 __device__ __forceinline__ void load64(uint32_t taddr, float (&x)[kM])
@@ -220,11 +228,15 @@ __device__ __forceinline__ float4* scratch_chunk(uint8_t* scratch, int row, int 
 __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint8_t* scratch,
                                             uint8_t* du_tile)
 {
-    float dot = 0.f;
+    f32x2 dot2 = pack2(0.f, 0.f);
 #pragma unroll
-    for (int j = 0; j < kM; ++j) dot = fmaf(p[j], dphi[j], dot);
+    for (int j = 0; j < kM; j += 2) dot2 = fma2(pack2(p[j], p[j + 1]), pack2(dphi[j], dphi[j + 1]), dot2);
+    float d0, d1;
+    unpack2(dot2, d0, d1);
+    const f32x2 ndot = pack2(-(d0 + d1), -(d0 + d1));
 #pragma unroll
-    for (int j = 0; j < kM; ++j) dphi[j] = p[j] * (dphi[j] - dot);
+    for (int j = 0; j < kM; j += 2)
+        unpack2(mul2(pack2(p[j], p[j + 1]), add2(pack2(dphi[j], dphi[j + 1]), ndot)), dphi[j], dphi[j + 1]);
     if (half == 1) {
 #pragma unroll
         for (int ch = 0; ch < 16; ++ch)
@@ -385,23 +397,24 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             load64(t_work + lane_base + half * kM, x);
             inv = 1.f / (sa[row] + sa[kTile + row]);
             const uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
-            float g0s = 0.f, g1s = 0.f;
+            f32x2 gs2 = pack2(0.f, 0.f);
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
                 const uint4 gv = *reinterpret_cast<const uint4*>(gblk + sw_chunk(row, ch));
                 const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    g0s = fmaf(__uint_as_float(gw[q] << 16), x[8 * ch + 2 * q], g0s);
-                    g1s = fmaf(__uint_as_float(gw[q] & 0xffff0000u), x[8 * ch + 2 * q + 1], g1s);
-                }
+                for (int q = 0; q < 4; ++q)
+                    gs2 = fma2(pack2(__uint_as_float(gw[q] << 16), __uint_as_float(gw[q] & 0xffff0000u)),
+                               pack2(x[8 * ch + 2 * q], x[8 * ch + 2 * q + 1]), gs2);
             }
+            float g0s, g1s;
+            unpack2(gs2, g0s, g1s);
             sb[half * kTile + row] = (g0s + g1s) * inv;   // this half's part of dO . o
             // phi / den over phi (the numerator MMA is done with it); p itself stays in registers for the softmax Jacobian
-            float ps[kM];
+            const f32x2 inv2 = pack2(inv, inv);
 #pragma unroll
-            for (int j = 0; j < kM; ++j) ps[j] = p[j] * inv;
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, ps);
+            for (int j = 0; j < kM; j += 2) unpack2(mul2(pack2(p[j], p[j + 1]), inv2), x[j], x[j + 1]);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
         }
         fence_proxy_async_smem();
         tcgen05_fence_before();
@@ -454,7 +467,10 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             float x[kM];
             load64(t_work + lane_base + half * kM, x);
 #pragma unroll
-            for (int j = 0; j < kM; ++j) x[j] = inv * fmaf(ngo, vec[half * kM + j], x[j]);   // dphi = (dO S^T - (dO . o) z) / den
+            for (int j = 0; j < kM; j += 2) {   // dphi = (dO S^T - (dO . o) z) / den
+                const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
+                unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
+            }
             du_exchange(half, row, p, x, c.smem + L::kL, c.smem + L::kG);
         }
         fence_proxy_async_smem();
