@@ -308,15 +308,21 @@ __device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_sme
 // Shared-memory layout, barriers and per-CTA state common to all three kernels
 // ======================================================================================================
 
-constexpr int kKStages = 3;   // key side: stages of (K tile, V tile)
+// Key side: K and V tiles have rings of their own.  A K slot is held from the issue of its load until the accumulation
+// MMA has consumed the phi written over it (load latency + logits MMA + feature map + MMA); a V tile is needed only
+// by that last MMA, so its load is issued one tile later and its slot lives about half as long: four K slots and
+// two V slots keep more loads in flight than three (K, V) pairs of the same 192 KB.
+constexpr int kKSlots = 4;
+constexpr int kVSlots = 2;
+constexpr int kVLag = 1;      // the load of V tile i is issued together with that of K tile i + kVLag
 constexpr int kQStages = 5;   // query side: stages of one Q tile (reused for phi(q) and then the output tile)
 constexpr int kThreads = 512; // 16 warps
 constexpr int kQPrefetchL2 = 3;   // fused kernel: Q tiles pulled into L2 while the CTA waits for S (measured: 2-3 best, 6+ slows the combine)
 
 struct Smem {
     // key side
-    static constexpr uint32_t kKStage = 2 * kTileBytes;                   // K (later phi) + V
-    static constexpr uint32_t kKW = kKStages * kKStage;                   // 2 x W_k^T
+    static constexpr uint32_t kKV = kKSlots * kTileBytes;                 // K slots (each later holds phi), then the V slots
+    static constexpr uint32_t kKW = (kKSlots + kVSlots) * kTileBytes;     // 2 x W_k^T
     static constexpr uint32_t kOnes = kKW + 2 * kWBytes;                  // 1 KB of bf16 ones
     static constexpr uint32_t kKEnd = kOnes + 1024;
     // query side (overlays the key-side region)
@@ -327,18 +333,20 @@ struct Smem {
     static constexpr uint32_t kQW = kQS + 2 * kSZBlock;                   // W_q^T (16 KB)
     static constexpr uint32_t kQEnd = kQW + kWBytes;
     static constexpr uint32_t kBars = kKEnd > kQEnd ? kKEnd : kQEnd;      // mbarriers, TMEM slot, abort word
-    static constexpr uint32_t kTotal = kBars + 512 + 1024;                // + alignment slack
+    static constexpr uint32_t kTotal = kBars + 640 + 1024;                // + alignment slack
 };
 
 // mbarrier indices
 enum : int {
     // key side
-    K_FULL = 0, K_EMPTY = 3, K_UFULL = 6, K_UEMPTY = 8, K_PHIFULL = 10, K_WFULL = 13, K_WFREE = 15, K_ACCFULL = 17, K_ACCFREE = 19,
+    K_FULL = 0, K_EMPTY = 4, K_PHIFULL = 8, K_VFULL = 12, K_VEMPTY = 14, K_UFULL = 16, K_UEMPTY = 18, K_WFULL = 20, K_WFREE = 22,
+    K_ACCFULL = 24, K_ACCFREE = 26,
     // query side
-    Q_FULL = 21, Q_EMPTY = 26, Q_PHIFULL = 31, Q_OFULL = 36, Q_UFULL = 41, Q_UEMPTY = 43, Q_DFULL = 45, Q_DEMPTY = 47,
-    Q_SEGFULL = 49, Q_SEGFREE = 50, Q_SREADY = 51, Q_WFULL = 52, Q_AFULL = 53,
-    NBARS = 58
+    Q_FULL = 28, Q_EMPTY = 33, Q_PHIFULL = 38, Q_OFULL = 43, Q_UFULL = 48, Q_UEMPTY = 50, Q_DFULL = 52, Q_DEMPTY = 54,
+    Q_SEGFULL = 56, Q_SEGFREE = 57, Q_SREADY = 58, Q_WFULL = 59, Q_AFULL = 60,
+    NBARS = 65
 };
+static_assert(kKSlots <= K_EMPTY - K_FULL && kVSlots <= K_VEMPTY - K_VFULL, "one mbarrier per ring slot: widen the enum before growing a ring");
 
 struct Cta {
     uint8_t* smem;
@@ -384,7 +392,8 @@ __device__ __forceinline__ Cta cta_setup(uint8_t* smem_raw, const Args& a, bool 
     if (threadIdx.x == 0) {
         *abort_word = 0u;
         if (init_k) {
-            for (int i = 0; i < kKStages; ++i) { mbar_init(c.bar(K_FULL + i), 1); mbar_init(c.bar(K_EMPTY + i), 1); mbar_init(c.bar(K_PHIFULL + i), 8); }
+            for (int i = 0; i < kKSlots; ++i) { mbar_init(c.bar(K_FULL + i), 1); mbar_init(c.bar(K_EMPTY + i), 1); mbar_init(c.bar(K_PHIFULL + i), 8); }
+            for (int i = 0; i < kVSlots; ++i) { mbar_init(c.bar(K_VFULL + i), 1); mbar_init(c.bar(K_VEMPTY + i), 1); }
             for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_UFULL + i), 1); mbar_init(c.bar(K_UEMPTY + i), 8); mbar_init(c.bar(K_WFULL + i), 1); mbar_init(c.bar(K_WFREE + i), 1); }
             for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_ACCFULL + i), 1); mbar_init(c.bar(K_ACCFREE + i), 4); }
         }
@@ -484,12 +493,27 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             tma_prefetch_desc(tmV);
             tma_prefetch_desc(tmW);
         }
-        Ring<kKStages> r;
-        int issued = 0;
-        for (; !w.done(); w.next(), r.next()) {
+        Ring<kKSlots> r;
+        Ring<kVSlots> vr;
+        TileWalk wv = w;                 // walks the V tiles, kVLag tiles behind the K tiles
+        int issued = 0, issued_v = 0;    // K and V loads issued so far
+        bool ok = true;
+        auto issue_v = [&]() {
+            if (issued_v >= kVSlots && !warp_wait(c.bar(K_VEMPTY + vr.s), vr.ph ^ 1u, c.wc, kErrProducer)) { ok = false; return; }
+            if (lane == 0) {
+                mbar_arrive_expect_tx(c.bar(K_VFULL + vr.s), kTileBytes);
+                const uint32_t vdst = sbase + Smem::kKV + vr.s * kTileBytes;
+                act_load<kLayout>(vdst, tmV, c.bar(K_VFULL + vr.s), 0, wv.lt * kTile, wv.g, a.H);
+                act_load<kLayout>(vdst + kHalfTileBytes, tmV, c.bar(K_VFULL + vr.s), 64, wv.lt * kTile, wv.g, a.H);
+            }
+            ++issued_v;
+            wv.next();
+            vr.next();
+        };
+        for (; !w.done() && ok; w.next(), r.next()) {
             if (kPhi == 0 && w.first()) {
                 const int wb = w.seg & 1;
-                if (w.seg >= 2 && !warp_wait(c.bar(K_WFREE + wb), ((w.seg >> 1) - 1) & 1, c.wc, kErrProducer)) break;
+                if (w.seg >= 2 && !warp_wait(c.bar(K_WFREE + wb), ((w.seg >> 1) - 1) & 1, c.wc, kErrProducer)) { ok = false; break; }
                 if (lane == 0) {
                     mbar_arrive_expect_tx(c.bar(K_WFULL + wb), kWBytes);
                     const uint32_t wdst = sbase + Smem::kKW + wb * kWBytes;
@@ -497,26 +521,28 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
                     tma_load_3d(wdst + kWBytes / 2, tmW, c.bar(K_WFULL + wb), 64, 0, w.g % a.H);
                 }
             }
-            if (w.i >= kKStages && !warp_wait(c.bar(K_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) break;
+            if (w.i >= kKSlots && !warp_wait(c.bar(K_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) { ok = false; break; }
             LA_TRACE(0, w.i, 0);
             if (lane == 0) {
-                mbar_arrive_expect_tx(c.bar(K_FULL + r.s), 2 * kTileBytes);
-                const uint32_t kdst = sbase + r.s * Smem::kKStage, vdst = kdst + kTileBytes;
+                mbar_arrive_expect_tx(c.bar(K_FULL + r.s), kTileBytes);
+                const uint32_t kdst = sbase + r.s * kTileBytes;
                 act_load<kLayout>(kdst, tmK, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
                 act_load<kLayout>(kdst + kHalfTileBytes, tmK, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
-                act_load<kLayout>(vdst, tmV, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
-                act_load<kLayout>(vdst + kHalfTileBytes, tmV, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
             }
             issued = w.i + 1;
+            if (w.i >= kVLag) issue_v();
         }
-        if (issued < w.count) {
+        while (ok && issued_v < issued) issue_v();
+        if (!ok) {
             // unwinding after a time-out: let the copies already in flight land before the CTA moves on
-            for (int i = (issued > kKStages ? issued - kKStages : 0); i < issued; ++i)
-                mbar_wait(c.bar(K_FULL + i % kKStages), (uint32_t)(i / kKStages) & 1u, kWaitLimitNs);
+            for (int i = (issued > kKSlots ? issued - kKSlots : 0); i < issued; ++i)
+                mbar_wait(c.bar(K_FULL + i % kKSlots), (uint32_t)(i / kKSlots) & 1u, kWaitLimitNs);
+            for (int i = (issued_v > kVSlots ? issued_v - kVSlots : 0); i < issued_v; ++i)
+                mbar_wait(c.bar(K_VFULL + i % kVSlots), (uint32_t)(i / kVSlots) & 1u, kWaitLimitNs);
         }
     } else if (warp == 9) {
         // ---------------- logits MMA issuer: U = K W_k ----------------
-        Ring<kKStages> r;
+        Ring<kKSlots> r;
         Ring<2> ur;
         for (; kPhi == 0 && !w.done(); w.next(), r.next(), ur.next()) {
             const int wb = w.seg & 1;
@@ -526,7 +552,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             if (w.i >= 2 && !warp_wait(c.bar(K_UEMPTY + ur.s), ur.ph ^ 1u, c.wc, kErrMmaU)) break;
             tcgen05_fence_after();
             if (elect_one()) {
-                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * Smem::kKStage, sbase + Smem::kKW + wb * kWBytes);
+                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + Smem::kKW + wb * kWBytes);
                 mma_commit(c.bar(K_UFULL + ur.s));
                 if (w.last()) mma_commit(c.bar(K_WFREE + wb));
             }
@@ -539,16 +565,18 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
         constexpr uint32_t idesc_z = make_idesc_bf16(kD, 16, 1, 0);   // B = ones (K-major, no swizzle)
         const uint64_t ones_desc = make_desc_noswizzle(sbase + Smem::kOnes, 128, 256);
         const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
-        Ring<kKStages> r;
-        for (; !w.done(); w.next(), r.next()) {
+        Ring<kKSlots> r;
+        Ring<kVSlots> vr;
+        for (; !w.done(); w.next(), r.next(), vr.next()) {
             if (!warp_wait(c.bar(K_PHIFULL + r.s), r.ph, c.wc, kErrMmaPhi)) break;
+            if (!warp_wait(c.bar(K_VFULL + vr.s), vr.ph, c.wc, kErrMmaLoad)) break;
             LA_TRACE(1, w.i, 2);
             const bool first = w.first();
             const int b = w.seg & 1;
             if (first && w.seg >= 2 && !warp_wait(c.bar(K_ACCFREE + b), (uint32_t)((w.seg >> 1) - 1) & 1u, c.wc, kErrMmaAcc)) break;
             tcgen05_fence_after();
             if (elect_one()) {
-                const uint32_t phi = sbase + r.s * Smem::kKStage, vt = phi + kTileBytes;
+                const uint32_t phi = sbase + r.s * kTileBytes, vt = sbase + Smem::kKV + vr.s * kTileBytes;
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k) {
                     const uint64_t da = desc_at(mnmajor, phi + k * 2048);
@@ -558,6 +586,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
                     mma_bf16_ss(tmem_z(b), da, ones_desc, idesc_z, acc);
                 }
                 mma_commit(c.bar(K_EMPTY + r.s));
+                mma_commit(c.bar(K_VEMPTY + vr.s));
                 if (w.last()) mma_commit(c.bar(K_ACCFULL + b));
             }
             __syncwarp();
@@ -565,10 +594,10 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
         }
     } else if (warp < 8 && kPhi == 1) {
         // ---------------- ReLU kernel function (warps 0-7) ----------------
-        Ring<kKStages> r;
+        Ring<kKSlots> r;
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(K_FULL + r.s), r.ph, c.wc, kErrSoftmaxU)) break;
-            relu_tile_in_place(c.smem + r.s * Smem::kKStage, threadIdx.x);
+            relu_tile_in_place(c.smem + r.s * kTileBytes, threadIdx.x);
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(c.bar(K_PHIFULL + r.s));
@@ -578,7 +607,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
         const int half = warp >> 2;                       // 0: softmax(+U), 1: softmax(-U)
         const int row = (warp & 3) * 32 + lane;           // token within the tile == TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        Ring<kKStages> r;
+        Ring<kKSlots> r;
         Ring<2> ur;
         for (; !w.done(); w.next(), r.next(), ur.next()) {
             if (!warp_wait(c.bar(K_UFULL + ur.s), ur.ph, c.wc, kErrSoftmaxU)) break;
@@ -591,7 +620,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             if (lane == 0) mbar_arrive(c.bar(K_UEMPTY + ur.s));
             if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 1);
             const float keep = (w.lt * kTile + row < a.n) ? 1.f : 0.f;
-            uint8_t* dst = c.smem + r.s * Smem::kKStage + half * kHalfTileBytes + row * 128;
+            uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
             if (half == 0) softmax_half_to_smem<false>(u, keep, dst, row);
             else softmax_half_to_smem<true>(u, keep, dst, row);
             fence_proxy_async_smem();
