@@ -766,6 +766,10 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         };
         for (; !w.done() && ok; w.next(), r.next()) {
             if (w.first()) {
+                // A first piece of the run shorter than the ring ends before its S, z were asked for (that load is put
+                // off until the ring is full): they are owed now, or the MMAs that free the single S buffer never run.
+                if (state_g >= 0) load_state();
+                if (!ok) break;
                 if (w.seg >= 1 && !warp_wait(c.bar(Q_SEGFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrSeg)) break;
                 if (kPhi == 0 && lane == 0) {
                     mbar_arrive_expect_tx(c.bar(Q_WFULL), kWBytes);

@@ -269,3 +269,26 @@ def test_forward_argument_errors():
         ctx.check()
     finally:
         ctx.destroy()
+
+
+@pytest.mark.parametrize("H,n", [(3, 9472), (3, 10240), (5, 9600), (8, 4736), (12, 2560)])
+def test_run_whose_first_piece_is_shorter_than_the_query_ring(H, n):
+    """Shapes for which some CTA of the fused kernel starts one to four tiles before a head boundary and goes on into
+    the next head: the first head's S, z must be fetched before the second head's are waited for."""
+    Tn = (n + 127) // 128
+    T, P = H * Tn, 148
+    assert T >= P
+    short = [c for c in range(P) if (c * T // P) % Tn != 0 and Tn - (c * T // P) % Tn < 5 and (c + 1) * T // P > c * T // P + Tn - (c * T // P) % Tn]
+    assert short, "the shape no longer exercises the case (148 SMs assumed)"
+    x = small_inputs(1, H, n, 128, torch.bfloat16, seed=40 + H)
+    ctx = linattn.LinAttn(H, 128, max_B=1, max_n=n)
+    try:
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        out = ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda())
+        ctx.check()
+        assert ctx.last_launch_count() == 1
+        rows = np.unique(np.concatenate([np.random.default_rng(H).choice(n, 400, replace=False), [0, n - 1]]))
+        want = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], rows=rows)
+        assert_parity(out.cpu()[:, :, torch.from_numpy(rows)].double().numpy(), want, f"H={H} n={n}")
+    finally:
+        ctx.destroy()
