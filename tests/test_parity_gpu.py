@@ -271,12 +271,22 @@ def test_forward_argument_errors():
         ctx.destroy()
 
 
-@pytest.mark.parametrize("H,n", [(3, 9472), (3, 10240), (5, 9600), (8, 4736), (12, 2560)])
+def _fused_ctas(G, T, sms=148):
+    """CTAs of the fused kernel (mirrors the library's rule: one per SM, or the same number per (b,h) pair when that
+    uses at least 95 % of the SMs)."""
+    if T <= sms:
+        return T
+    per_pair = sms // G
+    return G * per_pair if per_pair >= 1 and G * per_pair * 100 >= 95 * sms else sms
+
+
+@pytest.mark.parametrize("H,n", [(10, 2432), (10, 2688), (20, 1280), (20, 1536), (40, 768)])
 def test_run_whose_first_piece_is_shorter_than_the_query_ring(H, n):
     """Shapes for which some CTA of the fused kernel starts one to four tiles before a head boundary and goes on into
     the next head: the first head's S, z must be fetched before the second head's are waited for."""
     Tn = (n + 127) // 128
-    T, P = H * Tn, 148
+    T = H * Tn
+    P = _fused_ctas(H, T)
     assert T >= P
     short = [c for c in range(P) if (c * T // P) % Tn != 0 and Tn - (c * T // P) % Tn < 5 and (c + 1) * T // P > c * T // P + Tn - (c * T // P) % Tn]
     assert short, "the shape no longer exercises the case (148 SMs assumed)"
@@ -287,8 +297,7 @@ def test_run_whose_first_piece_is_shorter_than_the_query_ring(H, n):
         out = ctx.forward(x["q"].cuda(), x["k"].cuda(), x["v"].cuda())
         ctx.check()
         assert ctx.last_launch_count() == 1
-        rows = np.unique(np.concatenate([np.random.default_rng(H).choice(n, 400, replace=False), [0, n - 1]]))
-        want = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], rows=rows)
-        assert_parity(out.cpu()[:, :, torch.from_numpy(rows)].double().numpy(), want, f"H={H} n={n}")
+        want = oracle.ref_linear(x["q"], x["k"], x["v"], x["Wq"], x["Wk"])
+        assert_parity(out.cpu().double().numpy(), want, f"H={H} n={n}")
     finally:
         ctx.destroy()
