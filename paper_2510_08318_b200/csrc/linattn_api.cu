@@ -429,7 +429,7 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     const long long G = (long long)B * c->H;
     const long long Tn = ((long long)n + kTile - 1) / kTile;
     const long long T = G * Tn;
-    const long long P = choose_ctas(c, G, T);
+    const long long P = c->num_sms < T ? c->num_sms : T;   // these kernels are bound by per-tile latency, not bandwidth: every SM counts
     if (P + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
     // forward state (S as [c][f], z) and the hi image of S: left by the forward that just ran on these k, v (if the
     // caller allows it), else recomputed; q and out are not touched by the first two kernels of the forward
