@@ -301,3 +301,38 @@ def test_run_whose_first_piece_is_shorter_than_the_query_ring(H, n):
         assert_parity(out.cpu().double().numpy(), want, f"H={H} n={n}")
     finally:
         ctx.destroy()
+
+
+def test_fused_kernel_equals_the_three_launch_form_over_many_tile_splits():
+    """The fused kernel and the three-launch form split the tiles in the same way and sum the partials in the same
+    order, so their outputs must agree bit for bit.  Swept over head counts and lengths that give every kind of run:
+    one tile per CTA, runs inside a head, runs that cross one or several head boundaries at any offset, ragged tails."""
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev).manual_seed(123)
+    checked = 0
+    for G in (1, 2, 3, 5, 7, 10, 13, 20, 37, 40, 41, 50, 75, 149):
+        for Tn in (1, 2, 3, 4, 5, 6, 7, 9, 13, 21, 33):
+            if G * Tn > 3000:
+                continue
+            n = Tn * 128 - (17 if Tn % 2 else 0)
+            q, k, v = (torch.randn(1, G, n, 128, generator=g, device=dev).mul_(1 / math.sqrt(128)).bfloat16() for _ in range(3))
+            Wq, Wk = (torch.randn(G, 128, 64, generator=g, device=dev).bfloat16() for _ in range(2))
+            ctx = linattn.LinAttn(G, 128, max_B=1, max_n=n)
+            try:
+                ctx.set_feature_map(Wq, Wk)
+                fused = ctx.forward(q, k, v)
+                fused_mixed = ctx.forward_mixed(q, k, v, v, 0.25)
+                ctx.check()
+                assert ctx.last_launch_count() == 1
+                ctx.set_option(linattn.OPT_FUSE, 0)
+                unfused = ctx.forward(q, k, v)
+                unfused_mixed = ctx.forward_mixed(q, k, v, v, 0.25)
+                ctx.check()
+                assert ctx.last_launch_count() == 3
+                assert torch.isfinite(fused.float()).all(), f"G={G} tiles per head={Tn}"
+                assert torch.equal(fused, unfused), f"G={G} tiles per head={Tn}"
+                assert torch.equal(fused_mixed, unfused_mixed), f"mixed attention, G={G} tiles per head={Tn}"
+                checked += 1
+            finally:
+                ctx.destroy()
+    assert checked > 100
