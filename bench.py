@@ -148,7 +148,7 @@ def reference_arm(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl_name(args.config, wl), "B": B, "H": H, "n": n, "d": d, "sample": sample},
+        "config": config_dict(args, wl),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -159,13 +159,69 @@ def wl_name(config, wl):
     return f"config {config}: {wl.name} B={wl.B} H={wl.H} n={wl.n} d={wl.d} {wl.dtype}"
 
 
+def config_dict(args, wl):
+    """The workload as both arms (ours and --impl reference) name it: identical keys and values, so that the two
+    lines can be matched on it."""
+    rotate = wl.layers if wl.layers > 1 else ROTATE
+    return {"workload": wl_name(args.config, wl), "B": wl.B, "H": wl.H, "n": wl.n, "d": wl.d,
+            "layout": "[B][n][H][d]" if getattr(args, "layout", 0) else "[B][H][n][d]",
+            "l2": f"inputs larger than L2 and {rotate} input sets rotated (no set is re-read within {rotate - 1} steps)",
+            "multi_gpu": "replicas only: independent inputs per rank, no collective on the data path"}
+
+
+ALL_VARIANTS = [
+    ("forward, config 2 (the metric's workload)", ["--config", "2"]),
+    ("forward, config 3", ["--config", "3"]),
+    ("forward, config 4", ["--config", "4"]),
+    ("forward, config 5 (30 resident layers)", ["--config", "5"]),
+    ("forward, config 6 (CogVideoX-2B-shaped, d = 64)", ["--config", "6"]),
+    ("forward, config 2, token-major layout [B][n][H][d]", ["--config", "2", "--layout", "1"]),
+    ("mixed attention (Eq. 8), r = 0.5, config 2", ["--config", "2", "--mixed", "0.5"]),
+    ("ReLU kernel function, config 2", ["--config", "2", "--phi", "relu"]),
+    ("backward, config 2", ["--config", "2", "--backward"]),
+]
+
+
+def run_all(args):
+    """Child run of this script per variant (a fresh process each: fresh contexts, nothing resident from the previous
+    one); prints each child's JSON line and writes a markdown table of them."""
+    rows = []
+    for title, extra in ALL_VARIANTS:
+        steps = 300 if "--backward" not in extra else 100
+        cmd = [sys.executable, os.path.abspath(__file__), "--gpus", "1", "--steps", str(steps), "--warmup", "10", "--no-baselines"] + extra
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        line = next((l for l in reversed(res.stdout.splitlines()) if l.startswith("{")), None)
+        if res.returncode != 0 or line is None:
+            rows.append((title, None, (res.stderr or res.stdout)[-300:].replace("\n", " ")))
+            continue
+        print(line, flush=True)
+        rows.append((title, json.loads(line), ""))
+    out = ["# Benchmark table: every workload and variant, one B200", "",
+           f"Written by `python bench.py --all` (each row: `python bench.py --gpus 1 --steps 300 --warmup 10 --no-baselines <variant>`, "
+           f"100 steps for the backward), source digest {source_digest()}.", "",
+           "| variant | step (mean) | median / min | tokens/s | algorithmic GB/s | of measured peak | of nominal 8 TB/s | dominant kernel | SM clock (median), reasons |",
+           "|---|---|---|---|---|---|---|---|---|"]
+    for title, r, err in rows:
+        if r is None:
+            out.append(f"| {title} | failed: {err} | | | | | | | |")
+            continue
+        rf, ws, ck = r["roofline"], r["roofline"]["whole_step"], r.get("clocks") or {}
+        sp = rf["step_spread"]
+        out.append(f"| {title} | {1e3 * r['ms_per_step']:.1f} us | {1e3 * sp['median_ms']:.1f} / {1e3 * sp['min_ms']:.1f} us | {r['value']:.3e} | "
+                   f"{ws['achieved']:.0f} | {ws['frac']:.3f} | {ws['frac_of_nominal_8TBs']:.3f} | {rf['kernel']} ({1e3 * rf['kernel_ms']:.1f} us) | "
+                   f"{ck.get('sm_mhz')} MHz, {','.join(ck.get('reasons') or []) or 'none'} |")
+    os.makedirs(os.path.dirname(args.table_out), exist_ok=True)
+    with open(args.table_out, "w") as f:
+        f.write("\n".join(out) + "\n")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=2, choices=sorted(c_ for c_ in synth.CONFIGS if c_ >= 2))
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-baselines", action="store_true", help="skip the oracle and SDPA context baselines")
@@ -175,9 +231,23 @@ def main():
     ap.add_argument("--phi", default="hedgehog", choices=["hedgehog", "relu"],
                     help="kernel function: the Hedgehog feature map of Eq. 6 (the metric's) or the ReLU of the paper's ablation")
     ap.add_argument("--backward", action="store_true",
-                    help="time linattn_backward (gradients of the operator, CUDA-core kernels) instead of the forward")
+                    help="time linattn_backward (gradients of the operator; the kernels --path selects) instead of the forward")
+    ap.add_argument("--layout", type=int, default=0, choices=[0, 1],
+                    help="memory order of q, k, v, out: 0 = [B][H][n][d] (the metric's), 1 = [B][n][H][d] (LINATTN_OPT_LAYOUT)")
+    ap.add_argument("--source-digest", action="store_true",
+                    help="print the digest of the forward kernels' sources (what profiles/dram_traffic.txt is keyed by) and exit")
+    ap.add_argument("--all", action="store_true",
+                    help="run every workload and variant (configs 2-5 and the CogVideoX-shaped one, mixed attention, ReLU, backward, "
+                         "token-major layout) as child runs, print one JSON line each and write the table to --table-out")
+    ap.add_argument("--table-out", default=os.path.join(ROOT, "profiles", "bench_table.md"))
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.source_digest:
+        print(source_digest())
+        return
+    if args.all:
+        run_all(args)
+        return
     wl = synth.CONFIGS[args.config]
 
     if args.impl == "reference":
@@ -211,6 +281,7 @@ def main():
         c.set_option(linattn.OPT_PATH, args.path)
         c.set_option(linattn.OPT_SPLITS, args.splits)
         c.set_option(linattn.OPT_KERNEL_FUNCTION, linattn.PHI_RELU if args.phi == "relu" else linattn.PHI_HEDGEHOG)
+        c.set_option(linattn.OPT_LAYOUT, args.layout)   # i.i.d. synthetic values: the same storage read in the other order
         c.set_feature_map(s["Wq"], s["Wk"])
         ctxs.append(c)
     stream = torch.cuda.current_stream()
@@ -236,19 +307,41 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ladist.barrier()
     torch.cuda.synchronize()
+    t_region0 = time.time()
     ev0.record(stream)
     for i in range(args.steps):
         step(i)
     ev1.record(stream)
     torch.cuda.synchronize()
+    t_region1 = time.time()
     ladist.barrier()
     ms_total = ladist.max_over_ranks(ev0.elapsed_time(ev1))
-    clocks = sampler.stop() if rank == 0 else None
     for c in ctxs:
         c.check()
     ms_step = ms_total / args.steps
     tokens_per_step = ladist.sum_over_ranks(float(B * n))
     value = tokens_per_step / (ms_step * 1e-3)
+
+    # Second pass over the same steps, for the spread: an event pair around every step (around every block of 50 when
+    # there are more than 400), median and minimum.  The events sit between launches, so these are a little above the
+    # un-instrumented mean; `value` and `roofline.achieved` come from the first region only.
+    block = 1 if args.steps <= 400 else 50
+    nblk = max(1, args.steps // block)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(nblk + 1)]
+    torch.cuda.synchronize()
+    marks[0].record(stream)
+    for bi in range(nblk):
+        for i in range(bi * block, (bi + 1) * block):
+            step(i)
+        marks[bi + 1].record(stream)
+    torch.cuda.synchronize()
+    per_step = sorted(marks[bi].elapsed_time(marks[bi + 1]) / block for bi in range(nblk))
+    spread = {"median_ms": statistics.median(per_step), "min_ms": per_step[0], "max_ms": per_step[-1],
+              "events_around": f"every {'step' if block == 1 else f'{block} steps'}", "samples": nblk}
+    clocks = sampler.stop() if rank == 0 else None
+    if clocks is not None:
+        clocks["window"] = (f"warm-up end to the end of the per-step pass ({time.time() - t_region0:.3f} s, same steps twice); "
+                            f"the timed region itself lasted {t_region1 - t_region0:.4f} s")
 
     # per-kernel durations: a second pass of the same steps with events around every launch
     e = 2 if wl.dtype == "bf16" else 4
@@ -257,7 +350,7 @@ def main():
     alg_total = (7.0 if douts is not None else 4.0 if softs is None else 5.0) * B * H * n * d * e
     for c in ctxs:
         c.set_option(linattn.OPT_PROFILE, 1)
-    for i in range(args.steps):
+    for i in range(min(args.steps, 300)):
         step(i)
     torch.cuda.synchronize()
     kernels = ctxs[0].kernel_times()  # [(name, mean ms, launches, algorithmic bytes per launch)]
@@ -278,9 +371,10 @@ def main():
         timing = "mean over a second pass of the timed steps with CUDA events around each launch"
     achieved = dom["bytes"] / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom["name"], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                "peak_nominal": 8000.0, "frac_of_nominal": achieved / 8000.0, "traffic": None,
                 "kernel_ms": kernel_ms, "algorithmic_bytes_per_launch": dom["bytes"],
-                "timing": timing,
+                "timing": timing, "step_spread": spread,
                 "kernels": kernels,
                 "whole_step": {"achieved": alg_total / (ms_step * 1e-3) / 1e9,
                                "frac": alg_total / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -312,9 +406,7 @@ def main():
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": wl_name(args.config, wl), "B": B, "H": H, "n": n, "d": d, "path": args.path,
-                   "l2": f"inputs larger than L2 and {rotate} input sets rotated (no set is re-read within {rotate - 1} steps)",
-                   "multi_gpu": "replicas only: independent inputs per rank, no collective on the data path"},
+        "config": config_dict(args, wl), "kernel_path": args.path,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
     }
 

@@ -91,7 +91,10 @@ linattn_status linattn_set_feature_map(linattn_ctx* ctx, const void* Wq, const v
  *   stream  : a cudaStream_t of the context's device (NULL = default stream)
  * All accumulation (S, z, numerator, denominator) is fp32.  The call allocates nothing, does not
  * synchronise, and is deterministic: the same inputs give bit-identical outputs.  Calls on one
- * context must be stream-ordered (they share the context's workspace).
+ * context must be stream-ordered (they share the context's workspace).  The call may be recorded
+ * into a CUDA graph (stream capture): while `stream` is capturing, the tensor-core path records
+ * its three-launch form instead of the single cooperative kernel, because that kernel's
+ * grid-barrier targets are computed on the host for each launch and would be stale on replay.
  * Errors: INVALID_ARG, UNSUPPORTED, NO_FEATURE_MAP, WORKSPACE, CUDA (launch failure).
  */
 linattn_status linattn_forward(linattn_ctx* ctx, const void* q, const void* k, const void* v, void* out,
@@ -174,9 +177,12 @@ linattn_status linattn_read_state(linattn_ctx* ctx, float* S_host, float* z_host
  *   Wq, Wk       : device, fp32, 16-byte aligned, [H][d][d/2] (per_head != 0) or [d][d/2]; read, not copied
  *   limits       : B * H <= 16 and d in {64, 128}; any n >= 1.  A larger B * H returns
  *                  LINATTN_ERR_WORKSPACE ("request exceeds the workspace ...") and launches nothing.
- * Runs on the CURRENT device.  The first call on each device looks up the device address of the
- * scratch array and raises the kernels' shared-memory limit; make that first call before any
- * stream capture begins.  All calls on a device share the one scratch array: it keeps the previous
+ *   out          : must not overlap q, k or v (INVALID_ARG)
+ * Runs on the CURRENT device, which must be of compute capability 10.x (else UNSUPPORTED).  The first
+ * call on each device looks up the device address of the scratch array and raises the kernels'
+ * shared-memory limit; make that first call before any stream capture begins, and from ONE host
+ * thread (the set-up results are cached in unsynchronised host variables; later calls may come
+ * from any thread).  All calls on a device share the one scratch array: it keeps the previous
  * call's contents, every element a call reads is first written by that same call (nothing needs
  * clearing), and two calls whose kernels overlap on the GPU (different streams, no ordering) race
  * on it and give wrong results -- keep calls on one device stream-ordered.

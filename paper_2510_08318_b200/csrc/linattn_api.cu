@@ -66,6 +66,7 @@ struct linattn_ctx {
     float* bwd_part_w = nullptr;      // [partial_slots][d*d/2]    per-block sums of dW
     float* bwd_dstate = nullptr;      // [max_B*H][d*d + d]        dS, dz
     __nv_bfloat16* bwd_img[3] = {nullptr, nullptr, nullptr};   // tensor-core backward: lo image of S, hi and lo images of dS
+    bool bwd_ready = false;           // every allocation above succeeded
     // host-call staging and its pipeline: copies in, compute and copies out run on three streams, one (b,h) at a time
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     size_t stage_bytes = 0;
@@ -100,7 +101,10 @@ struct linattn_ctx {
     double prof_ms[kMaxKernels] = {};
     long long prof_cnt[kMaxKernels] = {};
     // bookkeeping
-    bool attr_done[9] = {};   // shared-memory limit raised on this context's device, per kernel family (function attributes are per device)
+    // shared-memory limit raised on this context's device, per kernel family (function attributes are per device)
+    enum AttrSlot { kAttrSimtFwd = 0 /* +0..3: (storage type, head dim) */, kAttrSimtBwd = 4 /* +0..3 */, kAttrTcFwd = 8,
+                    kAttrTcBwd = 9, kAttrSlots = 10 };
+    bool attr_done[kAttrSlots] = {};
     int last_launches = 0;
     int last_B = 0;
     bool state_transposed = false;  // the last forward left S in the workspace as [c][f] (tensor-core kernels) rather than [f][c]
@@ -203,7 +207,7 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
     if (G * splits > c->partial_slots) return LINATTN_ERR_WORKSPACE;
     constexpr int E = D * D + D;
 
-    bool& attr_done = c->attr_done[(sizeof(T) == 2 ? 2 : 0) + (D == 128 ? 1 : 0)];
+    bool& attr_done = c->attr_done[linattn_ctx::kAttrSimtFwd + (sizeof(T) == 2 ? 2 : 0) + (D == 128 ? 1 : 0)];
     if (!attr_done) {
         LA_CUDA(c, cudaFuncSetAttribute(kside_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kside_simt_smem<D>()));
@@ -249,7 +253,7 @@ linattn_status launch_backward_simt(linattn_ctx* c, const void* q, const void* k
     if (G * splits > c->partial_slots || G * blocks > c->partial_slots) return LINATTN_ERR_WORKSPACE;
     constexpr int E = D * D + D, DM = D * (D / 2);
 
-    bool& attr_done = c->attr_done[4 + (sizeof(T) == 2 ? 2 : 0) + (D == 128 ? 1 : 0)];
+    bool& attr_done = c->attr_done[linattn_ctx::kAttrSimtBwd + (sizeof(T) == 2 ? 2 : 0) + (D == 128 ? 1 : 0)];
     if (!attr_done) {
         LA_CUDA(c, cudaFuncSetAttribute(kside_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kside_simt_smem<D>()));
         LA_CUDA(c, cudaFuncSetAttribute(qside_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bwd_smem<D>()));
@@ -343,7 +347,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     const void* k_kside[2][2] = {LA_BY_PHI(kside_tc, 0), LA_BY_PHI(kside_tc, 1)};
 #undef LA_BY_PHI
     const int phi = c->opt_phi;
-    bool& attr_done = c->attr_done[8];
+    bool& attr_done = c->attr_done[linattn_ctx::kAttrTcFwd];
     if (!attr_done) {
         for (int i = 0; i < 2; ++i)
             for (int p = 0; p < 2; ++p) {
@@ -377,15 +381,23 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.trace = c->trace;
 #endif
     prof_begin(c, st);
-    if (c->opt_fuse && c->coop_ok && Pk == Pq && !state_only) {
+    // The fused kernel's grid-barrier targets are computed here, when the launch is enqueued, from a counter that only
+    // grows: a launch recorded into a CUDA graph would carry stale targets when the graph is replayed.  While the stream
+    // is being captured the three-launch form (no barrier, no host-side bookkeeping) is recorded instead.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+        cudaGetLastError();
+        cap = cudaStreamCaptureStatusNone;
+    }
+    if (c->opt_fuse && c->coop_ok && Pk == Pq && !state_only && cap == cudaStreamCaptureStatusNone) {
         // one cooperative launch: key side, grid barrier, combine, grid barrier, query side
         a.bar_target[0] = c->bar_total + (uint32_t)Pq;
         a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
-        c->bar_total += 2u * (uint32_t)Pq;
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
         const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout][phi], dim3((unsigned)Pq), dim3(kThreads),
                                                            params, Smem::kTotal, st);
         if (le == cudaSuccess) {
+            c->bar_total += 2u * (uint32_t)Pq;   // only a launch that was enqueued moves the counter
             prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
             c->last_launches = 1;
             return LINATTN_OK;
@@ -394,7 +406,6 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         // Not all CTAs can be resident at once (part of the GPU is taken, e.g. MIG or MPS limits): nothing was
         // launched; use the three-launch form from now on, which needs no co-residency.
         cudaGetLastError();
-        c->bar_total -= 2u * (uint32_t)Pq;
         c->coop_ok = false;
     }
     {
@@ -466,7 +477,7 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     }
     const void* k_q[2] = {(const void*)qside_bwd_tc<0>, (const void*)qside_bwd_tc<1>};
     const void* k_k[2] = {(const void*)kside_bwd_tc<0>, (const void*)kside_bwd_tc<1>};
-    bool& attr_done = c->attr_done[9];
+    bool& attr_done = c->attr_done[linattn_ctx::kAttrTcBwd];
     if (!attr_done) {
         for (int i = 0; i < 2; ++i) {
             LA_CUDA(c, cudaFuncSetAttribute(k_q[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemQ));
@@ -763,13 +774,28 @@ linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, co
     if (misaligned16(dWq) || misaligned16(dWk) || dWq == dWk) return LINATTN_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
-    if (!c->bwd_dstate) {
-        const size_t E = (size_t)d * d + d;
-        LA_CUDA(c, cudaMalloc(&c->bwd_part_state, sizeof(float) * E * (size_t)c->partial_slots));
-        LA_CUDA(c, cudaMalloc(&c->bwd_part_w, sizeof(float) * (size_t)d * (d / 2) * (size_t)c->partial_slots));
-        LA_CUDA(c, cudaMalloc(&c->bwd_dstate, sizeof(float) * E * (size_t)(c->max_B * c->H)));
+    if (!c->bwd_ready) {
+        // all or nothing: a failed allocation releases what the earlier ones got, so that the next call starts over
+        const size_t E = (size_t)d * d + d, G = (size_t)(c->max_B * c->H);
+        cudaError_t e = cudaMalloc(&c->bwd_part_state, sizeof(float) * E * (size_t)c->partial_slots);
+        if (e == cudaSuccess) e = cudaMalloc(&c->bwd_part_w, sizeof(float) * (size_t)d * (d / 2) * (size_t)c->partial_slots);
+        if (e == cudaSuccess) e = cudaMalloc(&c->bwd_dstate, sizeof(float) * E * G);
         if (d == 128)
-            for (__nv_bfloat16*& p : c->bwd_img) LA_CUDA(c, cudaMalloc(&p, sizeof(__nv_bfloat16) * (size_t)d * d * (size_t)(c->max_B * c->H)));
+            for (__nv_bfloat16*& p : c->bwd_img)
+                if (e == cudaSuccess) e = cudaMalloc(&p, sizeof(__nv_bfloat16) * (size_t)d * d * G);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(c->bwd_part_state);
+            cudaFree(c->bwd_part_w);
+            cudaFree(c->bwd_dstate);
+            c->bwd_part_state = c->bwd_part_w = c->bwd_dstate = nullptr;
+            for (__nv_bfloat16*& p : c->bwd_img) {
+                cudaFree(p);
+                p = nullptr;
+            }
+            return cuda_fail(c, e, "cudaMalloc (backward workspace)");
+        }
+        c->bwd_ready = true;
     }
     c->last_B = B;
     const int ph = per_head ? 1 : 0;

@@ -27,15 +27,28 @@ constexpr size_t kScratchFloats = (size_t)(kNoAllocPartialSlots + kNoAllocMaxGro
 // Every GPU that loads the library holds these ~5.3 MB until the process exits.
 static __device__ __align__(256) float g_noalloc_scratch[kScratchFloats];
 
+// Host-side caches, filled by the first call on each device.  They are plain variables: two host threads that make
+// their FIRST call on a device at the same moment would both run the set-up (each stores the same values), so the
+// documented rule is to make the first call on a device from one thread.
 constexpr int kMaxDevices = 64;
 float* g_scratch_ptr[kMaxDevices] = {};  // device address of g_noalloc_scratch on each device, set up on first use
 bool g_attr_done[kMaxDevices][4] = {};
+int g_cc_major[kMaxDevices] = {};        // compute capability (major) of each device, 0 = not asked yet
 
 // The array's name is only a host-side handle here; kernels need its device address, which the
 // runtime gives per device.  Done once per device, with that device current.
 linattn_status scratch_for_current_device(int dev, float** out)
 {
     if (dev < 0 || dev >= kMaxDevices) return LINATTN_ERR_UNSUPPORTED;
+    if (g_cc_major[dev] == 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return LINATTN_ERR_CUDA;
+        }
+        g_cc_major[dev] = major;
+    }
+    if (g_cc_major[dev] != 10) return LINATTN_ERR_UNSUPPORTED;   // the library is built for sm_100a only
     if (!g_scratch_ptr[dev]) {
         float* p = nullptr;
         if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
@@ -100,6 +113,13 @@ extern "C" linattn_status linattn_forward_noalloc(const void* q, const void* k, 
     if (G > kNoAllocMaxGroups) return LINATTN_ERR_WORKSPACE;  // beyond the fixed scratch
     const uintptr_t bits = (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out | (uintptr_t)Wq | (uintptr_t)Wk;
     if (bits & 15u) return LINATTN_ERR_INVALID_ARG;
+    // out is written while q, k, v are still being read: it must not overlap any of them
+    const size_t bytes = (size_t)G * (size_t)n * (size_t)d * (dtype == LINATTN_BF16 ? 2u : 4u);
+    const uintptr_t o0 = (uintptr_t)out;
+    for (const void* in : {q, k, v}) {
+        const uintptr_t i0 = (uintptr_t)in;
+        if (o0 < i0 + bytes && i0 < o0 + bytes) return LINATTN_ERR_INVALID_ARG;
+    }
 
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) {

@@ -2,13 +2,16 @@
 (a plug-in inside someone else's memory pool, a serving thread that must not trigger
 cudaMalloc's device-wide synchronisation).  Its scratch is a fixed device array shared by all
 calls, so the test makes two different calls in a row and checks each against the ordinary
-context-based entry point.  Collected last on purpose (file name), so a failure here cannot
-hide any other test in a run that stops at the first failure."""
+context-based entry point and against the fp64 CPU oracle (the context entry point runs the
+same CUDA-core kernels, so agreement with it alone would not catch a fault they share).
+Collected last on purpose (file name), so a failure here cannot hide any other test in a run
+that stops at the first failure."""
 import math
 
 import pytest
 import torch
 
+import oracle
 from paper_2510_08318_b200 import linattn
 from util import assert_parity
 
@@ -47,12 +50,20 @@ def test_two_calls_in_a_row_match_the_context_entry_point():
         torch.cuda.synchronize()
         want = _with_context(q, k, v, Wq, Wk)
         assert_parity(out.double().cpu().numpy(), want.double().cpu().numpy(), f"noalloc B={B} H={H} n={n} d={d}")
+        ref = oracle.ref_linear(q.cpu(), k.cpu(), v.cpu(), Wq.cpu(), Wk.cpu())
+        assert_parity(out.double().cpu().numpy(), ref, f"noalloc vs the oracle, B={B} H={H} n={n} d={d}")
     # shared weights ([d, d/2]) on the same scratch again
     q, k, v, Wq, Wk = _inputs(1, 2, 500, 128, torch.bfloat16, 23)
     out = torch.empty_like(q)
     linattn.forward_noalloc(q, k, v, Wq[0].contiguous(), Wk[0].contiguous(), out)
     want = _with_context(q, k, v, Wq[0].contiguous(), Wk[0].contiguous())
     assert_parity(out.double().cpu().numpy(), want.double().cpu().numpy(), "noalloc shared weights")
+    assert_parity(out.double().cpu().numpy(), oracle.ref_linear(q.cpu(), k.cpu(), v.cpu(), Wq[0].cpu(), Wk[0].cpu()),
+                  "noalloc shared weights vs the oracle")
+    # out may not overlap an input: refused before anything is launched
+    st = lib.linattn_forward_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), q.data_ptr(), Wq.data_ptr(), Wk.data_ptr(),
+                                     1, 1, 2, 500, 128, linattn.BF16, None)
+    assert st == linattn.ERR_INVALID_ARG
     # beyond the fixed scratch: B*H = 17 > 16 is refused with the workspace error, nothing is launched
     q, k, v, Wq, Wk = _inputs(1, 17, 64, 64, torch.bfloat16, 24)
     st = lib.linattn_forward_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), torch.empty_like(q).data_ptr(),
