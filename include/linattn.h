@@ -58,6 +58,13 @@ typedef enum {
                                (or backward) on the same k and v POINTERS, B, n and layout, with the same feature map.
                                The caller promises that the contents of k and v have not changed in between (the
                                forward -> backward order of a training step).  0 = always recompute (default) */
+    LINATTN_OPT_WAIT_LIMIT_US = 7, /* bound, in microseconds, of every wait inside the tensor-core forward kernels (on a
+                               shared-memory barrier or on another CTA): default 2,000,000.  A wait that runs out makes the
+                               kernel record a code, unwind and return; linattn_check then reports LINATTN_ERR_TIMEOUT */
+    LINATTN_OPT_TEST_UNMET_ARRIVAL = 8, /* for tests of the time-out path only: 1 = the single-kernel forward waits, at the
+                               points where the CTAs that share a head meet, for one arrival more than will ever come, so
+                               that its bounded wait runs out (nothing faults or hangs: the kernel gives up after the wait
+                               limit, the output is not produced, linattn_check reports TIMEOUT).  0 = off (default) */
     LINATTN_OPT_PROFILE = 2 /* 1 = record CUDA events around every kernel of each forward (see linattn_profile_get);
                                switching it on clears the accumulated figures; 0 = off (default) */
 } linattn_option;
@@ -91,10 +98,9 @@ linattn_status linattn_set_feature_map(linattn_ctx* ctx, const void* Wq, const v
  *   stream  : a cudaStream_t of the context's device (NULL = default stream)
  * All accumulation (S, z, numerator, denominator) is fp32.  The call allocates nothing, does not
  * synchronise, and is deterministic: the same inputs give bit-identical outputs.  Calls on one
- * context must be stream-ordered (they share the context's workspace).  The call may be recorded
- * into a CUDA graph (stream capture): while `stream` is capturing, the tensor-core path records
- * its three-launch form instead of the single cooperative kernel, because that kernel's
- * grid-barrier targets are computed on the host for each launch and would be stale on replay.
+ * context must be stream-ordered (they share the context's workspace).  Nothing about a launch
+ * depends on earlier launches (the single cooperative kernel of the tensor-core path leaves its
+ * synchronisation counters cleared), so the call may be recorded into a CUDA graph and replayed.
  * Errors: INVALID_ARG, UNSUPPORTED, NO_FEATURE_MAP, WORKSPACE, CUDA (launch failure).
  */
 linattn_status linattn_forward(linattn_ctx* ctx, const void* q, const void* k, const void* v, void* out,

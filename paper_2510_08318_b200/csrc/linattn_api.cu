@@ -54,8 +54,8 @@ struct linattn_ctx {
     __nv_bfloat16* z_img = nullptr;  // [max_B*H][2048] bf16 operand image of z (hi, lo)
     int num_sms = 0;
     bool coop_ok = false;            // device supports cooperative launches
-    uint32_t* sync_words = nullptr;  // grid-barrier arrival counter of the fused kernel (only ever grows)
-    uint32_t bar_total = 0;          // its value after the launches enqueued so far
+    uint32_t* sync_words = nullptr;  // fused kernel: 1 + 2 * max_B * H counters (exit count, two meeting points per (b,h) pair), zero between launches
+    size_t sync_bytes = 0;
     // workspace
     float* partial = nullptr;   // [partial_slots][d*d + d]
     long long partial_slots = 0;
@@ -83,6 +83,8 @@ struct linattn_ctx {
     int opt_layout = 0;   // 0: [B][H][n][d], 1: [B][n][H][d]
     int opt_phi = 0;      // 0: Hedgehog feature map (Eq. 6), 1: ReLU kernel function
     int opt_reuse = 0;    // 1: linattn_backward may take S, z from the forward that just ran on the same k, v
+    long long opt_wait_limit_us = 2000000;   // bound of every device-side wait
+    int opt_unmet = 0;    // test hook: the fused kernel's meeting points wait for one arrival that never comes
     // which problem the S, z (tensor-core layout, with the bf16 image of S) in the workspace belong to
     struct StateKey {
         const void* k = nullptr;
@@ -325,12 +327,13 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmS, tmA;   // tmA: the softmax branch's output (mixed attention), else a copy of tmQ
     const ActStrides as = act_strides(c, n);
     const int layout = c->opt_layout;
-    auto act_map = [&](CUtensorMap* m, const void* base) {
-        if (layout == 0) return make_tmap_bf16_3d(m, base, kD, (uint64_t)n, (uint64_t)G, kTile);
+    auto act_map = [&](CUtensorMap* m, const void* base, uint32_t box_rows = kTile) {
+        if (layout == 0) return make_tmap_bf16_3d(m, base, kD, (uint64_t)n, (uint64_t)G, box_rows);
         return make_tmap_bf16_act(m, base, kD, (uint64_t)n, (uint64_t)Hv, (uint64_t)B, (uint64_t)as.token * 2,
-                                  (uint64_t)as.head * 2, (uint64_t)as.batch * 2, kTile);
+                                  (uint64_t)as.head * 2, (uint64_t)as.batch * 2, box_rows);
     };
-    const bool ok = act_map(&tmK, k) && act_map(&tmV, v) && act_map(&tmQ, q) && act_map(&tmO, out) && act_map(&tmA, mix ? mix : q) &&
+    // V is fetched in half tiles (the key side's V ring), everything else in whole tiles
+    const bool ok = act_map(&tmK, k) && act_map(&tmV, v, kTile / 2) && act_map(&tmQ, q) && act_map(&tmO, out) && act_map(&tmA, mix ? mix : q) &&
                     make_tmap_bf16_3d(&tmWk, c->Wkt + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
                     make_tmap_bf16_3d(&tmWq, c->Wqt + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
                     make_tmap_bf16_3d(&tmS, c->s_img + (size_t)c->view_g0 * kD * kD, kD, kD, (uint64_t)G, kTile);
@@ -380,24 +383,17 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
 #ifdef LINATTN_TRACE
     a.trace = c->trace;
 #endif
+    a.wait_limit_us = (uint32_t)c->opt_wait_limit_us;
+    a.arrive_extra = (uint32_t)c->opt_unmet;
     prof_begin(c, st);
-    // The fused kernel's grid-barrier targets are computed here, when the launch is enqueued, from a counter that only
-    // grows: a launch recorded into a CUDA graph would carry stale targets when the graph is replayed.  While the stream
-    // is being captured the three-launch form (no barrier, no host-side bookkeeping) is recorded instead.
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
-        cudaGetLastError();
-        cap = cudaStreamCaptureStatusNone;
-    }
-    if (c->opt_fuse && c->coop_ok && Pk == Pq && !state_only && cap == cudaStreamCaptureStatusNone) {
-        // one cooperative launch: key side, grid barrier, combine, grid barrier, query side
-        a.bar_target[0] = c->bar_total + (uint32_t)Pq;
-        a.bar_target[1] = c->bar_total + 2u * (uint32_t)Pq;
+    if (c->opt_fuse && c->coop_ok && Pk == Pq && !state_only) {
+        // one cooperative launch: key side, per-head meeting point, combine, per-head meeting point, query side.  Its
+        // counters are zero between launches (the kernel clears them on its way out), so nothing here depends on
+        // earlier launches and the launch may be recorded in a CUDA graph.
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
         const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout][phi], dim3((unsigned)Pq), dim3(kThreads),
                                                            params, Smem::kTotal, st);
         if (le == cudaSuccess) {
-            c->bar_total += 2u * (uint32_t)Pq;   // only a launch that was enqueued moves the counter
             prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
             c->last_launches = 1;
             return LINATTN_OK;
@@ -612,8 +608,9 @@ linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, l
         e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device);
         c->coop_ok = (coop != 0);
     }
-    if (e == cudaSuccess) e = cudaMalloc(&c->sync_words, 2 * sizeof(uint32_t));
-    if (e == cudaSuccess) e = cudaMemset(c->sync_words, 0, 2 * sizeof(uint32_t));
+    c->sync_bytes = sizeof(uint32_t) * (size_t)(1 + 2 * G);
+    if (e == cudaSuccess) e = cudaMalloc(&c->sync_words, c->sync_bytes);
+    if (e == cudaSuccess) e = cudaMemset(c->sync_words, 0, c->sync_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->err_word, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->err_word, 0, sizeof(unsigned int));
     if (e != cudaSuccess) {
@@ -954,6 +951,14 @@ linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long 
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
             c->opt_reuse = (int)value;
             return LINATTN_OK;
+        case LINATTN_OPT_WAIT_LIMIT_US:
+            if (value < 1 || value > 60LL * 1000 * 1000) return LINATTN_ERR_INVALID_ARG;
+            c->opt_wait_limit_us = value;
+            return LINATTN_OK;
+        case LINATTN_OPT_TEST_UNMET_ARRIVAL:
+            if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
+            c->opt_unmet = (int)value;
+            return LINATTN_OK;
         case LINATTN_OPT_FUSE:
             if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
             c->opt_fuse = (int)value;
@@ -991,8 +996,7 @@ linattn_status linattn_check(linattn_ctx* c, void* stream)
     LA_CUDA(c, cudaStreamSynchronize(st));
     if (w != 0) {
         LA_CUDA(c, cudaMemsetAsync(c->err_word, 0, sizeof(w), st));
-        LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, 2 * sizeof(uint32_t), st));  // an aborted launch leaves the counter short
-        c->bar_total = 0;
+        LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, c->sync_bytes, st));  // an aborted launch does not clear its meeting-point counters
         snprintf(c->err_text, sizeof(c->err_text), "device-side wait gave up (code 0x%x)", w);
         return LINATTN_ERR_TIMEOUT;
     }

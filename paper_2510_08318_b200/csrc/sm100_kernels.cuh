@@ -1,7 +1,7 @@
 // Tensor-core kernels (tcgen05 + TMEM + TMA) for linear attention with the Hedgehog feature map,
 // bf16 storage, head dimension 128.  The forward has three steps, run either as ONE persistent
-// cooperative kernel (linattn_fused_tc: key side, grid barrier, combine, grid barrier, query side) or as
-// three launches:
+// cooperative kernel (linattn_fused_tc: key side, per-head meeting point, combine, per-head meeting point,
+// query side) or as three launches:
 //
 //   kside_tc   : persistent CTAs stream 128-token tiles of K and V.  Per tile
 //                  U = K W_k          (tcgen05.mma, 128x64x128, fp32 in TMEM)                 Eq. 6
@@ -21,7 +21,7 @@
 // Warp roles (16 warps): warps 0-3 feature map softmax(+U), warps 4-7 softmax(-U) (one token per thread),
 // warp 8 TMA producer, warp 9 issues the logits MMAs, warp 10 issues the accumulation MMAs, warp 11 issues
 // the TMA stores (query side), warps 12-15 query-side epilogue (num / den -> bf16 output tile) and, in the
-// fused kernel, the grid barriers and the combine step between the two sides.  Role loops are
+// fused kernel, warps 10-15 do the meeting points and the combine step between the two sides.  Role loops are
 // warp-uniform; single-thread work (TMA and MMA issue) is predicated inside them.
 // Every wait is bounded: on time-out the kernel records a code in *err, raises the CTA's abort word so
 // that the other roles stop waiting too, and unwinds.
@@ -46,7 +46,7 @@ constexpr uint32_t kTileBytes = kTile * kD * 2;       // 32 KB: one [128 x 128] 
 constexpr uint32_t kHalfTileBytes = kTileBytes / 2;   // one 64-column block of a tile
 constexpr uint32_t kWBytes = kM * kD * 2;             // 16 KB: W^T [64 x 128] bf16
 constexpr uint32_t kZBlkBytes = 2 * 16 * 128;         // 4 KB: z operand, [2 blocks][16 rows][64] bf16
-constexpr uint64_t kWaitLimitNs = 2000ull * 1000 * 1000;
+constexpr uint32_t kWaitLimitUs = 2000u * 1000u;   // default bound of every device-side wait: 2 s
 constexpr float kLog2e = 1.4426950408889634f;
 
 // error codes OR-ed into *err (which wait gave up)
@@ -107,12 +107,14 @@ template <int N> struct Ring {
 struct WaitCtx {
     uint32_t* err;        // global error word
     uint32_t abort_smem;  // shared-memory address of the CTA's abort word
+    uint32_t limit_us = kWaitLimitUs;   // bound of each wait
+    __device__ __forceinline__ uint64_t limit_ns() const { return (uint64_t)limit_us * 1000u; }
 };
 
 // All lanes wait (bounded); the verdict is made warp-uniform so that role loops never diverge.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc, uint32_t code)
 {
-    const bool ok = mbar_wait_abortable(bar, parity, kWaitLimitNs, wc.abort_smem);
+    const bool ok = mbar_wait_abortable(bar, parity, wc.limit_ns(), wc.abort_smem);
     const bool all = __all_sync(0xffffffffu, ok);
     if (!all && (threadIdx.x & 31) == 0) {
         atomicOr(wc.err, code);
@@ -308,22 +310,25 @@ __device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_sme
 // Shared-memory layout, barriers and per-CTA state common to all three kernels
 // ======================================================================================================
 
-// Key side: K and V tiles have rings of their own.  A K slot is held from the issue of its load until the accumulation
-// MMA has consumed the phi written over it (load latency + logits MMA + feature map + MMA); a V tile is needed only
-// by that last MMA, so its load is issued one tile later and its slot lives about half as long: four K slots and
-// two V slots keep more loads in flight than three (K, V) pairs of the same 192 KB.
+// Key side: K and V have rings of their own.  A K slot is held from the issue of its load until the accumulation
+// MMA has consumed the phi written over it (load latency + logits MMA + feature map + MMA).  V is needed only by that
+// last MMA; its ring works in HALF tiles (64 tokens, the tokens of four of the MMA's eight K steps), each half with its
+// own barriers, so that a half goes back to the producer as soon as its four K steps are done.  The rate of the key
+// side is set by the slower of the two rings' loops, (hold time) / (slots): with whole-tile V slots, two of them gave
+// (V load latency 2-3 us + MMA 0.8 us) / 2 = 1.75 us per tile against the 1.36 us per tile at which HBM delivers, and a
+// third did not fit; five half tiles do (the feature-map weights are single-buffered to make the room).
 constexpr int kKSlots = 4;
-constexpr int kVSlots = 2;
-constexpr int kVLag = 1;      // the load of V tile i is issued together with that of K tile i + kVLag
+constexpr int kVHalves = 5;   // V ring: half tiles of 64 tokens x 128 columns (16 KB)
+constexpr int kVLag = 1;      // the loads of V tile i are issued after that of K tile i + kVLag
 constexpr int kQStages = 5;   // query side: stages of one Q tile (reused for phi(q) and then the output tile)
 constexpr int kThreads = 512; // 16 warps
 constexpr int kQPrefetchL2 = 3;   // fused kernel: Q tiles pulled into L2 while the CTA waits for S (measured: 2-3 best, 6+ slows the combine)
 
 struct Smem {
     // key side
-    static constexpr uint32_t kKV = kKSlots * kTileBytes;                 // K slots (each later holds phi), then the V slots
-    static constexpr uint32_t kKW = (kKSlots + kVSlots) * kTileBytes;     // 2 x W_k^T
-    static constexpr uint32_t kOnes = kKW + 2 * kWBytes;                  // 1 KB of bf16 ones
+    static constexpr uint32_t kKV = kKSlots * kTileBytes;                 // K slots (each later holds phi), then the V half-tile slots
+    static constexpr uint32_t kKW = kKV + kVHalves * kHalfTileBytes;      // W_k^T
+    static constexpr uint32_t kOnes = kKW + kWBytes;                      // 1 KB of bf16 ones
     static constexpr uint32_t kKEnd = kOnes + 1024;
     // query side (overlays the key-side region)
     // [S | z] operand of the query side: per 64-feature block 144 rows of 128 bytes, rows 0-127 = S image [c][f],
@@ -339,14 +344,14 @@ struct Smem {
 // mbarrier indices
 enum : int {
     // key side
-    K_FULL = 0, K_EMPTY = 4, K_PHIFULL = 8, K_VFULL = 12, K_VEMPTY = 14, K_UFULL = 16, K_UEMPTY = 18, K_WFULL = 20, K_WFREE = 22,
-    K_ACCFULL = 24, K_ACCFREE = 26,
+    K_FULL = 0, K_EMPTY = 4, K_PHIFULL = 8, K_VFULL = 12, K_VEMPTY = 18, K_UFULL = 24, K_UEMPTY = 26, K_WFULL = 28, K_WFREE = 29,
+    K_ACCFULL = 30, K_ACCFREE = 32,
     // query side
-    Q_FULL = 28, Q_EMPTY = 33, Q_PHIFULL = 38, Q_OFULL = 43, Q_UFULL = 48, Q_UEMPTY = 50, Q_DFULL = 52, Q_DEMPTY = 54,
-    Q_SEGFULL = 56, Q_SEGFREE = 57, Q_SREADY = 58, Q_WFULL = 59, Q_AFULL = 60,
-    NBARS = 65
+    Q_FULL = 34, Q_EMPTY = 39, Q_PHIFULL = 44, Q_OFULL = 49, Q_UFULL = 54, Q_UEMPTY = 56, Q_DFULL = 58, Q_DEMPTY = 60,
+    Q_SEGFULL = 62, Q_SEGFREE = 63, Q_WFULL = 65, Q_AFULL = 66,
+    NBARS = 71
 };
-static_assert(kKSlots <= K_EMPTY - K_FULL && kVSlots <= K_VEMPTY - K_VFULL, "one mbarrier per ring slot: widen the enum before growing a ring");
+static_assert(kKSlots <= K_EMPTY - K_FULL && kVHalves <= K_VEMPTY - K_VFULL, "one mbarrier per ring slot: widen the enum before growing a ring");
 
 struct Cta {
     uint8_t* smem;
@@ -362,8 +367,10 @@ struct Args {
     __nv_bfloat16* s_img;        // [G][128][128] bf16 image of S, [c][f]
     __nv_bfloat16* z_img;        // [G][kZBlkBytes / 2] bf16 operand image of z (hi, lo)
     uint32_t* err;               // error word
-    uint32_t* sync;              // grid-barrier arrival counter of the fused kernel (monotonic over launches)
-    uint32_t bar_target[2];      // its value once every CTA has arrived at the first / second barrier of this launch
+    uint32_t* sync;              // fused kernel: [0] CTAs that have left their last wait; [1 + 2g], [2 + 2g] arrivals at the two
+                                 // per-head meeting points of (b,h) pair g.  All zero between launches (the kernel re-zeroes them)
+    uint32_t wait_limit_us;      // bound of every device-side wait
+    uint32_t arrive_extra;       // 0; a test sets 1, which makes every meeting point wait for one arrival more than will ever come
     const __nv_bfloat16* mix_src;  // Eq. 8: output of the softmax-attention branch [G][n][128], or nullptr (plain Eq. 5)
     float mix_r;                 // Eq. 8: the score r, already clipped into [0, 1]
     long long str_token, str_head, str_batch;  // element strides of q, k, v, out (and mix_src) between tokens, heads, batches
@@ -389,12 +396,15 @@ __device__ __forceinline__ Cta cta_setup(uint8_t* smem_raw, const Args& a, bool 
     c.lane = threadIdx.x & 31;
     c.wc.err = a.err;
     c.wc.abort_smem = smem_u32(abort_word);
+    c.wc.limit_us = a.wait_limit_us;
     if (threadIdx.x == 0) {
         *abort_word = 0u;
         if (init_k) {
             for (int i = 0; i < kKSlots; ++i) { mbar_init(c.bar(K_FULL + i), 1); mbar_init(c.bar(K_EMPTY + i), 1); mbar_init(c.bar(K_PHIFULL + i), 8); }
-            for (int i = 0; i < kVSlots; ++i) { mbar_init(c.bar(K_VFULL + i), 1); mbar_init(c.bar(K_VEMPTY + i), 1); }
-            for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_UFULL + i), 1); mbar_init(c.bar(K_UEMPTY + i), 8); mbar_init(c.bar(K_WFULL + i), 1); mbar_init(c.bar(K_WFREE + i), 1); }
+            for (int i = 0; i < kVHalves; ++i) { mbar_init(c.bar(K_VFULL + i), 1); mbar_init(c.bar(K_VEMPTY + i), 1); }
+            for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_UFULL + i), 1); mbar_init(c.bar(K_UEMPTY + i), 8); }
+            mbar_init(c.bar(K_WFULL), 1);
+            mbar_init(c.bar(K_WFREE), 1);
             for (int i = 0; i < 2; ++i) { mbar_init(c.bar(K_ACCFULL + i), 1); mbar_init(c.bar(K_ACCFREE + i), 4); }
         }
         if (init_q) {
@@ -402,7 +412,6 @@ __device__ __forceinline__ Cta cta_setup(uint8_t* smem_raw, const Args& a, bool 
             for (int i = 0; i < 2; ++i) { mbar_init(c.bar(Q_UFULL + i), 1); mbar_init(c.bar(Q_UEMPTY + i), 8); mbar_init(c.bar(Q_DFULL + i), 1); mbar_init(c.bar(Q_DEMPTY + i), 4); }
             mbar_init(c.bar(Q_SEGFULL), 1);
             mbar_init(c.bar(Q_SEGFREE), 1);
-            mbar_init(c.bar(Q_SREADY), 4);
             mbar_init(c.bar(Q_WFULL), 1);
         }
         fence_mbar_init();
@@ -443,6 +452,15 @@ __device__ __forceinline__ void act_store(const void* tm, uint32_t src, int x, i
     if (kLayout == 0) tma_store_3d(tm, src, x, t, g);
     else tma_store_4d(tm, src, x, t, g % H, g / H);
 }
+// The output tiles are stored with the L2 policy "evict last": the lines of the output then outlive, in L2, the lines of
+// q that stream through next to them (measured: 2 us of 82 at B=1, H=12, n=32760), and whatever consumes the output next
+// finds more of it on chip.
+template <int kLayout>
+__device__ __forceinline__ void act_store(const void* tm, uint32_t src, int x, int t, int g, int H, uint64_t policy)
+{
+    if (kLayout == 0) tma_store_3d_hint(tm, src, x, t, g, policy);
+    else tma_store_4d_hint(tm, src, x, t, g % H, g / H, policy);
+}
 template <int kLayout>
 __device__ __forceinline__ void act_prefetch_l2(const void* tm, int x, int t, int g, int H)
 {
@@ -467,15 +485,59 @@ __device__ __forceinline__ void relu_tile_in_place(uint8_t* tile, int t)
     }
 }
 
+// ---- Meeting points of the fused kernel ---------------------------------------------------------------
+// The one dependency of the forward: the query side of (b,h) pair g needs the S, z of ALL of g's keys.  The CTAs whose
+// runs touch g meet twice, on two counters of their own: once when each has written its partial record of g (then
+// each sums its share of the record), once when each has written its share of the sum (then each may load S, z).
+// A CTA waits only for the few CTAs that share a head with it, not for the slowest of the whole grid.  The counters
+// are zero when a launch starts and the kernel leaves them zero (the last CTA out clears them), so nothing about a
+// launch is computed on the host and a launch recorded in a CUDA graph can be replayed.  Co-residency of the CTAs is
+// what the cooperative launch guarantees.  Every wait is bounded and stops when the CTA's abort word is raised.
+
+// First CTA whose run touches (b,h) pair g, and how many do.
+__device__ __forceinline__ void head_ctas(const Args& a, long long P, int g, int& c0, int& cnt)
+{
+    c0 = (int)tile_owner((long long)g * a.tiles_per_head, a.total_tiles, P);
+    cnt = (int)tile_owner((long long)(g + 1) * a.tiles_per_head - 1, a.total_tiles, P) - c0 + 1;
+}
+constexpr uint32_t kDrainWarps = 4;   // arrivals per CTA at a head's first meeting point (one per drain warp)
+// Called by ONE thread after a warp- or CTA-level barrier: the release, together with that barrier, publishes what every
+// thread that took part in it wrote before.
+__device__ __forceinline__ void meet_arrive(uint32_t* ctr)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(ctr) : "memory");
+}
+// Called by ONE thread, followed by a CTA-level barrier (or a shuffle) that hands the verdict to the others.
+__device__ __forceinline__ bool meet_wait(const uint32_t* ctr, uint32_t target, const WaitCtx& wc)
+{
+    if (ld_acquire_gpu(ctr) >= target) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (ld_acquire_gpu(ctr) < target) {
+        if ((++spins & 15u) == 0u) {
+            uint32_t ab;
+            asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(ab) : "r"(wc.abort_smem) : "memory");
+            if (ab != 0u || globaltimer_ns() - t0 > wc.limit_ns()) return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void raise_abort(const WaitCtx& wc, uint32_t code)
+{
+    atomicOr(wc.err, code);
+    asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(wc.abort_smem), "r"(1u) : "memory");
+}
+
 // ======================================================================================================
 // Key side: partial S = sum phi(k)^T v and z = sum phi(k) over this CTA's tiles (Eq. 5 brackets, Eq. 6)
 // ======================================================================================================
 
 // kPhi: 0 = the Hedgehog feature map of Eq. 6; 1 = the ReLU kernel function (no projection, no softmax: the logits
 // warp idles and warps 0-7 rectify the K tile in place).
+// arrive: fused kernel; every partial record written is announced at its head's first meeting point.
 template <int kLayout, int kPhi>
 __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const CUtensorMap* tmK, const CUtensorMap* tmV,
-                                            const CUtensorMap* tmW)
+                                            const CUtensorMap* tmW, bool arrive)
 {
     const uint32_t tmem_u = c.tmem;            // 2 x 64 columns of logits
     // two accumulator sets, alternating by segment, so that one drains while the next accumulates
@@ -494,33 +556,26 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             tma_prefetch_desc(tmW);
         }
         Ring<kKSlots> r;
-        Ring<kVSlots> vr;
+        Ring<kVHalves> vr;
         TileWalk wv = w;                 // walks the V tiles, kVLag tiles behind the K tiles
-        int issued = 0, issued_v = 0;    // K and V loads issued so far
+        int issued = 0, issued_v = 0;    // K tiles and V half tiles whose loads have been issued so far
         bool ok = true;
+        // one half tile of V: tokens [64 h, 64 h + 64) of tile wv, as two boxes of 64 columns (the map's box is 64 rows high);
+        // a half that lies past the end of the sequence is zero-filled like any out-of-range row
         auto issue_v = [&]() {
-            if (issued_v >= kVSlots && !warp_wait(c.bar(K_VEMPTY + vr.s), vr.ph ^ 1u, c.wc, kErrProducer)) { ok = false; return; }
+            if (issued_v >= kVHalves && !warp_wait(c.bar(K_VEMPTY + vr.s), vr.ph ^ 1u, c.wc, kErrProducer)) { ok = false; return; }
             if (lane == 0) {
-                mbar_arrive_expect_tx(c.bar(K_VFULL + vr.s), kTileBytes);
-                const uint32_t vdst = sbase + Smem::kKV + vr.s * kTileBytes;
-                act_load<kLayout>(vdst, tmV, c.bar(K_VFULL + vr.s), 0, wv.lt * kTile, wv.g, a.H);
-                act_load<kLayout>(vdst + kHalfTileBytes, tmV, c.bar(K_VFULL + vr.s), 64, wv.lt * kTile, wv.g, a.H);
+                mbar_arrive_expect_tx(c.bar(K_VFULL + vr.s), kHalfTileBytes);
+                const uint32_t vdst = sbase + Smem::kKV + vr.s * kHalfTileBytes;
+                const int row = wv.lt * kTile + (issued_v & 1) * (kTile / 2);
+                act_load<kLayout>(vdst, tmV, c.bar(K_VFULL + vr.s), 0, row, wv.g, a.H);
+                act_load<kLayout>(vdst + kHalfTileBytes / 2, tmV, c.bar(K_VFULL + vr.s), 64, row, wv.g, a.H);
             }
+            if (issued_v & 1) wv.next();
             ++issued_v;
-            wv.next();
             vr.next();
         };
         for (; !w.done() && ok; w.next(), r.next()) {
-            if (kPhi == 0 && w.first()) {
-                const int wb = w.seg & 1;
-                if (w.seg >= 2 && !warp_wait(c.bar(K_WFREE + wb), ((w.seg >> 1) - 1) & 1, c.wc, kErrProducer)) { ok = false; break; }
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(c.bar(K_WFULL + wb), kWBytes);
-                    const uint32_t wdst = sbase + Smem::kKW + wb * kWBytes;
-                    tma_load_3d(wdst, tmW, c.bar(K_WFULL + wb), 0, 0, w.g % a.H);
-                    tma_load_3d(wdst + kWBytes / 2, tmW, c.bar(K_WFULL + wb), 64, 0, w.g % a.H);
-                }
-            }
             if (w.i >= kKSlots && !warp_wait(c.bar(K_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) { ok = false; break; }
             LA_TRACE(0, w.i, 0);
             if (lane == 0) {
@@ -530,31 +585,44 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
                 act_load<kLayout>(kdst + kHalfTileBytes, tmK, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
             }
             issued = w.i + 1;
-            if (w.i >= kVLag) issue_v();
+            if (w.i >= kVLag) {
+                issue_v();
+                if (ok) issue_v();
+            }
         }
-        while (ok && issued_v < issued) issue_v();
+        while (ok && issued_v < 2 * issued) issue_v();
         if (!ok) {
             // unwinding after a time-out: let the copies already in flight land before the CTA moves on
             for (int i = (issued > kKSlots ? issued - kKSlots : 0); i < issued; ++i)
-                mbar_wait(c.bar(K_FULL + i % kKSlots), (uint32_t)(i / kKSlots) & 1u, kWaitLimitNs);
-            for (int i = (issued_v > kVSlots ? issued_v - kVSlots : 0); i < issued_v; ++i)
-                mbar_wait(c.bar(K_VFULL + i % kVSlots), (uint32_t)(i / kVSlots) & 1u, kWaitLimitNs);
+                mbar_wait(c.bar(K_FULL + i % kKSlots), (uint32_t)(i / kKSlots) & 1u, c.wc.limit_ns());
+            for (int i = (issued_v > kVHalves ? issued_v - kVHalves : 0); i < issued_v; ++i)
+                mbar_wait(c.bar(K_VFULL + i % kVHalves), (uint32_t)(i / kVHalves) & 1u, c.wc.limit_ns());
         }
     } else if (warp == 9) {
         // ---------------- logits MMA issuer: U = K W_k ----------------
+        // This warp also fetches the head's W_k^T (one buffer): at a head boundary it waits for its own last logits MMAs
+        // of the previous head, loads the next head's matrix (16 KB, an L2 hit after the first CTA) and goes on; the K
+        // and V loads of the producer are not held up meanwhile.
         Ring<kKSlots> r;
         Ring<2> ur;
         for (; kPhi == 0 && !w.done(); w.next(), r.next(), ur.next()) {
-            const int wb = w.seg & 1;
-            if (w.first() && !warp_wait(c.bar(K_WFULL + wb), (uint32_t)(w.seg >> 1) & 1u, c.wc, kErrMmaLoad)) break;
+            if (w.first()) {
+                if (w.seg >= 1 && !warp_wait(c.bar(K_WFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrMmaLoad)) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(c.bar(K_WFULL), kWBytes);
+                    tma_load_3d(sbase + Smem::kKW, tmW, c.bar(K_WFULL), 0, 0, w.g % a.H);
+                    tma_load_3d(sbase + Smem::kKW + kWBytes / 2, tmW, c.bar(K_WFULL), 64, 0, w.g % a.H);
+                }
+                if (!warp_wait(c.bar(K_WFULL), (uint32_t)w.seg & 1u, c.wc, kErrMmaLoad)) break;
+            }
             if (!warp_wait(c.bar(K_FULL + r.s), r.ph, c.wc, kErrMmaLoad)) break;
             LA_TRACE(1, w.i, 0);
             if (w.i >= 2 && !warp_wait(c.bar(K_UEMPTY + ur.s), ur.ph ^ 1u, c.wc, kErrMmaU)) break;
             tcgen05_fence_after();
             if (elect_one()) {
-                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + Smem::kKW + wb * kWBytes);
+                issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + Smem::kKW);
                 mma_commit(c.bar(K_UFULL + ur.s));
-                if (w.last()) mma_commit(c.bar(K_WFREE + wb));
+                if (w.last()) mma_commit(c.bar(K_WFREE));
             }
             __syncwarp();
             LA_TRACE(1, w.i, 1);
@@ -564,32 +632,40 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
         constexpr uint32_t idesc_s = make_idesc_bf16(kD, kD, 1, 1);   // A = phi^T (MN-major), B = V (MN-major)
         constexpr uint32_t idesc_z = make_idesc_bf16(kD, 16, 1, 0);   // B = ones (K-major, no swizzle)
         const uint64_t ones_desc = make_desc_noswizzle(sbase + Smem::kOnes, 128, 256);
-        const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
+        const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);        // phi^T: blocks of 64 features 16 KB apart
+        const uint64_t mnmajor_v = make_desc_sw128(0, kHalfTileBytes / 2, 1024);  // V half tile: blocks of 64 columns 8 KB apart
         Ring<kKSlots> r;
-        Ring<kVSlots> vr;
-        for (; !w.done(); w.next(), r.next(), vr.next()) {
+        Ring<kVHalves> vr;
+        bool ok = true;
+        for (; !w.done() && ok; w.next(), r.next()) {
             if (!warp_wait(c.bar(K_PHIFULL + r.s), r.ph, c.wc, kErrMmaPhi)) break;
-            if (!warp_wait(c.bar(K_VFULL + vr.s), vr.ph, c.wc, kErrMmaLoad)) break;
-            LA_TRACE(1, w.i, 2);
             const bool first = w.first();
             const int b = w.seg & 1;
             if (first && w.seg >= 2 && !warp_wait(c.bar(K_ACCFREE + b), (uint32_t)((w.seg >> 1) - 1) & 1u, c.wc, kErrMmaAcc)) break;
-            tcgen05_fence_after();
-            if (elect_one()) {
-                const uint32_t phi = sbase + r.s * kTileBytes, vt = sbase + Smem::kKV + vr.s * kTileBytes;
+            // the tile's eight K steps (16 tokens each) in two halves, each against its own half tile of V
+            for (int h = 0; h < 2 && ok; ++h, vr.next()) {
+                if (!warp_wait(c.bar(K_VFULL + vr.s), vr.ph, c.wc, kErrMmaLoad)) { ok = false; break; }
+                if (h == 0) LA_TRACE(1, w.i, 2);
+                tcgen05_fence_after();
+                if (elect_one()) {
+                    const uint32_t phi = sbase + r.s * kTileBytes, vt = sbase + Smem::kKV + vr.s * kHalfTileBytes;
 #pragma unroll
-                for (int k = 0; k < kTile / 16; ++k) {
-                    const uint64_t da = desc_at(mnmajor, phi + k * 2048);
-                    const uint64_t db = desc_at(mnmajor, vt + k * 2048);
-                    const uint32_t acc = (first && k == 0) ? 0u : 1u;
-                    mma_bf16_ss(tmem_s(b), da, db, idesc_s, acc);
-                    mma_bf16_ss(tmem_z(b), da, ones_desc, idesc_z, acc);
+                    for (int kk = 0; kk < kTile / 32; ++kk) {
+                        const int k = h * (kTile / 32) + kk;
+                        const uint64_t da = desc_at(mnmajor, phi + k * 2048);
+                        const uint64_t db = desc_at(mnmajor_v, vt + kk * 2048);
+                        const uint32_t acc = (first && k == 0) ? 0u : 1u;
+                        mma_bf16_ss(tmem_s(b), da, db, idesc_s, acc);
+                        mma_bf16_ss(tmem_z(b), da, ones_desc, idesc_z, acc);
+                    }
+                    mma_commit(c.bar(K_VEMPTY + vr.s));
+                    if (h == 1) {
+                        mma_commit(c.bar(K_EMPTY + r.s));
+                        if (w.last()) mma_commit(c.bar(K_ACCFULL + b));
+                    }
                 }
-                mma_commit(c.bar(K_EMPTY + r.s));
-                mma_commit(c.bar(K_VEMPTY + vr.s));
-                if (w.last()) mma_commit(c.bar(K_ACCFULL + b));
+                __syncwarp();
             }
-            __syncwarp();
             LA_TRACE(1, w.i, 3);
         }
     } else if (warp < 8 && kPhi == 1) {
@@ -656,6 +732,9 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(c.bar(K_ACCFREE + b));
+            // each of the four drain warps announces its quarter of the record by itself (kDrainWarps arrivals per CTA
+            // and head): a CTA-level barrier here could be left waiting by a warp that gave up a wait
+            if (arrive && lane == 0) meet_arrive(a.sync + 1 + 2 * w.g);
         }
     }
 }
@@ -724,7 +803,7 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
 }
 
 // wait_state: the S and z images are produced earlier in the same kernel (fused path); loads of them
-// must wait for the Q_SREADY barrier.  Otherwise they were written by a previous launch.
+// must wait at the head's second meeting point.  Otherwise they were written by a previous launch.
 template <bool kMix, int kLayout, int kPhi>
 __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
                                             const CUtensorMap* tmW, const CUtensorMap* tmS, const CUtensorMap* tmA, bool wait_state)
@@ -750,8 +829,17 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         bool ok = true;
         auto load_state = [&]() {
             // S and z of head state_g; in the fused kernel they were written by other CTAs with ordinary
-            // stores and become readable once the grid barrier behind Q_SREADY has been passed
-            if (wait_state && !warp_wait(c.bar(Q_SREADY), 0u, c.wc, kErrSeg)) { ok = false; return; }
+            // stores and become readable once every sharer of the head has arrived at its second meeting point
+            if (wait_state) {
+                int c0, cnt;
+                head_ctas(a, gridDim.x, state_g, c0, cnt);
+                int got = 1;
+                if (lane == 0) {
+                    got = meet_wait(a.sync + 2 + 2 * state_g, (uint32_t)cnt + a.arrive_extra, c.wc) ? 1 : 0;
+                    if (!got) raise_abort(c.wc, kErrSeg);
+                }
+                if (!__shfl_sync(0xffffffffu, got, 0)) { ok = false; return; }
+            }
             if (lane == 0) {
                 if (wait_state) fence_proxy_async_all();
                 mbar_arrive_expect_tx(c.bar(Q_SEGFULL), kTileBytes + kZBlkBytes);
@@ -782,17 +870,19 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             }
             if (state_g >= 0 && w.i >= kQStages) {
                 if (wait_state && w.seg == 0) {
-                    // The ring is full and S does not exist yet.  Once every CTA has drained its accumulators
-                    // (first grid barrier) HBM has nothing to do until the query side starts: use the time to pull
-                    // the next Q tiles of this run into L2.
+                    // The ring is full and S does not exist yet.  Once the CTAs of this head have drained their
+                    // accumulators (first meeting point) HBM has little to do until the query side starts: use the time
+                    // to pull the next Q tiles of this run into L2.
                     bool passed = false;
                     if (lane == 0) {
+                        int c0, cnt;
+                        head_ctas(a, gridDim.x, w.g, c0, cnt);
                         const uint64_t t0 = globaltimer_ns();
-                        while (!(passed = (int32_t)(ld_acquire_gpu(a.sync) - a.bar_target[0]) >= 0)) {
+                        while (!(passed = ld_acquire_gpu(a.sync + 1 + 2 * w.g) >= kDrainWarps * (uint32_t)cnt)) {
                             __nanosleep(200);
                             uint32_t ab;
                             asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(ab) : "r"(c.wc.abort_smem) : "memory");
-                            if (ab != 0u || globaltimer_ns() - t0 > kWaitLimitNs) break;
+                            if (ab != 0u || globaltimer_ns() - t0 > c.wc.limit_ns()) break;
                         }
                         if (passed) {
                             TileWalk pw = w;
@@ -827,9 +917,18 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             issued = w.i + 1;
         }
         if (ok && state_g >= 0) load_state();
-        if (issued < w.count) {
+        if (wait_state && ok) {
+            // This CTA has left the last of its waits on the meeting points.  The last CTA to say so clears the counters
+            // for the next launch (nobody reads them any more: every CTA is past its last wait).
+            uint32_t old = 0;
+            if (lane == 0) old = atomicAdd(a.sync, 1u);
+            if (__shfl_sync(0xffffffffu, old, 0) == gridDim.x - 1)
+                for (int i = lane; i < 1 + 2 * a.G; i += 32) a.sync[i] = 0u;
+        }
+        if (!ok || issued < w.count) {
+            // unwinding: let the copies already in flight land before the CTA moves on
             for (int i = (issued > kQStages ? issued - kQStages : 0); i < issued; ++i)
-                mbar_wait(c.bar(Q_FULL + i % kQStages), (uint32_t)(i / kQStages) & 1u, kWaitLimitNs);
+                mbar_wait(c.bar(Q_FULL + i % kQStages), (uint32_t)(i / kQStages) & 1u, c.wc.limit_ns());
         }
     } else if (warp == 9) {
         // ---------------- logits MMA issuer: U = Q W_q ----------------
@@ -881,12 +980,13 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         // by itself): the query side runs at the rate at which slots come back, so every microsecond a slot is
         // held longer than needed costs throughput.
         if (lane == 0) tma_prefetch_desc(tmO);
+        const uint64_t keep = policy_evict_last();
         Ring<kQStages> r;
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(Q_OFULL + r.s), r.ph, c.wc, kErrStore)) break;
             if (lane == 0) {
-                act_store<kLayout>(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g, a.H);
-                act_store<kLayout>(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g, a.H);
+                act_store<kLayout>(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g, a.H, keep);
+                act_store<kLayout>(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g, a.H, keep);
                 bulk_commit_group();
                 bulk_wait_group_read<0>();
                 mbar_arrive(c.bar(Q_EMPTY + r.s));
@@ -1021,7 +1121,7 @@ kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtens
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, true, false);
-    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmW);
+    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmW, false);
     cta_teardown(c);
 }
 
@@ -1044,25 +1144,6 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
     cta_teardown(c);
 }
 
-// Grid-wide barrier for a cooperative launch (all CTAs resident).  Called by ONE thread per CTA after a
-// CTA-level barrier.  *counter only ever grows (over launches too); `target` is the value it has once all P
-// CTAs have arrived at this barrier, which the host knows when it enqueues the launch.  One fire-and-forget
-// add and a poll: no value has to come back before the wait can start.  Bounded: returns false on time-out.
-// Ordering: the add is a release at GPU scope and the poll an acquire, and the calling thread is joined to the
-// rest of its CTA by the CTA-level barriers before and after the call, so what any thread of any CTA wrote before
-// the barrier is visible to every thread after it; separate fences around the two were measured to cost 0.9 us
-// per forward and add nothing to that chain.
-__device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target)
-{
-    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
-    const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
-    while ((int32_t)(ld_acquire_gpu(counter) - target) < 0) {
-        if ((++spins & 63u) == 0u && globaltimer_ns() - t0 > kWaitLimitNs) return false;
-    }
-    return true;
-}
-
 // The whole forward in one cooperative launch of P <= #SMs persistent CTAs.
 template <bool kMix, int kLayout, int kPhi>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -1075,45 +1156,44 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     LA_TRACE_NS(0, 60, 0);
     const Cta c = cta_setup(smem_raw, a, true, true);
     LA_TRACE_NS(0, 60, 1);
-    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmWk);
-    // every role is done with the key-side buffers; the partials of this CTA are written
+    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmWk, true);
+    // every role is done with the key-side buffers; the partials of this CTA are written and announced
     tcgen05_fence_before();
     __syncthreads();
     tcgen05_fence_after();
     LA_TRACE_NS(0, 60, 2);
     constexpr int kHoleWarp0 = 10, kHoleThreads = (16 - kHoleWarp0) * 32;
     if (c.warp >= kHoleWarp0) {
-        // warps 10-15 (idle until S exists): grid barrier, combine (spread over all CTAs), grid barrier, then
-        // release the query side.  The other warps go straight on: Q tiles, W_q, the first logits and feature
-        // maps do not depend on S.
-        __shared__ uint32_t gb_ok;
-        const uint32_t P = gridDim.x;
+        // warps 10-15 (idle until S exists): for every head this CTA's run touches, wait at the head's first meeting
+        // point, sum this CTA's share of the head's record, announce it at the second.  The other warps go straight
+        // on: Q tiles, W_q, the first logits and feature maps do not depend on S.
+        __shared__ uint32_t met;
+        const long long P = gridDim.x;
         const int it = threadIdx.x - kHoleWarp0 * 32;
-        if (it == 0) {
-            gb_ok = grid_barrier(a.sync, a.bar_target[0]) ? 1u : 0u;
-            if (!gb_ok) {
-                atomicOr(a.err, (uint32_t)kErrGrid);
-                asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
+        TileWalk w;
+        w.init(a.total_tiles, a.tiles_per_head);
+        bool ok = true;
+        while (!w.done() && ok) {
+            const int g = w.g;
+            int c0, cnt;
+            head_ctas(a, P, g, c0, cnt);
+            if (it == 0) {
+                met = meet_wait(a.sync + 1 + 2 * g, kDrainWarps * (uint32_t)cnt + a.arrive_extra, c.wc) ? 1u : 0u;
+                if (!met) raise_abort(c.wc, kErrGrid);
             }
-        }
-        named_barrier_sync(1, kHoleThreads);
-        if (it == 0) LA_TRACE_NS1(0, 60, 3);
-        if (gb_ok) {
-            const int total = a.G * (kE / 4);   // float4 groups over all heads
-            for (int x = blockIdx.x * kHoleThreads + it; x < total; x += (int)P * kHoleThreads)
-                combine_quad(a, P, x / (kE / 4), (x % (kE / 4)) * 4);
-        }
-        named_barrier_sync(1, kHoleThreads);
-        if (it == 0) LA_TRACE_NS1(0, 61, 0);
-        if (it == 0 && gb_ok) {
-            if (!grid_barrier(a.sync, a.bar_target[1])) {
-                gb_ok = 0u;
-                atomicOr(a.err, (uint32_t)kErrGrid);
-                asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(c.wc.abort_smem), "r"(1u) : "memory");
+            named_barrier_sync(1, kHoleThreads);
+            ok = met != 0u;
+            if (it == 0 && w.seg == 0) LA_TRACE_NS1(0, 60, 3);
+            if (ok) {
+                const int j = (int)blockIdx.x - c0;
+                const int lo = j * (kE / 4) / cnt, hi = (j + 1) * (kE / 4) / cnt;   // this CTA's share: float4 groups [lo, hi)
+                for (int x = lo + it; x < hi; x += kHoleThreads) combine_quad(a, P, g, x * 4);
             }
+            named_barrier_sync(1, kHoleThreads);   // the share is written (and `met` has been read by everybody)
+            if (it == 0 && ok) meet_arrive(a.sync + 2 + 2 * g);
+            if (it == 0 && w.seg == 0) LA_TRACE_NS1(0, 61, 0);
+            do w.next(); while (!w.done() && w.g == g);
         }
-        named_barrier_sync(1, kHoleThreads);
-        if (c.warp >= 12 && c.lane == 0 && gb_ok) mbar_arrive(c.bar(Q_SREADY));
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
     qside_phase<kMix, kLayout, kPhi>(c, a, &tmQ, &tmO, &tmWq, &tmS, &tmA, true);

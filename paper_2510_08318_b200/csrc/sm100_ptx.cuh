@@ -162,6 +162,26 @@ __device__ __forceinline__ void tma_store_3d(const void* tmap, uint32_t src_smem
                  "r"(src_smem), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
+// L2 eviction-priority policy "evict last" for all of an access's lines (an operand of the stores below).
+__device__ __forceinline__ uint64_t policy_evict_last()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+// The tiled stores with an L2 cache hint.
+__device__ __forceinline__ void tma_store_3d_hint(const void* tmap, uint32_t src_smem, int x, int y, int z, uint64_t policy)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;" ::"l"(tmap),
+                 "r"(src_smem), "r"(x), "r"(y), "r"(z), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_4d_hint(const void* tmap, uint32_t src_smem, int x, int y, int z, int w, uint64_t policy)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4, %5}], [%1], %6;" ::"l"(tmap),
+                 "r"(src_smem), "r"(x), "r"(y), "r"(z), "r"(w), "l"(policy)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_group_read()
 {

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_PKG, "liblinattn.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FEATURE_MAP, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 F32, BF16 = 0, 1
 OPT_SPLITS, OPT_PATH, OPT_PROFILE, OPT_FUSE, OPT_LAYOUT, OPT_KERNEL_FUNCTION, OPT_REUSE_STATE = 0, 1, 2, 3, 4, 5, 6
+OPT_WAIT_LIMIT_US, OPT_TEST_UNMET_ARRIVAL = 7, 8
 PHI_HEDGEHOG, PHI_RELU = 0, 1
 LAYOUT_BHND, LAYOUT_BNHD = 0, 1
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
