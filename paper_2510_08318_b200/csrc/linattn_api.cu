@@ -57,8 +57,9 @@ struct linattn_ctx {
     uint32_t* sync_words = nullptr;  // fused kernel: 1 + 2 * max_B * H counters (exit count, two meeting points per (b,h) pair), zero between launches
     size_t sync_bytes = 0;
     // workspace
-    float* partial = nullptr;   // [partial_slots][d*d + d]
+    float* partial = nullptr;   // CUDA-core kernels: [partial_slots][d*d + d]; tensor-core kernels: [partial_slots_tc][128*128 + 128]
     long long partial_slots = 0;
+    long long partial_slots_tc = 0;
     float* state = nullptr;     // [max_B*H][d*d + d]
     unsigned int* err_word = nullptr;
     // workspace of the backward pass, allocated by the first linattn_backward
@@ -307,13 +308,16 @@ long long choose_ctas(const linattn_ctx* c, long long G, long long T)
     return c->num_sms;
 }
 
-// Tensor-core path: bf16, d = 128.
+// Tensor-core path: bf16, d = 128, or d = 64 with the heads taken two at a time (the kernels' kPair variant: a pair of
+// heads is one 128-feature unit of work with block-diagonal weights and state).
 linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B, int n,
                          cudaStream_t st, const void* mix, float mix_r, bool state_only = false)
 {
     using namespace linattn::tc;
     const int Hv = view_heads(c);
-    const long long G = (long long)B * Hv;
+    const int pair = (c->d == 64) ? 1 : 0;
+    const long long heads = (long long)B * Hv;
+    const long long G = pair ? (heads + 1) / 2 : heads;   // units of work
     const long long Tn = ((long long)n + kTile - 1) / kTile;
     const long long T = G * Tn;
     long long Pq = choose_ctas(c, G, T);
@@ -322,14 +326,14 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         Pk = G * c->opt_splits;
         if (Pk > T) Pk = T;
     }
-    if (Pk + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
+    if (Pk + G > c->partial_slots_tc) return LINATTN_ERR_WORKSPACE;
 
     CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmS, tmA;   // tmA: the softmax branch's output (mixed attention), else a copy of tmQ
     const ActStrides as = act_strides(c, n);
     const int layout = c->opt_layout;
     auto act_map = [&](CUtensorMap* m, const void* base, uint32_t box_rows = kTile) {
-        if (layout == 0) return make_tmap_bf16_3d(m, base, kD, (uint64_t)n, (uint64_t)G, box_rows);
-        return make_tmap_bf16_act(m, base, kD, (uint64_t)n, (uint64_t)Hv, (uint64_t)B, (uint64_t)as.token * 2,
+        if (layout == 0) return make_tmap_bf16_3d(m, base, (uint64_t)c->d, (uint64_t)n, (uint64_t)heads, box_rows);
+        return make_tmap_bf16_act(m, base, (uint64_t)c->d, (uint64_t)n, (uint64_t)Hv, (uint64_t)B, (uint64_t)as.token * 2,
                                   (uint64_t)as.head * 2, (uint64_t)as.batch * 2, box_rows);
     };
     // V is fetched in half tiles (the key side's V ring), everything else in whole tiles
@@ -341,31 +345,34 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         snprintf(c->err_text, sizeof(c->err_text), "cuTensorMapEncodeTiled failed");
         return LINATTN_ERR_CUDA;
     }
-    // one instantiation per (mixed attention or not, memory layout)
-#define LA_BY_PHI(K, ...) {(const void*)K<__VA_ARGS__, 0>, (const void*)K<__VA_ARGS__, 1>}
-    const void* k_fused[2][2][2] = {{LA_BY_PHI(linattn_fused_tc, false, 0), LA_BY_PHI(linattn_fused_tc, false, 1)},
-                                    {LA_BY_PHI(linattn_fused_tc, true, 0), LA_BY_PHI(linattn_fused_tc, true, 1)}};
-    const void* k_qside[2][2][2] = {{LA_BY_PHI(qside_tc, false, 0), LA_BY_PHI(qside_tc, false, 1)},
-                                    {LA_BY_PHI(qside_tc, true, 0), LA_BY_PHI(qside_tc, true, 1)}};
-    const void* k_kside[2][2] = {LA_BY_PHI(kside_tc, 0), LA_BY_PHI(kside_tc, 1)};
+    // one instantiation per (mixed attention or not, memory layout, kernel function, heads singly or in pairs)
+#define LA_BY_PAIR(K, ...) {(const void*)K<__VA_ARGS__, 0>, (const void*)K<__VA_ARGS__, 1>}
+#define LA_BY_PHI(K, ...) {LA_BY_PAIR(K, __VA_ARGS__, 0), LA_BY_PAIR(K, __VA_ARGS__, 1)}
+    const void* k_fused[2][2][2][2] = {{LA_BY_PHI(linattn_fused_tc, false, 0), LA_BY_PHI(linattn_fused_tc, false, 1)},
+                                       {LA_BY_PHI(linattn_fused_tc, true, 0), LA_BY_PHI(linattn_fused_tc, true, 1)}};
+    const void* k_qside[2][2][2][2] = {{LA_BY_PHI(qside_tc, false, 0), LA_BY_PHI(qside_tc, false, 1)},
+                                       {LA_BY_PHI(qside_tc, true, 0), LA_BY_PHI(qside_tc, true, 1)}};
+    const void* k_kside[2][2][2] = {LA_BY_PHI(kside_tc, 0), LA_BY_PHI(kside_tc, 1)};
 #undef LA_BY_PHI
+#undef LA_BY_PAIR
     const int phi = c->opt_phi;
     bool& attr_done = c->attr_done[linattn_ctx::kAttrTcFwd];
     if (!attr_done) {
         for (int i = 0; i < 2; ++i)
-            for (int p = 0; p < 2; ++p) {
-                LA_CUDA(c, cudaFuncSetAttribute(k_kside[i][p], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-                for (int j = 0; j < 2; ++j) {
-                    LA_CUDA(c, cudaFuncSetAttribute(k_fused[i][j][p], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-                    LA_CUDA(c, cudaFuncSetAttribute(k_qside[i][j][p], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+            for (int p = 0; p < 2; ++p)
+                for (int pr = 0; pr < 2; ++pr) {
+                    LA_CUDA(c, cudaFuncSetAttribute(k_kside[i][p][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                    for (int j = 0; j < 2; ++j) {
+                        LA_CUDA(c, cudaFuncSetAttribute(k_fused[i][j][p][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                        LA_CUDA(c, cudaFuncSetAttribute(k_qside[i][j][p][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                    }
                 }
-            }
         attr_done = true;
     }
-    const double side_bytes = 2.0 * (double)G * n * kD * 2;
+    const double side_bytes = 2.0 * (double)heads * n * c->d * 2;
     Args a{};
     a.partial = c->partial;
-    a.state = c->state + (size_t)c->view_g0 * kE;
+    a.state = c->state + (size_t)c->view_g0 * ((size_t)c->d * c->d + c->d);   // one record per head (per pair of heads only inside the kernels)
     a.s_img = c->s_img + (size_t)c->view_g0 * kD * kD;
     a.z_img = c->z_img + (size_t)c->view_g0 * (kZBlkBytes / 2);
     a.err = c->err_word;
@@ -378,6 +385,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.n = n;
     a.H = Hv;
     a.G = (int)G;
+    a.heads_total = (int)heads;
     a.tiles_per_head = (int)Tn;
     a.total_tiles = T;
 #ifdef LINATTN_TRACE
@@ -391,7 +399,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         // counters are zero between launches (the kernel clears them on its way out), so nothing here depends on
         // earlier launches and the launch may be recorded in a CUDA graph.
         void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
-        const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout][phi], dim3((unsigned)Pq), dim3(kThreads),
+        const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout][phi][pair], dim3((unsigned)Pq), dim3(kThreads),
                                                            params, Smem::kTotal, st);
         if (le == cudaSuccess) {
             prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
@@ -406,11 +414,12 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     }
     {
         void* kp[] = {&tmK, &tmV, &tmWk, &a};
-        LA_CUDA(c, cudaLaunchKernel(k_kside[layout][phi], dim3((unsigned)Pk), dim3(kThreads), kp, Smem::kTotal, st));
+        LA_CUDA(c, cudaLaunchKernel(k_kside[layout][phi][pair], dim3((unsigned)Pk), dim3(kThreads), kp, Smem::kTotal, st));
     }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_tc", side_bytes);
-    combine_tc<<<dim3((kE / 4 + 255) / 256, (unsigned)G), 256, 0, st>>>(a, Pk);
+    if (pair) combine_tc<1><<<dim3((kE / 4 + 255) / 256, (unsigned)G), 256, 0, st>>>(a, Pk);
+    else combine_tc<0><<<dim3((kE / 4 + 255) / 256, (unsigned)G), 256, 0, st>>>(a, Pk);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_tc", 0.0);
     if (state_only) {   // the backward pass wants S and z only
@@ -419,7 +428,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     }
     {
         void* qp[] = {&tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
-        LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout][phi], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
+        LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout][phi][pair], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
     }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);
@@ -437,7 +446,7 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     const long long Tn = ((long long)n + kTile - 1) / kTile;
     const long long T = G * Tn;
     const long long P = c->num_sms < T ? c->num_sms : T;   // these kernels are bound by per-tile latency, not bandwidth: every SM counts
-    if (P + G > c->partial_slots) return LINATTN_ERR_WORKSPACE;
+    if (P + G > c->partial_slots_tc) return LINATTN_ERR_WORKSPACE;
     // forward state (S as [c][f], z) and the hi image of S: left by the forward that just ran on these k, v (if the
     // caller allows it), else recomputed; q and out are not touched by the first two kernels of the forward
     const linattn_ctx::StateKey& sk = c->state_key;
@@ -588,17 +597,23 @@ linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, l
     const size_t E = (size_t)d * d + d;
     const size_t wbytes = sizeof(float) * (size_t)H * d * (d / 2);
     const long long G = max_B * H;
+    // The tensor-core kernels work on 128-feature units (one head of dimension 128, or a pair of heads of dimension 64:
+    // at most G units either way) with records of 128 * 128 + 128 floats, one per persistent CTA and unit it touches.
     c->partial_slots = kTargetCtas + G;
+    c->partial_slots_tc = kTargetCtas + G;
+    const size_t simt_bytes = sizeof(float) * E * (size_t)c->partial_slots;
+    const size_t tc_bytes = sizeof(float) * (size_t)linattn::tc::kE * (size_t)c->partial_slots_tc;
     cudaError_t e = cudaSuccess;
     if (e == cudaSuccess) e = cudaMalloc(&c->Wq, wbytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->Wk, wbytes);
-    if (e == cudaSuccess) e = cudaMalloc(&c->partial, sizeof(float) * E * (size_t)c->partial_slots);
+    if (e == cudaSuccess) e = cudaMalloc(&c->partial, simt_bytes > tc_bytes ? simt_bytes : tc_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&c->state, sizeof(float) * E * (size_t)G);
-    if (e == cudaSuccess && d == 128) {
-        const size_t wt = sizeof(__nv_bfloat16) * (size_t)H * d * (d / 2);
+    if (e == cudaSuccess) {
+        // weight images W^T [H][64][128] bf16 (d = 64: of each pair of consecutive heads), bf16 image of S and operand image of z per unit
+        const size_t wt = sizeof(__nv_bfloat16) * (size_t)H * linattn::tc::kM * linattn::tc::kD;
         e = cudaMalloc(&c->Wqt, wt);
         if (e == cudaSuccess) e = cudaMalloc(&c->Wkt, wt);
-        if (e == cudaSuccess) e = cudaMalloc(&c->s_img, sizeof(__nv_bfloat16) * (size_t)G * d * d);
+        if (e == cudaSuccess) e = cudaMalloc(&c->s_img, sizeof(__nv_bfloat16) * (size_t)G * linattn::tc::kD * linattn::tc::kD);
         if (e == cudaSuccess) e = cudaMalloc(&c->z_img, (size_t)G * linattn::tc::kZBlkBytes);
         if (e == cudaSuccess) e = cudaMemset(c->z_img, 0, (size_t)G * linattn::tc::kZBlkBytes);
     }
@@ -671,6 +686,16 @@ linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const voi
         convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wq, c->H, DM, per_head ? 1 : 0);
         convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wk, c->H, DM, per_head ? 1 : 0);
     }
+    if (c->d == 64) {
+        const unsigned tb = (unsigned)(((size_t)c->H * tc::kM * tc::kD + 255) / 256);
+        if (wdtype == LINATTN_F32) {
+            tc::pair_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
+            tc::pair_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
+        } else {
+            tc::pair_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
+            tc::pair_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
+        }
+    }
     if (c->d == 128) {
         const unsigned tb = (unsigned)(((size_t)c->H * DM + 255) / 256);
         if (wdtype == LINATTN_F32) {
@@ -711,19 +736,19 @@ static linattn_status forward_impl(linattn_ctx* c, const void* q, const void* k,
     return dispatch_forward(c, q, k, v, out, mix, mix_r, B, n, d, dtype, (cudaStream_t)stream);
 }
 
-// Choice of kernels for checked arguments.  The tensor-core kernels cover bf16 activations with head dimension 128
-// and bf16 feature-map weights; everything else runs on the CUDA-core kernels.
+// Choice of kernels for checked arguments.  The tensor-core kernels cover bf16 activations with bf16 feature-map
+// weights (head dimension 128, or 64 with the heads taken in pairs); everything else runs on the CUDA-core kernels.
 static linattn_status dispatch_forward(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, const void* mix,
                                        float mix_r, int B, int n, int d, linattn_dtype dtype, cudaStream_t st)
 {
-    const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && (c->map_is_bf16 || c->opt_phi == 1));
+    const bool tc_ok = (dtype == LINATTN_BF16 && (c->map_is_bf16 || c->opt_phi == 1));   // d = 128, or d = 64 with the heads in pairs
     if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
     c->last_B = B;
     c->state_transposed = tc_ok && c->opt_path != 1;
     c->state_key.valid = false;
     if (c->state_transposed) {
         const linattn_status s = launch_tc(c, q, k, v, out, B, n, st, mix, mix_r);
-        if (s == LINATTN_OK && c->opt_phi == 0 && c->view_H == 0) c->state_key = {k, v, B, n, c->opt_layout, true};
+        if (s == LINATTN_OK && c->opt_phi == 0 && c->view_H == 0 && d == 128) c->state_key = {k, v, B, n, c->opt_layout, true};
         return s;
     }
     if (dtype == LINATTN_BF16) {

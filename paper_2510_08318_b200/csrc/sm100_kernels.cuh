@@ -250,6 +250,58 @@ __device__ __forceinline__ void softmax_half_to_smem(float (&u)[kM], float keep,
     }
 }
 
+// The same for a PAIR of heads of dimension 64: u[0..31] are the token's logits under the first head's W, u[32..63]
+// under the second head's.  Each group of 32 gets its own softmax.  Head b's feature vector, [softmax(+u_b),
+// softmax(-u_b)], occupies block b of the tile (64 features): this thread's 32 values go to chunks 4 * kNeg .. 4 * kNeg + 3
+// of the token's row in block b.  `tile_row` = start of the token's row in block 0; block 1 is kHalfTileBytes further.
+template <bool kNeg>
+__device__ __forceinline__ void softmax_pair_to_smem(float (&u)[kM], float keep0, float keep1, uint8_t* tile_row, int row)
+{
+    const int sw = row & 7;
+#pragma unroll
+    for (int b = 0; b < 2; ++b) {
+        const int o = 32 * b;
+        float m = kNeg ? min3(u[o], u[o + 1], u[o + 2]) : max3(u[o], u[o + 1], u[o + 2]);
+#pragma unroll
+        for (int j = 3; j < 31; j += 2) m = kNeg ? min3(m, u[o + j], u[o + j + 1]) : max3(m, u[o + j], u[o + j + 1]);
+        m = kNeg ? fminf(m, u[o + 31]) : fmaxf(m, u[o + 31]);
+        const float sL = kNeg ? -kLog2e : kLog2e;
+        const float off = kNeg ? m * kLog2e : -m * kLog2e;
+        const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
+        f32x2 e[16];
+        f32x2 sum2 = pack2(0.f, 0.f);
+#pragma unroll
+        for (int p = 0; p < 16; ++p) {
+            const f32x2 x = fma2(pack2(u[o + 2 * p], u[o + 2 * p + 1]), scale, offset);
+            if ((p & 3) == 3) {
+                e[p] = exp2_poly2(x);
+            } else {
+                float x0, x1;
+                unpack2(x, x0, x1);
+                e[p] = pack2(ex2_approx(x0), ex2_approx(x1));
+            }
+            sum2 = add2(sum2, e[p]);
+        }
+        float s0, s1;
+        unpack2(sum2, s0, s1);
+        const float inv = __fdividef(b == 0 ? keep0 : keep1, s0 + s1);
+        const f32x2 inv2 = pack2(inv, inv);
+        uint8_t* dst = tile_row + b * kHalfTileBytes;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float x, y;
+                unpack2(mul2(e[4 * cc + q], inv2), x, y);
+                w[q] = pack_bf16(x, y);
+            }
+            const int chunk = (kNeg ? 4 : 0) + cc;
+            *reinterpret_cast<uint4*>(dst + ((chunk ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
 // Read this thread's 64 logits (its TMEM lane, columns [col, col+64)).
 __device__ __forceinline__ void load_logits(uint32_t taddr, float (&u)[kM])
 {
@@ -374,7 +426,8 @@ struct Args {
     const __nv_bfloat16* mix_src;  // Eq. 8: output of the softmax-attention branch [G][n][128], or nullptr (plain Eq. 5)
     float mix_r;                 // Eq. 8: the score r, already clipped into [0, 1]
     long long str_token, str_head, str_batch;  // element strides of q, k, v, out (and mix_src) between tokens, heads, batches
-    int n, H, G;
+    int n, H, G;                 // tokens; heads per batch entry (H); units of work: (b,h) pairs, or pairs of heads when d = 64
+    int heads_total;             // B * H
     int tiles_per_head;
     long long total_tiles;
 #ifdef LINATTN_TRACE
@@ -468,6 +521,33 @@ __device__ __forceinline__ void act_prefetch_l2(const void* tm, int x, int t, in
     else tma_prefetch_l2_4d(tm, x, t, g % H, g / H);
 }
 
+// Where the two 64-feature blocks of a 128-token tile come from.
+//   kPair = 0 (head dimension 128): features [0, 64) and [64, 128) of (b,h) pair g.
+//   kPair = 1 (head dimension 64): the 64 features of heads 2g and 2g + 1, taken over the flattened (batch, head)
+//   index: a PAIR of heads is processed as one 128-feature problem whose weight matrix, state S and normaliser z are
+//   block-diagonal (the combine step zeroes the off-diagonal blocks of S, the z operand has one hi+lo column pair per
+//   head), so every tensor-core shape, the shared-memory layout and the pipelines are those of d = 128.  If the number
+//   of heads in all is odd, the last pair's second head does not exist: its loads start past the end of the tensor
+//   (TMA fills zeros), its phi is forced to zero on the key side and its output block is not stored.
+template <int kLayout, int kPair> struct Blocks {
+    static __device__ __forceinline__ int head(int g, int blk) { return kPair ? 2 * g + blk : g; }
+    static __device__ __forceinline__ int x(int blk) { return kPair ? 0 : 64 * blk; }
+    static __device__ __forceinline__ void load(uint32_t dst, const void* tm, uint32_t bar, int blk, int t, int g, int H)
+    {
+        act_load<kLayout>(dst, tm, bar, x(blk), t, head(g, blk), H);
+    }
+    static __device__ __forceinline__ void store(const void* tm, uint32_t src, int blk, int t, int g, int H, uint64_t policy)
+    {
+        act_store<kLayout>(tm, src, x(blk), t, head(g, blk), H, policy);
+    }
+    static __device__ __forceinline__ void prefetch_l2(const void* tm, int blk, int t, int g, int H)
+    {
+        act_prefetch_l2<kLayout>(tm, x(blk), t, head(g, blk), H);
+    }
+    // which weight matrix (plane of the W^T tensor map) goes with (b,h) pair / pair of heads g
+    static __device__ __forceinline__ int weights(int g, int H) { return (kPair ? 2 * g : g) % H; }
+};
+
 // ReLU kernel function, phi(x) = max(x, 0) element by element: applied in place to a 128 x 128 bf16 tile exactly as
 // TMA left it in shared memory (element-wise, so the swizzled operand layout is kept); 256 threads, 128 bytes each.
 // Rows past the end of the sequence were zero-filled by TMA and stay zero.
@@ -535,7 +615,7 @@ __device__ __forceinline__ void raise_abort(const WaitCtx& wc, uint32_t code)
 // kPhi: 0 = the Hedgehog feature map of Eq. 6; 1 = the ReLU kernel function (no projection, no softmax: the logits
 // warp idles and warps 0-7 rectify the K tile in place).
 // arrive: fused kernel; every partial record written is announced at its head's first meeting point.
-template <int kLayout, int kPhi>
+template <int kLayout, int kPhi, int kPair>
 __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const CUtensorMap* tmK, const CUtensorMap* tmV,
                                             const CUtensorMap* tmW, bool arrive)
 {
@@ -568,8 +648,8 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
                 mbar_arrive_expect_tx(c.bar(K_VFULL + vr.s), kHalfTileBytes);
                 const uint32_t vdst = sbase + Smem::kKV + vr.s * kHalfTileBytes;
                 const int row = wv.lt * kTile + (issued_v & 1) * (kTile / 2);
-                act_load<kLayout>(vdst, tmV, c.bar(K_VFULL + vr.s), 0, row, wv.g, a.H);
-                act_load<kLayout>(vdst + kHalfTileBytes / 2, tmV, c.bar(K_VFULL + vr.s), 64, row, wv.g, a.H);
+                Blocks<kLayout, kPair>::load(vdst, tmV, c.bar(K_VFULL + vr.s), 0, row, wv.g, a.H);
+                Blocks<kLayout, kPair>::load(vdst + kHalfTileBytes / 2, tmV, c.bar(K_VFULL + vr.s), 1, row, wv.g, a.H);
             }
             if (issued_v & 1) wv.next();
             ++issued_v;
@@ -581,8 +661,8 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             if (lane == 0) {
                 mbar_arrive_expect_tx(c.bar(K_FULL + r.s), kTileBytes);
                 const uint32_t kdst = sbase + r.s * kTileBytes;
-                act_load<kLayout>(kdst, tmK, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
-                act_load<kLayout>(kdst + kHalfTileBytes, tmK, c.bar(K_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
+                Blocks<kLayout, kPair>::load(kdst, tmK, c.bar(K_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                Blocks<kLayout, kPair>::load(kdst + kHalfTileBytes, tmK, c.bar(K_FULL + r.s), 1, w.lt * kTile, w.g, a.H);
             }
             issued = w.i + 1;
             if (w.i >= kVLag) {
@@ -610,8 +690,8 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
                 if (w.seg >= 1 && !warp_wait(c.bar(K_WFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrMmaLoad)) break;
                 if (lane == 0) {
                     mbar_arrive_expect_tx(c.bar(K_WFULL), kWBytes);
-                    tma_load_3d(sbase + Smem::kKW, tmW, c.bar(K_WFULL), 0, 0, w.g % a.H);
-                    tma_load_3d(sbase + Smem::kKW + kWBytes / 2, tmW, c.bar(K_WFULL), 64, 0, w.g % a.H);
+                    tma_load_3d(sbase + Smem::kKW, tmW, c.bar(K_WFULL), 0, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
+                    tma_load_3d(sbase + Smem::kKW + kWBytes / 2, tmW, c.bar(K_WFULL), 64, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
                 }
                 if (!warp_wait(c.bar(K_WFULL), (uint32_t)w.seg & 1u, c.wc, kErrMmaLoad)) break;
             }
@@ -696,9 +776,16 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             if (lane == 0) mbar_arrive(c.bar(K_UEMPTY + ur.s));
             if ((warp & 3) == 0) LA_TRACE(2 + half, w.i, 1);
             const float keep = (w.lt * kTile + row < a.n) ? 1.f : 0.f;
-            uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
-            if (half == 0) softmax_half_to_smem<false>(u, keep, dst, row);
-            else softmax_half_to_smem<true>(u, keep, dst, row);
+            if (kPair) {
+                const float keep1 = (2 * w.g + 1 < a.heads_total) ? keep : 0.f;   // a last pair without a second head
+                uint8_t* tile_row = c.smem + r.s * kTileBytes + row * 128;
+                if (half == 0) softmax_pair_to_smem<false>(u, keep, keep1, tile_row, row);
+                else softmax_pair_to_smem<true>(u, keep, keep1, tile_row, row);
+            } else {
+                uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                if (half == 0) softmax_half_to_smem<false>(u, keep, dst, row);
+                else softmax_half_to_smem<true>(u, keep, dst, row);
+            }
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(c.bar(K_PHIFULL + r.s));
@@ -746,6 +833,11 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
 // Four consecutive elements (e4 .. e4+3, e4 a multiple of 4) of head g's record: sum the partials of the
 // CTAs that touched the head in ascending CTA index (so the result does not depend on timing), store the
 // fp32 state and the bf16 operand images.  All loads of a batch are issued before the first add.
+// kPair (head dimension 64, two heads per record): the record's off-diagonal blocks (one head's features against the
+// other head's columns) are dropped: zero in the bf16 image, so that the query side's product does not mix the heads;
+// the fp32 state goes to the two heads' own records ([c][f] of 64 x 64, then z) and the z operand gets one hi+lo pair
+// of rows per head (rows 0, 1: first head, features 0-63; rows 2, 3: second head, features 64-127; all else stays zero).
+template <int kPair>
 __device__ __forceinline__ void combine_quad(const Args& a, long long P, int g, int e4)
 {
     const long long c0 = tile_owner((long long)g * a.tiles_per_head, a.total_tiles, P);
@@ -769,15 +861,20 @@ __device__ __forceinline__ void combine_quad(const Args& a, long long P, int g, 
             }
         }
     }
-    *reinterpret_cast<float4*>(a.state + (size_t)g * kE + e4) = acc;
+    constexpr int kEh = 64 * 64 + 64;   // floats per head's state record when d = 64
+    if (!kPair) *reinterpret_cast<float4*>(a.state + (size_t)g * kE + e4) = acc;
     const float r[4] = {acc.x, acc.y, acc.z, acc.w};
     if (e4 < kD * kD) {
+        const int cc = e4 / kD, f0 = e4 % kD;   // column of V, first of the four features
+        const bool keep = !kPair || (cc >> 6) == (f0 >> 6);
         uint2 packed;
-        packed.x = pack_bf16(r[0], r[1]);
-        packed.y = pack_bf16(r[2], r[3]);
+        packed.x = keep ? pack_bf16(r[0], r[1]) : 0u;
+        packed.y = keep ? pack_bf16(r[2], r[3]) : 0u;
         *reinterpret_cast<uint2*>(a.s_img + (size_t)g * kD * kD + e4) = packed;
+        if (kPair && keep && 2 * g + (cc >> 6) < a.heads_total)
+            *reinterpret_cast<float4*>(a.state + (size_t)(2 * g + (cc >> 6)) * kEh + (cc & 63) * 64 + (f0 & 63)) = acc;
     } else {
-        // z[f]: hi and lo bf16 parts into rows 0 and 1 of the K-major operand block of feature block f / 64
+        // z[f]: hi and lo bf16 parts into two rows of the K-major operand block of feature block f / 64
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
             const int f = e4 - kD * kD + t;
@@ -785,8 +882,10 @@ __device__ __forceinline__ void combine_quad(const Args& a, long long P, int g, 
             const __nv_bfloat16 lo = __float2bfloat16_rn(r[t] - __bfloat162float(hi));
             __nv_bfloat16* blk = a.z_img + (size_t)g * (kZBlkBytes / 2) + (f >> 6) * (16 * 64);
             const int fi = f & 63, chunk = fi >> 3, within = fi & 7;
-            blk[0 * 64 + ((chunk ^ 0) << 3) + within] = hi;  // row 0: swizzle term (row & 7) = 0
-            blk[1 * 64 + ((chunk ^ 1) << 3) + within] = lo;  // row 1: swizzle term 1
+            const int row = kPair ? 2 * (f >> 6) : 0;   // rows (row, row + 1); the swizzle term of a row below 8 is the row itself
+            blk[row * 64 + ((chunk ^ row) << 3) + within] = hi;
+            blk[(row + 1) * 64 + ((chunk ^ (row + 1)) << 3) + within] = lo;
+            if (kPair && 2 * g + (f >> 6) < a.heads_total) a.state[(size_t)(2 * g + (f >> 6)) * kEh + 64 * 64 + fi] = r[t];
         }
     }
 }
@@ -804,7 +903,7 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
 
 // wait_state: the S and z images are produced earlier in the same kernel (fused path); loads of them
 // must wait at the head's second meeting point.  Otherwise they were written by a previous launch.
-template <bool kMix, int kLayout, int kPhi>
+template <bool kMix, int kLayout, int kPhi, int kPair>
 __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
                                             const CUtensorMap* tmW, const CUtensorMap* tmS, const CUtensorMap* tmA, bool wait_state)
 {
@@ -861,8 +960,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 if (w.seg >= 1 && !warp_wait(c.bar(Q_SEGFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrSeg)) break;
                 if (kPhi == 0 && lane == 0) {
                     mbar_arrive_expect_tx(c.bar(Q_WFULL), kWBytes);
-                    tma_load_3d(sbase + Smem::kQW, tmW, c.bar(Q_WFULL), 0, 0, w.g % a.H);
-                    tma_load_3d(sbase + Smem::kQW + kWBytes / 2, tmW, c.bar(Q_WFULL), 64, 0, w.g % a.H);
+                    tma_load_3d(sbase + Smem::kQW, tmW, c.bar(Q_WFULL), 0, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
+                    tma_load_3d(sbase + Smem::kQW + kWBytes / 2, tmW, c.bar(Q_WFULL), 64, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
                 }
                 state_g = w.g;
                 // the first head's state may not exist yet: get the first Q tiles moving before waiting for it
@@ -887,8 +986,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                         if (passed) {
                             TileWalk pw = w;
                             for (int j = 0; j < kQPrefetchL2 && !pw.done(); ++j, pw.next()) {
-                                act_prefetch_l2<kLayout>(tmQ, 0, pw.lt * kTile, pw.g, a.H);
-                                act_prefetch_l2<kLayout>(tmQ, 64, pw.lt * kTile, pw.g, a.H);
+                                Blocks<kLayout, kPair>::prefetch_l2(tmQ, 0, pw.lt * kTile, pw.g, a.H);
+                                Blocks<kLayout, kPair>::prefetch_l2(tmQ, 1, pw.lt * kTile, pw.g, a.H);
                             }
                         }
                     }
@@ -901,18 +1000,21 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             LA_TRACE(0, 24 + w.i, 0);
             if (lane == 0) {
                 mbar_arrive_expect_tx(c.bar(Q_FULL + r.s), kTileBytes);
-                act_load<kLayout>(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
-                act_load<kLayout>(sbase + r.s * kTileBytes + kHalfTileBytes, tmQ, c.bar(Q_FULL + r.s), 64, w.lt * kTile, w.g, a.H);
+                Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes, tmQ, c.bar(Q_FULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes + kHalfTileBytes, tmQ, c.bar(Q_FULL + r.s), 1, w.lt * kTile, w.g, a.H);
             }
             if (kMix) {
                 // Eq. 8: the epilogue will read this tile's rows of the softmax branch's output straight from
                 // global memory a few microseconds from now; start them on their way into L2 (the rows of a tile
                 // are contiguous: 256 lines of 128 bytes, fewer in the ragged tail tile)
                 const int rows = min(kTile, a.n - w.lt * kTile);
-                const __nv_bfloat16* base = a.mix_src + (size_t)(w.g / a.H) * a.str_batch + (size_t)(w.g % a.H) * a.str_head +
-                                            (size_t)w.lt * kTile * a.str_token;
-                for (int line = lane; line < rows * 2; line += 32)   // two 128-byte lines per row of 128 bf16
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (size_t)(line >> 1) * a.str_token + (line & 1) * 64));
+                for (int line = lane; line < rows * 2; line += 32) {   // two 128-byte lines per row of the tile (one per block)
+                    const int blk = line & 1, hd = Blocks<kLayout, kPair>::head(w.g, blk);
+                    if (kPair && hd >= a.heads_total) continue;
+                    const __nv_bfloat16* p = a.mix_src + (size_t)(hd / a.H) * a.str_batch + (size_t)(hd % a.H) * a.str_head +
+                                             ((size_t)w.lt * kTile + (line >> 1)) * a.str_token + Blocks<kLayout, kPair>::x(blk);
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+                }
             }
             issued = w.i + 1;
         }
@@ -985,8 +1087,9 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(Q_OFULL + r.s), r.ph, c.wc, kErrStore)) break;
             if (lane == 0) {
-                act_store<kLayout>(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g, a.H, keep);
-                act_store<kLayout>(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 64, w.lt * kTile, w.g, a.H, keep);
+                Blocks<kLayout, kPair>::store(tmO, sbase + r.s * kTileBytes, 0, w.lt * kTile, w.g, a.H, keep);
+                if (!kPair || 2 * w.g + 1 < a.heads_total)   // an odd number of heads in all: the last pair has no second head
+                    Blocks<kLayout, kPair>::store(tmO, sbase + r.s * kTileBytes + kHalfTileBytes, 1, w.lt * kTile, w.g, a.H, keep);
                 bulk_commit_group();
                 bulk_wait_group_read<0>();
                 mbar_arrive(c.bar(Q_EMPTY + r.s));
@@ -1021,9 +1124,15 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(c.bar(Q_UEMPTY + ur.s));
-            uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
-            if (half == 0) softmax_half_to_smem<false>(u, 1.f, dst, row);
-            else softmax_half_to_smem<true>(u, 1.f, dst, row);
+            if (kPair) {
+                uint8_t* tile_row = c.smem + r.s * kTileBytes + row * 128;
+                if (half == 0) softmax_pair_to_smem<false>(u, 1.f, 1.f, tile_row, row);
+                else softmax_pair_to_smem<true>(u, 1.f, 1.f, tile_row, row);
+            } else {
+                uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                if (half == 0) softmax_half_to_smem<false>(u, 1.f, dst, row);
+                else softmax_half_to_smem<true>(u, 1.f, dst, row);
+            }
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(c.bar(Q_PHIFULL + r.s));
@@ -1040,8 +1149,10 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             if (!warp_wait(c.bar(Q_DFULL + dr.s), dr.ph, c.wc, kErrEpilogue)) break;
             if (warp == 12) LA_TRACE(3, 24 + w.i, 0);
             tcgen05_fence_after();
-            uint32_t dv[2];
+            // columns of the denominator operand: d = 128: [z_hi, z_lo]; paired heads: [z_hi, z_lo] of the first head, then of the second
+            uint32_t dv[4];
             tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
+            if (kPair) tmem_ld_x2(tmem_den(dr.s) + lane_base + 2, dv + 2);
             constexpr bool mix = kMix;   // compile-time: the plain forward carries none of the blend's code
             if (mix) {
                 // Eq. 8 (mixed attention): the tensor core is done with phi(q) in this slot (that is what the barrier
@@ -1049,8 +1160,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 // (its lines are already on their way into L2), blended in place and stored from there.
                 if (warp == 12 && lane == 0) {
                     mbar_arrive_expect_tx(c.bar(Q_AFULL + r.s), kTileBytes);
-                    act_load<kLayout>(sbase + r.s * kTileBytes, tmA, c.bar(Q_AFULL + r.s), 0, w.lt * kTile, w.g, a.H);
-                    act_load<kLayout>(sbase + r.s * kTileBytes + kHalfTileBytes, tmA, c.bar(Q_AFULL + r.s), 64, w.lt * kTile, w.g, a.H);
+                    Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes, tmA, c.bar(Q_AFULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                    Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes + kHalfTileBytes, tmA, c.bar(Q_AFULL + r.s), 1, w.lt * kTile, w.g, a.H);
                 }
                 if (!warp_wait(c.bar(Q_AFULL + r.s), r.ph, c.wc, kErrEpilogue)) break;
             }
@@ -1066,7 +1177,8 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                     __syncwarp();
                     if (lane == 0) mbar_arrive(c.bar(Q_DEMPTY + dr.s));
                 }
-                const float inv = __fdividef(1.f, __uint_as_float(dv[0]) + __uint_as_float(dv[1]));
+                const int dsel = kPair ? 2 * half : 0;   // paired heads: output block `half` belongs to head `half` of the pair
+                const float inv = __fdividef(1.f, __uint_as_float(dv[dsel]) + __uint_as_float(dv[dsel + 1]));
                 uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
                 if (!mix) {
                     const f32x2 inv2 = pack2(inv, inv);
@@ -1114,25 +1226,26 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
 // Kernels
 // ======================================================================================================
 
-template <int kLayout, int kPhi>
+template <int kLayout, int kPhi, int kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
          const __grid_constant__ CUtensorMap tmW, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, true, false);
-    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmW, false);
+    kside_phase<kLayout, kPhi, kPair>(c, a, &tmK, &tmV, &tmW, false);
     cta_teardown(c);
 }
 
 // grid = (ceil(kE / 4 / 256), G)
-static __global__ void __launch_bounds__(256) combine_tc(const Args a, long long P)
+template <int kPair>
+__global__ void __launch_bounds__(256) combine_tc(const Args a, long long P)
 {
     const int q4 = blockIdx.x * 256 + threadIdx.x;
-    if (q4 < kE / 4) combine_quad(a, P, blockIdx.y, q4 * 4);
+    if (q4 < kE / 4) combine_quad<kPair>(a, P, blockIdx.y, q4 * 4);
 }
 
-template <bool kMix, int kLayout, int kPhi>
+template <bool kMix, int kLayout, int kPhi, int kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
          const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS,
@@ -1140,12 +1253,12 @@ qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtens
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, false, true);
-    qside_phase<kMix, kLayout, kPhi>(c, a, &tmQ, &tmO, &tmW, &tmS, &tmA, false);
+    qside_phase<kMix, kLayout, kPhi, kPair>(c, a, &tmQ, &tmO, &tmW, &tmS, &tmA, false);
     cta_teardown(c);
 }
 
 // The whole forward in one cooperative launch of P <= #SMs persistent CTAs.
-template <bool kMix, int kLayout, int kPhi>
+template <bool kMix, int kLayout, int kPhi, int kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmQ,
@@ -1156,7 +1269,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     LA_TRACE_NS(0, 60, 0);
     const Cta c = cta_setup(smem_raw, a, true, true);
     LA_TRACE_NS(0, 60, 1);
-    kside_phase<kLayout, kPhi>(c, a, &tmK, &tmV, &tmWk, true);
+    kside_phase<kLayout, kPhi, kPair>(c, a, &tmK, &tmV, &tmWk, true);
     // every role is done with the key-side buffers; the partials of this CTA are written and announced
     tcgen05_fence_before();
     __syncthreads();
@@ -1187,7 +1300,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (ok) {
                 const int j = (int)blockIdx.x - c0;
                 const int lo = j * (kE / 4) / cnt, hi = (j + 1) * (kE / 4) / cnt;   // this CTA's share: float4 groups [lo, hi)
-                for (int x = lo + it; x < hi; x += kHoleThreads) combine_quad(a, P, g, x * 4);
+                for (int x = lo + it; x < hi; x += kHoleThreads) combine_quad<kPair>(a, P, g, x * 4);
             }
             named_barrier_sync(1, kHoleThreads);   // the share is written (and `met` has been read by everybody)
             if (it == 0 && ok) meet_arrive(a.sync + 2 + 2 * g);
@@ -1196,7 +1309,7 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
-    qside_phase<kMix, kLayout, kPhi>(c, a, &tmQ, &tmO, &tmWq, &tmS, &tmA, true);
+    qside_phase<kMix, kLayout, kPhi, kPair>(c, a, &tmQ, &tmO, &tmWq, &tmS, &tmA, true);
     LA_TRACE_NS(0, 61, 2);
     cta_teardown(c);
     LA_TRACE_NS(0, 61, 3);
@@ -1211,6 +1324,27 @@ static __global__ void transpose_weights_bf16(const T* __restrict__ src, __nv_bf
     const int h = (int)(i / (kM * kD)), rem = (int)(i % (kM * kD)), j = rem / kD, dd = rem % kD;
     const size_t s = (size_t)(per_head ? h : 0) * kD * kM + (size_t)dd * kM + j;
     dst[i] = __float2bfloat16_rn((float)src[s]);
+}
+
+// Head dimension 64: the weight image of a PAIR of heads, as the logits MMA of the d = 128 kernels wants it.
+// dst [H][64 j'][128 d'] bf16, plane h0 for the pair (h0, h1 = (h0 + 1) mod H):
+//   rows  0..31: W_{h0}^T (32 x 64) in columns 0..63,   zeros in columns 64..127
+//   rows 32..63: zeros in columns 0..63,                W_{h1}^T in columns 64..127
+// so that [x_{h0}, x_{h1}] (128 features) times its transpose gives [u_{h0} (32 logits), u_{h1} (32 logits)].
+// src: W [H][64 d][32 j] (any supported type); per_head == 0: one matrix for every head.
+template <typename T>
+static __global__ void pair_weights_bf16(const T* __restrict__ src, __nv_bfloat16* __restrict__ dst, int H, int per_head)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)H * kM * kD) return;
+    const int h0 = (int)(i / (kM * kD)), rem = (int)(i % (kM * kD)), jp = rem / kD, dp = rem % kD;
+    const int blk = jp >> 5;   // which head of the pair this row of logits belongs to
+    float v = 0.f;
+    if ((dp >> 6) == blk) {
+        const int h = per_head ? (h0 + blk) % H : 0;
+        v = (float)src[(size_t)h * 64 * 32 + (size_t)(dp & 63) * 32 + (jp & 31)];
+    }
+    dst[i] = __float2bfloat16_rn(v);
 }
 
 }  // namespace tc

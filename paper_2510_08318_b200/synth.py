@@ -15,6 +15,9 @@ the paper, so these stand in for them:
                                           Student-t(3)/sqrt(d) (heavy tails)
   config 4  B=1 H=40 n=75600 d=128 bf16  as 2
   config 5  B=2 H=12 n=32760 d=128 bf16  as 2, 30 independent layers
+  config 6  B=1 H=30 n=17776 d=64  bf16  as 2: the shape of CogVideoX-2B's joint text + video self-attention
+                                          (30 heads of 64; 226 text tokens + 13 x 30 x 45 video tokens for 49 frames
+                                          of 480 x 720); the paper names the model but prints none of its dimensions
 
 W_q and W_k are drawn per head as N(0,1) / (sqrt(d) * sigma_x), sigma_x being the
 standard deviation of the inputs, so that the logits x W have unit variance: phi
@@ -51,6 +54,7 @@ CONFIGS = {
     3: Workload("wan14b-480p-heavytail", 1, 40, 32760, 128, "bf16", False, True),
     4: Workload("wan14b-720p", 1, 40, 75600, 128, "bf16", False, False),
     5: Workload("wan1.3b-cfg-pair-30-layers", 2, 12, 32760, 128, "bf16", False, False, 30),
+    6: Workload("cogvideox2b-480x720-49f", 1, 30, 17776, 64, "bf16", False, False),
 }
 
 
