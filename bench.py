@@ -65,14 +65,28 @@ def recorded_traffic(kernel):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples the SM clock and the clock-event (throttle) reasons while the benchmark runs: NVML polled from a thread
+    as fast as it answers (a few hundred microseconds per sample, so that even a timed region of a millisecond or two
+    gets samples of its own), with `nvidia-smi -lms 50` as the fallback when the NVML binding is missing.  Read-only."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    BITS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.nvml, self.stop_flag = index, [], None, None, False
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50"],
@@ -82,21 +96,41 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
+    def _poll(self):
+        n = self.nvml
+        while not self.stop_flag:
+            try:
+                t = time.time()
+                mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                bits = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                self.rows.append((t, mhz, bits))
+                time.sleep(0.0002)   # leave the interpreter to the thread that launches the kernels
+            except Exception:
+                break
+
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            f = [c.strip() for c in line.split(",")]
+            if len(f) >= 6 and f[0].replace(".", "").isdigit():
+                bits = sum(b for (nm, b), col in zip(self.BITS.items(), f[2:6]) if col == "Active")
+                self.max_mhz = float(f[1]) if f[1].replace(".", "").isdigit() else None
+                self.rows.append((time.time(), float(f[0]), bits))
 
-    def stop(self):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
+    def stop(self, t0=None, t1=None):
+        """Statistics over the samples taken inside [t0, t1] (the timed region) when there are any, else over all."""
+        if self.nvml is None and not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no NVML binding and no nvidia-smi"], "samples": 0}
+        self.stop_flag = True
+        if self.proc:
+            self.proc.terminate()
         self.thread.join(timeout=2)
-        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [nm for i, nm in enumerate(names) if any(len(r) >= 6 and r[2 + i] == "Active" for r in self.rows)]
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm)}
+        rows = list(self.rows)
+        inside = [r for r in rows if t0 is not None and t0 <= r[0] <= t1]
+        use, where = (inside, "timed region") if inside else (rows, "whole run of the benchmark's GPU passes")
+        reasons = [nm for nm, b in self.BITS.items() if any(r[2] & b for r in use)]
+        return {"sm_mhz": statistics.median(r[1] for r in use) if use else None, "sm_max_mhz": getattr(self, "max_mhz", None),
+                "reasons": reasons, "samples": len(use), "samples_from": where, "samples_all_passes": len(rows),
+                "source": "NVML" if self.nvml is not None else "nvidia-smi -lms 50"}
 
 
 def time_oracle(x, budget_s: float):
@@ -338,10 +372,9 @@ def main():
     per_step = sorted(marks[bi].elapsed_time(marks[bi + 1]) / block for bi in range(nblk))
     spread = {"median_ms": statistics.median(per_step), "min_ms": per_step[0], "max_ms": per_step[-1],
               "events_around": f"every {'step' if block == 1 else f'{block} steps'}", "samples": nblk}
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_region0, t_region1) if rank == 0 else None
     if clocks is not None:
-        clocks["window"] = (f"warm-up end to the end of the per-step pass ({time.time() - t_region0:.3f} s, same steps twice); "
-                            f"the timed region itself lasted {t_region1 - t_region0:.4f} s")
+        clocks["timed_region_s"] = t_region1 - t_region0
 
     # per-kernel durations: a second pass of the same steps with events around every launch
     e = 2 if wl.dtype == "bf16" else 4

@@ -9,6 +9,7 @@
 #include <string.h>
 
 #include <new>
+#include <type_traits>
 
 #include "simt_kernels.cuh"
 #include "simt_backward.cuh"
@@ -49,7 +50,9 @@ struct linattn_ctx {
     // weights for the tensor-core path: bf16 W^T [H][d/2][d] (d = 128 only)
     __nv_bfloat16* Wqt = nullptr;
     __nv_bfloat16* Wkt = nullptr;
-    bool map_is_bf16 = false;   // the caller supplied bf16 weights (the tensor-core path uses them unrounded)
+    __nv_bfloat16* Wqt_lo = nullptr;   // what the bf16 rounding of fp32 weights leaves, rounded to bf16 again: W = hi + lo
+    __nv_bfloat16* Wkt_lo = nullptr;
+    bool map_is_bf16 = false;   // the caller supplied bf16 weights: the images above are exact and the lo parts unused
     __nv_bfloat16* s_img = nullptr;  // [max_B*H][128*128] bf16 image of S for the query-side TMA
     __nv_bfloat16* z_img = nullptr;  // [max_B*H][2048] bf16 operand image of z (hi, lo)
     int num_sms = 0;
@@ -328,7 +331,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     }
     if (Pk + G > c->partial_slots_tc) return LINATTN_ERR_WORKSPACE;
 
-    CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmS, tmA;   // tmA: the softmax branch's output (mixed attention), else a copy of tmQ
+    CUtensorMap tmK, tmV, tmQ, tmO, tmWk, tmWq, tmWklo, tmWqlo, tmS, tmA;   // tmA: the softmax branch's output (mixed attention), else a copy of tmQ
     const ActStrides as = act_strides(c, n);
     const int layout = c->opt_layout;
     auto act_map = [&](CUtensorMap* m, const void* base, uint32_t box_rows = kTile) {
@@ -340,33 +343,41 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     const bool ok = act_map(&tmK, k) && act_map(&tmV, v, kTile / 2) && act_map(&tmQ, q) && act_map(&tmO, out) && act_map(&tmA, mix ? mix : q) &&
                     make_tmap_bf16_3d(&tmWk, c->Wkt + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
                     make_tmap_bf16_3d(&tmWq, c->Wqt + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
+                    make_tmap_bf16_3d(&tmWklo, c->Wkt_lo + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
+                    make_tmap_bf16_3d(&tmWqlo, c->Wqt_lo + (size_t)c->view_head0 * kD * kM, kD, kM, (uint64_t)Hv, kM) &&
                     make_tmap_bf16_3d(&tmS, c->s_img + (size_t)c->view_g0 * kD * kD, kD, kD, (uint64_t)G, kTile);
     if (!ok) {
         snprintf(c->err_text, sizeof(c->err_text), "cuTensorMapEncodeTiled failed");
         return LINATTN_ERR_CUDA;
     }
-    // one instantiation per (mixed attention or not, memory layout, kernel function, heads singly or in pairs)
-#define LA_BY_PAIR(K, ...) {(const void*)K<__VA_ARGS__, 0>, (const void*)K<__VA_ARGS__, 1>}
-#define LA_BY_PHI(K, ...) {LA_BY_PAIR(K, __VA_ARGS__, 0), LA_BY_PAIR(K, __VA_ARGS__, 1)}
-    const void* k_fused[2][2][2][2] = {{LA_BY_PHI(linattn_fused_tc, false, 0), LA_BY_PHI(linattn_fused_tc, false, 1)},
-                                       {LA_BY_PHI(linattn_fused_tc, true, 0), LA_BY_PHI(linattn_fused_tc, true, 1)}};
-    const void* k_qside[2][2][2][2] = {{LA_BY_PHI(qside_tc, false, 0), LA_BY_PHI(qside_tc, false, 1)},
-                                       {LA_BY_PHI(qside_tc, true, 0), LA_BY_PHI(qside_tc, true, 1)}};
-    const void* k_kside[2][2][2] = {LA_BY_PHI(kside_tc, 0), LA_BY_PHI(kside_tc, 1)};
+    // one instantiation per (mixed attention or not, memory layout, kernel function, heads singly or in pairs, weights exact
+    // in bf16 or split into hi + lo); the ReLU kernel function has no weights, so it has no split variant
+#define LA_BY_SPLIT(K, ...) {(const void*)K<__VA_ARGS__, 0>, (const void*)K<__VA_ARGS__, 1>}
+#define LA_NO_SPLIT(K, ...) {(const void*)K<__VA_ARGS__, 0>, nullptr}
+#define LA_BY_PHI(K, ...) {{LA_BY_SPLIT(K, __VA_ARGS__, 0, 0), LA_BY_SPLIT(K, __VA_ARGS__, 0, 1)}, {LA_NO_SPLIT(K, __VA_ARGS__, 1, 0), LA_NO_SPLIT(K, __VA_ARGS__, 1, 1)}}
+    // indices: [mixed][layout][kernel function][pair][split]
+    static const void* const k_fused[2][2][2][2][2] = {{LA_BY_PHI(linattn_fused_tc, false, 0), LA_BY_PHI(linattn_fused_tc, false, 1)},
+                                                       {LA_BY_PHI(linattn_fused_tc, true, 0), LA_BY_PHI(linattn_fused_tc, true, 1)}};
+    static const void* const k_qside[2][2][2][2][2] = {{LA_BY_PHI(qside_tc, false, 0), LA_BY_PHI(qside_tc, false, 1)},
+                                                       {LA_BY_PHI(qside_tc, true, 0), LA_BY_PHI(qside_tc, true, 1)}};
+    static const void* const k_kside[2][2][2][2] = {LA_BY_PHI(kside_tc, 0), LA_BY_PHI(kside_tc, 1)};
 #undef LA_BY_PHI
-#undef LA_BY_PAIR
+#undef LA_NO_SPLIT
+#undef LA_BY_SPLIT
     const int phi = c->opt_phi;
+    const int split = (phi == 0 && !c->map_is_bf16) ? 1 : 0;
     bool& attr_done = c->attr_done[linattn_ctx::kAttrTcFwd];
     if (!attr_done) {
         for (int i = 0; i < 2; ++i)
             for (int p = 0; p < 2; ++p)
-                for (int pr = 0; pr < 2; ++pr) {
-                    LA_CUDA(c, cudaFuncSetAttribute(k_kside[i][p][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-                    for (int j = 0; j < 2; ++j) {
-                        LA_CUDA(c, cudaFuncSetAttribute(k_fused[i][j][p][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
-                        LA_CUDA(c, cudaFuncSetAttribute(k_qside[i][j][p][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                for (int pr = 0; pr < 2; ++pr)
+                    for (int sp = 0; sp < 2 - p; ++sp) {
+                        LA_CUDA(c, cudaFuncSetAttribute(k_kside[i][p][pr][sp], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                        for (int j = 0; j < 2; ++j) {
+                            LA_CUDA(c, cudaFuncSetAttribute(k_fused[i][j][p][pr][sp], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                            LA_CUDA(c, cudaFuncSetAttribute(k_qside[i][j][p][pr][sp], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::kTotal));
+                        }
                     }
-                }
         attr_done = true;
     }
     const double side_bytes = 2.0 * (double)heads * n * c->d * 2;
@@ -398,8 +409,8 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         // one cooperative launch: key side, per-head meeting point, combine, per-head meeting point, query side.  Its
         // counters are zero between launches (the kernel clears them on its way out), so nothing here depends on
         // earlier launches and the launch may be recorded in a CUDA graph.
-        void* params[] = {&tmK, &tmV, &tmWk, &tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
-        const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout][phi][pair], dim3((unsigned)Pq), dim3(kThreads),
+        void* params[] = {&tmK, &tmV, &tmWk, &tmWklo, &tmQ, &tmO, &tmWq, &tmWqlo, &tmS, &tmA, &a};
+        const cudaError_t le = cudaLaunchCooperativeKernel(k_fused[mix ? 1 : 0][layout][phi][pair][split], dim3((unsigned)Pq), dim3(kThreads),
                                                            params, Smem::kTotal, st);
         if (le == cudaSuccess) {
             prof_mark(c, st, "linattn_fused_tc", 2.0 * side_bytes);
@@ -413,8 +424,8 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         c->coop_ok = false;
     }
     {
-        void* kp[] = {&tmK, &tmV, &tmWk, &a};
-        LA_CUDA(c, cudaLaunchKernel(k_kside[layout][phi][pair], dim3((unsigned)Pk), dim3(kThreads), kp, Smem::kTotal, st));
+        void* kp[] = {&tmK, &tmV, &tmWk, &tmWklo, &a};
+        LA_CUDA(c, cudaLaunchKernel(k_kside[layout][phi][pair][split], dim3((unsigned)Pk), dim3(kThreads), kp, Smem::kTotal, st));
     }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_tc", side_bytes);
@@ -427,8 +438,8 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
         return LINATTN_OK;
     }
     {
-        void* qp[] = {&tmQ, &tmO, &tmWq, &tmS, &tmA, &a};
-        LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout][phi][pair], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
+        void* qp[] = {&tmQ, &tmO, &tmWq, &tmWqlo, &tmS, &tmA, &a};
+        LA_CUDA(c, cudaLaunchKernel(k_qside[mix ? 1 : 0][layout][phi][pair][split], dim3((unsigned)Pq), dim3(kThreads), qp, Smem::kTotal, st));
     }
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_tc", side_bytes);
@@ -613,6 +624,8 @@ linattn_status linattn_create(linattn_ctx** out_ctx, int device, int H, int d, l
         const size_t wt = sizeof(__nv_bfloat16) * (size_t)H * linattn::tc::kM * linattn::tc::kD;
         e = cudaMalloc(&c->Wqt, wt);
         if (e == cudaSuccess) e = cudaMalloc(&c->Wkt, wt);
+        if (e == cudaSuccess) e = cudaMalloc(&c->Wqt_lo, wt);
+        if (e == cudaSuccess) e = cudaMalloc(&c->Wkt_lo, wt);
         if (e == cudaSuccess) e = cudaMalloc(&c->s_img, sizeof(__nv_bfloat16) * (size_t)G * linattn::tc::kD * linattn::tc::kD);
         if (e == cudaSuccess) e = cudaMalloc(&c->z_img, (size_t)G * linattn::tc::kZBlkBytes);
         if (e == cudaSuccess) e = cudaMemset(c->z_img, 0, (size_t)G * linattn::tc::kZBlkBytes);
@@ -650,6 +663,8 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->sync_words);
     cudaFree(c->Wqt);
     cudaFree(c->Wkt);
+    cudaFree(c->Wqt_lo);
+    cudaFree(c->Wkt_lo);
     cudaFree(c->s_img);
     cudaFree(c->z_img);
     cudaFree(c->bwd_part_state);
@@ -686,25 +701,27 @@ linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const voi
         convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wq, c->H, DM, per_head ? 1 : 0);
         convert_weights<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wk, c->H, DM, per_head ? 1 : 0);
     }
-    if (c->d == 64) {
+    {
+        // images for the tensor-core kernels: W^T [H][64][128] bf16 (d = 64: of each pair of consecutive heads); fp32 weights
+        // are kept as a bf16 hi + lo pair
         const unsigned tb = (unsigned)(((size_t)c->H * tc::kM * tc::kD + 255) / 256);
-        if (wdtype == LINATTN_F32) {
-            tc::pair_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
-            tc::pair_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
-        } else {
-            tc::pair_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
-            tc::pair_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
-        }
-    }
-    if (c->d == 128) {
-        const unsigned tb = (unsigned)(((size_t)c->H * DM + 255) / 256);
-        if (wdtype == LINATTN_F32) {
-            tc::transpose_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
-            tc::transpose_weights_bf16<float><<<tb, 256, 0, st>>>((const float*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
-        } else {
-            tc::transpose_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wq, c->Wqt, c->H, per_head ? 1 : 0);
-            tc::transpose_weights_bf16<__nv_bfloat16><<<tb, 256, 0, st>>>((const __nv_bfloat16*)Wk, c->Wkt, c->H, per_head ? 1 : 0);
-        }
+        const int ph = per_head ? 1 : 0;
+        auto images = [&](auto src_q, auto src_k) {
+            using T = std::remove_cv_t<std::remove_pointer_t<decltype(src_q)>>;
+            for (int lo = 0; lo < (wdtype == LINATTN_F32 ? 2 : 1); ++lo) {
+                __nv_bfloat16* dq = lo ? c->Wqt_lo : c->Wqt;
+                __nv_bfloat16* dk = lo ? c->Wkt_lo : c->Wkt;
+                if (c->d == 64) {
+                    tc::pair_weights_bf16<T><<<tb, 256, 0, st>>>(src_q, dq, c->H, ph, lo);
+                    tc::pair_weights_bf16<T><<<tb, 256, 0, st>>>(src_k, dk, c->H, ph, lo);
+                } else {
+                    tc::transpose_weights_bf16<T><<<tb, 256, 0, st>>>(src_q, dq, c->H, ph, lo);
+                    tc::transpose_weights_bf16<T><<<tb, 256, 0, st>>>(src_k, dk, c->H, ph, lo);
+                }
+            }
+        };
+        if (wdtype == LINATTN_F32) images((const float*)Wq, (const float*)Wk);
+        else images((const __nv_bfloat16*)Wq, (const __nv_bfloat16*)Wk);
     }
     LA_CUDA(c, cudaGetLastError());
     c->map_is_bf16 = (wdtype == LINATTN_BF16);
@@ -736,12 +753,13 @@ static linattn_status forward_impl(linattn_ctx* c, const void* q, const void* k,
     return dispatch_forward(c, q, k, v, out, mix, mix_r, B, n, d, dtype, (cudaStream_t)stream);
 }
 
-// Choice of kernels for checked arguments.  The tensor-core kernels cover bf16 activations with bf16 feature-map
-// weights (head dimension 128, or 64 with the heads taken in pairs); everything else runs on the CUDA-core kernels.
+// Choice of kernels for checked arguments.  The tensor-core kernels cover bf16 activations (head dimension 128, or 64
+// with the heads taken in pairs; feature-map weights given in fp32 enter as a bf16 hi + lo pair); fp32 activations run
+// on the CUDA-core kernels.
 static linattn_status dispatch_forward(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, const void* mix,
                                        float mix_r, int B, int n, int d, linattn_dtype dtype, cudaStream_t st)
 {
-    const bool tc_ok = (dtype == LINATTN_BF16 && (c->map_is_bf16 || c->opt_phi == 1));   // d = 128, or d = 64 with the heads in pairs
+    const bool tc_ok = (dtype == LINATTN_BF16);   // d = 128, or d = 64 with the heads in pairs; weights of either type
     if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
     c->last_B = B;
     c->state_transposed = tc_ok && c->opt_path != 1;

@@ -346,7 +346,9 @@ __device__ __forceinline__ uint64_t desc_at(uint64_t base_desc, uint32_t smem_ad
 }
 
 // U = X W (Eq. 6 logits) for one tile: A = X tile (K-major), B = W^T (K-major), D = 128 x 64 fp32.
-__device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_smem, uint32_t w_smem)
+// add = true: a second pass that adds X W_lo to the X W_hi already there (feature-map weights given in fp32 are held as
+// a bf16 hi + lo pair, W = W_hi + W_lo to 2^-17 relative, so that fp32 weights run on the tensor cores too).
+__device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_smem, uint32_t w_smem, bool add = false)
 {
     constexpr uint32_t idesc = make_idesc_bf16(kTile, kM, 0, 0);
     const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
@@ -354,7 +356,7 @@ __device__ __forceinline__ void issue_logits_mma(uint32_t d_tmem, uint32_t x_sme
     for (int k = 0; k < kD / 16; ++k) {
         const uint64_t da = desc_at(kmajor, x_smem + (k >> 2) * kHalfTileBytes + (k & 3) * 32);
         const uint64_t db = desc_at(kmajor, w_smem + (k >> 2) * (kWBytes / 2) + (k & 3) * 32);
-        mma_bf16_ss(d_tmem, da, db, idesc, k > 0);
+        mma_bf16_ss(d_tmem, da, db, idesc, (add || k > 0) ? 1u : 0u);
     }
 }
 
@@ -614,11 +616,16 @@ __device__ __forceinline__ void raise_abort(const WaitCtx& wc, uint32_t code)
 
 // kPhi: 0 = the Hedgehog feature map of Eq. 6; 1 = the ReLU kernel function (no projection, no softmax: the logits
 // warp idles and warps 0-7 rectify the K tile in place).
+// kSplit: 1 = the feature-map weights are a bf16 hi + lo pair (they were given in fp32): two logits passes per tile.  The
+// low parts live in the last slot of the V ring (key side) and of the Q ring (query side), which then run with one
+// slot fewer; a compile-time variant, so that the rings of the common case keep their compile-time sizes.
 // arrive: fused kernel; every partial record written is announced at its head's first meeting point.
-template <int kLayout, int kPhi, int kPair>
+template <int kLayout, int kPhi, int kPair, int kSplit>
 __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const CUtensorMap* tmK, const CUtensorMap* tmV,
-                                            const CUtensorMap* tmW, bool arrive)
+                                            const CUtensorMap* tmW, const CUtensorMap* tmWlo, bool arrive)
 {
+    constexpr int vh = kSplit ? kVHalves - 1 : kVHalves;   // half-tile slots of the V ring in use
+    const uint32_t wlo_smem = c.sbase + Smem::kKV + (kVHalves - 1) * kHalfTileBytes;
     const uint32_t tmem_u = c.tmem;            // 2 x 64 columns of logits
     // two accumulator sets, alternating by segment, so that one drains while the next accumulates
     auto tmem_s = [&](int b) { return c.tmem + 128 + b * 144; };   // 128 columns: S[f][c], lane = f
@@ -636,14 +643,14 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             tma_prefetch_desc(tmW);
         }
         Ring<kKSlots> r;
-        Ring<kVHalves> vr;
+        Ring<vh> vr;
         TileWalk wv = w;                 // walks the V tiles, kVLag tiles behind the K tiles
         int issued = 0, issued_v = 0;    // K tiles and V half tiles whose loads have been issued so far
         bool ok = true;
         // one half tile of V: tokens [64 h, 64 h + 64) of tile wv, as two boxes of 64 columns (the map's box is 64 rows high);
         // a half that lies past the end of the sequence is zero-filled like any out-of-range row
         auto issue_v = [&]() {
-            if (issued_v >= kVHalves && !warp_wait(c.bar(K_VEMPTY + vr.s), vr.ph ^ 1u, c.wc, kErrProducer)) { ok = false; return; }
+            if (issued_v >= vh && !warp_wait(c.bar(K_VEMPTY + vr.s), vr.ph ^ 1u, c.wc, kErrProducer)) { ok = false; return; }
             if (lane == 0) {
                 mbar_arrive_expect_tx(c.bar(K_VFULL + vr.s), kHalfTileBytes);
                 const uint32_t vdst = sbase + Smem::kKV + vr.s * kHalfTileBytes;
@@ -675,8 +682,8 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             // unwinding after a time-out: let the copies already in flight land before the CTA moves on
             for (int i = (issued > kKSlots ? issued - kKSlots : 0); i < issued; ++i)
                 mbar_wait(c.bar(K_FULL + i % kKSlots), (uint32_t)(i / kKSlots) & 1u, c.wc.limit_ns());
-            for (int i = (issued_v > kVHalves ? issued_v - kVHalves : 0); i < issued_v; ++i)
-                mbar_wait(c.bar(K_VFULL + i % kVHalves), (uint32_t)(i / kVHalves) & 1u, c.wc.limit_ns());
+            for (int i = (issued_v > vh ? issued_v - vh : 0); i < issued_v; ++i)
+                mbar_wait(c.bar(K_VFULL + i % vh), (uint32_t)(i / vh) & 1u, c.wc.limit_ns());
         }
     } else if (warp == 9) {
         // ---------------- logits MMA issuer: U = K W_k ----------------
@@ -689,9 +696,14 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             if (w.first()) {
                 if (w.seg >= 1 && !warp_wait(c.bar(K_WFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrMmaLoad)) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(c.bar(K_WFULL), kWBytes);
-                    tma_load_3d(sbase + Smem::kKW, tmW, c.bar(K_WFULL), 0, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
-                    tma_load_3d(sbase + Smem::kKW + kWBytes / 2, tmW, c.bar(K_WFULL), 64, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
+                    const int wi = Blocks<kLayout, kPair>::weights(w.g, a.H);
+                    mbar_arrive_expect_tx(c.bar(K_WFULL), kSplit ? 2 * kWBytes : kWBytes);
+                    tma_load_3d(sbase + Smem::kKW, tmW, c.bar(K_WFULL), 0, 0, wi);
+                    tma_load_3d(sbase + Smem::kKW + kWBytes / 2, tmW, c.bar(K_WFULL), 64, 0, wi);
+                    if (kSplit) {
+                        tma_load_3d(wlo_smem, tmWlo, c.bar(K_WFULL), 0, 0, wi);
+                        tma_load_3d(wlo_smem + kWBytes / 2, tmWlo, c.bar(K_WFULL), 64, 0, wi);
+                    }
                 }
                 if (!warp_wait(c.bar(K_WFULL), (uint32_t)w.seg & 1u, c.wc, kErrMmaLoad)) break;
             }
@@ -701,6 +713,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
             tcgen05_fence_after();
             if (elect_one()) {
                 issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + Smem::kKW);
+                if (kSplit) issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, wlo_smem, true);
                 mma_commit(c.bar(K_UFULL + ur.s));
                 if (w.last()) mma_commit(c.bar(K_WFREE));
             }
@@ -715,7 +728,7 @@ __device__ __forceinline__ void kside_phase(const Cta& c, const Args& a, const C
         const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);        // phi^T: blocks of 64 features 16 KB apart
         const uint64_t mnmajor_v = make_desc_sw128(0, kHalfTileBytes / 2, 1024);  // V half tile: blocks of 64 columns 8 KB apart
         Ring<kKSlots> r;
-        Ring<kVHalves> vr;
+        Ring<vh> vr;
         bool ok = true;
         for (; !w.done() && ok; w.next(), r.next()) {
             if (!warp_wait(c.bar(K_PHIFULL + r.s), r.ph, c.wc, kErrMmaPhi)) break;
@@ -903,10 +916,13 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src,
 
 // wait_state: the S and z images are produced earlier in the same kernel (fused path); loads of them
 // must wait at the head's second meeting point.  Otherwise they were written by a previous launch.
-template <bool kMix, int kLayout, int kPhi, int kPair>
+template <bool kMix, int kLayout, int kPhi, int kPair, int kSplit>
 __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const CUtensorMap* tmQ, const CUtensorMap* tmO,
-                                            const CUtensorMap* tmW, const CUtensorMap* tmS, const CUtensorMap* tmA, bool wait_state)
+                                            const CUtensorMap* tmW, const CUtensorMap* tmWlo, const CUtensorMap* tmS,
+                                            const CUtensorMap* tmA, bool wait_state)
 {
+    constexpr int qs = kSplit ? kQStages - 1 : kQStages;   // slots of the Q ring in use
+    const uint32_t wlo_smem = c.sbase + (kQStages - 1) * kTileBytes;
     const uint32_t tmem_u = c.tmem;  // 2 x 64 columns of logits
     auto tmem_num = [&](int db) { return c.tmem + 128 + db * 160; };   // 144 columns: num[token][c], c = 0..127, then
     auto tmem_den = [&](int db) { return c.tmem + 256 + db * 160; };   // 16 columns: [phi(q).z_hi, phi(q).z_lo, 0...]
@@ -922,7 +938,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             tma_prefetch_desc(tmW);
             tma_prefetch_desc(tmS);
         }
-        Ring<kQStages> r;
+        Ring<qs> r;
         int issued = 0;
         int state_g = -1;   // head whose S, z still have to be loaded (W already on its way)
         bool ok = true;
@@ -959,15 +975,20 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 if (!ok) break;
                 if (w.seg >= 1 && !warp_wait(c.bar(Q_SEGFREE), (uint32_t)(w.seg - 1) & 1u, c.wc, kErrSeg)) break;
                 if (kPhi == 0 && lane == 0) {
-                    mbar_arrive_expect_tx(c.bar(Q_WFULL), kWBytes);
-                    tma_load_3d(sbase + Smem::kQW, tmW, c.bar(Q_WFULL), 0, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
-                    tma_load_3d(sbase + Smem::kQW + kWBytes / 2, tmW, c.bar(Q_WFULL), 64, 0, Blocks<kLayout, kPair>::weights(w.g, a.H));
+                    const int wi = Blocks<kLayout, kPair>::weights(w.g, a.H);
+                    mbar_arrive_expect_tx(c.bar(Q_WFULL), kSplit ? 2 * kWBytes : kWBytes);
+                    tma_load_3d(sbase + Smem::kQW, tmW, c.bar(Q_WFULL), 0, 0, wi);
+                    tma_load_3d(sbase + Smem::kQW + kWBytes / 2, tmW, c.bar(Q_WFULL), 64, 0, wi);
+                    if (kSplit) {
+                        tma_load_3d(wlo_smem, tmWlo, c.bar(Q_WFULL), 0, 0, wi);
+                        tma_load_3d(wlo_smem + kWBytes / 2, tmWlo, c.bar(Q_WFULL), 64, 0, wi);
+                    }
                 }
                 state_g = w.g;
                 // the first head's state may not exist yet: get the first Q tiles moving before waiting for it
                 if (!(wait_state && w.seg == 0)) load_state();
             }
-            if (state_g >= 0 && w.i >= kQStages) {
+            if (state_g >= 0 && w.i >= qs) {
                 if (wait_state && w.seg == 0) {
                     // The ring is full and S does not exist yet.  Once the CTAs of this head have drained their
                     // accumulators (first meeting point) HBM has little to do until the query side starts: use the time
@@ -996,7 +1017,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
                 load_state();
             }
             if (!ok) break;
-            if (w.i >= kQStages && !warp_wait(c.bar(Q_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) break;
+            if (w.i >= qs && !warp_wait(c.bar(Q_EMPTY + r.s), r.ph ^ 1u, c.wc, kErrProducer)) break;
             LA_TRACE(0, 24 + w.i, 0);
             if (lane == 0) {
                 mbar_arrive_expect_tx(c.bar(Q_FULL + r.s), kTileBytes);
@@ -1029,12 +1050,12 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         }
         if (!ok || issued < w.count) {
             // unwinding: let the copies already in flight land before the CTA moves on
-            for (int i = (issued > kQStages ? issued - kQStages : 0); i < issued; ++i)
-                mbar_wait(c.bar(Q_FULL + i % kQStages), (uint32_t)(i / kQStages) & 1u, c.wc.limit_ns());
+            for (int i = (issued > qs ? issued - qs : 0); i < issued; ++i)
+                mbar_wait(c.bar(Q_FULL + i % qs), (uint32_t)(i / qs) & 1u, c.wc.limit_ns());
         }
     } else if (warp == 9) {
         // ---------------- logits MMA issuer: U = Q W_q ----------------
-        Ring<kQStages> r;
+        Ring<qs> r;
         Ring<2> ur;
         for (; kPhi == 0 && !w.done(); w.next(), r.next(), ur.next()) {
             if (w.first() && !warp_wait(c.bar(Q_WFULL), (uint32_t)w.seg & 1u, c.wc, kErrSeg)) break;
@@ -1044,6 +1065,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             tcgen05_fence_after();
             if (elect_one()) {
                 issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, sbase + Smem::kQW);
+                if (kSplit) issue_logits_mma(tmem_u + ur.s * kM, sbase + r.s * kTileBytes, wlo_smem, true);
                 mma_commit(c.bar(Q_UFULL + ur.s));
             }
             __syncwarp();
@@ -1054,7 +1076,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         constexpr uint32_t idesc_n = make_idesc_bf16(kTile, kD + 16, 0, 0);   // A = phi(q) (K-major), B = [S image [c][f]; z operand] (K-major)
         const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
         const uint64_t mnmajor = make_desc_sw128(0, kHalfTileBytes, 1024);
-        Ring<kQStages> r;
+        Ring<qs> r;
         Ring<2> dr;
         for (; !w.done(); w.next(), r.next(), dr.next()) {
             if (w.first() && !warp_wait(c.bar(Q_SEGFULL), (uint32_t)w.seg & 1u, c.wc, kErrSeg)) break;
@@ -1083,7 +1105,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         // held longer than needed costs throughput.
         if (lane == 0) tma_prefetch_desc(tmO);
         const uint64_t keep = policy_evict_last();
-        Ring<kQStages> r;
+        Ring<qs> r;
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(Q_OFULL + r.s), r.ph, c.wc, kErrStore)) break;
             if (lane == 0) {
@@ -1100,7 +1122,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         if (lane == 0) bulk_wait_group<0>();
     } else if (warp < 8 && kPhi == 1) {
         // ---------------- ReLU kernel function (warps 0-7): phi(q) in place in the tile's slot ----------------
-        Ring<kQStages> r;
+        Ring<qs> r;
         for (; !w.done(); w.next(), r.next()) {
             if (!warp_wait(c.bar(Q_FULL + r.s), r.ph, c.wc, kErrSoftmaxU)) break;
             relu_tile_in_place(c.smem + r.s * kTileBytes, threadIdx.x);
@@ -1113,7 +1135,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         const int half = warp >> 2;
         const int row = (warp & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        Ring<kQStages> r;
+        Ring<qs> r;
         Ring<2> ur;
         for (; !w.done(); w.next(), r.next(), ur.next()) {
             if (!warp_wait(c.bar(Q_UFULL + ur.s), ur.ph, c.wc, kErrSoftmaxU)) break;
@@ -1143,7 +1165,7 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         const int row = (warp & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int sw = row & 7;
-        Ring<kQStages> r;
+        Ring<qs> r;
         Ring<2> dr;
         for (; !w.done(); w.next(), r.next(), dr.next()) {
             if (!warp_wait(c.bar(Q_DFULL + dr.s), dr.ph, c.wc, kErrEpilogue)) break;
@@ -1226,14 +1248,14 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
 // Kernels
 // ======================================================================================================
 
-template <int kLayout, int kPhi, int kPair>
+template <int kLayout, int kPhi, int kPair, int kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 kside_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-         const __grid_constant__ CUtensorMap tmW, const Args a)
+         const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmWlo, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, true, false);
-    kside_phase<kLayout, kPhi, kPair>(c, a, &tmK, &tmV, &tmW, false);
+    kside_phase<kLayout, kPhi, kPair, kSplit>(c, a, &tmK, &tmV, &tmW, &tmWlo, false);
     cta_teardown(c);
 }
 
@@ -1245,31 +1267,32 @@ __global__ void __launch_bounds__(256) combine_tc(const Args a, long long P)
     if (q4 < kE / 4) combine_quad<kPair>(a, P, blockIdx.y, q4 * 4);
 }
 
-template <bool kMix, int kLayout, int kPhi, int kPair>
+template <bool kMix, int kLayout, int kPhi, int kPair, int kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 qside_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
-         const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmS,
-         const __grid_constant__ CUtensorMap tmA, const Args a)
+         const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmWlo,
+         const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmA, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     const Cta c = cta_setup(smem_raw, a, false, true);
-    qside_phase<kMix, kLayout, kPhi, kPair>(c, a, &tmQ, &tmO, &tmW, &tmS, &tmA, false);
+    qside_phase<kMix, kLayout, kPhi, kPair, kSplit>(c, a, &tmQ, &tmO, &tmW, &tmWlo, &tmS, &tmA, false);
     cta_teardown(c);
 }
 
 // The whole forward in one cooperative launch of P <= #SMs persistent CTAs.
-template <bool kMix, int kLayout, int kPhi, int kPair>
+template <bool kMix, int kLayout, int kPhi, int kPair, int kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                 const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmQ,
-                 const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmWq,
+                 const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmWklo,
+                 const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
+                 const __grid_constant__ CUtensorMap tmWq, const __grid_constant__ CUtensorMap tmWqlo,
                  const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmA, const Args a)
 {
     extern __shared__ uint8_t smem_raw[];
     LA_TRACE_NS(0, 60, 0);
     const Cta c = cta_setup(smem_raw, a, true, true);
     LA_TRACE_NS(0, 60, 1);
-    kside_phase<kLayout, kPhi, kPair>(c, a, &tmK, &tmV, &tmWk, true);
+    kside_phase<kLayout, kPhi, kPair, kSplit>(c, a, &tmK, &tmV, &tmWk, &tmWklo, true);
     // every role is done with the key-side buffers; the partials of this CTA are written and announced
     tcgen05_fence_before();
     __syncthreads();
@@ -1309,21 +1332,27 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
         if (it == 0) LA_TRACE_NS1(0, 61, 1);
     }
-    qside_phase<kMix, kLayout, kPhi, kPair>(c, a, &tmQ, &tmO, &tmWq, &tmS, &tmA, true);
+    qside_phase<kMix, kLayout, kPhi, kPair, kSplit>(c, a, &tmQ, &tmO, &tmWq, &tmWqlo, &tmS, &tmA, true);
     LA_TRACE_NS(0, 61, 2);
     cta_teardown(c);
     LA_TRACE_NS(0, 61, 3);
 }
 
 // W [H][128 d][64 j] (any supported type) -> W^T bf16 [H][64 j][128 d]; per_head == 0 replicates one matrix.
+// bf16 hi part of w, or (lo != 0) the bf16 rounding of what the hi part leaves: w = hi + lo to 2^-17 relative.
+__device__ __forceinline__ __nv_bfloat16 bf16_part(float w, int lo)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+    return lo ? __float2bfloat16_rn(w - __bfloat162float(hi)) : hi;
+}
 template <typename T>
-static __global__ void transpose_weights_bf16(const T* __restrict__ src, __nv_bfloat16* __restrict__ dst, int H, int per_head)
+static __global__ void transpose_weights_bf16(const T* __restrict__ src, __nv_bfloat16* __restrict__ dst, int H, int per_head, int lo)
 {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (size_t)H * kM * kD) return;
     const int h = (int)(i / (kM * kD)), rem = (int)(i % (kM * kD)), j = rem / kD, dd = rem % kD;
     const size_t s = (size_t)(per_head ? h : 0) * kD * kM + (size_t)dd * kM + j;
-    dst[i] = __float2bfloat16_rn((float)src[s]);
+    dst[i] = bf16_part((float)src[s], lo);
 }
 
 // Head dimension 64: the weight image of a PAIR of heads, as the logits MMA of the d = 128 kernels wants it.
@@ -1333,7 +1362,7 @@ static __global__ void transpose_weights_bf16(const T* __restrict__ src, __nv_bf
 // so that [x_{h0}, x_{h1}] (128 features) times its transpose gives [u_{h0} (32 logits), u_{h1} (32 logits)].
 // src: W [H][64 d][32 j] (any supported type); per_head == 0: one matrix for every head.
 template <typename T>
-static __global__ void pair_weights_bf16(const T* __restrict__ src, __nv_bfloat16* __restrict__ dst, int H, int per_head)
+static __global__ void pair_weights_bf16(const T* __restrict__ src, __nv_bfloat16* __restrict__ dst, int H, int per_head, int lo)
 {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (size_t)H * kM * kD) return;
@@ -1344,7 +1373,7 @@ static __global__ void pair_weights_bf16(const T* __restrict__ src, __nv_bfloat1
         const int h = per_head ? (h0 + blk) % H : 0;
         v = (float)src[(size_t)h * 64 * 32 + (size_t)(dp & 63) * 32 + (jp & 31)];
     }
-    dst[i] = __float2bfloat16_rn(v);
+    dst[i] = bf16_part(v, lo);
 }
 
 }  // namespace tc

@@ -208,7 +208,7 @@ def test_host_buffer_entry_point(B, H, n, d, dtype):
 
 
 def test_which_kernels_run():
-    """bf16, d = 128, bf16 weights -> the tensor-core kernels (one fused launch by default); fp32 -> CUDA cores."""
+    """bf16 activations -> the tensor-core kernels (one fused launch by default); fp32 activations -> CUDA cores."""
     x = small_inputs(1, 2, 700, 128, torch.bfloat16, seed=14)
     ctx = linattn.LinAttn(2, 128, max_B=1, max_n=700)
     try:
@@ -228,13 +228,52 @@ def test_which_kernels_run():
         assert names(linattn.PATH_TENSOR, 0) == (["kside_tc", "combine_tc", "qside_tc"], 3)
         assert names(linattn.PATH_SIMT, 1) == (["kside_simt", "combine_state", "qside_simt"], 3)
         ctx.check()
-        # fp32 weights with bf16 activations: the tensor-core path would have to round them, so it is not taken
+        # fp32 weights with bf16 activations stay on the tensor cores (the weights enter as a bf16 hi + lo pair)
         ctx.set_feature_map(x["Wq"].float().cuda(), x["Wk"].float().cuda())
-        assert names(linattn.PATH_AUTO, 1)[0][0] == "kside_simt"
+        assert names(linattn.PATH_AUTO, 1) == (["linattn_fused_tc"], 1)
+        ctx.check()
+    finally:
+        ctx.destroy()
+    # fp32 activations have no tensor-core kernels: asking for them is an error, not a silent detour
+    xf = small_inputs(1, 2, 700, 128, torch.float32, seed=14)
+    ctx = linattn.LinAttn(2, 128, max_B=1, max_n=700)
+    try:
+        ctx.set_feature_map(xf["Wq"].cuda(), xf["Wk"].cuda())
+        qf, kf, vf = xf["q"].cuda(), xf["k"].cuda(), xf["v"].cuda()
         lib = linattn.load_library()
         ctx.set_option(linattn.OPT_PATH, linattn.PATH_TENSOR)
-        assert lib.linattn_forward(ctx._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), torch.empty_like(q).data_ptr(),
-                                   1, 2, 700, 128, linattn.BF16, None) == linattn.ERR_UNSUPPORTED
+        assert lib.linattn_forward(ctx._h, qf.data_ptr(), kf.data_ptr(), vf.data_ptr(), torch.empty_like(qf).data_ptr(),
+                                   1, 2, 700, 128, linattn.F32, None) == linattn.ERR_UNSUPPORTED
+    finally:
+        ctx.destroy()
+
+
+@pytest.mark.parametrize("d", [128, 64])
+@pytest.mark.parametrize("scale", [1.0, 40.0])
+def test_fp32_feature_map_weights_on_the_tensor_cores(d, scale):
+    """Weights given in fp32 that are NOT bf16 values: the oracle gets the fp32 weights, the kernels a bf16 hi + lo pair.
+    With logits of magnitude ~50 (scale 40) weights rounded once to bf16 would be off by several per cent in phi."""
+    g = torch.Generator().manual_seed(77 + d)
+    B, H, n = 2, 3, 1500
+    sx = 1.0 / math.sqrt(d)
+    q, k, v = (torch.randn(B, H, n, d, generator=g).mul_(sx).bfloat16() for _ in range(3))
+    Wq, Wk = (torch.randn(H, d, d // 2, generator=g).mul_(scale / (math.sqrt(d) * sx)) for _ in range(2))   # fp32, full mantissas
+    assert not torch.equal(Wq.bfloat16().float(), Wq)
+    want = oracle.ref_linear(q, k, v, Wq, Wk)
+    ctx = linattn.LinAttn(H, d, max_B=B, max_n=n)
+    try:
+        ctx.set_feature_map(Wq.cuda(), Wk.cuda())
+        for fuse in (1, 0):
+            ctx.set_option(linattn.OPT_FUSE, fuse)
+            out = ctx.forward(q.cuda(), k.cuda(), v.cuda())
+            ctx.check()
+            assert ctx.last_launch_count() == (1 if fuse else 3)
+            assert_parity(out.cpu().double().numpy(), want, f"fp32 weights, d={d}, scale {scale}, fuse={fuse}")
+        # the same weights after a switch to bf16 values and back
+        ctx.set_feature_map(Wq.bfloat16().cuda(), Wk.bfloat16().cuda())
+        out_b = ctx.forward(q.cuda(), k.cuda(), v.cuda())
+        ctx.check()
+        assert_parity(out_b.cpu().double().numpy(), oracle.ref_linear(q, k, v, Wq.bfloat16(), Wk.bfloat16()), "bf16 weights afterwards")
     finally:
         ctx.destroy()
 
