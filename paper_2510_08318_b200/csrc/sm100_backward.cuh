@@ -57,11 +57,13 @@ struct BwdArgs {
 struct BwdSmemQ {   // query side
     static constexpr uint32_t kX = 0;                        // Q tile
     static constexpr uint32_t kG = kX + kTileBytes;          // dO tile -> du (first 16 KB)
-    static constexpr uint32_t kL = kG + kTileBytes;          // fp32 scratch for du, and for the dz sums at the end of a head
+    static constexpr uint32_t kL = kG + kTileBytes;          // du tile [128][64] bf16 (16 KB), then room for the dz sums at the end of a head
     static constexpr uint32_t kP = kL + kTileBytes;          // phi(q) -> phi(q) / den -> dq staging
     static constexpr uint32_t kShi = kP + kTileBytes;        // S image [c][f], hi part
     static constexpr uint32_t kSlo = kShi + kTileBytes;      // lo part
     static constexpr uint32_t kW = kSlo + kTileBytes;        // W_q^T [64][128]
+    static constexpr uint32_t kDu = kL;                      // du tile
+    static constexpr uint32_t kRed = kL + kWBytes;           // 16 x 128 floats: dz sums of the token groups
     static constexpr uint32_t kMisc = kW + kWBytes;
 };
 struct BwdSmemK {   // key side
@@ -80,13 +82,13 @@ struct BwdMisc {
     static constexpr uint32_t kA = 512;           // 2 x 128 floats: den halves, later dz halves
     static constexpr uint32_t kB = 1536;          // 2 x 128 floats: (dO . o) halves
     static constexpr uint32_t kDd = 2560;         // 128 floats: dden
-    static constexpr uint32_t kBars = 3072;       // 3 mbarriers, TMEM slot, abort word
+    static constexpr uint32_t kBars = 3072;       // 4 mbarriers, TMEM slot, abort word
     static constexpr uint32_t kBytes = 3072 + 64;
 };
 constexpr uint32_t kBwdSmemQ = BwdSmemQ::kMisc + BwdMisc::kBytes + 1024;
 constexpr uint32_t kBwdSmemK = BwdSmemK::kMisc + BwdMisc::kBytes + 1024;
 
-enum : int { BW_LOAD = 0, BW_SEG = 1, BW_MMA = 2 };
+enum : int { BW_LOAD = 0, BW_SEG = 1, BW_MMA = 2, BW_MMA2 = 3, BW_NBARS = 4 };
 
 struct BwdCta {
     uint8_t* smem;
@@ -104,13 +106,13 @@ __device__ __forceinline__ BwdCta bwd_setup(uint8_t* smem_raw, uint32_t misc_off
     c.misc = reinterpret_cast<float*>(c.smem + misc_off);
     uint64_t* bars = reinterpret_cast<uint64_t*>(c.smem + misc_off + BwdMisc::kBars);
     c.bar0 = smem_u32(bars);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[3]);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[BW_NBARS]);
     uint32_t* abort_word = tmem_slot + 1;
     c.wc.err = err;
     c.wc.abort_smem = smem_u32(abort_word);
     if (threadIdx.x == 0) {
         *abort_word = 0u;
-        for (int i = 0; i < 3; ++i) mbar_init(c.bar(i), 1);
+        for (int i = 0; i < BW_NBARS; ++i) mbar_init(c.bar(i), 1);
         fence_mbar_init();
     }
     if ((threadIdx.x >> 5) == 1) {
@@ -193,6 +195,43 @@ __device__ __forceinline__ float softmax_half_keep(float (&u)[kM], uint8_t* blk,
     return s0 + s1;
 }
 
+// The same without the store: p[64] (fp32) in place, its bf16 roundings packed two to a word in pk[32] (what a tensor
+// core operand built from p holds).  Returns sum_j bf16(p_j) * vec[j].
+template <bool kNeg>
+__device__ __forceinline__ float softmax_half_packed(float (&u)[kM], uint32_t (&pk)[kM / 2], const float* vec)
+{
+    float m = kNeg ? min3(u[0], u[1], u[2]) : max3(u[0], u[1], u[2]);
+#pragma unroll
+    for (int j = 3; j < kM - 1; j += 2) m = kNeg ? min3(m, u[j], u[j + 1]) : max3(m, u[j], u[j + 1]);
+    m = kNeg ? fminf(m, u[kM - 1]) : fmaxf(m, u[kM - 1]);
+    const float sL = kNeg ? -kLog2e : kLog2e, off = kNeg ? m * kLog2e : -m * kLog2e;
+    const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
+    f32x2 sum2 = pack2(0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < kM; j += 2) {
+        float x0, x1;
+        unpack2(fma2(pack2(u[j], u[j + 1]), scale, offset), x0, x1);
+        u[j] = ex2_approx(x0);
+        u[j + 1] = ex2_approx(x1);
+        sum2 = add2(sum2, pack2(u[j], u[j + 1]));
+    }
+    float s0, s1;
+    unpack2(sum2, s0, s1);
+    const float inv = __fdividef(1.f, s0 + s1);
+    const f32x2 inv2 = pack2(inv, inv);
+    f32x2 dot2 = pack2(0.f, 0.f);
+    const float2* vec2 = reinterpret_cast<const float2*>(vec);
+#pragma unroll
+    for (int j = 0; j < kM; j += 2) {
+        unpack2(mul2(pack2(u[j], u[j + 1]), inv2), u[j], u[j + 1]);
+        pk[j >> 1] = pack_bf16(u[j], u[j + 1]);
+        const float2 zv = vec2[j >> 1];
+        dot2 = fma2(pack2(__uint_as_float(pk[j >> 1] << 16), __uint_as_float(pk[j >> 1] & 0xffff0000u)), pack2(zv.x, zv.y), dot2);
+    }
+    unpack2(dot2, s0, s1);
+    return s0 + s1;
+}
+
 __device__ __forceinline__ void load64(uint32_t taddr, float (&x)[kM])
 {
     uint32_t r[kM];
@@ -215,18 +254,12 @@ __device__ __forceinline__ void store_row_bf16(uint8_t* blk, int row, const floa
     }
 }
 
-// fp32 scratch tile [128 tokens][64]: 16-byte chunk ch of row r sits at chunk ch ^ (r & 15) (no bank conflicts
-// when the threads of a warp, one row each, touch the same logical chunk).
-__device__ __forceinline__ float4* scratch_chunk(uint8_t* scratch, int row, int ch)
-{
-    return reinterpret_cast<float4*>(scratch + (size_t)row * 256 + ((ch ^ (row & 15)) << 4));
-}
-
 // Softmax backward of Eq. 6 for one token, split between the two threads of the token (half 0: softmax(+u),
-// half 1: softmax(-u)): each forms p (.) (dphi - p . dphi) for its half; half 1 parks its values in the scratch
-// tile, and after a CTA barrier half 0 subtracts them and writes du (bf16) to its row of the du tile.
-__device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint8_t* scratch,
-                                            uint8_t* du_tile)
+// half 1: softmax(-u)): each forms p (.) (dphi - p . dphi) for its half; half 1 parks its 64 values in 64 free columns
+// of the token's lane of tensor memory (`park`: the logits' columns, read long before; both threads of a token sit on
+// warps of the same lane quarter, so either can reach the lane), and after a CTA barrier half 0 takes them back,
+// subtracts and writes du (bf16) to its row of the du tile.
+__device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint32_t park, uint8_t* du_tile)
 {
     f32x2 dot2 = pack2(0.f, 0.f);
 #pragma unroll
@@ -238,20 +271,21 @@ __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[
     for (int j = 0; j < kM; j += 2)
         unpack2(mul2(pack2(p[j], p[j + 1]), add2(pack2(dphi[j], dphi[j + 1]), ndot)), dphi[j], dphi[j + 1]);
     if (half == 1) {
+        uint32_t r[kM];
 #pragma unroll
-        for (int ch = 0; ch < 16; ++ch)
-            *scratch_chunk(scratch, row, ch) = make_float4(dphi[4 * ch], dphi[4 * ch + 1], dphi[4 * ch + 2], dphi[4 * ch + 3]);
+        for (int j = 0; j < kM; ++j) r[j] = __float_as_uint(dphi[j]);
+        tmem_st_x32(park, r);
+        tmem_st_x32(park + 32, r + 32);
+        tmem_wait_st();
     }
+    tcgen05_fence_before();
     __syncthreads();
+    tcgen05_fence_after();
     if (half == 0) {
+        float o[kM];
+        load64(park, o);
 #pragma unroll
-        for (int ch = 0; ch < 16; ++ch) {
-            const float4 o = *scratch_chunk(scratch, row, ch);
-            dphi[4 * ch] -= o.x;
-            dphi[4 * ch + 1] -= o.y;
-            dphi[4 * ch + 2] -= o.z;
-            dphi[4 * ch + 3] -= o.w;
-        }
+        for (int j = 0; j < kM; ++j) dphi[j] -= o[j];
         store_row_bf16(du_tile, row, dphi);
     }
 }
@@ -306,7 +340,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     const uint32_t sb0 = c.sbase;
     const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
     const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
-    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0;
+    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0;
     float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
 #pragma unroll
     for (int e = 0; e < 8; ++e) dz_acc[e] = 0.f;
@@ -354,92 +388,78 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
         if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) break;
         LB_TRACE(1);
-        // ---- U = Q W_q ----
+        // ---- U = Q W_q, and T = dO S^T (S_hi, S_lo), which needs nothing but the loaded tiles and runs under the feature map ----
         if (tid == 0) {
             issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
             mma_commit(c.bar(BW_MMA));
-            bulk_wait_group_read<0>();   // the previous tile's dq has left the staging tile, which is phi's home again
-        }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
-        LB_TRACE(2);
-        // ---- phi(q): bf16 operand tile; p stays in registers; den = phi . z from the rounded values ----
-        float p[kM];
-        load64(t_u + lane_base, p);
-        {
-            uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
-            sa[half * kTile + row] = half == 0 ? softmax_half_keep<false>(p, blk, row, vec) : softmax_half_keep<true>(p, blk, row, vec + kM);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        LB_TRACE(3);
-        // ---- num = phi (S_hi + S_lo) ----
-        if (tid == 0) {
-            tcgen05_fence_after();
-            constexpr uint32_t idesc = make_idesc_bf16(kTile, kD, 0, 0);
-#pragma unroll
-            for (int pass = 0; pass < 2; ++pass)
-#pragma unroll
-                for (int k = 0; k < kD / 16; ++k)
-                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)),
-                                desc_at(kmajor, kstep_kmajor(sb0 + (pass == 0 ? L::kShi : L::kSlo), k, kHalfTileBytes)), idesc,
-                                (pass | k) != 0);
-            mma_commit(c.bar(BW_MMA));
-        }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrEpilogue)) break;
-        LB_TRACE(4);
-        // ---- den, dO . o.  The per-token factor 1 / den of dnum = dO / den is kept OUT of the tensor-core operands: dphi
-        // = (dO S^T) / den is scaled in the accumulator's epilogue, and dS = (phi / den)^T dO takes it into phi, so
-        // the dO tile itself, exact in bf16, is the operand of both products ----
-        float inv;
-        {
-            float x[kM];
-            load64(t_work + lane_base + half * kM, x);
-            inv = 1.f / (sa[row] + sa[kTile + row]);
-            const uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
-            f32x2 gs2 = pack2(0.f, 0.f);
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-                const uint4 gv = *reinterpret_cast<const uint4*>(gblk + sw_chunk(row, ch));
-                const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    gs2 = fma2(pack2(__uint_as_float(gw[q] << 16), __uint_as_float(gw[q] & 0xffff0000u)),
-                               pack2(x[8 * ch + 2 * q], x[8 * ch + 2 * q + 1]), gs2);
-            }
-            float g0s, g1s;
-            unpack2(gs2, g0s, g1s);
-            sb[half * kTile + row] = (g0s + g1s) * inv;   // this half's part of dO . o
-            // phi / den over phi (the numerator MMA is done with it); p itself stays in registers for the softmax Jacobian
-            const f32x2 inv2 = pack2(inv, inv);
-#pragma unroll
-            for (int j = 0; j < kM; j += 2) unpack2(mul2(pack2(p[j], p[j + 1]), inv2), x[j], x[j + 1]);
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        const float ngo = -(sb[row] + sb[kTile + row]);   // -(dO . o) = dden * den
-        if (half == 0) sdd[row] = ngo;
-        __syncthreads();
-        LB_TRACE(5);
-        // ---- dphi * den = dO S^T (S_hi, S_lo), dS += (phi / den)^T dO ----
-        if (tid == 0) {
-            tcgen05_fence_after();
-            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = dO (K-major over c), B = S image [c][f] (rows = K)
-            constexpr uint32_t idesc_ds = make_idesc_bf16(kD, kD, 1, 1);        // A = (phi / den)^T, B = dO, both read MN-major
+            constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kD, 0, 1);   // A = dO (K-major over c), B = S image [c][f] (rows = K)
 #pragma unroll
             for (int pass = 0; pass < 2; ++pass) {
                 const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k)
-                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kG, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
+                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kG, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_t,
                                 (pass | k) != 0);
             }
+            mma_commit(c.bar(BW_MMA2));
+            bulk_wait_group_read<0>();   // the previous tile's dq has left the staging tile, which is phi's home again
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
+        LB_TRACE(2);
+        // ---- phi(q): p stays in registers (fp32, and its bf16 roundings); den = phi . z from the rounded values ----
+        float p[kM];
+        uint32_t pk[kM / 2];
+        load64(t_u + lane_base, p);
+        sa[half * kTile + row] = half == 0 ? softmax_half_packed<false>(p, pk, vec) : softmax_half_packed<true>(p, pk, vec + kM);
+        LB_TRACE(3);
+        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrEpilogue)) break;   // T is there (and every thread's den part is visible)
+        LB_TRACE(4);
+        // ---- dO . o = (dO S^T) . phi / den: the numerator phi S itself is never formed.  The per-token factor 1 / den of
+        // dnum = dO / den is kept OUT of the tensor-core operands: dphi = (dO S^T - (dO . o) z) / den is scaled here, in
+        // the accumulator's epilogue, and dS = (phi / den)^T dO takes it into phi, so the dO tile itself, exact in bf16,
+        // is the operand of both products ----
+        float x[kM];
+        load64(t_work + lane_base + half * kM, x);
+        const float inv = 1.f / (sa[row] + sa[kTile + row]);
+        {
+            f32x2 gs2 = pack2(0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < kM; j += 2)
+                gs2 = fma2(pack2(__uint_as_float(pk[j >> 1] << 16), __uint_as_float(pk[j >> 1] & 0xffff0000u)), pack2(x[j], x[j + 1]), gs2);
+            float g0s, g1s;
+            unpack2(gs2, g0s, g1s);
+            sb[half * kTile + row] = (g0s + g1s) * inv;   // this half's part of dO . o
+            // phi / den (bf16) is the operand of dS and the factor of dz
+            float y[kM];
+            const f32x2 inv2 = pack2(inv, inv);
+#pragma unroll
+            for (int j = 0; j < kM; j += 2) unpack2(mul2(pack2(p[j], p[j + 1]), inv2), y[j], y[j + 1]);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, y);
+        }
+        __syncthreads();
+        const float ngo = -(sb[row] + sb[kTile + row]);   // -(dO . o) = dden * den
+        if (half == 0) sdd[row] = ngo;
+        LB_TRACE(5);
+        // ---- du (through the softmax of Eq. 6) ----
+#pragma unroll
+        for (int j = 0; j < kM; j += 2) {   // dphi = (dO S^T - (dO . o) z) / den
+            const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
+            unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
+        }
+        du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        LB_TRACE(8);
+        // ---- dS += (phi / den)^T dO, dq = du W_q^T, dW_q += Q^T du ----
+        if (tid == 0) {
+            tcgen05_fence_after();
+            constexpr uint32_t idesc_ds = make_idesc_bf16(kD, kD, 1, 1);        // A = (phi / den)^T, B = dO, both read MN-major
 #pragma unroll
             for (int k = 0; k < kTile / 16; ++k)
                 mma_bf16_ss(t_ds, desc_at(mn_tile, sb0 + L::kP + k * 2048), desc_at(mn_tile, sb0 + L::kG + k * 2048), idesc_ds,
                             (first && k == 0) ? 0u : 1u);
+            issue_dx_dw(t_work, t_dw, sb0 + L::kDu, sb0 + L::kX, sb0 + L::kW, first);
             mma_commit(c.bar(BW_MMA));
         }
         {
@@ -458,30 +478,6 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     dz_acc[2 * q + 1] = fmaf(dd, __uint_as_float(pw[q] & 0xffff0000u), dz_acc[2 * q + 1]);
                 }
             }
-        }
-        LB_TRACE(6);
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrMmaAcc)) break;
-        LB_TRACE(7);
-        // ---- du (through the softmax of Eq. 6) ----
-        {
-            float x[kM];
-            load64(t_work + lane_base + half * kM, x);
-#pragma unroll
-            for (int j = 0; j < kM; j += 2) {   // dphi = (dO S^T - (dO . o) z) / den
-                const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
-                unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
-            }
-            du_exchange(half, row, p, x, c.smem + L::kL, c.smem + L::kG);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        LB_TRACE(8);
-        // ---- dq = du W_q^T, dW_q += Q^T du ----
-        if (tid == 0) {
-            tcgen05_fence_after();
-            issue_dx_dw(t_work, t_dw, sb0 + L::kG, sb0 + L::kX, sb0 + L::kW, first);
-            mma_commit(c.bar(BW_MMA));
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
         LB_TRACE(9);
@@ -516,7 +512,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
             drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
             // dz: the 16 token groups' sums, in group order (the scratch tile is free at this point)
-            float* red = reinterpret_cast<float*>(c.smem + L::kL);
+            float* red = reinterpret_cast<float*>(c.smem + L::kRed);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 red[(tid >> 4) * kD + (tid & 15) * 8 + e] = dz_acc[e];
@@ -555,7 +551,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     const uint32_t sb0 = c.sbase;
     const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
     const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
-    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0;
+    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0;
     TileWalk w;
     w.init(a.total_tiles, a.tiles_per_head);
     if (tid == 0) {
@@ -597,10 +593,20 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) break;
         }
         if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) break;
-        // ---- U = K W_k ----
+        // ---- U = K W_k, and T = V dS^T (hi and lo parts of dS), which needs nothing but the loaded tiles ----
         if (tid == 0) {
             issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
             mma_commit(c.bar(BW_MMA));
+            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = V (K-major over c), B = dS image [c][f] (rows = K)
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass) {
+                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k)
+                    mma_bf16_ss(t_w1, desc_at(kmajor, kstep_kmajor(sb0 + L::kV, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
+                                (pass | k) != 0);
+            }
+            mma_commit(c.bar(BW_MMA2));
             bulk_wait_group_read<0>();   // the previous tile's dk has left phi's tile
         }
         if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
@@ -611,62 +617,58 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             if (half == 0) softmax_half_keep<false>(p, blk, row, vec);
             else softmax_half_keep<true>(p, blk, row, vec + kM);
         }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        // ---- dphi = V dS^T, dv = phi dS (hi and lo parts of dS) ----
-        if (tid == 0) {
-            tcgen05_fence_after();
-            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = V (K-major over c), B = dS image [c][f] (rows = K)
-            constexpr uint32_t idesc_dv = make_idesc_bf16(kTile, kD, 0, 0);     // A = phi (K-major over f), B = dS image [c][f] (rows = N)
-#pragma unroll
-            for (int pass = 0; pass < 2; ++pass) {
-                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
-#pragma unroll
-                for (int k = 0; k < kD / 16; ++k) {
-                    mma_bf16_ss(t_w1, desc_at(kmajor, kstep_kmajor(sb0 + L::kV, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
-                                (pass | k) != 0);
-                    mma_bf16_ss(t_w2, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)), desc_at(kmajor, kstep_kmajor(st, k, kHalfTileBytes)),
-                                idesc_dv, (pass | k) != 0);
-                }
-            }
-            mma_commit(c.bar(BW_MMA));
-        }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrMmaAcc)) break;
-        // ---- du; dv leaves through phi's tile ----
+        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrMmaAcc)) break;
+        // ---- dphi = V dS^T + dz -> du ----
         {
             float x[kM];
             load64(t_w1 + lane_base + half * kM, x);
 #pragma unroll
             for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
-            du_exchange(half, row, p, x, c.smem + L::kV, c.smem + L::kDu);
+            du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        // ---- dv = phi dS (hi and lo parts), dk = du W_k^T, dW_k += K^T du ----
+        if (tid == 0) {
+            tcgen05_fence_after();
+            constexpr uint32_t idesc_dv = make_idesc_bf16(kTile, kD, 0, 0);     // A = phi (K-major over f), B = dS image [c][f] (rows = N)
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass) {
+                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k)
+                    mma_bf16_ss(t_w2, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)), desc_at(kmajor, kstep_kmajor(st, k, kHalfTileBytes)),
+                                idesc_dv, (pass | k) != 0);
+            }
+            issue_dx_dw(t_w1, t_dw, sb0 + L::kDu, sb0 + L::kX, sb0 + L::kW, first);
+            mma_commit(c.bar(BW_MMA));
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
+        if (tid == 0) {
+            // K, V, phi and the du tile have been consumed: the next tile's loads start now and overlap this tile's stores
+            TileWalk nx = w;
+            nx.next();
+            if (!nx.done()) issue_loads(nx);
+        }
+        // ---- dv, then dk, leave through phi's tile ----
+        {
+            float x[kM];
             load64(t_w2 + lane_base + half * kM, x);
             store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
         }
         fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
-        // ---- dk = du W_k^T, dW_k += K^T du ----
-        if (tid == 0) {
-            tcgen05_fence_after();
-            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-            bulk_commit_group();
-            issue_dx_dw(t_w1, t_dw, sb0 + L::kDu, sb0 + L::kX, sb0 + L::kW, first);
-            mma_commit(c.bar(BW_MMA));
-        }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
-        if (tid == 0) {
-            // K, V (its tile served as scratch) and the du tile have been consumed: the next tile's loads start now and
-            // overlap this tile's stores; dk is staged in phi's tile once dv has left it
-            TileWalk nx = w;
-            nx.next();
-            if (!nx.done()) issue_loads(nx);
-            bulk_wait_group_read<0>();
-        }
-        __syncthreads();
         {
             float x[kM];
-            load64(t_w1 + lane_base + half * kM, x);
+            load64(t_w1 + lane_base + half * kM, x);   // dk comes out of tensor memory while dv's store reads the tile
+            if (tid == 0) {
+                for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                bulk_commit_group();
+                bulk_wait_group_read<0>();
+            }
+            __syncthreads();
             store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
         }
         fence_proxy_async_smem();
