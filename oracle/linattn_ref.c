@@ -314,9 +314,12 @@ static void phi_backward_row(const float *x, const float *W, int d, const double
     }
 }
 
-int linattn_ref_backward(const float *q, const float *k, const float *v, const float *Wq, const float *Wk,
-                         const float *dout, long G, int H, long n, int d, int per_head,
-                         double *dq, double *dk, double *dv, double *dWq, double *dWk)
+/* The chain rule above for an incoming gradient lin_scale * dout (lin_scale = 1 for the plain operator; Eq. 8 hands the
+ * linear branch (1 - r^) times the layer's gradient).  *sum_dout_o, if not NULL, receives sum_{g,i,c} dout * o with the
+ * UNSCALED dout: the part of dL/dr that comes from the linear branch. */
+static int backward_core(const float *q, const float *k, const float *v, const float *Wq, const float *Wk,
+                         const float *dout, double lin_scale, long G, int H, long n, int d, int per_head,
+                         double *dq, double *dk, double *dv, double *dWq, double *dWk, double *sum_dout_o)
 {
     if (d < 2 || d > 4096 || (d & 1) || n < 1 || G < 1 || H < 1) return 1;
     const int m = d / 2;
@@ -355,8 +358,10 @@ int linattn_ref_backward(const float *q, const float *k, const float *v, const f
                     double num = 0.0;
                     for (int f = 0; f < d; ++f) num += phi[f] * S[(size_t)f * d + c];
                     o[c] = num / den;
-                    go += (double)gg[(size_t)i * d + c] * o[c];
-                    dnum[c] = (double)gg[(size_t)i * d + c] / den;
+                    const double gin = lin_scale * (double)gg[(size_t)i * d + c];   /* gradient that reaches the linear branch */
+                    go += gin * o[c];
+                    dnum[c] = gin / den;
+                    if (sum_dout_o) *sum_dout_o += (double)gg[(size_t)i * d + c] * o[c];
                 }
                 const double dden = -go / den;
                 for (int f = 0; f < d; ++f) {
@@ -389,6 +394,43 @@ int linattn_ref_backward(const float *q, const float *k, const float *v, const f
         free(S); free(z); free(dS); free(dz); free(phi); free(dphi); free(o); free(dnum);
     }
     return fail;
+}
+
+int linattn_ref_backward(const float *q, const float *k, const float *v, const float *Wq, const float *Wk,
+                         const float *dout, long G, int H, long n, int d, int per_head,
+                         double *dq, double *dk, double *dv, double *dWq, double *dWk)
+{
+    return backward_core(q, k, v, Wq, Wk, dout, 1.0, G, H, n, d, per_head, dq, dk, dv, dWq, dWk, NULL);
+}
+
+/*
+ * Gradients through the mixed attention of Eq. 8,  out = r^ * a + (1 - r^) * lin(q, k, v),  r^ = clip(r, 0, 1), where a
+ * is the output of the softmax-attention branch (given) and lin the operator of Eq. 5 / Eq. 6.  For L = sum dout * out:
+ *
+ *   dL/da     = r^ * dout
+ *   dL/dlin   = (1 - r^) * dout      -> dq, dk, dv, dW_q, dW_k by the chain rule above with that incoming gradient
+ *   dL/dr     = sum dout * (a - lin)  if 0 <= r <= 1,  else 0
+ *
+ * Reading taken for the clip (the paper's footnote to Eq. 8 clips r into [0, 1] and says nothing of its derivative): the
+ * derivative of clip is 1 on the closed interval, ends included, and 0 outside.  The ends must be included for the
+ * method to work at all: the paper initialises every r to 1, and with a zero derivative at r = 1 no score could ever
+ * leave its initial value.  da may be NULL.  a: [G][n][d] float; dr: one double.
+ */
+int linattn_ref_backward_mixed(const float *q, const float *k, const float *v, const float *Wq, const float *Wk,
+                               const float *a, double r, const float *dout, long G, int H, long n, int d, int per_head,
+                               double *dq, double *dk, double *dv, double *dWq, double *dWk, double *da, double *dr)
+{
+    if (!dr || r != r) return 1;
+    const double rc = r < 0.0 ? 0.0 : (r > 1.0 ? 1.0 : r);
+    double sum_dout_o = 0.0;
+    if (backward_core(q, k, v, Wq, Wk, dout, 1.0 - rc, G, H, n, d, per_head, dq, dk, dv, dWq, dWk, &sum_dout_o)) return 1;
+    double sum_dout_a = 0.0;
+    for (size_t e = 0; e < (size_t)G * n * d; ++e) {
+        sum_dout_a += (double)dout[e] * (double)a[e];
+        if (da) da[e] = rc * (double)dout[e];
+    }
+    *dr = (r >= 0.0 && r <= 1.0) ? sum_dout_a - sum_dout_o : 0.0;
+    return 0;
 }
 
 /*
@@ -474,4 +516,74 @@ int linattn_ref_relu_linear(const float *q, const float *k, const float *v, long
     if (z_out) memcpy(z_out, z_all, (size_t)G * d * sizeof(double));
     free(S_all); free(z_all);
     return 0;
+}
+
+/*
+ * Gradients of Eq. 5 with the ReLU kernel function (reading above: phi(x) = max(x, 0), no weights).  The chain rule of
+ * the operator is the one written out before linattn_ref_backward; only the last step differs: d phi / d x is 1 where
+ * x > 0 and 0 elsewhere (at x = 0 the subgradient 0 is taken, as the automatic differentiation of max(x, 0) does), so
+ *   dq_i = dphi(q_i) (.) [q_i > 0]        dk_j = dphi(k_j) (.) [k_j > 0]        dv_j = dS^T phi(k_j).
+ * All arrays [G][n][d]; inputs float, outputs double.
+ */
+int linattn_ref_relu_backward(const float *q, const float *k, const float *v, const float *dout, long G, long n, int d,
+                              double *dq, double *dk, double *dv)
+{
+    if (d < 1 || d > 4096 || n < 1 || G < 1) return 1;
+    int fail = 0;
+#pragma omp parallel for schedule(dynamic)
+    for (long g = 0; g < G; ++g) {
+        const float *qg = q + (size_t)g * n * d, *kg = k + (size_t)g * n * d, *vg = v + (size_t)g * n * d;
+        const float *gg = dout + (size_t)g * n * d;
+        double *S = (double *)calloc((size_t)d * d, sizeof(double)), *z = (double *)calloc(d, sizeof(double));
+        double *dS = (double *)calloc((size_t)d * d, sizeof(double)), *dz = (double *)calloc(d, sizeof(double));
+        double *o = (double *)malloc((size_t)d * sizeof(double)), *dnum = (double *)malloc((size_t)d * sizeof(double));
+        if (!S || !z || !dS || !dz || !o || !dnum) {
+            fail = 1;
+        } else {
+            for (long j = 0; j < n; ++j)
+                for (int f = 0; f < d; ++f) {
+                    const double pf = relu(kg[(size_t)j * d + f]);
+                    z[f] += pf;
+                    for (int c = 0; c < d; ++c) S[(size_t)f * d + c] += pf * (double)vg[(size_t)j * d + c];
+                }
+            for (long i = 0; i < n; ++i) {
+                const float *qi = qg + (size_t)i * d;
+                double den = 0.0;
+                for (int f = 0; f < d; ++f) den += relu(qi[f]) * z[f];
+                double go = 0.0;
+                for (int c = 0; c < d; ++c) {
+                    double num = 0.0;
+                    for (int f = 0; f < d; ++f) num += relu(qi[f]) * S[(size_t)f * d + c];
+                    o[c] = num / den;
+                    go += (double)gg[(size_t)i * d + c] * o[c];
+                    dnum[c] = (double)gg[(size_t)i * d + c] / den;
+                }
+                const double dden = -go / den;
+                for (int f = 0; f < d; ++f) {
+                    double acc = dden * z[f];
+                    for (int c = 0; c < d; ++c) {
+                        acc += S[(size_t)f * d + c] * dnum[c];
+                        dS[(size_t)f * d + c] += relu(qi[f]) * dnum[c];
+                    }
+                    dz[f] += dden * relu(qi[f]);
+                    dq[((size_t)g * n + i) * d + f] = qi[f] > 0.0f ? acc : 0.0;
+                }
+            }
+            for (long j = 0; j < n; ++j) {
+                const float *kj = kg + (size_t)j * d;
+                double *dvj = dv + ((size_t)g * n + j) * d;
+                for (int c = 0; c < d; ++c) dvj[c] = 0.0;
+                for (int f = 0; f < d; ++f) {
+                    double acc = dz[f];
+                    for (int c = 0; c < d; ++c) {
+                        acc += dS[(size_t)f * d + c] * (double)vg[(size_t)j * d + c];
+                        dvj[c] += relu(kj[f]) * dS[(size_t)f * d + c];
+                    }
+                    dk[((size_t)g * n + j) * d + f] = kj[f] > 0.0f ? acc : 0.0;
+                }
+            }
+        }
+        free(S); free(z); free(dS); free(dz); free(o); free(dnum);
+    }
+    return fail;
 }

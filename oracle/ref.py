@@ -52,6 +52,9 @@ def _load():
         lib.linattn_ref_mix.argtypes = [dp, dp, ctypes.c_long, ctypes.c_double, dp]
         lib.linattn_ref_backward.argtypes = [fp, fp, fp, fp, fp, fp, ctypes.c_long, ctypes.c_int, ctypes.c_long,
                                              ctypes.c_int, ctypes.c_int, dp, dp, dp, dp, dp]
+        lib.linattn_ref_backward_mixed.argtypes = [fp, fp, fp, fp, fp, fp, ctypes.c_double, fp, ctypes.c_long, ctypes.c_int,
+                                                   ctypes.c_long, ctypes.c_int, ctypes.c_int, dp, dp, dp, dp, dp, dp, dp]
+        lib.linattn_ref_relu_backward.argtypes = [fp, fp, fp, fp, ctypes.c_long, ctypes.c_long, ctypes.c_int, dp, dp, dp]
         lib.linattn_ref_relu_quadratic.argtypes = [fp, fp, fp, ctypes.c_long, ctypes.c_long, ctypes.c_int, lp, ctypes.c_long, dp]
         lib.linattn_ref_relu_linear.argtypes = [fp, fp, fp, ctypes.c_long, ctypes.c_long, ctypes.c_int, lp, ctypes.c_long,
                                                 dp, dp, dp]
@@ -186,6 +189,38 @@ def ref_backward(q, k, v, Wq, Wk, dout):
     if rc:
         raise ValueError("oracle rejected the arguments or ran out of memory")
     return dq, dk, dv, dWq, dWk
+
+
+def ref_backward_mixed(q, k, v, Wq, Wk, o_softmax, r: float, dout):
+    """Gradients of sum(dout * out) through Eq. 8, out = clip(r) * o_softmax + (1 - clip(r)) * linear attention.
+    Returns float64 (dq, dk, dv, dWq, dWk, d_o_softmax, dr); dr is a Python float."""
+    q, k, v, Wq, Wk, B, H, n, d, per_head = _prep(q, k, v, Wq, Wk)
+    g, a = _f32(dout), _f32(o_softmax)
+    assert g.shape == q.shape and a.shape == q.shape
+    dq, dk, dv, da = (np.empty(q.shape, dtype=np.float64) for _ in range(4))
+    dWq, dWk = (np.empty(Wq.shape, dtype=np.float64) for _ in range(2))
+    dr = ctypes.c_double(0.0)
+    F, D = ctypes.c_float, ctypes.c_double
+    rc = _load().linattn_ref_backward_mixed(_ptr(q, F), _ptr(k, F), _ptr(v, F), _ptr(Wq, F), _ptr(Wk, F), _ptr(a, F), float(r),
+                                            _ptr(g, F), B * H, H, n, d, per_head, _ptr(dq, D), _ptr(dk, D), _ptr(dv, D),
+                                            _ptr(dWq, D), _ptr(dWk, D), _ptr(da, D), ctypes.byref(dr))
+    if rc:
+        raise ValueError("oracle rejected the arguments or ran out of memory")
+    return dq, dk, dv, dWq, dWk, da, float(dr.value)
+
+
+def ref_relu_backward(q, k, v, dout):
+    """Gradients of sum(dout * o) with the ReLU kernel function: float64 (dq, dk, dv)."""
+    q, k, v, g = (_f32(t) for t in (q, k, v, dout))
+    assert q.ndim == 4 and q.shape == k.shape == v.shape == g.shape
+    B, H, n, d = q.shape
+    dq, dk, dv = (np.empty(q.shape, dtype=np.float64) for _ in range(3))
+    F, D = ctypes.c_float, ctypes.c_double
+    rc = _load().linattn_ref_relu_backward(_ptr(q, F), _ptr(k, F), _ptr(v, F), _ptr(g, F), B * H, n, d,
+                                           _ptr(dq, D), _ptr(dk, D), _ptr(dv, D))
+    if rc:
+        raise ValueError("oracle rejected the arguments or ran out of memory")
+    return dq, dk, dv
 
 
 def ref_relu_quadratic(q, k, v, rows=None) -> np.ndarray:

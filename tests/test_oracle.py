@@ -426,3 +426,103 @@ def test_backward_closed_forms():
     for z in (dq, dk, dWq, dWk):
         assert np.abs(z).max() <= 1e-12
     np.testing.assert_allclose(dv, g.astype(np.float64), rtol=1e-13, atol=1e-15)
+
+
+# ---- gradients through Eq. 8 (mixed attention) and with the ReLU kernel function ------------------------------
+
+@pytest.mark.parametrize("r", [0.3, 0.0, 1.0, -0.2, 1.4])
+def test_mixed_backward_matches_autograd_of_an_independent_forward(r):
+    """torch fp64 autograd through clamp(r) * a + (1 - clamp(r)) * [Eq. 5, left form]: every gradient, the one of the
+    softmax branch's output and the one of r included.  torch's clamp passes the gradient on the closed interval
+    [0, 1] (ends included) and blocks it outside, which is the reading the oracle states."""
+    B, H, n, d = 2, 2, 7, 8
+    q, k, v, Wq, Wk = _rand(B, H, n, d, seed=80)
+    rng = np.random.default_rng(81)
+    g = rng.standard_normal((B, H, n, d)).astype(np.float32)
+    a = rng.standard_normal((B, H, n, d)).astype(np.float32)
+    t = [torch.from_numpy(x).double().requires_grad_(True) for x in (q, k, v, Wq, Wk, a)]
+    rt = torch.tensor(r, dtype=torch.float64, requires_grad=True)
+    rc = torch.clamp(rt, 0.0, 1.0)
+    out = rc * t[5] + (1.0 - rc) * _torch_forward(*t[:5])
+    (out * torch.from_numpy(g).double()).sum().backward()
+    got = oracle.ref_backward_mixed(q, k, v, Wq, Wk, a, r, g)
+    for name, x, y in zip(("dq", "dk", "dv", "dWq", "dWk", "da"), got[:6], t):
+        np.testing.assert_allclose(x, y.grad.numpy(), rtol=1e-9, atol=1e-12, err_msg=name)
+    np.testing.assert_allclose(got[6], rt.grad.item(), rtol=1e-9, atol=1e-12)
+    if r < 0.0 or r > 1.0:
+        assert got[6] == 0.0
+
+
+def test_mixed_backward_special_cases_and_central_difference_in_r():
+    B, H, n, d = 1, 2, 6, 4
+    q, k, v, Wq, Wk = _rand(B, H, n, d, seed=82)
+    rng = np.random.default_rng(83)
+    g = rng.standard_normal((B, H, n, d)).astype(np.float32)
+    a = rng.standard_normal((B, H, n, d)).astype(np.float32)
+    # r = 0: the layer IS the linear branch
+    plain = oracle.ref_backward(q, k, v, Wq, Wk, g)
+    at0 = oracle.ref_backward_mixed(q, k, v, Wq, Wk, a, 0.0, g)
+    for x, y in zip(plain, at0[:5]):
+        np.testing.assert_array_equal(x, y)
+    assert np.abs(at0[5]).max() == 0.0
+    # r = 1: nothing reaches the linear branch, the softmax branch gets dout unchanged
+    at1 = oracle.ref_backward_mixed(q, k, v, Wq, Wk, a, 1.0, g)
+    for x in at1[:5]:
+        assert np.abs(x).max() == 0.0
+    np.testing.assert_array_equal(at1[5], g.astype(np.float64))
+    # dr against a central difference of the pinned forward (ref_mix of ref_linear); the blend is affine in r^
+    lin = oracle.ref_linear(q, k, v, Wq, Wk)
+    h = 2.0 ** -12
+    fd = ((oracle.ref_mix(a, lin, 0.4 + h) - oracle.ref_mix(a, lin, 0.4 - h)) * g.astype(np.float64)).sum() / (2 * h)
+    dr = oracle.ref_backward_mixed(q, k, v, Wq, Wk, a, 0.4, g)[6]
+    assert abs(fd - dr) <= 1e-8 * max(1.0, abs(dr))
+    # and linear in (1 - r^) for everything that passes through the linear branch
+    half = oracle.ref_backward_mixed(q, k, v, Wq, Wk, a, 0.5, g)
+    for x, y in zip(plain, half[:5]):
+        np.testing.assert_allclose(0.5 * x, y, rtol=1e-13, atol=1e-15)
+
+
+def _torch_relu_forward(q, k, v):
+    a = torch.einsum("bhif,bhjf->bhij", torch.relu(q), torch.relu(k))
+    return torch.einsum("bhij,bhjd->bhid", a / a.sum(-1, keepdim=True), v)
+
+
+@pytest.mark.parametrize("B,H,n,d", [(1, 1, 5, 4), (2, 3, 11, 8)])
+def test_relu_backward_matches_autograd_and_central_differences(B, H, n, d):
+    q, k, v = _qkv(B, H, n, d, seed=90 + n)
+    g = np.random.default_rng(91).standard_normal((B, H, n, d)).astype(np.float32)
+    t = [torch.from_numpy(x).double().requires_grad_(True) for x in (q, k, v)]
+    (_torch_relu_forward(*t) * torch.from_numpy(g).double()).sum().backward()
+    got = oracle.ref_relu_backward(q, k, v, g)
+    for name, x, y in zip(("dq", "dk", "dv"), got, t):
+        np.testing.assert_allclose(x, y.grad.numpy(), rtol=1e-9, atol=1e-12, err_msg=name)
+    # central differences of the pinned ReLU forward oracle (away from the kink: |x| > 2h for the sampled entries)
+    h = 2.0 ** -10
+    rng = np.random.default_rng(92)
+    args = [q, k, v]
+    for a_i, (arr, grad) in enumerate(zip(args, got)):
+        done = 0
+        while done < 5:
+            idx = tuple(rng.integers(0, s) for s in arr.shape)
+            if abs(arr[idx]) <= 4 * h:
+                continue
+            plus, minus = [x.copy() for x in args], [x.copy() for x in args]
+            plus[a_i][idx] += h
+            minus[a_i][idx] -= h
+            fd = ((oracle.ref_relu_linear(*plus) - oracle.ref_relu_linear(*minus)) * g.astype(np.float64)).sum() / (2 * h)
+            assert abs(fd - grad[idx]) <= 1e-5 * max(1.0, abs(grad[idx])), (a_i, idx, fd, grad[idx])
+            done += 1
+
+
+def test_relu_backward_closed_forms():
+    """Negative entries of q and k get no gradient; n = 1 returns v, so dv = dO and dq = dk = 0."""
+    rng = np.random.default_rng(93)
+    q, k, v = (rng.standard_normal((1, 2, 9, 8)).astype(np.float32) for _ in range(3))
+    g = rng.standard_normal((1, 2, 9, 8)).astype(np.float32)
+    dq, dk, dv = oracle.ref_relu_backward(q, k, v, g)
+    assert np.abs(dq[q <= 0]).max() == 0.0 and np.abs(dk[k <= 0]).max() == 0.0
+    assert np.abs(dq[q > 0]).min() > 0.0
+    q1, k1, v1, g1 = (x[:, :, :1].copy() for x in (np.abs(q) + 0.1, np.abs(k) + 0.1, v, g))
+    dq, dk, dv = oracle.ref_relu_backward(q1, k1, v1, g1)
+    assert np.abs(dq).max() <= 1e-12 and np.abs(dk).max() <= 1e-12
+    np.testing.assert_allclose(dv, g1.astype(np.float64), rtol=1e-13, atol=1e-15)
