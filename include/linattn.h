@@ -51,8 +51,9 @@ typedef enum {
                                kernel function of the paper's comparison across kernel functions, phi(x) = max(x, 0)
                                element by element on the d features of the head: no weights (set_feature_map is not
                                needed), no epsilon (a query whose phi is orthogonal to every key's gives a non-finite
-                               row).  Applies to linattn_forward, _mixed and _host; linattn_backward then returns
-                               UNSUPPORTED */
+                               row).  Applies to every entry point; the gradients (linattn_backward, _backward_mixed) then
+                               run on the CUDA-core kernels, have no weight gradients (dWq, dWk are ignored and may be
+                               NULL), and take d phi / d x = 1 where x > 0, else 0 */
     LINATTN_OPT_REUSE_STATE = 6, /* 1 = linattn_backward (tensor-core path) takes S and z from the workspace instead of
                                recomputing them when the most recent state-producing call on this context was a forward
                                (or backward) on the same k and v POINTERS, B, n and layout, with the same feature map.
@@ -146,6 +147,27 @@ linattn_status linattn_forward_mixed(linattn_ctx* ctx, const void* q, const void
 linattn_status linattn_backward(linattn_ctx* ctx, const void* q, const void* k, const void* v, const void* dout,
                                 void* dq, void* dk, void* dv, float* dWq, float* dWk, int per_head,
                                 int B, int H, int n, int d, linattn_dtype dtype, void* stream);
+
+/*
+ * Gradients through mixed attention, Eq. 8: out = r^ * o_softmax + (1 - r^) * [Eq. 5 applied to q, k, v], r^ = clip(r, 0, 1),
+ * the layer that the objective of Eq. 14 is back-propagated through while softmax attention is being transferred to
+ * linear attention.  Given dout = dL/d(out):
+ *   dq, dk, dv, dWq, dWk : the gradients of linattn_backward for the incoming gradient (1 - r^) * dout (the factor is
+ *                          applied inside the kernels, to the fp32 accumulators: nothing is rounded twice)
+ *   d_o_softmax          : r^ * dout, the gradient that reaches the softmax branch (device, shape and type of dout;
+ *                          may be NULL: not computed); must not overlap any other argument
+ *   dr                   : device, ONE float, 4-byte aligned: dL/dr = sum dout * (o_softmax - linear attention) if
+ *                          0 <= r <= 1, else 0.  (The paper clips r and says nothing of the clip's derivative; it is taken
+ *                          as 1 on the closed interval: every r starts at 1, and with a zero derivative there it could
+ *                          never move.)  Summed in a fixed order: bit-reproducible.
+ *   o_softmax            : the softmax branch's output as given to linattn_forward_mixed (read-only)
+ * Everything else (layouts, the two sets of kernels, workspace, errors) as for linattn_backward; r = NaN is INVALID_ARG.
+ */
+linattn_status linattn_backward_mixed(linattn_ctx* ctx, const void* q, const void* k, const void* v,
+                                      const void* o_softmax, float r, const void* dout,
+                                      void* dq, void* dk, void* dv, float* dWq, float* dWk, int per_head,
+                                      void* d_o_softmax, float* dr,
+                                      int B, int H, int n, int d, linattn_dtype dtype, void* stream);
 
 /*
  * The same operation on HOST buffers (pageable or pinned; pinned buffers let the copies overlap).  For the

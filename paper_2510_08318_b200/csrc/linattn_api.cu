@@ -69,6 +69,7 @@ struct linattn_ctx {
     float* bwd_part_state = nullptr;  // [partial_slots][d*d + d]  per-block sums of dS, dz
     float* bwd_part_w = nullptr;      // [partial_slots][d*d/2]    per-block sums of dW
     float* bwd_dstate = nullptr;      // [max_B*H][d*d + d]        dS, dz
+    float* bwd_part_dr = nullptr;     // [partial_slots]           per-block sums of dout . (a - o), the terms of Eq. 8's dL/dr
     __nv_bfloat16* bwd_img[3] = {nullptr, nullptr, nullptr};   // tensor-core backward: lo image of S, hi and lo images of dS
     bool bwd_ready = false;           // every allocation above succeeded
     // host-call staging and its pipeline: copies in, compute and copies out run on three streams, one (b,h) at a time
@@ -244,9 +245,18 @@ linattn_status launch_simt(linattn_ctx* c, const void* q, const void* k, const v
 
 // Gradients on the CUDA-core kernels: S, z as in the forward, then the query side (dq, dS, dz, dW_q), then the key
 // side (dk, dv, dW_k).
+// What Eq. 8 adds to a backward call (all unused for the plain operator: lin_scale = 1, the rest null).
+struct MixGrad {
+    const void* a = nullptr;   // output of the softmax branch
+    float lin_scale = 1.f;     // 1 - r^: factor of the gradient that reaches the linear branch
+    int r_in_range = 0;        // 0 <= r <= 1: the clip passes the gradient of r
+    float* dr = nullptr;       // device, one float
+};
+
 template <typename T, int D>
 linattn_status launch_backward_simt(linattn_ctx* c, const void* q, const void* k, const void* v, const void* dout, void* dq,
-                                    void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int n, cudaStream_t st)
+                                    void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int n, cudaStream_t st,
+                                    const MixGrad& mg)
 {
     const long long G = (long long)B * c->H;
     int splits = choose_splits(G, n, c->opt_splits);
@@ -270,31 +280,45 @@ linattn_status launch_backward_simt(linattn_ctx* c, const void* q, const void* k
     const double tensor_bytes = (double)G * n * D * sizeof(T);
     const dim3 grid((unsigned)blocks, (unsigned)G);
     prof_begin(c, st);
+    const int relu = c->opt_phi;
     kside_simt<T, D><<<dim3(splits, (unsigned)G), kSimtThreads, kside_simt_smem<D>(), st>>>(
-        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, as, 0);
+        (const T*)k, (const T*)v, c->Wk, c->partial, c->H, n, chunk, as, relu);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_simt", 2.0 * tensor_bytes);
     combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->partial, c->state, splits, E);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_state", 0.0);
     qside_bwd<T, D><<<grid, kSimtThreads, bwd_smem<D>(), st>>>((const T*)q, (const T*)dout, c->Wq, c->state, (T*)dq,
-                                                              c->bwd_part_state, c->bwd_part_w, c->H, n, as);
+                                                              c->bwd_part_state, c->bwd_part_w, c->H, n, as, relu, (const T*)mg.a,
+                                                              mg.lin_scale, mg.dr ? c->bwd_part_dr : nullptr);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "qside_bwd", 3.0 * tensor_bytes);
+    int launches = 5;
     combine_state<<<dim3((E + 255) / 256, (unsigned)G), 256, 0, st>>>(c->bwd_part_state, c->bwd_dstate, (int)blocks, E);
     LA_CUDA(c, cudaGetLastError());
     const dim3 wgrid((DM + 255) / 256, per_head ? (unsigned)c->H : 1u);
-    combine_wgrad<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWq, (int)blocks, (int)G, c->H, DM, per_head);
-    LA_CUDA(c, cudaGetLastError());
+    if (!relu) {   // the ReLU kernel function has no weights
+        combine_wgrad<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWq, (int)blocks, (int)G, c->H, DM, per_head);
+        LA_CUDA(c, cudaGetLastError());
+        ++launches;
+    }
+    if (mg.dr) {
+        combine_dr<<<1, 32, 0, st>>>(c->bwd_part_dr, (int)(G * blocks), mg.r_in_range, mg.dr);
+        LA_CUDA(c, cudaGetLastError());
+        ++launches;
+    }
     prof_mark(c, st, "combine_dstate_dWq", 0.0);
     kside_bwd<T, D><<<grid, kSimtThreads, bwd_smem<D>(), st>>>((const T*)k, (const T*)v, c->Wk, c->bwd_dstate, (T*)dk, (T*)dv,
-                                                              c->bwd_part_w, c->H, n, as);
+                                                              c->bwd_part_w, c->H, n, as, relu);
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "kside_bwd", 4.0 * tensor_bytes);
-    combine_wgrad<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWk, (int)blocks, (int)G, c->H, DM, per_head);
-    LA_CUDA(c, cudaGetLastError());
+    if (!relu) {
+        combine_wgrad<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWk, (int)blocks, (int)G, c->H, DM, per_head);
+        LA_CUDA(c, cudaGetLastError());
+        ++launches;
+    }
     prof_mark(c, st, "combine_dWk", 0.0);
-    c->last_launches = 7;
+    c->last_launches = launches;
     return LINATTN_OK;
 }
 
@@ -450,7 +474,8 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
 // Gradients on the tensor-core kernels (bf16, d = 128, bf16 feature-map weights): S, z by the forward's key-side
 // kernels, then the query side (dq; dS, dz, dW_q records), the combines, and the key side (dk, dv; dW_k records).
 linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, const void* v, const void* dout, void* dq,
-                                  void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int n, cudaStream_t st)
+                                  void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int n, cudaStream_t st,
+                                  const MixGrad& mg)
 {
     using namespace linattn::tc;
     const long long G = (long long)B * c->H;
@@ -491,12 +516,13 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
         snprintf(c->err_text, sizeof(c->err_text), "cuTensorMapEncodeTiled failed");
         return LINATTN_ERR_CUDA;
     }
-    const void* k_q[2] = {(const void*)qside_bwd_tc<0>, (const void*)qside_bwd_tc<1>};
+    const void* k_q[2][2] = {{(const void*)qside_bwd_tc<0, 0>, (const void*)qside_bwd_tc<0, 1>},
+                             {(const void*)qside_bwd_tc<1, 0>, (const void*)qside_bwd_tc<1, 1>}};   // [layout][Eq. 8 terms]
     const void* k_k[2] = {(const void*)kside_bwd_tc<0>, (const void*)kside_bwd_tc<1>};
     bool& attr_done = c->attr_done[linattn_ctx::kAttrTcBwd];
     if (!attr_done) {
         for (int i = 0; i < 2; ++i) {
-            LA_CUDA(c, cudaFuncSetAttribute(k_q[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemQ));
+            for (int j = 0; j < 2; ++j) LA_CUDA(c, cudaFuncSetAttribute(k_q[i][j], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemQ));
             LA_CUDA(c, cudaFuncSetAttribute(k_k[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBwdSmemK));
         }
         attr_done = true;
@@ -507,6 +533,12 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     a.part_w = c->bwd_part_w;
     a.state = c->state;
     a.err = c->err_word;
+    a.mix_a = (const __nv_bfloat16*)mg.a;
+    a.part_dr = c->bwd_part_dr;
+    a.lin_scale = mg.lin_scale;
+    a.str_token = as.token;
+    a.str_head = as.head;
+    a.str_batch = as.batch;
     a.n = n;
     a.H = c->H;
     a.G = (int)G;
@@ -520,9 +552,14 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     LA_CUDA(c, cudaGetLastError());
     {
         void* p[] = {&tmQ, &tmG, &tmDQ, &tmWq, &tmShi, &tmSlo, &a};
-        LA_CUDA(c, cudaLaunchKernel(k_q[layout], dim3((unsigned)P), dim3(kBwdThreads), p, kBwdSmemQ, st));
+        LA_CUDA(c, cudaLaunchKernel(k_q[layout][mg.dr ? 1 : 0], dim3((unsigned)P), dim3(kBwdThreads), p, kBwdSmemQ, st));
     }
-    prof_mark(c, st, "qside_bwd_tc", 3.0 * tensor_bytes);
+    prof_mark(c, st, "qside_bwd_tc", (mg.dr ? 4.0 : 3.0) * tensor_bytes);
+    if (mg.dr) {
+        combine_dr<<<1, 32, 0, st>>>(c->bwd_part_dr, (int)P, mg.r_in_range, mg.dr);
+        LA_CUDA(c, cudaGetLastError());
+        ++launches;
+    }
     combine_slots<<<dim3((kE + 255) / 256, (unsigned)G), 256, 0, st>>>(c->bwd_part_state, c->bwd_dstate, kE, (int)Tn, T, P);
     LA_CUDA(c, cudaGetLastError());
     hilo_images<<<dim3(kD * kD / 256, (unsigned)G), 256, 0, st>>>(c->bwd_dstate, c->bwd_img[1], c->bwd_img[2]);
@@ -670,6 +707,7 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->bwd_part_state);
     cudaFree(c->bwd_part_w);
     cudaFree(c->bwd_dstate);
+    cudaFree(c->bwd_part_dr);
     for (void* p : c->bwd_img) cudaFree(p);
     for (void* p : c->stage) cudaFree(p);
     if (c->copy_in) cudaStreamDestroy(c->copy_in);
@@ -791,27 +829,39 @@ linattn_status linattn_forward_mixed(linattn_ctx* c, const void* q, const void* 
     return forward_impl(c, q, k, v, out, o_softmax, r, B, H, n, d, dtype, stream);
 }
 
-linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, const void* v, const void* dout, void* dq,
-                                void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int H, int n, int d,
-                                linattn_dtype dtype, void* stream)
+// Shared by linattn_backward (a == NULL) and linattn_backward_mixed.
+static linattn_status backward_impl(linattn_ctx* c, const void* q, const void* k, const void* v, const void* a, float r,
+                                    const void* dout, void* dq, void* dk, void* dv, float* dWq, float* dWk, int per_head,
+                                    void* d_a, float* dr, int B, int H, int n, int d, linattn_dtype dtype, void* stream)
 {
-    if (!dout || !dk || !dv || !dWq || !dWk) return LINATTN_ERR_INVALID_ARG;
-    if (c && c->opt_phi != 0) return LINATTN_ERR_UNSUPPORTED;   // gradients exist for the feature map of Eq. 6 only
+    if (!dout || !dk || !dv) return LINATTN_ERR_INVALID_ARG;
+    const bool relu = c && c->opt_phi != 0;
+    if (!relu && (!dWq || !dWk)) return LINATTN_ERR_INVALID_ARG;   // the ReLU kernel function has no weights: its dWq, dWk are ignored
     linattn_status s = check_forward_args(c, q, k, v, dq, B, H, n, d, dtype);
     if (s != LINATTN_OK) return s;
-    const void* ins[4] = {q, k, v, dout};
-    void* outs[3] = {dq, dk, dv};
+    const void* ins[5] = {q, k, v, dout, a};
+    void* outs[4] = {dq, dk, dv, d_a};
     const size_t bytes = (size_t)B * H * n * d * elem_size(dtype);
     for (const void* p : ins)
-        if (misaligned16(p)) return LINATTN_ERR_INVALID_ARG;
-    for (int i = 0; i < 3; ++i) {
+        if (p && misaligned16(p)) return LINATTN_ERR_INVALID_ARG;
+    for (int i = 0; i < 4; ++i) {
+        if (!outs[i]) continue;
         if (misaligned16(outs[i])) return LINATTN_ERR_INVALID_ARG;
         for (const void* p : ins)
-            if (overlaps(outs[i], p, bytes)) return LINATTN_ERR_INVALID_ARG;
+            if (p && overlaps(outs[i], p, bytes)) return LINATTN_ERR_INVALID_ARG;
         for (int j = 0; j < i; ++j)
-            if (overlaps(outs[i], outs[j], bytes)) return LINATTN_ERR_INVALID_ARG;
+            if (outs[j] && overlaps(outs[i], outs[j], bytes)) return LINATTN_ERR_INVALID_ARG;
     }
-    if (misaligned16(dWq) || misaligned16(dWk) || dWq == dWk) return LINATTN_ERR_INVALID_ARG;
+    if (!relu && (misaligned16(dWq) || misaligned16(dWk) || dWq == dWk)) return LINATTN_ERR_INVALID_ARG;
+    MixGrad mg;
+    if (a) {
+        if (!dr || (reinterpret_cast<uintptr_t>(dr) & 3u) || !(r == r)) return LINATTN_ERR_INVALID_ARG;
+        const float rc = r < 0.f ? 0.f : (r > 1.f ? 1.f : r);   // footnote to Eq. 8: r is clipped into [0, 1]
+        mg.a = a;
+        mg.lin_scale = 1.f - rc;
+        mg.r_in_range = (r >= 0.f && r <= 1.f) ? 1 : 0;   // the clip passes r's gradient on the closed interval
+        mg.dr = dr;
+    }
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (!c->bwd_ready) {
@@ -820,6 +870,7 @@ linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, co
         cudaError_t e = cudaMalloc(&c->bwd_part_state, sizeof(float) * E * (size_t)c->partial_slots);
         if (e == cudaSuccess) e = cudaMalloc(&c->bwd_part_w, sizeof(float) * (size_t)d * (d / 2) * (size_t)c->partial_slots);
         if (e == cudaSuccess) e = cudaMalloc(&c->bwd_dstate, sizeof(float) * E * G);
+        if (e == cudaSuccess) e = cudaMalloc(&c->bwd_part_dr, sizeof(float) * (size_t)c->partial_slots);
         if (d == 128)
             for (__nv_bfloat16*& p : c->bwd_img)
                 if (e == cudaSuccess) e = cudaMalloc(&p, sizeof(__nv_bfloat16) * (size_t)d * d * G);
@@ -828,7 +879,8 @@ linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, co
             cudaFree(c->bwd_part_state);
             cudaFree(c->bwd_part_w);
             cudaFree(c->bwd_dstate);
-            c->bwd_part_state = c->bwd_part_w = c->bwd_dstate = nullptr;
+            cudaFree(c->bwd_part_dr);
+            c->bwd_part_state = c->bwd_part_w = c->bwd_dstate = c->bwd_part_dr = nullptr;
             for (__nv_bfloat16*& p : c->bwd_img) {
                 cudaFree(p);
                 p = nullptr;
@@ -839,20 +891,48 @@ linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, co
     }
     c->last_B = B;
     const int ph = per_head ? 1 : 0;
-    const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && c->map_is_bf16);
+    // the gradient that reaches the softmax branch, r^ * dout: element by element, whatever the layout
+    if (a && d_a) {
+        const size_t count = (size_t)B * H * n * d;
+        const unsigned blocks = (unsigned)((count + 256 * 8 - 1) / (256 * 8) < 1184 * 4 ? (count + 256 * 8 - 1) / (256 * 8) : 1184 * 4);
+        if (dtype == LINATTN_BF16) scale_copy<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dout, (__nv_bfloat16*)d_a, count, 1.f - mg.lin_scale);
+        else scale_copy<float><<<blocks, 256, 0, st>>>((const float*)dout, (float*)d_a, count, 1.f - mg.lin_scale);
+        LA_CUDA(c, cudaGetLastError());
+    }
+    // tensor-core kernels: Eq. 6 with bf16 weights, bf16 activations, d = 128; everything else on the CUDA cores
+    const bool tc_ok = (dtype == LINATTN_BF16 && d == 128 && c->map_is_bf16 && !relu);
     if (c->opt_path == 2 && !tc_ok) return LINATTN_ERR_UNSUPPORTED;
+    linattn_status res;
     if (tc_ok && c->opt_path != 1) {
         c->state_transposed = true;
-        return launch_backward_tc(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
+        res = launch_backward_tc(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st, mg);
+    } else {
+        c->state_transposed = false;
+        c->state_key.valid = false;
+        if (dtype == LINATTN_BF16)
+            res = d == 128 ? launch_backward_simt<__nv_bfloat16, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st, mg)
+                           : launch_backward_simt<__nv_bfloat16, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st, mg);
+        else
+            res = d == 128 ? launch_backward_simt<float, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st, mg)
+                           : launch_backward_simt<float, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st, mg);
     }
-    c->state_transposed = false;
-    c->state_key.valid = false;
-    if (dtype == LINATTN_BF16) {
-        return d == 128 ? launch_backward_simt<__nv_bfloat16, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st)
-                        : launch_backward_simt<__nv_bfloat16, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
-    }
-    return d == 128 ? launch_backward_simt<float, 128>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st)
-                    : launch_backward_simt<float, 64>(c, q, k, v, dout, dq, dk, dv, dWq, dWk, ph, B, n, st);
+    if (res == LINATTN_OK && a && d_a) c->last_launches += 1;
+    return res;
+}
+
+linattn_status linattn_backward(linattn_ctx* c, const void* q, const void* k, const void* v, const void* dout, void* dq,
+                                void* dk, void* dv, float* dWq, float* dWk, int per_head, int B, int H, int n, int d,
+                                linattn_dtype dtype, void* stream)
+{
+    return backward_impl(c, q, k, v, nullptr, 0.f, dout, dq, dk, dv, dWq, dWk, per_head, nullptr, nullptr, B, H, n, d, dtype, stream);
+}
+
+linattn_status linattn_backward_mixed(linattn_ctx* c, const void* q, const void* k, const void* v, const void* o_softmax, float r,
+                                      const void* dout, void* dq, void* dk, void* dv, float* dWq, float* dWk, int per_head,
+                                      void* d_o_softmax, float* dr, int B, int H, int n, int d, linattn_dtype dtype, void* stream)
+{
+    if (!o_softmax) return LINATTN_ERR_INVALID_ARG;
+    return backward_impl(c, q, k, v, o_softmax, r, dout, dq, dk, dv, dWq, dWk, per_head, d_o_softmax, dr, B, H, n, d, dtype, stream);
 }
 
 linattn_status linattn_forward_host(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B,

@@ -60,11 +60,12 @@ template <int D>
 __device__ __forceinline__ void bwd_load_constants(const BwdSmem<D>& s, const float* __restrict__ Wg, const float* __restrict__ state)
 {
     constexpr int M = D / 2, P = BwdShape<D>::P;
-    for (int e = threadIdx.x; e < D * M; e += kSimtThreads) {
-        const float w = Wg[e];
-        s.W[e] = w;
-        s.Wt[(e % M) * D + e / M] = w;
-    }
+    if (Wg)   // the ReLU kernel function has no weights
+        for (int e = threadIdx.x; e < D * M; e += kSimtThreads) {
+            const float w = Wg[e];
+            s.W[e] = w;
+            s.Wt[(e % M) * D + e / M] = w;
+        }
     for (int e = threadIdx.x; e < D * D; e += kSimtThreads) s.A[(e / D) * P + e % D] = state[e];
     for (int e = threadIdx.x; e < D; e += kSimtThreads) s.a[e] = state[D * D + e];
 }
@@ -199,7 +200,37 @@ __device__ __forceinline__ void dx_store(const BwdSmem<D>& s, T* __restrict__ ds
     }
 }
 
+// ReLU kernel function, phi(x) = max(x, 0): dx[t][c] = dphi[t][c] where x[t][c] > 0, else 0 (no weights, no softmax).
+template <typename T, int D>
+__device__ __forceinline__ void relu_dx_store(const BwdSmem<D>& s, T* __restrict__ dst, long long row_stride, int valid)
+{
+    constexpr int P = BwdShape<D>::P;
+    for (int e = threadIdx.x; e < kSimtTokens * D; e += kSimtThreads) {
+        const int r = e / D, c = e % D;
+        if (r < valid) store_out(&dst[(size_t)r * row_stride + c], s.x[r * P + c] > 0.f ? s.dphi[r * P + c] : 0.f);
+    }
+}
+
+// Sum of one value per thread over the block in a fixed order (thread 0 adds them up); every thread gets the result.
+__device__ __forceinline__ float block_sum_ordered(float v, float* scratch)
+{
+    __syncthreads();
+    scratch[threadIdx.x] = v;
+    __syncthreads();
+    float acc = 0.f;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kSimtThreads; ++i) acc += scratch[i];
+        scratch[0] = acc;
+    }
+    __syncthreads();
+    return scratch[0];
+}
+
 // grid = (blocks_per_group, G).  Block x handles chunks x, x + gridDim.x, ... of kSimtTokens tokens.
+//   relu      : 1 = the ReLU kernel function instead of Eq. 6 (no weights: Wq is NULL, part_w is not written)
+//   mix_a, lin_scale, part_dr : Eq. 8.  The gradient that reaches the linear branch is lin_scale * dout (lin_scale = 1 - r^);
+//               when mix_a (the softmax branch's output, laid out like q) is given, part_dr [G][gridDim.x] receives the
+//               block's sum of dout . (a - o), the terms of dL/dr
 //   state     : [G][D*D + D]  S row-major [f][c], then z   (from the forward's key side)
 //   dq        : same layout and type as q
 //   part_state: [G][gridDim.x][D*D + D]  the block's sums of dS ([f][c]) and dz
@@ -207,17 +238,20 @@ __device__ __forceinline__ void dx_store(const BwdSmem<D>& s, T* __restrict__ ds
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 qside_bwd(const T* __restrict__ q, const T* __restrict__ dout, const float* __restrict__ Wq, const float* __restrict__ state,
-          T* __restrict__ dq, float* __restrict__ part_state, float* __restrict__ part_w, int H, int n, ActStrides st)
+          T* __restrict__ dq, float* __restrict__ part_state, float* __restrict__ part_w, int H, int n, ActStrides st, int relu,
+          const T* __restrict__ mix_a, float lin_scale, float* __restrict__ part_dr)
 {
     using Sh = BwdShape<D>;
     constexpr int M = Sh::M, P = Sh::P, CG = Sh::CG, FB = Sh::FB, CB = Sh::CB;
     extern __shared__ __align__(16) float smem[];
     const BwdSmem<D> s(smem);
     const int g = blockIdx.y, tid = threadIdx.x;
-    bwd_load_constants<D>(s, Wq + (size_t)(g % H) * D * M, state + (size_t)g * (D * D + D));
+    bwd_load_constants<D>(s, relu ? nullptr : Wq + (size_t)(g % H) * D * M, state + (size_t)g * (D * D + D));
 
     const T* qg = q + st.base(g, H);
     const T* gg = dout + st.base(g, H);
+    const T* ag = mix_a ? mix_a + st.base(g, H) : nullptr;
+    float dr_acc = 0.f;   // this thread's share of sum dout . (a - o)
     T* dqg = dq + st.base(g, H);
     const int tt = tid >> 3, cg = tid & 7;
     const int fy = tid >> 4, cx = tid & 15;
@@ -242,7 +276,8 @@ qside_bwd(const T* __restrict__ q, const T* __restrict__ dout, const float* __re
         load_chunk<T, D>(qg + (size_t)t * st.token, st.token, s.x, valid);
         load_chunk<T, D>(gg + (size_t)t * st.token, st.token, s.y, valid);
         __syncthreads();
-        feature_map_chunk<D>(s.x, s.W, s.phi, valid);   // rows past `valid` get phi = 0
+        if (relu) relu_chunk<D>(s.x, s.phi, valid);
+        else feature_map_chunk<D>(s.x, s.W, s.phi, valid);   // rows past `valid` get phi = 0
         __syncthreads();
         {
             // forward quantities of the token, then dnum (over dO in place) and dden
@@ -252,6 +287,7 @@ qside_bwd(const T* __restrict__ q, const T* __restrict__ dout, const float* __re
 #pragma unroll 8
             for (int f = 0; f < D; ++f) den = fmaf(s.phi[tt * P + f], s.a[f], den);
             const float inv = (tt < valid) ? 1.f / den : 0.f;
+            const float sc = lin_scale * inv;   // the linear branch's incoming gradient is lin_scale * dO
             float go = 0.f;
 #pragma unroll
             for (int r = 0; r < CG; ++r) {
@@ -261,12 +297,20 @@ qside_bwd(const T* __restrict__ q, const T* __restrict__ dout, const float* __re
                 go = fmaf(gv.y, num[r][1] * inv, go);
                 go = fmaf(gv.z, num[r][2] * inv, go);
                 go = fmaf(gv.w, num[r][3] * inv, go);
-                gv.x *= inv; gv.y *= inv; gv.z *= inv; gv.w *= inv;
+                if (ag && tt < valid) {   // Eq. 8: dO . a, the softmax branch's part of dL/dr
+                    const T* ap = ag + (size_t)(t + tt) * st.token + r * 32 + cg * 4;
+                    dr_acc = fmaf(gv.x, to_f32(ap[0]), dr_acc);
+                    dr_acc = fmaf(gv.y, to_f32(ap[1]), dr_acc);
+                    dr_acc = fmaf(gv.z, to_f32(ap[2]), dr_acc);
+                    dr_acc = fmaf(gv.w, to_f32(ap[3]), dr_acc);
+                }
+                gv.x *= sc; gv.y *= sc; gv.z *= sc; gv.w *= sc;
                 *gp = gv;
             }
+            dr_acc -= go;   // ... minus dO . o, each thread its own columns' share
 #pragma unroll
             for (int o = 1; o < 8; o <<= 1) go += __shfl_xor_sync(0xffffffffu, go, o);
-            if (cg == 0) s.dd[tt] = -go * inv;
+            if (cg == 0) s.dd[tt] = -go * sc;
         }
         __syncthreads();
         dphi_chunk<D>(s, s.dd);
@@ -289,13 +333,21 @@ qside_bwd(const T* __restrict__ q, const T* __restrict__ dout, const float* __re
             }
         }
         __syncthreads();
-        du_chunk<D>(s);
-        __syncthreads();
-        dx_store<T, D>(s, dqg + (size_t)t * st.token, st.token, valid);
-        dw_accumulate<D>(s, dw);
+        if (relu) {
+            relu_dx_store<T, D>(s, dqg + (size_t)t * st.token, st.token, valid);
+        } else {
+            du_chunk<D>(s);
+            __syncthreads();
+            dx_store<T, D>(s, dqg + (size_t)t * st.token, st.token, valid);
+            dw_accumulate<D>(s, dw);
+        }
     }
 
     const size_t slot = (size_t)g * gridDim.x + blockIdx.x;
+    if (part_dr) {
+        const float total = block_sum_ordered(dr_acc, s.phi);   // the token tiles are free now
+        if (tid == 0) part_dr[slot] = total;
+    }
     float* ps = part_state + slot * (D * D + D);
 #pragma unroll
     for (int a = 0; a < FB; ++a) {
@@ -305,7 +357,7 @@ qside_bwd(const T* __restrict__ q, const T* __restrict__ dout, const float* __re
             *reinterpret_cast<float4*>(&ps[f * D + (b / 4) * 64 + cx * 4]) = *reinterpret_cast<float4*>(&dS[a][b]);
         if (cx == 0) ps[D * D + f] = dz[a];
     }
-    dw_store<D>(part_w + slot * (D * M), dw);
+    if (!relu) dw_store<D>(part_w + slot * (D * M), dw);
 }
 
 // grid = (blocks_per_group, G).
@@ -315,14 +367,14 @@ qside_bwd(const T* __restrict__ q, const T* __restrict__ dout, const float* __re
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 kside_bwd(const T* __restrict__ k, const T* __restrict__ v, const float* __restrict__ Wk, const float* __restrict__ dstate,
-          T* __restrict__ dk, T* __restrict__ dv, float* __restrict__ part_w, int H, int n, ActStrides st)
+          T* __restrict__ dk, T* __restrict__ dv, float* __restrict__ part_w, int H, int n, ActStrides st, int relu)
 {
     using Sh = BwdShape<D>;
     constexpr int M = Sh::M, P = Sh::P, CG = Sh::CG;
     extern __shared__ __align__(16) float smem[];
     const BwdSmem<D> s(smem);
     const int g = blockIdx.y, tid = threadIdx.x;
-    bwd_load_constants<D>(s, Wk + (size_t)(g % H) * D * M, dstate + (size_t)g * (D * D + D));
+    bwd_load_constants<D>(s, relu ? nullptr : Wk + (size_t)(g % H) * D * M, dstate + (size_t)g * (D * D + D));
 
     const T* kg = k + st.base(g, H);
     const T* vg = v + st.base(g, H);
@@ -344,7 +396,8 @@ kside_bwd(const T* __restrict__ k, const T* __restrict__ v, const float* __restr
         load_chunk<T, D>(kg + (size_t)t * st.token, st.token, s.x, valid);
         load_chunk<T, D>(vg + (size_t)t * st.token, st.token, s.y, valid);
         __syncthreads();
-        feature_map_chunk<D>(s.x, s.W, s.phi, valid);
+        if (relu) relu_chunk<D>(s.x, s.phi, valid);
+        else feature_map_chunk<D>(s.x, s.W, s.phi, valid);
         __syncthreads();
         dphi_chunk<D>(s, nullptr);
         {
@@ -359,12 +412,16 @@ kside_bwd(const T* __restrict__ k, const T* __restrict__ v, const float* __restr
             }
         }
         __syncthreads();
-        du_chunk<D>(s);
-        __syncthreads();
-        dx_store<T, D>(s, dkg + (size_t)t * st.token, st.token, valid);
-        dw_accumulate<D>(s, dw);
+        if (relu) {
+            relu_dx_store<T, D>(s, dkg + (size_t)t * st.token, st.token, valid);
+        } else {
+            du_chunk<D>(s);
+            __syncthreads();
+            dx_store<T, D>(s, dkg + (size_t)t * st.token, st.token, valid);
+            dw_accumulate<D>(s, dw);
+        }
     }
-    dw_store<D>(part_w + ((size_t)g * gridDim.x + blockIdx.x) * (D * M), dw);
+    if (!relu) dw_store<D>(part_w + ((size_t)g * gridDim.x + blockIdx.x) * (D * M), dw);
 }
 
 // dW[w][e] = sum over the groups g that use weight matrix w (per_head: g % H == w; shared: all g), g ascending, and
@@ -381,6 +438,23 @@ combine_wgrad(const float* __restrict__ part_w, float* __restrict__ dW, int bloc
         for (int b = 0; b < blocks; ++b) acc += p[(size_t)b * DM];
     }
     dW[(size_t)w * DM + e] = acc;
+}
+
+// Eq. 8: dL/dr = sum of the partial sums of dout . (a - o), in index order, if r lies in [0, 1] (the clip passes the
+// gradient on the closed interval), else 0.  One thread.
+static __global__ void combine_dr(const float* __restrict__ part_dr, int count, int in_range, float* __restrict__ dr)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    float acc = 0.f;
+    for (int i = 0; i < count; ++i) acc += part_dr[i];
+    *dr = in_range ? acc : 0.f;
+}
+
+// Eq. 8: the gradient that reaches the softmax branch, d_a = r^ * dout, element by element (any layout: `count` elements).
+template <typename T>
+static __global__ void __launch_bounds__(256) scale_copy(const T* __restrict__ src, T* __restrict__ dst, size_t count, float f)
+{
+    for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < count; i += (size_t)gridDim.x * 256) store_out(&dst[i], f * to_f32(src[i]));
 }
 
 }  // namespace linattn

@@ -38,6 +38,13 @@ struct BwdArgs {
     float* part_w;         // [slots][kWRec]: per (CTA, head) sums of dW as [j][c]
     const float* state;    // [G][kE]: query side: S as [c][f], then z; key side: dS as [c][f], then dz
     uint32_t* err;
+    // Eq. 8 (mixed attention): the linear branch's incoming gradient is lin_scale * dout, lin_scale = 1 - r^ (1 for the
+    // plain operator); with mix_a (the softmax branch's output, laid out like q) the query side also sums
+    // dout . (a - o) into part_dr [CTA], the terms of dL/dr
+    const __nv_bfloat16* mix_a;
+    float* part_dr;
+    float lin_scale;
+    long long str_token, str_head, str_batch;   // element strides of the activations (for the reads of mix_a)
     int n, H, G, tiles_per_head;
     long long total_tiles;
 #ifdef LINATTN_TRACE
@@ -320,7 +327,7 @@ __device__ __forceinline__ void drain_dw(uint32_t t_dw, uint32_t lane_base, int 
     for (int j = 0; j < 32; ++j) rec[(size_t)(half * 32 + j) * kD + row] = __uint_as_float(v[j]);
 }
 
-template <int kLayout>
+template <int kLayout, int kMixB>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
              const __grid_constant__ CUtensorMap tmDQ, const __grid_constant__ CUtensorMap tmW,
@@ -341,6 +348,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
     const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
     uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0;
+    float dr_acc = 0.f;   // Eq. 8: this thread's share of sum dout . (a - o)
     float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
 #pragma unroll
     for (int e = 0; e < 8; ++e) dz_acc[e] = 0.f;
@@ -420,7 +428,8 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         // is the operand of both products ----
         float x[kM];
         load64(t_work + lane_base + half * kM, x);
-        const float inv = 1.f / (sa[row] + sa[kTile + row]);
+        const float inv1 = 1.f / (sa[row] + sa[kTile + row]);
+        const float inv = inv1 * a.lin_scale;   // every gradient below is linear in the incoming one: its factor rides on 1 / den
         {
             f32x2 gs2 = pack2(0.f, 0.f);
 #pragma unroll
@@ -428,7 +437,37 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 gs2 = fma2(pack2(__uint_as_float(pk[j >> 1] << 16), __uint_as_float(pk[j >> 1] & 0xffff0000u)), pack2(x[j], x[j + 1]), gs2);
             float g0s, g1s;
             unpack2(gs2, g0s, g1s);
-            sb[half * kTile + row] = (g0s + g1s) * inv;   // this half's part of dO . o
+            sb[half * kTile + row] = (g0s + g1s) * inv1;   // this half's part of dO . o
+            if (kMixB) {
+                // Eq. 8: dout . a over this thread's 64 columns (dout from its tile, a straight from memory: one
+                // 128-byte line per thread, started towards L2 a tile ago), minus this half's part of dout . o
+                dr_acc -= (g0s + g1s) * inv1;
+                const int token = w.lt * kTile + row;
+                if (token < a.n) {
+                    const __nv_bfloat16* ap = a.mix_a + (size_t)(w.g / a.H) * a.str_batch + (size_t)(w.g % a.H) * a.str_head +
+                                              (size_t)token * a.str_token + half * kM;
+                    const uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
+                    f32x2 da2 = pack2(0.f, 0.f);
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        const uint4 av = __ldg(reinterpret_cast<const uint4*>(ap) + ch);
+                        const uint4 gv = *reinterpret_cast<const uint4*>(gblk + sw_chunk(row, ch));
+                        const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            da2 = fma2(pack2(__uint_as_float(gw[q] << 16), __uint_as_float(gw[q] & 0xffff0000u)),
+                                       pack2(__uint_as_float(aw[q] << 16), __uint_as_float(aw[q] & 0xffff0000u)), da2);
+                    }
+                    float d0, d1;
+                    unpack2(da2, d0, d1);
+                    dr_acc += d0 + d1;
+                }
+                TileWalk nx = w;
+                nx.next();
+                if (!nx.done() && nx.lt * kTile + row < a.n)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.mix_a + (size_t)(nx.g / a.H) * a.str_batch + (size_t)(nx.g % a.H) * a.str_head +
+                                                                 (size_t)(nx.lt * kTile + row) * a.str_token + half * kM));
+            }
             // phi / den (bf16) is the operand of dS and the factor of dz
             float y[kM];
             const f32x2 inv2 = pack2(inv, inv);
@@ -529,6 +568,18 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         tcgen05_fence_before();
         __syncthreads();
         LB_TRACE(11);
+    }
+    if (kMixB) {
+        // the CTA's sum of dout . (a - o), thread by thread in index order (bit-reproducible)
+        float* red = reinterpret_cast<float*>(c.smem + L::kRed);
+        __syncthreads();
+        red[tid] = dr_acc;
+        __syncthreads();
+        if (tid == 0) {
+            float acc = 0.f;
+            for (int i = 0; i < kBwdThreads; ++i) acc += red[i];
+            a.part_dr[blockIdx.x] = acc;
+        }
     }
     bwd_teardown(c);
 }

@@ -32,6 +32,8 @@ SIGNATURES = {
     "linattn_forward": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_mixed": (_i, [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
+    "linattn_backward_mixed": (_i, [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp,
+                                    _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_host": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "linattn_forward_noalloc": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "linattn_read_state": (_i, [_vp, _vp, _vp, _i, _vp]),
@@ -177,6 +179,26 @@ class LinAttn:
                    dk.data_ptr(), dv.data_ptr(), dWq.data_ptr(), dWk.data_ptr(), 1 if per_head else 0, B, H, n, d,
                    _DTYPES[q.dtype], _stream_ptr(stream))
         return dq, dk, dv, dWq, dWk
+
+    def backward_mixed(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, o_softmax: torch.Tensor, r: float,
+                       dout: torch.Tensor, per_head: bool = True, want_d_o_softmax: bool = True, stream=None):
+        """Gradients through Eq. 8: returns (dq, dk, dv, dWq, dWk, d_o_softmax or None, dr); dr is a CUDA tensor of one float."""
+        for t in (q, k, v, o_softmax, dout):
+            assert t.is_cuda and t.is_contiguous()
+        assert q.shape == k.shape == v.shape == dout.shape == o_softmax.shape
+        assert q.dtype == k.dtype == v.dtype == dout.dtype == o_softmax.dtype
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+        da = torch.empty_like(q) if want_d_o_softmax else None
+        wshape = (self.H, self.d, self.d // 2) if per_head else (self.d, self.d // 2)
+        dWq = torch.empty(wshape, dtype=torch.float32, device=q.device)
+        dWk = torch.empty(wshape, dtype=torch.float32, device=q.device)
+        dr = torch.empty(1, dtype=torch.float32, device=q.device)
+        B, H, n, d = q.shape
+        self._call(self._lib.linattn_backward_mixed, q.data_ptr(), k.data_ptr(), v.data_ptr(), o_softmax.data_ptr(), float(r),
+                   dout.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dWq.data_ptr(), dWk.data_ptr(),
+                   1 if per_head else 0, da.data_ptr() if da is not None else None, dr.data_ptr(), B, H, n, d,
+                   _DTYPES[q.dtype], _stream_ptr(stream))
+        return dq, dk, dv, dWq, dWk, da, dr
 
     def forward_host(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
                      stream=None) -> torch.Tensor:

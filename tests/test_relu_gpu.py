@@ -83,7 +83,10 @@ def test_switching_back_to_the_hedgehog_map_on_one_context():
         assert_parity(hedge.cpu().double().numpy(), oracle.ref_linear(q, k, v, Wq, Wk), "hedgehog after relu")
         with pytest.raises(linattn.LinAttnError):
             ctx.set_option(linattn.OPT_KERNEL_FUNCTION, 2)
+        # the gradients exist for the ReLU kernel function too (CUDA-core kernels; tests/test_backward_mixed_gpu.py),
+        # but there are no tensor-core kernels for them: asking for those is an error, not a silent detour
         ctx.set_option(linattn.OPT_KERNEL_FUNCTION, linattn.PHI_RELU)
+        ctx.set_option(linattn.OPT_PATH, linattn.PATH_TENSOR)
         with pytest.raises(linattn.LinAttnError) as e:
             ctx.backward(q.cuda(), k.cuda(), v.cuda(), q.cuda())
         assert e.value.status == linattn.ERR_UNSUPPORTED
