@@ -21,7 +21,7 @@
 // Warp roles (16 warps): warps 0-3 feature map softmax(+U), warps 4-7 softmax(-U) (one token per thread),
 // warp 8 TMA producer, warp 9 issues the logits MMAs, warp 10 issues the accumulation MMAs, warp 11 issues
 // the TMA stores (query side), warps 12-15 query-side epilogue (num / den -> bf16 output tile) and, in the
-// fused kernel, warps 10-15 do the meeting points and the combine step between the two sides.  Role loops are
+// fused kernel, every warp but 8 and 9 takes part in the meeting points and the combine step between the two sides.  Role loops are
 // warp-uniform; single-thread work (TMA and MMA issue) is predicated inside them.
 // Every wait is bounded: on time-out the kernel records a code in *err, raises the CTA's abort word so
 // that the other roles stop waiting too, and unwinds.
@@ -1298,14 +1298,16 @@ linattn_fused_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     __syncthreads();
     tcgen05_fence_after();
     LA_TRACE_NS(0, 60, 2);
-    constexpr int kHoleWarp0 = 10, kHoleThreads = (16 - kHoleWarp0) * 32;
-    if (c.warp >= kHoleWarp0) {
-        // warps 10-15 (idle until S exists): for every head this CTA's run touches, wait at the head's first meeting
-        // point, sum this CTA's share of the head's record, announce it at the second.  The other warps go straight
-        // on: Q tiles, W_q, the first logits and feature maps do not depend on S.
+    constexpr int kHoleThreads = 14 * 32;
+    if (c.warp != 8 && c.warp != 9) {
+        // Every warp but the producer and the logits issuer (which go straight on: Q tiles, W_q and the first logits do not
+        // depend on S): for every head this CTA's run touches, wait at the head's first meeting point, sum this CTA's
+        // share of the head's record, announce it at the second.  With 448 threads a share of a twelfth of a record (344
+        // groups of four) is one group per thread: ONE round of loads from L2 instead of two (the step took 4 us with the
+        // six warps that are idle anyway; the feature-map warps have nothing urgent to do until S exists either).
         __shared__ uint32_t met;
         const long long P = gridDim.x;
-        const int it = threadIdx.x - kHoleWarp0 * 32;
+        const int it = c.warp < 8 ? (int)threadIdx.x : (int)threadIdx.x - 64;
         TileWalk w;
         w.init(a.total_tiles, a.tiles_per_head);
         bool ok = true;
