@@ -36,7 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xptxas", "-v" if verbose else "-O3",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", tmp] + _sources()
+           "-o", tmp] + _sources() + ["-ldl"]   # -ldl: the header-only NVTX loads a profiler's library on demand
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)

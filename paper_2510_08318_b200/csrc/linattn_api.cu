@@ -11,6 +11,8 @@
 #include <new>
 #include <type_traits>
 
+#include <nvtx3/nvToolsExt.h>   // header-only: the ranges cost a pointer check unless a profiler is attached
+
 #include "simt_kernels.cuh"
 #include "simt_backward.cuh"
 #include "sm100_kernels.cuh"
@@ -23,6 +25,14 @@ namespace {
 
 constexpr int kTargetCtas = 296;  // key-side CTAs aimed for: two waves of the 148 SMs
 constexpr int kMaxSplits = 512;
+
+// A named range around each entry point's work on the host (validation, tensor maps, launches), for timelines.
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange&) = delete;
+    NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 struct DeviceGuard {
     int prev = -1;
@@ -725,6 +735,7 @@ linattn_status linattn_destroy(linattn_ctx* c)
 linattn_status linattn_set_feature_map(linattn_ctx* c, const void* Wq, const void* Wk, int per_head,
                                        linattn_dtype wdtype, void* stream)
 {
+    NvtxRange range("linattn_set_feature_map");
     if (!c || !Wq || !Wk) return LINATTN_ERR_INVALID_ARG;
     if (wdtype != LINATTN_F32 && wdtype != LINATTN_BF16) return LINATTN_ERR_UNSUPPORTED;
     DeviceGuard guard(c->device);
@@ -776,6 +787,7 @@ static linattn_status forward_impl(linattn_ctx* c, const void* q, const void* k,
                                    const void* mix, float mix_r, int B, int H, int n, int d, linattn_dtype dtype,
                                    void* stream)
 {
+    NvtxRange range(mix ? "linattn_forward_mixed" : "linattn_forward");
     linattn_status s = check_forward_args(c, q, k, v, out, B, H, n, d, dtype);
     if (s != LINATTN_OK) return s;
     if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(out)) return LINATTN_ERR_INVALID_ARG;
@@ -834,6 +846,7 @@ static linattn_status backward_impl(linattn_ctx* c, const void* q, const void* k
                                     const void* dout, void* dq, void* dk, void* dv, float* dWq, float* dWk, int per_head,
                                     void* d_a, float* dr, int B, int H, int n, int d, linattn_dtype dtype, void* stream)
 {
+    NvtxRange range(a ? "linattn_backward_mixed" : "linattn_backward");
     if (!dout || !dk || !dv) return LINATTN_ERR_INVALID_ARG;
     const bool relu = c && c->opt_phi != 0;
     if (!relu && (!dWq || !dWk)) return LINATTN_ERR_INVALID_ARG;   // the ReLU kernel function has no weights: its dWq, dWk are ignored
@@ -938,6 +951,7 @@ linattn_status linattn_backward_mixed(linattn_ctx* c, const void* q, const void*
 linattn_status linattn_forward_host(linattn_ctx* c, const void* q, const void* k, const void* v, void* out, int B,
                                     int H, int n, int d, linattn_dtype dtype, void* stream)
 {
+    NvtxRange range("linattn_forward_host");
     linattn_status s = check_forward_args(c, q, k, v, out, B, H, n, d, dtype);
     if (s != LINATTN_OK) return s;
     DeviceGuard guard(c->device);
