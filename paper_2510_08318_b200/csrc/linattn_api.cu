@@ -78,6 +78,7 @@ struct linattn_ctx {
     // workspace of the backward pass, allocated by the first linattn_backward
     float* bwd_part_state = nullptr;  // [partial_slots][d*d + d]  per-block sums of dS, dz
     float* bwd_part_w = nullptr;      // [partial_slots][d*d/2]    per-block sums of dW
+    float* bwd_part_w2 = nullptr;     // the same for dW_k on the tensor-core path (both weight gradients are summed by one launch at the end)
     float* bwd_dstate = nullptr;      // [max_B*H][d*d + d]        dS, dz
     float* bwd_part_dr = nullptr;     // [partial_slots]           per-block sums of dout . (a - o), the terms of Eq. 8's dL/dr
     __nv_bfloat16* bwd_img[3] = {nullptr, nullptr, nullptr};   // tensor-core backward: lo image of S, hi and lo images of dS
@@ -106,6 +107,7 @@ struct linattn_ctx {
         const void* v = nullptr;
         int B = 0, n = 0, layout = 0;
         bool valid = false;
+        bool has_lo = false;   // the lo image of S (the backward's second operand) was written along with the state
     } state_key;
     // per-kernel timing (LINATTN_OPT_PROFILE)
     static constexpr int kMaxKernels = 8;
@@ -419,6 +421,9 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.partial = c->partial;
     a.state = c->state + (size_t)c->view_g0 * ((size_t)c->d * c->d + c->d);   // one record per head (per pair of heads only inside the kernels)
     a.s_img = c->s_img + (size_t)c->view_g0 * kD * kD;
+    // the backward's tensor-core kernels (d = 128) read S as a bf16 hi + lo pair: the lo image is written along with the
+    // state when this call is the backward's own, or when the backward may take the state over from this forward
+    a.s_img_lo = (!pair && c->bwd_img[0] && c->view_H == 0 && (state_only || c->opt_reuse)) ? c->bwd_img[0] : nullptr;
     a.z_img = c->z_img + (size_t)c->view_g0 * (kZBlkBytes / 2);
     a.err = c->err_word;
     a.sync = c->sync_words;
@@ -497,15 +502,17 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     // caller allows it), else recomputed; q and out are not touched by the first two kernels of the forward
     const linattn_ctx::StateKey& sk = c->state_key;
     const bool reuse = c->opt_reuse && sk.valid && sk.k == k && sk.v == v && sk.B == B && sk.n == n && sk.layout == c->opt_layout;
-    int launches = 7;
+    int launches = 4;   // qside_bwd_tc, combine of dS and dz, kside_bwd_tc, combine of both weight gradients
+    bool need_lo = false;
     if (reuse) {
         prof_begin(c, st);
+        need_lo = !sk.has_lo;
     } else {
         c->state_key.valid = false;
-        const linattn_status s = launch_tc(c, k, k, v, dk, B, n, st, nullptr, 0.f, true);
+        const linattn_status s = launch_tc(c, k, k, v, dk, B, n, st, nullptr, 0.f, true);   // writes the lo image of S too
         if (s != LINATTN_OK) return s;
-        c->state_key = {k, v, B, n, c->opt_layout, true};
-        launches = 9;
+        c->state_key = {k, v, B, n, c->opt_layout, true, true};
+        launches = 6;
     }
 
     const ActStrides as = act_strides(c, n);
@@ -558,8 +565,12 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     a.trace = c->trace;
 #endif
     const dim3 wgrid(kWRec / 256, per_head ? (unsigned)c->H : 1u);
-    hilo_images<<<dim3(kD * kD / 256, (unsigned)G), 256, 0, st>>>(c->state, nullptr, c->bwd_img[0]);
-    LA_CUDA(c, cudaGetLastError());
+    if (need_lo) {   // the state was taken over from a forward that ran before the backward's workspace existed
+        hilo_images<<<dim3(kD * kD / 256, (unsigned)G), 256, 0, st>>>(c->state, nullptr, c->bwd_img[0]);
+        LA_CUDA(c, cudaGetLastError());
+        c->state_key.has_lo = true;
+        ++launches;
+    }
     {
         void* p[] = {&tmQ, &tmG, &tmDQ, &tmWq, &tmShi, &tmSlo, &a};
         LA_CUDA(c, cudaLaunchKernel(k_q[layout][mg.dr ? 1 : 0], dim3((unsigned)P), dim3(kBwdThreads), p, kBwdSmemQ, st));
@@ -570,22 +581,20 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
         LA_CUDA(c, cudaGetLastError());
         ++launches;
     }
-    combine_slots<<<dim3((kE + 255) / 256, (unsigned)G), 256, 0, st>>>(c->bwd_part_state, c->bwd_dstate, kE, (int)Tn, T, P);
+    combine_slots_hilo<<<dim3((kE + 255) / 256, (unsigned)G), 256, 0, st>>>(c->bwd_part_state, c->bwd_dstate, c->bwd_img[1], c->bwd_img[2],
+                                                                           (int)Tn, T, P);
     LA_CUDA(c, cudaGetLastError());
-    hilo_images<<<dim3(kD * kD / 256, (unsigned)G), 256, 0, st>>>(c->bwd_dstate, c->bwd_img[1], c->bwd_img[2]);
-    LA_CUDA(c, cudaGetLastError());
-    combine_wgrad_slots<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWq, (int)G, c->H, per_head, (int)Tn, T, P);
-    LA_CUDA(c, cudaGetLastError());
-    prof_mark(c, st, "combine_dstate_dWq", 0.0);
+    prof_mark(c, st, "combine_dstate", 0.0);
     a.state = c->bwd_dstate;
+    a.part_w = c->bwd_part_w2;   // dW_k's records; dW_q's stay in part_w until both are summed at the end
     {
         void* p[] = {&tmK, &tmV, &tmDK, &tmDV, &tmWk, &tmDShi, &tmDSlo, &a};
         LA_CUDA(c, cudaLaunchKernel(k_k[layout], dim3((unsigned)P), dim3(kBwdThreads), p, kBwdSmemK, st));
     }
     prof_mark(c, st, "kside_bwd_tc", 4.0 * tensor_bytes);
-    combine_wgrad_slots<<<wgrid, 256, 0, st>>>(c->bwd_part_w, dWk, (int)G, c->H, per_head, (int)Tn, T, P);
+    combine_wgrad_slots2<<<dim3(wgrid.x, wgrid.y, 2), 256, 0, st>>>(c->bwd_part_w, c->bwd_part_w2, dWq, dWk, (int)G, c->H, per_head, (int)Tn, T, P);
     LA_CUDA(c, cudaGetLastError());
-    prof_mark(c, st, "combine_dWk", 0.0);
+    prof_mark(c, st, "combine_dWq_dWk", 0.0);
     c->last_launches = launches;
     return LINATTN_OK;
 }
@@ -716,6 +725,7 @@ linattn_status linattn_destroy(linattn_ctx* c)
     cudaFree(c->z_img);
     cudaFree(c->bwd_part_state);
     cudaFree(c->bwd_part_w);
+    cudaFree(c->bwd_part_w2);
     cudaFree(c->bwd_dstate);
     cudaFree(c->bwd_part_dr);
     for (void* p : c->bwd_img) cudaFree(p);
@@ -816,7 +826,8 @@ static linattn_status dispatch_forward(linattn_ctx* c, const void* q, const void
     c->state_key.valid = false;
     if (c->state_transposed) {
         const linattn_status s = launch_tc(c, q, k, v, out, B, n, st, mix, mix_r);
-        if (s == LINATTN_OK && c->opt_phi == 0 && c->view_H == 0 && d == 128) c->state_key = {k, v, B, n, c->opt_layout, true};
+        if (s == LINATTN_OK && c->opt_phi == 0 && c->view_H == 0 && d == 128)
+            c->state_key = {k, v, B, n, c->opt_layout, true, c->opt_reuse && c->bwd_img[0] != nullptr};
         return s;
     }
     if (dtype == LINATTN_BF16) {
@@ -882,6 +893,7 @@ static linattn_status backward_impl(linattn_ctx* c, const void* q, const void* k
         const size_t E = (size_t)d * d + d, G = (size_t)(c->max_B * c->H);
         cudaError_t e = cudaMalloc(&c->bwd_part_state, sizeof(float) * E * (size_t)c->partial_slots);
         if (e == cudaSuccess) e = cudaMalloc(&c->bwd_part_w, sizeof(float) * (size_t)d * (d / 2) * (size_t)c->partial_slots);
+        if (e == cudaSuccess && d == 128) e = cudaMalloc(&c->bwd_part_w2, sizeof(float) * (size_t)d * (d / 2) * (size_t)c->partial_slots);
         if (e == cudaSuccess) e = cudaMalloc(&c->bwd_dstate, sizeof(float) * E * G);
         if (e == cudaSuccess) e = cudaMalloc(&c->bwd_part_dr, sizeof(float) * (size_t)c->partial_slots);
         if (d == 128)
@@ -891,9 +903,10 @@ static linattn_status backward_impl(linattn_ctx* c, const void* q, const void* k
             cudaGetLastError();
             cudaFree(c->bwd_part_state);
             cudaFree(c->bwd_part_w);
+            cudaFree(c->bwd_part_w2);
             cudaFree(c->bwd_dstate);
             cudaFree(c->bwd_part_dr);
-            c->bwd_part_state = c->bwd_part_w = c->bwd_dstate = c->bwd_part_dr = nullptr;
+            c->bwd_part_state = c->bwd_part_w = c->bwd_part_w2 = c->bwd_dstate = c->bwd_part_dr = nullptr;
             for (__nv_bfloat16*& p : c->bwd_img) {
                 cudaFree(p);
                 p = nullptr;

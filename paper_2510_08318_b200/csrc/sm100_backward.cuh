@@ -753,6 +753,27 @@ combine_slots(const float* __restrict__ part, float* __restrict__ out, int E, in
     out[(size_t)g * E + e] = acc;
 }
 
+// The two steps in one for dS, dz: fixed-order sum of the (CTA, head) records, fp32 state and, for the matrix part, the
+// bf16 hi and lo images the key side reads.  grid = (ceil(kE/256), G).
+static __global__ void __launch_bounds__(256)
+combine_slots_hilo(const float* __restrict__ part, float* __restrict__ out, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                   int tiles_per_head, long long total_tiles, long long P)
+{
+    const int e = blockIdx.x * 256 + threadIdx.x;
+    if (e >= kE) return;
+    const int g = blockIdx.y;
+    const long long c0 = tile_owner((long long)g * tiles_per_head, total_tiles, P);
+    const long long c1 = tile_owner((long long)(g + 1) * tiles_per_head - 1, total_tiles, P);
+    float acc = 0.f;
+    for (long long cta = c0; cta <= c1; ++cta) acc += part[(size_t)(cta + g) * kE + e];
+    out[(size_t)g * kE + e] = acc;
+    if (e < kD * kD) {
+        const __nv_bfloat16 h = __float2bfloat16_rn(acc);
+        hi[(size_t)g * kD * kD + e] = h;
+        lo[(size_t)g * kD * kD + e] = __float2bfloat16_rn(acc - __bfloat162float(h));
+    }
+}
+
 // Matrix part of a state record ([c][f] fp32) -> bf16 hi and lo images (either may be NULL).  grid = (64, G).
 static __global__ void __launch_bounds__(256)
 hilo_images(const float* __restrict__ state, __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo)
@@ -771,6 +792,24 @@ combine_wgrad_slots(const float* __restrict__ part_w, float* __restrict__ dW, in
                     long long total_tiles, long long P)
 {
     const int r = blockIdx.x * 256 + threadIdx.x;   // index in a record, j * 128 + c: neighbouring threads read neighbouring words
+    const int j = r / kD, cc = r % kD, wsel = blockIdx.y;
+    float acc = 0.f;
+    for (int g = per_head ? wsel : 0; g < G; g += per_head ? H : 1) {
+        const long long c0 = tile_owner((long long)g * tiles_per_head, total_tiles, P);
+        const long long c1 = tile_owner((long long)(g + 1) * tiles_per_head - 1, total_tiles, P);
+        for (long long cta = c0; cta <= c1; ++cta) acc += part_w[(size_t)(cta + g) * kWRec + r];
+    }
+    dW[(size_t)wsel * kWRec + (size_t)cc * kM + j] = acc;
+}
+
+// Both weight gradients in one launch: blockIdx.z = 0: dW_q from part_wq, 1: dW_k from part_wk.  grid = (kWRec / 256, per_head ? H : 1, 2).
+static __global__ void __launch_bounds__(256)
+combine_wgrad_slots2(const float* __restrict__ part_wq, const float* __restrict__ part_wk, float* __restrict__ dWq, float* __restrict__ dWk,
+                     int G, int H, int per_head, int tiles_per_head, long long total_tiles, long long P)
+{
+    const float* part_w = blockIdx.z == 0 ? part_wq : part_wk;
+    float* dW = blockIdx.z == 0 ? dWq : dWk;
+    const int r = blockIdx.x * 256 + threadIdx.x;
     const int j = r / kD, cc = r % kD, wsel = blockIdx.y;
     float acc = 0.f;
     for (int g = per_head ? wsel : 0; g < G; g += per_head ? H : 1) {

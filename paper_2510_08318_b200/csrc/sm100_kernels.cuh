@@ -419,6 +419,7 @@ struct Args {
     float* partial;              // [slots][kE] partial (S, z) records, slot = cta + g; S as [c][f] (c = column of V, f = feature)
     float* state;                // [G][kE] combined S, z (fp32), same layout
     __nv_bfloat16* s_img;        // [G][128][128] bf16 image of S, [c][f]
+    __nv_bfloat16* s_img_lo;     // or nullptr: bf16 image of what s_img leaves of S (S = hi + lo; the backward's operand pair)
     __nv_bfloat16* z_img;        // [G][kZBlkBytes / 2] bf16 operand image of z (hi, lo)
     uint32_t* err;               // error word
     uint32_t* sync;              // fused kernel: [0] CTAs that have left their last wait; [1 + 2g], [2 + 2g] arrivals at the two
@@ -884,6 +885,12 @@ __device__ __forceinline__ void combine_quad(const Args& a, long long P, int g, 
         packed.x = keep ? pack_bf16(r[0], r[1]) : 0u;
         packed.y = keep ? pack_bf16(r[2], r[3]) : 0u;
         *reinterpret_cast<uint2*>(a.s_img + (size_t)g * kD * kD + e4) = packed;
+        if (a.s_img_lo) {   // never with kPair (the backward's tensor-core kernels are d = 128 only)
+            uint2 lo;
+            lo.x = pack_bf16(r[0] - __uint_as_float(packed.x << 16), r[1] - __uint_as_float(packed.x & 0xffff0000u));
+            lo.y = pack_bf16(r[2] - __uint_as_float(packed.y << 16), r[3] - __uint_as_float(packed.y & 0xffff0000u));
+            *reinterpret_cast<uint2*>(a.s_img_lo + (size_t)g * kD * kD + e4) = lo;
+        }
         if (kPair && keep && 2 * g + (cc >> 6) < a.heads_total)
             *reinterpret_cast<float4*>(a.state + (size_t)(2 * g + (cc >> 6)) * kEh + (cc & 63) * 64 + (f0 & 63)) = acc;
     } else {

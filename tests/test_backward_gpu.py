@@ -61,7 +61,7 @@ def _run(x, per_head=True, layout=linattn.LAYOUT_BHND, path=linattn.PATH_AUTO):
         got = ctx.backward(*args, per_head=per_head)
         again = ctx.backward(*args, per_head=per_head)
         ctx.check()
-        assert ctx.last_launch_count() == (9 if _tensor_core(x, path) else 7)   # tensor-core kernels for bf16, d = 128
+        assert ctx.last_launch_count() == (6 if _tensor_core(x, path) else 7)   # tensor-core kernels for bf16, d = 128
         for a, b in zip(got, again):
             assert torch.equal(a, b), "the gradients are not bit-reproducible"
         if layout == linattn.LAYOUT_BNHD:
@@ -92,7 +92,8 @@ def test_gradients_match_the_oracle(B, H, n, d, dtype, path):
         # o = v whatever q and k are: every gradient but dv vanishes, so only absolute checks make sense
         for name, t in zip(NAMES, got):
             if name != "dv":
-                assert float(t.abs().max()) <= (1e-5 if dtype == torch.float32 else 2e-2), f"{name} must vanish for a single token"
+                # (bf16, tensor-core kernels: what is left of the cancellation dO S^T - (dO . o) z with S as a bf16 hi + lo pair)
+                assert float(t.abs().max()) <= (1e-5 if dtype == torch.float32 else 2e-3), f"{name} must vanish for a single token"
         assert torch.allclose(got[2].cpu().float(), x["dout"].float(), rtol=1e-6 if dtype == torch.float32 else 1e-2, atol=0)
         assert np.abs(want[2] - x["dout"].double().numpy()).max() <= 1e-12
         return
@@ -169,31 +170,49 @@ def test_state_left_by_the_forward_is_reused_only_when_it_belongs_to_the_same_pr
         dy = [y[s].cuda() for s in ("q", "k", "v", "dout")]
         ref_x = ctx.backward(*dx)
         ref_y = ctx.backward(*dy)
-        assert ctx.last_launch_count() == 9
+        assert ctx.last_launch_count() == 6
         ctx.set_option(linattn.OPT_REUSE_STATE, 1)
         ctx.forward(dx[0], dx[1], dx[2])
         got = ctx.backward(*dx)                       # same k, v as the forward: S, z are taken over
-        assert ctx.last_launch_count() == 7
+        assert ctx.last_launch_count() == 4
         for a, b in zip(got, ref_x):
             assert torch.equal(a, b)
         got = ctx.backward(*dy)                       # other k, v: recomputed
-        assert ctx.last_launch_count() == 9
+        assert ctx.last_launch_count() == 6
         for a, b in zip(got, ref_y):
             assert torch.equal(a, b)
         got = ctx.backward(*dy)                       # the backward's own state counts too
-        assert ctx.last_launch_count() == 7
+        assert ctx.last_launch_count() == 4
         for a, b in zip(got, ref_y):
             assert torch.equal(a, b)
         ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())   # new weights: nothing is taken over
         ctx.backward(*dy)
-        assert ctx.last_launch_count() == 9
+        assert ctx.last_launch_count() == 6
         ctx.forward(dx[0], dx[1], dx[2])
         ctx.set_option(linattn.OPT_REUSE_STATE, 0)
         ctx.backward(*dx)
-        assert ctx.last_launch_count() == 9
+        assert ctx.last_launch_count() == 6
         ctx.check()
     finally:
         ctx.destroy()
+    # a forward that ran before the backward's workspace existed left no lo image of S: the first backward makes it
+    fresh = linattn.LinAttn(3, 128, max_B=1, max_n=900)
+    try:
+        fresh.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        fresh.set_option(linattn.OPT_REUSE_STATE, 1)
+        fresh.forward(dx[0], dx[1], dx[2])
+        got = fresh.backward(*dx)
+        assert fresh.last_launch_count() == 5
+        for a, b in zip(got, ref_x):
+            assert torch.equal(a, b)
+        fresh.forward(dx[0], dx[1], dx[2])
+        got = fresh.backward(*dx)
+        assert fresh.last_launch_count() == 4
+        for a, b in zip(got, ref_x):
+            assert torch.equal(a, b)
+        fresh.check()
+    finally:
+        fresh.destroy()
 
 
 def test_argument_errors():
