@@ -294,6 +294,9 @@ def main():
     assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torchrun --nproc-per-node {args.gpus}"
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    sampler = ClockSampler(local)   # started this early so that it is polling steadily by the time the timed region runs
+    if rank == 0:
+        sampler.start()
 
     # inputs: `rotate` independent sets per rank (different layers' seeds), resident in HBM; the 30-layer workload
     # keeps every layer resident and walks through them back to back on the one stream
@@ -329,16 +332,17 @@ def main():
         else:
             ctxs[j].forward_mixed(sets[j]["q"], sets[j]["k"], sets[j]["v"], softs[j], args.mixed, out=outs[j], stream=stream)
 
-    # the backward allocates its workspace on a context's first call: every context gets one call before the warm-up
-    for i in range(max(args.warmup, rotate if douts is not None else 0)):
+    # every context's first call (function attributes, the backward's workspace allocation) happens before the warm-up
+    for i in range(rotate):
         step(i)
     ctxs[0].check()
     launches_per_step = ctxs[0].last_launch_count()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # the W warm-up steps run right before the timed region, with no host-side pause in between in which the GPU could
+    # fall back to its idle clocks
+    for i in range(args.warmup):
+        step(i)
     ladist.barrier()
     torch.cuda.synchronize()
     t_region0 = time.time()
