@@ -1172,43 +1172,29 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
         const int row = (warp & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int sw = row & 7;
-        Ring<qs> r;
-        Ring<2> dr;
-        for (; !w.done(); w.next(), r.next(), dr.next()) {
-            if (!warp_wait(c.bar(Q_DFULL + dr.s), dr.ph, c.wc, kErrEpilogue)) break;
-            if (warp == 12) LA_TRACE(3, 24 + w.i, 0);
-            tcgen05_fence_after();
+        constexpr bool mix = kMix;   // compile-time: the plain forward carries none of the blend's code
+        // One finished tile: o = num / den (blended with the softmax branch's tile under Eq. 8), bf16, into slot `rs`.
+        auto finish = [&](int rs, uint32_t rph, int ds) -> bool {
             // columns of the denominator operand: d = 128: [z_hi, z_lo]; paired heads: [z_hi, z_lo] of the first head, then of the second
             uint32_t dv[4];
-            tmem_ld_x2(tmem_den(dr.s) + lane_base, dv);
-            if (kPair) tmem_ld_x2(tmem_den(dr.s) + lane_base + 2, dv + 2);
-            constexpr bool mix = kMix;   // compile-time: the plain forward carries none of the blend's code
-            if (mix) {
-                // Eq. 8 (mixed attention): the tensor core is done with phi(q) in this slot (that is what the barrier
-                // above says), so the tile of the softmax branch's output is brought into the very same slot by TMA
-                // (its lines are already on their way into L2), blended in place and stored from there.
-                if (warp == 12 && lane == 0) {
-                    mbar_arrive_expect_tx(c.bar(Q_AFULL + r.s), kTileBytes);
-                    Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes, tmA, c.bar(Q_AFULL + r.s), 0, w.lt * kTile, w.g, a.H);
-                    Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes + kHalfTileBytes, tmA, c.bar(Q_AFULL + r.s), 1, w.lt * kTile, w.g, a.H);
-                }
-                if (!warp_wait(c.bar(Q_AFULL + r.s), r.ph, c.wc, kErrEpilogue)) break;
-            }
+            tmem_ld_x2(tmem_den(ds) + lane_base, dv);
+            if (kPair) tmem_ld_x2(tmem_den(ds) + lane_base + 2, dv + 2);
+            if (mix && !warp_wait(c.bar(Q_AFULL + rs), rph, c.wc, kErrEpilogue)) return false;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[64];
-                tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64, v);
-                tmem_ld_x32(tmem_num(dr.s) + lane_base + half * 64 + 32, v + 32);
+                tmem_ld_x32(tmem_num(ds) + lane_base + half * 64, v);
+                tmem_ld_x32(tmem_num(ds) + lane_base + half * 64 + 32, v + 32);
                 tmem_wait_ld();
                 if (half == 1) {
                     // everything this tile needs from TMEM is in registers: release the accumulator
                     tcgen05_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(c.bar(Q_DEMPTY + dr.s));
+                    if (lane == 0) mbar_arrive(c.bar(Q_DEMPTY + ds));
                 }
                 const int dsel = kPair ? 2 * half : 0;   // paired heads: output block `half` belongs to head `half` of the pair
                 const float inv = __fdividef(1.f, __uint_as_float(dv[dsel]) + __uint_as_float(dv[dsel + 1]));
-                uint8_t* dst = c.smem + r.s * kTileBytes + half * kHalfTileBytes + row * 128;
+                uint8_t* dst = c.smem + rs * kTileBytes + half * kHalfTileBytes + row * 128;
                 if (!mix) {
                     const f32x2 inv2 = pack2(inv, inv);
 #pragma unroll
@@ -1245,8 +1231,39 @@ __device__ __forceinline__ void qside_phase(const Cta& c, const Args& a, const C
             }
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(c.bar(Q_OFULL + r.s));
+            if (lane == 0) mbar_arrive(c.bar(Q_OFULL + rs));
+            return true;
+        };
+        Ring<qs> r;
+        Ring<2> dr;
+        // Eq. 8 (mixed attention): once the tensor core is done with phi(q) in a slot (that is what Q_DFULL says), the
+        // tile of the softmax branch's output is brought into the very same slot by TMA (its lines are already on their
+        // way into L2), blended in place and stored from there.  The blend of a tile runs one tile late, so that the
+        // copy's latency passes under the blend of the tile before it instead of in front of its own.
+        int prev_rs = -1, prev_ds = 0;
+        uint32_t prev_rph = 0;
+        bool ok = true;
+        for (; !w.done(); w.next(), r.next(), dr.next()) {
+            if (!warp_wait(c.bar(Q_DFULL + dr.s), dr.ph, c.wc, kErrEpilogue)) { ok = false; break; }
+            if (warp == 12) LA_TRACE(3, 24 + w.i, 0);
+            tcgen05_fence_after();
+            if (mix) {
+                if (warp == 12 && lane == 0) {
+                    mbar_arrive_expect_tx(c.bar(Q_AFULL + r.s), kTileBytes);
+                    Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes, tmA, c.bar(Q_AFULL + r.s), 0, w.lt * kTile, w.g, a.H);
+                    Blocks<kLayout, kPair>::load(sbase + r.s * kTileBytes + kHalfTileBytes, tmA, c.bar(Q_AFULL + r.s), 1, w.lt * kTile, w.g, a.H);
+                }
+                if (prev_rs >= 0 && !finish(prev_rs, prev_rph, prev_ds)) { ok = false; break; }
+                prev_rs = r.s;
+                prev_rph = r.ph;
+                prev_ds = dr.s;
+            } else if (!finish(r.s, r.ph, dr.s)) { ok = false; break; }
             if (warp == 12) LA_TRACE(3, 24 + w.i, 1);
+        }
+        if (mix && prev_rs >= 0) {
+            // the last tile; after a wait that gave up, only so that the copy in flight has landed before the CTA moves on
+            if (ok) finish(prev_rs, prev_rph, prev_ds);
+            else if (warp == 12) mbar_wait(c.bar(Q_AFULL + prev_rs), prev_rph, c.wc.limit_ns());
         }
     }
 }
