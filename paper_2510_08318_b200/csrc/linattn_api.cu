@@ -1147,7 +1147,8 @@ linattn_status linattn_check(linattn_ctx* c, void* stream)
     if (w != 0) {
         LA_CUDA(c, cudaMemsetAsync(c->err_word, 0, sizeof(w), st));
         LA_CUDA(c, cudaMemsetAsync(c->sync_words, 0, c->sync_bytes, st));  // an aborted launch does not clear its meeting-point counters
-        snprintf(c->err_text, sizeof(c->err_text), "device-side wait gave up (code 0x%x)", w);
+        if (w & tc::kErrSmem) snprintf(c->err_text, sizeof(c->err_text), "a kernel's shared-memory window did not hold its layout (code 0x%x)", w);
+        else snprintf(c->err_text, sizeof(c->err_text), "device-side wait gave up (code 0x%x)", w);
         return LINATTN_ERR_TIMEOUT;
     }
     return LINATTN_OK;

@@ -7,10 +7,11 @@
 //     dphi(k_j) = dS v_j + dz                dv_j = dS^T phi(k_j)
 //     du = p+ (.) (dphi+ - p+ . dphi+) - p- (.) (dphi- - p- . dphi-)       dx = du W^T       dW += x^T du
 //
-// Two kernels of persistent CTAs, each walking its contiguous run of 128-token tiles one tile at a time; the
-// stages of a tile run one after the other (no software pipeline: the first aim here is a correct tensor-core
-// path; every matrix product is a tcgen05.mma with fp32 accumulators in TMEM, every element-wise step runs on all
-// 256 threads, thread = (token, half of the features)):
+// Two kernels of persistent CTAs, each walking its contiguous run of 128-token tiles.  Every matrix product is a
+// tcgen05.mma with fp32 accumulators in TMEM, every element-wise step runs on all 256 threads, thread = (token, half of
+// the features); thread 0 issues the copies and the products.  Within a head the tiles are software-pipelined two deep:
+// the tile that feeds the logits is double-buffered, the next tile's logits are issued ahead of this tile's last
+// tensor-core stage, and this tile's results leave tensor memory after the next tile's feature map:
 //
 //   qside_bwd_tc : U = Q W_q -> phi(q) -> num = phi S, den, dO . o -> dphi = (dO S^T - (dO . o) z) / den,
 //                  dS += (phi / den)^T dO, dz += (phi / den)^T (dden den) -> du -> dq = du W_q^T (TMA store),
@@ -61,21 +62,26 @@ struct BwdArgs {
 #define LB_TRACE(ev) do { } while (0)
 #endif
 
+// Shared memory, both kernels: two buffers for the tile that feeds the logits (the next tile's is fetched while this
+// tile is worked on), one for the other input tile, the staging tile, the hi and lo images, the weights and the du
+// tile: 224 KB, then the small block below.  The total is the 227 KB a CTA may have, to within 448 bytes: the
+// kernels leave with an error if the base of the dynamic array is not aligned well enough for that.
 struct BwdSmemQ {   // query side
-    static constexpr uint32_t kX = 0;                        // Q tile
-    static constexpr uint32_t kG = kX + kTileBytes;          // dO tile -> du (first 16 KB)
-    static constexpr uint32_t kL = kG + kTileBytes;          // du tile [128][64] bf16 (16 KB), then room for the dz sums at the end of a head
-    static constexpr uint32_t kP = kL + kTileBytes;          // phi(q) -> phi(q) / den -> dq staging
+    static constexpr uint32_t kX0 = 0;                       // Q tile, even tiles of the run
+    static constexpr uint32_t kX1 = kX0 + kTileBytes;        // Q tile, odd tiles
+    static constexpr uint32_t kG = kX1 + kTileBytes;         // dO tile
+    static constexpr uint32_t kP = kG + kTileBytes;          // phi(q) / den -> dq staging
     static constexpr uint32_t kShi = kP + kTileBytes;        // S image [c][f], hi part
     static constexpr uint32_t kSlo = kShi + kTileBytes;      // lo part
     static constexpr uint32_t kW = kSlo + kTileBytes;        // W_q^T [64][128]
-    static constexpr uint32_t kDu = kL;                      // du tile
-    static constexpr uint32_t kRed = kL + kWBytes;           // 16 x 128 floats: dz sums of the token groups
-    static constexpr uint32_t kMisc = kW + kWBytes;
+    static constexpr uint32_t kDu = kW + kWBytes;            // du tile [128][64] bf16 (16 KB)
+    static constexpr uint32_t kRed = kDu;                    // at the end of a head (du consumed): 16 x 128 floats, dz sums of the token groups
+    static constexpr uint32_t kMisc = kDu + kWBytes;
 };
 struct BwdSmemK {   // key side
-    static constexpr uint32_t kX = 0;                        // K tile
-    static constexpr uint32_t kV = kX + kTileBytes;          // V tile -> fp32 scratch for du
+    static constexpr uint32_t kX0 = 0;                       // K tile, even tiles of the run
+    static constexpr uint32_t kX1 = kX0 + kTileBytes;        // K tile, odd tiles
+    static constexpr uint32_t kV = kX1 + kTileBytes;         // V tile
     static constexpr uint32_t kP = kV + kTileBytes;          // phi(k) -> dv staging -> dk staging
     static constexpr uint32_t kShi = kP + kTileBytes;        // dS image [c][f], hi part
     static constexpr uint32_t kSlo = kShi + kTileBytes;
@@ -86,16 +92,18 @@ struct BwdSmemK {   // key side
 // misc block: z / dz vector, per-token scalars, barriers, TMEM slot, abort word
 struct BwdMisc {
     static constexpr uint32_t kVec = 0;           // 128 floats: z (query side) or dz (key side)
-    static constexpr uint32_t kA = 512;           // 2 x 128 floats: den halves, later dz halves
-    static constexpr uint32_t kB = 1536;          // 2 x 128 floats: (dO . o) halves
-    static constexpr uint32_t kDd = 2560;         // 128 floats: dden
-    static constexpr uint32_t kBars = 3072;       // 4 mbarriers, TMEM slot, abort word
-    static constexpr uint32_t kBytes = 3072 + 64;
+    static constexpr uint32_t kA = 512;           // 2 x 128 floats: den halves
+    static constexpr uint32_t kB = 1536;          // 2 x 128 floats: (dO . o) halves; then, in the first 128, dden den of the tile
+    static constexpr uint32_t kBars = 2560;       // 6 mbarriers, TMEM slot, abort word
+    static constexpr uint32_t kBytes = 2560 + 64;
 };
-constexpr uint32_t kBwdSmemQ = BwdSmemQ::kMisc + BwdMisc::kBytes + 1024;
-constexpr uint32_t kBwdSmemK = BwdSmemK::kMisc + BwdMisc::kBytes + 1024;
+constexpr uint32_t kBwdSmemQ = BwdSmemQ::kMisc + BwdMisc::kBytes;
+constexpr uint32_t kBwdSmemK = BwdSmemK::kMisc + BwdMisc::kBytes;
+static_assert(kBwdSmemQ <= 232448 && kBwdSmemK <= 232448, "a CTA has 227 KB of shared memory");
 
-enum : int { BW_LOAD = 0, BW_SEG = 1, BW_MMA = 2, BW_MMA2 = 3, BW_NBARS = 4 };
+// BW_LOAD: the tile that feeds the logits; BW_LOAD2: the other input tile; BW_MMA: logits; BW_MMA2: the product with the
+// hi and lo images; BW_G: the tile's last tensor-core stage
+enum : int { BW_LOAD = 0, BW_SEG = 1, BW_MMA = 2, BW_MMA2 = 3, BW_G = 4, BW_LOAD2 = 5, BW_NBARS = 6 };
 
 struct BwdCta {
     uint8_t* smem;
@@ -104,6 +112,20 @@ struct BwdCta {
     WaitCtx wc;
     __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * (uint32_t)i; }
 };
+
+// The layout above leaves no room for rounding the base of the dynamic shared memory up to the 1024 bytes the swizzled
+// tiles need.  These kernels have no static shared memory, so their dynamic array starts at the CTA's window, which is
+// so aligned; this check (the same verdict in every thread, before any barrier or allocation) makes a launch whose
+// array came out otherwise report it and leave instead of writing past its end.
+__device__ __forceinline__ bool bwd_smem_fits(const uint8_t* smem_raw, uint32_t need, uint32_t* err)
+{
+    uint32_t have;
+    asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(have));
+    const uint32_t pad = (1024u - (smem_u32(smem_raw) & 1023u)) & 1023u;
+    if (pad + need <= have) return true;
+    if (threadIdx.x == 0) atomicOr(err, kErrSmem);
+    return false;
+}
 
 __device__ __forceinline__ BwdCta bwd_setup(uint8_t* smem_raw, uint32_t misc_off, uint32_t* err)
 {
@@ -156,53 +178,7 @@ __device__ __forceinline__ bool cta_wait(const BwdCta& c, int b, uint32_t& phase
 // Byte offset of 16-byte chunk `ch` (8 bf16) of row `row` inside a 64-column block of a TMA tile (128-byte swizzle).
 __device__ __forceinline__ uint32_t sw_chunk(int row, int ch) { return (uint32_t)row * 128u + (uint32_t)((ch ^ (row & 7)) << 4); }
 
-// One softmax half of Eq. 6 for one token: u[64] logits in, p[64] (fp32) out in place; the bf16 values go to the
-// token's 128-byte row of the half's 64-feature block (operand layout).  Returns sum_j bf16(p_j) * vec[j].
-template <bool kNeg>
-__device__ __forceinline__ float softmax_half_keep(float (&u)[kM], uint8_t* blk, int row, const float* vec)
-{
-    float m = kNeg ? min3(u[0], u[1], u[2]) : max3(u[0], u[1], u[2]);
-#pragma unroll
-    for (int j = 3; j < kM - 1; j += 2) m = kNeg ? min3(m, u[j], u[j + 1]) : max3(m, u[j], u[j + 1]);
-    m = kNeg ? fminf(m, u[kM - 1]) : fmaxf(m, u[kM - 1]);
-    // exp(u - max) = 2^(u*log2e - max*log2e);   exp(-u - max(-u)) = 2^(min*log2e - u*log2e)
-    const float sL = kNeg ? -kLog2e : kLog2e, off = kNeg ? m * kLog2e : -m * kLog2e;
-    // two lanes of arithmetic per instruction (packed fp32 pairs), as in the forward
-    const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
-    f32x2 sum2 = pack2(0.f, 0.f);
-#pragma unroll
-    for (int j = 0; j < kM; j += 2) {
-        float x0, x1;
-        unpack2(fma2(pack2(u[j], u[j + 1]), scale, offset), x0, x1);
-        u[j] = ex2_approx(x0);
-        u[j + 1] = ex2_approx(x1);
-        sum2 = add2(sum2, pack2(u[j], u[j + 1]));
-    }
-    float s0, s1;
-    unpack2(sum2, s0, s1);
-    const float inv = __fdividef(1.f, s0 + s1);
-    const f32x2 inv2 = pack2(inv, inv);
-    f32x2 dot2 = pack2(0.f, 0.f);
-    const float2* vec2 = reinterpret_cast<const float2*>(vec);
-#pragma unroll
-    for (int ch = 0; ch < 8; ++ch) {
-        uint32_t w[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int j = 8 * ch + 2 * q;
-            unpack2(mul2(pack2(u[j], u[j + 1]), inv2), u[j], u[j + 1]);
-            w[q] = pack_bf16(u[j], u[j + 1]);
-            const float2 zv = vec2[j >> 1];
-            // the rounded values, as the tensor core sees them
-            dot2 = fma2(pack2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xffff0000u)), pack2(zv.x, zv.y), dot2);
-        }
-        *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-    unpack2(dot2, s0, s1);
-    return s0 + s1;
-}
-
-// The same without the store: p[64] (fp32) in place, its bf16 roundings packed two to a word in pk[32] (what a tensor
+// One softmax half of Eq. 6 for one token: u[64] logits in, p[64] (fp32) out in place, its bf16 roundings packed two to a word in pk[32] (what a tensor
 // core operand built from p holds).  Returns sum_j bf16(p_j) * vec[j].
 template <bool kNeg>
 __device__ __forceinline__ float softmax_half_packed(float (&u)[kM], uint32_t (&pk)[kM / 2], const float* vec)
@@ -333,9 +309,10 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
              const __grid_constant__ CUtensorMap tmDQ, const __grid_constant__ CUtensorMap tmW,
              const __grid_constant__ CUtensorMap tmShi, const __grid_constant__ CUtensorMap tmSlo, const BwdArgs a)
 {
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ uint8_t bwd_smem[];
     using L = BwdSmemQ;
-    const BwdCta c = bwd_setup(smem_raw, L::kMisc, a.err);
+    if (!bwd_smem_fits(bwd_smem, kBwdSmemQ, a.err)) return;
+    const BwdCta c = bwd_setup(bwd_smem, L::kMisc, a.err);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int half = warp >> 2, row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -343,11 +320,11 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     float* vec = c.misc + BwdMisc::kVec / 4;
     float* sa = c.misc + BwdMisc::kA / 4;
     float* sb = c.misc + BwdMisc::kB / 4;
-    float* sdd = c.misc + BwdMisc::kDd / 4;
+    float* sdd = sb;   // dden den of the tile's tokens takes the place of the first half of sb once both halves have been read
     const uint32_t sb0 = c.sbase;
     const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
     const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
-    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0;
+    uint32_t ph_load = 0, ph_load2 = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0, ph_g = 0;
     float dr_acc = 0.f;   // Eq. 8: this thread's share of sum dout . (a - o)
     float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
 #pragma unroll
@@ -360,59 +337,120 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         tma_prefetch_desc(&tmDQ);
     }
 
-    // Loads of one tile (issued by one thread): Q and dO, at the start of a head also S (hi, lo) and W_q^T; the tile
-    // after it starts on its way into L2.
-    auto issue_loads = [&](const TileWalk& t) {
-        if (t.first()) {
-            mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
-            for (int b = 0; b < 2; ++b) {
-                tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
-                tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
-                tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
-            }
-        }
-        mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
+    // ---- copies, each issued by thread 0 ----
+    auto xbuf = [&](int b) { return sb0 + (b ? L::kX1 : L::kX0); };
+    auto load_seg = [&](const TileWalk& t) {   // S (hi, lo) and W_q^T of the head
+        mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
         for (int b = 0; b < 2; ++b) {
-            act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmQ, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
-            act_load<kLayout>(sb0 + L::kG + b * kHalfTileBytes, &tmG, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+            tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
+            tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
+            tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
         }
+    };
+    auto load_q = [&](const TileWalk& t, int buf) {
+        mbar_arrive_expect_tx(c.bar(BW_LOAD), kTileBytes);
+        for (int b = 0; b < 2; ++b) act_load<kLayout>(xbuf(buf) + b * kHalfTileBytes, &tmQ, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+    };
+    auto load_g = [&](const TileWalk& t) {   // dO; the tile after it starts on its way into L2
+        mbar_arrive_expect_tx(c.bar(BW_LOAD2), kTileBytes);
+        for (int b = 0; b < 2; ++b) act_load<kLayout>(sb0 + L::kG + b * kHalfTileBytes, &tmG, c.bar(BW_LOAD2), 64 * b, t.lt * kTile, t.g, a.H);
         TileWalk nx = t;
         nx.next();
         if (!nx.done())
-            for (int b = 0; b < 2; ++b) {
-                act_prefetch_l2<kLayout>(&tmQ, 64 * b, nx.lt * kTile, nx.g, a.H);
-                act_prefetch_l2<kLayout>(&tmG, 64 * b, nx.lt * kTile, nx.g, a.H);
-            }
+            for (int b = 0; b < 2; ++b) act_prefetch_l2<kLayout>(&tmG, 64 * b, nx.lt * kTile, nx.g, a.H);
     };
-    if (tid == 0 && !w.done()) issue_loads(w);
+    // ---- tensor-core stages, each issued by thread 0 ----
+    auto issue_t = [&]() {   // T = dO S^T (S_hi, S_lo): A = dO (K-major over c), B = S image [c][f] (rows = K)
+        constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kD, 0, 1);
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+            const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
+#pragma unroll
+            for (int k = 0; k < kD / 16; ++k)
+                mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kG, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_t,
+                            (pass | k) != 0);
+        }
+        mma_commit(c.bar(BW_MMA2));
+    };
+    // dz += phi^T dden = (phi / den)^T (dden den) of the tile whose phi / den is in the staging tile, on the CUDA cores:
+    // thread = (16-byte chunk of 8 features, group of 8 tokens)
+    auto dz_tile = [&]() {
+        const int fc = tid & 15, t0 = (tid >> 4) * 8;
+        const uint8_t* blk = c.smem + L::kP + (fc >> 3) * kHalfTileBytes;
+#pragma unroll
+        for (int t = t0; t < t0 + 8; ++t) {
+            const uint4 pv = *reinterpret_cast<const uint4*>(blk + sw_chunk(t, fc & 7));
+            const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
+            const float dd = sdd[t];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                dz_acc[2 * q] = fmaf(dd, __uint_as_float(pw[q] << 16), dz_acc[2 * q]);
+                dz_acc[2 * q + 1] = fmaf(dd, __uint_as_float(pw[q] & 0xffff0000u), dz_acc[2 * q + 1]);
+            }
+        }
+    };
+    // dq of tile (lt, g) leaves tensor memory through the staging tile (its last tensor-core stage has completed)
+    auto store_dq = [&](int lt, int g) {
+        {
+            float x[kM];
+            load64(t_work + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, sb0 + L::kP + b * kHalfTileBytes, 64 * b, lt * kTile, g, a.H);
+            bulk_commit_group();
+        }
+    };
 
-    for (; !w.done(); w.next()) {
+    // Software pipeline over the tiles of a head: the next tile's Q is fetched into the other Q buffer while this tile is
+    // worked on, and its logits are issued AHEAD of this tile's last tensor-core stage (dS, dq, dW), so that the next
+    // tile's feature map runs on the CUDA cores while the tensor core finishes this tile; dq of this tile then leaves
+    // after the next tile's feature map.  The first tile of a head starts from scratch (S and W_q change there).
+    bool ok = true;
+    bool pre = false;              // this tile's logits were issued during the previous tile
+    bool pend_q = false, pend_g = false, pend_seg = false;   // copies requested and not yet waited for (what an unwinding CTA waits for)
+    int xb = 0, prev_lt = 0, prev_g = 0;
+    if (!w.done()) {
+        if (tid == 0) {
+            load_seg(w);
+            load_q(w, 0);
+            load_g(w);
+        }
+        pend_q = pend_g = pend_seg = true;
+    }
+    for (; !w.done(); w.next(), xb ^= 1) {
         const bool first = w.first(), last = w.last();
+        TileWalk nx = w;
+        nx.next();
+        const bool ahead = !last && !nx.done();   // the next tile belongs to the same head
         LB_TRACE(0);
-        // ---- this tile's Q and dO (and, at the start of a head, S hi/lo, W_q^T) were requested one tile ago ----
         if (first) {
             if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];
-            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) break;
+            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
+            pend_seg = false;
         }
-        if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) break;
-        LB_TRACE(1);
-        // ---- U = Q W_q, and T = dO S^T (S_hi, S_lo), which needs nothing but the loaded tiles and runs under the feature map ----
-        if (tid == 0) {
-            issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
-            mma_commit(c.bar(BW_MMA));
-            constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kD, 0, 1);   // A = dO (K-major over c), B = S image [c][f] (rows = K)
-#pragma unroll
-            for (int pass = 0; pass < 2; ++pass) {
-                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
-#pragma unroll
-                for (int k = 0; k < kD / 16; ++k)
-                    mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kG, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_t,
-                                (pass | k) != 0);
+        if (!pre) {
+            // ---- from scratch: U = Q W_q once Q is there, T = dO S^T once dO is there ----
+            if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) { ok = false; break; }
+            pend_q = false;
+            if (tid == 0) {
+                issue_logits_mma(t_u, xbuf(xb), sb0 + L::kW);
+                mma_commit(c.bar(BW_MMA));
+                if (ahead) load_q(nx, xb ^ 1);
             }
-            mma_commit(c.bar(BW_MMA2));
-            bulk_wait_group_read<0>();   // the previous tile's dq has left the staging tile, which is phi's home again
+            pend_q = ahead;
+            if (!cta_wait(c, BW_LOAD2, ph_load2, kErrMmaLoad)) { ok = false; break; }
+            pend_g = false;
+            if (tid == 0) {
+                issue_t();
+                bulk_wait_group_read<0>();   // the previous tile's dq has left the staging tile, which is phi's home again
+            }
         }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
+        LB_TRACE(1);
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) { ok = false; break; }
         LB_TRACE(2);
         // ---- phi(q): p stays in registers (fp32, and its bf16 roundings); den = phi . z from the rounded values ----
         float p[kM];
@@ -420,7 +458,28 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         load64(t_u + lane_base, p);
         sa[half * kTile + row] = half == 0 ? softmax_half_packed<false>(p, pk, vec) : softmax_half_packed<true>(p, pk, vec + kM);
         LB_TRACE(3);
-        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrEpilogue)) break;   // T is there (and every thread's den part is visible)
+        if (pre) {
+            // ---- the previous tile's last stage has had the time of a feature map: its dO and (two tiles back) Q buffers
+            // are free for the copies of this tile's dO and the next tile's Q, and its dq leaves ----
+            if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
+            LB_TRACE(6);
+            if (tid == 0) {
+                load_g(w);
+                if (ahead) load_q(nx, xb ^ 1);
+            }
+            pend_g = true;
+            pend_q = ahead;
+            store_dq(prev_lt, prev_g);
+            LB_TRACE(7);
+            if (!cta_wait(c, BW_LOAD2, ph_load2, kErrMmaLoad)) { ok = false; break; }
+            LB_TRACE(12);
+            pend_g = false;
+            if (tid == 0) {
+                issue_t();
+                bulk_wait_group_read<0>();   // dq has left the staging tile
+            }
+        }
+        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrEpilogue)) { ok = false; break; }   // T is there (and every thread's den part is visible)
         LB_TRACE(4);
         // ---- dO . o = (dO S^T) . phi / den: the numerator phi S itself is never formed.  The per-token factor 1 / den of
         // dnum = dO / den is kept OUT of the tensor-core operands: dphi = (dO S^T - (dO . o) z) / den is scaled here, in
@@ -462,8 +521,6 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     unpack2(da2, d0, d1);
                     dr_acc += d0 + d1;
                 }
-                TileWalk nx = w;
-                nx.next();
                 if (!nx.done() && nx.lt * kTile + row < a.n)
                     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.mix_a + (size_t)(nx.g / a.H) * a.str_batch + (size_t)(nx.g % a.H) * a.str_head +
                                                                  (size_t)(nx.lt * kTile + row) * a.str_token + half * kM));
@@ -477,7 +534,6 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
         __syncthreads();
         const float ngo = -(sb[row] + sb[kTile + row]);   // -(dO . o) = dden * den
-        if (half == 0) sdd[row] = ngo;
         LB_TRACE(5);
         // ---- du (through the softmax of Eq. 6) ----
 #pragma unroll
@@ -485,62 +541,58 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
             unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
         }
-        du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
+        du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);   // (a CTA barrier inside: both halves of sb have been read)
+        if (half == 0) sdd[row] = ngo;
         fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
         LB_TRACE(8);
-        // ---- dS += (phi / den)^T dO, dq = du W_q^T, dW_q += Q^T du ----
+        // ---- the next tile's U = Q W_q first (it waits for nothing else), then dS += (phi / den)^T dO, dq = du W_q^T,
+        // dW_q += Q^T du ----
         if (tid == 0) {
             tcgen05_fence_after();
+            if (ahead) {
+                if (mbar_wait_abortable(c.bar(BW_LOAD), ph_load, c.wc.limit_ns(), c.wc.abort_smem)) {
+                    issue_logits_mma(t_u, xbuf(xb ^ 1), sb0 + L::kW);
+                    mma_commit(c.bar(BW_MMA));
+                } else {
+                    raise_abort(c.wc, kErrMmaLoad);   // the CTA leaves at its next wait
+                }
+            }
             constexpr uint32_t idesc_ds = make_idesc_bf16(kD, kD, 1, 1);        // A = (phi / den)^T, B = dO, both read MN-major
 #pragma unroll
             for (int k = 0; k < kTile / 16; ++k)
                 mma_bf16_ss(t_ds, desc_at(mn_tile, sb0 + L::kP + k * 2048), desc_at(mn_tile, sb0 + L::kG + k * 2048), idesc_ds,
                             (first && k == 0) ? 0u : 1u);
-            issue_dx_dw(t_work, t_dw, sb0 + L::kDu, sb0 + L::kX, sb0 + L::kW, first);
-            mma_commit(c.bar(BW_MMA));
+            issue_dx_dw(t_work, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
+            mma_commit(c.bar(BW_G));
         }
-        {
-            // dz += phi^T dden = (phi / den)^T (dden den) on the CUDA cores while the tensor core works: thread =
-            // (16-byte chunk of 8 features, group of 8 tokens)
-            const int fc = tid & 15, t0 = (tid >> 4) * 8;
-            const uint8_t* blk = c.smem + L::kP + (fc >> 3) * kHalfTileBytes;
-#pragma unroll
-            for (int t = t0; t < t0 + 8; ++t) {
-                const uint4 pv = *reinterpret_cast<const uint4*>(blk + sw_chunk(t, fc & 7));
-                const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
-                const float dd = sdd[t];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    dz_acc[2 * q] = fmaf(dd, __uint_as_float(pw[q] << 16), dz_acc[2 * q]);
-                    dz_acc[2 * q + 1] = fmaf(dd, __uint_as_float(pw[q] & 0xffff0000u), dz_acc[2 * q + 1]);
-                }
-            }
+        if (ahead) {
+            ph_load ^= 1u;   // thread 0 has waited for that phase on everybody's behalf
+            pend_q = false;
         }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
+        LB_TRACE(13);
+        dz_tile();   // while the tensor core works
+        LB_TRACE(14);
+        pre = ahead;
+        prev_lt = w.lt;
+        prev_g = w.g;
+        if (ahead) continue;
+
+        // ---- the last tile of the head (or of the run): finished here, nothing of the next tile in flight ----
+        if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
         LB_TRACE(9);
-        if (tid == 0) {
-            // every operand tile of this tile has been consumed: the next tile's loads overlap the store of this one
-            TileWalk nx = w;
-            nx.next();
-            if (!nx.done()) issue_loads(nx);
+        if (tid == 0 && !nx.done()) {
+            // S, W_q and every tile buffer are free: the next head's copies overlap this tile's stores
+            load_seg(nx);
+            load_q(nx, xb ^ 1);
+            load_g(nx);
         }
-        {
-            float x[kM];
-            load64(t_work + lane_base + half * kM, x);
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
+        if (!nx.done()) pend_q = pend_g = pend_seg = true;
+        store_dq(w.lt, w.g);
         LB_TRACE(10);
-        if (tid == 0) {
-            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-            bulk_commit_group();
-        }
         // ---- end of this CTA's part of the head: the accumulators go to the (CTA, head) records ----
-        if (last) {
+        {
             tcgen05_fence_after();
             float* rec = a.part_state + (size_t)(blockIdx.x + w.g) * kE;
             {
@@ -550,7 +602,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 for (int j = 0; j < kM; ++j) rec[(size_t)(half * kM + j) * kD + row] = x[j];
             }
             drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
-            // dz: the 16 token groups' sums, in group order (the scratch tile is free at this point)
+            // dz: the 16 token groups' sums, in group order (the du tile has been consumed)
             float* red = reinterpret_cast<float*>(c.smem + L::kRed);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -568,6 +620,12 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         tcgen05_fence_before();
         __syncthreads();
         LB_TRACE(11);
+    }
+    if (!ok && tid == 0) {
+        // unwinding: let the copies already requested land before the CTA gives its shared memory back
+        if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
+        if (pend_q) mbar_wait(c.bar(BW_LOAD), ph_load, c.wc.limit_ns());
+        if (pend_g) mbar_wait(c.bar(BW_LOAD2), ph_load2, c.wc.limit_ns());
     }
     if (kMixB) {
         // the CTA's sum of dout . (a - o), thread by thread in index order (bit-reproducible)
@@ -591,18 +649,20 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
              const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmShi,
              const __grid_constant__ CUtensorMap tmSlo, const BwdArgs a)
 {
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ uint8_t bwd_smem[];
     using L = BwdSmemK;
-    const BwdCta c = bwd_setup(smem_raw, L::kMisc, a.err);
+    if (!bwd_smem_fits(bwd_smem, kBwdSmemK, a.err)) return;
+    const BwdCta c = bwd_setup(bwd_smem, L::kMisc, a.err);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int half = warp >> 2, row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t t_u = c.tmem, t_w1 = c.tmem + 64, t_w2 = c.tmem + 192, t_dw = c.tmem + 320;
+    // tensor memory: logits | T = V dS^T | dv | dW_k | dk
+    const uint32_t t_u = c.tmem, t_t = c.tmem + 64, t_dv = c.tmem + 192, t_dw = c.tmem + 320, t_dk = c.tmem + 384;
     float* vec = c.misc + BwdMisc::kVec / 4;
     const uint32_t sb0 = c.sbase;
     const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
     const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
-    uint32_t ph_load = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0;
+    uint32_t ph_load = 0, ph_load2 = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0, ph_g = 0;
     TileWalk w;
     w.init(a.total_tiles, a.tiles_per_head);
     if (tid == 0) {
@@ -612,129 +672,203 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         tma_prefetch_desc(&tmDV);
     }
 
-    // Loads of one tile (issued by one thread): K and V, at the start of a head also dS (hi, lo) and W_k^T.
-    auto issue_loads = [&](const TileWalk& t) {
-        if (t.first()) {
-            mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
-            for (int b = 0; b < 2; ++b) {
-                tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
-                tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
-                tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
-            }
-        }
-        mbar_arrive_expect_tx(c.bar(BW_LOAD), 2 * kTileBytes);
+    // ---- copies, each issued by thread 0 ----
+    auto xbuf = [&](int b) { return sb0 + (b ? L::kX1 : L::kX0); };
+    auto load_seg = [&](const TileWalk& t) {   // dS (hi, lo) and W_k^T of the head
+        mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
         for (int b = 0; b < 2; ++b) {
-            act_load<kLayout>(sb0 + L::kX + b * kHalfTileBytes, &tmK, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
-            act_load<kLayout>(sb0 + L::kV + b * kHalfTileBytes, &tmV, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+            tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
+            tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
+            tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
         }
+    };
+    auto load_k = [&](const TileWalk& t, int buf) {
+        mbar_arrive_expect_tx(c.bar(BW_LOAD), kTileBytes);
+        for (int b = 0; b < 2; ++b) act_load<kLayout>(xbuf(buf) + b * kHalfTileBytes, &tmK, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
+    };
+    auto load_v = [&](const TileWalk& t) {   // V; the tile after it starts on its way into L2
+        mbar_arrive_expect_tx(c.bar(BW_LOAD2), kTileBytes);
+        for (int b = 0; b < 2; ++b) act_load<kLayout>(sb0 + L::kV + b * kHalfTileBytes, &tmV, c.bar(BW_LOAD2), 64 * b, t.lt * kTile, t.g, a.H);
         TileWalk nx = t;
         nx.next();
         if (!nx.done())
-            for (int b = 0; b < 2; ++b) {
-                act_prefetch_l2<kLayout>(&tmK, 64 * b, nx.lt * kTile, nx.g, a.H);
-                act_prefetch_l2<kLayout>(&tmV, 64 * b, nx.lt * kTile, nx.g, a.H);
-            }
+            for (int b = 0; b < 2; ++b) act_prefetch_l2<kLayout>(&tmV, 64 * b, nx.lt * kTile, nx.g, a.H);
     };
-    if (tid == 0 && !w.done()) issue_loads(w);
-
-    for (; !w.done(); w.next()) {
-        const bool first = w.first(), last = w.last();
-        if (first) {
-            if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // dz
-            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) break;
-        }
-        if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) break;
-        // ---- U = K W_k, and T = V dS^T (hi and lo parts of dS), which needs nothing but the loaded tiles ----
-        if (tid == 0) {
-            issue_logits_mma(t_u, sb0 + L::kX, sb0 + L::kW);
-            mma_commit(c.bar(BW_MMA));
-            constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);   // A = V (K-major over c), B = dS image [c][f] (rows = K)
+    // ---- T = V dS^T (hi and lo parts of dS): A = V (K-major over c), B = dS image [c][f] (rows = K); issued by thread 0 ----
+    auto issue_t = [&]() {
+        constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);
 #pragma unroll
-            for (int pass = 0; pass < 2; ++pass) {
-                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
+        for (int pass = 0; pass < 2; ++pass) {
+            const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
 #pragma unroll
-                for (int k = 0; k < kD / 16; ++k)
-                    mma_bf16_ss(t_w1, desc_at(kmajor, kstep_kmajor(sb0 + L::kV, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
-                                (pass | k) != 0);
-            }
-            mma_commit(c.bar(BW_MMA2));
-            bulk_wait_group_read<0>();   // the previous tile's dk has left phi's tile
+            for (int k = 0; k < kD / 16; ++k)
+                mma_bf16_ss(t_t, desc_at(kmajor, kstep_kmajor(sb0 + L::kV, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
+                            (pass | k) != 0);
         }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) break;
-        float p[kM];
-        load64(t_u + lane_base, p);
-        {
-            uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
-            if (half == 0) softmax_half_keep<false>(p, blk, row, vec);
-            else softmax_half_keep<true>(p, blk, row, vec + kM);
-        }
-        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrMmaAcc)) break;
-        // ---- dphi = V dS^T + dz -> du ----
+        mma_commit(c.bar(BW_MMA2));
+    };
+    // dv and dk of tile (lt, g) leave tensor memory (the tile's last tensor-core stage has completed): dv through phi's
+    // tile, dk through V's (this tile's V dS^T has been formed; thread 0 asks for the next V only once the store has read it)
+    auto store_dv_dk = [&](int lt, int g) {
         {
             float x[kM];
-            load64(t_w1 + lane_base + half * kM, x);
-#pragma unroll
-            for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
-            du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
+            load64(t_dv + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
+        }
+        {
+            float x[kM];
+            load64(t_dk + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kV + half * kHalfTileBytes, row, x);
         }
         fence_proxy_async_smem();
         tcgen05_fence_before();
         __syncthreads();
-        // ---- dv = phi dS (hi and lo parts), dk = du W_k^T, dW_k += K^T du ----
+        if (tid == 0) {
+            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, lt * kTile, g, a.H);
+            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, sb0 + L::kV + b * kHalfTileBytes, 64 * b, lt * kTile, g, a.H);
+            bulk_commit_group();
+        }
+    };
+
+    // Software pipeline over the tiles of a head, as on the query side: the next tile's K is fetched into the other K
+    // buffer, its V into V's tile once dk has left it, and its logits and V dS^T are issued around this tile's last
+    // tensor-core stage (dv, dk, dW), so that the next tile's feature map runs while the tensor core finishes this tile.
+    bool ok = true;
+    bool pre = false;              // this tile's logits and V dS^T were issued during the previous tile
+    bool pend_k = false, pend_v = false, pend_seg = false;   // copies requested and not yet waited for
+    int xb = 0, prev_lt = 0, prev_g = 0;
+    if (!w.done()) {
+        if (tid == 0) {
+            load_seg(w);
+            load_k(w, 0);
+            load_v(w);
+        }
+        pend_k = pend_v = pend_seg = true;
+    }
+    for (; !w.done(); w.next(), xb ^= 1) {
+        const bool first = w.first(), last = w.last();
+        TileWalk nx = w;
+        nx.next();
+        const bool ahead = !last && !nx.done();   // the next tile belongs to the same head
+        if (first) {
+            if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // dz
+            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
+            pend_seg = false;
+        }
+        if (!pre) {
+            // ---- from scratch: U = K W_k once K is there, T = V dS^T once V is there ----
+            if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) { ok = false; break; }
+            pend_k = false;
+            if (tid == 0) {
+                issue_logits_mma(t_u, xbuf(xb), sb0 + L::kW);
+                mma_commit(c.bar(BW_MMA));
+                if (ahead) load_k(nx, xb ^ 1);
+            }
+            pend_k = ahead;
+            if (!cta_wait(c, BW_LOAD2, ph_load2, kErrMmaLoad)) { ok = false; break; }
+            pend_v = false;
+            if (tid == 0) issue_t();
+        }
+        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) { ok = false; break; }
+        // ---- phi(k): p stays in registers (fp32, and its bf16 roundings, which go to phi's tile once that is free) ----
+        float p[kM];
+        uint32_t pk[kM / 2];
+        load64(t_u + lane_base, p);
+        if (half == 0) softmax_half_packed<false>(p, pk, vec);
+        else softmax_half_packed<true>(p, pk, vec + kM);
+        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrMmaAcc)) { ok = false; break; }   // T is there: V's tile is free
+        if (pre) {
+            // ---- the previous tile's last stage has had the time of a feature map: its dv and dk leave, and the K buffer
+            // two tiles back takes the next tile's K ----
+            if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
+            if (tid == 0 && ahead) load_k(nx, xb ^ 1);
+            pend_k = ahead;
+            store_dv_dk(prev_lt, prev_g);
+        }
+        // ---- dphi = V dS^T + dz -> du ----
+        {
+            float x[kM];
+            load64(t_t + lane_base + half * kM, x);
+#pragma unroll
+            for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
+            if (tid == 0) {
+                bulk_wait_group_read<0>();   // the stores have read phi's and V's tiles
+                if (ahead) load_v(nx);
+            }
+            du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);   // (a CTA barrier inside: phi's tile is free for everybody)
+        }
+        pend_v = ahead;
+        {
+            uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch)
+                *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+        }
+        fence_proxy_async_smem();
+        tcgen05_fence_before();
+        __syncthreads();
+        // ---- the next tile's U = K W_k first, then dv = phi dS (hi and lo parts), dk = du W_k^T, dW_k += K^T du, then the
+        // next tile's V dS^T ----
         if (tid == 0) {
             tcgen05_fence_after();
+            if (ahead) {
+                if (mbar_wait_abortable(c.bar(BW_LOAD), ph_load, c.wc.limit_ns(), c.wc.abort_smem)) {
+                    issue_logits_mma(t_u, xbuf(xb ^ 1), sb0 + L::kW);
+                    mma_commit(c.bar(BW_MMA));
+                } else {
+                    raise_abort(c.wc, kErrMmaLoad);   // the CTA leaves at its next wait
+                }
+            }
             constexpr uint32_t idesc_dv = make_idesc_bf16(kTile, kD, 0, 0);     // A = phi (K-major over f), B = dS image [c][f] (rows = N)
 #pragma unroll
             for (int pass = 0; pass < 2; ++pass) {
                 const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k)
-                    mma_bf16_ss(t_w2, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)), desc_at(kmajor, kstep_kmajor(st, k, kHalfTileBytes)),
+                    mma_bf16_ss(t_dv, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)), desc_at(kmajor, kstep_kmajor(st, k, kHalfTileBytes)),
                                 idesc_dv, (pass | k) != 0);
             }
-            issue_dx_dw(t_w1, t_dw, sb0 + L::kDu, sb0 + L::kX, sb0 + L::kW, first);
-            mma_commit(c.bar(BW_MMA));
-        }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrStore)) break;
-        if (tid == 0) {
-            // K, V, phi and the du tile have been consumed: the next tile's loads start now and overlap this tile's stores
-            TileWalk nx = w;
-            nx.next();
-            if (!nx.done()) issue_loads(nx);
-        }
-        // ---- dv, then dk, leave through phi's tile ----
-        {
-            float x[kM];
-            load64(t_w2 + lane_base + half * kM, x);
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        {
-            float x[kM];
-            load64(t_w1 + lane_base + half * kM, x);   // dk comes out of tensor memory while dv's store reads the tile
-            if (tid == 0) {
-                for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-                bulk_commit_group();
-                bulk_wait_group_read<0>();
+            issue_dx_dw(t_dk, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
+            mma_commit(c.bar(BW_G));
+            if (ahead) {
+                if (mbar_wait_abortable(c.bar(BW_LOAD2), ph_load2, c.wc.limit_ns(), c.wc.abort_smem)) issue_t();
+                else raise_abort(c.wc, kErrMmaLoad);
             }
-            __syncthreads();
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
         }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
+        if (ahead) {
+            ph_load ^= 1u;    // thread 0 has waited for these phases on everybody's behalf
+            ph_load2 ^= 1u;
+            pend_k = pend_v = false;
+        }
+        pre = ahead;
+        prev_lt = w.lt;
+        prev_g = w.g;
+        if (ahead) continue;
+
+        // ---- the last tile of the head (or of the run): finished here, nothing of the next tile in flight ----
+        if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
+        if (tid == 0 && !nx.done()) {
+            // dS, W_k and the K buffers are free: the next head's copies overlap this tile's stores
+            load_seg(nx);
+            load_k(nx, xb ^ 1);
+        }
+        if (!nx.done()) pend_k = pend_seg = true;
+        store_dv_dk(w.lt, w.g);
         if (tid == 0) {
-            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-            bulk_commit_group();
+            bulk_wait_group_read<0>();
+            if (!nx.done()) load_v(nx);
         }
-        if (last) {
-            tcgen05_fence_after();
-            drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
-        }
+        if (!nx.done()) pend_v = true;
+        tcgen05_fence_after();
+        drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
         tcgen05_fence_before();
         __syncthreads();
+    }
+    if (!ok && tid == 0) {
+        // unwinding: let the copies already requested land before the CTA gives its shared memory back
+        if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
+        if (pend_k) mbar_wait(c.bar(BW_LOAD), ph_load, c.wc.limit_ns());
+        if (pend_v) mbar_wait(c.bar(BW_LOAD2), ph_load2, c.wc.limit_ns());
     }
     bwd_teardown(c);
 }

@@ -52,7 +52,8 @@ constexpr float kLog2e = 1.4426950408889634f;
 // error codes OR-ed into *err (which wait gave up)
 enum : uint32_t {
     kErrProducer = 1u, kErrMmaLoad = 2u, kErrMmaU = 4u, kErrMmaPhi = 8u, kErrMmaAcc = 16u,
-    kErrSoftmaxU = 32u, kErrDrain = 64u, kErrEpilogue = 128u, kErrSeg = 256u, kErrStore = 512u, kErrGrid = 1024u
+    kErrSoftmaxU = 32u, kErrDrain = 64u, kErrEpilogue = 128u, kErrSeg = 256u, kErrStore = 512u, kErrGrid = 1024u,
+    kErrSmem = 2048u   // not a wait: the kernel's shared-memory window did not hold its layout
 };
 
 // CTA that owns tile t when T tiles are split over P CTAs (CTA c owns [c*T/P, (c+1)*T/P)).

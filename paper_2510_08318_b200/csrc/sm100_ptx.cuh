@@ -116,6 +116,27 @@ __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// Barrier `id` over `threads` threads that also AND-reduces a predicate: every participant gets the same verdict.
+__device__ __forceinline__ bool named_barrier_and(uint32_t id, uint32_t threads, bool pred)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %3, 0;\n\t"
+        "bar.red.and.pred p, %1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(out)
+        : "r"(id), "r"(threads), "r"(pred ? 1u : 0u)
+        : "memory");
+    return out != 0u;
+}
+// Registers per thread of the executing warp group (4 consecutive warps, all of which execute this): give some back, or
+// take more from the pool the other groups gave back to.
+template <int kRegs> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs)); }
+template <int kRegs> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs)); }
+
 // ---- TMA (tiled, rank 3, this GPU's memory only, never multicast) --------------------------------
 
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap)
