@@ -31,7 +31,15 @@
 namespace linattn {
 namespace tc {
 
-constexpr int kBwdThreads = 256;
+// Warps 0-7 do the element-wise work (thread = (token, half of the features)); warp 8 issues every copy and every
+// tensor-core product; warps 9-11 only complete warp 8's group of four, which gives most of its registers to the others.
+constexpr int kBwdThreads = 384;
+constexpr int kBwdCompute = 256;
+constexpr int kBwdIssuer = 8;
+// Registers per thread after the split.  A CTA of 384 threads starts with 168 each, and what the three warp groups hold
+// afterwards can only come out of that: 2 x element-wise + issuer <= 3 x 168 (a request beyond it would wait for ever).
+constexpr int kBwdRegsCompute = 216, kBwdRegsIssuer = 72;
+static_assert(2 * kBwdRegsCompute + kBwdRegsIssuer <= 3 * 168 && kBwdRegsCompute % 8 == 0 && kBwdRegsIssuer % 8 == 0, "register split");
 constexpr int kWRec = kM * kD;   // floats per weight-gradient record, stored [j][c]
 
 struct BwdArgs {
@@ -94,16 +102,19 @@ struct BwdMisc {
     static constexpr uint32_t kVec = 0;           // 128 floats: z (query side) or dz (key side)
     static constexpr uint32_t kA = 512;           // 2 x 128 floats: den halves
     static constexpr uint32_t kB = 1536;          // 2 x 128 floats: (dO . o) halves; then, in the first 128, dden den of the tile
-    static constexpr uint32_t kBars = 2560;       // 6 mbarriers, TMEM slot, abort word
-    static constexpr uint32_t kBytes = 2560 + 64;
+    static constexpr uint32_t kBars = 2560;       // 10 mbarriers, TMEM slot, abort word
+    static constexpr uint32_t kBytes = 2560 + 96;
 };
 constexpr uint32_t kBwdSmemQ = BwdSmemQ::kMisc + BwdMisc::kBytes;
 constexpr uint32_t kBwdSmemK = BwdSmemK::kMisc + BwdMisc::kBytes;
 static_assert(kBwdSmemQ <= 232448 && kBwdSmemK <= 232448, "a CTA has 227 KB of shared memory");
 
-// BW_LOAD: the tile that feeds the logits; BW_LOAD2: the other input tile; BW_MMA: logits; BW_MMA2: the product with the
-// hi and lo images; BW_G: the tile's last tensor-core stage
-enum : int { BW_LOAD = 0, BW_SEG = 1, BW_MMA = 2, BW_MMA2 = 3, BW_G = 4, BW_LOAD2 = 5, BW_NBARS = 6 };
+// mbarriers.  Copies: BW_X0 / BW_X1 the two buffers of the tile that feeds the logits, BW_IN2 the other input tile,
+// BW_SEG the head's images and weights.  Issuer -> element-wise warps: BW_LFULL logits, BW_TFULL the product with the
+// images, BW_GFULL the tile's last tensor-core stage, BW_PFREE the staging tile has been read by its store.
+// Element-wise warps -> issuer (one arrival per warp): BW_OPS the operands of the last stage are written, BW_STAGED the
+// results have been staged for their stores.
+enum : int { BW_X0 = 0, BW_X1 = 1, BW_IN2 = 2, BW_SEG = 3, BW_LFULL = 4, BW_TFULL = 5, BW_GFULL = 6, BW_PFREE = 7, BW_OPS = 8, BW_STAGED = 9, BW_NBARS = 10 };
 
 struct BwdCta {
     uint8_t* smem;
@@ -141,7 +152,7 @@ __device__ __forceinline__ BwdCta bwd_setup(uint8_t* smem_raw, uint32_t misc_off
     c.wc.abort_smem = smem_u32(abort_word);
     if (threadIdx.x == 0) {
         *abort_word = 0u;
-        for (int i = 0; i < BW_NBARS; ++i) mbar_init(c.bar(i), 1);
+        for (int i = 0; i < BW_NBARS; ++i) mbar_init(c.bar(i), (i == BW_OPS || i == BW_STAGED) ? kBwdCompute / 32 : 1);
         fence_mbar_init();
     }
     if ((threadIdx.x >> 5) == 1) {
@@ -158,21 +169,41 @@ __device__ __forceinline__ BwdCta bwd_setup(uint8_t* smem_raw, uint32_t misc_off
 
 __device__ __forceinline__ void bwd_teardown(const BwdCta& c)
 {
-    if (threadIdx.x == 0) bulk_wait_group<0>();
     tcgen05_fence_before();
     __syncthreads();
     if ((threadIdx.x >> 5) == 1) tmem_dealloc(c.tmem, 512);
 }
 
-// All threads of the CTA wait (bounded) for the barrier's phase; the verdict is the same for every thread, so the
-// stage loop never leaves some threads behind at a CTA barrier.
-__device__ __forceinline__ bool cta_wait(const BwdCta& c, int b, uint32_t& phase, uint32_t code)
+// Barrier of the element-wise warps.
+__device__ __forceinline__ void cbar() { named_barrier_sync(1, kBwdCompute); }
+// The same with a verdict: false for everybody if any thread brings false (a wait of its own that gave up).
+__device__ __forceinline__ bool cbar_and(bool ok) { return named_barrier_and(1, kBwdCompute, ok); }
+
+// All element-wise threads wait (bounded) for the barrier's phase and meet; the verdict is the same for every one of
+// them, so the stage loop never leaves some of them behind at a barrier.  `ok` carries the verdict of earlier waits
+// that did not meet (wait_only).
+__device__ __forceinline__ bool compute_wait(const BwdCta& c, int b, uint32_t& phase, uint32_t code, bool ok = true)
 {
-    const bool ok = warp_wait(c.bar(b), phase, c.wc, code);
+    const bool mine = warp_wait(c.bar(b), phase, c.wc, code);
     phase ^= 1u;
-    const bool all = __syncthreads_and(ok ? 1 : 0) != 0;
+    const bool all = cbar_and(ok && mine);
     tcgen05_fence_after();
     return all;
+}
+__device__ __forceinline__ bool wait_only(const BwdCta& c, int b, uint32_t& phase, uint32_t code)
+{
+    const bool mine = warp_wait(c.bar(b), phase, c.wc, code);
+    phase ^= 1u;
+    tcgen05_fence_after();
+    return mine;
+}
+// What a warp has written (shared memory for the tensor core or a store, tensor memory reads done) is announced to the issuer.
+__device__ __forceinline__ void warp_announce(const BwdCta& c, int b)
+{
+    fence_proxy_async_smem();
+    tcgen05_fence_before();
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(c.bar(b));
 }
 
 // Byte offset of 16-byte chunk `ch` (8 bf16) of row `row` inside a 64-column block of a TMA tile (128-byte swizzle).
@@ -240,7 +271,7 @@ __device__ __forceinline__ void store_row_bf16(uint8_t* blk, int row, const floa
 // Softmax backward of Eq. 6 for one token, split between the two threads of the token (half 0: softmax(+u),
 // half 1: softmax(-u)): each forms p (.) (dphi - p . dphi) for its half; half 1 parks its 64 values in 64 free columns
 // of the token's lane of tensor memory (`park`: the logits' columns, read long before; both threads of a token sit on
-// warps of the same lane quarter, so either can reach the lane), and after a CTA barrier half 0 takes them back,
+// warps of the same lane quarter, so either can reach the lane), and after a barrier of these warps half 0 takes them back,
 // subtracts and writes du (bf16) to its row of the du tile.
 __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint32_t park, uint8_t* du_tile)
 {
@@ -262,7 +293,7 @@ __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[
         tmem_wait_st();
     }
     tcgen05_fence_before();
-    __syncthreads();
+    cbar();
     tcgen05_fence_after();
     if (half == 0) {
         float o[kM];
@@ -273,24 +304,62 @@ __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[
     }
 }
 
-// K-major operand (rows x K, K contiguous in 64-element blocks `blk_bytes` apart): address of K step k (16 elements).
-__device__ __forceinline__ uint32_t kstep_kmajor(uint32_t base, int k, uint32_t blk_bytes) { return base + (uint32_t)(k >> 2) * blk_bytes + (uint32_t)(k & 3) * 32u; }
+// n products D (+)= A_k B_k issued by one thread, the operands' start addresses advancing by fixed byte steps.  The loop
+// is NOT unrolled on purpose: the issuer warp runs on few registers, and the descriptor arithmetic of unrolled products
+// is hoisted out of the tile loop and spilled.
+__device__ __forceinline__ void mma_chain(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t step_a, uint32_t step_b, uint32_t idesc, int n,
+                                          uint32_t acc_first)
+{
+#pragma unroll 1
+    for (int k = 0; k < n; ++k) {
+        mma_bf16_ss(d_tmem, da, db, idesc, k > 0 ? 1u : acc_first);
+        da += step_a >> 4;
+        db += step_b >> 4;
+    }
+}
+// K-major operand tiles are two 64-element blocks of four K steps each (32 bytes apart).
+__device__ __forceinline__ uint64_t kmajor_desc() { return make_desc_sw128(0, 16, 1024); }
+__device__ __forceinline__ uint64_t mn_desc(uint32_t blk_bytes) { return make_desc_sw128(0, blk_bytes, 1024); }
 
-// dx = du W^T and dW += x^T du for one tile (issued by one thread): A of the first product is the du tile (K-major,
-// K = 64), B the W^T image [j][c] read MN-major; the second product reads the x tile MN-major (x^T) and du MN-major.
-__device__ __forceinline__ void issue_dx_dw(uint32_t t_dx, uint32_t t_dw, uint32_t du, uint32_t x, uint32_t w, bool first_of_segment)
+// U = X W (logits) of one tile: A = X tile, B = W^T image, both K-major.
+__device__ __forceinline__ void chain_logits(uint32_t d_tmem, uint32_t x, uint32_t w)
+{
+    constexpr uint32_t idesc = make_idesc_bf16(kTile, kM, 0, 0);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), x), desc_at(kmajor_desc(), w), 32, 32, idesc, 4, 0u);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), x + kHalfTileBytes), desc_at(kmajor_desc(), w + kWBytes / 2), 32, 32, idesc, 4, 1u);
+}
+// T = Y (S_hi + S_lo)^T: A = Y tile (K-major over c), B = image [c][f] read with rows = K (hi pass, then lo pass).
+__device__ __forceinline__ void chain_images(uint32_t d_tmem, uint32_t y, uint32_t img_hi, uint32_t img_lo)
+{
+    constexpr uint32_t idesc = make_idesc_bf16(kTile, kD, 0, 1);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), y), desc_at(mn_desc(kHalfTileBytes), img_hi), 32, 2048, idesc, 4, 0u);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), y + kHalfTileBytes), desc_at(mn_desc(kHalfTileBytes), img_hi + 4 * 2048), 32, 2048, idesc, 4, 1u);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), y), desc_at(mn_desc(kHalfTileBytes), img_lo), 32, 2048, idesc, 4, 1u);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), y + kHalfTileBytes), desc_at(mn_desc(kHalfTileBytes), img_lo + 4 * 2048), 32, 2048, idesc, 4, 1u);
+}
+// dv = phi (dS_hi + dS_lo): A = phi tile (K-major over f), B = image [c][f] read with rows = N (both K-major).
+__device__ __forceinline__ void chain_dv(uint32_t d_tmem, uint32_t phi, uint32_t img_hi, uint32_t img_lo)
+{
+    constexpr uint32_t idesc = make_idesc_bf16(kTile, kD, 0, 0);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), phi), desc_at(kmajor_desc(), img_hi), 32, 32, idesc, 4, 0u);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), phi + kHalfTileBytes), desc_at(kmajor_desc(), img_hi + kHalfTileBytes), 32, 32, idesc, 4, 1u);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), phi), desc_at(kmajor_desc(), img_lo), 32, 32, idesc, 4, 1u);
+    mma_chain(d_tmem, desc_at(kmajor_desc(), phi + kHalfTileBytes), desc_at(kmajor_desc(), img_lo + kHalfTileBytes), 32, 32, idesc, 4, 1u);
+}
+// dS += (phi / den)^T dO: A and B are token tiles read MN-major (K = the tile's tokens).
+__device__ __forceinline__ void chain_ds(uint32_t d_tmem, uint32_t phi, uint32_t g, bool first_of_segment)
+{
+    constexpr uint32_t idesc = make_idesc_bf16(kD, kD, 1, 1);
+    mma_chain(d_tmem, desc_at(mn_desc(kHalfTileBytes), phi), desc_at(mn_desc(kHalfTileBytes), g), 2048, 2048, idesc, kTile / 16, first_of_segment ? 0u : 1u);
+}
+// dx = du W^T and dW += x^T du for one tile: A of the first product is the du tile (K-major, K = 64), B the W^T image
+// [j][c] read MN-major; the second product reads the x tile MN-major (x^T) and du MN-major.
+__device__ __forceinline__ void chain_dx_dw(uint32_t t_dx, uint32_t t_dw, uint32_t du, uint32_t x, uint32_t w, bool first_of_segment)
 {
     constexpr uint32_t idesc_dx = make_idesc_bf16(kTile, kD, 0, 1);
     constexpr uint32_t idesc_dw = make_idesc_bf16(kD, kM, 1, 1);
-    const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
-    const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
-    const uint64_t mn_w = make_desc_sw128(0, kWBytes / 2, 1024);
-#pragma unroll
-    for (int k = 0; k < kM / 16; ++k)
-        mma_bf16_ss(t_dx, desc_at(kmajor, du + k * 32), desc_at(mn_w, w + k * 2048), idesc_dx, k > 0);
-#pragma unroll
-    for (int k = 0; k < kTile / 16; ++k)
-        mma_bf16_ss(t_dw, desc_at(mn_tile, x + k * 2048), desc_at(mn_tile, du + k * 2048), idesc_dw, (first_of_segment && k == 0) ? 0u : 1u);
+    mma_chain(t_dx, desc_at(kmajor_desc(), du), desc_at(mn_desc(kWBytes / 2), w), 32, 2048, idesc_dx, kM / 16, 0u);
+    mma_chain(t_dw, desc_at(mn_desc(kHalfTileBytes), x), desc_at(mn_desc(kHalfTileBytes), du), 2048, 2048, idesc_dw, kTile / 16, first_of_segment ? 0u : 1u);
 }
 
 // Write the weight-gradient accumulator (TMEM: lane = input feature c, 64 columns = logits j) as a [j][c] record.
@@ -303,6 +372,23 @@ __device__ __forceinline__ void drain_dw(uint32_t t_dw, uint32_t lane_base, int 
     for (int j = 0; j < 32; ++j) rec[(size_t)(half * 32 + j) * kD + row] = __uint_as_float(v[j]);
 }
 
+// The issuer's waits: the whole warp waits (bounded), the verdict is warp-uniform.
+__device__ __forceinline__ bool issuer_wait(const BwdCta& c, int b, uint32_t& phase, uint32_t code)
+{
+    const bool ok = warp_wait(c.bar(b), phase, c.wc, code);
+    phase ^= 1u;
+    tcgen05_fence_after();
+    return ok;
+}
+
+// Schedule of a head's tiles, both kernels (i = tile):
+//   issuer:        wait OPS(i) | logits(i+1), last stage(i) | copies into the buffers that stage frees | T(i+1) |
+//                  wait STAGED(i), stores of tile i, PFREE
+//   element-wise:  feature map(i+1) | wait GFULL(i), results of tile i to their staging tiles, STAGED(i) |
+//                  wait TFULL(i+1), ... du(i+1), operands of the last stage written, OPS(i+1)
+// so the tensor core works on tile i's last stage and tile i+1's first products while the CUDA cores run tile i+1's
+// feature map and convert tile i's results.  The first tile of a head starts from scratch (images and weights change
+// there) and the last one is finished before the next head's copies are requested.
 template <int kLayout, int kMixB>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmG,
@@ -314,329 +400,319 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (!bwd_smem_fits(bwd_smem, kBwdSmemQ, a.err)) return;
     const BwdCta c = bwd_setup(bwd_smem, L::kMisc, a.err);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int half = warp >> 2, row = (warp & 3) * 32 + lane;
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t t_u = c.tmem, t_work = c.tmem + 64, t_ds = c.tmem + 208, t_dw = c.tmem + 336;
-    float* vec = c.misc + BwdMisc::kVec / 4;
-    float* sa = c.misc + BwdMisc::kA / 4;
-    float* sb = c.misc + BwdMisc::kB / 4;
-    float* sdd = sb;   // dden den of the tile's tokens takes the place of the first half of sb once both halves have been read
+    // tensor memory: logits (later the du exchange) | T = dO S^T | dS | dW_q | dq
+    const uint32_t t_u = c.tmem, t_t = c.tmem + 64, t_ds = c.tmem + 192, t_dw = c.tmem + 320, t_dq = c.tmem + 384;
     const uint32_t sb0 = c.sbase;
-    const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
-    const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
-    uint32_t ph_load = 0, ph_load2 = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0, ph_g = 0;
-    float dr_acc = 0.f;   // Eq. 8: this thread's share of sum dout . (a - o)
-    float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
-#pragma unroll
-    for (int e = 0; e < 8; ++e) dz_acc[e] = 0.f;
     TileWalk w;
     w.init(a.total_tiles, a.tiles_per_head);
-    if (tid == 0) {
-        tma_prefetch_desc(&tmQ);
-        tma_prefetch_desc(&tmG);
-        tma_prefetch_desc(&tmDQ);
-    }
 
-    // ---- copies, each issued by thread 0 ----
-    auto xbuf = [&](int b) { return sb0 + (b ? L::kX1 : L::kX0); };
-    auto load_seg = [&](const TileWalk& t) {   // S (hi, lo) and W_q^T of the head
-        mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
-        for (int b = 0; b < 2; ++b) {
-            tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
-            tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
-            tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
-        }
-    };
-    auto load_q = [&](const TileWalk& t, int buf) {
-        mbar_arrive_expect_tx(c.bar(BW_LOAD), kTileBytes);
-        for (int b = 0; b < 2; ++b) act_load<kLayout>(xbuf(buf) + b * kHalfTileBytes, &tmQ, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
-    };
-    auto load_g = [&](const TileWalk& t) {   // dO; the tile after it starts on its way into L2
-        mbar_arrive_expect_tx(c.bar(BW_LOAD2), kTileBytes);
-        for (int b = 0; b < 2; ++b) act_load<kLayout>(sb0 + L::kG + b * kHalfTileBytes, &tmG, c.bar(BW_LOAD2), 64 * b, t.lt * kTile, t.g, a.H);
-        TileWalk nx = t;
-        nx.next();
-        if (!nx.done())
-            for (int b = 0; b < 2; ++b) act_prefetch_l2<kLayout>(&tmG, 64 * b, nx.lt * kTile, nx.g, a.H);
-    };
-    // ---- tensor-core stages, each issued by thread 0 ----
-    auto issue_t = [&]() {   // T = dO S^T (S_hi, S_lo): A = dO (K-major over c), B = S image [c][f] (rows = K)
-        constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kD, 0, 1);
-#pragma unroll
-        for (int pass = 0; pass < 2; ++pass) {
-            const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
-#pragma unroll
-            for (int k = 0; k < kD / 16; ++k)
-                mma_bf16_ss(t_work, desc_at(kmajor, kstep_kmajor(sb0 + L::kG, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_t,
-                            (pass | k) != 0);
-        }
-        mma_commit(c.bar(BW_MMA2));
-    };
-    // dz += phi^T dden = (phi / den)^T (dden den) of the tile whose phi / den is in the staging tile, on the CUDA cores:
-    // thread = (16-byte chunk of 8 features, group of 8 tokens)
-    auto dz_tile = [&]() {
-        const int fc = tid & 15, t0 = (tid >> 4) * 8;
-        const uint8_t* blk = c.smem + L::kP + (fc >> 3) * kHalfTileBytes;
-#pragma unroll
-        for (int t = t0; t < t0 + 8; ++t) {
-            const uint4 pv = *reinterpret_cast<const uint4*>(blk + sw_chunk(t, fc & 7));
-            const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
-            const float dd = sdd[t];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                dz_acc[2 * q] = fmaf(dd, __uint_as_float(pw[q] << 16), dz_acc[2 * q]);
-                dz_acc[2 * q + 1] = fmaf(dd, __uint_as_float(pw[q] & 0xffff0000u), dz_acc[2 * q + 1]);
+    if (warp >= kBwdIssuer) {
+        setmaxnreg_dec<kBwdRegsIssuer>();
+        if (warp == kBwdIssuer) {
+            // =================== issuer: every copy, every tensor-core product, every store ===================
+            const bool one = lane == 0;
+            if (one) {
+                tma_prefetch_desc(&tmQ);
+                tma_prefetch_desc(&tmG);
+                tma_prefetch_desc(&tmDQ);
             }
-        }
-    };
-    // dq of tile (lt, g) leaves tensor memory through the staging tile (its last tensor-core stage has completed)
-    auto store_dq = [&](int lt, int g) {
-        {
-            float x[kM];
-            load64(t_work + lane_base + half * kM, x);
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, sb0 + L::kP + b * kHalfTileBytes, 64 * b, lt * kTile, g, a.H);
-            bulk_commit_group();
-        }
-    };
-
-    // Software pipeline over the tiles of a head: the next tile's Q is fetched into the other Q buffer while this tile is
-    // worked on, and its logits are issued AHEAD of this tile's last tensor-core stage (dS, dq, dW), so that the next
-    // tile's feature map runs on the CUDA cores while the tensor core finishes this tile; dq of this tile then leaves
-    // after the next tile's feature map.  The first tile of a head starts from scratch (S and W_q change there).
-    bool ok = true;
-    bool pre = false;              // this tile's logits were issued during the previous tile
-    bool pend_q = false, pend_g = false, pend_seg = false;   // copies requested and not yet waited for (what an unwinding CTA waits for)
-    int xb = 0, prev_lt = 0, prev_g = 0;
-    if (!w.done()) {
-        if (tid == 0) {
-            load_seg(w);
-            load_q(w, 0);
-            load_g(w);
-        }
-        pend_q = pend_g = pend_seg = true;
-    }
-    for (; !w.done(); w.next(), xb ^= 1) {
-        const bool first = w.first(), last = w.last();
-        TileWalk nx = w;
-        nx.next();
-        const bool ahead = !last && !nx.done();   // the next tile belongs to the same head
-        LB_TRACE(0);
-        if (first) {
-            if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];
-            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
-            pend_seg = false;
-        }
-        if (!pre) {
-            // ---- from scratch: U = Q W_q once Q is there, T = dO S^T once dO is there ----
-            if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) { ok = false; break; }
-            pend_q = false;
-            if (tid == 0) {
-                issue_logits_mma(t_u, xbuf(xb), sb0 + L::kW);
-                mma_commit(c.bar(BW_MMA));
-                if (ahead) load_q(nx, xb ^ 1);
+            auto xbuf = [&](int b) { return sb0 + (b ? L::kX1 : L::kX0); };
+            auto load_seg = [&](const TileWalk& t) {   // S (hi, lo) and W_q^T of the head
+                mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
+                    tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
+                    tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
+                }
+            };
+            auto load_q = [&](const TileWalk& t, int buf) {
+                mbar_arrive_expect_tx(c.bar(BW_X0 + buf), kTileBytes);
+                for (int b = 0; b < 2; ++b) act_load<kLayout>(xbuf(buf) + b * kHalfTileBytes, &tmQ, c.bar(BW_X0 + buf), 64 * b, t.lt * kTile, t.g, a.H);
+            };
+            auto load_g = [&](const TileWalk& t) {   // dO; the tile after it starts on its way into L2
+                mbar_arrive_expect_tx(c.bar(BW_IN2), kTileBytes);
+                for (int b = 0; b < 2; ++b) act_load<kLayout>(sb0 + L::kG + b * kHalfTileBytes, &tmG, c.bar(BW_IN2), 64 * b, t.lt * kTile, t.g, a.H);
+                TileWalk n2 = t;
+                n2.next();
+                if (!n2.done())
+                    for (int b = 0; b < 2; ++b) act_prefetch_l2<kLayout>(&tmG, 64 * b, n2.lt * kTile, n2.g, a.H);
+            };
+            auto issue_t = [&]() {   // T = dO S^T (S_hi, S_lo)
+                chain_images(t_t, sb0 + L::kG, sb0 + L::kShi, sb0 + L::kSlo);
+                mma_commit(c.bar(BW_TFULL));
+            };
+            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_staged = 0, ph_g = 0;
+            bool pend_x[2] = {false, false}, pend_in2 = false, pend_seg = false;   // copies requested and not yet waited for
+            bool ok = true, pre = false;
+            int xb = 0;
+            if (!w.done()) {
+                if (one) {
+                    load_seg(w);
+                    load_q(w, 0);
+                    load_g(w);
+                }
+                pend_seg = pend_x[0] = pend_in2 = true;
             }
-            pend_q = ahead;
-            if (!cta_wait(c, BW_LOAD2, ph_load2, kErrMmaLoad)) { ok = false; break; }
-            pend_g = false;
-            if (tid == 0) {
-                issue_t();
-                bulk_wait_group_read<0>();   // the previous tile's dq has left the staging tile, which is phi's home again
-            }
-        }
-        LB_TRACE(1);
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) { ok = false; break; }
-        LB_TRACE(2);
-        // ---- phi(q): p stays in registers (fp32, and its bf16 roundings); den = phi . z from the rounded values ----
-        float p[kM];
-        uint32_t pk[kM / 2];
-        load64(t_u + lane_base, p);
-        sa[half * kTile + row] = half == 0 ? softmax_half_packed<false>(p, pk, vec) : softmax_half_packed<true>(p, pk, vec + kM);
-        LB_TRACE(3);
-        if (pre) {
-            // ---- the previous tile's last stage has had the time of a feature map: its dO and (two tiles back) Q buffers
-            // are free for the copies of this tile's dO and the next tile's Q, and its dq leaves ----
-            if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
-            LB_TRACE(6);
-            if (tid == 0) {
-                load_g(w);
-                if (ahead) load_q(nx, xb ^ 1);
-            }
-            pend_g = true;
-            pend_q = ahead;
-            store_dq(prev_lt, prev_g);
-            LB_TRACE(7);
-            if (!cta_wait(c, BW_LOAD2, ph_load2, kErrMmaLoad)) { ok = false; break; }
-            LB_TRACE(12);
-            pend_g = false;
-            if (tid == 0) {
-                issue_t();
-                bulk_wait_group_read<0>();   // dq has left the staging tile
-            }
-        }
-        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrEpilogue)) { ok = false; break; }   // T is there (and every thread's den part is visible)
-        LB_TRACE(4);
-        // ---- dO . o = (dO S^T) . phi / den: the numerator phi S itself is never formed.  The per-token factor 1 / den of
-        // dnum = dO / den is kept OUT of the tensor-core operands: dphi = (dO S^T - (dO . o) z) / den is scaled here, in
-        // the accumulator's epilogue, and dS = (phi / den)^T dO takes it into phi, so the dO tile itself, exact in bf16,
-        // is the operand of both products ----
-        float x[kM];
-        load64(t_work + lane_base + half * kM, x);
-        const float inv1 = 1.f / (sa[row] + sa[kTile + row]);
-        const float inv = inv1 * a.lin_scale;   // every gradient below is linear in the incoming one: its factor rides on 1 / den
-        {
-            f32x2 gs2 = pack2(0.f, 0.f);
-#pragma unroll
-            for (int j = 0; j < kM; j += 2)
-                gs2 = fma2(pack2(__uint_as_float(pk[j >> 1] << 16), __uint_as_float(pk[j >> 1] & 0xffff0000u)), pack2(x[j], x[j + 1]), gs2);
-            float g0s, g1s;
-            unpack2(gs2, g0s, g1s);
-            sb[half * kTile + row] = (g0s + g1s) * inv1;   // this half's part of dO . o
-            if (kMixB) {
-                // Eq. 8: dout . a over this thread's 64 columns (dout from its tile, a straight from memory: one
-                // 128-byte line per thread, started towards L2 a tile ago), minus this half's part of dout . o
-                dr_acc -= (g0s + g1s) * inv1;
-                const int token = w.lt * kTile + row;
-                if (token < a.n) {
-                    const __nv_bfloat16* ap = a.mix_a + (size_t)(w.g / a.H) * a.str_batch + (size_t)(w.g % a.H) * a.str_head +
-                                              (size_t)token * a.str_token + half * kM;
-                    const uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
-                    f32x2 da2 = pack2(0.f, 0.f);
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        const uint4 av = __ldg(reinterpret_cast<const uint4*>(ap) + ch);
-                        const uint4 gv = *reinterpret_cast<const uint4*>(gblk + sw_chunk(row, ch));
-                        const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            da2 = fma2(pack2(__uint_as_float(gw[q] << 16), __uint_as_float(gw[q] & 0xffff0000u)),
-                                       pack2(__uint_as_float(aw[q] << 16), __uint_as_float(aw[q] & 0xffff0000u)), da2);
+            for (; !w.done(); w.next(), xb ^= 1) {
+                const bool first = w.first(), last = w.last();
+                TileWalk nx = w;
+                nx.next();
+                TileWalk nn = nx;
+                nn.next();
+                const bool ahead = !last && !nx.done();               // the next tile belongs to the same head
+                const bool ahead2 = ahead && !nx.last() && !nn.done();  // and so does the one after it
+                if (!pre) {
+                    // ---- the head's first tile: U = Q W_q once Q, W_q are there, T = dO S^T once dO, S are there ----
+                    if (first) {
+                        if (!issuer_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
+                        pend_seg = false;
                     }
-                    float d0, d1;
-                    unpack2(da2, d0, d1);
-                    dr_acc += d0 + d1;
+                    if (!issuer_wait(c, BW_X0 + xb, ph_x[xb], kErrMmaLoad)) { ok = false; break; }
+                    pend_x[xb] = false;
+                    if (one) {
+                        chain_logits(t_u, xbuf(xb), sb0 + L::kW);
+                        mma_commit(c.bar(BW_LFULL));
+                        if (ahead) load_q(nx, xb ^ 1);
+                    }
+                    pend_x[xb ^ 1] = ahead;
+                    if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
+                    pend_in2 = false;
+                    if (one) issue_t();
+                    __syncwarp();
                 }
-                if (!nx.done() && nx.lt * kTile + row < a.n)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.mix_a + (size_t)(nx.g / a.H) * a.str_batch + (size_t)(nx.g % a.H) * a.str_head +
-                                                                 (size_t)(nx.lt * kTile + row) * a.str_token + half * kM));
-            }
-            // phi / den (bf16) is the operand of dS and the factor of dz
-            float y[kM];
-            const f32x2 inv2 = pack2(inv, inv);
-#pragma unroll
-            for (int j = 0; j < kM; j += 2) unpack2(mul2(pack2(p[j], p[j + 1]), inv2), y[j], y[j + 1]);
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, y);
-        }
-        __syncthreads();
-        const float ngo = -(sb[row] + sb[kTile + row]);   // -(dO . o) = dden * den
-        LB_TRACE(5);
-        // ---- du (through the softmax of Eq. 6) ----
-#pragma unroll
-        for (int j = 0; j < kM; j += 2) {   // dphi = (dO S^T - (dO . o) z) / den
-            const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
-            unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
-        }
-        du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);   // (a CTA barrier inside: both halves of sb have been read)
-        if (half == 0) sdd[row] = ngo;
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        LB_TRACE(8);
-        // ---- the next tile's U = Q W_q first (it waits for nothing else), then dS += (phi / den)^T dO, dq = du W_q^T,
-        // dW_q += Q^T du ----
-        if (tid == 0) {
-            tcgen05_fence_after();
-            if (ahead) {
-                if (mbar_wait_abortable(c.bar(BW_LOAD), ph_load, c.wc.limit_ns(), c.wc.abort_smem)) {
-                    issue_logits_mma(t_u, xbuf(xb ^ 1), sb0 + L::kW);
-                    mma_commit(c.bar(BW_MMA));
-                } else {
-                    raise_abort(c.wc, kErrMmaLoad);   // the CTA leaves at its next wait
+                // ---- phi / den and du of this tile are written: the next tile's logits first (the feature map waits for
+                // nothing else), then dS += (phi / den)^T dO, dq = du W_q^T, dW_q += Q^T du ----
+                if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
+                if (ahead) {
+                    if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
+                    pend_x[xb ^ 1] = false;
                 }
+                if (one) {
+                    if (ahead) {
+                        chain_logits(t_u, xbuf(xb ^ 1), sb0 + L::kW);
+                        mma_commit(c.bar(BW_LFULL));
+                    }
+                    chain_ds(t_ds, sb0 + L::kP, sb0 + L::kG, first);
+                    chain_dx_dw(t_dq, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
+                    mma_commit(c.bar(BW_GFULL));
+                }
+                __syncwarp();
+                // ---- that stage done: dO's tile, this tile's Q buffer (and, at the end of a head, S and W_q) are free ----
+                if (!issuer_wait(c, BW_GFULL, ph_g, kErrMmaAcc)) { ok = false; break; }
+                if (ahead) {
+                    if (one) {
+                        load_g(nx);
+                        if (ahead2) load_q(nn, xb);
+                    }
+                    pend_in2 = true;
+                    pend_x[xb] = ahead2;
+                    if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
+                    pend_in2 = false;
+                    if (one) issue_t();   // the element-wise warps took this tile's T out of tensor memory before they announced its operands
+                    __syncwarp();
+                } else if (!nx.done()) {
+                    if (one) {
+                        load_seg(nx);
+                        load_q(nx, xb ^ 1);
+                        load_g(nx);
+                    }
+                    pend_seg = pend_x[xb ^ 1] = pend_in2 = true;
+                }
+                // ---- dq of this tile has been staged: store it; the staging tile is phi's home again once the store has read it ----
+                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
+                if (one) {
+                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                    bulk_commit_group();
+                    bulk_wait_group_read<0>();
+                    mbar_arrive(c.bar(BW_PFREE));
+                }
+                __syncwarp();
+                pre = ahead;
             }
-            constexpr uint32_t idesc_ds = make_idesc_bf16(kD, kD, 1, 1);        // A = (phi / den)^T, B = dO, both read MN-major
+            if (!ok) {
+                // unwinding: let the copies already requested land before the CTA gives its shared memory back
+                if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
+                for (int b = 0; b < 2; ++b)
+                    if (pend_x[b]) mbar_wait(c.bar(BW_X0 + b), ph_x[b], c.wc.limit_ns());
+                if (pend_in2) mbar_wait(c.bar(BW_IN2), ph_in2, c.wc.limit_ns());
+            }
+            if (one) bulk_wait_group<0>();
+        }
+    } else {
+        setmaxnreg_inc<kBwdRegsCompute>();
+        // =================== element-wise warps ===================
+        const int half = warp >> 2, row = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        float* vec = c.misc + BwdMisc::kVec / 4;
+        float* sa = c.misc + BwdMisc::kA / 4;
+        float* sb = c.misc + BwdMisc::kB / 4;
+        float* sdd = sb;   // dden den of the tile's tokens takes the place of the first half of sb once both halves have been read
+        uint32_t ph_l = 0, ph_t = 0, ph_g = 0, ph_p = 0;
+        float dr_acc = 0.f;   // Eq. 8: this thread's share of sum dout . (a - o)
+        float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
 #pragma unroll
-            for (int k = 0; k < kTile / 16; ++k)
-                mma_bf16_ss(t_ds, desc_at(mn_tile, sb0 + L::kP + k * 2048), desc_at(mn_tile, sb0 + L::kG + k * 2048), idesc_ds,
-                            (first && k == 0) ? 0u : 1u);
-            issue_dx_dw(t_work, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
-            mma_commit(c.bar(BW_G));
-        }
-        if (ahead) {
-            ph_load ^= 1u;   // thread 0 has waited for that phase on everybody's behalf
-            pend_q = false;
-        }
-        LB_TRACE(13);
-        dz_tile();   // while the tensor core works
-        LB_TRACE(14);
-        pre = ahead;
-        prev_lt = w.lt;
-        prev_g = w.g;
-        if (ahead) continue;
-
-        // ---- the last tile of the head (or of the run): finished here, nothing of the next tile in flight ----
-        if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
-        LB_TRACE(9);
-        if (tid == 0 && !nx.done()) {
-            // S, W_q and every tile buffer are free: the next head's copies overlap this tile's stores
-            load_seg(nx);
-            load_q(nx, xb ^ 1);
-            load_g(nx);
-        }
-        if (!nx.done()) pend_q = pend_g = pend_seg = true;
-        store_dq(w.lt, w.g);
-        LB_TRACE(10);
-        // ---- end of this CTA's part of the head: the accumulators go to the (CTA, head) records ----
-        {
-            tcgen05_fence_after();
-            float* rec = a.part_state + (size_t)(blockIdx.x + w.g) * kE;
+        for (int e = 0; e < 8; ++e) dz_acc[e] = 0.f;
+        // dq of a tile leaves tensor memory for the staging tile (the tile's last tensor-core stage has completed)
+        auto stage_dq = [&]() {
+            float x[kM];
+            load64(t_dq + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
+            warp_announce(c, BW_STAGED);
+        };
+        bool pre = false;   // the previous tile belongs to the same head: its dq is still in tensor memory
+        for (; !w.done(); w.next()) {
+            const bool first = w.first(), last = w.last();
+            TileWalk nx = w;
+            nx.next();
+            LB_TRACE(0);
+            if (first && tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // z (read after the next barrier)
+            bool okl = wait_only(c, BW_LFULL, ph_l, kErrSoftmaxU);   // verdict of this warp's waits since the last barrier with a verdict
+            LB_TRACE(2);
+            if (first && !cbar_and(okl)) break;
+            // ---- phi(q): p stays in registers (fp32, and its bf16 roundings); den = phi . z from the rounded values ----
+            float p[kM];
+            uint32_t pk[kM / 2];
+            load64(t_u + lane_base, p);
+            sa[half * kTile + row] = half == 0 ? softmax_half_packed<false>(p, pk, vec) : softmax_half_packed<true>(p, pk, vec + kM);
+            LB_TRACE(3);
+            if (pre) {
+                // ---- the previous tile's last stage has had the time of a feature map: its dq leaves ----
+                if (!compute_wait(c, BW_GFULL, ph_g, kErrStore, okl)) break;
+                LB_TRACE(6);
+                stage_dq();
+                LB_TRACE(7);
+            }
+            if (!compute_wait(c, BW_TFULL, ph_t, kErrEpilogue, okl)) break;   // T is there (and every thread's den part is visible)
+            LB_TRACE(4);
+            // ---- dO . o = (dO S^T) . phi / den: the numerator phi S itself is never formed.  The per-token factor 1 / den of
+            // dnum = dO / den is kept OUT of the tensor-core operands: dphi = (dO S^T - (dO . o) z) / den is scaled here, in
+            // the accumulator's epilogue, and dS = (phi / den)^T dO takes it into phi, so the dO tile itself, exact in bf16,
+            // is the operand of both products ----
+            float x[kM];
+            load64(t_t + lane_base + half * kM, x);
+            const float inv1 = 1.f / (sa[row] + sa[kTile + row]);
+            const float inv = inv1 * a.lin_scale;   // every gradient below is linear in the incoming one: its factor rides on 1 / den
             {
-                float x[kM];
-                load64(t_ds + lane_base + half * kM, x);   // lane = feature f, columns = c
+                f32x2 gs2 = pack2(0.f, 0.f);
 #pragma unroll
-                for (int j = 0; j < kM; ++j) rec[(size_t)(half * kM + j) * kD + row] = x[j];
-            }
-            drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
-            // dz: the 16 token groups' sums, in group order (the du tile has been consumed)
-            float* red = reinterpret_cast<float*>(c.smem + L::kRed);
+                for (int j = 0; j < kM; j += 2)
+                    gs2 = fma2(pack2(__uint_as_float(pk[j >> 1] << 16), __uint_as_float(pk[j >> 1] & 0xffff0000u)), pack2(x[j], x[j + 1]), gs2);
+                float g0s, g1s;
+                unpack2(gs2, g0s, g1s);
+                sb[half * kTile + row] = (g0s + g1s) * inv1;   // this half's part of dO . o
+                if (kMixB) {
+                    // Eq. 8: dout . a over this thread's 64 columns (dout from its tile, a straight from memory: one
+                    // 128-byte line per thread, started towards L2 a tile ago), minus this half's part of dout . o
+                    dr_acc -= (g0s + g1s) * inv1;
+                    const int token = w.lt * kTile + row;
+                    if (token < a.n) {
+                        const __nv_bfloat16* ap = a.mix_a + (size_t)(w.g / a.H) * a.str_batch + (size_t)(w.g % a.H) * a.str_head +
+                                                  (size_t)token * a.str_token + half * kM;
+                        const uint8_t* gblk = c.smem + L::kG + half * kHalfTileBytes;
+                        f32x2 da2 = pack2(0.f, 0.f);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                red[(tid >> 4) * kD + (tid & 15) * 8 + e] = dz_acc[e];
-                dz_acc[e] = 0.f;
-            }
-            __syncthreads();
-            if (tid < kD) {
-                float acc = 0.f;
+                        for (int ch = 0; ch < 8; ++ch) {
+                            const uint4 av = __ldg(reinterpret_cast<const uint4*>(ap) + ch);
+                            const uint4 gv = *reinterpret_cast<const uint4*>(gblk + sw_chunk(row, ch));
+                            const uint32_t aw[4] = {av.x, av.y, av.z, av.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
 #pragma unroll
-                for (int gidx = 0; gidx < 16; ++gidx) acc += red[gidx * kD + tid];
-                rec[kD * kD + tid] = acc;
+                            for (int q = 0; q < 4; ++q)
+                                da2 = fma2(pack2(__uint_as_float(gw[q] << 16), __uint_as_float(gw[q] & 0xffff0000u)),
+                                           pack2(__uint_as_float(aw[q] << 16), __uint_as_float(aw[q] & 0xffff0000u)), da2);
+                        }
+                        float d0, d1;
+                        unpack2(da2, d0, d1);
+                        dr_acc += d0 + d1;
+                    }
+                    if (!nx.done() && nx.lt * kTile + row < a.n)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(a.mix_a + (size_t)(nx.g / a.H) * a.str_batch + (size_t)(nx.g % a.H) * a.str_head +
+                                                                     (size_t)(nx.lt * kTile + row) * a.str_token + half * kM));
+                }
+                // phi / den (bf16) is the operand of dS and the factor of dz; its tile is free once the previous dq's store has read it
+                float y[kM];
+                const f32x2 inv2 = pack2(inv, inv);
+#pragma unroll
+                for (int j = 0; j < kM; j += 2) unpack2(mul2(pack2(p[j], p[j + 1]), inv2), y[j], y[j + 1]);
+                okl = w.i == 0 || wait_only(c, BW_PFREE, ph_p, kErrEpilogue);
+                store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, y);
             }
+            if (!cbar_and(okl)) break;
+            const float ngo = -(sb[row] + sb[kTile + row]);   // -(dO . o) = dden * den
+            LB_TRACE(5);
+            // ---- du (through the softmax of Eq. 6) ----
+#pragma unroll
+            for (int j = 0; j < kM; j += 2) {   // dphi = (dO S^T - (dO . o) z) / den
+                const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
+                unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
+            }
+            du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);   // (a barrier inside: both halves of sb have been read)
+            if (half == 0) sdd[row] = ngo;
+            warp_announce(c, BW_OPS);
+            cbar();
+            LB_TRACE(8);
+            {
+                // dz += phi^T dden = (phi / den)^T (dden den) on the CUDA cores: thread = (16-byte chunk of 8 features,
+                // group of 8 tokens)
+                const int fc = tid & 15, t0 = (tid >> 4) * 8;
+                const uint8_t* blk = c.smem + L::kP + (fc >> 3) * kHalfTileBytes;
+#pragma unroll
+                for (int t = t0; t < t0 + 8; ++t) {
+                    const uint4 pv = *reinterpret_cast<const uint4*>(blk + sw_chunk(t, fc & 7));
+                    const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
+                    const float dd = sdd[t];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        dz_acc[2 * q] = fmaf(dd, __uint_as_float(pw[q] << 16), dz_acc[2 * q]);
+                        dz_acc[2 * q + 1] = fmaf(dd, __uint_as_float(pw[q] & 0xffff0000u), dz_acc[2 * q + 1]);
+                    }
+                }
+            }
+            LB_TRACE(9);
+            pre = !last && !nx.done();
+            if (pre) continue;
+
+            // ---- the last tile of the head (or of the run): finished here; the accumulators go to the (CTA, head) records ----
+            if (!compute_wait(c, BW_GFULL, ph_g, kErrStore)) break;
+            stage_dq();
+            {
+                float* rec = a.part_state + (size_t)(blockIdx.x + w.g) * kE;
+                {
+                    float x[kM];
+                    load64(t_ds + lane_base + half * kM, x);   // lane = feature f, columns = c
+#pragma unroll
+                    for (int j = 0; j < kM; ++j) rec[(size_t)(half * kM + j) * kD + row] = x[j];
+                }
+                drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
+                // dz: the 16 token groups' sums, in group order (the du tile has been consumed)
+                float* red = reinterpret_cast<float*>(c.smem + L::kRed);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    red[(tid >> 4) * kD + (tid & 15) * 8 + e] = dz_acc[e];
+                    dz_acc[e] = 0.f;
+                }
+                cbar();
+                if (tid < kD) {
+                    float acc = 0.f;
+#pragma unroll
+                    for (int gidx = 0; gidx < 16; ++gidx) acc += red[gidx * kD + tid];
+                    rec[kD * kD + tid] = acc;
+                }
+            }
+            tcgen05_fence_before();
+            cbar();
+            LB_TRACE(11);
         }
-        tcgen05_fence_before();
-        __syncthreads();
-        LB_TRACE(11);
-    }
-    if (!ok && tid == 0) {
-        // unwinding: let the copies already requested land before the CTA gives its shared memory back
-        if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
-        if (pend_q) mbar_wait(c.bar(BW_LOAD), ph_load, c.wc.limit_ns());
-        if (pend_g) mbar_wait(c.bar(BW_LOAD2), ph_load2, c.wc.limit_ns());
-    }
-    if (kMixB) {
-        // the CTA's sum of dout . (a - o), thread by thread in index order (bit-reproducible)
-        float* red = reinterpret_cast<float*>(c.smem + L::kRed);
-        __syncthreads();
-        red[tid] = dr_acc;
-        __syncthreads();
-        if (tid == 0) {
-            float acc = 0.f;
-            for (int i = 0; i < kBwdThreads; ++i) acc += red[i];
-            a.part_dr[blockIdx.x] = acc;
+        if (kMixB) {
+            // the CTA's sum of dout . (a - o), thread by thread in index order (bit-reproducible)
+            float* red = reinterpret_cast<float*>(c.smem + L::kRed);
+            cbar();
+            red[tid] = dr_acc;
+            cbar();
+            if (tid == 0) {
+                float acc = 0.f;
+                for (int i = 0; i < kBwdCompute; ++i) acc += red[i];
+                a.part_dr[blockIdx.x] = acc;
+            }
         }
     }
     bwd_teardown(c);
@@ -654,221 +730,219 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (!bwd_smem_fits(bwd_smem, kBwdSmemK, a.err)) return;
     const BwdCta c = bwd_setup(bwd_smem, L::kMisc, a.err);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int half = warp >> 2, row = (warp & 3) * 32 + lane;
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    // tensor memory: logits | T = V dS^T | dv | dW_k | dk
+    // tensor memory: logits (later the du exchange) | T = V dS^T | dv | dW_k | dk
     const uint32_t t_u = c.tmem, t_t = c.tmem + 64, t_dv = c.tmem + 192, t_dw = c.tmem + 320, t_dk = c.tmem + 384;
-    float* vec = c.misc + BwdMisc::kVec / 4;
     const uint32_t sb0 = c.sbase;
-    const uint64_t kmajor = make_desc_sw128(0, 16, 1024);
-    const uint64_t mn_tile = make_desc_sw128(0, kHalfTileBytes, 1024);
-    uint32_t ph_load = 0, ph_load2 = 0, ph_seg = 0, ph_mma = 0, ph_mma2 = 0, ph_g = 0;
     TileWalk w;
     w.init(a.total_tiles, a.tiles_per_head);
-    if (tid == 0) {
-        tma_prefetch_desc(&tmK);
-        tma_prefetch_desc(&tmV);
-        tma_prefetch_desc(&tmDK);
-        tma_prefetch_desc(&tmDV);
-    }
 
-    // ---- copies, each issued by thread 0 ----
-    auto xbuf = [&](int b) { return sb0 + (b ? L::kX1 : L::kX0); };
-    auto load_seg = [&](const TileWalk& t) {   // dS (hi, lo) and W_k^T of the head
-        mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
-        for (int b = 0; b < 2; ++b) {
-            tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
-            tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
-            tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
-        }
-    };
-    auto load_k = [&](const TileWalk& t, int buf) {
-        mbar_arrive_expect_tx(c.bar(BW_LOAD), kTileBytes);
-        for (int b = 0; b < 2; ++b) act_load<kLayout>(xbuf(buf) + b * kHalfTileBytes, &tmK, c.bar(BW_LOAD), 64 * b, t.lt * kTile, t.g, a.H);
-    };
-    auto load_v = [&](const TileWalk& t) {   // V; the tile after it starts on its way into L2
-        mbar_arrive_expect_tx(c.bar(BW_LOAD2), kTileBytes);
-        for (int b = 0; b < 2; ++b) act_load<kLayout>(sb0 + L::kV + b * kHalfTileBytes, &tmV, c.bar(BW_LOAD2), 64 * b, t.lt * kTile, t.g, a.H);
-        TileWalk nx = t;
-        nx.next();
-        if (!nx.done())
-            for (int b = 0; b < 2; ++b) act_prefetch_l2<kLayout>(&tmV, 64 * b, nx.lt * kTile, nx.g, a.H);
-    };
-    // ---- T = V dS^T (hi and lo parts of dS): A = V (K-major over c), B = dS image [c][f] (rows = K); issued by thread 0 ----
-    auto issue_t = [&]() {
-        constexpr uint32_t idesc_dphi = make_idesc_bf16(kTile, kD, 0, 1);
-#pragma unroll
-        for (int pass = 0; pass < 2; ++pass) {
-            const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
-#pragma unroll
-            for (int k = 0; k < kD / 16; ++k)
-                mma_bf16_ss(t_t, desc_at(kmajor, kstep_kmajor(sb0 + L::kV, k, kHalfTileBytes)), desc_at(mn_tile, st + k * 2048), idesc_dphi,
-                            (pass | k) != 0);
-        }
-        mma_commit(c.bar(BW_MMA2));
-    };
-    // dv and dk of tile (lt, g) leave tensor memory (the tile's last tensor-core stage has completed): dv through phi's
-    // tile, dk through V's (this tile's V dS^T has been formed; thread 0 asks for the next V only once the store has read it)
-    auto store_dv_dk = [&](int lt, int g) {
-        {
-            float x[kM];
-            load64(t_dv + lane_base + half * kM, x);
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
-        }
-        {
-            float x[kM];
-            load64(t_dk + lane_base + half * kM, x);
-            store_row_bf16(c.smem + L::kV + half * kHalfTileBytes, row, x);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, lt * kTile, g, a.H);
-            for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, sb0 + L::kV + b * kHalfTileBytes, 64 * b, lt * kTile, g, a.H);
-            bulk_commit_group();
-        }
-    };
-
-    // Software pipeline over the tiles of a head, as on the query side: the next tile's K is fetched into the other K
-    // buffer, its V into V's tile once dk has left it, and its logits and V dS^T are issued around this tile's last
-    // tensor-core stage (dv, dk, dW), so that the next tile's feature map runs while the tensor core finishes this tile.
-    bool ok = true;
-    bool pre = false;              // this tile's logits and V dS^T were issued during the previous tile
-    bool pend_k = false, pend_v = false, pend_seg = false;   // copies requested and not yet waited for
-    int xb = 0, prev_lt = 0, prev_g = 0;
-    if (!w.done()) {
-        if (tid == 0) {
-            load_seg(w);
-            load_k(w, 0);
-            load_v(w);
-        }
-        pend_k = pend_v = pend_seg = true;
-    }
-    for (; !w.done(); w.next(), xb ^= 1) {
-        const bool first = w.first(), last = w.last();
-        TileWalk nx = w;
-        nx.next();
-        const bool ahead = !last && !nx.done();   // the next tile belongs to the same head
-        if (first) {
-            if (tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // dz
-            if (!cta_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
-            pend_seg = false;
-        }
-        if (!pre) {
-            // ---- from scratch: U = K W_k once K is there, T = V dS^T once V is there ----
-            if (!cta_wait(c, BW_LOAD, ph_load, kErrMmaLoad)) { ok = false; break; }
-            pend_k = false;
-            if (tid == 0) {
-                issue_logits_mma(t_u, xbuf(xb), sb0 + L::kW);
-                mma_commit(c.bar(BW_MMA));
-                if (ahead) load_k(nx, xb ^ 1);
+    if (warp >= kBwdIssuer) {
+        setmaxnreg_dec<kBwdRegsIssuer>();
+        if (warp == kBwdIssuer) {
+            // =================== issuer ===================
+            const bool one = lane == 0;
+            if (one) {
+                tma_prefetch_desc(&tmK);
+                tma_prefetch_desc(&tmV);
+                tma_prefetch_desc(&tmDK);
+                tma_prefetch_desc(&tmDV);
             }
-            pend_k = ahead;
-            if (!cta_wait(c, BW_LOAD2, ph_load2, kErrMmaLoad)) { ok = false; break; }
-            pend_v = false;
-            if (tid == 0) issue_t();
-        }
-        if (!cta_wait(c, BW_MMA, ph_mma, kErrSoftmaxU)) { ok = false; break; }
-        // ---- phi(k): p stays in registers (fp32, and its bf16 roundings, which go to phi's tile once that is free) ----
-        float p[kM];
-        uint32_t pk[kM / 2];
-        load64(t_u + lane_base, p);
-        if (half == 0) softmax_half_packed<false>(p, pk, vec);
-        else softmax_half_packed<true>(p, pk, vec + kM);
-        if (!cta_wait(c, BW_MMA2, ph_mma2, kErrMmaAcc)) { ok = false; break; }   // T is there: V's tile is free
-        if (pre) {
-            // ---- the previous tile's last stage has had the time of a feature map: its dv and dk leave, and the K buffer
-            // two tiles back takes the next tile's K ----
-            if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
-            if (tid == 0 && ahead) load_k(nx, xb ^ 1);
-            pend_k = ahead;
-            store_dv_dk(prev_lt, prev_g);
-        }
-        // ---- dphi = V dS^T + dz -> du ----
-        {
-            float x[kM];
-            load64(t_t + lane_base + half * kM, x);
-#pragma unroll
-            for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
-            if (tid == 0) {
-                bulk_wait_group_read<0>();   // the stores have read phi's and V's tiles
-                if (ahead) load_v(nx);
-            }
-            du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);   // (a CTA barrier inside: phi's tile is free for everybody)
-        }
-        pend_v = ahead;
-        {
-            uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch)
-                *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-        }
-        fence_proxy_async_smem();
-        tcgen05_fence_before();
-        __syncthreads();
-        // ---- the next tile's U = K W_k first, then dv = phi dS (hi and lo parts), dk = du W_k^T, dW_k += K^T du, then the
-        // next tile's V dS^T ----
-        if (tid == 0) {
-            tcgen05_fence_after();
-            if (ahead) {
-                if (mbar_wait_abortable(c.bar(BW_LOAD), ph_load, c.wc.limit_ns(), c.wc.abort_smem)) {
-                    issue_logits_mma(t_u, xbuf(xb ^ 1), sb0 + L::kW);
-                    mma_commit(c.bar(BW_MMA));
-                } else {
-                    raise_abort(c.wc, kErrMmaLoad);   // the CTA leaves at its next wait
+            auto xbuf = [&](int b) { return sb0 + (b ? L::kX1 : L::kX0); };
+            auto load_seg = [&](const TileWalk& t) {   // dS (hi, lo) and W_k^T of the head
+                mbar_arrive_expect_tx(c.bar(BW_SEG), 2 * kTileBytes + kWBytes);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_3d(sb0 + L::kShi + b * kHalfTileBytes, &tmShi, c.bar(BW_SEG), 64 * b, 0, t.g);
+                    tma_load_3d(sb0 + L::kSlo + b * kHalfTileBytes, &tmSlo, c.bar(BW_SEG), 64 * b, 0, t.g);
+                    tma_load_3d(sb0 + L::kW + b * (kWBytes / 2), &tmW, c.bar(BW_SEG), 64 * b, 0, t.g % a.H);
                 }
+            };
+            auto load_k = [&](const TileWalk& t, int buf) {
+                mbar_arrive_expect_tx(c.bar(BW_X0 + buf), kTileBytes);
+                for (int b = 0; b < 2; ++b) act_load<kLayout>(xbuf(buf) + b * kHalfTileBytes, &tmK, c.bar(BW_X0 + buf), 64 * b, t.lt * kTile, t.g, a.H);
+                TileWalk n2 = t;
+                n2.next();
+                if (!n2.done())
+                    for (int b = 0; b < 2; ++b) act_prefetch_l2<kLayout>(&tmK, 64 * b, n2.lt * kTile, n2.g, a.H);
+            };
+            auto load_v = [&](const TileWalk& t) {
+                mbar_arrive_expect_tx(c.bar(BW_IN2), kTileBytes);
+                for (int b = 0; b < 2; ++b) act_load<kLayout>(sb0 + L::kV + b * kHalfTileBytes, &tmV, c.bar(BW_IN2), 64 * b, t.lt * kTile, t.g, a.H);
+                TileWalk n2 = t;
+                n2.next();
+                if (!n2.done())
+                    for (int b = 0; b < 2; ++b) act_prefetch_l2<kLayout>(&tmV, 64 * b, n2.lt * kTile, n2.g, a.H);
+            };
+            auto issue_t = [&]() {   // T = V dS^T (hi and lo parts of dS)
+                chain_images(t_t, sb0 + L::kV, sb0 + L::kShi, sb0 + L::kSlo);
+                mma_commit(c.bar(BW_TFULL));
+            };
+            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_staged = 0, ph_t = 0;
+            bool pend_x[2] = {false, false}, pend_in2 = false, pend_seg = false;
+            bool ok = true, pre = false;
+            int xb = 0;
+            if (!w.done()) {
+                if (one) {
+                    load_seg(w);
+                    load_k(w, 0);
+                    load_v(w);
+                }
+                pend_seg = pend_x[0] = pend_in2 = true;
             }
-            constexpr uint32_t idesc_dv = make_idesc_bf16(kTile, kD, 0, 0);     // A = phi (K-major over f), B = dS image [c][f] (rows = N)
+            for (; !w.done(); w.next(), xb ^= 1) {
+                const bool first = w.first(), last = w.last();
+                TileWalk nx = w;
+                nx.next();
+                TileWalk nn = nx;
+                nn.next();
+                const bool ahead = !last && !nx.done();
+                const bool ahead2 = ahead && !nx.last() && !nn.done();
+                if (!pre) {
+                    // ---- the head's first tile: U = K W_k once K, W_k are there, T = V dS^T once V, dS are there; V's tile then
+                    // takes the next tile's V ----
+                    if (first) {
+                        if (!issuer_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
+                        pend_seg = false;
+                    }
+                    if (!issuer_wait(c, BW_X0 + xb, ph_x[xb], kErrMmaLoad)) { ok = false; break; }
+                    pend_x[xb] = false;
+                    if (one) {
+                        chain_logits(t_u, xbuf(xb), sb0 + L::kW);
+                        mma_commit(c.bar(BW_LFULL));
+                        if (ahead) load_k(nx, xb ^ 1);
+                    }
+                    pend_x[xb ^ 1] = ahead;
+                    if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
+                    pend_in2 = false;
+                    if (one) issue_t();
+                    __syncwarp();
+                    if (!issuer_wait(c, BW_TFULL, ph_t, kErrMmaAcc)) { ok = false; break; }
+                    if (ahead && one) load_v(nx);
+                    pend_in2 = ahead;
+                }
+                // ---- phi and du of this tile are written: the next tile's logits first, then dv = phi dS (hi and lo parts),
+                // dk = du W_k^T, dW_k += K^T du, then the next tile's V dS^T ----
+                if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
+                if (ahead) {
+                    if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
+                    pend_x[xb ^ 1] = false;
+                    if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
+                    pend_in2 = false;
+                }
+                if (one) {
+                    if (ahead) {
+                        chain_logits(t_u, xbuf(xb ^ 1), sb0 + L::kW);
+                        mma_commit(c.bar(BW_LFULL));
+                    }
+                    chain_dv(t_dv, sb0 + L::kP, sb0 + L::kShi, sb0 + L::kSlo);
+                    chain_dx_dw(t_dk, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
+                    mma_commit(c.bar(BW_GFULL));
+                    if (ahead) issue_t();   // the element-wise warps took this tile's T out of tensor memory before they announced its operands
+                }
+                __syncwarp();
+                if (ahead) {
+                    // V's tile is free once that product is done: the V of the tile after the next
+                    if (!issuer_wait(c, BW_TFULL, ph_t, kErrMmaAcc)) { ok = false; break; }
+                    if (ahead2 && one) load_v(nn);
+                    pend_in2 = ahead2;
+                }
+                // ---- dv (in phi's tile) and dk (in this tile's K buffer) have been staged: store them; the buffers are free
+                // once the stores have read them ----
+                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
+                if (one) {
+                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, xbuf(xb) + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                    bulk_commit_group();
+                    bulk_wait_group_read<0>();
+                    mbar_arrive(c.bar(BW_PFREE));
+                    if (ahead2) load_k(nn, xb);
+                    else if (!ahead && !nx.done()) {
+                        // the next head: the staged results were drained after this tile's last stage, so every buffer is free
+                        load_seg(nx);
+                        load_k(nx, xb ^ 1);
+                        load_v(nx);
+                    }
+                }
+                __syncwarp();
+                if (ahead2) pend_x[xb] = true;
+                else if (!ahead && !nx.done()) pend_seg = pend_x[xb ^ 1] = pend_in2 = true;
+                pre = ahead;
+            }
+            if (!ok) {
+                if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
+                for (int b = 0; b < 2; ++b)
+                    if (pend_x[b]) mbar_wait(c.bar(BW_X0 + b), ph_x[b], c.wc.limit_ns());
+                if (pend_in2) mbar_wait(c.bar(BW_IN2), ph_in2, c.wc.limit_ns());
+            }
+            if (one) bulk_wait_group<0>();
+        }
+    } else {
+        setmaxnreg_inc<kBwdRegsCompute>();
+        // =================== element-wise warps ===================
+        const int half = warp >> 2, row = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        float* vec = c.misc + BwdMisc::kVec / 4;
+        uint32_t ph_l = 0, ph_t = 0, ph_g = 0, ph_p = 0;
+        // dv and dk of a tile leave tensor memory (its last tensor-core stage has completed): dv to phi's tile, dk to the
+        // tile's own K buffer
+        auto stage_dv_dk = [&](int buf) {
+            {
+                float x[kM];
+                load64(t_dv + lane_base + half * kM, x);
+                store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
+            }
+            {
+                float x[kM];
+                load64(t_dk + lane_base + half * kM, x);
+                store_row_bf16(c.smem + (buf ? L::kX1 : L::kX0) + half * kHalfTileBytes, row, x);
+            }
+            warp_announce(c, BW_STAGED);
+        };
+        bool pre = false;
+        bool okl = true;   // verdict of this warp's waits since the last barrier with a verdict (a warp leaves only at such a barrier)
+        int xb = 0;
+        for (; !w.done(); w.next(), xb ^= 1) {
+            const bool first = w.first(), last = w.last();
+            TileWalk nx = w;
+            nx.next();
+            if (first && tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // dz (read after the next barrier)
+            okl = wait_only(c, BW_LFULL, ph_l, kErrSoftmaxU) && okl;
+            // ---- phi(k): p stays in registers (fp32, and its bf16 roundings, which go to phi's tile once that is free) ----
+            float p[kM];
+            uint32_t pk[kM / 2];
+            load64(t_u + lane_base, p);
+            if (half == 0) softmax_half_packed<false>(p, pk, vec);   // (the returned dot product is not needed here: vec may still be the old one)
+            else softmax_half_packed<true>(p, pk, vec + kM);
+            if (pre) {
+                // ---- the previous tile's last stage has had the time of a feature map: its dv and dk leave ----
+                if (!compute_wait(c, BW_GFULL, ph_g, kErrStore, okl)) break;
+                stage_dv_dk(xb ^ 1);
+            }
+            if (!compute_wait(c, BW_TFULL, ph_t, kErrMmaAcc, okl)) break;
+            // ---- dphi = V dS^T + dz -> du ----
+            {
+                float x[kM];
+                load64(t_t + lane_base + half * kM, x);
 #pragma unroll
-            for (int pass = 0; pass < 2; ++pass) {
-                const uint32_t st = sb0 + (pass == 0 ? L::kShi : L::kSlo);
+                for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
+                du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
+            }
+            if (w.i > 0) okl = wait_only(c, BW_PFREE, ph_p, kErrEpilogue) && okl;
+            {
+                uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
 #pragma unroll
-                for (int k = 0; k < kD / 16; ++k)
-                    mma_bf16_ss(t_dv, desc_at(kmajor, kstep_kmajor(sb0 + L::kP, k, kHalfTileBytes)), desc_at(kmajor, kstep_kmajor(st, k, kHalfTileBytes)),
-                                idesc_dv, (pass | k) != 0);
+                for (int ch = 0; ch < 8; ++ch)
+                    *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
             }
-            issue_dx_dw(t_dk, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
-            mma_commit(c.bar(BW_G));
-            if (ahead) {
-                if (mbar_wait_abortable(c.bar(BW_LOAD2), ph_load2, c.wc.limit_ns(), c.wc.abort_smem)) issue_t();
-                else raise_abort(c.wc, kErrMmaLoad);
-            }
+            warp_announce(c, BW_OPS);
+            pre = !last && !nx.done();
+            if (pre) continue;
+            // ---- the last tile of the head (or of the run): finished here ----
+            if (!compute_wait(c, BW_GFULL, ph_g, kErrStore, okl)) break;
+            stage_dv_dk(xb);
+            drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
+            tcgen05_fence_before();
+            cbar();
         }
-        if (ahead) {
-            ph_load ^= 1u;    // thread 0 has waited for these phases on everybody's behalf
-            ph_load2 ^= 1u;
-            pend_k = pend_v = false;
-        }
-        pre = ahead;
-        prev_lt = w.lt;
-        prev_g = w.g;
-        if (ahead) continue;
-
-        // ---- the last tile of the head (or of the run): finished here, nothing of the next tile in flight ----
-        if (!cta_wait(c, BW_G, ph_g, kErrStore)) { ok = false; break; }
-        if (tid == 0 && !nx.done()) {
-            // dS, W_k and the K buffers are free: the next head's copies overlap this tile's stores
-            load_seg(nx);
-            load_k(nx, xb ^ 1);
-        }
-        if (!nx.done()) pend_k = pend_seg = true;
-        store_dv_dk(w.lt, w.g);
-        if (tid == 0) {
-            bulk_wait_group_read<0>();
-            if (!nx.done()) load_v(nx);
-        }
-        if (!nx.done()) pend_v = true;
-        tcgen05_fence_after();
-        drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
-        tcgen05_fence_before();
-        __syncthreads();
-    }
-    if (!ok && tid == 0) {
-        // unwinding: let the copies already requested land before the CTA gives its shared memory back
-        if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
-        if (pend_k) mbar_wait(c.bar(BW_LOAD), ph_load, c.wc.limit_ns());
-        if (pend_v) mbar_wait(c.bar(BW_LOAD2), ph_load2, c.wc.limit_ns());
     }
     bwd_teardown(c);
 }
