@@ -102,8 +102,8 @@ struct BwdMisc {
     static constexpr uint32_t kVec = 0;           // 128 floats: z (query side) or dz (key side)
     static constexpr uint32_t kA = 512;           // 2 x 128 floats: den halves
     static constexpr uint32_t kB = 1536;          // 2 x 128 floats: (dO . o) halves; then, in the first 128, dden den of the tile
-    static constexpr uint32_t kBars = 2560;       // 10 mbarriers, TMEM slot, abort word
-    static constexpr uint32_t kBytes = 2560 + 96;
+    static constexpr uint32_t kBars = 2560;       // 12 mbarriers, TMEM slot, abort word
+    static constexpr uint32_t kBytes = 2560 + 112;
 };
 constexpr uint32_t kBwdSmemQ = BwdSmemQ::kMisc + BwdMisc::kBytes;
 constexpr uint32_t kBwdSmemK = BwdSmemK::kMisc + BwdMisc::kBytes;
@@ -111,10 +111,13 @@ static_assert(kBwdSmemQ <= 232448 && kBwdSmemK <= 232448, "a CTA has 227 KB of s
 
 // mbarriers.  Copies: BW_X0 / BW_X1 the two buffers of the tile that feeds the logits, BW_IN2 the other input tile,
 // BW_SEG the head's images and weights.  Issuer -> element-wise warps: BW_LFULL logits, BW_TFULL the product with the
-// images, BW_GFULL the tile's last tensor-core stage, BW_PFREE the staging tile has been read by its store.
-// Element-wise warps -> issuer (one arrival per warp): BW_OPS the operands of the last stage are written, BW_STAGED the
+// images, BW_G1 / BW_GFULL the first part / all of the tile's last tensor-core stage.  Element-wise warps -> issuer (one
+// arrival per warp): BW_OPS1 / BW_OPS the first / all operands of the last stage are written, BW_STAGED1 / BW_STAGED
 // results have been staged for their stores.
-enum : int { BW_X0 = 0, BW_X1 = 1, BW_IN2 = 2, BW_SEG = 3, BW_LFULL = 4, BW_TFULL = 5, BW_GFULL = 6, BW_PFREE = 7, BW_OPS = 8, BW_STAGED = 9, BW_NBARS = 10 };
+enum : int {
+    BW_X0 = 0, BW_X1 = 1, BW_IN2 = 2, BW_SEG = 3, BW_LFULL = 4, BW_TFULL = 5, BW_G1 = 6, BW_GFULL = 7,
+    BW_OPS1 = 8, BW_OPS = 9, BW_STAGED1 = 10, BW_STAGED = 11, BW_NBARS = 12
+};
 
 struct BwdCta {
     uint8_t* smem;
@@ -152,7 +155,7 @@ __device__ __forceinline__ BwdCta bwd_setup(uint8_t* smem_raw, uint32_t misc_off
     c.wc.abort_smem = smem_u32(abort_word);
     if (threadIdx.x == 0) {
         *abort_word = 0u;
-        for (int i = 0; i < BW_NBARS; ++i) mbar_init(c.bar(i), (i == BW_OPS || i == BW_STAGED) ? kBwdCompute / 32 : 1);
+        for (int i = 0; i < BW_NBARS; ++i) mbar_init(c.bar(i), i >= BW_OPS1 ? kBwdCompute / 32 : 1);
         fence_mbar_init();
     }
     if ((threadIdx.x >> 5) == 1) {
@@ -441,7 +444,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 chain_images(t_t, sb0 + L::kG, sb0 + L::kShi, sb0 + L::kSlo);
                 mma_commit(c.bar(BW_TFULL));
             };
-            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_staged = 0, ph_g = 0;
+            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops1 = 0, ph_ops = 0, ph_staged = 0, ph_g1 = 0;
             bool pend_x[2] = {false, false}, pend_in2 = false, pend_seg = false;   // copies requested and not yet waited for
             bool ok = true, pre = false;
             int xb = 0;
@@ -480,8 +483,22 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     if (one) issue_t();
                     __syncwarp();
                 }
-                // ---- phi / den and du of this tile are written: the next tile's logits first (the feature map waits for
-                // nothing else), then dS += (phi / den)^T dO, dq = du W_q^T, dW_q += Q^T du ----
+                // ---- phi / den of this tile is written: dS += (phi / den)^T dO at once, so that dO's tile is free for the
+                // next tile's dO while this tile's du is still being formed ----
+                if (!issuer_wait(c, BW_OPS1, ph_ops1, kErrMmaPhi)) { ok = false; break; }
+                if (one) {
+                    chain_ds(t_ds, sb0 + L::kP, sb0 + L::kG, first);
+                    mma_commit(c.bar(BW_G1));
+                }
+                __syncwarp();
+                if (!issuer_wait(c, BW_G1, ph_g1, kErrMmaAcc)) { ok = false; break; }
+                if (ahead) {
+                    if (one) load_g(nx);
+                    pend_in2 = true;
+                }
+                // ---- du is written: the next tile's logits first (its feature map waits for nothing else), then
+                // dq = du W_q^T, dW_q += Q^T du, then the next tile's T = dO S^T (the element-wise warps took this tile's T
+                // out of tensor memory before they announced phi / den) ----
                 if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
                 if (ahead) {
                     if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
@@ -492,41 +509,37 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                         chain_logits(t_u, xbuf(xb ^ 1), sb0 + L::kW);
                         mma_commit(c.bar(BW_LFULL));
                     }
-                    chain_ds(t_ds, sb0 + L::kP, sb0 + L::kG, first);
                     chain_dx_dw(t_dq, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
                     mma_commit(c.bar(BW_GFULL));
                 }
                 __syncwarp();
-                // ---- that stage done: dO's tile, this tile's Q buffer (and, at the end of a head, S and W_q) are free ----
-                if (!issuer_wait(c, BW_GFULL, ph_g, kErrMmaAcc)) { ok = false; break; }
                 if (ahead) {
-                    if (one) {
-                        load_g(nx);
-                        if (ahead2) load_q(nn, xb);
-                    }
-                    pend_in2 = true;
-                    pend_x[xb] = ahead2;
                     if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
                     pend_in2 = false;
-                    if (one) issue_t();   // the element-wise warps took this tile's T out of tensor memory before they announced its operands
+                    if (one) issue_t();
                     __syncwarp();
-                } else if (!nx.done()) {
-                    if (one) {
+                }
+                // ---- dq of this tile has been staged in the tile's own Q buffer (so its last stage is complete): store it;
+                // the buffer then takes the Q of the tile after the next, or, at the end of a head, everything is free
+                // for the next head's copies ----
+                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
+                if (one) {
+                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, xbuf(xb) + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                    bulk_commit_group();
+                    if (!ahead && !nx.done()) {
+                        bulk_wait_group_read<0>();   // (the store before this one read the other Q buffer)
                         load_seg(nx);
                         load_q(nx, xb ^ 1);
                         load_g(nx);
                     }
-                    pend_seg = pend_x[xb ^ 1] = pend_in2 = true;
-                }
-                // ---- dq of this tile has been staged: store it; the staging tile is phi's home again once the store has read it ----
-                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
-                if (one) {
-                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-                    bulk_commit_group();
-                    bulk_wait_group_read<0>();
-                    mbar_arrive(c.bar(BW_PFREE));
+                    if (ahead2) {
+                        bulk_wait_group_read<0>();
+                        load_q(nn, xb);
+                    }
                 }
                 __syncwarp();
+                if (!ahead && !nx.done()) pend_seg = pend_x[xb ^ 1] = pend_in2 = true;
+                if (ahead2) pend_x[xb] = true;
                 pre = ahead;
             }
             if (!ok) {
@@ -547,20 +560,21 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         float* sa = c.misc + BwdMisc::kA / 4;
         float* sb = c.misc + BwdMisc::kB / 4;
         float* sdd = sb;   // dden den of the tile's tokens takes the place of the first half of sb once both halves have been read
-        uint32_t ph_l = 0, ph_t = 0, ph_g = 0, ph_p = 0;
+        uint32_t ph_l = 0, ph_t = 0, ph_g = 0;
         float dr_acc = 0.f;   // Eq. 8: this thread's share of sum dout . (a - o)
         float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
 #pragma unroll
         for (int e = 0; e < 8; ++e) dz_acc[e] = 0.f;
-        // dq of a tile leaves tensor memory for the staging tile (the tile's last tensor-core stage has completed)
-        auto stage_dq = [&]() {
+        // dq of a tile leaves tensor memory for the tile's own Q buffer (the tile's last tensor-core stage has completed)
+        auto stage_dq = [&](int buf) {
             float x[kM];
             load64(t_dq + lane_base + half * kM, x);
-            store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
+            store_row_bf16(c.smem + (buf ? L::kX1 : L::kX0) + half * kHalfTileBytes, row, x);
             warp_announce(c, BW_STAGED);
         };
         bool pre = false;   // the previous tile belongs to the same head: its dq is still in tensor memory
-        for (; !w.done(); w.next()) {
+        int xb = 0;
+        for (; !w.done(); w.next(), xb ^= 1) {
             const bool first = w.first(), last = w.last();
             TileWalk nx = w;
             nx.next();
@@ -579,7 +593,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 // ---- the previous tile's last stage has had the time of a feature map: its dq leaves ----
                 if (!compute_wait(c, BW_GFULL, ph_g, kErrStore, okl)) break;
                 LB_TRACE(6);
-                stage_dq();
+                stage_dq(xb ^ 1);
                 LB_TRACE(7);
             }
             if (!compute_wait(c, BW_TFULL, ph_t, kErrEpilogue, okl)) break;   // T is there (and every thread's den part is visible)
@@ -628,15 +642,15 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(a.mix_a + (size_t)(nx.g / a.H) * a.str_batch + (size_t)(nx.g % a.H) * a.str_head +
                                                                      (size_t)(nx.lt * kTile + row) * a.str_token + half * kM));
                 }
-                // phi / den (bf16) is the operand of dS and the factor of dz; its tile is free once the previous dq's store has read it
+                // phi / den (bf16) is the operand of dS and the factor of dz (the previous tile's dS and dz are done with the tile)
                 float y[kM];
                 const f32x2 inv2 = pack2(inv, inv);
 #pragma unroll
                 for (int j = 0; j < kM; j += 2) unpack2(mul2(pack2(p[j], p[j + 1]), inv2), y[j], y[j + 1]);
-                okl = w.i == 0 || wait_only(c, BW_PFREE, ph_p, kErrEpilogue);
                 store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, y);
+                warp_announce(c, BW_OPS1);
             }
-            if (!cbar_and(okl)) break;
+            cbar();
             const float ngo = -(sb[row] + sb[kTile + row]);   // -(dO . o) = dden * den
             LB_TRACE(5);
             // ---- du (through the softmax of Eq. 6) ----
@@ -673,7 +687,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
             // ---- the last tile of the head (or of the run): finished here; the accumulators go to the (CTA, head) records ----
             if (!compute_wait(c, BW_GFULL, ph_g, kErrStore)) break;
-            stage_dq();
+            stage_dq(xb);
             {
                 float* rec = a.part_state + (size_t)(blockIdx.x + w.g) * kE;
                 {
@@ -776,7 +790,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 chain_images(t_t, sb0 + L::kV, sb0 + L::kShi, sb0 + L::kSlo);
                 mma_commit(c.bar(BW_TFULL));
             };
-            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_staged = 0, ph_t = 0;
+            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_staged1 = 0, ph_staged = 0, ph_t = 0;
             bool pend_x[2] = {false, false}, pend_in2 = false, pend_seg = false;
             bool ok = true, pre = false;
             int xb = 0;
@@ -815,55 +829,73 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                     pend_in2 = false;
                     if (one) issue_t();
                     __syncwarp();
-                    if (!issuer_wait(c, BW_TFULL, ph_t, kErrMmaAcc)) { ok = false; break; }
-                    if (ahead && one) load_v(nx);
-                    pend_in2 = ahead;
+                    if (ahead) {
+                        if (!issuer_wait(c, BW_TFULL, ph_t, kErrMmaAcc)) { ok = false; break; }
+                        if (one) load_v(nx);
+                        pend_in2 = true;
+                    } else {
+                        ph_t ^= 1u;   // (that phase is not waited for here)
+                    }
+                } else {
+                    ph_t ^= 1u;       // this tile's V dS^T was issued during the previous tile
                 }
-                // ---- phi and du of this tile are written: the next tile's logits first, then dv = phi dS (hi and lo parts),
-                // dk = du W_k^T, dW_k += K^T du, then the next tile's V dS^T ----
+                // ---- phi and du of this tile are written: the next tile's logits first, then dk = du W_k^T and
+                // dW_k += K^T du (the du tile and this tile's K buffer are free after them), the next tile's V dS^T, and
+                // dv = phi dS (hi and lo parts) last ----
                 if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
                 if (ahead) {
                     if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
                     pend_x[xb ^ 1] = false;
-                    if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
-                    pend_in2 = false;
                 }
                 if (one) {
                     if (ahead) {
                         chain_logits(t_u, xbuf(xb ^ 1), sb0 + L::kW);
                         mma_commit(c.bar(BW_LFULL));
                     }
-                    chain_dv(t_dv, sb0 + L::kP, sb0 + L::kShi, sb0 + L::kSlo);
                     chain_dx_dw(t_dk, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
-                    mma_commit(c.bar(BW_GFULL));
-                    if (ahead) issue_t();   // the element-wise warps took this tile's T out of tensor memory before they announced its operands
+                    mma_commit(c.bar(BW_G1));
                 }
                 __syncwarp();
                 if (ahead) {
-                    // V's tile is free once that product is done: the V of the tile after the next
-                    if (!issuer_wait(c, BW_TFULL, ph_t, kErrMmaAcc)) { ok = false; break; }
-                    if (ahead2 && one) load_v(nn);
-                    pend_in2 = ahead2;
+                    if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
+                    pend_in2 = false;
+                    if (one) issue_t();   // the element-wise warps took this tile's T out of tensor memory before they announced its operands
                 }
-                // ---- dv (in phi's tile) and dk (in this tile's K buffer) have been staged: store them; the buffers are free
-                // once the stores have read them ----
-                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
                 if (one) {
-                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kP + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                    chain_dv(t_dv, sb0 + L::kP, sb0 + L::kShi, sb0 + L::kSlo);
+                    mma_commit(c.bar(BW_GFULL));
+                }
+                __syncwarp();
+                // ---- dk has been staged in this tile's K buffer: store it; the buffer then takes the K of the tile after the next ----
+                if (!issuer_wait(c, BW_STAGED1, ph_staged1, kErrStore)) { ok = false; break; }
+                if (one) {
                     for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, xbuf(xb) + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
                     bulk_commit_group();
-                    bulk_wait_group_read<0>();
-                    mbar_arrive(c.bar(BW_PFREE));
-                    if (ahead2) load_k(nn, xb);
-                    else if (!ahead && !nx.done()) {
-                        // the next head: the staged results were drained after this tile's last stage, so every buffer is free
+                    if (ahead2) {
+                        bulk_wait_group_read<0>();
+                        load_k(nn, xb);
+                    }
+                }
+                __syncwarp();
+                if (ahead2) pend_x[xb] = true;
+                // ---- dv has been staged in V's tile (the next tile's V dS^T is done with it): store it; the tile then takes
+                // the V of the tile after the next, or, at the end of a head, everything is free for the next head's copies ----
+                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
+                if (one) {
+                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kV + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                    bulk_commit_group();
+                    if (ahead2) {
+                        bulk_wait_group_read<0>();
+                        load_v(nn);
+                    } else if (!ahead && !nx.done()) {
+                        bulk_wait_group_read<0>();
                         load_seg(nx);
                         load_k(nx, xb ^ 1);
                         load_v(nx);
                     }
                 }
                 __syncwarp();
-                if (ahead2) pend_x[xb] = true;
+                if (ahead2) pend_in2 = true;
                 else if (!ahead && !nx.done()) pend_seg = pend_x[xb ^ 1] = pend_in2 = true;
                 pre = ahead;
             }
@@ -881,20 +913,19 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
         const int half = warp >> 2, row = (warp & 3) * 32 + lane;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         float* vec = c.misc + BwdMisc::kVec / 4;
-        uint32_t ph_l = 0, ph_t = 0, ph_g = 0, ph_p = 0;
-        // dv and dk of a tile leave tensor memory (its last tensor-core stage has completed): dv to phi's tile, dk to the
-        // tile's own K buffer
-        auto stage_dv_dk = [&](int buf) {
-            {
-                float x[kM];
-                load64(t_dv + lane_base + half * kM, x);
-                store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, x);
-            }
-            {
-                float x[kM];
-                load64(t_dk + lane_base + half * kM, x);
-                store_row_bf16(c.smem + (buf ? L::kX1 : L::kX0) + half * kHalfTileBytes, row, x);
-            }
+        uint32_t ph_l = 0, ph_t = 0, ph_g1 = 0, ph_g = 0;
+        // dk of a tile leaves tensor memory for the tile's own K buffer (dk and dW_k are complete: the buffer has been read)
+        auto stage_dk = [&](int buf) {
+            float x[kM];
+            load64(t_dk + lane_base + half * kM, x);
+            store_row_bf16(c.smem + (buf ? L::kX1 : L::kX0) + half * kHalfTileBytes, row, x);
+            warp_announce(c, BW_STAGED1);
+        };
+        // dv leaves for V's tile (the V dS^T that read it last is complete)
+        auto stage_dv = [&]() {
+            float x[kM];
+            load64(t_dv + lane_base + half * kM, x);
+            store_row_bf16(c.smem + L::kV + half * kHalfTileBytes, row, x);
             warp_announce(c, BW_STAGED);
         };
         bool pre = false;
@@ -913,9 +944,9 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             if (half == 0) softmax_half_packed<false>(p, pk, vec);   // (the returned dot product is not needed here: vec may still be the old one)
             else softmax_half_packed<true>(p, pk, vec + kM);
             if (pre) {
-                // ---- the previous tile's last stage has had the time of a feature map: its dv and dk leave ----
-                if (!compute_wait(c, BW_GFULL, ph_g, kErrStore, okl)) break;
-                stage_dv_dk(xb ^ 1);
+                // ---- the previous tile's dk and dW_k have had the time of a feature map: dk leaves, the du tile is free ----
+                if (!compute_wait(c, BW_G1, ph_g1, kErrStore, okl)) break;
+                stage_dk(xb ^ 1);
             }
             if (!compute_wait(c, BW_TFULL, ph_t, kErrMmaAcc, okl)) break;
             // ---- dphi = V dS^T + dz -> du ----
@@ -926,7 +957,11 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
                 du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
             }
-            if (w.i > 0) okl = wait_only(c, BW_PFREE, ph_p, kErrEpilogue) && okl;
+            if (pre) {
+                // ---- the previous tile's dv is complete: it leaves through V's tile, and phi's tile is free ----
+                if (!compute_wait(c, BW_GFULL, ph_g, kErrStore)) break;
+                stage_dv();
+            }
             {
                 uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
 #pragma unroll
@@ -937,8 +972,10 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             pre = !last && !nx.done();
             if (pre) continue;
             // ---- the last tile of the head (or of the run): finished here ----
-            if (!compute_wait(c, BW_GFULL, ph_g, kErrStore, okl)) break;
-            stage_dv_dk(xb);
+            if (!compute_wait(c, BW_G1, ph_g1, kErrStore)) break;
+            stage_dk(xb);
+            if (!compute_wait(c, BW_GFULL, ph_g, kErrStore)) break;
+            stage_dv();
             drain_dw(t_dw, lane_base, half, row, a.part_w + (size_t)(blockIdx.x + w.g) * kWRec);
             tcgen05_fence_before();
             cbar();
