@@ -31,8 +31,10 @@
 namespace linattn {
 namespace tc {
 
-// Warps 0-7 do the element-wise work (thread = (token, half of the features)); warp 8 issues every copy and every
-// tensor-core product; warps 9-11 only complete warp 8's group of four, which gives most of its registers to the others.
+// Warps 0-7 do the element-wise work (thread = (token, half of the features)); warp 8 issues the tensor-core products
+// and the copies they wait for; warp 9 stores the staged results and, once a store has read its buffer, requests the
+// tile that comes into it next (a wait the issuer must not sit in); warps 10-11 only complete the group of four, which
+// gives most of its registers to the element-wise warps.
 constexpr int kBwdThreads = 384;
 constexpr int kBwdCompute = 256;
 constexpr int kBwdIssuer = 8;
@@ -66,8 +68,13 @@ struct BwdArgs {
     do {                                                                                                              \
         if (a.trace && threadIdx.x == 0 && w.i < 8) a.trace[((size_t)blockIdx.x * 8 + w.i) * 16 + (ev)] = clock64(); \
     } while (0)
+#define LB_TRACE_K(ev)                                                                                                \
+    do {                                                                                                              \
+        if (a.trace && threadIdx.x == 0 && w.i < 8) a.trace[((size_t)(148 + blockIdx.x) * 8 + w.i) * 16 + (ev)] = clock64(); \
+    } while (0)
 #else
 #define LB_TRACE(ev) do { } while (0)
+#define LB_TRACE_K(ev) do { } while (0)
 #endif
 
 // Shared memory, both kernels: two buffers for the tile that feeds the logits (the next tile's is fetched while this
@@ -375,7 +382,19 @@ __device__ __forceinline__ void drain_dw(uint32_t t_dw, uint32_t lane_base, int 
     for (int j = 0; j < 32; ++j) rec[(size_t)(half * 32 + j) * kD + row] = __uint_as_float(v[j]);
 }
 
-// The issuer's waits: the whole warp waits (bounded), the verdict is warp-uniform.
+// Unwinding after a wait that gave up: whatever copies into shared memory are still in flight (requested by this warp or
+// by the store warp, which requests none after the two have met) get a short while to land before the CTA gives its shared
+// memory back.  A barrier whose current phase has no copy outstanding just runs out the short limit.
+__device__ __forceinline__ void settle_copies(const BwdCta& c, uint32_t ph_seg, uint32_t ph_x0, uint32_t ph_x1, uint32_t ph_in2)
+{
+    constexpr uint64_t kSettleNs = 20000;
+    mbar_wait(c.bar(BW_SEG), ph_seg, kSettleNs);
+    mbar_wait(c.bar(BW_X0), ph_x0, kSettleNs);
+    mbar_wait(c.bar(BW_X1), ph_x1, kSettleNs);
+    mbar_wait(c.bar(BW_IN2), ph_in2, kSettleNs);
+}
+
+// The issuer's and the store warp's waits: the whole warp waits (bounded), the verdict is warp-uniform.
 __device__ __forceinline__ bool issuer_wait(const BwdCta& c, int b, uint32_t& phase, uint32_t code)
 {
     const bool ok = warp_wait(c.bar(b), phase, c.wc, code);
@@ -411,8 +430,8 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
     if (warp >= kBwdIssuer) {
         setmaxnreg_dec<kBwdRegsIssuer>();
-        if (warp == kBwdIssuer) {
-            // =================== issuer: every copy, every tensor-core product, every store ===================
+        if (warp <= kBwdIssuer + 1) {
+            // =================== issuer (warp 8) and store warp (warp 9) ===================
             const bool one = lane == 0;
             if (one) {
                 tma_prefetch_desc(&tmQ);
@@ -444,42 +463,66 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 chain_images(t_t, sb0 + L::kG, sb0 + L::kShi, sb0 + L::kSlo);
                 mma_commit(c.bar(BW_TFULL));
             };
-            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops1 = 0, ph_ops = 0, ph_staged = 0, ph_g1 = 0;
-            bool pend_x[2] = {false, false}, pend_in2 = false, pend_seg = false;   // copies requested and not yet waited for
+            if (warp == kBwdIssuer + 1) {
+                // =================== store warp ===================
+                uint32_t ph_staged = 0;
+                int xb = 0;
+                for (; !w.done(); w.next(), xb ^= 1) {
+                    const bool last = w.last();
+                    TileWalk nx = w;
+                    nx.next();
+                    TileWalk nn = nx;
+                    nn.next();
+                    const bool ahead = !last && !nx.done();
+                    const bool ahead2 = ahead && !nx.last() && !nn.done();
+                    // dq of this tile has been staged in the tile's own Q buffer (so its last stage is complete): store it; the
+                    // buffer then takes the Q of the tile after the next, or, at the end of a head, everything is free for
+                    // the next head's copies
+                    if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) break;
+                    if (one) {
+                        for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, xbuf(xb) + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                        bulk_commit_group();
+                        if (ahead2) {
+                            bulk_wait_group_read<0>();
+                            load_q(nn, xb);
+                        } else if (!ahead && !nx.done()) {
+                            bulk_wait_group_read<0>();   // (the store before this one read the other Q buffer)
+                            load_seg(nx);
+                            load_q(nx, xb ^ 1);
+                            load_g(nx);
+                        }
+                    }
+                    __syncwarp();
+                }
+                if (one) bulk_wait_group<0>();
+                named_barrier_sync(2, 64);   // no copy is requested after this point
+            } else {
+            // =================== issuer ===================
+            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops1 = 0, ph_ops = 0, ph_g1 = 0;
             bool ok = true, pre = false;
             int xb = 0;
-            if (!w.done()) {
-                if (one) {
-                    load_seg(w);
-                    load_q(w, 0);
-                    load_g(w);
-                }
-                pend_seg = pend_x[0] = pend_in2 = true;
+            if (!w.done() && one) {
+                load_seg(w);
+                load_q(w, 0);
+                load_g(w);
             }
             for (; !w.done(); w.next(), xb ^= 1) {
                 const bool first = w.first(), last = w.last();
                 TileWalk nx = w;
                 nx.next();
-                TileWalk nn = nx;
-                nn.next();
-                const bool ahead = !last && !nx.done();               // the next tile belongs to the same head
-                const bool ahead2 = ahead && !nx.last() && !nn.done();  // and so does the one after it
+                const bool ahead = !last && !nx.done();   // the next tile belongs to the same head
                 if (!pre) {
                     // ---- the head's first tile: U = Q W_q once Q, W_q are there, T = dO S^T once dO, S are there ----
                     if (first) {
                         if (!issuer_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
-                        pend_seg = false;
                     }
                     if (!issuer_wait(c, BW_X0 + xb, ph_x[xb], kErrMmaLoad)) { ok = false; break; }
-                    pend_x[xb] = false;
                     if (one) {
                         chain_logits(t_u, xbuf(xb), sb0 + L::kW);
                         mma_commit(c.bar(BW_LFULL));
                         if (ahead) load_q(nx, xb ^ 1);
                     }
-                    pend_x[xb ^ 1] = ahead;
                     if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
-                    pend_in2 = false;
                     if (one) issue_t();
                     __syncwarp();
                 }
@@ -492,17 +535,13 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
                 __syncwarp();
                 if (!issuer_wait(c, BW_G1, ph_g1, kErrMmaAcc)) { ok = false; break; }
-                if (ahead) {
-                    if (one) load_g(nx);
-                    pend_in2 = true;
-                }
+                if (ahead && one) load_g(nx);
                 // ---- du is written: the next tile's logits first (its feature map waits for nothing else), then
                 // dq = du W_q^T, dW_q += Q^T du, then the next tile's T = dO S^T (the element-wise warps took this tile's T
                 // out of tensor memory before they announced phi / den) ----
                 if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
                 if (ahead) {
                     if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
-                    pend_x[xb ^ 1] = false;
                 }
                 if (one) {
                     if (ahead) {
@@ -515,41 +554,14 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 __syncwarp();
                 if (ahead) {
                     if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
-                    pend_in2 = false;
                     if (one) issue_t();
                     __syncwarp();
                 }
-                // ---- dq of this tile has been staged in the tile's own Q buffer (so its last stage is complete): store it;
-                // the buffer then takes the Q of the tile after the next, or, at the end of a head, everything is free
-                // for the next head's copies ----
-                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
-                if (one) {
-                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDQ, xbuf(xb) + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-                    bulk_commit_group();
-                    if (!ahead && !nx.done()) {
-                        bulk_wait_group_read<0>();   // (the store before this one read the other Q buffer)
-                        load_seg(nx);
-                        load_q(nx, xb ^ 1);
-                        load_g(nx);
-                    }
-                    if (ahead2) {
-                        bulk_wait_group_read<0>();
-                        load_q(nn, xb);
-                    }
-                }
-                __syncwarp();
-                if (!ahead && !nx.done()) pend_seg = pend_x[xb ^ 1] = pend_in2 = true;
-                if (ahead2) pend_x[xb] = true;
                 pre = ahead;
             }
-            if (!ok) {
-                // unwinding: let the copies already requested land before the CTA gives its shared memory back
-                if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
-                for (int b = 0; b < 2; ++b)
-                    if (pend_x[b]) mbar_wait(c.bar(BW_X0 + b), ph_x[b], c.wc.limit_ns());
-                if (pend_in2) mbar_wait(c.bar(BW_IN2), ph_in2, c.wc.limit_ns());
+            named_barrier_sync(2, 64);
+            if (!ok) settle_copies(c, ph_seg, ph_x[0], ph_x[1], ph_in2);
             }
-            if (one) bulk_wait_group<0>();
         }
     } else {
         setmaxnreg_inc<kBwdRegsCompute>();
@@ -752,8 +764,8 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
 
     if (warp >= kBwdIssuer) {
         setmaxnreg_dec<kBwdRegsIssuer>();
-        if (warp == kBwdIssuer) {
-            // =================== issuer ===================
+        if (warp <= kBwdIssuer + 1) {
+            // =================== issuer (warp 8) and store warp (warp 9) ===================
             const bool one = lane == 0;
             if (one) {
                 tma_prefetch_desc(&tmK);
@@ -790,49 +802,83 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 chain_images(t_t, sb0 + L::kV, sb0 + L::kShi, sb0 + L::kSlo);
                 mma_commit(c.bar(BW_TFULL));
             };
-            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_staged1 = 0, ph_staged = 0, ph_t = 0;
-            bool pend_x[2] = {false, false}, pend_in2 = false, pend_seg = false;
+            if (warp == kBwdIssuer + 1) {
+                // =================== store warp ===================
+                uint32_t ph_staged1 = 0, ph_staged = 0;
+                int xb = 0;
+                for (; !w.done(); w.next(), xb ^= 1) {
+                    const bool last = w.last();
+                    TileWalk nx = w;
+                    nx.next();
+                    TileWalk nn = nx;
+                    nn.next();
+                    const bool ahead = !last && !nx.done();
+                    const bool ahead2 = ahead && !nx.last() && !nn.done();
+                    // dk has been staged in this tile's K buffer (dk and dW_k are complete): store it; the buffer then takes the
+                    // K of the tile after the next
+                    if (!issuer_wait(c, BW_STAGED1, ph_staged1, kErrStore)) break;
+                    if (one) {
+                        for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, xbuf(xb) + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                        bulk_commit_group();
+                        if (ahead2) {
+                            bulk_wait_group_read<0>();
+                            load_k(nn, xb);
+                        }
+                    }
+                    __syncwarp();
+                    // dv has been staged in V's tile (the next tile's V dS^T is done with it): store it; the tile then takes the V
+                    // of the tile after the next, or, at the end of a head, everything is free for the next head's copies
+                    if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) break;
+                    if (one) {
+                        for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kV + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
+                        bulk_commit_group();
+                        if (ahead2) {
+                            bulk_wait_group_read<0>();
+                            load_v(nn);
+                        } else if (!ahead && !nx.done()) {
+                            bulk_wait_group_read<0>();
+                            load_seg(nx);
+                            load_k(nx, xb ^ 1);
+                            load_v(nx);
+                        }
+                    }
+                    __syncwarp();
+                }
+                if (one) bulk_wait_group<0>();
+                named_barrier_sync(2, 64);   // no copy is requested after this point
+            } else {
+            // =================== issuer ===================
+            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_t = 0;
             bool ok = true, pre = false;
             int xb = 0;
-            if (!w.done()) {
-                if (one) {
-                    load_seg(w);
-                    load_k(w, 0);
-                    load_v(w);
-                }
-                pend_seg = pend_x[0] = pend_in2 = true;
+            if (!w.done() && one) {
+                load_seg(w);
+                load_k(w, 0);
+                load_v(w);
             }
             for (; !w.done(); w.next(), xb ^= 1) {
                 const bool first = w.first(), last = w.last();
                 TileWalk nx = w;
                 nx.next();
-                TileWalk nn = nx;
-                nn.next();
                 const bool ahead = !last && !nx.done();
-                const bool ahead2 = ahead && !nx.last() && !nn.done();
                 if (!pre) {
                     // ---- the head's first tile: U = K W_k once K, W_k are there, T = V dS^T once V, dS are there; V's tile then
                     // takes the next tile's V ----
                     if (first) {
                         if (!issuer_wait(c, BW_SEG, ph_seg, kErrSeg)) { ok = false; break; }
-                        pend_seg = false;
                     }
                     if (!issuer_wait(c, BW_X0 + xb, ph_x[xb], kErrMmaLoad)) { ok = false; break; }
-                    pend_x[xb] = false;
                     if (one) {
                         chain_logits(t_u, xbuf(xb), sb0 + L::kW);
                         mma_commit(c.bar(BW_LFULL));
                         if (ahead) load_k(nx, xb ^ 1);
                     }
-                    pend_x[xb ^ 1] = ahead;
                     if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
-                    pend_in2 = false;
                     if (one) issue_t();
                     __syncwarp();
                     if (ahead) {
                         if (!issuer_wait(c, BW_TFULL, ph_t, kErrMmaAcc)) { ok = false; break; }
                         if (one) load_v(nx);
-                        pend_in2 = true;
                     } else {
                         ph_t ^= 1u;   // (that phase is not waited for here)
                     }
@@ -845,7 +891,6 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
                 if (ahead) {
                     if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
-                    pend_x[xb ^ 1] = false;
                 }
                 if (one) {
                     if (ahead) {
@@ -858,7 +903,6 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 __syncwarp();
                 if (ahead) {
                     if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
-                    pend_in2 = false;
                     if (one) issue_t();   // the element-wise warps took this tile's T out of tensor memory before they announced its operands
                 }
                 if (one) {
@@ -866,46 +910,11 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                     mma_commit(c.bar(BW_GFULL));
                 }
                 __syncwarp();
-                // ---- dk has been staged in this tile's K buffer: store it; the buffer then takes the K of the tile after the next ----
-                if (!issuer_wait(c, BW_STAGED1, ph_staged1, kErrStore)) { ok = false; break; }
-                if (one) {
-                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDK, xbuf(xb) + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-                    bulk_commit_group();
-                    if (ahead2) {
-                        bulk_wait_group_read<0>();
-                        load_k(nn, xb);
-                    }
-                }
-                __syncwarp();
-                if (ahead2) pend_x[xb] = true;
-                // ---- dv has been staged in V's tile (the next tile's V dS^T is done with it): store it; the tile then takes
-                // the V of the tile after the next, or, at the end of a head, everything is free for the next head's copies ----
-                if (!issuer_wait(c, BW_STAGED, ph_staged, kErrStore)) { ok = false; break; }
-                if (one) {
-                    for (int b = 0; b < 2; ++b) act_store<kLayout>(&tmDV, sb0 + L::kV + b * kHalfTileBytes, 64 * b, w.lt * kTile, w.g, a.H);
-                    bulk_commit_group();
-                    if (ahead2) {
-                        bulk_wait_group_read<0>();
-                        load_v(nn);
-                    } else if (!ahead && !nx.done()) {
-                        bulk_wait_group_read<0>();
-                        load_seg(nx);
-                        load_k(nx, xb ^ 1);
-                        load_v(nx);
-                    }
-                }
-                __syncwarp();
-                if (ahead2) pend_in2 = true;
-                else if (!ahead && !nx.done()) pend_seg = pend_x[xb ^ 1] = pend_in2 = true;
                 pre = ahead;
             }
-            if (!ok) {
-                if (pend_seg) mbar_wait(c.bar(BW_SEG), ph_seg, c.wc.limit_ns());
-                for (int b = 0; b < 2; ++b)
-                    if (pend_x[b]) mbar_wait(c.bar(BW_X0 + b), ph_x[b], c.wc.limit_ns());
-                if (pend_in2) mbar_wait(c.bar(BW_IN2), ph_in2, c.wc.limit_ns());
+            named_barrier_sync(2, 64);
+            if (!ok) settle_copies(c, ph_seg, ph_x[0], ph_x[1], ph_in2);
             }
-            if (one) bulk_wait_group<0>();
         }
     } else {
         setmaxnreg_inc<kBwdRegsCompute>();
@@ -935,20 +944,26 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             const bool first = w.first(), last = w.last();
             TileWalk nx = w;
             nx.next();
+            LB_TRACE_K(0);
             if (first && tid < kD) vec[tid] = a.state[(size_t)w.g * kE + kD * kD + tid];   // dz (read after the next barrier)
             okl = wait_only(c, BW_LFULL, ph_l, kErrSoftmaxU) && okl;
+            LB_TRACE_K(2);
             // ---- phi(k): p stays in registers (fp32, and its bf16 roundings, which go to phi's tile once that is free) ----
             float p[kM];
             uint32_t pk[kM / 2];
             load64(t_u + lane_base, p);
             if (half == 0) softmax_half_packed<false>(p, pk, vec);   // (the returned dot product is not needed here: vec may still be the old one)
             else softmax_half_packed<true>(p, pk, vec + kM);
+            LB_TRACE_K(3);
             if (pre) {
                 // ---- the previous tile's dk and dW_k have had the time of a feature map: dk leaves, the du tile is free ----
                 if (!compute_wait(c, BW_G1, ph_g1, kErrStore, okl)) break;
+                LB_TRACE_K(6);
                 stage_dk(xb ^ 1);
+                LB_TRACE_K(7);
             }
             if (!compute_wait(c, BW_TFULL, ph_t, kErrMmaAcc, okl)) break;
+            LB_TRACE_K(4);
             // ---- dphi = V dS^T + dz -> du ----
             {
                 float x[kM];
@@ -957,10 +972,13 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
                 du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
             }
+            LB_TRACE_K(5);
             if (pre) {
                 // ---- the previous tile's dv is complete: it leaves through V's tile, and phi's tile is free ----
                 if (!compute_wait(c, BW_GFULL, ph_g, kErrStore)) break;
+                LB_TRACE_K(10);
                 stage_dv();
+                LB_TRACE_K(11);
             }
             {
                 uint8_t* blk = c.smem + L::kP + half * kHalfTileBytes;
@@ -969,6 +987,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                     *reinterpret_cast<uint4*>(blk + sw_chunk(row, ch)) = make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
             }
             warp_announce(c, BW_OPS);
+            LB_TRACE_K(8);
             pre = !last && !nx.done();
             if (pre) continue;
             // ---- the last tile of the head (or of the run): finished here ----
