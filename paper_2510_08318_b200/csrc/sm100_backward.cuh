@@ -72,9 +72,14 @@ struct BwdArgs {
     do {                                                                                                              \
         if (a.trace && threadIdx.x == 0 && w.i < 8) a.trace[((size_t)(148 + blockIdx.x) * 8 + w.i) * 16 + (ev)] = clock64(); \
     } while (0)
+#define LB_TRACE_I(region, ev)                                                                                        \
+    do {                                                                                                              \
+        if (a.trace && one && w.i < 8) a.trace[((size_t)((region) * 148 + blockIdx.x) * 8 + w.i) * 16 + (ev)] = clock64(); \
+    } while (0)
 #else
 #define LB_TRACE(ev) do { } while (0)
 #define LB_TRACE_K(ev) do { } while (0)
+#define LB_TRACE_I(region, ev) do { } while (0)
 #endif
 
 // Shared memory, both kernels: two buffers for the tile that feeds the logits (the next tile's is fetched while this
@@ -280,8 +285,8 @@ __device__ __forceinline__ void store_row_bf16(uint8_t* blk, int row, const floa
 
 // Softmax backward of Eq. 6 for one token, split between the two threads of the token (half 0: softmax(+u),
 // half 1: softmax(-u)): each forms p (.) (dphi - p . dphi) for its half; half 1 parks its 64 values in 64 free columns
-// of the token's lane of tensor memory (`park`: the logits' columns, read long before; both threads of a token sit on
-// warps of the same lane quarter, so either can reach the lane), and after a barrier of these warps half 0 takes them back,
+// of the token's lane of tensor memory (`park`: the columns of T that half 1 itself has just read; both threads of a token
+// sit on warps of the same lane quarter, so either can reach the lane), and after a barrier of these warps half 0 takes them back,
 // subtracts and writes du (bf16) to its row of the du tile.
 __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint32_t park, uint8_t* du_tile)
 {
@@ -422,7 +427,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (!bwd_smem_fits(bwd_smem, kBwdSmemQ, a.err)) return;
     const BwdCta c = bwd_setup(bwd_smem, L::kMisc, a.err);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // tensor memory: logits (later the du exchange) | T = dO S^T | dS | dW_q | dq
+    // tensor memory: logits | T = dO S^T (later the du exchange) | dS | dW_q | dq
     const uint32_t t_u = c.tmem, t_t = c.tmem + 64, t_ds = c.tmem + 192, t_dw = c.tmem + 320, t_dq = c.tmem + 384;
     const uint32_t sb0 = c.sbase;
     TileWalk w;
@@ -529,33 +534,43 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 // ---- phi / den of this tile is written: dS += (phi / den)^T dO at once, so that dO's tile is free for the
                 // next tile's dO while this tile's du is still being formed ----
                 if (!issuer_wait(c, BW_OPS1, ph_ops1, kErrMmaPhi)) { ok = false; break; }
+                LB_TRACE_I(2, 0);
                 if (one) {
                     chain_ds(t_ds, sb0 + L::kP, sb0 + L::kG, first);
                     mma_commit(c.bar(BW_G1));
                 }
                 __syncwarp();
-                if (!issuer_wait(c, BW_G1, ph_g1, kErrMmaAcc)) { ok = false; break; }
-                if (ahead && one) load_g(nx);
-                // ---- du is written: the next tile's logits first (its feature map waits for nothing else), then
-                // dq = du W_q^T, dW_q += Q^T du, then the next tile's T = dO S^T (the element-wise warps took this tile's T
-                // out of tensor memory before they announced phi / den) ----
-                if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
+                LB_TRACE_I(2, 1);
                 if (ahead) {
+                    // the next tile's logits (this tile's have long been read, and its Q came in a tile ago)
                     if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
-                }
-                if (one) {
-                    if (ahead) {
+                    if (one) {
                         chain_logits(t_u, xbuf(xb ^ 1), sb0 + L::kW);
                         mma_commit(c.bar(BW_LFULL));
                     }
+                    __syncwarp();
+                }
+                LB_TRACE_I(2, 2);
+                if (!issuer_wait(c, BW_G1, ph_g1, kErrMmaAcc)) { ok = false; break; }
+                LB_TRACE_I(2, 3);
+                if (ahead && one) load_g(nx);
+                // ---- du is written: dq = du W_q^T, dW_q += Q^T du, then the next tile's T = dO S^T (the element-wise warps
+                // took this tile's T out of tensor memory before they announced phi / den, and are done with the columns
+                // they exchange du through) ----
+                if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
+                LB_TRACE_I(2, 4);
+                if (one) {
                     chain_dx_dw(t_dq, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
                     mma_commit(c.bar(BW_GFULL));
                 }
                 __syncwarp();
+                LB_TRACE_I(2, 5);
                 if (ahead) {
                     if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
+                    LB_TRACE_I(2, 6);
                     if (one) issue_t();
                     __syncwarp();
+                    LB_TRACE_I(2, 7);
                 }
                 pre = ahead;
             }
@@ -671,7 +686,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
                 unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
             }
-            du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);   // (a barrier inside: both halves of sb have been read)
+            du_exchange(half, row, p, x, t_t + kM + lane_base, c.smem + L::kDu);   // (a barrier inside: both halves of sb have been read)
             if (half == 0) sdd[row] = ngo;
             warp_announce(c, BW_OPS);
             cbar();
@@ -756,7 +771,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
     if (!bwd_smem_fits(bwd_smem, kBwdSmemK, a.err)) return;
     const BwdCta c = bwd_setup(bwd_smem, L::kMisc, a.err);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // tensor memory: logits (later the du exchange) | T = V dS^T | dv | dW_k | dk
+    // tensor memory: logits | T = V dS^T (later the du exchange) | dv | dW_k | dk
     const uint32_t t_u = c.tmem, t_t = c.tmem + 64, t_dv = c.tmem + 192, t_dw = c.tmem + 320, t_dk = c.tmem + 384;
     const uint32_t sb0 = c.sbase;
     TileWalk w;
@@ -848,7 +863,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 named_barrier_sync(2, 64);   // no copy is requested after this point
             } else {
             // =================== issuer ===================
-            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops = 0, ph_t = 0;
+            uint32_t ph_x[2] = {0u, 0u}, ph_in2 = 0, ph_seg = 0, ph_ops1 = 0, ph_ops = 0, ph_t = 0;
             bool ok = true, pre = false;
             int xb = 0;
             if (!w.done() && one) {
@@ -885,31 +900,41 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 } else {
                     ph_t ^= 1u;       // this tile's V dS^T was issued during the previous tile
                 }
-                // ---- phi and du of this tile are written: the next tile's logits first, then dk = du W_k^T and
-                // dW_k += K^T du (the du tile and this tile's K buffer are free after them), the next tile's V dS^T, and
-                // dv = phi dS (hi and lo parts) last ----
-                if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
+                // ---- this tile's logits have been read: the next tile's; then, phi and du of this tile written,
+                // dk = du W_k^T and dW_k += K^T du (the du tile and this tile's K buffer are free after them), the next
+                // tile's V dS^T, and dv = phi dS (hi and lo parts) last ----
+                if (!issuer_wait(c, BW_OPS1, ph_ops1, kErrMmaU)) { ok = false; break; }
+                LB_TRACE_I(3, 0);
                 if (ahead) {
                     if (!issuer_wait(c, BW_X0 + (xb ^ 1), ph_x[xb ^ 1], kErrMmaLoad)) { ok = false; break; }
-                }
-                if (one) {
-                    if (ahead) {
+                    if (one) {
                         chain_logits(t_u, xbuf(xb ^ 1), sb0 + L::kW);
                         mma_commit(c.bar(BW_LFULL));
                     }
+                    __syncwarp();
+                }
+                LB_TRACE_I(3, 1);
+                if (!issuer_wait(c, BW_OPS, ph_ops, kErrMmaPhi)) { ok = false; break; }
+                LB_TRACE_I(3, 2);
+                if (one) {
                     chain_dx_dw(t_dk, t_dw, sb0 + L::kDu, xbuf(xb), sb0 + L::kW, first);
                     mma_commit(c.bar(BW_G1));
                 }
                 __syncwarp();
+                LB_TRACE_I(3, 3);
                 if (ahead) {
                     if (!issuer_wait(c, BW_IN2, ph_in2, kErrMmaLoad)) { ok = false; break; }
+                    LB_TRACE_I(3, 4);
                     if (one) issue_t();   // the element-wise warps took this tile's T out of tensor memory before they announced its operands
                 }
+                __syncwarp();
+                LB_TRACE_I(3, 5);
                 if (one) {
                     chain_dv(t_dv, sb0 + L::kP, sb0 + L::kShi, sb0 + L::kSlo);
                     mma_commit(c.bar(BW_GFULL));
                 }
                 __syncwarp();
+                LB_TRACE_I(3, 6);
                 pre = ahead;
             }
             named_barrier_sync(2, 64);
@@ -952,6 +977,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
             float p[kM];
             uint32_t pk[kM / 2];
             load64(t_u + lane_base, p);
+            warp_announce(c, BW_OPS1);   // the logits' columns may take the next tile's
             if (half == 0) softmax_half_packed<false>(p, pk, vec);   // (the returned dot product is not needed here: vec may still be the old one)
             else softmax_half_packed<true>(p, pk, vec + kM);
             LB_TRACE_K(3);
@@ -970,7 +996,7 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 load64(t_t + lane_base + half * kM, x);
 #pragma unroll
                 for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
-                du_exchange(half, row, p, x, t_u + lane_base, c.smem + L::kDu);
+                du_exchange(half, row, p, x, t_t + kM + lane_base, c.smem + L::kDu);
             }
             LB_TRACE_K(5);
             if (pre) {
