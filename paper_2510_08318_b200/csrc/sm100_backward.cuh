@@ -319,18 +319,27 @@ __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[
     }
 }
 
-// n products D (+)= A_k B_k issued by one thread, the operands' start addresses advancing by fixed byte steps.  The loop
-// is NOT unrolled on purpose: the issuer warp runs on few registers, and the descriptor arithmetic of unrolled products
-// is hoisted out of the tile loop and spilled.
+// n products D (+)= A_k B_k issued by one thread, the operands' start addresses advancing by fixed byte steps.  Unrolled,
+// so that each descriptor is the first one plus a constant; the first ones pass through `opaque` so that this arithmetic
+// stays inside the tile loop (hoisted out of it, the descriptors of a whole tile would not fit the issuer's registers).
+__device__ __forceinline__ uint64_t opaque(uint64_t v)
+{
+    asm volatile("" : "+l"(v));
+    return v;
+}
+template <int kN>
+__device__ __forceinline__ void mma_chain_n(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t step_a, uint32_t step_b, uint32_t idesc, uint32_t acc_first)
+{
+    da = opaque(da);
+    db = opaque(db);
+#pragma unroll
+    for (int k = 0; k < kN; ++k) mma_bf16_ss(d_tmem, da + (uint64_t)(k * (step_a >> 4)), db + (uint64_t)(k * (step_b >> 4)), idesc, k > 0 ? 1u : acc_first);
+}
 __device__ __forceinline__ void mma_chain(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t step_a, uint32_t step_b, uint32_t idesc, int n,
                                           uint32_t acc_first)
 {
-#pragma unroll 1
-    for (int k = 0; k < n; ++k) {
-        mma_bf16_ss(d_tmem, da, db, idesc, k > 0 ? 1u : acc_first);
-        da += step_a >> 4;
-        db += step_b >> 4;
-    }
+    if (n == 4) mma_chain_n<4>(d_tmem, da, db, step_a, step_b, idesc, acc_first);
+    else mma_chain_n<8>(d_tmem, da, db, step_a, step_b, idesc, acc_first);
 }
 // K-major operand tiles are two 64-element blocks of four K steps each (32 bytes apart).
 __device__ __forceinline__ uint64_t kmajor_desc() { return make_desc_sw128(0, 16, 1024); }
