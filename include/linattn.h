@@ -59,13 +59,16 @@ typedef enum {
                                (or backward) on the same k and v POINTERS, B, n and layout, with the same feature map.
                                The caller promises that the contents of k and v have not changed in between (the
                                forward -> backward order of a training step).  0 = always recompute (default) */
-    LINATTN_OPT_WAIT_LIMIT_US = 7, /* bound, in microseconds, of every wait inside the tensor-core forward kernels (on a
-                               shared-memory barrier or on another CTA): default 2,000,000.  A wait that runs out makes the
-                               kernel record a code, unwind and return; linattn_check then reports LINATTN_ERR_TIMEOUT */
-    LINATTN_OPT_TEST_UNMET_ARRIVAL = 8, /* for tests of the time-out path only: 1 = the single-kernel forward waits, at the
-                               points where the CTAs that share a head meet, for one arrival more than will ever come, so
-                               that its bounded wait runs out (nothing faults or hangs: the kernel gives up after the wait
-                               limit, the output is not produced, linattn_check reports TIMEOUT).  0 = off (default) */
+    LINATTN_OPT_WAIT_LIMIT_US = 7, /* bound, in microseconds, of every wait inside the tensor-core kernels, forward and
+                               backward (on a shared-memory barrier or on another CTA): default 2,000,000.  A wait that
+                               runs out makes the kernel record a code, unwind and return; linattn_check then reports
+                               LINATTN_ERR_TIMEOUT */
+    LINATTN_OPT_TEST_UNMET_ARRIVAL = 8, /* for tests of the time-out path only.  1 = the single-kernel forward waits, at the
+                               points where the CTAs that share a head meet, for one arrival more than will ever come;
+                               2 / 3 = in the query-side / key-side kernel of the tensor-core backward one warp of every
+                               CTA leaves out one arrival that the warp issuing the tensor-core products waits for.  The
+                               bounded wait runs out (nothing faults or hangs: the kernel gives up after the wait limit,
+                               its output is not produced, linattn_check reports TIMEOUT).  0 = off (default) */
     LINATTN_OPT_PROFILE = 2 /* 1 = record CUDA events around every kernel of each forward (see linattn_profile_get);
                                switching it on clears the accumulated figures; 0 = off (default) */
 } linattn_option;

@@ -442,7 +442,7 @@ linattn_status launch_tc(linattn_ctx* c, const void* q, const void* k, const voi
     a.trace = c->trace;
 #endif
     a.wait_limit_us = (uint32_t)c->opt_wait_limit_us;
-    a.arrive_extra = (uint32_t)c->opt_unmet;
+    a.arrive_extra = c->opt_unmet == 1 ? 1u : 0u;
     prof_begin(c, st);
     if (c->opt_fuse && c->coop_ok && Pk == Pq && !state_only) {
         // one cooperative launch: key side, per-head meeting point, combine, per-head meeting point, query side.  Its
@@ -561,6 +561,8 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     a.G = (int)G;
     a.tiles_per_head = (int)Tn;
     a.total_tiles = T;
+    a.wait_limit_us = (uint32_t)c->opt_wait_limit_us;
+    a.test_unmet = c->opt_unmet == 2 ? 1 : 0;
 #ifdef LINATTN_TRACE
     a.trace = c->trace;
 #endif
@@ -586,6 +588,7 @@ linattn_status launch_backward_tc(linattn_ctx* c, const void* q, const void* k, 
     LA_CUDA(c, cudaGetLastError());
     prof_mark(c, st, "combine_dstate", 0.0);
     a.state = c->bwd_dstate;
+    a.test_unmet = c->opt_unmet == 3 ? 1 : 0;
     a.part_w = c->bwd_part_w2;   // dW_k's records; dW_q's stay in part_w until both are summed at the end
     {
         void* p[] = {&tmK, &tmV, &tmDK, &tmDV, &tmWk, &tmDShi, &tmDSlo, &a};
@@ -1106,7 +1109,7 @@ linattn_status linattn_set_option(linattn_ctx* c, linattn_option opt, long long 
             c->opt_wait_limit_us = value;
             return LINATTN_OK;
         case LINATTN_OPT_TEST_UNMET_ARRIVAL:
-            if (value != 0 && value != 1) return LINATTN_ERR_INVALID_ARG;
+            if (value < 0 || value > 3) return LINATTN_ERR_INVALID_ARG;
             c->opt_unmet = (int)value;
             return LINATTN_OK;
         case LINATTN_OPT_FUSE:

@@ -3,6 +3,10 @@ wait, where the CTAs that share a head meet, for one arrival more than will ever
 millisecond.  The wait runs out, the kernel records where, unwinds (copies in flight land, tensor memory is freed) and
 returns; the host reads the status.  The context must then be usable again and give the same bits as before.
 
+The tensor-core backward gets the same treatment: one warp of every CTA leaves out one arrival that the warp issuing
+the tensor-core products waits for, in the query-side or in the key-side kernel; every role of the kernel (issuer, store
+warp, element-wise warps) has to notice, unwind and meet at the kernel's last barrier.
+
 Also here: the forward recorded in a CUDA graph and replayed (its synchronisation counters are cleared by the kernel
 itself, so a replay starts from the same state as a fresh launch)."""
 import math
@@ -57,13 +61,45 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(H, n):
         fresh.destroy()
 
 
+@pytest.mark.parametrize("side", [2, 3])                    # query-side kernel, key-side kernel
+@pytest.mark.parametrize("H,n", [(2, 1024), (3, 32768)])     # at most one tile per CTA; five or six tiles per CTA (the pipelined path)
+def test_a_backward_wait_that_runs_out_is_reported_and_the_context_recovers(side, H, n):
+    q, k, v, Wq, Wk = _inputs(1, H, n, 128, seed=n + side)
+    g = torch.Generator().manual_seed(99)
+    dout = torch.randn(1, H, n, 128, generator=g).bfloat16().cuda()
+    ctx = linattn.LinAttn(H, 128, max_B=1, max_n=n)
+    try:
+        ctx.set_feature_map(Wq, Wk)
+        ref = ctx.backward(q, k, v, dout)
+        ctx.check()
+        assert ctx.last_launch_count() == 6, "the test is about the tensor-core backward"
+
+        ctx.set_option(linattn.OPT_WAIT_LIMIT_US, 1000)
+        ctx.set_option(linattn.OPT_TEST_UNMET_ARRIVAL, side)
+        ctx.backward(q, k, v, dout)
+        with pytest.raises(linattn.LinAttnError) as info:
+            ctx.check()
+        assert info.value.status == linattn.ERR_TIMEOUT
+        assert "gave up" in str(info.value)
+        ctx.check()   # the error word was cleared by the check that reported it
+
+        ctx.set_option(linattn.OPT_TEST_UNMET_ARRIVAL, 0)
+        ctx.set_option(linattn.OPT_WAIT_LIMIT_US, 2_000_000)
+        again = ctx.backward(q, k, v, dout)
+        ctx.check()
+        for x, y in zip(again, ref):
+            assert torch.equal(x, y), "the context must give the same bits after a timed-out launch"
+    finally:
+        ctx.destroy()
+
+
 def test_wait_limit_option_range():
     lib = linattn.load_library()
     ctx = linattn.LinAttn(2, 128, max_B=1, max_n=128)
     try:
         assert lib.linattn_set_option(ctx._h, linattn.OPT_WAIT_LIMIT_US, 0) == linattn.ERR_INVALID_ARG
         assert lib.linattn_set_option(ctx._h, linattn.OPT_WAIT_LIMIT_US, 10**9) == linattn.ERR_INVALID_ARG
-        assert lib.linattn_set_option(ctx._h, linattn.OPT_TEST_UNMET_ARRIVAL, 2) == linattn.ERR_INVALID_ARG
+        assert lib.linattn_set_option(ctx._h, linattn.OPT_TEST_UNMET_ARRIVAL, 4) == linattn.ERR_INVALID_ARG
         assert lib.linattn_set_option(ctx._h, linattn.OPT_WAIT_LIMIT_US, 5000) == linattn.OK
     finally:
         ctx.destroy()
