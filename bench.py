@@ -213,6 +213,8 @@ ALL_VARIANTS = [
     ("mixed attention (Eq. 8), r = 0.5, config 2", ["--config", "2", "--mixed", "0.5"]),
     ("ReLU kernel function, config 2", ["--config", "2", "--phi", "relu"]),
     ("backward, config 2", ["--config", "2", "--backward"]),
+    ("backward, config 3", ["--config", "3", "--backward"]),
+    ("backward, config 4", ["--config", "4", "--backward"]),
 ]
 
 
