@@ -72,8 +72,9 @@ class ClockSampler:
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
     BITS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, period_s: float = 0.0002):
         self.index, self.rows, self.proc, self.nvml, self.stop_flag = index, [], None, None, False
+        self.period_s = period_s
 
     def start(self):
         try:
@@ -104,7 +105,7 @@ class ClockSampler:
                 mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
                 bits = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
                 self.rows.append((t, mhz, bits))
-                time.sleep(0.0002)   # leave the interpreter to the thread that launches the kernels
+                time.sleep(self.period_s)   # leave the interpreter to the thread that launches the kernels
             except Exception:
                 break
 
@@ -261,6 +262,7 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="0 auto, 1 CUDA-core kernels, 2 tensor-core kernels")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-baselines", action="store_true", help="skip the oracle and SDPA context baselines")
+    ap.add_argument("--clock-period-ms", type=float, default=0.2, help="pause between two NVML samples of the SM clock (ms)")
     ap.add_argument("--mixed", type=float, default=None, metavar="R",
                     help="time mixed attention (Eq. 8) with score R instead: linattn_forward_mixed on a resident "
                          "softmax-branch output (5 tensors of traffic instead of 4)")
@@ -296,7 +298,7 @@ def main():
     assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torchrun --nproc-per-node {args.gpus}"
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    sampler = ClockSampler(local)   # started this early so that it is polling steadily by the time the timed region runs
+    sampler = ClockSampler(local, args.clock_period_ms * 1e-3)   # started this early so that it is polling steadily by the time the timed region runs
     if rank == 0:
         sampler.start()
 
