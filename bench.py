@@ -41,12 +41,14 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "source": "fallback"}
 
 
-def source_digest():
-    """Digest of the sources the forward's tensor-core kernels are built from (the kernels, their PTX wrappers and
-    the tensor maps): DRAM counters taken with ncu are only quoted for the code they were taken on."""
+def source_digest(kernel: str = "linattn_fused_tc"):
+    """Digest of the sources `kernel` is built from (the forward's tensor-core kernels, their PTX wrappers and the tensor
+    maps; for the backward's kernels their own file as well): DRAM counters taken with ncu are only quoted for the code
+    they were taken on."""
     import hashlib
     h = hashlib.sha256()
-    for name in ("sm100_kernels.cuh", "sm100_ptx.cuh", "tensor_map.hpp"):
+    names = ["sm100_kernels.cuh", "sm100_ptx.cuh", "tensor_map.hpp"] + (["sm100_backward.cuh"] if "bwd" in kernel else [])
+    for name in names:
         h.update(open(os.path.join(ROOT, "paper_2510_08318_b200", "csrc", name), "rb").read())
     return h.hexdigest()[:16]
 
@@ -59,7 +61,7 @@ def recorded_traffic(kernel):
         return None
     for line in open(path):
         f = line.split()
-        if len(f) == 3 and f[0] == kernel and f[2] == source_digest():
+        if len(f) == 3 and f[0] == kernel and f[2] == source_digest(kernel):
             return float(f[1])
     return None
 
@@ -281,7 +283,7 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.source_digest:
-        print(source_digest())
+        print(source_digest(), "(forward kernels)", source_digest("qside_bwd_tc"), "(backward kernels)")
         return
     if args.all:
         run_all(args)
@@ -421,7 +423,9 @@ def main():
                                "frac": alg_total / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                "frac_of_nominal_8TBs": alg_total / (ms_step * 1e-3) / 1e9 / 8000.0,
                                "algorithmic_bytes": alg_total}}
-    roofline["traffic"] = recorded_traffic(dom["name"]) if softs is None and douts is None and args.phi == "hedgehog" else None
+    # recorded at config 2, default layout, Eq. 6 feature map only
+    plain = softs is None and args.phi == "hedgehog" and args.config == 2 and args.layout == 0
+    roofline["traffic"] = recorded_traffic(dom["name"]) if plain else None
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host tensor out
     pin = {k_: host0[k_].pin_memory() for k_ in ("q", "k", "v")}
