@@ -264,6 +264,42 @@ __device__ __forceinline__ float softmax_half_packed(float (&u)[kM], uint32_t (&
     return s0 + s1;
 }
 
+// The same without the roundings: p[64] (fp32) in place; returns sum_j p_j * vec[j].
+template <bool kNeg>
+__device__ __forceinline__ float softmax_half_plain(float (&u)[kM], const float* vec)
+{
+    float m = kNeg ? min3(u[0], u[1], u[2]) : max3(u[0], u[1], u[2]);
+#pragma unroll
+    for (int j = 3; j < kM - 1; j += 2) m = kNeg ? min3(m, u[j], u[j + 1]) : max3(m, u[j], u[j + 1]);
+    m = kNeg ? fminf(m, u[kM - 1]) : fmaxf(m, u[kM - 1]);
+    const float sL = kNeg ? -kLog2e : kLog2e, off = kNeg ? m * kLog2e : -m * kLog2e;
+    const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
+    f32x2 sum2 = pack2(0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < kM; j += 2) {
+        float x0, x1;
+        unpack2(fma2(pack2(u[j], u[j + 1]), scale, offset), x0, x1);
+        u[j] = ex2_approx(x0);
+        u[j + 1] = ex2_approx(x1);
+        sum2 = add2(sum2, pack2(u[j], u[j + 1]));
+    }
+    float s0, s1;
+    unpack2(sum2, s0, s1);
+    const float inv = __fdividef(1.f, s0 + s1);
+    const f32x2 inv2 = pack2(inv, inv);
+    f32x2 dot2 = pack2(0.f, 0.f);
+    const float2* vec2 = reinterpret_cast<const float2*>(vec);
+#pragma unroll
+    for (int j = 0; j < kM; j += 2) {
+        const f32x2 pj = mul2(pack2(u[j], u[j + 1]), inv2);
+        unpack2(pj, u[j], u[j + 1]);
+        const float2 zv = vec2[j >> 1];
+        dot2 = fma2(pj, pack2(zv.x, zv.y), dot2);
+    }
+    unpack2(dot2, s0, s1);
+    return s0 + s1;
+}
+
 __device__ __forceinline__ void load64(uint32_t taddr, float (&x)[kM])
 {
     uint32_t r[kM];
@@ -624,9 +660,8 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             if (first && !cbar_and(okl)) break;
             // ---- phi(q): p stays in registers (fp32, and its bf16 roundings); den = phi . z from the rounded values ----
             float p[kM];
-            uint32_t pk[kM / 2];
             load64(t_u + lane_base, p);
-            sa[half * kTile + row] = half == 0 ? softmax_half_packed<false>(p, pk, vec) : softmax_half_packed<true>(p, pk, vec + kM);
+            sa[half * kTile + row] = half == 0 ? softmax_half_plain<false>(p, vec) : softmax_half_plain<true>(p, vec + kM);
             LB_TRACE(3);
             if (pre) {
                 // ---- the previous tile's last stage has had the time of a feature map: its dq leaves ----
@@ -649,7 +684,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 f32x2 gs2 = pack2(0.f, 0.f);
 #pragma unroll
                 for (int j = 0; j < kM; j += 2)
-                    gs2 = fma2(pack2(__uint_as_float(pk[j >> 1] << 16), __uint_as_float(pk[j >> 1] & 0xffff0000u)), pack2(x[j], x[j + 1]), gs2);
+                    gs2 = fma2(pack2(p[j], p[j + 1]), pack2(x[j], x[j + 1]), gs2);
                 float g0s, g1s;
                 unpack2(gs2, g0s, g1s);
                 sb[half * kTile + row] = (g0s + g1s) * inv1;   // this half's part of dO . o
