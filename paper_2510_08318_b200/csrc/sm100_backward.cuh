@@ -352,8 +352,9 @@ __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[
     if (half == 0) {
         float o[kM];
         load64(park, o);
+        const f32x2 minus1 = pack2(-1.f, -1.f);
 #pragma unroll
-        for (int j = 0; j < kM; ++j) dphi[j] -= o[j];
+        for (int j = 0; j < kM; j += 2) unpack2(fma2(pack2(o[j], o[j + 1]), minus1, pack2(dphi[j], dphi[j + 1])), dphi[j], dphi[j + 1]);
         store_row_bf16(du_tile, row, dphi);
     }
 }
@@ -637,9 +638,9 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         float* sdd = sb;   // dden den of the tile's tokens takes the place of the first half of sb once both halves have been read
         uint32_t ph_l = 0, ph_t = 0, ph_g = 0;
         float dr_acc = 0.f;   // Eq. 8: this thread's share of sum dout . (a - o)
-        float dz_acc[8];      // thread (8 consecutive features, 8 of the tile's tokens); summed over the token groups at the end of a segment
+        f32x2 dz2[4];         // thread (8 consecutive features as 4 pairs, 8 of the tile's tokens); summed over the token groups at the end of a segment
 #pragma unroll
-        for (int e = 0; e < 8; ++e) dz_acc[e] = 0.f;
+        for (int e = 0; e < 4; ++e) dz2[e] = pack2(0.f, 0.f);
         // dq of a tile leaves tensor memory for the tile's own Q buffer (the tile's last tensor-core stage has completed)
         auto stage_dq = [&](int buf) {
             float x[kM];
@@ -748,11 +749,10 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     const uint4 pv = *reinterpret_cast<const uint4*>(blk + sw_chunk(t, fc & 7));
                     const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
                     const float dd = sdd[t];
+                    const f32x2 dd2 = pack2(dd, dd);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        dz_acc[2 * q] = fmaf(dd, __uint_as_float(pw[q] << 16), dz_acc[2 * q]);
-                        dz_acc[2 * q + 1] = fmaf(dd, __uint_as_float(pw[q] & 0xffff0000u), dz_acc[2 * q + 1]);
-                    }
+                    for (int q = 0; q < 4; ++q)
+                        dz2[q] = fma2(dd2, pack2(__uint_as_float(pw[q] << 16), __uint_as_float(pw[q] & 0xffff0000u)), dz2[q]);
                 }
             }
             LB_TRACE(9);
@@ -774,9 +774,12 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 // dz: the 16 token groups' sums, in group order (the du tile has been consumed)
                 float* red = reinterpret_cast<float*>(c.smem + L::kRed);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    red[(tid >> 4) * kD + (tid & 15) * 8 + e] = dz_acc[e];
-                    dz_acc[e] = 0.f;
+                for (int e = 0; e < 4; ++e) {
+                    float d0, d1;
+                    unpack2(dz2[e], d0, d1);
+                    red[(tid >> 4) * kD + (tid & 15) * 8 + 2 * e] = d0;
+                    red[(tid >> 4) * kD + (tid & 15) * 8 + 2 * e + 1] = d1;
+                    dz2[e] = pack2(0.f, 0.f);
                 }
                 cbar();
                 if (tid < kD) {
@@ -1042,7 +1045,10 @@ kside_bwd_tc(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CU
                 float x[kM];
                 load64(t_t + lane_base + half * kM, x);
 #pragma unroll
-                for (int j = 0; j < kM; ++j) x[j] += vec[half * kM + j];
+                for (int j = 0; j < kM; j += 2) {
+                    const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
+                    unpack2(add2(pack2(x[j], x[j + 1]), pack2(zv.x, zv.y)), x[j], x[j + 1]);
+                }
                 du_exchange(half, row, p, x, t_t + kM + lane_base, c.smem + L::kDu);
             }
             LB_TRACE_K(5);
