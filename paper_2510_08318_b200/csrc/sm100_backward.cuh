@@ -264,9 +264,10 @@ __device__ __forceinline__ float softmax_half_packed(float (&u)[kM], uint32_t (&
     return s0 + s1;
 }
 
-// The same without the roundings: p[64] (fp32) in place; returns sum_j p_j * vec[j].
+// The same without roundings and without the division: u[64] becomes e_j = exp(+-u_j - max), `inv_sum` 1 / sum_j e_j
+// (p_j = e_j * inv_sum: the callers fold that factor into what they multiply p by); returns sum_j e_j * vec[j].
 template <bool kNeg>
-__device__ __forceinline__ float softmax_half_plain(float (&u)[kM], const float* vec)
+__device__ __forceinline__ float softmax_half_raw(float (&u)[kM], float& inv_sum, const float* vec)
 {
     float m = kNeg ? min3(u[0], u[1], u[2]) : max3(u[0], u[1], u[2]);
 #pragma unroll
@@ -274,28 +275,22 @@ __device__ __forceinline__ float softmax_half_plain(float (&u)[kM], const float*
     m = kNeg ? fminf(m, u[kM - 1]) : fmaxf(m, u[kM - 1]);
     const float sL = kNeg ? -kLog2e : kLog2e, off = kNeg ? m * kLog2e : -m * kLog2e;
     const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
-    f32x2 sum2 = pack2(0.f, 0.f);
+    f32x2 sum2 = pack2(0.f, 0.f), dot2 = pack2(0.f, 0.f);
+    const float2* vec2 = reinterpret_cast<const float2*>(vec);
 #pragma unroll
     for (int j = 0; j < kM; j += 2) {
         float x0, x1;
         unpack2(fma2(pack2(u[j], u[j + 1]), scale, offset), x0, x1);
         u[j] = ex2_approx(x0);
         u[j + 1] = ex2_approx(x1);
-        sum2 = add2(sum2, pack2(u[j], u[j + 1]));
+        const f32x2 e = pack2(u[j], u[j + 1]);
+        sum2 = add2(sum2, e);
+        const float2 zv = vec2[j >> 1];
+        dot2 = fma2(e, pack2(zv.x, zv.y), dot2);
     }
     float s0, s1;
     unpack2(sum2, s0, s1);
-    const float inv = __fdividef(1.f, s0 + s1);
-    const f32x2 inv2 = pack2(inv, inv);
-    f32x2 dot2 = pack2(0.f, 0.f);
-    const float2* vec2 = reinterpret_cast<const float2*>(vec);
-#pragma unroll
-    for (int j = 0; j < kM; j += 2) {
-        const f32x2 pj = mul2(pack2(u[j], u[j + 1]), inv2);
-        unpack2(pj, u[j], u[j + 1]);
-        const float2 zv = vec2[j >> 1];
-        dot2 = fma2(pj, pack2(zv.x, zv.y), dot2);
-    }
+    inv_sum = __fdividef(1.f, s0 + s1);
     unpack2(dot2, s0, s1);
     return s0 + s1;
 }
@@ -327,17 +322,20 @@ __device__ __forceinline__ void store_row_bf16(uint8_t* blk, int row, const floa
 // of the token's lane of tensor memory (`park`: the columns of T that half 1 itself has just read; both threads of a token
 // sit on warps of the same lane quarter, so either can reach the lane), and after a barrier of these warps half 0 takes them back,
 // subtracts and writes du (bf16) to its row of the du tile.
-__device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint32_t park, uint8_t* du_tile)
+__device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint32_t park, uint8_t* du_tile,
+                                            float p_scale = 1.f)
 {
+    // p = p_scale * p[] (the query side keeps the exponentials and their normaliser apart)
     f32x2 dot2 = pack2(0.f, 0.f);
 #pragma unroll
     for (int j = 0; j < kM; j += 2) dot2 = fma2(pack2(p[j], p[j + 1]), pack2(dphi[j], dphi[j + 1]), dot2);
     float d0, d1;
     unpack2(dot2, d0, d1);
-    const f32x2 ndot = pack2(-(d0 + d1), -(d0 + d1));
+    const float nd = -(d0 + d1) * p_scale * p_scale;
+    const f32x2 ndot = pack2(nd, nd), ps2 = pack2(p_scale, p_scale);
 #pragma unroll
     for (int j = 0; j < kM; j += 2)
-        unpack2(mul2(pack2(p[j], p[j + 1]), add2(pack2(dphi[j], dphi[j + 1]), ndot)), dphi[j], dphi[j + 1]);
+        unpack2(mul2(pack2(p[j], p[j + 1]), fma2(pack2(dphi[j], dphi[j + 1]), ps2, ndot)), dphi[j], dphi[j + 1]);
     if (half == 1) {
         uint32_t r[kM];
 #pragma unroll
@@ -662,7 +660,11 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             // ---- phi(q): p stays in registers (fp32, and its bf16 roundings); den = phi . z from the rounded values ----
             float p[kM];
             load64(t_u + lane_base, p);
-            sa[half * kTile + row] = half == 0 ? softmax_half_plain<false>(p, vec) : softmax_half_plain<true>(p, vec + kM);
+            float invs;   // p_j = invs * p[j] from here on
+            {
+                const float ez = half == 0 ? softmax_half_raw<false>(p, invs, vec) : softmax_half_raw<true>(p, invs, vec + kM);
+                sa[half * kTile + row] = ez * invs;
+            }
             LB_TRACE(3);
             if (pre) {
                 // ---- the previous tile's last stage has had the time of a feature map: its dq leaves ----
@@ -688,6 +690,8 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     gs2 = fma2(pack2(p[j], p[j + 1]), pack2(x[j], x[j + 1]), gs2);
                 float g0s, g1s;
                 unpack2(gs2, g0s, g1s);
+                g0s *= invs;
+                g1s *= invs;
                 sb[half * kTile + row] = (g0s + g1s) * inv1;   // this half's part of dO . o
                 if (kMixB) {
                     // Eq. 8: dout . a over this thread's 64 columns (dout from its tile, a straight from memory: one
@@ -719,7 +723,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
                 // phi / den (bf16) is the operand of dS and the factor of dz (the previous tile's dS and dz are done with the tile)
                 float y[kM];
-                const f32x2 inv2 = pack2(inv, inv);
+                const f32x2 inv2 = pack2(inv * invs, inv * invs);
 #pragma unroll
                 for (int j = 0; j < kM; j += 2) unpack2(mul2(pack2(p[j], p[j + 1]), inv2), y[j], y[j + 1]);
                 store_row_bf16(c.smem + L::kP + half * kHalfTileBytes, row, y);
@@ -734,7 +738,7 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
                 unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
             }
-            du_exchange(half, row, p, x, t_t + kM + lane_base, c.smem + L::kDu);   // (a barrier inside: both halves of sb have been read)
+            du_exchange(half, row, p, x, t_t + kM + lane_base, c.smem + L::kDu, invs);   // (a barrier inside: both halves of sb have been read)
             if (half == 0) sdd[row] = ngo;
             if (!(a.test_unmet && warp == 0 && w.i == 0)) warp_announce(c, BW_OPS);   // (left out once by the test of the time-out path)
             cbar();
