@@ -276,17 +276,20 @@ __device__ __forceinline__ float softmax_half_raw(float (&u)[kM], float& inv_sum
     const float sL = kNeg ? -kLog2e : kLog2e, off = kNeg ? m * kLog2e : -m * kLog2e;
     const f32x2 scale = pack2(sL, sL), offset = pack2(off, off);
     f32x2 sum2 = pack2(0.f, 0.f), dot2 = pack2(0.f, 0.f);
-    const float2* vec2 = reinterpret_cast<const float2*>(vec);
+    const float4* vec4 = reinterpret_cast<const float4*>(vec);
 #pragma unroll
-    for (int j = 0; j < kM; j += 2) {
-        float x0, x1;
-        unpack2(fma2(pack2(u[j], u[j + 1]), scale, offset), x0, x1);
-        u[j] = ex2_approx(x0);
-        u[j + 1] = ex2_approx(x1);
-        const f32x2 e = pack2(u[j], u[j + 1]);
-        sum2 = add2(sum2, e);
-        const float2 zv = vec2[j >> 1];
-        dot2 = fma2(e, pack2(zv.x, zv.y), dot2);
+    for (int j = 0; j < kM; j += 4) {
+        const float4 zv = vec4[j >> 2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float x0, x1;
+            unpack2(fma2(pack2(u[j + 2 * h], u[j + 2 * h + 1]), scale, offset), x0, x1);
+            u[j + 2 * h] = ex2_approx(x0);
+            u[j + 2 * h + 1] = ex2_approx(x1);
+            const f32x2 e = pack2(u[j + 2 * h], u[j + 2 * h + 1]);
+            sum2 = add2(sum2, e);
+            dot2 = fma2(e, h ? pack2(zv.z, zv.w) : pack2(zv.x, zv.y), dot2);
+        }
     }
     float s0, s1;
     unpack2(sum2, s0, s1);
@@ -323,19 +326,21 @@ __device__ __forceinline__ void store_row_bf16(uint8_t* blk, int row, const floa
 // sit on warps of the same lane quarter, so either can reach the lane), and after a barrier of these warps half 0 takes them back,
 // subtracts and writes du (bf16) to its row of the du tile.
 __device__ __forceinline__ void du_exchange(int half, int row, const float (&p)[kM], float (&dphi)[kM], uint32_t park, uint8_t* du_tile,
-                                            float p_scale = 1.f)
+                                            float p_scale = 1.f, float dphi_scale = 1.f)
 {
-    // p = p_scale * p[] (the query side keeps the exponentials and their normaliser apart)
+    // the feature values are p_scale * p[], the gradients dphi_scale * dphi[] (the query side keeps the exponentials and
+    // their normaliser apart, and the per-token factor 1 / den out of dphi): du_j = a p_j (dphi_j - b sum_i p_i dphi_i) with
+    // a = p_scale dphi_scale, b = p_scale
     f32x2 dot2 = pack2(0.f, 0.f);
 #pragma unroll
     for (int j = 0; j < kM; j += 2) dot2 = fma2(pack2(p[j], p[j + 1]), pack2(dphi[j], dphi[j + 1]), dot2);
     float d0, d1;
     unpack2(dot2, d0, d1);
-    const float nd = -(d0 + d1) * p_scale * p_scale;
-    const f32x2 ndot = pack2(nd, nd), ps2 = pack2(p_scale, p_scale);
+    const float as = p_scale * dphi_scale, nd = -(d0 + d1) * p_scale * as;
+    const f32x2 ndot = pack2(nd, nd), as2 = pack2(as, as);
 #pragma unroll
     for (int j = 0; j < kM; j += 2)
-        unpack2(mul2(pack2(p[j], p[j + 1]), fma2(pack2(dphi[j], dphi[j + 1]), ps2, ndot)), dphi[j], dphi[j + 1]);
+        unpack2(mul2(pack2(p[j], p[j + 1]), fma2(pack2(dphi[j], dphi[j + 1]), as2, ndot)), dphi[j], dphi[j + 1]);
     if (half == 1) {
         uint32_t r[kM];
 #pragma unroll
@@ -734,11 +739,12 @@ qside_bwd_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             LB_TRACE(5);
             // ---- du (through the softmax of Eq. 6) ----
 #pragma unroll
-            for (int j = 0; j < kM; j += 2) {   // dphi = (dO S^T - (dO . o) z) / den
-                const float2 zv = *reinterpret_cast<const float2*>(&vec[half * kM + j]);
-                unpack2(mul2(pack2(inv, inv), fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1]))), x[j], x[j + 1]);
+            for (int j = 0; j < kM; j += 4) {   // dphi = (dO S^T - (dO . o) z) / den, its factor 1 / den left to the next step
+                const float4 zv = *reinterpret_cast<const float4*>(&vec[half * kM + j]);
+                unpack2(fma2(pack2(ngo, ngo), pack2(zv.x, zv.y), pack2(x[j], x[j + 1])), x[j], x[j + 1]);
+                unpack2(fma2(pack2(ngo, ngo), pack2(zv.z, zv.w), pack2(x[j + 2], x[j + 3])), x[j + 2], x[j + 3]);
             }
-            du_exchange(half, row, p, x, t_t + kM + lane_base, c.smem + L::kDu, invs);   // (a barrier inside: both halves of sb have been read)
+            du_exchange(half, row, p, x, t_t + kM + lane_base, c.smem + L::kDu, invs, inv);   // (a barrier inside: both halves of sb have been read)
             if (half == 0) sdd[row] = ngo;
             if (!(a.test_unmet && warp == 0 && w.i == 0)) warp_announce(c, BW_OPS);   // (left out once by the test of the time-out path)
             cbar();
