@@ -8,16 +8,18 @@
 //     du = p+ (.) (dphi+ - p+ . dphi+) - p- (.) (dphi- - p- . dphi-)       dx = du W^T       dW += x^T du
 //
 // Two kernels of persistent CTAs, each walking its contiguous run of 128-token tiles.  Every matrix product is a
-// tcgen05.mma with fp32 accumulators in TMEM, every element-wise step runs on all 256 threads, thread = (token, half of
-// the features); thread 0 issues the copies and the products.  Within a head the tiles are software-pipelined two deep:
-// the tile that feeds the logits is double-buffered, the next tile's logits are issued ahead of this tile's last
-// tensor-core stage, and this tile's results leave tensor memory after the next tile's feature map:
+// tcgen05.mma with fp32 accumulators in TMEM.  Warp-specialised: eight element-wise warps (thread = (token, half of the
+// features)), a warp that issues the products and the copies they wait for, a warp that stores the staged results and
+// requests the tile that follows into a buffer once its store has read it; mbarriers both ways.  Within a head the tiles
+// are software-pipelined two deep: the tile that feeds the logits is double-buffered, the next tile's logits and first
+// products are issued around this tile's last tensor-core stage, and this tile's results leave tensor memory after the
+// next tile's feature map (the schedule is written out above qside_bwd_tc):
 //
-//   qside_bwd_tc : U = Q W_q -> phi(q) -> num = phi S, den, dO . o -> dphi = (dO S^T - (dO . o) z) / den,
-//                  dS += (phi / den)^T dO, dz += (phi / den)^T (dden den) -> du -> dq = du W_q^T (TMA store),
-//                  dW_q += Q^T du
-//   kside_bwd_tc : U = K W_k -> phi(k) -> dphi = V dS^T (+ dz), dv = phi dS (TMA store) -> du ->
-//                  dk = du W_k^T (TMA store), dW_k += K^T du
+//   qside_bwd_tc : U = Q W_q -> phi(q), den = phi . z -> T = dO S^T -> dO . o = (T . phi) / den ->
+//                  dphi = (T - (dO . o) z) / den, dS += (phi / den)^T dO, dz += (phi / den)^T (dden den) -> du ->
+//                  dq = du W_q^T (TMA store), dW_q += Q^T du
+//   kside_bwd_tc : U = K W_k -> phi(k) -> dphi = V dS^T (+ dz) -> du -> dk = du W_k^T (TMA store), dW_k += K^T du,
+//                  dv = phi dS (TMA store)
 //
 // Operands that carry a difference of nearly equal terms downstream are kept exact or split into bf16 hi + lo
 // parts: S and dS are hi + lo images written by the combine kernels (two passes each); dnum = dO / den is never
