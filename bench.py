@@ -216,6 +216,7 @@ ALL_VARIANTS = [
     ("mixed attention (Eq. 8), r = 0.5, config 2", ["--config", "2", "--mixed", "0.5"]),
     ("ReLU kernel function, config 2", ["--config", "2", "--phi", "relu"]),
     ("backward, config 2", ["--config", "2", "--backward"]),
+    ("training step (forward, then backward with the forward's S and z), config 2", ["--config", "2", "--train-step"]),
     ("backward, config 3", ["--config", "3", "--backward"]),
     ("backward, config 4", ["--config", "4", "--backward"]),
 ]
@@ -226,7 +227,7 @@ def run_all(args):
     one); prints each child's JSON line and writes a markdown table of them."""
     rows = []
     for title, extra in ALL_VARIANTS:
-        steps = 300 if "--backward" not in extra else 100
+        steps = 300 if "--backward" not in extra and "--train-step" not in extra else 100
         cmd = [sys.executable, os.path.abspath(__file__), "--gpus", "1", "--steps", str(steps), "--warmup", "10", "--no-baselines"] + extra
         res = subprocess.run(cmd, capture_output=True, text=True)
         line = next((l for l in reversed(res.stdout.splitlines()) if l.startswith("{")), None)
@@ -270,6 +271,9 @@ def main():
                          "softmax-branch output (5 tensors of traffic instead of 4)")
     ap.add_argument("--phi", default="hedgehog", choices=["hedgehog", "relu"],
                     help="kernel function: the Hedgehog feature map of Eq. 6 (the metric's) or the ReLU of the paper's ablation")
+    ap.add_argument("--train-step", action="store_true",
+                    help="time a training step of the layer: linattn_forward followed by linattn_backward on the same q, k, v, "
+                         "with LINATTN_OPT_REUSE_STATE = 1 (the backward takes S and z over from the forward that just ran)")
     ap.add_argument("--backward", action="store_true",
                     help="time linattn_backward (gradients of the operator; the kernels --path selects) instead of the forward")
     ap.add_argument("--layout", type=int, default=0, choices=[0, 1],
@@ -317,7 +321,7 @@ def main():
         sets.append({k_: t.to(dev) for k_, t in x.items()})
     outs = [torch.empty_like(s["q"]) for s in sets]
     softs = [torch.randn_like(s["q"]) for s in sets] if args.mixed is not None else None
-    douts = [torch.randn_like(s["q"]) for s in sets] if args.backward else None
+    douts = [torch.randn_like(s["q"]) for s in sets] if (args.backward or args.train_step) else None
     ctxs = []
     for s in sets:  # one context per input set: its own feature map, as one layer would have
         c = linattn.LinAttn(H, d, max_B=B, max_n=n, device=local)
@@ -325,13 +329,18 @@ def main():
         c.set_option(linattn.OPT_SPLITS, args.splits)
         c.set_option(linattn.OPT_KERNEL_FUNCTION, linattn.PHI_RELU if args.phi == "relu" else linattn.PHI_HEDGEHOG)
         c.set_option(linattn.OPT_LAYOUT, args.layout)   # i.i.d. synthetic values: the same storage read in the other order
+        if args.train_step:
+            c.set_option(linattn.OPT_REUSE_STATE, 1)
         c.set_feature_map(s["Wq"], s["Wk"])
         ctxs.append(c)
     stream = torch.cuda.current_stream()
 
     def step(i):
         j = i % rotate
-        if douts is not None:
+        if args.train_step:
+            ctxs[j].forward(sets[j]["q"], sets[j]["k"], sets[j]["v"], out=outs[j], stream=stream)
+            ctxs[j].backward(sets[j]["q"], sets[j]["k"], sets[j]["v"], douts[j], stream=stream)
+        elif douts is not None:
             ctxs[j].backward(sets[j]["q"], sets[j]["k"], sets[j]["v"], douts[j], stream=stream)
         elif softs is None:
             ctxs[j].forward(sets[j]["q"], sets[j]["k"], sets[j]["v"], out=outs[j], stream=stream)
@@ -343,6 +352,11 @@ def main():
         step(i)
     ctxs[0].check()
     launches_per_step = ctxs[0].last_launch_count()
+    if args.train_step:   # one more step on the first context, counting both calls (its very first backward also split S into hi + lo)
+        ctxs[0].forward(sets[0]["q"], sets[0]["k"], sets[0]["v"], out=outs[0], stream=stream)
+        launches_per_step = ctxs[0].last_launch_count()
+        ctxs[0].backward(sets[0]["q"], sets[0]["k"], sets[0]["v"], douts[0], stream=stream)
+        launches_per_step += ctxs[0].last_launch_count()
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     # the W warm-up steps run right before the timed region, with no host-side pause in between in which the GPU could
@@ -390,7 +404,7 @@ def main():
     e = 2 if wl.dtype == "bf16" else 4
     # tensors of [B,H,n,d] one step must move: q, k, v in and o out; + the softmax branch for Eq. 8; for the
     # gradients q, k, v, dO in and dq, dk, dv out
-    alg_total = (7.0 if douts is not None else 4.0 if softs is None else 5.0) * B * H * n * d * e
+    alg_total = (11.0 if args.train_step else 7.0 if douts is not None else 4.0 if softs is None else 5.0) * B * H * n * d * e
     for c in ctxs:
         c.set_option(linattn.OPT_PROFILE, 1)
     for i in range(min(args.steps, 300)):
@@ -446,7 +460,7 @@ def main():
     if douts is not None:
         e2e["note"] = "this is the forward's host-buffer entry point; the backward has no host-buffer form"
     result = {
-        "metric": ("linear-attention bwd tokens/s" if douts is not None else "mixed-attention (Eq. 8) fwd tokens/s" if softs is not None
+        "metric": ("linear-attention fwd+bwd tokens/s" if args.train_step else "linear-attention bwd tokens/s" if douts is not None else "mixed-attention (Eq. 8) fwd tokens/s" if softs is not None
                    else "linear-attention (ReLU kernel function) fwd tokens/s" if args.phi == "relu" else METRIC), "value": value, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
