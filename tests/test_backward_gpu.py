@@ -215,6 +215,39 @@ def test_state_left_by_the_forward_is_reused_only_when_it_belongs_to_the_same_pr
         fresh.destroy()
 
 
+@pytest.mark.parametrize("n", [1000, 2700])   # a ragged last tile; about one and about three tiles per CTA
+def test_gradient_guard_bands_are_untouched(n):
+    """dq, dk, dv are written by TMA stores that clip at the end of the sequence, the weight gradients by a kernel of
+    their own: canaries on both sides of every output buffer must survive (called through the C-ABI, which takes the
+    output pointers as they are)."""
+    B, H, d = 2, 3, 128
+    x = _inputs(B, H, n, d, torch.bfloat16, seed=300 + n)
+    want = oracle.ref_backward(x["q"], x["k"], x["v"], x["Wq"], x["Wk"], x["dout"])
+    pad = 4096
+
+    def guarded(numel, dtype):
+        buf = torch.full((pad + numel + pad,), 7.0, dtype=dtype, device="cuda")
+        return buf, buf[pad:pad + numel]
+
+    bufs = [guarded(B * H * n * d, torch.bfloat16) for _ in range(3)] + [guarded(H * d * (d // 2), torch.float32) for _ in range(2)]
+    ctx = linattn.LinAttn(H, d, max_B=B, max_n=n)
+    try:
+        ctx.set_feature_map(x["Wq"].cuda(), x["Wk"].cuda())
+        q, k, v, dout = (x[s].cuda() for s in ("q", "k", "v", "dout"))
+        st = ctx._lib.linattn_backward(ctx._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), dout.data_ptr(),
+                                       *[inner.data_ptr() for _, inner in bufs], 1, B, H, n, d, linattn.BF16,
+                                       torch.cuda.current_stream().cuda_stream)
+        assert st == linattn.OK
+        ctx.check()
+        assert ctx.last_launch_count() == 6
+        for buf, _ in bufs:
+            assert (buf[:pad] == 7.0).all() and (buf[-pad:] == 7.0).all(), "a gradient kernel wrote outside its output"
+        got = [bufs[i][1].view(B, H, n, d) for i in range(3)] + [bufs[i][1].view(H, d, d // 2) for i in (3, 4)]
+        _assert_grads(got, want, f"guarded outputs, n={n}")
+    finally:
+        ctx.destroy()
+
+
 def test_argument_errors():
     lib = linattn.load_library()
     x = _inputs(1, 2, 128, 64, torch.float32, seed=35)
