@@ -82,6 +82,7 @@ def _run(x, per_head=True, layout=linattn.LAYOUT_BHND, path=linattn.PATH_AUTO):
     (1, 1, 1, 128, torch.bfloat16),
     (2, 5, 700, 128, torch.bfloat16),    # more heads than one CTA's run covers: segments of several heads per CTA
     (1, 2, 33000, 128, torch.bfloat16),  # runs of many tiles per CTA
+    (2, 20, 1500, 128, torch.bfloat16),  # three to four tiles per CTA and twelve per head: most runs cross into another head
 ])
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_gradients_match_the_oracle(B, H, n, d, dtype, path):
